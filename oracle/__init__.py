@@ -1,0 +1,203 @@
+"""CPU oracle of the folded quantized linear layer (test infrastructure only).
+
+Thin numpy/ctypes front end over ``fq_oracle.c``; every numerical step lives in
+that C file, which restates Eq. 3, Eq. 5, Eq. 8 and Algorithm 1 of the paper.
+Only tests, the smoke check and the benchmark's CPU-baseline leg may import
+this package; the CUDA product path never does.
+
+bfloat16 tensors are numpy ``uint16`` arrays holding the raw bit patterns and
+are tagged with ``dtype="bf16"``; everything else is ``float32``.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from typing import Optional, Sequence, Tuple
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "fq_oracle.c")
+_LIB = os.path.join(_HERE, "libfq_oracle.so")
+
+F32, BF16 = 0, 1
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (strict IEEE: no FMA contraction)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        cmd = ["gcc", "-O2", "-std=c11", "-ffp-contract=off", "-fno-fast-math", "-fopenmp",
+               "-fPIC", "-shared", "-o", _LIB, _SRC, "-lm"]
+        subprocess.run(cmd, check=True)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        build()
+        _lib = ctypes.CDLL(_LIB)
+        _lib.fqo_num_threads.restype = ctypes.c_int
+    return _lib
+
+
+def num_threads() -> int:
+    return int(_load().fqo_num_threads())
+
+
+def _dt(dtype: str) -> int:
+    if dtype in ("f32", "fp32", "float32"):
+        return F32
+    if dtype in ("bf16", "bfloat16"):
+        return BF16
+    raise ValueError(dtype)
+
+
+def _mat(x: np.ndarray, dtype: str) -> np.ndarray:
+    want = np.float32 if _dt(dtype) == F32 else np.uint16
+    x = np.ascontiguousarray(x)
+    if x.dtype != want:
+        raise TypeError(f"expected {want} for dtype={dtype}, got {x.dtype}")
+    return x
+
+
+def _p(a: Optional[np.ndarray]):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _f32(a) -> Optional[np.ndarray]:
+    return None if a is None else np.ascontiguousarray(a, dtype=np.float32)
+
+
+def _check(rc: int, what: str):
+    if rc != 0:
+        raise RuntimeError(f"oracle {what} failed with code {rc}")
+
+
+def fwht_block(v: np.ndarray) -> np.ndarray:
+    """Unnormalised Sylvester-Hadamard product of one block (length = beta)."""
+    out = np.array(v, dtype=np.float32, copy=True).reshape(-1)
+    _load().fqo_fwht_block(_p(out), ctypes.c_int(out.size))
+    return out
+
+
+def multiplier(smooth, K: int, beta: int, for_weights: bool) -> np.ndarray:
+    g = np.empty(K, dtype=np.float32)
+    s = _f32(smooth)
+    _check(_load().fqo_multiplier(_p(s), ctypes.c_int64(K), ctypes.c_int(beta),
+                                  ctypes.c_int(1 if for_weights else 0), _p(g)), "multiplier")
+    return g
+
+
+def smooth_scale(a, w, alpha: float) -> np.ndarray:
+    a = _f32(a)
+    w = _f32(w)
+    s = np.empty_like(a)
+    _check(_load().fqo_smooth_scale(_p(a), _p(w), ctypes.c_int64(a.size), ctypes.c_double(alpha),
+                                    _p(s)), "smooth_scale")
+    return s
+
+
+def col_absmax(x: np.ndarray, dtype: str = "f32") -> np.ndarray:
+    x = _mat(x, dtype)
+    M, K = x.shape
+    out = np.empty(K, dtype=np.float32)
+    _check(_load().fqo_col_absmax(_p(x), ctypes.c_int(_dt(dtype)), ctypes.c_int64(M),
+                                  ctypes.c_int64(K), ctypes.c_int64(K), _p(out)), "col_absmax")
+    return out
+
+
+def pack(codes: np.ndarray, bits: int) -> np.ndarray:
+    codes = np.ascontiguousarray(codes, dtype=np.int32)
+    rows, K = codes.shape
+    out = np.empty((rows, K * bits // 8), dtype=np.uint8)
+    _check(_load().fqo_pack(_p(codes), ctypes.c_int64(rows), ctypes.c_int64(K), ctypes.c_int(bits),
+                            _p(out)), "pack")
+    return out
+
+
+def unpack(packed: np.ndarray, K: int, bits: int) -> np.ndarray:
+    packed = np.ascontiguousarray(packed).view(np.uint8)
+    rows = packed.shape[0]
+    out = np.empty((rows, K), dtype=np.int32)
+    _check(_load().fqo_unpack(_p(packed), ctypes.c_int64(rows), ctypes.c_int64(K),
+                              ctypes.c_int(bits), _p(out)), "unpack")
+    return out
+
+
+def quantize_act(x: np.ndarray, dtype: str, g, beta: int, bits: int, clip_ratio: float = 1.0,
+                 return_z: bool = False):
+    """Runtime prologue: returns (codes[M, K*bits/8] u8, delta[M] f32[, z[M, K] f32])."""
+    x = _mat(x, dtype)
+    M, K = x.shape
+    g = _f32(g)
+    codes = np.zeros((M, K * bits // 8), dtype=np.uint8)
+    delta = np.zeros(M, dtype=np.float32)
+    z = np.zeros((M, K), dtype=np.float32) if return_z else None
+    _check(_load().fqo_quantize_act(_p(x), ctypes.c_int(_dt(dtype)), ctypes.c_int64(M),
+                                    ctypes.c_int64(K), ctypes.c_int64(K), _p(g), ctypes.c_int(beta),
+                                    ctypes.c_int(bits), ctypes.c_float(clip_ratio), _p(codes),
+                                    _p(delta), _p(z)), "quantize_act")
+    return (codes, delta, z) if return_z else (codes, delta)
+
+
+def fold_weights(W: np.ndarray, dtype: str, smooth, beta: int, bits: int, return_wt: bool = False):
+    """Offline fold + RTN + pack: returns (codes, w_scale[N], mult_g[K][, W~[N, K]])."""
+    W = _mat(W, dtype)
+    N, K = W.shape
+    s = _f32(smooth)
+    codes = np.zeros((N, K * bits // 8), dtype=np.uint8)
+    w_scale = np.zeros(N, dtype=np.float32)
+    g = np.zeros(K, dtype=np.float32)
+    wt = np.zeros((N, K), dtype=np.float32) if return_wt else None
+    _check(_load().fqo_fold_weights(_p(W), ctypes.c_int(_dt(dtype)), ctypes.c_int64(N),
+                                    ctypes.c_int64(K), ctypes.c_int64(K), _p(s), ctypes.c_int(beta),
+                                    ctypes.c_int(bits), _p(codes), _p(w_scale), _p(g), _p(wt)),
+           "fold_weights")
+    return (codes, w_scale, g, wt) if return_wt else (codes, w_scale, g)
+
+
+def gemm_i32(a_codes: np.ndarray, w_codes: np.ndarray, K: int, bits: int) -> np.ndarray:
+    a = np.ascontiguousarray(a_codes).view(np.uint8)
+    w = np.ascontiguousarray(w_codes).view(np.uint8)
+    M, N = a.shape[0], w.shape[0]
+    acc = np.zeros((M, N), dtype=np.int32)
+    _check(_load().fqo_gemm_i32(_p(a), _p(w), ctypes.c_int64(M), ctypes.c_int64(N),
+                                ctypes.c_int64(K), ctypes.c_int(bits), _p(acc)), "gemm_i32")
+    return acc
+
+
+def epilogue(acc: np.ndarray, delta, w_scale, bias, out_dtype: str = "f32") -> np.ndarray:
+    acc = np.ascontiguousarray(acc, dtype=np.int32)
+    M, N = acc.shape
+    y = np.zeros((M, N), dtype=np.float32 if _dt(out_dtype) == F32 else np.uint16)
+    _check(_load().fqo_epilogue(_p(acc), _p(_f32(delta)), _p(_f32(w_scale)), _p(_f32(bias)),
+                                ctypes.c_int64(M), ctypes.c_int64(N), _p(y),
+                                ctypes.c_int(_dt(out_dtype)), ctypes.c_int64(N)), "epilogue")
+    return y
+
+
+def linear(x: np.ndarray, xdtype: str, g, beta: int, bits: int, clip_ratio: float,
+           w_codes: np.ndarray, w_scale, bias, out_dtype: str = "f32",
+           rows: Optional[Sequence[int]] = None) -> Tuple[np.ndarray, np.ndarray, np.ndarray, np.ndarray]:
+    """Whole runtime path. Returns (y, a_codes, delta, acc); with ``rows`` the
+    integer product and epilogue run on those token rows only."""
+    x = _mat(x, xdtype)
+    M, K = x.shape
+    w = np.ascontiguousarray(w_codes).view(np.uint8)
+    N = w.shape[0]
+    sel = None if rows is None else np.ascontiguousarray(rows, dtype=np.int64)
+    Ms = M if sel is None else sel.size
+    y = np.zeros((Ms, N), dtype=np.float32 if _dt(out_dtype) == F32 else np.uint16)
+    codes = np.zeros((M, K * bits // 8), dtype=np.uint8)
+    delta = np.zeros(M, dtype=np.float32)
+    acc = np.zeros((Ms, N), dtype=np.int32)
+    _check(_load().fqo_linear(_p(x), ctypes.c_int(_dt(xdtype)), ctypes.c_int64(M), ctypes.c_int64(K),
+                              ctypes.c_int64(K), _p(_f32(g)), ctypes.c_int(beta), ctypes.c_int(bits),
+                              ctypes.c_float(clip_ratio), _p(w), _p(_f32(w_scale)), _p(_f32(bias)),
+                              ctypes.c_int64(N), _p(sel), ctypes.c_int64(0 if sel is None else sel.size),
+                              _p(y), ctypes.c_int(_dt(out_dtype)), ctypes.c_int64(N), _p(codes),
+                              _p(delta), _p(acc)), "linear")
+    return y, codes, delta, acc

@@ -1,0 +1,360 @@
+/*
+ * FoldQuant linear layer -- CPU ORACLE (test infrastructure, not product code).
+ *
+ * A plain, slow, step-by-step restatement of the folded quantized linear layer:
+ *   offline : fold  W~ = W S R^T  (fold-before transform family, Eq. 3),
+ *             round to nearest per output channel, nibble-pack        (Alg. 1 offline half)
+ *   runtime : z_t = R S^-1 x_t, per-token symmetric quantization      (Eq. 5)
+ *             integer product with int32 accumulation, rescale + bias (Eq. 8, Alg. 1 runtime half)
+ *
+ * Only tests, the smoke check and the benchmark's CPU-baseline leg may call
+ * this file.  It shares no code, header, table or helper with the CUDA path.
+ *
+ * Arithmetic contract (so that integer stages can be compared bit for bit):
+ *   - every floating-point step of the transform and the quantizer is one
+ *     IEEE-754 binary32 operation, round-to-nearest-even, no fused
+ *     multiply-add (build with -ffp-contract=off), denormals preserved;
+ *   - butterflies run with ascending stride h = 1, 2, ..., beta/2; the lower
+ *     index receives a+b, the upper a-b (natural / Sylvester ordering);
+ *   - the epilogue is evaluated in binary64 and rounded once.
+ *
+ * Readings the paper leaves open (fixed here, "parity unpinned" by the paper
+ * itself): ties in round() go to even; two 4-bit codes share a byte with the
+ * even channel in the low nibble, two's complement; smoothing-scale floors
+ * 1e-5 and bounds [1e-5, 1e5].
+ */
+#include <float.h>
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+#define FQO_F32 0
+#define FQO_BF16 1
+
+int fqo_num_threads(void) {
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+/* bfloat16 <-> float. Widening is exact; narrowing rounds to nearest even. */
+static float bf16_to_f32(uint16_t h) {
+    uint32_t u = (uint32_t)h << 16;
+    float f;
+    memcpy(&f, &u, 4);
+    return f;
+}
+
+static uint16_t f32_to_bf16(float f) {
+    uint32_t u;
+    memcpy(&u, &f, 4);
+    if ((u & 0x7fffffffu) > 0x7f800000u) return (uint16_t)((u >> 16) | 0x40u); /* NaN */
+    uint32_t lsb = (u >> 16) & 1u;
+    u += 0x7fffu + lsb;
+    return (uint16_t)(u >> 16);
+}
+
+static float load_elem(const void* base, int dtype, int64_t idx) {
+    if (dtype == FQO_BF16) return bf16_to_f32(((const uint16_t*)base)[idx]);
+    return ((const float*)base)[idx];
+}
+
+static int valid_block(int beta, int64_t K) {
+    if (beta < 2 || beta > 256 || (beta & (beta - 1)) != 0) return 0;
+    return K > 0 && K % beta == 0;
+}
+
+static float qmax_of(int bits) { return bits == 4 ? 7.0f : 127.0f; }
+
+/* Section "Transforms supported by the runtime": unnormalised Sylvester
+ * Hadamard product of one block of beta values, in place, by butterflies. */
+void fqo_fwht_block(float* v, int beta) {
+    for (int h = 1; h < beta; h <<= 1) {
+        for (int i = 0; i < beta; ++i) {
+            if ((i & h) == 0) {
+                float a = v[i];
+                float b = v[i + h];
+                v[i] = a + b;
+                v[i + h] = a - b;
+            }
+        }
+    }
+}
+
+/* u = (I (x) H_beta) v over a row of K channels, unnormalised. */
+void fqo_fwht_row(float* v, int64_t K, int beta) {
+    for (int64_t c0 = 0; c0 < K; c0 += beta) fqo_fwht_block(v + c0, beta);
+}
+
+/* Per-channel multiplier that carries both the diagonal factor of the
+ * fold-before transform and the beta^(-1/2) normalisation of R.
+ *   for_weights = 0 : g_c = (1/s_c) * beta^(-1/2)   (runtime side, S^-1)
+ *   for_weights = 1 : g_c =    s_c  * beta^(-1/2)   (offline side, S)
+ * smooth == NULL means S = I. */
+int fqo_multiplier(const float* smooth, int64_t K, int beta, int for_weights, float* g) {
+    if (!valid_block(beta, K) || !g) return 1;
+    float c = (float)(1.0 / sqrt((double)beta));
+    for (int64_t i = 0; i < K; ++i) {
+        if (!smooth) {
+            g[i] = c;
+        } else if (for_weights) {
+            g[i] = smooth[i] * c;
+        } else {
+            float inv = 1.0f / smooth[i];
+            g[i] = inv * c;
+        }
+    }
+    return 0;
+}
+
+/* SmoothQuant channel scale s_c = a_c^alpha / w_c^(1-alpha) with floors and
+ * bounds (section "Transforms supported by the runtime").  a = calibrated
+ * activation max-abs per channel, w = largest weight magnitude per input
+ * channel over all consumers of the site.  binary64, cast once. */
+int fqo_smooth_scale(const float* a, const float* w, int64_t K, double alpha, float* s) {
+    if (!a || !w || !s || alpha < 0.0 || alpha > 1.0) return 1;
+    for (int64_t i = 0; i < K; ++i) {
+        double ac = a[i] > 1e-5 ? (double)a[i] : 1e-5;
+        double wc = w[i] > 1e-5 ? (double)w[i] : 1e-5;
+        double v = pow(ac, alpha) / pow(wc, 1.0 - alpha);
+        if (v < 1e-5) v = 1e-5;
+        if (v > 1e5) v = 1e5;
+        s[i] = (float)v;
+    }
+    return 0;
+}
+
+/* Column-wise max |x| over the rows of a [M, K] matrix (calibration statistic). */
+int fqo_col_absmax(const void* x, int dtype, int64_t M, int64_t K, int64_t ldx, float* out) {
+    if (!x || !out) return 1;
+    for (int64_t c = 0; c < K; ++c) out[c] = 0.0f;
+    for (int64_t t = 0; t < M; ++t)
+        for (int64_t c = 0; c < K; ++c) {
+            float v = fabsf(load_elem(x, dtype, t * ldx + c));
+            if (v > out[c]) out[c] = v;
+        }
+    return 0;
+}
+
+/* Store one row of signed codes.  4 bits: byte i = code[2i] in the low nibble,
+ * code[2i+1] in the high nibble, two's complement.  8 bits: one int8 each. */
+static void pack_row(const int* code, int64_t K, int bits, uint8_t* out) {
+    if (bits == 4) {
+        for (int64_t i = 0; i < K / 2; ++i)
+            out[i] = (uint8_t)((code[2 * i] & 0xF) | ((code[2 * i + 1] & 0xF) << 4));
+    } else {
+        for (int64_t i = 0; i < K; ++i) out[i] = (uint8_t)(int8_t)code[i];
+    }
+}
+
+static int code_at(const uint8_t* row, int64_t c, int bits) {
+    if (bits == 8) return (int)(int8_t)row[c];
+    int nib = (row[c >> 1] >> ((c & 1) * 4)) & 0xF;
+    return nib >= 8 ? nib - 16 : nib;
+}
+
+int fqo_pack(const int32_t* codes, int64_t rows, int64_t K, int bits, uint8_t* out) {
+    if ((bits != 4 && bits != 8) || (bits == 4 && (K & 1))) return 1;
+    int64_t pitch = K * bits / 8;
+    int* tmp = (int*)malloc(sizeof(int) * (size_t)(K > 0 ? K : 1));
+    for (int64_t r = 0; r < rows; ++r) {
+        for (int64_t c = 0; c < K; ++c) tmp[c] = codes[r * K + c];
+        pack_row(tmp, K, bits, out + r * pitch);
+    }
+    free(tmp);
+    return 0;
+}
+
+int fqo_unpack(const uint8_t* packed, int64_t rows, int64_t K, int bits, int32_t* codes) {
+    if ((bits != 4 && bits != 8) || (bits == 4 && (K & 1))) return 1;
+    int64_t pitch = K * bits / 8;
+    for (int64_t r = 0; r < rows; ++r)
+        for (int64_t c = 0; c < K; ++c) codes[r * K + c] = code_at(packed + r * pitch, c, bits);
+    return 0;
+}
+
+/* Eq. 5 applied to one already-transformed row u: per-row step
+ * delta = (r * max|u|) / q, codes = clip(round(u * (1/delta)), -q, q).
+ * A row whose step would fall below the smallest normal float is the zero
+ * token: (codes, delta) = (0, 0). */
+static float quantize_row(const float* u, int64_t K, int bits, float clip_ratio, int* code) {
+    float qf = qmax_of(bits);
+    int q = (int)qf;
+    float m = 0.0f;
+    for (int64_t c = 0; c < K; ++c) {
+        float a = fabsf(u[c]);
+        if (a > m) m = a;
+    }
+    float rm = clip_ratio * m;
+    float delta = rm / qf;
+    if (!(delta >= FLT_MIN)) {
+        for (int64_t c = 0; c < K; ++c) code[c] = 0;
+        return 0.0f;
+    }
+    float inv = 1.0f / delta;
+    for (int64_t c = 0; c < K; ++c) {
+        float scaled = u[c] * inv;
+        int v = (int)rintf(scaled); /* default rounding mode: ties to even */
+        if (v > q) v = q;
+        if (v < -q) v = -q;
+        code[c] = v;
+    }
+    return delta;
+}
+
+/* Runtime prologue (Alg. 1, runtime half, first two lines): for each token
+ * z_t = R S^-1 x_t then Eq. 5.  g is the runtime multiplier of
+ * fqo_multiplier(for_weights = 0), or NULL for S = I.
+ * If z_out != NULL it receives the transformed rows [M, K] (for tests). */
+int fqo_quantize_act(const void* x, int dtype, int64_t M, int64_t K, int64_t ldx, const float* g,
+                     int beta, int bits, float clip_ratio, uint8_t* codes, float* delta,
+                     float* z_out) {
+    if (!valid_block(beta, K) || (bits != 4 && bits != 8)) return 1;
+    if (!(clip_ratio > 0.0f && clip_ratio <= 1.0f)) return 1;
+    if (M < 0 || ldx < K || (M > 0 && (!x || !codes || !delta))) return 1;
+    float c = (float)(1.0 / sqrt((double)beta));
+    int64_t pitch = K * bits / 8;
+#pragma omp parallel
+    {
+        float* v = (float*)malloc(sizeof(float) * (size_t)K);
+        int* code = (int*)malloc(sizeof(int) * (size_t)K);
+#pragma omp for schedule(static)
+        for (int64_t t = 0; t < M; ++t) {
+            for (int64_t i = 0; i < K; ++i) {
+                float xv = load_elem(x, dtype, t * ldx + i);
+                float gi = g ? g[i] : c;
+                v[i] = xv * gi;
+            }
+            fqo_fwht_row(v, K, beta);
+            if (z_out) memcpy(z_out + t * K, v, sizeof(float) * (size_t)K);
+            delta[t] = quantize_row(v, K, bits, clip_ratio, code);
+            pack_row(code, K, bits, codes + t * pitch);
+        }
+        free(v);
+        free(code);
+    }
+    return 0;
+}
+
+/* Offline half of Alg. 1 for one consumer with round-to-nearest:
+ * row j of W~ = W S R^T is R (s (.) w_j) because the block Hadamard matrix is
+ * symmetric.  Per-output-channel step s^W_j = max|W~_j| / q, no clipping.
+ * mult_g (optional) receives the matching RUNTIME multiplier (1/s)*beta^-1/2.
+ * wt_out (optional) receives W~ [N, K] in float (for tests). */
+int fqo_fold_weights(const void* W, int dtype, int64_t N, int64_t K, int64_t ldw,
+                     const float* smooth, int beta, int bits, uint8_t* codes, float* w_scale,
+                     float* mult_g, float* wt_out) {
+    if (!valid_block(beta, K) || (bits != 4 && bits != 8)) return 1;
+    if (N < 0 || ldw < K || (N > 0 && (!W || !codes || !w_scale))) return 1;
+    float* gw = (float*)malloc(sizeof(float) * (size_t)K);
+    fqo_multiplier(smooth, K, beta, 1, gw);
+    if (mult_g) fqo_multiplier(smooth, K, beta, 0, mult_g);
+    int64_t pitch = K * bits / 8;
+#pragma omp parallel
+    {
+        float* v = (float*)malloc(sizeof(float) * (size_t)K);
+        int* code = (int*)malloc(sizeof(int) * (size_t)K);
+#pragma omp for schedule(static)
+        for (int64_t j = 0; j < N; ++j) {
+            for (int64_t i = 0; i < K; ++i) v[i] = load_elem(W, dtype, j * ldw + i) * gw[i];
+            fqo_fwht_row(v, K, beta);
+            if (wt_out) memcpy(wt_out + j * K, v, sizeof(float) * (size_t)K);
+            w_scale[j] = quantize_row(v, K, bits, 1.0f, code);
+            pack_row(code, K, bits, codes + j * pitch);
+        }
+        free(v);
+        free(code);
+    }
+    free(gw);
+    return 0;
+}
+
+/* Integer product of Eq. 8: acc[t][j] = sum_c qA[t][c] * qW[j][c], summed in
+ * 64 bits and required to fit 32.  Returns 2 if any sum does not fit. */
+int fqo_gemm_i32(const uint8_t* a_codes, const uint8_t* w_codes, int64_t M, int64_t N, int64_t K,
+                 int bits, int32_t* acc) {
+    if ((bits != 4 && bits != 8) || (K & 1)) return 1;
+    int64_t pitch = K * bits / 8;
+    int overflow = 0;
+#pragma omp parallel
+    {
+        int* arow = (int*)malloc(sizeof(int) * (size_t)(K > 0 ? K : 1));
+#pragma omp for schedule(static) reduction(| : overflow)
+        for (int64_t t = 0; t < M; ++t) {
+            for (int64_t c = 0; c < K; ++c) arow[c] = code_at(a_codes + t * pitch, c, bits);
+            for (int64_t j = 0; j < N; ++j) {
+                const uint8_t* wrow = w_codes + j * pitch;
+                int64_t s = 0;
+                for (int64_t c = 0; c < K; ++c) s += (int64_t)arow[c] * (int64_t)code_at(wrow, c, bits);
+                if (s > INT32_MAX || s < INT32_MIN) overflow = 1;
+                acc[t * N + j] = (int32_t)s;
+            }
+        }
+        free(arow);
+    }
+    return overflow ? 2 : 0;
+}
+
+/* Rescale + bias of Eq. 8: y[t][j] = s^W_j * delta_t * acc[t][j] + b_j in
+ * binary64, rounded once to the output type.  bias == NULL means b = 0. */
+int fqo_epilogue(const int32_t* acc, const float* delta, const float* w_scale, const float* bias,
+                 int64_t M, int64_t N, void* y, int ydtype, int64_t ldy) {
+    if (ldy < N) return 1;
+#pragma omp parallel for schedule(static)
+    for (int64_t t = 0; t < M; ++t) {
+        for (int64_t j = 0; j < N; ++j) {
+            double v = (double)w_scale[j] * (double)delta[t] * (double)acc[t * N + j] +
+                       (bias ? (double)bias[j] : 0.0);
+            float f = (float)v;
+            if (ydtype == FQO_BF16)
+                ((uint16_t*)y)[t * ldy + j] = f32_to_bf16(f);
+            else
+                ((float*)y)[t * ldy + j] = f;
+        }
+    }
+    return 0;
+}
+
+/* Whole runtime path for one consumer: prologue, integer product, epilogue.
+ * rows_sel (optional, n_sel entries) restricts the integer product and the
+ * epilogue to those token rows (output then has n_sel rows); the prologue
+ * always runs on all M rows. acc_out is optional. */
+int fqo_linear(const void* x, int xdtype, int64_t M, int64_t K, int64_t ldx, const float* g, int beta,
+               int bits, float clip_ratio, const uint8_t* w_codes, const float* w_scale,
+               const float* bias, int64_t N, const int64_t* rows_sel, int64_t n_sel, void* y,
+               int ydtype, int64_t ldy, uint8_t* a_codes_out, float* delta_out, int32_t* acc_out) {
+    int64_t pitch = K * bits / 8;
+    uint8_t* codes = a_codes_out ? a_codes_out : (uint8_t*)malloc((size_t)(M * pitch + 1));
+    float* delta = delta_out ? delta_out : (float*)malloc(sizeof(float) * (size_t)(M + 1));
+    int rc = fqo_quantize_act(x, xdtype, M, K, ldx, g, beta, bits, clip_ratio, codes, delta, NULL);
+    if (rc == 0) {
+        int64_t Ms = rows_sel ? n_sel : M;
+        uint8_t* ca = codes;
+        float* da = delta;
+        if (rows_sel) {
+            ca = (uint8_t*)malloc((size_t)(Ms * pitch + 1));
+            da = (float*)malloc(sizeof(float) * (size_t)(Ms + 1));
+            for (int64_t i = 0; i < Ms; ++i) {
+                memcpy(ca + i * pitch, codes + rows_sel[i] * pitch, (size_t)pitch);
+                da[i] = delta[rows_sel[i]];
+            }
+        }
+        int32_t* acc = acc_out ? acc_out : (int32_t*)malloc(sizeof(int32_t) * (size_t)(Ms * N + 1));
+        rc = fqo_gemm_i32(ca, w_codes, Ms, N, K, bits, acc);
+        if (rc == 0) rc = fqo_epilogue(acc, da, w_scale, bias, Ms, N, y, ydtype, ldy);
+        if (!acc_out) free(acc);
+        if (rows_sel) {
+            free(ca);
+            free(da);
+        }
+    }
+    if (!a_codes_out) free(codes);
+    if (!delta_out) free(delta);
+    return rc;
+}

@@ -1,0 +1,372 @@
+"""Pins for the CPU oracle: every check here compares the oracle with something
+other than itself -- an explicit Sylvester matrix product, hand-worked quantizer
+and packing cases, brute-force loops, closed forms and the identities the paper
+states (fold identity, H H^T = beta I, norm preservation, amplitude invariance,
+zero token -> bias)."""
+import os
+
+import numpy as np
+import pytest
+
+import oracle
+from paper_2609_24433_b200 import synth
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def sylvester(n: int) -> np.ndarray:
+    """H_1 = [1], H_2n = [[H, H], [H, -H]] (entries +-1), built independently of the oracle."""
+    H = np.array([[1]], dtype=np.int64)
+    while H.shape[0] < n:
+        H = np.block([[H, H], [H, -H]])
+    return H
+
+
+def inv_transform(z: np.ndarray, beta: int) -> np.ndarray:
+    """x with R x = z for the normalised block Hadamard R (R is an involution): exact
+    float64 matrix product, used only to craft oracle inputs."""
+    H = sylvester(beta).astype(np.float64)
+    zb = z.reshape(-1, beta).astype(np.float64)
+    return (zb @ H.T / np.sqrt(beta)).reshape(z.shape)
+
+
+# ------------------------------------------------------------------ FWHT ----
+@pytest.mark.parametrize("beta", [2, 4, 8, 16, 32, 64, 128, 256])
+def test_fwht_basis_vectors_give_sylvester_columns(beta):
+    H = sylvester(beta)
+    # entry rule H[i][j] = (-1)^popcount(i & j)
+    i, j = np.meshgrid(np.arange(beta), np.arange(beta), indexing="ij")
+    pop = np.array([[bin(a & b).count("1") for b in range(beta)] for a in range(beta)])
+    assert np.array_equal(H, (-1) ** pop)
+    for col in range(beta):
+        e = np.zeros(beta, dtype=np.float32)
+        e[col] = 1.0
+        assert np.array_equal(oracle.fwht_block(e).astype(np.int64), H[:, col])
+
+
+@pytest.mark.parametrize("beta", [2, 4, 8, 16, 32, 64, 128, 256])
+def test_fwht_integer_inputs_equal_exact_matrix_product(beta):
+    rng = np.random.default_rng(beta)
+    H = sylvester(beta)
+    for _ in range(8):
+        x = rng.integers(-1024, 1025, size=beta)
+        got = oracle.fwht_block(x.astype(np.float32))
+        assert np.array_equal(got.astype(np.int64), H @ x)          # exact in binary32
+        # H H^T = beta I  (applying the butterfly network twice)
+        if beta <= 64:
+            twice = oracle.fwht_block(got)
+            assert np.array_equal(twice.astype(np.int64), beta * x)
+
+
+def test_fwht_is_not_symmetric_mistake_detector():
+    # A non-symmetric probe: a wrong pairing (i, i+h swapped, or descending order with
+    # wrong sign) changes the image of this vector.
+    x = np.array([1, 2, 3, 4, 5, 6, 7, 8], dtype=np.float32)
+    assert np.array_equal(oracle.fwht_block(x), np.array([36, -4, -8, 0, -16, 0, 0, 0], np.float32))
+
+
+@pytest.mark.parametrize("beta", [32, 64, 128, 256])
+def test_normalised_rotation_preserves_norm_and_is_involution(beta):
+    rng = np.random.default_rng(7)
+    K = 4 * beta
+    x = rng.standard_normal((3, K)).astype(np.float32)
+    _, _, z = oracle.quantize_act(x, "f32", None, beta, 8, return_z=True)
+    assert np.allclose((z.astype(np.float64) ** 2).sum(1), (x.astype(np.float64) ** 2).sum(1), rtol=1e-5)
+    _, _, back = oracle.quantize_act(z, "f32", None, beta, 8, return_z=True)
+    assert np.allclose(back, x, rtol=0, atol=2e-5)
+    # against the explicit normalised matrix in float64
+    H = sylvester(beta) / np.sqrt(beta)
+    ref = (x.reshape(3, -1, beta).astype(np.float64) @ H.T).reshape(3, K)
+    assert np.allclose(z, ref, rtol=0, atol=1e-5)
+
+
+@pytest.mark.parametrize("beta", [4, 16, 64, 256])
+def test_power_of_two_normalisation_commutes_exactly(beta):
+    # beta^(-1/2) is a power of two: scaling before or after the butterflies is bit-identical.
+    rng = np.random.default_rng(11)
+    x = rng.standard_normal((2, 2 * beta)).astype(np.float32)
+    _, _, z = oracle.quantize_act(x, "f32", None, beta, 8, return_z=True)
+    post = np.stack([np.concatenate([oracle.fwht_block(r[b:b + beta]) for b in range(0, r.size, beta)])
+                     for r in x]) * np.float32(1.0 / np.sqrt(beta))
+    assert np.array_equal(z, post.astype(np.float32))
+
+
+def test_blocks_are_independent():
+    beta, K = 32, 96
+    x = np.zeros((1, K), dtype=np.float32)
+    x[0, 40] = 3.0                                     # lives in block 1 only
+    _, _, z = oracle.quantize_act(x, "f32", np.ones(K, np.float32), beta, 8, return_z=True)
+    assert np.all(z[0, :32] == 0) and np.all(z[0, 64:] == 0)
+    assert np.array_equal(np.abs(z[0, 32:64]), np.full(32, 3.0, np.float32))
+
+
+# ------------------------------------------------------------- quantizer ----
+def _read_quant_cases():
+    cases = []
+    with open(os.path.join(GOLDEN, "quantizer_cases.txt")) as f:
+        for line in f:
+            line = line.strip()
+            if not line or line.startswith("#"):
+                continue
+            bits, r, z, delta, codes = [p.strip() for p in line.split("|")]
+            cases.append((int(bits), float(r), np.array(z.split(), dtype=np.float64), float(delta),
+                          np.array(codes.split(), dtype=np.int32)))
+    return cases
+
+
+@pytest.mark.parametrize("case", _read_quant_cases())
+def test_quantizer_hand_cases(case):
+    bits, r, z, delta, codes = case
+    x = inv_transform(z, 4).astype(np.float32)[None, :]   # exact: dyadic values
+    got_codes, got_delta, got_z = oracle.quantize_act(x, "f32", None, 4, bits, r, return_z=True)
+    assert np.array_equal(got_z[0].astype(np.float64), z)
+    assert got_delta[0] == np.float32(delta)
+    assert np.array_equal(oracle.unpack(got_codes, z.size, bits)[0], codes)
+
+
+@pytest.mark.parametrize("bits", [4, 8])
+def test_codes_range_and_extreme_code_is_q(bits):
+    q = 7 if bits == 4 else 127
+    d = synth.make_site(synth.Site("t", 37, 512, [("p", 8)], beta=64, bits=bits, x_dtype="f32"), seed=3)
+    codes, delta = oracle.quantize_act(d.x, "f32", None, 64, bits)
+    c = oracle.unpack(codes, 512, bits)
+    assert c.min() >= -q and c.max() <= q
+    assert np.array_equal(np.abs(c).max(1), np.full(37, q))
+    assert np.all(delta > 0)
+
+
+@pytest.mark.parametrize("bits", [4, 8])
+def test_step_is_absmax_over_whole_token(bits):
+    # two Hadamard blocks with very different ranges share one step
+    q = 7.0 if bits == 4 else 127.0
+    z = np.concatenate([np.full(4, 0.5), np.array([64.0, 0, 0, 0])])
+    x = inv_transform(z, 4).astype(np.float32)[None, :]
+    codes, delta = oracle.quantize_act(x, "f32", None, 4, bits)
+    assert delta[0] == np.float32(np.float32(64.0) / np.float32(q))
+    c = oracle.unpack(codes, 8, bits)[0]
+    assert c[4] == q and np.all(c[:4] == int(np.rint(0.5 / (64.0 / q))))
+
+
+@pytest.mark.parametrize("bits", [4, 8])
+@pytest.mark.parametrize("k", [-20, -3, 1, 9])
+def test_amplitude_invariance(bits, k):
+    # Proposition 2: scaling a token by 2^k leaves the codes and scales the step exactly.
+    d = synth.make_site(synth.Site("t", 16, 256, [("p", 8)], beta=64, bits=bits, x_dtype="f32"), seed=5)
+    c0, d0 = oracle.quantize_act(d.x, "f32", None, 64, bits)
+    c1, d1 = oracle.quantize_act(d.x * np.float32(2.0 ** k), "f32", None, 64, bits)
+    assert np.array_equal(c0, c1)
+    assert np.array_equal(d1, d0 * np.float32(2.0 ** k))
+
+
+@pytest.mark.parametrize("bits", [4, 8])
+def test_zero_and_tiny_tokens_give_zero_codes_and_bias_output(bits):
+    K, N = 128, 16
+    rng = np.random.default_rng(1)
+    x = rng.standard_normal((4, K)).astype(np.float32)
+    x[1] = 0.0
+    x[2] = np.float32(1e-42)                            # denormal token: step below FLT_MIN
+    W = synth.draw_weights(rng, N, K)
+    bias = rng.standard_normal(N).astype(np.float32)
+    wc, ws, g = oracle.fold_weights(W, "f32", None, 32, bits)
+    y, codes, delta, acc = oracle.linear(x, "f32", g, 32, bits, 1.0, wc, ws, bias)
+    for t in (1, 2):
+        assert delta[t] == 0.0 and not codes[t].any() and not acc[t].any()
+        assert np.array_equal(y[t], bias)
+    assert delta[0] > 0 and delta[3] > 0
+
+
+# ------------------------------------------------------------------ pack ----
+def test_pack_hand_cases_and_roundtrip():
+    with open(os.path.join(GOLDEN, "pack_cases.txt")) as f:
+        for line in f:
+            line = line.strip()
+            if not line or line.startswith("#"):
+                continue
+            codes, hexes = [p.strip() for p in line.split("|")]
+            c = np.array(codes.split(), dtype=np.int32)[None, :]
+            want = np.array([int(h, 16) for h in hexes.split()], dtype=np.uint8)
+            assert np.array_equal(oracle.pack(c, 4)[0], want)
+    rng = np.random.default_rng(0)
+    for bits, q in ((4, 7), (8, 127)):
+        c = rng.integers(-q, q + 1, size=(5, 64)).astype(np.int32)
+        assert np.array_equal(oracle.unpack(oracle.pack(c, bits), 64, bits), c)
+    assert np.array_equal(oracle.pack(np.array([[-128, 127, -1]], np.int32)[:, :2], 8).view(np.int8)[0],
+                          np.array([-128, 127], np.int8))
+
+
+# ------------------------------------------------------------------ GEMM ----
+@pytest.mark.parametrize("bits", [4, 8])
+def test_integer_gemm_equals_brute_force(bits):
+    q = 7 if bits == 4 else 127
+    rng = np.random.default_rng(bits)
+    M, N, K = 5, 7, 64
+    a = rng.integers(-q, q + 1, size=(M, K)).astype(np.int32)
+    w = rng.integers(-q, q + 1, size=(N, K)).astype(np.int32)
+    got = oracle.gemm_i32(oracle.pack(a, bits), oracle.pack(w, bits), K, bits)
+    want = np.zeros((M, N), dtype=np.int64)
+    for t in range(M):
+        for j in range(N):
+            s = 0
+            for c in range(K):
+                s += int(a[t, c]) * int(w[j, c])
+            want[t, j] = s
+    assert np.array_equal(got.astype(np.int64), want)
+    # a transposed-operand mistake would change this non-square case
+    assert got.shape == (M, N)
+
+
+@pytest.mark.parametrize("bits", [4, 8])
+def test_integer_gemm_extremes_and_one_hot(bits):
+    q = 7 if bits == 4 else 127
+    K = 4096
+    a = np.full((2, K), q, np.int32)
+    w = np.full((3, K), -q, np.int32)
+    assert np.all(oracle.gemm_i32(oracle.pack(a, bits), oracle.pack(w, bits), K, bits) == -q * q * K)
+    rng = np.random.default_rng(2)
+    w = rng.integers(-q, q + 1, size=(6, 32)).astype(np.int32)
+    a = np.zeros((32, 32), np.int32)
+    a[np.arange(32), np.arange(32)] = 1                   # one-hot rows pick single weights
+    assert np.array_equal(oracle.gemm_i32(oracle.pack(a, bits), oracle.pack(w, bits), 32, bits), w.T)
+    assert 127 * 127 * 131072 < 2 ** 31                   # accumulator bound at the largest K accepted
+
+
+# ------------------------------------------------------------------ fold ----
+@pytest.mark.parametrize("beta", [32, 64, 128, 256])
+@pytest.mark.parametrize("smoothed", [False, True])
+def test_fold_identity_before_rounding(beta, smoothed):
+    # (W S R^T)(R S^-1 x) = W x
+    rng = np.random.default_rng(beta)
+    K, N, M = 512, 24, 9
+    x = rng.standard_normal((M, K)).astype(np.float32)
+    W = synth.draw_weights(rng, N, K)
+    s = np.exp(rng.uniform(-2, 2, K)).astype(np.float32) if smoothed else None
+    _, _, g, wt = oracle.fold_weights(W, "f32", s, beta, 8, return_wt=True)
+    _, _, z = oracle.quantize_act(x, "f32", g, beta, 8, return_z=True)
+    want = x.astype(np.float64) @ W.astype(np.float64).T
+    got = z.astype(np.float64) @ wt.astype(np.float64).T
+    assert np.abs(got - want).max() <= 1e-5 * np.abs(want).max()
+    if not smoothed:
+        assert np.allclose(np.linalg.norm(wt, axis=1), np.linalg.norm(W, axis=1), rtol=1e-5)
+        assert np.array_equal(g, np.full(K, np.float32(1.0 / np.sqrt(beta))))
+    else:
+        c = np.float32(1.0 / np.sqrt(beta))
+        assert np.array_equal(g, (np.float32(1.0) / s) * c)
+
+
+def test_fold_mismatch_is_detected():
+    # A consumer folded with another block size than the runtime uses is badly wrong.
+    rng = np.random.default_rng(0)
+    K, N, M = 512, 32, 16
+    x = rng.standard_normal((M, K)).astype(np.float32)
+    W = synth.draw_weights(rng, N, K)
+    want = x.astype(np.float64) @ W.astype(np.float64).T
+    wc, ws, g = oracle.fold_weights(W, "f32", None, 64, 8)
+    good = oracle.linear(x, "f32", g, 64, 8, 1.0, wc, ws, None)[0]
+    bad = oracle.linear(x, "f32", oracle.multiplier(None, K, 128, False), 128, 8, 1.0, wc, ws, None)[0]
+    rel = lambda y: np.linalg.norm(y - want) / np.linalg.norm(want)
+    assert rel(good) < 0.02 and rel(bad) > 0.5
+
+
+@pytest.mark.parametrize("bits", [4, 8])
+def test_weight_rounding_is_rtn_per_output_channel(bits):
+    q = 7 if bits == 4 else 127
+    rng = np.random.default_rng(4)
+    W = synth.draw_weights(rng, 10, 256)
+    W[3] = 0.0
+    codes, ws, _, wt = oracle.fold_weights(W, "f32", None, 64, bits, return_wt=True)
+    c = oracle.unpack(codes, 256, bits)
+    assert ws[3] == 0 and not c[3].any()
+    rows = [j for j in range(10) if j != 3]
+    assert np.array_equal(np.abs(c[rows]).max(1), np.full(9, q))
+    assert np.array_equal(ws[rows], (np.abs(wt[rows]).max(1) / np.float32(q)).astype(np.float32))
+    # nearest code: |W~ - s*code| <= s/2 (+ rounding slack)
+    err = np.abs(wt[rows] - ws[rows, None] * c[rows])
+    assert np.all(err <= 0.5 * ws[rows, None] * (1 + 1e-5))
+
+
+# -------------------------------------------------------------- epilogue ----
+@pytest.mark.parametrize("bits", [4, 8])
+def test_eq8_equals_product_of_dequantised_operands(bits):
+    d = synth.make_site(synth.Site("t", 12, 256, [("p", 40)], beta=64, bits=bits, x_dtype="f32",
+                                   y_dtype="f32"), seed=9)
+    W, b = d.W["p"], d.bias["p"]
+    wc, ws, g = oracle.fold_weights(W, "f32", None, 64, bits)
+    y, codes, delta, acc = oracle.linear(d.x, "f32", g, 64, bits, 1.0, wc, ws, b)
+    zhat = delta[:, None].astype(np.float64) * oracle.unpack(codes, 256, bits)
+    what = ws[:, None].astype(np.float64) * oracle.unpack(wc, 256, bits)
+    want = zhat @ what.T + b
+    assert np.abs(y - want).max() <= 1e-6 * np.abs(want).max()
+    # bf16 output is the float result rounded to nearest even
+    yb = oracle.epilogue(acc, delta, ws, b, "bf16")
+    assert np.array_equal(yb, synth.f32_to_bf16_bits(y))
+
+
+def test_int8_sites_are_more_accurate_than_int4():
+    d = synth.make_site(synth.Site("t", 64, 1024, [("p", 128)], beta=128, bits=4, x_dtype="f32"), seed=21)
+    W = d.W["p"]
+    want = d.x.astype(np.float64) @ W.astype(np.float64).T
+    rel = {}
+    for bits in (4, 8):
+        wc, ws, g = oracle.fold_weights(W, "f32", None, 128, bits)
+        y = oracle.linear(d.x, "f32", g, 128, bits, 1.0, wc, ws, None)[0]
+        rel[bits] = np.linalg.norm(y - want) / np.linalg.norm(want)
+    assert rel[8] < 0.03 and rel[8] < rel[4] < 0.5
+
+
+def test_rows_subset_matches_full():
+    d = synth.make_site(synth.Site("t", 20, 256, [("p", 24)], beta=32, bits=4, x_dtype="bf16"), seed=2)
+    wc, ws, g = oracle.fold_weights(d.W["p"], "f32", None, 32, 4)
+    full = oracle.linear(d.x, "bf16", g, 32, 4, 1.0, wc, ws, d.bias["p"], "bf16")
+    sub = oracle.linear(d.x, "bf16", g, 32, 4, 1.0, wc, ws, d.bias["p"], "bf16", rows=[19, 0, 7])
+    assert np.array_equal(sub[0], full[0][[19, 0, 7]])
+    assert np.array_equal(sub[3], full[3][[19, 0, 7]])
+
+
+# --------------------------------------------------------- smoothing scale ----
+def test_smoothing_scale_closed_forms():
+    rng = np.random.default_rng(3)
+    a = np.exp(rng.uniform(-3, 3, 64)).astype(np.float32)
+    w = np.exp(rng.uniform(-3, 1, 64)).astype(np.float32)
+    s1 = oracle.smooth_scale(a, w, 1.0)
+    assert np.allclose(a / s1, 1.0, rtol=1e-6)             # alpha = 1 equalises calibrated ranges
+    s0 = oracle.smooth_scale(a, w, 0.0)
+    assert np.allclose(s0 * w, 1.0, rtol=1e-6)
+    sh = oracle.smooth_scale(a, w, 0.5)
+    assert np.allclose(a / sh, w * sh, rtol=1e-5)           # alpha = 1/2 balances both sides
+    assert np.allclose(sh, np.sqrt(a.astype(np.float64) / w.astype(np.float64)), rtol=1e-6)
+    # floors and bounds
+    s = oracle.smooth_scale(np.array([0.0, 1e9], np.float32), np.array([1e9, 0.0], np.float32), 0.5)
+    assert s[0] == np.float32(1e-5) and s[1] == np.float32(1e5)
+
+
+def test_col_absmax_against_numpy():
+    rng = np.random.default_rng(8)
+    x = rng.standard_normal((33, 48)).astype(np.float32)
+    assert np.array_equal(oracle.col_absmax(x), np.abs(x).max(0))
+    xb = synth.f32_to_bf16_bits(x)
+    assert np.array_equal(oracle.col_absmax(xb, "bf16"), np.abs(synth.bf16_bits_to_f32(xb)).max(0))
+
+
+def test_smoothing_moves_outliers_into_weights():
+    site = synth.config1_site()
+    d = synth.make_site(site, seed=0, calib_tokens=512)
+    a = oracle.col_absmax(d.calib)
+    w = oracle.col_absmax(d.W["proj"])
+    s = oracle.smooth_scale(a, w, site.alpha)
+    ch = d.outlier_channels
+    assert s[ch].min() > 3 * np.median(s)
+    want = d.x.astype(np.float64) @ d.W["proj"].astype(np.float64).T
+    wc, ws, g = oracle.fold_weights(d.W["proj"], "f32", s, site.beta, 4)
+    y = oracle.linear(d.x, "f32", g, site.beta, 4, 1.0, wc, ws, None)[0]
+    assert np.linalg.norm(y - want) / np.linalg.norm(want) < 0.35
+
+
+# ------------------------------------------------------------ bf16 helpers ----
+def test_bf16_helpers_match_torch():
+    import torch
+    rng = np.random.default_rng(0)
+    x = (rng.standard_normal(4096) * np.exp(rng.uniform(-20, 20, 4096))).astype(np.float32)
+    want = torch.from_numpy(x).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    assert np.array_equal(synth.f32_to_bf16_bits(x), want)
+    assert np.array_equal(synth.bf16_bits_to_f32(want),
+                          torch.from_numpy(x).to(torch.bfloat16).float().numpy())
