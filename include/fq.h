@@ -1,0 +1,152 @@
+/*
+ * fq.h -- C ABI of the B200 (sm_100a) folded quantized linear layer.
+ *
+ * One projection site of the method runs as
+ *   offline : W~ = W S R^T, round to nearest per output channel, pack   (Alg. 1, offline half; Eq. 3)
+ *   runtime : z_t = R S^-1 x_t, per-token symmetric quantization         (Alg. 1 runtime half; Eq. 5)
+ *             c = q^W q^A (int32), y = delta_t (s^W (.) c) + b           (Eq. 8)
+ * with R the normalised block Hadamard transform applied as an FWHT.
+ *
+ * Conventions that hold for every entry point
+ *   - "device" pointers are CUDA global-memory addresses on the current device,
+ *     "host" pointers are ordinary process memory.  The kind is stated per argument.
+ *   - Matrices are row-major; a leading dimension (ld*) counts ELEMENTS between rows.
+ *     Activations are [M tokens, K channels]; weights are [N output channels, K].
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *     All work is enqueued on it; no entry point synchronises unless it says so.
+ *   - The caller owns every buffer except the memory inside an fq_weights handle.
+ *     Inputs are never written.  Output rows >= M and bytes outside the stated
+ *     shapes are never touched.
+ *   - Errors are return codes.  Nothing aborts, throws or traps.  Argument checks run
+ *     on the host before any launch; a failed check launches nothing.
+ *   - Inputs must be finite; NaN/Inf give unspecified codes (never a fault).
+ *   - Supported sizes: hadamard_block a power of two in [2, 256] dividing K;
+ *     K a multiple of 32 and <= 131072 (int32 accumulator bound; the prologue and the fold
+ *     keep a whole token in one thread block and accept K <= 32768); N a multiple of 8;
+ *     bits 4 or 8; clip_ratio in (0, 1].  M = 0 or N = 0 succeeds and does nothing.
+ *   - Device pointers must be 16-byte aligned and ld* a multiple of 8 elements.
+ *   - Arithmetic of the transform and quantizer is IEEE binary32, round to nearest
+ *     even, no fused multiply-add, ascending butterfly strides; ties in round() go
+ *     to even.  4-bit codes are two's-complement nibbles, even channel in the low
+ *     nibble, row pitch K/2 bytes; 8-bit codes are int8, row pitch K bytes.
+ */
+#ifndef FQ_H_
+#define FQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    FQ_OK = 0,
+    FQ_ERR_INVALID_ARG = 1, /* NULL where data is required, negative size, bits not 4/8, bad clip ratio */
+    FQ_ERR_UNSUPPORTED = 2, /* size or block outside the supported set, handle/call bit width mismatch */
+    FQ_ERR_ALIGNMENT = 3,   /* pointer not 16-byte aligned or leading dimension not a multiple of 8 */
+    FQ_ERR_ARCH = 4,        /* current device is not compute capability 10.x */
+    FQ_ERR_CUDA = 5,        /* a CUDA runtime/driver call failed */
+    FQ_ERR_NOMEM = 6,       /* allocation failed, or caller workspace too small */
+    FQ_ERR_TIMEOUT = 7      /* a bounded device-side wait expired (see fq_device_status) */
+} fq_status;
+
+typedef enum { FQ_F32 = 0, FQ_BF16 = 1 } fq_dtype;
+
+/* Opaque folded-weight pack of one consumer projection (or several consumers of one
+ * site concatenated along N).  Owns device memory; immutable after creation. */
+typedef struct fq_weights fq_weights;
+
+const char* fq_status_string(fq_status s);
+
+/* ---- offline: fold + round + pack (Alg. 1 offline half, Eq. 3 fold-before, RTN) ----------
+ * W      device, [N, K] of dtype wt, leading dimension ldw.
+ * smooth device float[K] SmoothQuant scales s_c, or NULL for S = I.
+ * bias   device float[N] or NULL (= 0); copied into the handle unchanged (output transform is I).
+ * Creates *out holding: packed codes [N, K*bits/8], s^W[N], bias[N] and the runtime multiplier
+ * g[K] = (1/s_c) * block^-1/2.  Allocates with cudaMalloc (this call only); work is async on stream.
+ * Row j of W~ is FWHT(s (.) w_j * block^-1/2); s^W_j = max|W~_j| / q; no weight clipping. */
+fq_status fq_fold_weights(const void* W, fq_dtype wt, int64_t N, int64_t K, int64_t ldw,
+                          const float* smooth, const float* bias, int hadamard_block, int bits,
+                          void* stream, fq_weights** out);
+
+/* Frees the handle's device memory (cudaFree synchronises the device). NULL is accepted. */
+fq_status fq_weights_destroy(fq_weights* w);
+
+/* Shape query (host). Any out pointer may be NULL. */
+fq_status fq_weights_info(const fq_weights* w, int64_t* N, int64_t* K, int* hadamard_block, int* bits);
+
+/* Device pointer to the handle's runtime multiplier g[K] (valid until destroy). */
+const float* fq_weights_multiplier(const fq_weights* w);
+
+/* Copy the canonical pack out of / into a handle.  All pointers are device pointers with
+ * the shapes listed for fq_fold_weights; any destination may be NULL to skip it.
+ * Import allocates a new handle; bias may be NULL (= 0). */
+fq_status fq_weights_export(const fq_weights* w, void* codes, float* w_scale, float* mult_g, float* bias,
+                            void* stream);
+fq_status fq_weights_import(const void* codes, const float* w_scale, const float* mult_g,
+                            const float* bias, int64_t N, int64_t K, int hadamard_block, int bits,
+                            void* stream, fq_weights** out);
+
+/* ---- calibration support (section "Transforms supported by the runtime", SmoothQuant scale) --
+ * fq_col_absmax: out[c] = max(out[c] if accumulate else 0, max_t |x[t][c]|); x device [M, K].
+ * fq_smooth_scale: s_c = clamp(max(a_c,1e-5)^alpha / max(w_c,1e-5)^(1-alpha), 1e-5, 1e5) in
+ * binary64 on the device; a, w, s device float[K]; alpha in [0, 1]. */
+fq_status fq_col_absmax(const void* x, fq_dtype xt, int64_t M, int64_t K, int64_t ldx, int accumulate,
+                        float* out, void* stream);
+fq_status fq_smooth_scale(const float* a, const float* w, int64_t K, double alpha, float* s, void* stream);
+
+/* ---- runtime prologue (Alg. 1 runtime half lines 1-2; Eq. 5) ----------------------------------
+ * x       device [M, K] of dtype xt, leading dimension ldx.
+ * mult_g  device float[K] (fq_weights_multiplier of any consumer of the site) or NULL (S = I).
+ * codes_out device, [M, K*bits/8] bytes, canonical packing, pitch K*bits/8.
+ * delta_out device float[M]: delta_t = (clip_ratio * max_c|z_tc|) / q, 0 for a zero token
+ * (a token whose step would be below FLT_MIN), whose codes are all 0. */
+fq_status fq_quantize_act(const void* x, fq_dtype xt, int64_t M, int64_t K, int64_t ldx,
+                          const float* mult_g, int hadamard_block, int bits, float clip_ratio,
+                          void* codes_out, float* delta_out, void* stream);
+
+/* ---- integer GEMM + rescale/bias epilogue on pre-quantized activations (Eq. 8) -----------------
+ * a_codes device, canonical codes from fq_quantize_act with the same bit width as W.
+ * a_delta device float[M].   y device [M, N] of dtype yt, leading dimension ldy.
+ * workspace device, at least fq_workspace_bytes(M, K, N, bits) bytes, 256-byte aligned; contents
+ * are scratch (calls sharing a workspace must be stream-ordered).
+ * Shared sites: quantize once, then call this once per consumer handle. */
+fq_status fq_gemm_w4a4(const void* a_codes, const float* a_delta, int64_t M, const fq_weights* W,
+                       void* y, fq_dtype yt, int64_t ldy, void* workspace, size_t ws_bytes, void* stream);
+fq_status fq_gemm_w8a8(const void* a_codes, const float* a_delta, int64_t M, const fq_weights* W,
+                       void* y, fq_dtype yt, int64_t ldy, void* workspace, size_t ws_bytes, void* stream);
+
+/* ---- whole runtime path of one consumer: prologue + GEMM + epilogue (Alg. 1 runtime half) ------
+ * Equivalent to fq_quantize_act (codes and delta kept in the workspace) followed by fq_gemm_*.
+ * K, N, block and bits come from the handle; the handle's bit width must match the entry point. */
+fq_status fq_linear_w4a4(const void* x, fq_dtype xt, int64_t M, int64_t ldx, const fq_weights* W,
+                         float clip_ratio, void* y, fq_dtype yt, int64_t ldy, void* workspace,
+                         size_t ws_bytes, void* stream);
+fq_status fq_linear_w8a8(const void* x, fq_dtype xt, int64_t M, int64_t ldx, const fq_weights* W,
+                         float clip_ratio, void* y, fq_dtype yt, int64_t ldy, void* workspace,
+                         size_t ws_bytes, void* stream);
+
+/* Bytes of workspace that fq_gemm_* / fq_linear_* need for this shape (host computation). */
+size_t fq_workspace_bytes(int64_t M, int64_t K, int64_t N, int bits);
+
+/* Parity/debug: raw int32 accumulators acc[M, N] (device, pitch N) of Eq. 8's integer sum. */
+fq_status fq_gemm_acc_i32(const void* a_codes, int64_t M, const fq_weights* W, int32_t* acc,
+                          void* workspace, size_t ws_bytes, void* stream);
+
+/* On-device second witness (Eq. 8 with CUDA-core dp4a arithmetic, untuned): same arguments as
+ * fq_gemm_*; if acc != NULL it receives raw int32 accumulators [M, N] and y is ignored.  Used by the
+ * tests to cross-check the tensor-core kernel at sizes where the CPU oracle can only sample. */
+fq_status fq_gemm_simt(const void* a_codes, const float* a_delta, int64_t M, const fq_weights* W, void* y,
+                       fq_dtype yt, int64_t ldy, int32_t* acc, void* workspace, size_t ws_bytes, void* stream);
+
+/* Device-side wait watchdog.  Every spin on an mbarrier inside the kernels is bounded; a wait
+ * that expires records a code in a device word and the kernel winds down normally.  This call
+ * SYNCHRONISES the device, returns FQ_ERR_TIMEOUT if any kernel recorded an expiry since the
+ * last call (and clears the record), else FQ_OK.  *detail (host, may be NULL) gets the raw word. */
+fq_status fq_device_status(uint32_t* detail);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FQ_H_ */

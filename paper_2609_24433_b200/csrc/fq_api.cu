@@ -1,0 +1,386 @@
+// C ABI of the library (see include/fq.h): host-side argument checks, handle
+// management and stream-ordered dispatch.  No entry point below touches data on
+// the host; every step of the path runs in the kernels of this library.
+#include <math.h>
+#include <new>
+
+#include "fq_common.cuh"
+
+using namespace fq;
+
+namespace {
+
+constexpr int64_t kMaxK = 131072;       // 127^2 * K and 256 * 49 * K stay below 2^31
+constexpr int64_t kMaxPrologueK = 32768; // one token must fit the registers of one CTA
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+bool valid_block(int block, int64_t K) {
+    return block >= 2 && block <= 256 && (block & (block - 1)) == 0 && K > 0 && K % block == 0;
+}
+
+float block_norm(int block) { return (float)(1.0 / sqrt((double)block)); }
+
+fq_status check_arch() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return FQ_ERR_CUDA;
+    int major = 0;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return FQ_ERR_CUDA;
+    return major == 10 ? FQ_OK : FQ_ERR_ARCH;
+}
+
+fq_status check_shape(int64_t N, int64_t K, int block, int bits) {
+    if (N < 0 || K <= 0) return FQ_ERR_INVALID_ARG;
+    if (bits != 4 && bits != 8) return FQ_ERR_INVALID_ARG;
+    if (!valid_block(block, K) || K % 32 != 0 || K > kMaxK || N % 8 != 0) return FQ_ERR_UNSUPPORTED;
+    return FQ_OK;
+}
+
+fq_status alloc_handle(int64_t N, int64_t K, int block, int bits, Weights** out) {
+    Weights* w = new (std::nothrow) Weights();
+    if (!w) return FQ_ERR_NOMEM;
+    w->N = N; w->K = K; w->block = block; w->bits = bits;
+    cudaGetDevice(&w->device);
+    const size_t code_bytes = (size_t)N * (size_t)K * bits / 8;
+    bool ok = true;
+    ok = ok && cudaMalloc(&w->codes, code_bytes > 0 ? code_bytes : 16) == cudaSuccess;
+    ok = ok && cudaMalloc(&w->w_scale, sizeof(float) * (size_t)(N > 0 ? N : 4)) == cudaSuccess;
+    ok = ok && cudaMalloc(&w->bias, sizeof(float) * (size_t)(N > 0 ? N : 4)) == cudaSuccess;
+    ok = ok && cudaMalloc(&w->mult_g, sizeof(float) * (size_t)K) == cudaSuccess;
+    if (!ok) {
+        cudaGetLastError();
+        cudaFree(w->codes); cudaFree(w->w_scale); cudaFree(w->bias); cudaFree(w->mult_g);
+        delete w;
+        return FQ_ERR_NOMEM;
+    }
+    *out = w;
+    return FQ_OK;
+}
+
+struct Workspace {
+    int8_t* a8;
+    float* delta;
+};
+
+size_t ws_bytes_needed(int64_t M, int64_t K) {
+    return align_up((size_t)M * (size_t)K, 256) + align_up(sizeof(float) * (size_t)M, 256);
+}
+
+fq_status carve(void* workspace, size_t ws_bytes, int64_t M, int64_t K, Workspace* ws) {
+    if (!workspace) return FQ_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return FQ_ERR_ALIGNMENT;
+    if (ws_bytes < ws_bytes_needed(M, K)) return FQ_ERR_NOMEM;
+    ws->a8 = static_cast<int8_t*>(workspace);
+    ws->delta = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + align_up((size_t)M * (size_t)K, 256));
+    return FQ_OK;
+}
+
+fq_status check_y(const void* y, fq_dtype yt, int64_t ldy, int64_t N) {
+    if (!y) return FQ_ERR_INVALID_ARG;
+    if (yt != FQ_F32 && yt != FQ_BF16) return FQ_ERR_INVALID_ARG;
+    if (ldy < N) return FQ_ERR_INVALID_ARG;
+    if (!aligned16(y) || ldy % 8 != 0) return FQ_ERR_ALIGNMENT;
+    return FQ_OK;
+}
+
+// a_codes: canonical codes of width W->bits.  Produces the int8 operand of the GEMM.
+fq_status gemm_from_codes(const void* a_codes, const float* a_delta, int64_t M, const fq_weights* Wp, int bits,
+                          const GemmOut& out, void* workspace, size_t ws_bytes, cudaStream_t stream, bool simt) {
+    const Weights* W = reinterpret_cast<const Weights*>(Wp);
+    if (!W || M < 0) return FQ_ERR_INVALID_ARG;
+    if (W->bits != bits) return FQ_ERR_UNSUPPORTED;
+    if (M == 0 || W->N == 0) return FQ_OK;
+    if (!a_codes || (!a_delta && !out.acc)) return FQ_ERR_INVALID_ARG;
+    if (!aligned16(a_codes)) return FQ_ERR_ALIGNMENT;
+    fq_status st = check_arch();
+    if (st != FQ_OK) return st;
+    const int8_t* a8 = static_cast<const int8_t*>(a_codes);
+    int shift = 0;
+    if (bits == 4) {
+        Workspace ws;
+        st = carve(workspace, ws_bytes, M, W->K, &ws);
+        if (st != FQ_OK) return st;
+        if (launch_expand_nibbles(a_codes, M, W->K, ws.a8, stream) != cudaSuccess) return FQ_ERR_CUDA;
+        a8 = ws.a8;
+        shift = 8;   // both operands carry 16*code
+    }
+    if (simt) return launch_gemm_simt(a8, M, *W, shift, out, stream) == cudaSuccess ? FQ_OK : FQ_ERR_CUDA;
+    return launch_gemm_tcgen05(a8, M, *W, shift, out, stream);
+}
+
+fq_status linear_impl(const void* x, fq_dtype xt, int64_t M, int64_t ldx, const fq_weights* Wp, int bits,
+                      float clip_ratio, void* y, fq_dtype yt, int64_t ldy, void* workspace, size_t ws_bytes,
+                      void* stream) {
+    const Weights* W = reinterpret_cast<const Weights*>(Wp);
+    if (!W || M < 0) return FQ_ERR_INVALID_ARG;
+    if (W->bits != bits) return FQ_ERR_UNSUPPORTED;
+    if (!(clip_ratio > 0.0f && clip_ratio <= 1.0f)) return FQ_ERR_INVALID_ARG;
+    if (xt != FQ_F32 && xt != FQ_BF16) return FQ_ERR_INVALID_ARG;
+    if (M == 0 || W->N == 0) return FQ_OK;
+    if (!x || ldx < W->K) return FQ_ERR_INVALID_ARG;
+    if (!aligned16(x) || ldx % 8 != 0) return FQ_ERR_ALIGNMENT;
+    if (W->K > kMaxPrologueK) return FQ_ERR_UNSUPPORTED;
+    fq_status st = check_y(y, yt, ldy, W->N);
+    if (st != FQ_OK) return st;
+    st = check_arch();
+    if (st != FQ_OK) return st;
+    Workspace ws;
+    st = carve(workspace, ws_bytes, M, W->K, &ws);
+    if (st != FQ_OK) return st;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // Prologue writes one int8 per code into the workspace (4-bit codes stay in [-7, 7]).
+    const int qmax = bits == 4 ? 7 : 127;
+    if (launch_transform_quantize(x, xt, M, W->K, ldx, W->mult_g, block_norm(W->block), W->block, qmax, clip_ratio,
+                                  StoreFmt::Int8, ws.a8, ws.delta, s) != cudaSuccess)
+        return FQ_ERR_CUDA;
+    GemmOut out;
+    out.y = y; out.yt = yt; out.ldy = ldy; out.a_delta = ws.delta;
+    // 4-bit weights are expanded to 16*code on chip: accumulator = 16 * integer sum.
+    return launch_gemm_tcgen05(ws.a8, M, *W, bits == 4 ? 4 : 0, out, s);
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* fq_status_string(fq_status s) {
+    switch (s) {
+        case FQ_OK: return "ok";
+        case FQ_ERR_INVALID_ARG: return "invalid argument";
+        case FQ_ERR_UNSUPPORTED: return "unsupported size or configuration";
+        case FQ_ERR_ALIGNMENT: return "misaligned pointer or leading dimension";
+        case FQ_ERR_ARCH: return "device is not sm_100";
+        case FQ_ERR_CUDA: return "CUDA call failed";
+        case FQ_ERR_NOMEM: return "out of memory or workspace too small";
+        case FQ_ERR_TIMEOUT: return "bounded device wait expired";
+    }
+    return "unknown status";
+}
+
+fq_status fq_fold_weights(const void* Wsrc, fq_dtype wt, int64_t N, int64_t K, int64_t ldw, const float* smooth,
+                          const float* bias, int hadamard_block, int bits, void* stream, fq_weights** out) {
+    if (!out) return FQ_ERR_INVALID_ARG;
+    *out = nullptr;
+    fq_status st = check_shape(N, K, hadamard_block, bits);
+    if (st != FQ_OK) return st;
+    if (wt != FQ_F32 && wt != FQ_BF16) return FQ_ERR_INVALID_ARG;
+    if (K > kMaxPrologueK) return FQ_ERR_UNSUPPORTED;
+    if (N > 0 && (!Wsrc || ldw < K)) return FQ_ERR_INVALID_ARG;
+    if (N > 0 && (!aligned16(Wsrc) || ldw % 8 != 0)) return FQ_ERR_ALIGNMENT;
+    if ((smooth && !aligned16(smooth)) || (bias && !aligned16(bias))) return FQ_ERR_ALIGNMENT;
+    st = check_arch();
+    if (st != FQ_OK) return st;
+    Weights* w = nullptr;
+    st = alloc_handle(N, K, hadamard_block, bits, &w);
+    if (st != FQ_OK) return st;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    float* mult_w = nullptr;   // s_c * block^-1/2, only needed while folding
+    if (cudaMalloc(&mult_w, sizeof(float) * (size_t)K) != cudaSuccess) {
+        fq_weights_destroy(reinterpret_cast<fq_weights*>(w));
+        return FQ_ERR_NOMEM;
+    }
+    const float cn = block_norm(hadamard_block);
+    bool ok = launch_multipliers(smooth, K, cn, mult_w, w->mult_g, s) == cudaSuccess;
+    ok = ok && launch_transform_quantize(Wsrc, wt, N, K, ldw, mult_w, cn, hadamard_block, bits == 4 ? 7 : 127, 1.0f,
+                                         bits == 4 ? StoreFmt::Nibble : StoreFmt::Int8, w->codes, w->w_scale,
+                                         s) == cudaSuccess;
+    if (N > 0) {
+        if (bias)
+            ok = ok && cudaMemcpyAsync(w->bias, bias, sizeof(float) * (size_t)N, cudaMemcpyDeviceToDevice, s) == cudaSuccess;
+        else
+            ok = ok && cudaMemsetAsync(w->bias, 0, sizeof(float) * (size_t)N, s) == cudaSuccess;
+    }
+    ok = ok && cudaStreamSynchronize(s) == cudaSuccess;   // mult_w is freed below; folding is offline
+    cudaFree(mult_w);
+    if (ok) ok = build_weight_tmap(*w) == FQ_OK;
+    if (!ok) {
+        fq_weights_destroy(reinterpret_cast<fq_weights*>(w));
+        return FQ_ERR_CUDA;
+    }
+    *out = reinterpret_cast<fq_weights*>(w);
+    return FQ_OK;
+}
+
+fq_status fq_weights_destroy(fq_weights* wp) {
+    Weights* w = reinterpret_cast<Weights*>(wp);
+    if (!w) return FQ_OK;
+    cudaFree(w->codes); cudaFree(w->w_scale); cudaFree(w->bias); cudaFree(w->mult_g);
+    delete w;
+    return FQ_OK;
+}
+
+fq_status fq_weights_info(const fq_weights* wp, int64_t* N, int64_t* K, int* hadamard_block, int* bits) {
+    const Weights* w = reinterpret_cast<const Weights*>(wp);
+    if (!w) return FQ_ERR_INVALID_ARG;
+    if (N) *N = w->N;
+    if (K) *K = w->K;
+    if (hadamard_block) *hadamard_block = w->block;
+    if (bits) *bits = w->bits;
+    return FQ_OK;
+}
+
+const float* fq_weights_multiplier(const fq_weights* wp) {
+    const Weights* w = reinterpret_cast<const Weights*>(wp);
+    return w ? w->mult_g : nullptr;
+}
+
+fq_status fq_weights_export(const fq_weights* wp, void* codes, float* w_scale, float* mult_g, float* bias,
+                            void* stream) {
+    const Weights* w = reinterpret_cast<const Weights*>(wp);
+    if (!w) return FQ_ERR_INVALID_ARG;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t code_bytes = (size_t)w->N * (size_t)w->K * w->bits / 8;
+    bool ok = true;
+    if (codes && code_bytes) ok = ok && cudaMemcpyAsync(codes, w->codes, code_bytes, cudaMemcpyDeviceToDevice, s) == cudaSuccess;
+    if (w_scale && w->N) ok = ok && cudaMemcpyAsync(w_scale, w->w_scale, sizeof(float) * (size_t)w->N, cudaMemcpyDeviceToDevice, s) == cudaSuccess;
+    if (bias && w->N) ok = ok && cudaMemcpyAsync(bias, w->bias, sizeof(float) * (size_t)w->N, cudaMemcpyDeviceToDevice, s) == cudaSuccess;
+    if (mult_g) ok = ok && cudaMemcpyAsync(mult_g, w->mult_g, sizeof(float) * (size_t)w->K, cudaMemcpyDeviceToDevice, s) == cudaSuccess;
+    return ok ? FQ_OK : FQ_ERR_CUDA;
+}
+
+fq_status fq_weights_import(const void* codes, const float* w_scale, const float* mult_g, const float* bias,
+                            int64_t N, int64_t K, int hadamard_block, int bits, void* stream, fq_weights** out) {
+    if (!out) return FQ_ERR_INVALID_ARG;
+    *out = nullptr;
+    fq_status st = check_shape(N, K, hadamard_block, bits);
+    if (st != FQ_OK) return st;
+    if (N > 0 && (!codes || !w_scale)) return FQ_ERR_INVALID_ARG;
+    st = check_arch();
+    if (st != FQ_OK) return st;
+    Weights* w = nullptr;
+    st = alloc_handle(N, K, hadamard_block, bits, &w);
+    if (st != FQ_OK) return st;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t code_bytes = (size_t)N * (size_t)K * bits / 8;
+    bool ok = true;
+    if (N > 0) {
+        ok = ok && cudaMemcpyAsync(w->codes, codes, code_bytes, cudaMemcpyDeviceToDevice, s) == cudaSuccess;
+        ok = ok && cudaMemcpyAsync(w->w_scale, w_scale, sizeof(float) * (size_t)N, cudaMemcpyDeviceToDevice, s) == cudaSuccess;
+        if (bias)
+            ok = ok && cudaMemcpyAsync(w->bias, bias, sizeof(float) * (size_t)N, cudaMemcpyDeviceToDevice, s) == cudaSuccess;
+        else
+            ok = ok && cudaMemsetAsync(w->bias, 0, sizeof(float) * (size_t)N, s) == cudaSuccess;
+    }
+    if (mult_g)
+        ok = ok && cudaMemcpyAsync(w->mult_g, mult_g, sizeof(float) * (size_t)K, cudaMemcpyDeviceToDevice, s) == cudaSuccess;
+    else
+        ok = ok && launch_multipliers(nullptr, K, block_norm(hadamard_block), nullptr, w->mult_g, s) == cudaSuccess;
+    if (ok) ok = build_weight_tmap(*w) == FQ_OK;
+    if (!ok) {
+        fq_weights_destroy(reinterpret_cast<fq_weights*>(w));
+        return FQ_ERR_CUDA;
+    }
+    *out = reinterpret_cast<fq_weights*>(w);
+    return FQ_OK;
+}
+
+fq_status fq_col_absmax(const void* x, fq_dtype xt, int64_t M, int64_t K, int64_t ldx, int accumulate, float* out,
+                        void* stream) {
+    if (M < 0 || K <= 0 || !out || (M > 0 && (!x || ldx < K))) return FQ_ERR_INVALID_ARG;
+    if (xt != FQ_F32 && xt != FQ_BF16) return FQ_ERR_INVALID_ARG;
+    return launch_col_absmax(x, xt, M, K, ldx, accumulate, out, static_cast<cudaStream_t>(stream)) == cudaSuccess
+               ? FQ_OK : FQ_ERR_CUDA;
+}
+
+fq_status fq_smooth_scale(const float* a, const float* w, int64_t K, double alpha, float* s, void* stream) {
+    if (!a || !w || !s || K <= 0 || !(alpha >= 0.0 && alpha <= 1.0)) return FQ_ERR_INVALID_ARG;
+    return launch_smooth_scale(a, w, K, alpha, s, static_cast<cudaStream_t>(stream)) == cudaSuccess ? FQ_OK
+                                                                                                     : FQ_ERR_CUDA;
+}
+
+fq_status fq_quantize_act(const void* x, fq_dtype xt, int64_t M, int64_t K, int64_t ldx, const float* mult_g,
+                          int hadamard_block, int bits, float clip_ratio, void* codes_out, float* delta_out,
+                          void* stream) {
+    if (M < 0 || K <= 0) return FQ_ERR_INVALID_ARG;
+    if (bits != 4 && bits != 8) return FQ_ERR_INVALID_ARG;
+    if (!(clip_ratio > 0.0f && clip_ratio <= 1.0f)) return FQ_ERR_INVALID_ARG;
+    if (xt != FQ_F32 && xt != FQ_BF16) return FQ_ERR_INVALID_ARG;
+    if (!valid_block(hadamard_block, K) || K % 32 != 0 || K > kMaxPrologueK) return FQ_ERR_UNSUPPORTED;
+    if (M == 0) return FQ_OK;
+    if (!x || !codes_out || !delta_out || ldx < K) return FQ_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(codes_out) || ldx % 8 != 0 || (mult_g && !aligned16(mult_g)))
+        return FQ_ERR_ALIGNMENT;
+    fq_status st = check_arch();
+    if (st != FQ_OK) return st;
+    cudaError_t e = launch_transform_quantize(x, xt, M, K, ldx, mult_g, block_norm(hadamard_block), hadamard_block,
+                                              bits == 4 ? 7 : 127, clip_ratio,
+                                              bits == 4 ? StoreFmt::Nibble : StoreFmt::Int8, codes_out, delta_out,
+                                              static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? FQ_OK : FQ_ERR_CUDA;
+}
+
+fq_status fq_gemm_w4a4(const void* a_codes, const float* a_delta, int64_t M, const fq_weights* W, void* y,
+                       fq_dtype yt, int64_t ldy, void* workspace, size_t ws_bytes, void* stream) {
+    if (!W) return FQ_ERR_INVALID_ARG;
+    if (M > 0 && reinterpret_cast<const Weights*>(W)->N > 0) {
+        fq_status st = check_y(y, yt, ldy, reinterpret_cast<const Weights*>(W)->N);
+        if (st != FQ_OK) return st;
+    }
+    GemmOut out;
+    out.y = y; out.yt = yt; out.ldy = ldy; out.a_delta = a_delta;
+    return gemm_from_codes(a_codes, a_delta, M, W, 4, out, workspace, ws_bytes, static_cast<cudaStream_t>(stream), false);
+}
+
+fq_status fq_gemm_w8a8(const void* a_codes, const float* a_delta, int64_t M, const fq_weights* W, void* y,
+                       fq_dtype yt, int64_t ldy, void* workspace, size_t ws_bytes, void* stream) {
+    if (!W) return FQ_ERR_INVALID_ARG;
+    if (M > 0 && reinterpret_cast<const Weights*>(W)->N > 0) {
+        fq_status st = check_y(y, yt, ldy, reinterpret_cast<const Weights*>(W)->N);
+        if (st != FQ_OK) return st;
+    }
+    GemmOut out;
+    out.y = y; out.yt = yt; out.ldy = ldy; out.a_delta = a_delta;
+    return gemm_from_codes(a_codes, a_delta, M, W, 8, out, workspace, ws_bytes, static_cast<cudaStream_t>(stream), false);
+}
+
+fq_status fq_linear_w4a4(const void* x, fq_dtype xt, int64_t M, int64_t ldx, const fq_weights* W, float clip_ratio,
+                         void* y, fq_dtype yt, int64_t ldy, void* workspace, size_t ws_bytes, void* stream) {
+    return linear_impl(x, xt, M, ldx, W, 4, clip_ratio, y, yt, ldy, workspace, ws_bytes, stream);
+}
+
+fq_status fq_linear_w8a8(const void* x, fq_dtype xt, int64_t M, int64_t ldx, const fq_weights* W, float clip_ratio,
+                         void* y, fq_dtype yt, int64_t ldy, void* workspace, size_t ws_bytes, void* stream) {
+    return linear_impl(x, xt, M, ldx, W, 8, clip_ratio, y, yt, ldy, workspace, ws_bytes, stream);
+}
+
+size_t fq_workspace_bytes(int64_t M, int64_t K, int64_t N, int bits) {
+    (void)N; (void)bits;
+    if (M <= 0 || K <= 0) return 256;
+    return ws_bytes_needed(M, K);
+}
+
+fq_status fq_gemm_acc_i32(const void* a_codes, int64_t M, const fq_weights* W, int32_t* acc, void* workspace,
+                          size_t ws_bytes, void* stream) {
+    if (!W) return FQ_ERR_INVALID_ARG;
+    const Weights* w = reinterpret_cast<const Weights*>(W);
+    if (M > 0 && w->N > 0 && !acc) return FQ_ERR_INVALID_ARG;
+    GemmOut out;
+    out.acc = acc;
+    return gemm_from_codes(a_codes, nullptr, M, W, w->bits, out, workspace, ws_bytes, static_cast<cudaStream_t>(stream), false);
+}
+
+fq_status fq_gemm_simt(const void* a_codes, const float* a_delta, int64_t M, const fq_weights* W, void* y,
+                       fq_dtype yt, int64_t ldy, int32_t* acc, void* workspace, size_t ws_bytes, void* stream) {
+    if (!W) return FQ_ERR_INVALID_ARG;
+    const Weights* w = reinterpret_cast<const Weights*>(W);
+    GemmOut out;
+    if (acc) {
+        out.acc = acc;
+    } else {
+        if (M > 0 && w->N > 0) {
+            fq_status st = check_y(y, yt, ldy, w->N);
+            if (st != FQ_OK) return st;
+        }
+        out.y = y; out.yt = yt; out.ldy = ldy; out.a_delta = a_delta;
+    }
+    return gemm_from_codes(a_codes, a_delta, M, W, w->bits, out, workspace, ws_bytes, static_cast<cudaStream_t>(stream), true);
+}
+
+fq_status fq_device_status(uint32_t* detail) {
+    uint32_t word = 0;
+    if (read_and_clear_watchdog(&word) != cudaSuccess) return FQ_ERR_CUDA;
+    if (detail) *detail = word;
+    return word ? FQ_ERR_TIMEOUT : FQ_OK;
+}
+
+}  // extern "C"

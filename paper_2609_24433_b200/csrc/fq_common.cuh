@@ -1,0 +1,76 @@
+// Internal declarations shared by the translation units of the library
+// (never installed; the public boundary is include/fq.h).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda.h>
+#include <stdint.h>
+
+#include "fq.h"
+
+namespace fq {
+
+// Folded-weight pack of one projection (Alg. 1, offline half: packed codes,
+// output-channel scales, bias) plus the constants the runtime prologue needs.
+struct Weights {
+    int64_t N = 0, K = 0;
+    int block = 0, bits = 0;
+    int device = 0;
+    uint8_t* codes = nullptr;   // [N, K*bits/8], canonical packing
+    float* w_scale = nullptr;   // [N]
+    float* bias = nullptr;      // [N]
+    float* mult_g = nullptr;    // [K] runtime multiplier (1/s_c) * block^-1/2
+    CUtensorMap tmap;           // TMA view of `codes` for the GEMM's weight operand
+    bool tmap_valid = false;
+};
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// ---- launchers (host side, defined next to their kernels) -------------------
+enum class StoreFmt : int { Nibble = 0, Int8 = 1 };
+
+// Runtime prologue / offline fold share one kernel: multiply by mult[K] (or the
+// constant `cnorm` if mult == nullptr), block FWHT, per-row absmax, quantize to
+// +-qmax, store codes in `fmt`, store per-row step to delta.
+cudaError_t launch_transform_quantize(const void* x, fq_dtype xt, int64_t rows, int64_t K, int64_t ldx,
+                                      const float* mult, float cnorm, int block, int qmax,
+                                      float clip_ratio, StoreFmt fmt, void* codes, float* delta,
+                                      cudaStream_t stream);
+
+// mult_w[c] = s_c * cnorm, mult_g[c] = (1/s_c) * cnorm (smooth == nullptr: both = cnorm).
+cudaError_t launch_multipliers(const float* smooth, int64_t K, float cnorm, float* mult_w, float* mult_g,
+                               cudaStream_t stream);
+
+cudaError_t launch_col_absmax(const void* x, fq_dtype xt, int64_t M, int64_t K, int64_t ldx, int accumulate,
+                              float* out, cudaStream_t stream);
+cudaError_t launch_smooth_scale(const float* a, const float* w, int64_t K, double alpha, float* s,
+                                cudaStream_t stream);
+
+// packed nibbles [rows, K/2] -> int8 [rows, K] holding 16*code (natural channel order).
+cudaError_t launch_expand_nibbles(const void* packed, int64_t rows, int64_t K, void* out, cudaStream_t stream);
+
+// Epilogue selector of the GEMM kernels.
+struct GemmOut {
+    void* y = nullptr;          // [M, N] of yt, leading dimension ldy   (nullptr when acc is used)
+    fq_dtype yt = FQ_F32;
+    int64_t ldy = 0;
+    int32_t* acc = nullptr;     // raw accumulators [M, N] (debug/parity)
+    const float* a_delta = nullptr;
+};
+
+// Reference-grade CUDA-core integer GEMM (dp4a); a8 = int8 activations [M, K].
+cudaError_t launch_gemm_simt(const int8_t* a8, int64_t M, const Weights& W, int acc_shift, const GemmOut& out,
+                             cudaStream_t stream);
+
+// tcgen05 integer GEMM; a8 = int8 activations [M, K] (pitch K), 16-byte aligned.
+fq_status launch_gemm_tcgen05(const int8_t* a8, int64_t M, const Weights& W, int acc_shift, const GemmOut& out,
+                              cudaStream_t stream);
+
+// Builds the weight-operand tensor map of a handle (after `codes` is allocated).
+fq_status build_weight_tmap(Weights& W);
+
+// Device watchdog word (see fq_device_status).
+cudaError_t read_and_clear_watchdog(uint32_t* word);
+uint32_t* watchdog_device_ptr();
+
+}  // namespace fq

@@ -1,0 +1,516 @@
+// Integer GEMM of Eq. 8 on the 5th-generation tensor cores (sm_100a):
+//   acc[j][t] = sum_c qW[j][c] * qA[t][c]   tcgen05.mma kind::i8, int32 accumulators in TMEM
+//   y[t][j]   = delta_t * s^W_j * acc + b_j fused epilogue straight out of TMEM
+//
+// Orientation.  The 128 rows of an MMA tile are OUTPUT CHANNELS (weight rows),
+// the MMA's N dimension (16..256, any multiple of 16) is a tile of TOKENS.  A
+// TMEM lane therefore owns one output channel: its scale and bias are per-thread
+// scalars in the epilogue, a warp stores 32 consecutive channels of one token
+// (coalesced), and ragged token counts (M = 50, 816, ...) are absorbed by the
+// free N dimension instead of padding a fixed 128-row tile.
+//
+// Operands.  Both are K-major with 128-byte rows in the 128B-swizzled shared
+// memory layout.  Activations arrive as int8 by TMA.  8-bit weights arrive the
+// same way.  4-bit weights stay packed in HBM and in the TMA stage; four unpack
+// warps expand each 128 x 64-byte packed tile into a 128 x 128-byte int8 tile
+// holding 16*code (nibble moved to the high half of the byte: no sign extension
+// needed), so the accumulator is an exact multiple of 2^acc_shift that the
+// epilogue shifts away.
+//
+// Roles (warp specialised, persistent over tiles):
+//   warp 0     TMA producer          warp 1  MMA issuer + TMEM allocator
+//   warps 2-5  epilogue (one TMEM lane quadrant each)
+//   warps 6-9  nibble unpack (4-bit weights only)
+// Every mbarrier wait is bounded by wall-clock time; on expiry the CTA records a
+// code in the watchdog word, stops issuing work, and still frees its TMEM.
+#include <cuda_bf16.h>
+
+#include "fq_common.cuh"
+
+namespace fq {
+
+__device__ uint32_t g_watchdog_word = 0;
+
+uint32_t* watchdog_device_ptr() {
+    uint32_t* p = nullptr;
+    if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_watchdog_word) != cudaSuccess) return nullptr;
+    return p;
+}
+
+cudaError_t read_and_clear_watchdog(uint32_t* word) {
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) return e;
+    e = cudaMemcpyFromSymbol(word, g_watchdog_word, sizeof(uint32_t));
+    if (e != cudaSuccess) return e;
+    const uint32_t zero = 0;
+    return cudaMemcpyToSymbol(g_watchdog_word, &zero, sizeof(uint32_t));
+}
+
+namespace {
+
+constexpr int kTileN = 128;          // output channels per tile (MMA M)
+constexpr int kBlockK = 128;         // int8 elements (= bytes) of K per pipeline stage
+constexpr int kMmaK = 32;            // K per tcgen05.mma.kind::i8
+constexpr int kAccStages = 2;
+constexpr int kMaxStages = 8;
+constexpr uint64_t kWaitLimitNs = 2000000000ull;   // 2 s per wait
+
+struct Params {
+    int64_t M, N, K;
+    int bt;              // tokens per tile (MMA N), multiple of 16, <= 256
+    int stages;
+    int m_tiles, n_tiles;
+    int tmem_cols;
+    int acc_shift;
+    const float* w_scale;
+    const float* bias;
+    GemmOut out;
+    uint32_t* watchdog;
+};
+
+// ---- PTX wrappers ------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.b32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ uint64_t global_timer_ns() {
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
+// Bounded wait.  Returns false if the CTA is aborting or the limit expired
+// (in which case the abort flag and the watchdog word are set).
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                            uint32_t* watchdog, uint32_t code) {
+    const uint64_t t0 = global_timer_ns();
+    for (uint32_t spin = 1;; ++spin) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((spin & 0xff) == 0) {
+            if (*abort_flag) return false;
+            if (global_timer_ns() - t0 > kWaitLimitNs) {
+                *abort_flag = 1;
+                atomicOr(watchdog, code);
+                return false;
+            }
+        }
+    }
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          uint32_t* watchdog, uint32_t code) {
+#pragma unroll 1
+    for (int i = 0; i < 64; ++i)
+        if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait_slow(bar, parity, abort_flag, watchdog, code);
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ void fence_proxy_async_smem() {
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void mma_i8(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                       uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void mma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* r) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor: K-major operand, 128-byte rows, 128B swizzle,
+// 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr & 0x3FFFFu) >> 4);   // start address, 16-byte units
+    d |= (uint64_t)1 << 16;                    // leading byte offset (unused for swizzled K-major)
+    d |= (uint64_t)(1024 >> 4) << 32;          // stride byte offset between 8-row groups
+    d |= (uint64_t)1 << 46;                    // descriptor version of this architecture
+    d |= (uint64_t)2 << 61;                    // 128-byte swizzle
+    return d;
+}
+// Instruction descriptor: s8 x s8 -> s32, both operands K-major, M = 128, N = n.
+__device__ __forceinline__ uint32_t instr_desc_i8(int n) {
+    return (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTileN >> 4) << 24);
+}
+
+enum : uint32_t {
+    kWdProducer = 1u, kWdMmaFull = 2u, kWdMmaAcc = 4u, kWdEpilogue = 8u, kWdUnpackFull = 16u,
+    kWdUnpackEmpty = 32u, kWdDrain = 64u
+};
+
+template <int BITS>
+__global__ void __launch_bounds__(BITS == 4 ? 320 : 192, 1)
+gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_w,
+                    const Params p) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint64_t s_full_tma[kMaxStages];
+    __shared__ uint64_t s_full_w8[kMaxStages];
+    __shared__ uint64_t s_empty[kMaxStages];
+    __shared__ uint64_t s_acc_full[kAccStages];
+    __shared__ uint64_t s_acc_empty[kAccStages];
+    __shared__ uint32_t s_tmem_base;
+    __shared__ int s_abort;
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    volatile int* abort_flag = &s_abort;
+
+    // carve dynamic shared memory: [A8 stages][W8 stages][packed stages], all 1024-byte aligned
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t a_bytes = (uint32_t)p.bt * kBlockK;
+    const uint32_t w_bytes = kTileN * kBlockK;
+    const uint32_t pk_bytes = kTileN * kBlockK / 2;
+    const uint32_t smem_a = base;
+    const uint32_t smem_w = smem_a + (uint32_t)p.stages * a_bytes;
+    const uint32_t smem_p = smem_w + (uint32_t)p.stages * w_bytes;
+    uint8_t* gen_base = smem_raw + (base - smem_u32(smem_raw));   // generic pointer to `base`
+
+    if (threadIdx.x == 0) {
+        s_abort = 0;
+        for (int s = 0; s < p.stages; ++s) {
+            mbar_init(smem_u32(&s_full_tma[s]), 1);
+            mbar_init(smem_u32(&s_full_w8[s]), 4);
+            mbar_init(smem_u32(&s_empty[s]), 1);
+        }
+        for (int a = 0; a < kAccStages; ++a) {
+            mbar_init(smem_u32(&s_acc_full[a]), 1);
+            mbar_init(smem_u32(&s_acc_empty[a]), 4);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        fence_proxy_async_smem();
+    }
+    if (warp == 1) tmem_alloc(smem_u32(&s_tmem_base), (uint32_t)p.tmem_cols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = s_tmem_base;
+
+    const int num_tiles = p.m_tiles * p.n_tiles;
+    const int k_blocks = (int)((p.K + kBlockK - 1) / kBlockK);
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            const uint32_t tx = a_bytes + (BITS == 4 ? pk_bytes : w_bytes);
+            bool ok = true;
+            int issued = 0;
+            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+                const int n0 = (tile / p.m_tiles) * kTileN;
+                const int t0 = (tile % p.m_tiles) * p.bt;
+                for (int kb = 0; kb < k_blocks; ++kb) {
+                    ok = mbar_wait(smem_u32(&s_empty[stage]), phase ^ 1u, abort_flag, p.watchdog, kWdProducer);
+                    if (!ok) break;
+                    const uint32_t bar = smem_u32(&s_full_tma[stage]);
+                    mbar_arrive_expect_tx(bar, tx);
+                    tma_load_2d(smem_a + stage * a_bytes, &map_a, kb * kBlockK, t0, bar);
+                    if (BITS == 4)
+                        tma_load_2d(smem_p + stage * pk_bytes, &map_w, kb * (kBlockK / 2), n0, bar);
+                    else
+                        tma_load_2d(smem_w + stage * w_bytes, &map_w, kb * kBlockK, n0, bar);
+                    ++issued;
+                    if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+                }
+            }
+            if (!ok) {
+                // Winding down after an expired wait: let the copies already issued land
+                // before the CTA gives its shared memory back.
+                int back = issued < p.stages ? issued : p.stages;
+                int s = stage;
+                uint32_t ph = phase;
+                for (int i = 0; i < back; ++i) {
+                    if (--s < 0) { s = p.stages - 1; ph ^= 1u; }
+                    const uint64_t t0 = global_timer_ns();
+                    while (!mbar_try_wait(smem_u32(&s_full_tma[s]), ph)) {
+                        if (global_timer_ns() - t0 > kWaitLimitNs) { atomicOr(p.watchdog, kWdDrain); break; }
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // -------------------------------------------------------------- MMA issuer
+        if (lane == 0) {
+            const uint32_t idesc = instr_desc_i8(p.bt);
+            int stage = 0;
+            uint32_t phase = 0;
+            int acc_stage = 0;
+            uint32_t acc_phase = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+                ok = mbar_wait(smem_u32(&s_acc_empty[acc_stage]), acc_phase ^ 1u, abort_flag, p.watchdog, kWdMmaAcc);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(acc_stage * p.bt);
+                for (int kb = 0; kb < k_blocks; ++kb) {
+                    ok = mbar_wait(smem_u32(&s_full_tma[stage]), phase, abort_flag, p.watchdog, kWdMmaFull);
+                    if (ok && BITS == 4)
+                        ok = mbar_wait(smem_u32(&s_full_w8[stage]), phase, abort_flag, p.watchdog, kWdMmaFull);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint64_t wdesc = smem_desc_sw128(smem_w + stage * w_bytes);
+                    const uint64_t adesc = smem_desc_sw128(smem_a + stage * a_bytes);
+#pragma unroll
+                    for (int k = 0; k < kBlockK / kMmaK; ++k) {
+                        // step 32 bytes along K inside the swizzle atom: +2 in 16-byte address units
+                        mma_i8(d_tmem, wdesc + (uint64_t)(2 * k), adesc + (uint64_t)(2 * k), idesc,
+                               (kb | k) != 0 ? 1u : 0u);
+                    }
+                    mma_commit(smem_u32(&s_empty[stage]));          // frees this stage when the MMAs retire
+                    if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+                }
+                if (!ok) break;
+                mma_commit(smem_u32(&s_acc_full[acc_stage]));        // accumulator complete
+                if (++acc_stage == kAccStages) { acc_stage = 0; acc_phase ^= 1u; }
+            }
+        }
+    } else if (warp < 6) {
+        // ---------------------------------------------------------------- epilogue
+        const int quad = warp & 3;                       // TMEM lanes [32*quad, 32*quad + 32)
+        int acc_stage = 0;
+        uint32_t acc_phase = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+            const int64_t j = (int64_t)(tile / p.m_tiles) * kTileN + quad * 32 + lane;
+            const int64_t t0 = (int64_t)(tile % p.m_tiles) * p.bt;
+            const bool j_ok = j < p.N;
+            float sw = 0.0f, bj = 0.0f;
+            if (j_ok && p.out.acc == nullptr) {
+                sw = __ldg(p.w_scale + j);
+                bj = __ldg(p.bias + j);
+            }
+            ok = mbar_wait(smem_u32(&s_acc_full[acc_stage]), acc_phase, abort_flag, p.watchdog, kWdEpilogue);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc_stage * p.bt);
+            for (int c = 0; c < p.bt; c += 16) {
+                if (t0 + c >= p.M) break;                // tokens beyond M: nothing to store (warp-uniform)
+                uint32_t r[16];
+                tmem_ld16(taddr + (uint32_t)c, r);
+                tmem_ld_wait();
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    const int64_t t = t0 + c + i;
+                    if (t < p.M && j_ok) {
+                        const int acc = ((int)r[i]) >> p.acc_shift;
+                        if (p.out.acc != nullptr) {
+                            p.out.acc[t * p.N + j] = acc;
+                        } else {
+                            const float v = fmaf((float)acc, __ldg(p.out.a_delta + t) * sw, bj);
+                            if (p.out.yt == FQ_F32)
+                                static_cast<float*>(p.out.y)[t * p.out.ldy + j] = v;
+                            else
+                                static_cast<__nv_bfloat16*>(p.out.y)[t * p.out.ldy + j] = __float2bfloat16_rn(v);
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&s_acc_empty[acc_stage]));
+            if (++acc_stage == kAccStages) { acc_stage = 0; acc_phase ^= 1u; }
+        }
+    } else if (BITS == 4) {
+        // ------------------------------------------------------------ nibble unpack
+        const int ut = threadIdx.x - 192;                // 0..127
+        int stage = 0;
+        uint32_t phase = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+            for (int kb = 0; kb < k_blocks; ++kb) {
+                ok = mbar_wait(smem_u32(&s_full_tma[stage]), phase, abort_flag, p.watchdog, kWdUnpackFull);
+                if (ok) ok = mbar_wait(smem_u32(&s_empty[stage]), phase ^ 1u, abort_flag, p.watchdog, kWdUnpackEmpty);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                const uint8_t* src = gen_base + (smem_p - base) + stage * pk_bytes;
+                uint8_t* dst = gen_base + (smem_w - base) + stage * w_bytes;
+#pragma unroll
+                for (int it = 0; it < 4; ++it) {
+                    const int idx = it * 128 + ut;       // 16-byte packed chunk index
+                    const int row = idx >> 2;
+                    const int cp = idx & 3;
+                    const uint4 pk = *reinterpret_cast<const uint4*>(src + idx * 16);
+                    const uint32_t w[4] = {pk.x, pk.y, pk.z, pk.w};
+                    uint32_t o[8];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const uint32_t lo = (w[q] << 4) & 0xF0F0F0F0u;
+                        const uint32_t hi = w[q] & 0xF0F0F0F0u;
+                        o[2 * q + 0] = __byte_perm(lo, hi, 0x5140);
+                        o[2 * q + 1] = __byte_perm(lo, hi, 0x7362);
+                    }
+                    uint8_t* drow = dst + row * 128;
+                    const int sw = row & 7;
+                    *reinterpret_cast<uint4*>(drow + (((2 * cp) ^ sw) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
+                    *reinterpret_cast<uint4*>(drow + (((2 * cp + 1) ^ sw) << 4)) = make_uint4(o[4], o[5], o[6], o[7]);
+                }
+                fence_proxy_async_smem();                // generic-proxy writes -> visible to the tensor core
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&s_full_w8[stage]));
+                if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+            }
+        }
+    }
+
+    // ------------------------------------------------------------------ teardown
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, (uint32_t)p.tmem_cols);
+    }
+}
+
+// ---- host side ---------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* sym = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(sym);
+    }
+    return fn;
+}
+
+// 2-D byte tensor [rows, row_bytes] (row pitch = row_bytes), box [box_rows, box_bytes].
+bool encode_2d(CUtensorMap* map, const void* ptr, uint64_t row_bytes, uint64_t rows, uint32_t box_bytes,
+               uint32_t box_rows, bool swizzle128) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {row_bytes, rows};
+    const cuuint64_t strides[1] = {row_bytes};
+    const cuuint32_t box[2] = {box_bytes, box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int next_pow2(int v) {
+    int r = 32;
+    while (r < v) r <<= 1;
+    return r;
+}
+
+}  // namespace
+
+fq_status build_weight_tmap(Weights& W) {
+    W.tmap_valid = false;
+    if (W.N == 0) return FQ_OK;
+    const bool ok = W.bits == 4
+                        ? encode_2d(&W.tmap, W.codes, (uint64_t)W.K / 2, (uint64_t)W.N, kBlockK / 2, kTileN, false)
+                        : encode_2d(&W.tmap, W.codes, (uint64_t)W.K, (uint64_t)W.N, kBlockK, kTileN, true);
+    if (!ok) return FQ_ERR_CUDA;
+    W.tmap_valid = true;
+    return FQ_OK;
+}
+
+fq_status launch_gemm_tcgen05(const int8_t* a8, int64_t M, const Weights& W, int acc_shift, const GemmOut& out,
+                              cudaStream_t stream) {
+    if (M == 0 || W.N == 0) return FQ_OK;
+    if (!W.tmap_valid) return FQ_ERR_CUDA;
+
+    Params p{};
+    p.M = M; p.N = W.N; p.K = W.K;
+    const int m_tiles = (int)((M + 255) / 256);
+    int bt = (int)(((M + m_tiles - 1) / m_tiles + 15) / 16 * 16);
+    p.bt = bt;
+    p.m_tiles = (int)((M + bt - 1) / bt);
+    p.n_tiles = (int)((W.N + kTileN - 1) / kTileN);
+    p.acc_shift = acc_shift;
+    p.w_scale = W.w_scale;
+    p.bias = W.bias;
+    p.out = out;
+    p.watchdog = watchdog_device_ptr();
+    if (!p.watchdog) return FQ_ERR_CUDA;
+    p.tmem_cols = next_pow2(kAccStages * bt);
+
+    const size_t stage_bytes = (size_t)bt * kBlockK + kTileN * kBlockK + (W.bits == 4 ? kTileN * kBlockK / 2 : 0);
+    const size_t budget = 227 * 1024 - 1024 /*alignment slack*/ - 1024 /*static*/;
+    int stages = (int)(budget / stage_bytes);
+    if (stages > kMaxStages) stages = kMaxStages;
+    if (stages < 2) return FQ_ERR_UNSUPPORTED;
+    p.stages = stages;
+    const size_t smem = stage_bytes * stages + 1024;
+
+    CUtensorMap map_a;
+    if (!encode_2d(&map_a, a8, (uint64_t)W.K, (uint64_t)M, kBlockK, (uint32_t)bt, true)) return FQ_ERR_CUDA;
+
+    int dev = 0, sms = 148;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int num_tiles = p.m_tiles * p.n_tiles;
+    const int grid = num_tiles < sms ? num_tiles : sms;
+
+    cudaError_t e;
+    if (W.bits == 4) {
+        e = cudaFuncSetAttribute(gemm_tcgen05_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return FQ_ERR_CUDA;
+        gemm_tcgen05_kernel<4><<<grid, 320, smem, stream>>>(map_a, W.tmap, p);
+    } else {
+        e = cudaFuncSetAttribute(gemm_tcgen05_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return FQ_ERR_CUDA;
+        gemm_tcgen05_kernel<8><<<grid, 192, smem, stream>>>(map_a, W.tmap, p);
+    }
+    return cudaGetLastError() == cudaSuccess ? FQ_OK : FQ_ERR_CUDA;
+}
+
+}  // namespace fq

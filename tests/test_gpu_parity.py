@@ -1,0 +1,345 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the same
+seeded inputs.  Integer stages (packed codes, per-token steps, folded weight codes and scales,
+int32 accumulators) must match bit for bit; floating-point outputs within 1e-3 (fp32) or
+1e-2 (bf16) relative."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from helpers import assert_close, concat_consumers, oracle_smooth, to_dev, to_np
+from paper_2609_24433_b200 import fq, synth
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(autouse=True)
+def _watchdog_clean():
+    yield
+    st, word = fq.device_status()
+    assert st == fq.OK, f"device wait watchdog fired: {word:#x}"
+
+
+def make_x(M, K, dtype, seed, frac=0.01):
+    site = synth.Site("t", M, K, [("p", 8)], beta=32, bits=4, x_dtype=dtype, outlier_frac=frac)
+    return synth.make_site(site, seed, with_weights=False).x
+
+
+# ----------------------------------------------------------------- prologue ----
+ACT_CASES = [
+    # M, K, block, bits, dtype, smooth, clip
+    (64, 1024, 128, 4, "f32", True, 1.0),
+    (50, 1024, 64, 4, "bf16", False, 1.0),
+    (50, 4096, 64, 4, "bf16", False, 1.0),
+    (816, 2048, 128, 4, "bf16", True, 1.0),
+    (816, 2048, 128, 8, "bf16", False, 1.0),
+    (203, 16384, 256, 8, "bf16", False, 1.0),
+    (131, 16384, 256, 4, "f32", True, 0.8),
+    (5, 32, 32, 4, "f32", False, 1.0),
+    (3, 64, 2, 8, "bf16", False, 1.0),
+    (9, 96, 32, 4, "bf16", True, 1.0),
+    (33, 256, 4, 4, "f32", False, 1.0),
+    (33, 512, 8, 8, "bf16", False, 0.5),
+    (17, 3072, 16, 4, "bf16", False, 1.0),
+    (7, 3072, 128, 8, "f32", True, 0.9),
+    (300, 8192, 32, 4, "bf16", False, 1.0),
+    (19, 8192, 256, 8, "f32", False, 1.0),
+    (4, 32768, 256, 4, "bf16", True, 1.0),
+    (3, 32768, 64, 8, "f32", False, 0.75),
+    (1, 2048, 128, 4, "bf16", False, 1.0),
+    (2500, 1024, 64, 4, "bf16", False, 1.0),
+]
+
+
+@pytest.mark.parametrize("M,K,block,bits,dtype,smooth,clip", ACT_CASES)
+def test_quantize_act_bit_exact(M, K, block, bits, dtype, smooth, clip):
+    x = make_x(M, K, dtype, seed=M + K + block)
+    rng = np.random.default_rng(K)
+    s = np.exp(rng.uniform(-2, 2, K)).astype(np.float32) if smooth else None
+    g = oracle.multiplier(s, K, block, False) if smooth else None
+    want_codes, want_delta = oracle.quantize_act(x, dtype, g, block, bits, clip)
+    codes, delta = fq.quantize_act(to_dev(x, dtype), to_dev(g), block, bits, clip)
+    assert np.array_equal(to_np(delta).view(np.uint32), want_delta.view(np.uint32))
+    assert np.array_equal(to_np(codes), want_codes)
+
+
+@pytest.mark.parametrize("bits", [4, 8])
+def test_quantize_act_zero_tiny_and_strided_rows(bits):
+    M, K, block = 37, 1024, 128
+    x = make_x(M, K, "f32", seed=1).copy()
+    x[3] = 0.0
+    x[11] = np.float32(1e-42)
+    x[20] = np.float32(-3e-39)
+    want_codes, want_delta = oracle.quantize_act(x, "f32", None, block, bits)
+    assert want_delta[3] == 0 and want_delta[11] == 0
+    wide = torch.full((M, K + 64), 7.0, dtype=torch.float32, device="cuda")   # leading dimension > K
+    wide[:, :K] = to_dev(x)
+    codes = torch.full((M + 1, K * bits // 8), 0xAB, dtype=torch.uint8, device="cuda")
+    delta = torch.full((M + 1,), -1.0, dtype=torch.float32, device="cuda")
+    fq.quantize_act(wide[:, :K], None, block, bits, 1.0, codes=codes[:M], delta=delta[:M])
+    assert np.array_equal(to_np(codes[:M]), want_codes)
+    assert np.array_equal(to_np(delta[:M]).view(np.uint32), want_delta.view(np.uint32))
+    assert (codes[M] == 0xAB).all() and delta[M] == -1.0      # nothing written past row M
+
+
+def test_quantize_act_amplitude_invariance_on_device():
+    x = make_x(64, 2048, "f32", seed=4)
+    c0, d0 = fq.quantize_act(to_dev(x), None, 64, 4)
+    for k in (-7, 5):
+        c1, d1 = fq.quantize_act(to_dev(x * np.float32(2.0 ** k)), None, 64, 4)
+        assert torch.equal(c0, c1) and torch.equal(d1, d0 * (2.0 ** k))
+
+
+def test_quantize_act_empty_batch():
+    x = torch.empty((0, 1024), dtype=torch.bfloat16, device="cuda")
+    codes, delta = fq.quantize_act(x, None, 128, 4)
+    assert codes.shape == (0, 512) and delta.shape == (0,)
+
+
+# --------------------------------------------------------------------- fold ----
+FOLD_CASES = [
+    # N, K, block, bits, wdtype, smooth
+    (1024, 1024, 128, 4, "f32", True),
+    (256, 2048, 128, 8, "f32", False),
+    (264, 4096, 64, 4, "bf16", True),
+    (8, 32, 32, 4, "f32", False),
+    (24, 16384, 256, 8, "bf16", False),
+    (16, 16384, 256, 4, "f32", True),
+    (40, 96, 32, 8, "f32", True),
+]
+
+
+@pytest.mark.parametrize("N,K,block,bits,wdtype,smooth", FOLD_CASES)
+def test_fold_weights_bit_exact(N, K, block, bits, wdtype, smooth):
+    rng = np.random.default_rng(N + K)
+    W = synth.as_dtype(synth.draw_weights(rng, N, K), wdtype)
+    if N > 2:
+        W[2] = 0                                                   # zero output channel
+    bias = rng.standard_normal(N).astype(np.float32)
+    s = np.exp(rng.uniform(-2, 2, K)).astype(np.float32) if smooth else None
+    want_codes, want_scale, want_g = oracle.fold_weights(W, wdtype, s, block, bits)
+    h = fq.fold_weights(to_dev(W, wdtype), to_dev(s), to_dev(bias), block, bits)
+    assert (h.N, h.K, h.block, h.bits) == (N, K, block, bits)
+    codes, scale, g, b = h.export()
+    assert np.array_equal(to_np(g).view(np.uint32), want_g.view(np.uint32))
+    assert np.array_equal(to_np(scale).view(np.uint32), want_scale.view(np.uint32))
+    assert np.array_equal(to_np(codes), want_codes)
+    assert np.array_equal(to_np(b), bias)
+    # import of the exported pack behaves like the original handle
+    h2 = fq.weights_import(codes, scale, g, b, K, block, bits)
+    c2, s2, g2, b2 = h2.export()
+    assert torch.equal(c2, codes) and torch.equal(s2, scale) and torch.equal(g2, g) and torch.equal(b2, b)
+
+
+# ------------------------------------------------------------ integer GEMM ----
+def random_codes(rng, rows, K, bits):
+    q = 7 if bits == 4 else 127
+    return oracle.pack(rng.integers(-q, q + 1, size=(rows, K)).astype(np.int32), bits)
+
+
+def import_codes(wc, K, bits, block=32, scale=None, bias=None):
+    N = wc.shape[0]
+    scale = np.ones(N, np.float32) if scale is None else scale
+    return fq.weights_import(to_dev(wc), to_dev(scale), None, to_dev(bias), K, block, bits)
+
+
+GEMM_CASES = [
+    # M, N, K, bits
+    (64, 1024, 1024, 4),
+    (50, 3072, 1024, 4),
+    (50, 1024, 4096, 4),
+    (1, 256, 2048, 4),
+    (16, 8, 32, 4),
+    (17, 24, 96, 8),
+    (130, 136, 160, 4),
+    (300, 264, 2048, 8),
+    (816, 512, 2048, 4),
+    (816, 256, 2048, 8),
+    (257, 384, 16384, 8),
+    (520, 128, 8192, 4),
+]
+
+
+@pytest.mark.parametrize("M,N,K,bits", GEMM_CASES)
+@pytest.mark.parametrize("kernel", ["tcgen05", "simt"])
+def test_int32_accumulators_bit_exact(M, N, K, bits, kernel):
+    rng = np.random.default_rng(M * 7 + N * 3 + K + bits)
+    a = random_codes(rng, M, K, bits)
+    w = random_codes(rng, N, K, bits)
+    want = oracle.gemm_i32(a, w, K, bits)
+    h = import_codes(w, K, bits)
+    if kernel == "tcgen05":
+        got = fq.gemm_acc_i32(to_dev(a), h)
+    else:
+        got = fq.gemm_simt(to_dev(a), None, h, raw_acc=True)
+    assert np.array_equal(to_np(got), want)
+
+
+@pytest.mark.parametrize("bits", [4, 8])
+def test_accumulator_extremes_and_one_hot(bits):
+    q = 7 if bits == 4 else 127
+    K, M, N = 16384, 40, 136
+    a = oracle.pack(np.full((M, K), q, np.int32), bits)
+    w = oracle.pack(np.full((N, K), -q, np.int32), bits)
+    got = fq.gemm_acc_i32(to_dev(a), import_codes(w, K, bits))
+    assert (got == -q * q * K).all()
+    # one-hot activations pick single weight codes: catches any K permutation or operand swap
+    K = 256
+    rng = np.random.default_rng(0)
+    wi = rng.integers(-q, q + 1, size=(N, K)).astype(np.int32)
+    eye = np.eye(K, dtype=np.int32)
+    got = fq.gemm_acc_i32(to_dev(oracle.pack(eye, bits)), import_codes(oracle.pack(wi, bits), K, bits))
+    assert np.array_equal(to_np(got), wi.T)
+
+
+def test_gemm_is_deterministic_run_to_run():
+    rng = np.random.default_rng(5)
+    a, w = random_codes(rng, 333, 2048, 4), random_codes(rng, 520, 2048, 4)
+    h = import_codes(w, 2048, 4)
+    first = fq.gemm_acc_i32(to_dev(a), h)
+    for _ in range(3):
+        assert torch.equal(fq.gemm_acc_i32(to_dev(a), h), first)
+
+
+# ------------------------------------------------------- whole runtime path ----
+def run_site(data: synth.SiteData, rows=None, clip=1.0):
+    """Fold + run one site on the GPU and in the oracle; returns dicts of results."""
+    site = data.site
+    s = oracle_smooth(data)
+    W, b = concat_consumers(data)
+    wc, ws, g = oracle.fold_weights(W, "f32", s, site.beta, site.bits)
+    y_ref, codes_ref, delta_ref, acc_ref = oracle.linear(data.x, site.x_dtype, g, site.beta, site.bits, clip, wc, ws,
+                                                         b, site.y_dtype, rows=rows)
+    h = fq.fold_weights(to_dev(W), to_dev(s), to_dev(b), site.beta, site.bits)
+    ydt = torch.float32 if site.y_dtype == "f32" else torch.bfloat16
+    x_dev = to_dev(data.x, site.x_dtype)
+    y = fq.linear(x_dev, h, clip, ydt)
+    codes, delta = fq.quantize_act(x_dev, h, site.beta, site.bits, clip)
+    return dict(h=h, y=y, codes=codes, delta=delta, x=x_dev), dict(y=y_ref, codes=codes_ref, delta=delta_ref,
+                                                                  acc=acc_ref, wc=wc, ws=ws, g=g)
+
+
+def test_config1_single_w4a4_linear_full_parity():
+    data = synth.make_site(synth.config1_site(), seed=0, calib_tokens=512)
+    gpu, ref = run_site(data)
+    assert np.array_equal(to_np(gpu["codes"]), ref["codes"])
+    assert np.array_equal(to_np(gpu["delta"]).view(np.uint32), ref["delta"].view(np.uint32))
+    hc, hs, hg, _ = gpu["h"].export()
+    assert np.array_equal(to_np(hc), ref["wc"]) and np.array_equal(to_np(hs), ref["ws"])
+    acc = fq.gemm_acc_i32(gpu["codes"], gpu["h"])
+    assert np.array_equal(to_np(acc), ref["acc"])
+    assert_close(to_np(gpu["y"]), ref["y"], "f32", "config 1 fused")
+    y2 = fq.gemm_w4a4(gpu["codes"], gpu["delta"], gpu["h"], torch.float32)
+    assert_close(to_np(y2), ref["y"], "f32", "config 1 two-call")
+    # and the layer does what it is for: close to the unquantised projection
+    want = data.x.astype(np.float64) @ data.W["proj"].astype(np.float64).T + data.bias["proj"]
+    assert np.linalg.norm(to_np(gpu["y"]) - want) / np.linalg.norm(want) < 0.35
+
+
+@pytest.mark.parametrize("site_idx", [0, 1, 3])
+@pytest.mark.parametrize("selective", [True, False])
+def test_backbone_layer_sites_small_n(site_idx, selective):
+    """Backbone-layer shapes (M = 816, K = 2048 / 16384) with N cut to 512 so the oracle runs in full."""
+    site = synth.backbone_layer_sites(selective)[site_idx]
+    site.consumers = [(n, min(k, 256)) for n, k in site.consumers][:2]
+    data = synth.make_site(site, seed=2 + site_idx)
+    gpu, ref = run_site(data)
+    assert np.array_equal(to_np(gpu["codes"]), ref["codes"])
+    assert np.array_equal(to_np(gpu["delta"]).view(np.uint32), ref["delta"].view(np.uint32))
+    assert np.array_equal(to_np(fq.gemm_acc_i32(gpu["codes"], gpu["h"])), ref["acc"])
+    assert_close(to_np(gpu["y"]), ref["y"], site.y_dtype, site.name)
+
+
+def test_shared_site_consumers_see_the_same_codes():
+    """q/k/v run as one concatenated GEMM equal three separate consumer calls bit for bit."""
+    site = synth.backbone_layer_sites()[0]
+    site.M = 200
+    data = synth.make_site(site, seed=11)
+    s = oracle_smooth(data)
+    W, b = concat_consumers(data)
+    x = to_dev(data.x, "bf16")
+    h_all = fq.fold_weights(to_dev(W), to_dev(s), to_dev(b), site.beta, 4)
+    codes, delta = fq.quantize_act(x, h_all, site.beta, 4)
+    y_all = fq.gemm_w4a4(codes, delta, h_all, torch.bfloat16)
+    col = 0
+    for name, n in site.consumers:
+        h = fq.fold_weights(to_dev(data.W[name]), to_dev(s), to_dev(data.bias[name]), site.beta, 4)
+        y = fq.gemm_w4a4(codes, delta, h, torch.bfloat16)
+        assert torch.equal(y, y_all[:, col:col + n]), name
+        col += n
+
+
+@pytest.mark.parametrize("bits", [4, 8])
+def test_zero_token_gives_bias_and_rows_beyond_m_are_untouched(bits):
+    M, K, N = 70, 1024, 264
+    rng = np.random.default_rng(3)
+    x = make_x(M, K, "bf16", seed=8).copy()
+    x[5] = 0
+    W = synth.draw_weights(rng, N, K)
+    bias = rng.standard_normal(N).astype(np.float32)
+    h = fq.fold_weights(to_dev(W), None, to_dev(bias), 128, bits)
+    y = torch.full((M + 2, N + 8), 123.0, dtype=torch.float32, device="cuda")
+    fq.linear(to_dev(x, "bf16"), h, 1.0, y=y[:M, :N])
+    assert np.array_equal(to_np(y[5, :N]), bias)
+    assert (y[M:] == 123.0).all() and (y[:, N:] == 123.0).all()
+    wc, ws, g = oracle.fold_weights(W, "f32", None, 128, bits)
+    ref = oracle.linear(x, "bf16", g, 128, bits, 1.0, wc, ws, bias, "f32")[0]
+    assert_close(to_np(y[:M, :N]), ref, "f32", "strided output")
+
+
+def test_expert_layer_sites_and_amplitude_drift():
+    """Action-expert shapes (M = 50, block 64, W4A4) at two denoising amplitudes."""
+    for sigma in (1.0, 0.1):
+        for site in synth.expert_layer_sites(sigma=sigma):
+            data = synth.make_site(site, seed=3)
+            gpu, ref = run_site(data)
+            assert np.array_equal(to_np(gpu["codes"]), ref["codes"]), site.name
+            assert np.array_equal(to_np(gpu["delta"]).view(np.uint32), ref["delta"].view(np.uint32))
+            assert np.array_equal(to_np(fq.gemm_acc_i32(gpu["codes"], gpu["h"])), ref["acc"]), site.name
+            assert_close(to_np(gpu["y"]), ref["y"], site.y_dtype, f"{site.name} sigma={sigma}")
+
+
+def test_full_size_backbone_sites_sampled_rows_and_second_witness():
+    """Full-size backbone layer (gate/up N = 32768, down K = 16384): prologue checked in full,
+    outputs checked on sampled token rows, accumulators checked against the dp4a kernel."""
+    rows = [0, 1, 127, 128, 207, 208, 415, 500, 623, 624, 799, 815]
+    for site in synth.backbone_layer_sites(True):
+        data = synth.make_site(site, seed=2)
+        gpu, ref = run_site(data, rows=rows)
+        assert np.array_equal(to_np(gpu["codes"]), ref["codes"]), site.name
+        assert np.array_equal(to_np(gpu["delta"]).view(np.uint32), ref["delta"].view(np.uint32))
+        assert_close(to_np(gpu["y"][rows]), ref["y"], site.y_dtype, site.name)
+        acc = fq.gemm_acc_i32(gpu["codes"], gpu["h"])
+        assert np.array_equal(to_np(acc[rows]), ref["acc"]), site.name
+        assert torch.equal(acc, fq.gemm_simt(gpu["codes"], None, gpu["h"], raw_acc=True)), site.name
+
+
+def test_calibration_helpers_match_oracle():
+    data = synth.make_site(synth.config1_site(), seed=0, calib_tokens=512)
+    a = fq.col_absmax(to_dev(data.calib))
+    w = fq.col_absmax(to_dev(data.W["proj"]))
+    assert np.array_equal(to_np(a), oracle.col_absmax(data.calib))
+    assert np.array_equal(to_np(w), oracle.col_absmax(data.W["proj"]))
+    w2 = fq.col_absmax(to_dev(2 * data.W["proj"][:100]), out=w.clone())      # accumulate over consumers
+    assert np.array_equal(to_np(w2), np.maximum(oracle.col_absmax(data.W["proj"]),
+                                                oracle.col_absmax(2 * data.W["proj"][:100])))
+    s = fq.smooth_scale(a, w, 0.5)
+    assert np.allclose(to_np(s), oracle.smooth_scale(to_np(a), to_np(w), 0.5), rtol=1e-6)
+
+
+def test_error_codes_on_device_arguments():
+    x = torch.zeros((8, 1024), dtype=torch.float32, device="cuda")
+    W = torch.zeros((16, 1024), dtype=torch.float32, device="cuda")
+    h8 = fq.fold_weights(W, None, None, 128, 8)
+    with pytest.raises(fq.FqError) as e:
+        fq.linear_w4a4(x, h8)                                   # handle is 8-bit
+    assert e.value.status == fq.ERR_UNSUPPORTED
+    with pytest.raises(fq.FqError) as e:
+        fq.linear_w8a8(x, h8, workspace=torch.empty(256, dtype=torch.uint8, device="cuda"))
+    assert e.value.status == fq.ERR_NOMEM
+    with pytest.raises(fq.FqError) as e:
+        fq.quantize_act(x[:, 1:1 + 992], None, 32, 4)           # misaligned base pointer
+    assert e.value.status == fq.ERR_ALIGNMENT
+    with pytest.raises(fq.FqError) as e:
+        fq.linear_w8a8(x, h8, clip_ratio=0.0)
+    assert e.value.status == fq.ERR_INVALID_ARG
