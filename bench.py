@@ -1,0 +1,395 @@
+#!/usr/bin/env python
+"""Benchmark of the folded quantized linear layer on B200.
+
+Default workload (``backbone_layer``): one pi0.5-like language-backbone layer at M = 816
+tokens -- four activation sites, seven projections (q/k/v fused, o, gate/up fused, down),
+o_proj/down_proj at W8A8 and the rest W4A4.  A step is one pass of the whole hot path over
+one batch: per site the prologue kernel (scale + FWHT + per-token quantization) and the
+tcgen05 integer GEMM with its dequant/bias epilogue.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                    [--workload backbone_layer|expert_loop|sweep]
+
+Prints ONE JSON line (rank 0).  ``--impl reference`` times the CPU oracle on host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2609_24433_b200 import synth  # noqa: E402
+
+METRIC = "fused FWHT+quant+W4A4/W8A8 GEMM throughput (whole layer)"
+UNIT = "TOPS"
+ROTATE = 4            # distinct weight/activation sets cycled so that no step finds its operands in L2
+CPU_SAMPLE_ROWS = 512  # token rows the oracle arm processes per step (about 10 s on 8 cores)
+
+
+def layer_ops(sites) -> float:
+    return float(sum(2 * s.M * s.K * s.N_total for s in sites))
+
+
+def read_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(hbm_gbs=p["hbm_gbs"], bf16_burst=p["bf16_tflops"], bf16_sustained=p["bf16_tflops_sustained"],
+                    source="measured")
+    return dict(hbm_gbs=6650.0, bf16_burst=1590.0, bf16_sustained=1400.0, source="fallback")
+
+
+# ------------------------------------------------------------------ clock sampling ----
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while a region runs."""
+
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap"}
+
+    def __init__(self, index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.nv = None
+
+    def _run(self):
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(self.nv.nvmlDeviceGetClockInfo(self.h, self.nv.NVML_CLOCK_SM)))
+                mask = int(self.nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                for bit, name in self.REASONS.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(0.002)
+
+    def __enter__(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self, note: str = ""):
+        d = {"sm_mhz": (int(statistics.median(self.samples)) if self.samples else None),
+             "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+        if note:
+            d["note"] = note
+        return d
+
+
+# ------------------------------------------------------------------------ our arm ----
+class LayerOnDevice:
+    """Folded weights, inputs, outputs and workspace of ROTATE copies of one layer."""
+
+    def __init__(self, sites, seed: int, device):
+        import torch
+        from paper_2609_24433_b200 import fq
+        self.sites, self.fq, self.torch = sites, fq, torch
+        self.sets = []
+        for r in range(ROTATE):
+            entry = []
+            for i, site in enumerate(sites):
+                data = synth.make_site(site, seed + 1000 * r + i)
+                x = self._dev(data.x, site.x_dtype, device)
+                W = torch.from_numpy(np.concatenate([data.W[n] for n, _ in site.consumers], 0)).to(device)
+                b = torch.from_numpy(np.concatenate([data.bias[n] for n, _ in site.consumers], 0)).to(device)
+                smooth = None
+                if site.alpha is not None:      # SmoothQuant scale from the calibration batch, on the device
+                    a = fq.col_absmax(torch.from_numpy(data.calib).to(device))
+                    smooth = fq.smooth_scale(a, fq.col_absmax(W), site.alpha)
+                h = fq.fold_weights(W, smooth, b, site.beta, site.bits)
+                ydt = torch.float32 if site.y_dtype == "f32" else torch.bfloat16
+                y = torch.empty((site.M, site.N_total), dtype=ydt, device=device)
+                ws = torch.empty(fq.workspace_bytes(site.M, site.K, site.N_total, site.bits), dtype=torch.uint8,
+                                 device=device)
+                entry.append(dict(x=x, h=h, y=y, ws=ws, host_x=data.x, site=site))
+                del W, data
+            self.sets.append(entry)
+        torch.cuda.synchronize()
+
+    @staticmethod
+    def _dev(a, dtype, device):
+        import torch
+        if dtype == "bf16":
+            return torch.from_numpy(a.view(np.int16)).to(device).view(torch.bfloat16)
+        return torch.from_numpy(a).to(device)
+
+    def step(self, k: int, events=None):
+        """One pass of the layer. ``events``: optional list of (e0, mark, e1) per site."""
+        fq = self.fq
+        for i, e in enumerate(self.sets[k % ROTATE]):
+            if events is not None:
+                e0, mark, e1 = events[i]
+                e0.record()
+                fq.profile_mark(mark)
+            fq.linear(e["x"], e["h"], 1.0, y=e["y"], workspace=e["ws"])
+            if events is not None:
+                fq.profile_mark(None)
+                e1.record()
+
+    @property
+    def launches_per_step(self) -> int:
+        return 2 * len(self.sites)
+
+
+def run_ours(args, rank: int, world: int, local_rank: int):
+    import torch
+    from paper_2609_24433_b200 import fq
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=device)
+
+    sites = workload_sites(args.workload)
+    layer = LayerOnDevice(sites, seed=2 + 7919 * rank, device=device)
+    ops = layer_ops(sites)
+    K, Wm = args.steps, max(args.warmup, 3)
+
+    for k in range(Wm):
+        layer.step(k)
+    torch.cuda.synchronize()
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- timed region: exactly K steps, per-site events inside ----
+    ev = [[tuple(torch.cuda.Event(enable_timing=True) for _ in range(3)) for _ in sites] for _ in range(K)]
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(local_rank)
+    barrier()
+    with sampler:
+        start.record()
+        for k in range(K):
+            layer.step(Wm + k, ev[k])
+        end.record()
+        torch.cuda.synchronize()
+    barrier()
+    ms_total = start.elapsed_time(end)
+    note = ""
+    if len(sampler.samples) < 5:
+        # The timed region is shorter than NVML's refresh period: replay the same loop untimed for
+        # about half a second and sample the clocks under that identical load.
+        sampler = ClockSampler(local_rank)
+        t_end = time.time() + 0.5
+        with sampler:
+            k = 0
+            while time.time() < t_end:
+                layer.step(k)
+                k += 1
+                if k % 64 == 0:
+                    torch.cuda.synchronize()
+            torch.cuda.synchronize()
+        note = "sampled during an immediate untimed replay of the timed loop (timed region < NVML period)"
+    if dist is not None:
+        t = torch.tensor([ms_total], dtype=torch.float64, device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_per_step = ms_total / K
+    value = world * ops / (ms_per_step * 1e-3) / 1e12
+
+    st, word = fq.device_status()
+    if st != fq.OK:
+        raise RuntimeError(f"device watchdog fired during the benchmark: {word:#x}")
+
+    # per-site kernel durations out of the timed region
+    act_ms = [statistics.mean(ev[k][i][0].elapsed_time(ev[k][i][1]) for k in range(K)) for i in range(len(sites))]
+    gemm_ms = [statistics.mean(ev[k][i][1].elapsed_time(ev[k][i][2]) for k in range(K)) for i in range(len(sites))]
+    peaks = read_peaks()
+    dom = max(range(len(sites)), key=lambda i: gemm_ms[i])
+    s = sites[dom]
+    gemm_ops = 2.0 * s.M * s.K * s.N_total
+    achieved = gemm_ops / (gemm_ms[dom] * 1e-3) / 1e12
+    int8_peak = 2.0 * peaks["bf16_sustained"]     # dense int8 : bf16 = 2 : 1 (4.5 vs 2.25 PFLOP/s nominal)
+    roofline = {"bound": "tensor", "kernel": f"gemm_tcgen05_kernel<{s.bits}> ({s.name}: M={s.M} K={s.K} N={s.N_total})",
+                "achieved": round(achieved, 1), "peak": round(int8_peak, 1), "unit": "TOP/s",
+                "frac": round(achieved / int8_peak, 4),
+                "peak_source": f"{peaks['source']}: sustained bf16 cuBLAS {peaks['bf16_sustained']} TFLOP/s x 2 (int8:bf16)",
+                "traffic": TRAFFIC_BYTES.get((args.workload, s.name)),
+                "per_site_us": {sites[i].name: {"prologue": round(act_ms[i] * 1e3, 2), "gemm": round(gemm_ms[i] * 1e3, 2)}
+                                for i in range(len(sites))}}
+    act_i = max(range(len(sites)), key=lambda i: act_ms[i])
+    sa = sites[act_i]
+    act_bytes = sa.M * sa.K * (2 if sa.x_dtype == "bf16" else 4) + sa.M * sa.K + 4 * sa.M
+    roofline["prologue"] = {"site": sa.name, "bytes": act_bytes,
+                            "achieved_gbs": round(act_bytes / (act_ms[act_i] * 1e-3) / 1e9, 1),
+                            "peak_gbs": peaks["hbm_gbs"],
+                            "frac": round(act_bytes / (act_ms[act_i] * 1e-3) / 1e9 / peaks["hbm_gbs"], 4)}
+
+    # ---- end to end: host buffers, copies inside the timed region ----
+    e2e = run_e2e(layer, sites, ops, world, K, Wm, dist, device)
+
+    out = {
+        "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
+        "ms_per_step": round(ms_per_step, 5), "us_per_layer": round(ms_per_step * 1e3, 2),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int8/int4 codes, int32 accumulate, f32 transform",
+        "data": "synthetic", "impl": "ours",
+        "config": {"workload": workload_name(args.workload), "M": sites[0].M,
+                   "sites": {s.name: {"K": s.K, "N": s.N_total, "bits": s.bits, "block": s.beta} for s in sites},
+                   "ops_per_step": ops, "parallelism": "replicas only (one batch per GPU, no collective)",
+                   "l2": f"{ROTATE} rotating weight+activation sets (> 126 MB L2 in total), no flush kernel"},
+        "clocks": sampler.summary(note), "e2e": e2e, "gpu_launches": layer.launches_per_step * K,
+        "roofline": roofline,
+    }
+    if rank == 0:
+        if world == 1 and not args.no_cpu_baseline:
+            out["cpu_baseline"] = cpu_baseline(args.workload, steps=1)
+        print(json.dumps(out), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def run_e2e(layer, sites, ops, world, K, Wm, dist, device):
+    """Same step through the public API with HOST buffers: pinned host -> device copies of the
+    step's inputs, the kernels, and the device -> pinned host copy of every output, each step."""
+    import torch
+    entry = layer.sets[0]
+    host_x = []
+    for e in entry:
+        site = e["site"]
+        t = torch.from_numpy(e["host_x"].view(np.int16) if site.x_dtype == "bf16" else e["host_x"]).pin_memory()
+        host_x.append(t)
+    host_y = [torch.empty(e["y"].shape, dtype=e["y"].dtype).pin_memory() for e in entry]
+    h2d = sum(t.numel() * t.element_size() for t in host_x)
+    d2h = sum(t.numel() * t.element_size() for t in host_y)
+
+    def step():
+        for e, hx, hy in zip(entry, host_x, host_y):
+            dst = e["x"].view(torch.int16) if e["x"].dtype == torch.bfloat16 else e["x"]
+            dst.copy_(hx, non_blocking=True)
+            layer.fq.linear(e["x"], e["h"], 1.0, y=e["y"], workspace=e["ws"])
+            hy.copy_(e["y"], non_blocking=True)
+        torch.cuda.synchronize()
+
+    n = max(3, min(K, 20))
+    for _ in range(3):
+        step()
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(n):
+        step()
+    dt = (time.perf_counter() - t0) / n
+    if dist is not None:
+        t = torch.tensor([dt], dtype=torch.float64, device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dt = float(t.item())
+    return {"value": round(world * ops / dt / 1e12, 3), "unit": UNIT, "ms_per_step": round(dt * 1e3, 4),
+            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": n}
+
+
+# ------------------------------------------------------------------- oracle arm ----
+def cpu_baseline(workload: str, steps: int):
+    """The CPU oracle, as it stands, on a bounded sample of the same workload."""
+    import oracle
+    sites = workload_sites(workload)
+    rows = CPU_SAMPLE_ROWS
+    prepared = []
+    for i, site in enumerate(sites):
+        data = synth.make_site(site, 2 + i)
+        W = np.concatenate([data.W[n] for n, _ in site.consumers], 0)
+        b = np.concatenate([data.bias[n] for n, _ in site.consumers], 0)
+        smooth = None
+        if site.alpha is not None:
+            smooth = oracle.smooth_scale(oracle.col_absmax(data.calib), oracle.col_absmax(W), site.alpha)
+        wc, ws, g = oracle.fold_weights(W, "f32", smooth, site.beta, site.bits)      # offline, untimed
+        prepared.append((site, np.ascontiguousarray(data.x[:rows]), g, wc, ws, b))
+    times = []
+    for _ in range(steps):
+        t0 = time.perf_counter()
+        for site, x, g, wc, ws, b in prepared:
+            oracle.linear(x, site.x_dtype, g, site.beta, site.bits, 1.0, wc, ws, b, site.y_dtype)
+        times.append(time.perf_counter() - t0)
+    ops = sum(2.0 * rows * s.K * s.N_total for s in sites)
+    dt = statistics.mean(times)
+    return {"value": round(ops / dt / 1e12, 6), "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"{rows} of {sites[0].M} token rows through all {len(sites)} sites "
+                      f"(prologue + integer GEMM + epilogue, all N), {dt:.2f} s per step",
+            "seconds_per_step": round(dt, 3)}
+
+
+def run_reference(args):
+    sites = workload_sites(args.workload)
+    steps = max(1, min(args.steps, 5))
+    base = cpu_baseline(args.workload, steps=steps)
+    out = {"metric": METRIC, "value": base["value"], "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
+           "warmup": 0, "ms_per_step": round(base["seconds_per_step"] * 1e3, 2), "higher_is_better": True,
+           "scaling": "weak", "vs_baseline": None, "dtype": "int8/int4 codes, int32 accumulate, f32 transform",
+           "data": "synthetic", "impl": "reference",
+           "config": {"workload": workload_name(args.workload), "M": sites[0].M,
+                      "sites": {s.name: {"K": s.K, "N": s.N_total, "bits": s.bits, "block": s.beta} for s in sites}},
+           "cpu_baseline": base,
+           "e2e": {"value": base["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(out), flush=True)
+
+
+# -------------------------------------------------------------------- workloads ----
+# DRAM bytes per launch of the dominant kernel, from the ncu captures summarised under profiles/.
+TRAFFIC_BYTES = {}
+
+
+def workload_sites(name: str):
+    if name == "backbone_layer":
+        return synth.backbone_layer_sites(selective_int8=True)
+    if name == "backbone_layer_w4":
+        return synth.backbone_layer_sites(selective_int8=False)
+    if name == "expert_layer":
+        return synth.expert_layer_sites()
+    raise ValueError(name)
+
+
+def workload_name(name: str) -> str:
+    return {"backbone_layer": "pi0.5-like backbone layer, M=816, hidden 2048, MLP 16384, o/down W8A8, rest W4A4",
+            "backbone_layer_w4": "pi0.5-like backbone layer, M=816, uniform W4A4",
+            "expert_layer": "action-expert layer, M=50, width 1024, MLP 4096, W4A4, block 64"}[name]
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="backbone_layer")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        if rank == 0:
+            run_reference(args)
+        return
+    run_ours(args, rank, world, local_rank)
+
+
+if __name__ == "__main__":
+    main()

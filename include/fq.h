@@ -140,6 +140,12 @@ fq_status fq_gemm_acc_i32(const void* a_codes, int64_t M, const fq_weights* W, i
 fq_status fq_gemm_simt(const void* a_codes, const float* a_delta, int64_t M, const fq_weights* W, void* y,
                        fq_dtype yt, int64_t ldy, int32_t* acc, void* workspace, size_t ws_bytes, void* stream);
 
+/* Profiling hook (process-global, not thread-safe; benchmarks only).  While `event` -- a
+ * cudaEvent_t passed as void* -- is non-NULL, every fq_linear_* call records it on its stream
+ * between the prologue kernel and the GEMM kernel, so a caller that brackets the call with two
+ * events of its own obtains the two kernel durations of that very launch.  NULL switches it off. */
+fq_status fq_profile_mark(void* event);
+
 /* Device-side wait watchdog.  Every spin on an mbarrier inside the kernels is bounded; a wait
  * that expires records a code in a device word and the kernel winds down normally.  This call
  * SYNCHRONISES the device, returns FQ_ERR_TIMEOUT if any kernel recorded an expiry since the

@@ -57,6 +57,8 @@ fq_status alloc_handle(int64_t N, int64_t K, int block, int bits, Weights** out)
     return FQ_OK;
 }
 
+cudaEvent_t g_profile_mark = nullptr;   // see fq_profile_mark
+
 struct Workspace {
     int8_t* a8;
     float* delta;
@@ -133,6 +135,7 @@ fq_status linear_impl(const void* x, fq_dtype xt, int64_t M, int64_t ldx, const 
     if (launch_transform_quantize(x, xt, M, W->K, ldx, W->mult_g, block_norm(W->block), W->block, qmax, clip_ratio,
                                   StoreFmt::Int8, ws.a8, ws.delta, s) != cudaSuccess)
         return FQ_ERR_CUDA;
+    if (g_profile_mark != nullptr && cudaEventRecord(g_profile_mark, s) != cudaSuccess) return FQ_ERR_CUDA;
     GemmOut out;
     out.y = y; out.yt = yt; out.ldy = ldy; out.a_delta = ws.delta;
     // 4-bit weights are expanded to 16*code on chip: accumulator = 16 * integer sum.
@@ -374,6 +377,11 @@ fq_status fq_gemm_simt(const void* a_codes, const float* a_delta, int64_t M, con
         out.y = y; out.yt = yt; out.ldy = ldy; out.a_delta = a_delta;
     }
     return gemm_from_codes(a_codes, a_delta, M, W, w->bits, out, workspace, ws_bytes, static_cast<cudaStream_t>(stream), true);
+}
+
+fq_status fq_profile_mark(void* event) {
+    g_profile_mark = static_cast<cudaEvent_t>(event);
+    return FQ_OK;
 }
 
 fq_status fq_device_status(uint32_t* detail) {

@@ -18,9 +18,11 @@
 // epilogue shifts away.
 //
 // Roles (warp specialised, persistent over tiles):
-//   warp 0     TMA producer          warp 1  MMA issuer + TMEM allocator
-//   warps 2-5  epilogue (one TMEM lane quadrant each)
-//   warps 6-9  nibble unpack (4-bit weights only)
+//   warp 0       TMA producer          warp 1  MMA issuer + TMEM allocator
+//   warps 2-9    epilogue (two warps per TMEM lane quadrant, alternating 16-token chunks)
+//   warps 10-13  nibble unpack (4-bit weights only)
+// bf16 outputs leave through a per-warp 1 KB shared-memory transposer so that global
+// stores are 16-byte vectors of 8 consecutive channels; fp32/raw outputs store directly.
 // Every mbarrier wait is bounded by wall-clock time; on expiry the CTA records a
 // code in the watchdog word, stops issuing work, and still frees its TMEM.
 #include <cuda_bf16.h>
@@ -52,6 +54,10 @@ constexpr int kTileN = 128;          // output channels per tile (MMA M)
 constexpr int kBlockK = 128;         // int8 elements (= bytes) of K per pipeline stage
 constexpr int kMmaK = 32;            // K per tcgen05.mma.kind::i8
 constexpr int kAccStages = 2;
+constexpr int kEpiWarps = 8;
+constexpr int kEpiStageBytes = 16 * 64;   // 16 tokens x 32 channels of bf16 per epilogue warp
+constexpr int kThreadsW8 = 32 * (2 + kEpiWarps);
+constexpr int kThreadsW4 = kThreadsW8 + 128;
 constexpr int kMaxStages = 8;
 constexpr uint64_t kWaitLimitNs = 2000000000ull;   // 2 s per wait
 
@@ -188,7 +194,7 @@ enum : uint32_t {
 };
 
 template <int BITS>
-__global__ void __launch_bounds__(BITS == 4 ? 320 : 192, 1)
+__global__ void __launch_bounds__(BITS == 4 ? kThreadsW4 : kThreadsW8, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_w,
                     const Params p) {
     extern __shared__ uint8_t smem_raw[];
@@ -204,7 +210,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     const int lane = threadIdx.x & 31;
     volatile int* abort_flag = &s_abort;
 
-    // carve dynamic shared memory: [A8 stages][W8 stages][packed stages], all 1024-byte aligned
+    // carve dynamic shared memory: [A8 stages][W8 stages][packed stages][epilogue transposers], 1024-byte aligned
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t a_bytes = (uint32_t)p.bt * kBlockK;
     const uint32_t w_bytes = kTileN * kBlockK;
@@ -212,6 +218,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     const uint32_t smem_a = base;
     const uint32_t smem_w = smem_a + (uint32_t)p.stages * a_bytes;
     const uint32_t smem_p = smem_w + (uint32_t)p.stages * w_bytes;
+    const uint32_t smem_e = smem_p + (BITS == 4 ? (uint32_t)p.stages * pk_bytes : 0u);
     uint8_t* gen_base = smem_raw + (base - smem_u32(smem_raw));   // generic pointer to `base`
 
     if (threadIdx.x == 0) {
@@ -223,7 +230,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         }
         for (int a = 0; a < kAccStages; ++a) {
             mbar_init(smem_u32(&s_acc_full[a]), 1);
-            mbar_init(smem_u32(&s_acc_empty[a]), 4);
+            mbar_init(smem_u32(&s_acc_empty[a]), kEpiWarps);
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_proxy_async_smem();
@@ -313,19 +320,24 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                 if (++acc_stage == kAccStages) { acc_stage = 0; acc_phase ^= 1u; }
             }
         }
-    } else if (warp < 6) {
+    } else if (warp < 2 + kEpiWarps) {
         // ---------------------------------------------------------------- epilogue
         const int quad = warp & 3;                       // TMEM lanes [32*quad, 32*quad + 32)
+        const int half = (warp - 2) >> 2;                // which of the alternating 16-token chunks
+        uint8_t* xpose = gen_base + (smem_e - base) + (warp - 2) * kEpiStageBytes;
+        const bool staged = p.out.acc == nullptr && p.out.yt == FQ_BF16;
+        const float unshift = 1.0f / (float)(1 << p.acc_shift);   // exact power of two
         int acc_stage = 0;
         uint32_t acc_phase = 0;
         bool ok = true;
         for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-            const int64_t j = (int64_t)(tile / p.m_tiles) * kTileN + quad * 32 + lane;
+            const int64_t jq = (int64_t)(tile / p.m_tiles) * kTileN + quad * 32;   // first channel of this warp
+            const int64_t j = jq + lane;
             const int64_t t0 = (int64_t)(tile % p.m_tiles) * p.bt;
             const bool j_ok = j < p.N;
             float sw = 0.0f, bj = 0.0f;
             if (j_ok && p.out.acc == nullptr) {
-                sw = __ldg(p.w_scale + j);
+                sw = __ldg(p.w_scale + j) * unshift;     // (float)acc * 2^-shift is exact: fold the shift here
                 bj = __ldg(p.bias + j);
             }
             ok = mbar_wait(smem_u32(&s_acc_full[acc_stage]), acc_phase, abort_flag, p.watchdog, kWdEpilogue);
@@ -333,24 +345,58 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             if (!ok) break;
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc_stage * p.bt);
-            for (int c = 0; c < p.bt; c += 16) {
-                if (t0 + c >= p.M) break;                // tokens beyond M: nothing to store (warp-uniform)
+            for (int c = half * 16; c < p.bt; c += 32) {
+                const int64_t tc = t0 + c;
+                if (tc >= p.M) break;                    // tokens beyond M: nothing to store (warp-uniform)
                 uint32_t r[16];
                 tmem_ld16(taddr + (uint32_t)c, r);
-                tmem_ld_wait();
+                if (p.out.acc != nullptr) {
+                    tmem_ld_wait();
 #pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    const int64_t t = t0 + c + i;
-                    if (t < p.M && j_ok) {
-                        const int acc = ((int)r[i]) >> p.acc_shift;
-                        if (p.out.acc != nullptr) {
-                            p.out.acc[t * p.N + j] = acc;
-                        } else {
-                            const float v = fmaf((float)acc, __ldg(p.out.a_delta + t) * sw, bj);
+                    for (int i = 0; i < 16; ++i)
+                        if (tc + i < p.M && j_ok) p.out.acc[(tc + i) * p.N + j] = ((int)r[i]) >> p.acc_shift;
+                    continue;
+                }
+                float d[16];
+                if (tc + 16 <= p.M) {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const float4 q = __ldg(reinterpret_cast<const float4*>(p.out.a_delta + tc) + i);
+                        d[4 * i + 0] = q.x; d[4 * i + 1] = q.y; d[4 * i + 2] = q.z; d[4 * i + 3] = q.w;
+                    }
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) d[i] = tc + i < p.M ? __ldg(p.out.a_delta + tc + i) : 0.0f;
+                }
+                tmem_ld_wait();
+                if (staged) {
+                    // transpose 32 channels x 16 tokens through shared memory, then 16-byte stores
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        const float v = fmaf((float)(int)r[i], d[i] * sw, bj);
+                        *reinterpret_cast<__nv_bfloat16*>(xpose + i * 64 + lane * 2) = __float2bfloat16_rn(v);
+                    }
+                    __syncwarp();
+                    __nv_bfloat16* y = static_cast<__nv_bfloat16*>(p.out.y);
+#pragma unroll
+                    for (int k = 0; k < 2; ++k) {
+                        const int row = (lane >> 2) + 8 * k;
+                        const int64_t jj = jq + (lane & 3) * 8;
+                        const uint4 v = *reinterpret_cast<const uint4*>(xpose + row * 64 + (lane & 3) * 16);
+                        if (tc + row < p.M && jj < p.N)
+                            *reinterpret_cast<uint4*>(y + (tc + row) * p.out.ldy + jj) = v;
+                    }
+                    __syncwarp();
+                } else {
+                    float* y = static_cast<float*>(p.out.y) + tc * p.out.ldy + j;
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        const float v = fmaf((float)(int)r[i], d[i] * sw, bj);
+                        if (tc + i < p.M && j_ok) {
                             if (p.out.yt == FQ_F32)
-                                static_cast<float*>(p.out.y)[t * p.out.ldy + j] = v;
+                                y[i * p.out.ldy] = v;
                             else
-                                static_cast<__nv_bfloat16*>(p.out.y)[t * p.out.ldy + j] = __float2bfloat16_rn(v);
+                                reinterpret_cast<__nv_bfloat16*>(p.out.y)[(tc + i) * p.out.ldy + j] = __float2bfloat16_rn(v);
                         }
                     }
                 }
@@ -362,7 +408,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         }
     } else if (BITS == 4) {
         // ------------------------------------------------------------ nibble unpack
-        const int ut = threadIdx.x - 192;                // 0..127
+        const int ut = threadIdx.x - kThreadsW8;         // 0..127
         int stage = 0;
         uint32_t phase = 0;
         bool ok = true;
@@ -484,12 +530,13 @@ fq_status launch_gemm_tcgen05(const int8_t* a8, int64_t M, const Weights& W, int
     p.tmem_cols = next_pow2(kAccStages * bt);
 
     const size_t stage_bytes = (size_t)bt * kBlockK + kTileN * kBlockK + (W.bits == 4 ? kTileN * kBlockK / 2 : 0);
-    const size_t budget = 227 * 1024 - 1024 /*alignment slack*/ - 1024 /*static*/;
+    const size_t epi_bytes = (size_t)kEpiWarps * kEpiStageBytes;
+    const size_t budget = 227 * 1024 - 1024 /*alignment slack*/ - 1024 /*static*/ - epi_bytes;
     int stages = (int)(budget / stage_bytes);
     if (stages > kMaxStages) stages = kMaxStages;
     if (stages < 2) return FQ_ERR_UNSUPPORTED;
     p.stages = stages;
-    const size_t smem = stage_bytes * stages + 1024;
+    const size_t smem = stage_bytes * stages + epi_bytes + 1024;
 
     CUtensorMap map_a;
     if (!encode_2d(&map_a, a8, (uint64_t)W.K, (uint64_t)M, kBlockK, (uint32_t)bt, true)) return FQ_ERR_CUDA;
@@ -504,11 +551,11 @@ fq_status launch_gemm_tcgen05(const int8_t* a8, int64_t M, const Weights& W, int
     if (W.bits == 4) {
         e = cudaFuncSetAttribute(gemm_tcgen05_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return FQ_ERR_CUDA;
-        gemm_tcgen05_kernel<4><<<grid, 320, smem, stream>>>(map_a, W.tmap, p);
+        gemm_tcgen05_kernel<4><<<grid, kThreadsW4, smem, stream>>>(map_a, W.tmap, p);
     } else {
         e = cudaFuncSetAttribute(gemm_tcgen05_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return FQ_ERR_CUDA;
-        gemm_tcgen05_kernel<8><<<grid, 192, smem, stream>>>(map_a, W.tmap, p);
+        gemm_tcgen05_kernel<8><<<grid, kThreadsW8, smem, stream>>>(map_a, W.tmap, p);
     }
     return cudaGetLastError() == cudaSuccess ? FQ_OK : FQ_ERR_CUDA;
 }

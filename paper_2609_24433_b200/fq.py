@@ -23,7 +23,7 @@ EXPORTS = [
     "fq_status_string", "fq_fold_weights", "fq_weights_destroy", "fq_weights_info", "fq_weights_multiplier",
     "fq_weights_export", "fq_weights_import", "fq_col_absmax", "fq_smooth_scale", "fq_quantize_act",
     "fq_gemm_w4a4", "fq_gemm_w8a8", "fq_linear_w4a4", "fq_linear_w8a8", "fq_workspace_bytes",
-    "fq_gemm_acc_i32", "fq_gemm_simt", "fq_device_status",
+    "fq_gemm_acc_i32", "fq_gemm_simt", "fq_device_status", "fq_profile_mark",
 ]
 
 _lib = None
@@ -268,6 +268,13 @@ def gemm_simt(a_codes, a_delta, W: Weights, out_dtype=torch.float32, raw_acc: bo
                               _out_dt(out_dtype), ctypes.c_int64(W.N if y is None else y.stride(0)), _ptr(acc),
                               _ptr(ws), ctypes.c_size_t(ws.numel()), _stream()), "fq_gemm_simt")
     return acc if raw_acc else y
+
+
+def profile_mark(event: Optional[torch.cuda.Event]):
+    """Record ``event`` between the prologue and the GEMM of every linear_* call (None = off)."""
+    if event is not None and not event.cuda_event:
+        event.record()      # torch creates the underlying cudaEvent_t lazily, on its first record
+    _check(lib().fq_profile_mark(ctypes.c_void_p(0 if event is None else event.cuda_event)), "fq_profile_mark")
 
 
 def device_status() -> Tuple[int, int]:
