@@ -150,6 +150,42 @@ class LayerOnDevice:
                 fq.profile_mark(None)
                 e1.record()
 
+    def capture(self):
+        """One CUDA graph per rotating set (the step's kernels back to back, no host launch gaps),
+        and a second graph per set that also carries external event-record nodes around and
+        inside every site so that single-kernel durations can be read after a replay."""
+        torch = self.torch
+        self.graphs, self.ev_graphs, self.ev = [], [], []
+        for r in range(ROTATE):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                self.step(r)
+            self.graphs.append(g)
+            evs = [tuple(torch.cuda.Event(enable_timing=True, external=True) for _ in range(3)) for _ in self.sites]
+            for trio in evs:
+                for e in trio:
+                    e.record()          # creates the underlying event before the capture
+            torch.cuda.synchronize()
+            g2 = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g2):
+                self.step(r, evs)
+            self.ev_graphs.append(g2)
+            self.ev.append(evs)
+        torch.cuda.synchronize()
+
+    def kernel_durations(self, replays: int):
+        """Mean (prologue_ms, gemm_ms) per site over ``replays`` replays of the evented graphs."""
+        torch = self.torch
+        act = [[] for _ in self.sites]
+        gemm = [[] for _ in self.sites]
+        for k in range(replays):
+            self.ev_graphs[k % ROTATE].replay()
+            torch.cuda.synchronize()
+            for i, (e0, mark, e1) in enumerate(self.ev[k % ROTATE]):
+                act[i].append(e0.elapsed_time(mark))
+                gemm[i].append(mark.elapsed_time(e1))
+        return [statistics.mean(a) for a in act], [statistics.mean(g) for g in gemm]
+
     @property
     def launches_per_step(self) -> int:
         return 2 * len(self.sites)
@@ -180,15 +216,17 @@ def run_ours(args, rank: int, world: int, local_rank: int):
             dist.barrier()
         torch.cuda.synchronize()
 
-    # ---- timed region: exactly K steps, per-site events inside ----
-    ev = [[tuple(torch.cuda.Event(enable_timing=True) for _ in range(3)) for _ in sites] for _ in range(K)]
+    # ---- timed region: exactly K steps, each one replay of a captured step graph ----
+    layer.capture()
+    for k in range(Wm):
+        layer.graphs[k % ROTATE].replay()
     start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     sampler = ClockSampler(local_rank)
     barrier()
     with sampler:
         start.record()
         for k in range(K):
-            layer.step(Wm + k, ev[k])
+            layer.graphs[(Wm + k) % ROTATE].replay()
         end.record()
         torch.cuda.synchronize()
     barrier()
@@ -202,7 +240,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         with sampler:
             k = 0
             while time.time() < t_end:
-                layer.step(k)
+                layer.graphs[k % ROTATE].replay()
                 k += 1
                 if k % 64 == 0:
                     torch.cuda.synchronize()
@@ -219,9 +257,8 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     if st != fq.OK:
         raise RuntimeError(f"device watchdog fired during the benchmark: {word:#x}")
 
-    # per-site kernel durations out of the timed region
-    act_ms = [statistics.mean(ev[k][i][0].elapsed_time(ev[k][i][1]) for k in range(K)) for i in range(len(sites))]
-    gemm_ms = [statistics.mean(ev[k][i][1].elapsed_time(ev[k][i][2]) for k in range(K)) for i in range(len(sites))]
+    # per-kernel durations: the same step graphs with event-record nodes between the kernels
+    act_ms, gemm_ms = layer.kernel_durations(max(8, min(K, 40)))
     peaks = read_peaks()
     dom = max(range(len(sites)), key=lambda i: gemm_ms[i])
     s = sites[dom]
@@ -254,7 +291,8 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         "config": {"workload": workload_name(args.workload), "M": sites[0].M,
                    "sites": {s.name: {"K": s.K, "N": s.N_total, "bits": s.bits, "block": s.beta} for s in sites},
                    "ops_per_step": ops, "parallelism": "replicas only (one batch per GPU, no collective)",
-                   "l2": f"{ROTATE} rotating weight+activation sets (> 126 MB L2 in total), no flush kernel"},
+                   "l2": f"{ROTATE} rotating weight+activation sets (> 126 MB L2 in total), no flush kernel",
+                   "launch": "one CUDA-graph replay per step"},
         "clocks": sampler.summary(note), "e2e": e2e, "gpu_launches": layer.launches_per_step * K,
         "roofline": roofline,
     }

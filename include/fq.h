@@ -143,7 +143,8 @@ fq_status fq_gemm_simt(const void* a_codes, const float* a_delta, int64_t M, con
 /* Profiling hook (process-global, not thread-safe; benchmarks only).  While `event` -- a
  * cudaEvent_t passed as void* -- is non-NULL, every fq_linear_* call records it on its stream
  * between the prologue kernel and the GEMM kernel, so a caller that brackets the call with two
- * events of its own obtains the two kernel durations of that very launch.  NULL switches it off. */
+ * events of its own obtains the two kernel durations of that very launch.  During a stream capture
+ * the mark becomes an external event-record node of the graph.  NULL switches it off. */
 fq_status fq_profile_mark(void* event);
 
 /* Device-side wait watchdog.  Every spin on an mbarrier inside the kernels is bounded; a wait

@@ -135,7 +135,13 @@ fq_status linear_impl(const void* x, fq_dtype xt, int64_t M, int64_t ldx, const 
     if (launch_transform_quantize(x, xt, M, W->K, ldx, W->mult_g, block_norm(W->block), W->block, qmax, clip_ratio,
                                   StoreFmt::Int8, ws.a8, ws.delta, s) != cudaSuccess)
         return FQ_ERR_CUDA;
-    if (g_profile_mark != nullptr && cudaEventRecord(g_profile_mark, s) != cudaSuccess) return FQ_ERR_CUDA;
+    if (g_profile_mark != nullptr) {
+        // Inside a stream capture the mark must be an external event-record node to stay readable.
+        cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+        if (cudaStreamIsCapturing(s, &cap) != cudaSuccess) return FQ_ERR_CUDA;
+        const unsigned flags = cap == cudaStreamCaptureStatusActive ? cudaEventRecordExternal : cudaEventRecordDefault;
+        if (cudaEventRecordWithFlags(g_profile_mark, s, flags) != cudaSuccess) return FQ_ERR_CUDA;
+    }
     GemmOut out;
     out.y = y; out.yt = yt; out.ldy = ldy; out.a_delta = ws.delta;
     // 4-bit weights are expanded to 16*code on chip: accumulator = 16 * integer sum.
