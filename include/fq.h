@@ -127,6 +127,29 @@ fq_status fq_linear_w8a8(const void* x, fq_dtype xt, int64_t M, int64_t ldx, con
                          float clip_ratio, void* y, fq_dtype yt, int64_t ldy, void* workspace,
                          size_t ws_bytes, void* stream);
 
+/* ---- fused W4A4 linear without a workspace, for callers that cannot allocate ------------------
+ * (The paper has no counterpart: this is a deployment convenience of this library.)
+ * Same result as fq_linear_w4a4, but the quantized activations and per-token steps that sit
+ * between the two kernels live in a scratch area built into the library image instead of a
+ * caller workspace.  It is meant for code that has no way to obtain device memory at call time:
+ * plugin enqueue callbacks that are forbidden to call cudaMalloc, control loops that cannot
+ * tolerate the device-wide synchronisation an allocation can imply, processes whose device
+ * memory was all handed out at start-up.  The call performs no cudaMalloc/cudaFree and calls no
+ * allocating library routine; the caller still provides x and y.
+ *   Limits: M * K <= FQ_STATIC_MAX_CODE_BYTES (4 MiB) and M <= FQ_STATIC_MAX_TOKENS (16384);
+ *   anything larger returns FQ_ERR_NOMEM and launches nothing.  The scratch (4 MiB + 64 KiB) is
+ *   held by every GPU that loads the library until the process exits.
+ *   The first call on each device looks up the scratch's device address (once, with that device
+ *   current); make that first call before any stream capture.
+ *   All calls on a device share the one scratch.  Nothing in it needs clearing -- each call
+ *   rewrites every row it later reads -- but it keeps the previous call's contents, and two calls
+ *   whose kernels may overlap on the GPU (different streams without an ordering between them)
+ *   race on it: keep calls to this entry point stream-ordered per device. */
+#define FQ_STATIC_MAX_CODE_BYTES (4ll << 20)
+#define FQ_STATIC_MAX_TOKENS 16384ll
+fq_status fq_linear_w4a4_static(const void* x, fq_dtype xt, int64_t M, int64_t ldx, const fq_weights* W,
+                                float clip_ratio, void* y, fq_dtype yt, int64_t ldy, void* stream);
+
 /* Bytes of workspace that fq_gemm_* / fq_linear_* need for this shape (host computation). */
 size_t fq_workspace_bytes(int64_t M, int64_t K, int64_t N, int bits);
 

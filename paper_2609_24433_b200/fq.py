@@ -23,7 +23,7 @@ EXPORTS = [
     "fq_status_string", "fq_fold_weights", "fq_weights_destroy", "fq_weights_info", "fq_weights_multiplier",
     "fq_weights_export", "fq_weights_import", "fq_col_absmax", "fq_smooth_scale", "fq_quantize_act",
     "fq_gemm_w4a4", "fq_gemm_w8a8", "fq_linear_w4a4", "fq_linear_w8a8", "fq_workspace_bytes",
-    "fq_gemm_acc_i32", "fq_gemm_simt", "fq_device_status", "fq_profile_mark",
+    "fq_gemm_acc_i32", "fq_gemm_simt", "fq_device_status", "fq_profile_mark", "fq_linear_w4a4_static",
 ]
 
 _lib = None
@@ -239,6 +239,24 @@ def linear_w4a4(x, W: Weights, clip_ratio: float = 1.0, out_dtype=torch.float32,
 
 def linear_w8a8(x, W: Weights, clip_ratio: float = 1.0, out_dtype=torch.float32, y=None, workspace=None):
     return _linear("fq_linear_w8a8", x, W, clip_ratio, out_dtype, y, workspace)
+
+
+STATIC_MAX_CODE_BYTES = 4 << 20
+STATIC_MAX_TOKENS = 16384
+
+
+def linear_w4a4_static(x, W: Weights, clip_ratio: float = 1.0, out_dtype=torch.float32, y=None):
+    """fq_linear_w4a4 on the library's built-in scratch: for callers that cannot allocate device
+    memory at call time.  Only the output tensor is created here when ``y`` is not passed in, and
+    the entry point itself allocates nothing; M*K must fit STATIC_MAX_CODE_BYTES."""
+    x = _rowmajor(x)
+    M = x.shape[0]
+    if y is None:
+        y = torch.empty((M, W.N), dtype=out_dtype, device=x.device)
+    _check(lib().fq_linear_w4a4_static(_ptr(x), _dt(x), ctypes.c_int64(M), ctypes.c_int64(x.stride(0)), W.handle,
+                                       ctypes.c_float(clip_ratio), _ptr(y), _out_dt(y.dtype),
+                                       ctypes.c_int64(y.stride(0)), _stream()), "fq_linear_w4a4_static")
+    return y
 
 
 def linear(x, W: Weights, clip_ratio: float = 1.0, out_dtype=torch.float32, y=None, workspace=None):
