@@ -1,0 +1,31 @@
+// Device helpers shared by the two prologue kernels.
+#pragma once
+
+#include <stdint.h>
+
+namespace fq {
+
+// Round-to-nearest-even code extraction: bits(t + 1.5*2^23) = 0x4B400000 + rint(t) for |t| < 2^22.
+constexpr uint32_t kMagicBits = 0x4B400000u;
+
+// Pack 8 four-bit (or 4 eight-bit) two's-complement codes from the raw bit patterns
+// b[i] = kMagicBits + code_i (element 0 in the lowest field) with one shift-add per code:
+// the Horner sum of the raw patterns equals the Horner sum of the codes plus a constant;
+// adding half the field range to every field removes the borrows between fields, and
+// flipping each field's top bit afterwards turns offset binary into two's complement.
+template <int FMT>
+__device__ __forceinline__ uint32_t pack_word(const uint32_t* b) {
+    if (FMT == 0) {
+        uint32_t w = b[7];
+#pragma unroll
+        for (int i = 6; i >= 0; --i) w = (w << 4) + b[i];
+        return (w + (0x88888888u - kMagicBits * 0x11111111u)) ^ 0x88888888u;
+    } else {
+        uint32_t w = b[3];
+#pragma unroll
+        for (int i = 2; i >= 0; --i) w = (w << 8) + b[i];
+        return (w + (0x80808080u - kMagicBits * 0x01010101u)) ^ 0x80808080u;
+    }
+}
+
+}  // namespace fq

@@ -21,6 +21,7 @@
 #include <float.h>
 
 #include "fq_common.cuh"
+#include "act_common.cuh"
 
 namespace fq {
 namespace {
@@ -69,12 +70,6 @@ struct RawRow<__nv_bfloat16, E> {
         }
     }
 };
-
-__device__ __forceinline__ uint32_t bfi(uint32_t src, uint32_t dst, int pos, int len) {
-    uint32_t r;
-    asm("bfi.b32 %0, %1, %2, %3, %4;" : "=r"(r) : "r"(src), "r"(dst), "r"(pos), "r"(len));
-    return r;
-}
 
 // FMT: 0 = two 4-bit codes per byte, 1 = one int8 per code.  CLAMP: clip_ratio < 1.
 // CACHE: keep the multiplier slice in registers across tokens and prefetch the next
@@ -198,18 +193,18 @@ transform_quantize_kernel(const XT* __restrict__ x, int64_t rows, int K, int64_t
 
         // round to nearest even through the 1.5*2^23 trick: the low mantissa bits of
         // (t + 12582912) hold the two's-complement integer rint(t) for |t| < 2^22
-        uint32_t w[FMT == 0 ? E / 8 : E / 4];
+        constexpr int kPer = FMT == 0 ? 8 : 4;               // codes per 32-bit word
+        uint32_t w[E / kPer];
 #pragma unroll
-        for (int i = 0; i < (FMT == 0 ? E / 8 : E / 4); ++i) w[i] = 0u;
+        for (int j = 0; j < E / kPer; ++j) {
+            uint32_t b[kPer];
 #pragma unroll
-        for (int i = 0; i < E; ++i) {
-            float t = __fmul_rn(v[i], inv);
-            if (CLAMP) t = fminf(fmaxf(t, -qmax), qmax);
-            const uint32_t b = __float_as_uint(__fadd_rn(t, 12582912.0f));
-            if (FMT == 0)
-                w[i / 8] = bfi(b, w[i / 8], 4 * (i % 8), 4);
-            else
-                w[i / 4] = bfi(b, w[i / 4], 8 * (i % 4), 8);
+            for (int i = 0; i < kPer; ++i) {
+                float t = __fmul_rn(v[j * kPer + i], inv);
+                if (CLAMP) t = fminf(fmaxf(t, -qmax), qmax);
+                b[i] = __float_as_uint(__fadd_rn(t, 12582912.0f));
+            }
+            w[j] = pack_word<FMT>(b);
         }
         if (row_ok) {
             if (FMT == 0) {
@@ -350,6 +345,11 @@ cudaError_t launch_transform_quantize(const void* x, fq_dtype xt, int64_t rows, 
                                       const float* mult, float cnorm, int block, int qmax, float clip_ratio,
                                       StoreFmt fmt, void* codes, float* delta, cudaStream_t stream) {
     if (rows == 0) return cudaSuccess;
+    {   // long batches stream through the TMA-fed ring; everything else stays in registers
+        const cudaError_t e = launch_transform_quantize_ring(x, xt, rows, K, ldx, mult, cnorm, block, qmax, clip_ratio,
+                                                             fmt, codes, delta, stream);
+        if (e != cudaErrorNotSupported) return e;
+    }
     const int k = (int)K;
     if (xt == FQ_F32) {
         const float* p = static_cast<const float*>(x);

@@ -66,6 +66,17 @@ cudaError_t launch_gemm_simt(const int8_t* a8, int64_t M, const Weights& W, int 
 fq_status launch_gemm_tcgen05(const int8_t* a8, int64_t M, const Weights& W, int acc_shift, const GemmOut& out,
                               cudaStream_t stream);
 
+// cuTensorMapEncodeTiled through the runtime's driver entry point (no link-time libcuda dependency).
+// dims/box innermost first; strides_bytes has rank-1 entries (dimension 0 is contiguous).
+bool encode_tiled(CUtensorMap* map, CUtensorMapDataType dt, uint32_t rank, const void* ptr, const uint64_t* dims,
+                  const uint64_t* strides_bytes, const uint32_t* box, bool swizzle128);
+
+// Streaming variant of the prologue (TMA-fed shared-memory ring). Returns cudaErrorNotSupported
+// when the shape does not fit it; the caller then uses the register-only kernel.
+cudaError_t launch_transform_quantize_ring(const void* x, fq_dtype xt, int64_t rows, int64_t K, int64_t ldx,
+                                           const float* mult, float cnorm, int block, int qmax, float clip_ratio,
+                                           StoreFmt fmt, void* codes, float* delta, cudaStream_t stream);
+
 // Builds the weight-operand tensor map of a handle (after `codes` is allocated).
 fq_status build_weight_tmap(Weights& W);
 

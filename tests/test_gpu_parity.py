@@ -48,6 +48,11 @@ ACT_CASES = [
     (3, 32768, 64, 8, "f32", False, 0.75),
     (1, 2048, 128, 4, "bf16", False, 1.0),
     (2500, 1024, 64, 4, "bf16", False, 1.0),
+    (600, 2048, 128, 4, "f32", True, 0.8),
+    (400, 4096, 256, 8, "f32", False, 1.0),
+    (333, 3072, 128, 4, "bf16", True, 1.0),
+    (1000, 16384, 256, 4, "bf16", True, 1.0),
+    (700, 8192, 32, 8, "bf16", False, 0.6),
 ]
 
 
