@@ -20,12 +20,16 @@
 // Roles (warp specialised, persistent over tiles):
 //   warp 0       TMA producer          warp 1  MMA issuer + TMEM allocator
 //   warps 2-9    epilogue (two warps per TMEM lane quadrant, alternating 16-token chunks)
-//   warps 10-13  nibble unpack (4-bit weights only)
+//   warps 10-13  nibble unpack, warp 14 TMA producer of packed weights (4-bit weights only)
+// With 4-bit weights three rings are decoupled: activations (TMA -> MMA), packed weights
+// (TMA -> unpack, deep and cheap: 8 KB a stage) and unpacked weights (unpack -> MMA, 3 stages),
+// so the unpack latency sits beside, not inside, the TMA round trip.
 // bf16 outputs leave through a per-warp 1 KB shared-memory transposer so that global
 // stores are 16-byte vectors of 8 consecutive channels; fp32/raw outputs store directly.
 // Every mbarrier wait is bounded by wall-clock time; on expiry the CTA records a
 // code in the watchdog word, stops issuing work, and still frees its TMEM.
 #include <cuda_bf16.h>
+#include <stdlib.h>
 
 #include "fq_common.cuh"
 #include "ptx_sm100.cuh"
@@ -58,13 +62,16 @@ constexpr int kAccStages = 2;
 constexpr int kEpiWarps = 8;
 constexpr int kEpiStageBytes = 16 * 64;   // 16 tokens x 32 channels of bf16 per epilogue warp
 constexpr int kThreadsW8 = 32 * (2 + kEpiWarps);
-constexpr int kThreadsW4 = kThreadsW8 + 128;
+constexpr int kThreadsW4 = kThreadsW8 + 128 + 32;
+constexpr int kMaxStagesW = 4;
 constexpr int kMaxStages = 8;
 
 struct Params {
     int64_t M, N, K;
     int bt;              // tokens per tile (MMA N), multiple of 16, <= 256
-    int stages;
+    int stages;          // activation ring (and int8 weight ring, in lockstep, for 8-bit weights)
+    int stages_p;        // packed-weight ring (4-bit weights)
+    int stages_w;        // unpacked-weight ring (4-bit weights)
     int m_tiles, n_tiles;
     int tmem_cols;
     int acc_shift;
@@ -140,9 +147,12 @@ __global__ void __launch_bounds__(BITS == 4 ? kThreadsW4 : kThreadsW8, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_w,
                     const Params p) {
     extern __shared__ uint8_t smem_raw[];
-    __shared__ uint64_t s_full_tma[kMaxStages];
-    __shared__ uint64_t s_full_w8[kMaxStages];
-    __shared__ uint64_t s_empty[kMaxStages];
+    __shared__ uint64_t s_full_tma[kMaxStages];     // activations (+ int8 weights) landed
+    __shared__ uint64_t s_empty[kMaxStages];        // ... consumed by the MMAs
+    __shared__ uint64_t s_full_p[kMaxStages];       // packed weights landed
+    __shared__ uint64_t s_empty_p[kMaxStages];      // ... read by the unpack warps
+    __shared__ uint64_t s_full_w8[kMaxStagesW];     // unpacked weights written
+    __shared__ uint64_t s_empty_w8[kMaxStagesW];    // ... consumed by the MMAs
     __shared__ uint64_t s_acc_full[kAccStages];
     __shared__ uint64_t s_acc_empty[kAccStages];
     __shared__ uint32_t s_tmem_base;
@@ -159,16 +169,25 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     const uint32_t pk_bytes = kTileN * kBlockK / 2;
     const uint32_t smem_a = base;
     const uint32_t smem_w = smem_a + (uint32_t)p.stages * a_bytes;
-    const uint32_t smem_p = smem_w + (uint32_t)p.stages * w_bytes;
-    const uint32_t smem_e = smem_p + (BITS == 4 ? (uint32_t)p.stages * pk_bytes : 0u);
+    const uint32_t smem_p = smem_w + (uint32_t)(BITS == 4 ? p.stages_w : p.stages) * w_bytes;
+    const uint32_t smem_e = smem_p + (BITS == 4 ? (uint32_t)p.stages_p * pk_bytes : 0u);
     uint8_t* gen_base = smem_raw + (base - smem_u32(smem_raw));   // generic pointer to `base`
 
     if (threadIdx.x == 0) {
         s_abort = 0;
         for (int s = 0; s < p.stages; ++s) {
             mbar_init(smem_u32(&s_full_tma[s]), 1);
-            mbar_init(smem_u32(&s_full_w8[s]), 4);
             mbar_init(smem_u32(&s_empty[s]), 1);
+        }
+        if (BITS == 4) {
+            for (int s = 0; s < p.stages_p; ++s) {
+                mbar_init(smem_u32(&s_full_p[s]), 1);
+                mbar_init(smem_u32(&s_empty_p[s]), 4);
+            }
+            for (int s = 0; s < p.stages_w; ++s) {
+                mbar_init(smem_u32(&s_full_w8[s]), 4);
+                mbar_init(smem_u32(&s_empty_w8[s]), 1);
+            }
         }
         for (int a = 0; a < kAccStages; ++a) {
             mbar_init(smem_u32(&s_acc_full[a]), 1);
@@ -191,7 +210,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         if (lane == 0) {
             int stage = 0;
             uint32_t phase = 0;
-            const uint32_t tx = a_bytes + (BITS == 4 ? pk_bytes : w_bytes);
+            const uint32_t tx = a_bytes + (BITS == 4 ? 0u : w_bytes);
             bool ok = true;
             int issued = 0;
             for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
@@ -203,10 +222,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                     const uint32_t bar = smem_u32(&s_full_tma[stage]);
                     mbar_arrive_expect_tx(bar, tx);
                     tma_load_2d(smem_a + stage * a_bytes, &map_a, kb * kBlockK, t0, bar);
-                    if (BITS == 4)
-                        tma_load_2d(smem_p + stage * pk_bytes, &map_w, kb * (kBlockK / 2), n0, bar);
-                    else
-                        tma_load_2d(smem_w + stage * w_bytes, &map_w, kb * kBlockK, n0, bar);
+                    if (BITS == 8) tma_load_2d(smem_w + stage * w_bytes, &map_w, kb * kBlockK, n0, bar);
                     ++issued;
                     if (++stage == p.stages) { stage = 0; phase ^= 1u; }
                 }
@@ -230,8 +246,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         // -------------------------------------------------------------- MMA issuer
         if (lane == 0) {
             const uint32_t idesc = instr_desc_i8(p.bt);
-            int stage = 0;
-            uint32_t phase = 0;
+            int stage = 0, wstage = 0;
+            uint32_t phase = 0, wphase = 0;
             int acc_stage = 0;
             uint32_t acc_phase = 0;
             bool ok = true;
@@ -243,10 +259,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                 for (int kb = 0; kb < k_blocks; ++kb) {
                     ok = mbar_wait(smem_u32(&s_full_tma[stage]), phase, abort_flag, p.watchdog, kWdMmaFull);
                     if (ok && BITS == 4)
-                        ok = mbar_wait(smem_u32(&s_full_w8[stage]), phase, abort_flag, p.watchdog, kWdMmaFull);
+                        ok = mbar_wait(smem_u32(&s_full_w8[wstage]), wphase, abort_flag, p.watchdog, kWdMmaFull);
                     if (!ok) break;
                     tc_fence_after();
-                    const uint64_t wdesc = smem_desc_sw128(smem_w + stage * w_bytes);
+                    const uint64_t wdesc = smem_desc_sw128(smem_w + (BITS == 4 ? wstage : stage) * w_bytes);
                     const uint64_t adesc = smem_desc_sw128(smem_a + stage * a_bytes);
 #pragma unroll
                     for (int k = 0; k < kBlockK / kMmaK; ++k) {
@@ -256,6 +272,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                     }
                     mma_commit(smem_u32(&s_empty[stage]));          // frees this stage when the MMAs retire
                     if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+                    if (BITS == 4) {
+                        mma_commit(smem_u32(&s_empty_w8[wstage]));
+                        if (++wstage == p.stages_w) { wstage = 0; wphase ^= 1u; }
+                    }
                 }
                 if (!ok) break;
                 mma_commit(smem_u32(&s_acc_full[acc_stage]));        // accumulator complete
@@ -348,27 +368,31 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             if (lane == 0) mbar_arrive(smem_u32(&s_acc_empty[acc_stage]));
             if (++acc_stage == kAccStages) { acc_stage = 0; acc_phase ^= 1u; }
         }
-    } else if (BITS == 4) {
+    } else if (BITS == 4 && warp < 2 + kEpiWarps + 4) {
         // ------------------------------------------------------------ nibble unpack
         const int ut = threadIdx.x - kThreadsW8;         // 0..127
-        int stage = 0;
-        uint32_t phase = 0;
+        int ps = 0, ws = 0;
+        uint32_t pph = 0, wph = 0;
         bool ok = true;
         for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
             for (int kb = 0; kb < k_blocks; ++kb) {
-                ok = mbar_wait(smem_u32(&s_full_tma[stage]), phase, abort_flag, p.watchdog, kWdUnpackFull);
-                if (ok) ok = mbar_wait(smem_u32(&s_empty[stage]), phase ^ 1u, abort_flag, p.watchdog, kWdUnpackEmpty);
+                ok = mbar_wait(smem_u32(&s_full_p[ps]), pph, abort_flag, p.watchdog, kWdUnpackFull);
+                if (ok) ok = mbar_wait(smem_u32(&s_empty_w8[ws]), wph ^ 1u, abort_flag, p.watchdog, kWdUnpackEmpty);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
-                const uint8_t* src = gen_base + (smem_p - base) + stage * pk_bytes;
-                uint8_t* dst = gen_base + (smem_w - base) + stage * w_bytes;
+                const uint8_t* src = gen_base + (smem_p - base) + ps * pk_bytes;
+                uint8_t* dst = gen_base + (smem_w - base) + ws * w_bytes;
+                uint4 pk[4];
+#pragma unroll
+                for (int it = 0; it < 4; ++it) pk[it] = *reinterpret_cast<const uint4*>(src + (it * 128 + ut) * 16);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&s_empty_p[ps]));   // packed stage read: give it back
 #pragma unroll
                 for (int it = 0; it < 4; ++it) {
                     const int idx = it * 128 + ut;       // 16-byte packed chunk index
                     const int row = idx >> 2;
                     const int cp = idx & 3;
-                    const uint4 pk = *reinterpret_cast<const uint4*>(src + idx * 16);
-                    const uint32_t w[4] = {pk.x, pk.y, pk.z, pk.w};
+                    const uint32_t w[4] = {pk[it].x, pk[it].y, pk[it].z, pk[it].w};
                     uint32_t o[8];
 #pragma unroll
                     for (int q = 0; q < 4; ++q) {
@@ -384,8 +408,41 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                 }
                 fence_proxy_async_smem();                // generic-proxy writes -> visible to the tensor core
                 __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&s_full_w8[stage]));
-                if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+                if (lane == 0) mbar_arrive(smem_u32(&s_full_w8[ws]));
+                if (++ps == p.stages_p) { ps = 0; pph ^= 1u; }
+                if (++ws == p.stages_w) { ws = 0; wph ^= 1u; }
+            }
+        }
+    } else if (BITS == 4) {
+        // ------------------------------------------------- TMA producer, packed weights
+        if (lane == 0) {
+            int ps = 0;
+            uint32_t pph = 0;
+            bool ok = true;
+            int issued = 0;
+            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+                const int n0 = (tile / p.m_tiles) * kTileN;
+                for (int kb = 0; kb < k_blocks; ++kb) {
+                    ok = mbar_wait(smem_u32(&s_empty_p[ps]), pph ^ 1u, abort_flag, p.watchdog, kWdProducer);
+                    if (!ok) break;
+                    const uint32_t bar = smem_u32(&s_full_p[ps]);
+                    mbar_arrive_expect_tx(bar, pk_bytes);
+                    tma_load_2d(smem_p + ps * pk_bytes, &map_w, kb * (kBlockK / 2), n0, bar);
+                    ++issued;
+                    if (++ps == p.stages_p) { ps = 0; pph ^= 1u; }
+                }
+            }
+            if (!ok) {
+                int back = issued < p.stages_p ? issued : p.stages_p;
+                int sidx = ps;
+                uint32_t ph = pph;
+                for (int i = 0; i < back; ++i) {
+                    if (--sidx < 0) { sidx = p.stages_p - 1; ph ^= 1u; }
+                    const uint64_t t0 = global_timer_ns();
+                    while (!mbar_try_wait(smem_u32(&s_full_p[sidx]), ph)) {
+                        if (global_timer_ns() - t0 > kWaitLimitNs) { atomicOr(p.watchdog, kWdDrain); break; }
+                    }
+                }
             }
         }
     }
@@ -477,6 +534,7 @@ fq_status launch_gemm_tcgen05(const int8_t* a8, int64_t M, const Weights& W, int
     p.M = M; p.N = W.N; p.K = W.K;
     const int m_tiles = (int)((M + 255) / 256);
     int bt = (int)(((M + m_tiles - 1) / m_tiles + 15) / 16 * 16);
+    if (const char* e = getenv("FQ_DEBUG_BT")) bt = atoi(e);   // TEMP experiment
     p.bt = bt;
     p.m_tiles = (int)((M + bt - 1) / bt);
     p.n_tiles = (int)((W.N + kTileN - 1) / kTileN);
@@ -488,14 +546,29 @@ fq_status launch_gemm_tcgen05(const int8_t* a8, int64_t M, const Weights& W, int
     if (!p.watchdog) return FQ_ERR_CUDA;
     p.tmem_cols = next_pow2(kAccStages * bt);
 
-    const size_t stage_bytes = (size_t)bt * kBlockK + kTileN * kBlockK + (W.bits == 4 ? kTileN * kBlockK / 2 : 0);
     const size_t epi_bytes = (size_t)kEpiWarps * kEpiStageBytes;
     const size_t budget = 227 * 1024 - 1024 /*alignment slack*/ - 1024 /*static*/ - epi_bytes;
-    int stages = (int)(budget / stage_bytes);
-    if (stages > kMaxStages) stages = kMaxStages;
-    if (stages < 2) return FQ_ERR_UNSUPPORTED;
-    p.stages = stages;
-    const size_t smem = stage_bytes * stages + epi_bytes + 1024;
+    const size_t a_bytes = (size_t)bt * kBlockK, w_bytes = (size_t)kTileN * kBlockK, pk_bytes = w_bytes / 2;
+    size_t smem;
+    if (W.bits == 4) {
+        p.stages_w = 3;
+        int sa = (int)((budget - p.stages_w * w_bytes - 2 * pk_bytes) / a_bytes);
+        if (sa > 6) sa = 6;
+        if (sa < 2) return FQ_ERR_UNSUPPORTED;
+        int sp = (int)((budget - p.stages_w * w_bytes - sa * a_bytes) / pk_bytes);
+        if (sp > kMaxStages) sp = kMaxStages;
+        p.stages = sa;
+        p.stages_p = sp;
+        smem = sa * a_bytes + p.stages_w * w_bytes + sp * pk_bytes + epi_bytes + 1024;
+    } else {
+        int stages = (int)(budget / (a_bytes + w_bytes));
+        if (stages > kMaxStages) stages = kMaxStages;
+        if (stages < 2) return FQ_ERR_UNSUPPORTED;
+        p.stages = stages;
+        p.stages_p = 0;
+        p.stages_w = 0;
+        smem = (a_bytes + w_bytes) * stages + epi_bytes + 1024;
+    }
 
     CUtensorMap map_a;
     if (!encode_2d(&map_a, a8, (uint64_t)W.K, (uint64_t)M, kBlockK, (uint32_t)bt, true)) return FQ_ERR_CUDA;
