@@ -128,7 +128,7 @@ transform_quantize_ring_kernel(const __grid_constant__ CUtensorMap map_x, const 
     int n = 0, d = 0;
     uint32_t ph = 0;
     for (int row = first; row < rows; row += step, ++n) {
-        bool ok = mbar_wait(smem_u32(&full0[d]), ph, abort_flag, p.watchdog, 0x100u);
+        bool ok = mbar_wait_warp(smem_u32(&full0[d]), ph, abort_flag, p.watchdog, 0x100u);
 
         float v[E];
         const uint8_t* slot = gen + slots_off + (size_t)(group * p.depth + d) * p.slot_bytes + xoff0;

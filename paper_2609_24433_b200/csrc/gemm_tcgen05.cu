@@ -9,21 +9,24 @@
 // (coalesced), and ragged token counts (M = 50, 816, ...) are absorbed by the
 // free N dimension instead of padding a fixed 128-row tile.
 //
-// Operands.  Both are K-major with 128-byte rows in the 128B-swizzled shared
-// memory layout.  Activations arrive as int8 by TMA.  8-bit weights arrive the
-// same way.  4-bit weights stay packed in HBM and in the TMA stage; four unpack
-// warps expand each 128 x 64-byte packed tile into a 128 x 128-byte int8 tile
-// holding 16*code (nibble moved to the high half of the byte: no sign extension
-// needed), so the accumulator is an exact multiple of 2^acc_shift that the
-// epilogue shifts away.
+// Operands.  Activations (the MMA's B operand) arrive as int8 by TMA, K-major with
+// 128-byte rows in the 128B-swizzled shared memory layout.  8-bit weights (the A
+// operand) arrive the same way.  4-bit weights stay packed in HBM and in their TMA
+// stage; four unpack warps expand each row's 64 packed bytes to 128 int8 holding
+// 16*code (nibble moved to the high half of the byte: no sign extension needed) and
+// write them with tcgen05.st straight into TENSOR MEMORY, from where the MMA takes
+// its A operand -- the unpacked weights never touch shared memory, which is the
+// bandwidth that bounds this kernel.  The accumulator is then an exact multiple of
+// 2^acc_shift that the epilogue folds into the scale.
 //
 // Roles (warp specialised, persistent over tiles):
 //   warp 0       TMA producer          warp 1  MMA issuer + TMEM allocator
 //   warps 2-9    epilogue (two warps per TMEM lane quadrant, alternating 16-token chunks)
-//   warps 10-13  nibble unpack, warp 14 TMA producer of packed weights (4-bit weights only)
+//   warps 10-17  nibble unpack (two sets of four, alternating k-blocks), warp 18 TMA producer
+//                of packed weights (4-bit weights only)
 // With 4-bit weights three rings are decoupled: activations (TMA -> MMA), packed weights
-// (TMA -> unpack, deep and cheap: 8 KB a stage) and unpacked weights (unpack -> MMA, 3 stages),
-// so the unpack latency sits beside, not inside, the TMA round trip.
+// (TMA -> unpack, deep and cheap: 8 KB a stage) and unpacked weights (unpack -> MMA, 3 stages
+// of 32 TMEM columns), so the unpack latency sits beside, not inside, the TMA round trip.
 // bf16 outputs leave through a per-warp 1 KB shared-memory transposer so that global
 // stores are 16-byte vectors of 8 consecutive channels; fp32/raw outputs store directly.
 // Every mbarrier wait is bounded by wall-clock time; on expiry the CTA records a
@@ -62,9 +65,14 @@ constexpr int kAccStages = 2;
 constexpr int kEpiWarps = 8;
 constexpr int kEpiStageBytes = 16 * 64;   // 16 tokens x 32 channels of bf16 per epilogue warp
 constexpr int kThreadsW8 = 32 * (2 + kEpiWarps);
-constexpr int kThreadsW4 = kThreadsW8 + 128 + 32;
-constexpr int kMaxStagesW = 4;
+constexpr int kUnpackSets = 2;          // sets of four unpack warps, one TMEM lane quadrant each
+constexpr int kThreadsW4 = kThreadsW8 + kUnpackSets * 128 + 32;
+constexpr int kMaxStagesW = 8;
+constexpr int kStagesW = 3;            // unpacked-weight stages in tensor memory (4-bit weights)
+constexpr int kColsW = kBlockK / 4;     // TMEM columns of one unpacked k-block (128 int8 per lane)
 constexpr int kMaxStages = 8;
+constexpr int kMaxStagesP = 16;
+constexpr int kProducerLanes = 1;      // threads that issue TMA copies, k-blocks dealt round-robin
 
 struct Params {
     int64_t M, N, K;
@@ -107,6 +115,22 @@ __device__ __forceinline__ void mma_i8(uint32_t d_tmem, uint64_t a_desc, uint64_
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
+// A operand from tensor memory (lane = row, 4 int8 per 32-bit column), B from shared memory.
+__device__ __forceinline__ void mma_i8_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t* r) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                 ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void mma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
                  : "memory");
@@ -137,6 +161,13 @@ __device__ __forceinline__ uint32_t instr_desc_i8(int n) {
     return (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTileN >> 4) << 24);
 }
 
+// After an expired wait a producer lets the copies it already issued land before the CTA gives its
+// shared memory back: they complete within microseconds, so a bounded pause suffices.
+__device__ __forceinline__ void drain_after_abort() {
+    const uint64_t t0 = global_timer_ns();
+    while (global_timer_ns() - t0 < 100000ull) __nanosleep(1000);
+}
+
 enum : uint32_t {
     kWdProducer = 1u, kWdMmaFull = 2u, kWdMmaAcc = 4u, kWdEpilogue = 8u, kWdUnpackFull = 16u,
     kWdUnpackEmpty = 32u, kWdDrain = 64u
@@ -149,8 +180,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t s_full_tma[kMaxStages];     // activations (+ int8 weights) landed
     __shared__ uint64_t s_empty[kMaxStages];        // ... consumed by the MMAs
-    __shared__ uint64_t s_full_p[kMaxStages];       // packed weights landed
-    __shared__ uint64_t s_empty_p[kMaxStages];      // ... read by the unpack warps
+    __shared__ uint64_t s_full_p[kMaxStagesP];      // packed weights landed
+    __shared__ uint64_t s_empty_p[kMaxStagesP];     // ... read by the unpack warps
     __shared__ uint64_t s_full_w8[kMaxStagesW];     // unpacked weights written
     __shared__ uint64_t s_empty_w8[kMaxStagesW];    // ... consumed by the MMAs
     __shared__ uint64_t s_acc_full[kAccStages];
@@ -169,7 +200,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     const uint32_t pk_bytes = kTileN * kBlockK / 2;
     const uint32_t smem_a = base;
     const uint32_t smem_w = smem_a + (uint32_t)p.stages * a_bytes;
-    const uint32_t smem_p = smem_w + (uint32_t)(BITS == 4 ? p.stages_w : p.stages) * w_bytes;
+    const uint32_t smem_p = smem_w + (BITS == 4 ? 0u : (uint32_t)p.stages * w_bytes);
     const uint32_t smem_e = smem_p + (BITS == 4 ? (uint32_t)p.stages_p * pk_bytes : 0u);
     uint8_t* gen_base = smem_raw + (base - smem_u32(smem_raw));   // generic pointer to `base`
 
@@ -207,40 +238,27 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
-        if (lane == 0) {
-            int stage = 0;
-            uint32_t phase = 0;
+        // One thread sustains only about one bulk-tensor copy per ~400 cycles (measured), so the
+        // k-blocks are dealt round-robin to kProducerLanes lanes, each waiting on its own stages.
+        if (lane < kProducerLanes) {
             const uint32_t tx = a_bytes + (BITS == 4 ? 0u : w_bytes);
+            const int total_kb = ((num_tiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1) * k_blocks;
             bool ok = true;
-            int issued = 0;
-            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+            for (int n = lane; n < total_kb; n += kProducerLanes) {
+                const int tile = (int)blockIdx.x + (n / k_blocks) * (int)gridDim.x;
+                const int kb = n % k_blocks;
                 const int n0 = (tile / p.m_tiles) * kTileN;
                 const int t0 = (tile % p.m_tiles) * p.bt;
-                for (int kb = 0; kb < k_blocks; ++kb) {
-                    ok = mbar_wait(smem_u32(&s_empty[stage]), phase ^ 1u, abort_flag, p.watchdog, kWdProducer);
-                    if (!ok) break;
-                    const uint32_t bar = smem_u32(&s_full_tma[stage]);
-                    mbar_arrive_expect_tx(bar, tx);
-                    tma_load_2d(smem_a + stage * a_bytes, &map_a, kb * kBlockK, t0, bar);
-                    if (BITS == 8) tma_load_2d(smem_w + stage * w_bytes, &map_w, kb * kBlockK, n0, bar);
-                    ++issued;
-                    if (++stage == p.stages) { stage = 0; phase ^= 1u; }
-                }
+                const int stage = n % p.stages;
+                const uint32_t phase = (uint32_t)((n / p.stages) & 1);
+                ok = mbar_wait(smem_u32(&s_empty[stage]), phase ^ 1u, abort_flag, p.watchdog, kWdProducer);
+                if (!ok) break;
+                const uint32_t bar = smem_u32(&s_full_tma[stage]);
+                mbar_arrive_expect_tx(bar, tx);
+                tma_load_2d(smem_a + stage * a_bytes, &map_a, kb * kBlockK, t0, bar);
+                if (BITS == 8) tma_load_2d(smem_w + stage * w_bytes, &map_w, kb * kBlockK, n0, bar);
             }
-            if (!ok) {
-                // Winding down after an expired wait: let the copies already issued land
-                // before the CTA gives its shared memory back.
-                int back = issued < p.stages ? issued : p.stages;
-                int s = stage;
-                uint32_t ph = phase;
-                for (int i = 0; i < back; ++i) {
-                    if (--s < 0) { s = p.stages - 1; ph ^= 1u; }
-                    const uint64_t t0 = global_timer_ns();
-                    while (!mbar_try_wait(smem_u32(&s_full_tma[s]), ph)) {
-                        if (global_timer_ns() - t0 > kWaitLimitNs) { atomicOr(p.watchdog, kWdDrain); break; }
-                    }
-                }
-            }
+            if (!ok) drain_after_abort();
         }
     } else if (warp == 1) {
         // -------------------------------------------------------------- MMA issuer
@@ -262,13 +280,21 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                         ok = mbar_wait(smem_u32(&s_full_w8[wstage]), wphase, abort_flag, p.watchdog, kWdMmaFull);
                     if (!ok) break;
                     tc_fence_after();
-                    const uint64_t wdesc = smem_desc_sw128(smem_w + (BITS == 4 ? wstage : stage) * w_bytes);
                     const uint64_t adesc = smem_desc_sw128(smem_a + stage * a_bytes);
+                    if (BITS == 4) {
+                        const uint32_t w_tmem = tmem_base + (uint32_t)(kAccStages * p.bt + wstage * kColsW);
 #pragma unroll
-                    for (int k = 0; k < kBlockK / kMmaK; ++k) {
-                        // step 32 bytes along K inside the swizzle atom: +2 in 16-byte address units
-                        mma_i8(d_tmem, wdesc + (uint64_t)(2 * k), adesc + (uint64_t)(2 * k), idesc,
-                               (kb | k) != 0 ? 1u : 0u);
+                        for (int k = 0; k < kBlockK / kMmaK; ++k)   // 32 int8 of K = 8 TMEM columns per MMA
+                            mma_i8_ts(d_tmem, w_tmem + (uint32_t)(8 * k), adesc + (uint64_t)(2 * k), idesc,
+                                      (kb | k) != 0 ? 1u : 0u);
+                    } else {
+                        const uint64_t wdesc = smem_desc_sw128(smem_w + stage * w_bytes);
+#pragma unroll
+                        for (int k = 0; k < kBlockK / kMmaK; ++k) {
+                            // step 32 bytes along K inside the swizzle atom: +2 in 16-byte address units
+                            mma_i8(d_tmem, wdesc + (uint64_t)(2 * k), adesc + (uint64_t)(2 * k), idesc,
+                                   (kb | k) != 0 ? 1u : 0u);
+                        }
                     }
                     mma_commit(smem_u32(&s_empty[stage]));          // frees this stage when the MMAs retire
                     if (++stage == p.stages) { stage = 0; phase ^= 1u; }
@@ -302,8 +328,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                 sw = __ldg(p.w_scale + j) * unshift;     // (float)acc * 2^-shift is exact: fold the shift here
                 bj = __ldg(p.bias + j);
             }
-            ok = mbar_wait(smem_u32(&s_acc_full[acc_stage]), acc_phase, abort_flag, p.watchdog, kWdEpilogue);
-            ok = __all_sync(0xffffffffu, ok);
+            ok = mbar_wait_warp_relaxed(smem_u32(&s_acc_full[acc_stage]), acc_phase, abort_flag, p.watchdog, kWdEpilogue);
             if (!ok) break;
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc_stage * p.bt);
@@ -368,82 +393,71 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             if (lane == 0) mbar_arrive(smem_u32(&s_acc_empty[acc_stage]));
             if (++acc_stage == kAccStages) { acc_stage = 0; acc_phase ^= 1u; }
         }
-    } else if (BITS == 4 && warp < 2 + kEpiWarps + 4) {
+    } else if (BITS == 4 && warp < 2 + kEpiWarps + 4 * kUnpackSets) {
         // ------------------------------------------------------------ nibble unpack
-        const int ut = threadIdx.x - kThreadsW8;         // 0..127
-        int ps = 0, ws = 0;
-        uint32_t pph = 0, wph = 0;
+        // A thread owns one weight row (= one TMEM lane of its warp's quadrant).  The packed tile is
+        // 128 rows x 64 bytes with the 64-byte TMA swizzle: 16-byte chunk c of row r sits at
+        // chunk c ^ ((r >> 1) & 3), which makes the row-per-thread reads bank-conflict free.
+        const int row = (warp & 3) * 32 + lane;
+        const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
+        const int swz = (row >> 1) & 3;
+        // Set `uset` takes the k-blocks whose running index n is congruent to it modulo kUnpackSets,
+        // so two k-blocks are in flight per quadrant and one set's store latency hides behind the other.
+        const int uset = (warp - 2 - kEpiWarps) >> 2;
+        const int total_kb = ((num_tiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1) * k_blocks;
         bool ok = true;
-        for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-            for (int kb = 0; kb < k_blocks; ++kb) {
-                ok = mbar_wait(smem_u32(&s_full_p[ps]), pph, abort_flag, p.watchdog, kWdUnpackFull);
-                if (ok) ok = mbar_wait(smem_u32(&s_empty_w8[ws]), wph ^ 1u, abort_flag, p.watchdog, kWdUnpackEmpty);
-                ok = __all_sync(0xffffffffu, ok);
+        for (int n = uset; n < total_kb && ok; n += kUnpackSets) {
+            {
+                const int ps = n % p.stages_p, ws = n % p.stages_w;
+                const uint32_t pph = (uint32_t)((n / p.stages_p) & 1), wph = (uint32_t)((n / p.stages_w) & 1);
+                ok = mbar_wait_warp(smem_u32(&s_full_p[ps]), pph, abort_flag, p.watchdog, kWdUnpackFull);
+                if (ok) ok = mbar_wait_warp(smem_u32(&s_empty_w8[ws]), wph ^ 1u, abort_flag, p.watchdog, kWdUnpackEmpty);
                 if (!ok) break;
-                const uint8_t* src = gen_base + (smem_p - base) + ps * pk_bytes;
-                uint8_t* dst = gen_base + (smem_w - base) + ws * w_bytes;
+                tc_fence_after();
+                const uint8_t* src = gen_base + (smem_p - base) + ps * pk_bytes + row * 64;
                 uint4 pk[4];
 #pragma unroll
-                for (int it = 0; it < 4; ++it) pk[it] = *reinterpret_cast<const uint4*>(src + (it * 128 + ut) * 16);
+                for (int c = 0; c < 4; ++c) pk[c] = *reinterpret_cast<const uint4*>(src + ((c ^ swz) << 4));
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&s_empty_p[ps]));   // packed stage read: give it back
+                const uint32_t w_tmem = tmem_base + lane_addr + (uint32_t)(kAccStages * p.bt + ws * kColsW);
 #pragma unroll
-                for (int it = 0; it < 4; ++it) {
-                    const int idx = it * 128 + ut;       // 16-byte packed chunk index
-                    const int row = idx >> 2;
-                    const int cp = idx & 3;
-                    const uint32_t w[4] = {pk[it].x, pk[it].y, pk[it].z, pk[it].w};
+                for (int c = 0; c < 4; ++c) {            // 32 codes -> 32 int8 = 8 TMEM columns
+                    const uint32_t w[4] = {pk[c].x, pk[c].y, pk[c].z, pk[c].w};
                     uint32_t o[8];
 #pragma unroll
                     for (int q = 0; q < 4; ++q) {
-                        const uint32_t lo = (w[q] << 4) & 0xF0F0F0F0u;
-                        const uint32_t hi = w[q] & 0xF0F0F0F0u;
+                        const uint32_t lo = (w[q] << 4) & 0xF0F0F0F0u;   // even channels, 16*code
+                        const uint32_t hi = w[q] & 0xF0F0F0F0u;          // odd channels
                         o[2 * q + 0] = __byte_perm(lo, hi, 0x5140);
                         o[2 * q + 1] = __byte_perm(lo, hi, 0x7362);
                     }
-                    uint8_t* drow = dst + row * 128;
-                    const int sw = row & 7;
-                    *reinterpret_cast<uint4*>(drow + (((2 * cp) ^ sw) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
-                    *reinterpret_cast<uint4*>(drow + (((2 * cp + 1) ^ sw) << 4)) = make_uint4(o[4], o[5], o[6], o[7]);
+                    tmem_st8(w_tmem + (uint32_t)(8 * c), o);
                 }
-                fence_proxy_async_smem();                // generic-proxy writes -> visible to the tensor core
+                tmem_st_wait();
+                tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&s_full_w8[ws]));
-                if (++ps == p.stages_p) { ps = 0; pph ^= 1u; }
-                if (++ws == p.stages_w) { ws = 0; wph ^= 1u; }
             }
         }
     } else if (BITS == 4) {
         // ------------------------------------------------- TMA producer, packed weights
-        if (lane == 0) {
-            int ps = 0;
-            uint32_t pph = 0;
+        if (lane < kProducerLanes) {
+            const int total_kb = ((num_tiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1) * k_blocks;
             bool ok = true;
-            int issued = 0;
-            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+            for (int n = lane; n < total_kb; n += kProducerLanes) {
+                const int tile = (int)blockIdx.x + (n / k_blocks) * (int)gridDim.x;
+                const int kb = n % k_blocks;
                 const int n0 = (tile / p.m_tiles) * kTileN;
-                for (int kb = 0; kb < k_blocks; ++kb) {
-                    ok = mbar_wait(smem_u32(&s_empty_p[ps]), pph ^ 1u, abort_flag, p.watchdog, kWdProducer);
-                    if (!ok) break;
-                    const uint32_t bar = smem_u32(&s_full_p[ps]);
-                    mbar_arrive_expect_tx(bar, pk_bytes);
-                    tma_load_2d(smem_p + ps * pk_bytes, &map_w, kb * (kBlockK / 2), n0, bar);
-                    ++issued;
-                    if (++ps == p.stages_p) { ps = 0; pph ^= 1u; }
-                }
+                const int ps = n % p.stages_p;
+                const uint32_t pph = (uint32_t)((n / p.stages_p) & 1);
+                ok = mbar_wait(smem_u32(&s_empty_p[ps]), pph ^ 1u, abort_flag, p.watchdog, kWdProducer);
+                if (!ok) break;
+                const uint32_t bar = smem_u32(&s_full_p[ps]);
+                mbar_arrive_expect_tx(bar, pk_bytes);
+                tma_load_2d(smem_p + ps * pk_bytes, &map_w, kb * (kBlockK / 2), n0, bar);
             }
-            if (!ok) {
-                int back = issued < p.stages_p ? issued : p.stages_p;
-                int sidx = ps;
-                uint32_t ph = pph;
-                for (int i = 0; i < back; ++i) {
-                    if (--sidx < 0) { sidx = p.stages_p - 1; ph ^= 1u; }
-                    const uint64_t t0 = global_timer_ns();
-                    while (!mbar_try_wait(smem_u32(&s_full_p[sidx]), ph)) {
-                        if (global_timer_ns() - t0 > kWaitLimitNs) { atomicOr(p.watchdog, kWdDrain); break; }
-                    }
-                }
-            }
+            if (!ok) drain_after_abort();
         }
     }
 
@@ -477,7 +491,7 @@ EncodeTiledFn encode_fn() {
 
 // 2-D byte tensor [rows, row_bytes] (row pitch = row_bytes), box [box_rows, box_bytes].
 bool encode_2d(CUtensorMap* map, const void* ptr, uint64_t row_bytes, uint64_t rows, uint32_t box_bytes,
-               uint32_t box_rows, bool swizzle128) {
+               uint32_t box_rows, CUtensorMapSwizzle swizzle) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
     const cuuint64_t dims[2] = {row_bytes, rows};
@@ -485,7 +499,7 @@ bool encode_2d(CUtensorMap* map, const void* ptr, uint64_t row_bytes, uint64_t r
     const cuuint32_t box[2] = {box_bytes, box_rows};
     const cuuint32_t estr[2] = {1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(ptr), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle,
               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -518,8 +532,10 @@ fq_status build_weight_tmap(Weights& W) {
     W.tmap_valid = false;
     if (W.N == 0) return FQ_OK;
     const bool ok = W.bits == 4
-                        ? encode_2d(&W.tmap, W.codes, (uint64_t)W.K / 2, (uint64_t)W.N, kBlockK / 2, kTileN, false)
-                        : encode_2d(&W.tmap, W.codes, (uint64_t)W.K, (uint64_t)W.N, kBlockK, kTileN, true);
+                        ? encode_2d(&W.tmap, W.codes, (uint64_t)W.K / 2, (uint64_t)W.N, kBlockK / 2, kTileN,
+                                    CU_TENSOR_MAP_SWIZZLE_64B)
+                        : encode_2d(&W.tmap, W.codes, (uint64_t)W.K, (uint64_t)W.N, kBlockK, kTileN,
+                                    CU_TENSOR_MAP_SWIZZLE_128B);
     if (!ok) return FQ_ERR_CUDA;
     W.tmap_valid = true;
     return FQ_OK;
@@ -532,7 +548,10 @@ fq_status launch_gemm_tcgen05(const int8_t* a8, int64_t M, const Weights& W, int
 
     Params p{};
     p.M = M; p.N = W.N; p.K = W.K;
-    const int m_tiles = (int)((M + 255) / 256);
+    // Token tile: as large as TMEM allows (two accumulator stages, plus the unpacked-weight ring
+    // for 4-bit weights: 2*bt + 3*32 <= 512 columns), split evenly so ragged M wastes little.
+    const int bt_max = W.bits == 4 ? 208 : 256;
+    const int m_tiles = (int)((M + bt_max - 1) / bt_max);
     int bt = (int)(((M + m_tiles - 1) / m_tiles + 15) / 16 * 16);
     if (const char* e = getenv("FQ_DEBUG_BT")) bt = atoi(e);   // TEMP experiment
     p.bt = bt;
@@ -544,22 +563,27 @@ fq_status launch_gemm_tcgen05(const int8_t* a8, int64_t M, const Weights& W, int
     p.out = out;
     p.watchdog = watchdog_device_ptr();
     if (!p.watchdog) return FQ_ERR_CUDA;
-    p.tmem_cols = next_pow2(kAccStages * bt);
+    // 4-bit weights: every TMEM column the accumulators leave free becomes unpacked-weight ring
+    int stages_w = W.bits == 4 ? (512 - kAccStages * bt) / kColsW : 0;
+    if (stages_w > kMaxStagesW) stages_w = kMaxStagesW;
+    p.tmem_cols = next_pow2(kAccStages * bt + stages_w * kColsW);
 
     const size_t epi_bytes = (size_t)kEpiWarps * kEpiStageBytes;
     const size_t budget = 227 * 1024 - 1024 /*alignment slack*/ - 1024 /*static*/ - epi_bytes;
     const size_t a_bytes = (size_t)bt * kBlockK, w_bytes = (size_t)kTileN * kBlockK, pk_bytes = w_bytes / 2;
     size_t smem;
     if (W.bits == 4) {
-        p.stages_w = 3;
-        int sa = (int)((budget - p.stages_w * w_bytes - 2 * pk_bytes) / a_bytes);
-        if (sa > 6) sa = 6;
+        p.stages_w = stages_w;
+        // Both TMA rings need the same look-ahead in k-blocks (their latencies are the same):
+        // split the budget evenly, then give the remainder to the cheaper packed ring.
+        int sa = (int)(budget / (a_bytes + pk_bytes));
+        if (sa > kMaxStages) sa = kMaxStages;
         if (sa < 2) return FQ_ERR_UNSUPPORTED;
-        int sp = (int)((budget - p.stages_w * w_bytes - sa * a_bytes) / pk_bytes);
-        if (sp > kMaxStages) sp = kMaxStages;
+        int sp = (int)((budget - sa * a_bytes) / pk_bytes);
+        if (sp > kMaxStagesP) sp = kMaxStagesP;
         p.stages = sa;
         p.stages_p = sp;
-        smem = sa * a_bytes + p.stages_w * w_bytes + sp * pk_bytes + epi_bytes + 1024;
+        smem = sa * a_bytes + sp * pk_bytes + epi_bytes + 1024;
     } else {
         int stages = (int)(budget / (a_bytes + w_bytes));
         if (stages > kMaxStages) stages = kMaxStages;
@@ -571,7 +595,8 @@ fq_status launch_gemm_tcgen05(const int8_t* a8, int64_t M, const Weights& W, int
     }
 
     CUtensorMap map_a;
-    if (!encode_2d(&map_a, a8, (uint64_t)W.K, (uint64_t)M, kBlockK, (uint32_t)bt, true)) return FQ_ERR_CUDA;
+    if (!encode_2d(&map_a, a8, (uint64_t)W.K, (uint64_t)M, kBlockK, (uint32_t)bt, CU_TENSOR_MAP_SWIZZLE_128B))
+        return FQ_ERR_CUDA;
 
     int dev = 0, sms = 148;
     cudaGetDevice(&dev);

@@ -30,6 +30,19 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
+// Same, but the thread may stay suspended for up to `hint_ns` before the instruction returns:
+// long waits then cost far fewer issue slots (and less power) than a tight polling loop.
+__device__ __forceinline__ bool mbar_try_wait_hint(uint32_t bar, uint32_t parity, uint32_t hint_ns) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.b32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity), "r"(hint_ns)
+        : "memory");
+    return ok != 0;
+}
 __device__ __forceinline__ uint64_t global_timer_ns() {
     uint64_t t;
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
@@ -59,6 +72,35 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     for (int i = 0; i < 64; ++i)
         if (mbar_try_wait(bar, parity)) return true;
     return mbar_wait_slow(bar, parity, abort_flag, watchdog, code);
+}
+// Wait for latency-tolerant roles (epilogue): lane 0 polls with a short sleep between tries so that
+// an idle warp does not compete for issue slots with the warps feeding the tensor core.
+__device__ __forceinline__ bool mbar_wait_warp_relaxed(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                                       uint32_t* watchdog, uint32_t code) {
+    int ok = 1;
+    if ((threadIdx.x & 31) == 0) {
+        const uint64_t t0 = global_timer_ns();
+        for (uint32_t spin = 1; !mbar_try_wait(bar, parity); ++spin) {
+            __nanosleep(200);
+            if ((spin & 0x3f) == 0) {
+                if (*abort_flag) { ok = 0; break; }
+                if (global_timer_ns() - t0 > kWaitLimitNs) {
+                    *abort_flag = 1;
+                    atomicOr(watchdog, code);
+                    ok = 0;
+                    break;
+                }
+            }
+        }
+    }
+    return __shfl_sync(0xffffffffu, ok, 0) != 0;
+}
+// Warp-collective wait: lane 0 waits, the result is broadcast (one poller per warp instead of 32).
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                               uint32_t* watchdog, uint32_t code) {
+    int ok = 1;
+    if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity, abort_flag, watchdog, code) ? 1 : 0;
+    return __shfl_sync(0xffffffffu, ok, 0) != 0;
 }
 
 __device__ __forceinline__ void fence_proxy_async_smem() {
