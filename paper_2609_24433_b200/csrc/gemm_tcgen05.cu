@@ -32,7 +32,6 @@
 // Every mbarrier wait is bounded by wall-clock time; on expiry the CTA records a
 // code in the watchdog word, stops issuing work, and still frees its TMEM.
 #include <cuda_bf16.h>
-#include <stdlib.h>
 
 #include "fq_common.cuh"
 #include "ptx_sm100.cuh"
@@ -64,9 +63,10 @@ constexpr int kMmaK = 32;            // K per tcgen05.mma.kind::i8
 constexpr int kAccStages = 2;
 constexpr int kEpiWarps = 8;
 constexpr int kEpiStageBytes = 16 * 64;   // 16 tokens x 32 channels of bf16 per epilogue warp
-constexpr int kThreadsW8 = 32 * (2 + kEpiWarps);
+constexpr int kThreadsW8 = 32 * (2 + kEpiWarps + 1);   // + one warp: TMA producer of int8 weights
+constexpr int kFirstUnpackWarp = 2 + kEpiWarps;
 constexpr int kUnpackSets = 2;          // sets of four unpack warps, one TMEM lane quadrant each
-constexpr int kThreadsW4 = kThreadsW8 + kUnpackSets * 128 + 32;
+constexpr int kThreadsW4 = 32 * (2 + kEpiWarps) + kUnpackSets * 128 + 32;
 constexpr int kMaxStagesW = 8;
 constexpr int kStagesW = 3;            // unpacked-weight stages in tensor memory (4-bit weights)
 constexpr int kColsW = kBlockK / 4;     // TMEM columns of one unpacked k-block (128 int8 per lane)
@@ -95,45 +95,122 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
         ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(bar)
         : "memory");
 }
+// ---- CTA-pair (cta_group::2) helpers -----------------------------------------------------
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// Arrive on the barrier at the same shared-memory offset in CTA `rank` of the cluster.
+__device__ __forceinline__ void mbar_arrive_cta(uint32_t bar, uint32_t rank) {
+    asm volatile(
+        "{\n\t.reg .b32 ra;\n\t"
+        "mapa.shared::cluster.u32 ra, %0, %1;\n\t"
+        "mbarrier.arrive.shared::cluster.b64 _, [ra];\n\t}"
+        ::"r"(bar), "r"(rank)
+        : "memory");
+}
+// Pair variant of the tiled load: issued by both CTAs into their own shared memory, but the
+// bytes are counted on the barrier of the pair's even CTA (address with the peer bit cleared).
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(bar & 0xFEFFFFFFu)
+        : "memory");
+}
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
+template <int CTAS>
 __device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols)
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    if (CTAS == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    } else {   // same warp index in both CTAs of the pair, same destination offset
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
 }
+template <int CTAS>
 __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+    if (CTAS == 1)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+    else
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
 }
+template <int CTAS>
 __device__ __forceinline__ void mma_i8(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
                                        uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-        : "memory");
+    if (CTAS == 1)
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "setp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+            ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+            : "memory");
+    else
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "setp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::2.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+            ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+            : "memory");
 }
 // A operand from tensor memory (lane = row, 4 int8 per 32-bit column), B from shared memory.
+template <int CTAS>
 __device__ __forceinline__ void mma_i8_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
                                           uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::i8 [%0], [%1], %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
-        : "memory");
+    if (CTAS == 1)
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "setp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::i8 [%0], [%1], %2, %3, p;\n\t}"
+            ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+            : "memory");
+    else
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "setp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::2.kind::i8 [%0], [%1], %2, %3, p;\n\t}"
+            ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+            : "memory");
 }
 __device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t* r) {
     asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
                  ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
                  : "memory");
 }
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+          "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]),
+          "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]),
+          "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+        : "memory");
+}
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+// Arrive on `bar` once every MMA issued so far by this thread has retired; for a CTA pair the
+// arrival is delivered to the barrier at that offset in BOTH CTAs.
+template <int CTAS>
 __device__ __forceinline__ void mma_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
-                 : "memory");
+    if (CTAS == 1) {
+        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
+                     : "memory");
+    } else {
+        const uint16_t mask = 3;
+        asm volatile(
+            "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+            ::"r"(bar), "h"(mask)
+            : "memory");
+    }
 }
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* r) {
     asm volatile(
@@ -156,9 +233,9 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
     d |= (uint64_t)2 << 61;                    // 128-byte swizzle
     return d;
 }
-// Instruction descriptor: s8 x s8 -> s32, both operands K-major, M = 128, N = n.
-__device__ __forceinline__ uint32_t instr_desc_i8(int n) {
-    return (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTileN >> 4) << 24);
+// Instruction descriptor: s8 x s8 -> s32, both operands K-major, M = m (128, or 256 for a CTA pair), N = n.
+__device__ __forceinline__ uint32_t instr_desc_i8(int m, int n) {
+    return (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 
 // After an expired wait a producer lets the copies it already issued land before the CTA gives its
@@ -173,7 +250,11 @@ enum : uint32_t {
     kWdUnpackEmpty = 32u, kWdDrain = 64u
 };
 
-template <int BITS>
+// CTAS = 2: two CTAs of a cluster work as a pair on a 256-channel x bt-token tile (cta_group::2):
+// each loads its own 128 weight rows and HALF of the token tile, the even CTA issues the MMAs for
+// both, and every MMA reads the token halves out of both CTAs' shared memory.  This halves the
+// activation bytes each SM pulls from L2, which is what bounds the single-CTA kernel.
+template <int BITS, int CTAS>
 __global__ void __launch_bounds__(BITS == 4 ? kThreadsW4 : kThreadsW8, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_w,
                     const Params p) {
@@ -192,10 +273,13 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     volatile int* abort_flag = &s_abort;
+    const uint32_t cta_rank = CTAS == 2 ? cluster_ctarank() : 0u;
+    const bool leader = cta_rank == 0;
+    const int bt_cta = p.bt / CTAS;                 // token rows this CTA loads
 
     // carve dynamic shared memory: [A8 stages][W8 stages][packed stages][epilogue transposers], 1024-byte aligned
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t a_bytes = (uint32_t)p.bt * kBlockK;
+    const uint32_t a_bytes = (uint32_t)bt_cta * kBlockK;
     const uint32_t w_bytes = kTileN * kBlockK;
     const uint32_t pk_bytes = kTileN * kBlockK / 2;
     const uint32_t smem_a = base;
@@ -207,7 +291,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     if (threadIdx.x == 0) {
         s_abort = 0;
         for (int s = 0; s < p.stages; ++s) {
-            mbar_init(smem_u32(&s_full_tma[s]), 1);
+            mbar_init(smem_u32(&s_full_tma[s]), BITS == 8 ? 2 : 1);   // 8-bit: activation and weight producers
             mbar_init(smem_u32(&s_empty[s]), 1);
         }
         if (BITS == 4) {
@@ -216,24 +300,28 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                 mbar_init(smem_u32(&s_empty_p[s]), 4);
             }
             for (int s = 0; s < p.stages_w; ++s) {
-                mbar_init(smem_u32(&s_full_w8[s]), 4);
+                mbar_init(smem_u32(&s_full_w8[s]), 4 * CTAS);
                 mbar_init(smem_u32(&s_empty_w8[s]), 1);
             }
         }
         for (int a = 0; a < kAccStages; ++a) {
             mbar_init(smem_u32(&s_acc_full[a]), 1);
-            mbar_init(smem_u32(&s_acc_empty[a]), kEpiWarps);
+            mbar_init(smem_u32(&s_acc_empty[a]), kEpiWarps * CTAS);
         }
         fence_mbarrier_init();
         fence_proxy_async_smem();
     }
-    if (warp == 1) tmem_alloc(smem_u32(&s_tmem_base), (uint32_t)p.tmem_cols);
+    if (warp == 1) tmem_alloc<CTAS>(smem_u32(&s_tmem_base), (uint32_t)p.tmem_cols);
     tc_fence_before();
     __syncthreads();
+    if (CTAS == 2) cluster_sync_all();              // the peer's barriers exist before anyone signals them
     tc_fence_after();
     const uint32_t tmem_base = s_tmem_base;
 
+    // work units: (super-tile of 128*CTAS channels) x (token tile); one unit per CTA or CTA pair at a time
     const int num_tiles = p.m_tiles * p.n_tiles;
+    const int unit0 = (int)blockIdx.x / CTAS;
+    const int unit_step = (int)gridDim.x / CTAS;
     const int k_blocks = (int)((p.K + kBlockK - 1) / kBlockK);
 
     if (warp == 0) {
@@ -241,35 +329,39 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         // One thread sustains only about one bulk-tensor copy per ~400 cycles (measured), so the
         // k-blocks are dealt round-robin to kProducerLanes lanes, each waiting on its own stages.
         if (lane < kProducerLanes) {
-            const uint32_t tx = a_bytes + (BITS == 4 ? 0u : w_bytes);
-            const int total_kb = ((num_tiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1) * k_blocks;
+            const uint32_t tx = a_bytes;
+            const int total_kb = ((num_tiles - 1 - unit0) / unit_step + 1) * k_blocks;
             bool ok = true;
             for (int n = lane; n < total_kb; n += kProducerLanes) {
-                const int tile = (int)blockIdx.x + (n / k_blocks) * (int)gridDim.x;
+                const int tile = unit0 + (n / k_blocks) * unit_step;
                 const int kb = n % k_blocks;
-                const int n0 = (tile / p.m_tiles) * kTileN;
-                const int t0 = (tile % p.m_tiles) * p.bt;
+                const int t0 = (tile % p.m_tiles) * p.bt + (int)cta_rank * bt_cta;
                 const int stage = n % p.stages;
                 const uint32_t phase = (uint32_t)((n / p.stages) & 1);
                 ok = mbar_wait(smem_u32(&s_empty[stage]), phase ^ 1u, abort_flag, p.watchdog, kWdProducer);
                 if (!ok) break;
                 const uint32_t bar = smem_u32(&s_full_tma[stage]);
-                mbar_arrive_expect_tx(bar, tx);
-                tma_load_2d(smem_a + stage * a_bytes, &map_a, kb * kBlockK, t0, bar);
-                if (BITS == 8) tma_load_2d(smem_w + stage * w_bytes, &map_w, kb * kBlockK, n0, bar);
+                if (CTAS == 1) {
+                    mbar_arrive_expect_tx(bar, tx);
+                    tma_load_2d(smem_a + stage * a_bytes, &map_a, kb * kBlockK, t0, bar);
+                } else {
+                    // the pair's bytes are all counted on the even CTA's barrier, which it arms for both
+                    if (leader) mbar_arrive_expect_tx(bar, tx * CTAS);
+                    tma_load_2d_pair(smem_a + stage * a_bytes, &map_a, kb * kBlockK, t0, bar);
+                }
             }
             if (!ok) drain_after_abort();
         }
     } else if (warp == 1) {
         // -------------------------------------------------------------- MMA issuer
-        if (lane == 0) {
-            const uint32_t idesc = instr_desc_i8(p.bt);
+        if (lane == 0 && leader) {
+            const uint32_t idesc = instr_desc_i8(kTileN * CTAS, p.bt);
             int stage = 0, wstage = 0;
             uint32_t phase = 0, wphase = 0;
             int acc_stage = 0;
             uint32_t acc_phase = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+            for (int tile = unit0; tile < num_tiles && ok; tile += unit_step) {
                 ok = mbar_wait(smem_u32(&s_acc_empty[acc_stage]), acc_phase ^ 1u, abort_flag, p.watchdog, kWdMmaAcc);
                 if (!ok) break;
                 tc_fence_after();
@@ -285,26 +377,26 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                         const uint32_t w_tmem = tmem_base + (uint32_t)(kAccStages * p.bt + wstage * kColsW);
 #pragma unroll
                         for (int k = 0; k < kBlockK / kMmaK; ++k)   // 32 int8 of K = 8 TMEM columns per MMA
-                            mma_i8_ts(d_tmem, w_tmem + (uint32_t)(8 * k), adesc + (uint64_t)(2 * k), idesc,
+                            mma_i8_ts<CTAS>(d_tmem, w_tmem + (uint32_t)(8 * k), adesc + (uint64_t)(2 * k), idesc,
                                       (kb | k) != 0 ? 1u : 0u);
                     } else {
                         const uint64_t wdesc = smem_desc_sw128(smem_w + stage * w_bytes);
 #pragma unroll
                         for (int k = 0; k < kBlockK / kMmaK; ++k) {
                             // step 32 bytes along K inside the swizzle atom: +2 in 16-byte address units
-                            mma_i8(d_tmem, wdesc + (uint64_t)(2 * k), adesc + (uint64_t)(2 * k), idesc,
+                            mma_i8<CTAS>(d_tmem, wdesc + (uint64_t)(2 * k), adesc + (uint64_t)(2 * k), idesc,
                                    (kb | k) != 0 ? 1u : 0u);
                         }
                     }
-                    mma_commit(smem_u32(&s_empty[stage]));          // frees this stage when the MMAs retire
+                    mma_commit<CTAS>(smem_u32(&s_empty[stage]));          // frees this stage when the MMAs retire
                     if (++stage == p.stages) { stage = 0; phase ^= 1u; }
                     if (BITS == 4) {
-                        mma_commit(smem_u32(&s_empty_w8[wstage]));
+                        mma_commit<CTAS>(smem_u32(&s_empty_w8[wstage]));
                         if (++wstage == p.stages_w) { wstage = 0; wphase ^= 1u; }
                     }
                 }
                 if (!ok) break;
-                mma_commit(smem_u32(&s_acc_full[acc_stage]));        // accumulator complete
+                mma_commit<CTAS>(smem_u32(&s_acc_full[acc_stage]));        // accumulator complete
                 if (++acc_stage == kAccStages) { acc_stage = 0; acc_phase ^= 1u; }
             }
         }
@@ -318,8 +410,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         int acc_stage = 0;
         uint32_t acc_phase = 0;
         bool ok = true;
-        for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-            const int64_t jq = (int64_t)(tile / p.m_tiles) * kTileN + quad * 32;   // first channel of this warp
+        for (int tile = unit0; tile < num_tiles && ok; tile += unit_step) {
+            const int64_t jq = (int64_t)(tile / p.m_tiles) * (kTileN * CTAS) + (int64_t)cta_rank * kTileN + quad * 32;   // first channel of this warp
             const int64_t j = jq + lane;
             const int64_t t0 = (int64_t)(tile % p.m_tiles) * p.bt;
             const bool j_ok = j < p.N;
@@ -390,10 +482,38 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&s_acc_empty[acc_stage]));
+            if (lane == 0) {
+                if (CTAS == 1) mbar_arrive(smem_u32(&s_acc_empty[acc_stage]));
+                else mbar_arrive_cta(smem_u32(&s_acc_empty[acc_stage]), 0);   // the even CTA issues the MMAs
+            }
             if (++acc_stage == kAccStages) { acc_stage = 0; acc_phase ^= 1u; }
         }
-    } else if (BITS == 4 && warp < 2 + kEpiWarps + 4 * kUnpackSets) {
+    } else if (BITS == 8) {
+        // ------------------------------------------------- TMA producer, int8 weights
+        // (a thread sustains only about one bulk-tensor copy per ~400 cycles: one producer per operand)
+        if (lane == 0) {
+            const int total_kb = ((num_tiles - 1 - unit0) / unit_step + 1) * k_blocks;
+            bool ok = true;
+            for (int n = 0; n < total_kb; ++n) {
+                const int tile = unit0 + (n / k_blocks) * unit_step;
+                const int kb = n % k_blocks;
+                const int n0 = (tile / p.m_tiles) * (kTileN * CTAS) + (int)cta_rank * kTileN;
+                const int stage = n % p.stages;
+                const uint32_t phase = (uint32_t)((n / p.stages) & 1);
+                ok = mbar_wait(smem_u32(&s_empty[stage]), phase ^ 1u, abort_flag, p.watchdog, kWdProducer);
+                if (!ok) break;
+                const uint32_t bar = smem_u32(&s_full_tma[stage]);
+                if (CTAS == 1) {
+                    mbar_arrive_expect_tx(bar, w_bytes);
+                    tma_load_2d(smem_w + stage * w_bytes, &map_w, kb * kBlockK, n0, bar);
+                } else {
+                    if (leader) mbar_arrive_expect_tx(bar, w_bytes * CTAS);
+                    tma_load_2d_pair(smem_w + stage * w_bytes, &map_w, kb * kBlockK, n0, bar);
+                }
+            }
+            if (!ok) drain_after_abort();
+        }
+    } else if (warp < kFirstUnpackWarp + 4 * kUnpackSets) {
         // ------------------------------------------------------------ nibble unpack
         // A thread owns one weight row (= one TMEM lane of its warp's quadrant).  The packed tile is
         // 128 rows x 64 bytes with the 64-byte TMA swizzle: 16-byte chunk c of row r sits at
@@ -403,15 +523,16 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         const int swz = (row >> 1) & 3;
         // Set `uset` takes the k-blocks whose running index n is congruent to it modulo kUnpackSets,
         // so two k-blocks are in flight per quadrant and one set's store latency hides behind the other.
-        const int uset = (warp - 2 - kEpiWarps) >> 2;
-        const int total_kb = ((num_tiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1) * k_blocks;
+        const int uset = (warp - kFirstUnpackWarp) >> 2;
+        const int total_kb = ((num_tiles - 1 - unit0) / unit_step + 1) * k_blocks;
         bool ok = true;
         for (int n = uset; n < total_kb && ok; n += kUnpackSets) {
             {
                 const int ps = n % p.stages_p, ws = n % p.stages_w;
                 const uint32_t pph = (uint32_t)((n / p.stages_p) & 1), wph = (uint32_t)((n / p.stages_w) & 1);
-                ok = mbar_wait_warp(smem_u32(&s_full_p[ps]), pph, abort_flag, p.watchdog, kWdUnpackFull);
-                if (ok) ok = mbar_wait_warp(smem_u32(&s_empty_w8[ws]), wph ^ 1u, abort_flag, p.watchdog, kWdUnpackEmpty);
+                ok = mbar_wait(smem_u32(&s_full_p[ps]), pph, abort_flag, p.watchdog, kWdUnpackFull);
+                if (ok) ok = mbar_wait(smem_u32(&s_empty_w8[ws]), wph ^ 1u, abort_flag, p.watchdog, kWdUnpackEmpty);
+                ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 tc_fence_after();
                 const uint8_t* src = gen_base + (smem_p - base) + ps * pk_bytes + row * 64;
@@ -421,34 +542,37 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&s_empty_p[ps]));   // packed stage read: give it back
                 const uint32_t w_tmem = tmem_base + lane_addr + (uint32_t)(kAccStages * p.bt + ws * kColsW);
+                uint32_t o[32];                          // 128 codes -> 128 int8 = 32 TMEM columns
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {            // 32 codes -> 32 int8 = 8 TMEM columns
+                for (int c = 0; c < 4; ++c) {
                     const uint32_t w[4] = {pk[c].x, pk[c].y, pk[c].z, pk[c].w};
-                    uint32_t o[8];
 #pragma unroll
                     for (int q = 0; q < 4; ++q) {
                         const uint32_t lo = (w[q] << 4) & 0xF0F0F0F0u;   // even channels, 16*code
                         const uint32_t hi = w[q] & 0xF0F0F0F0u;          // odd channels
-                        o[2 * q + 0] = __byte_perm(lo, hi, 0x5140);
-                        o[2 * q + 1] = __byte_perm(lo, hi, 0x7362);
+                        o[8 * c + 2 * q + 0] = __byte_perm(lo, hi, 0x5140);
+                        o[8 * c + 2 * q + 1] = __byte_perm(lo, hi, 0x7362);
                     }
-                    tmem_st8(w_tmem + (uint32_t)(8 * c), o);
                 }
+                tmem_st32(w_tmem, o);
                 tmem_st_wait();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&s_full_w8[ws]));
+                if (lane == 0) {
+                    if (CTAS == 1) mbar_arrive(smem_u32(&s_full_w8[ws]));
+                    else mbar_arrive_cta(smem_u32(&s_full_w8[ws]), 0);
+                }
             }
         }
     } else if (BITS == 4) {
         // ------------------------------------------------- TMA producer, packed weights
         if (lane < kProducerLanes) {
-            const int total_kb = ((num_tiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1) * k_blocks;
+            const int total_kb = ((num_tiles - 1 - unit0) / unit_step + 1) * k_blocks;
             bool ok = true;
             for (int n = lane; n < total_kb; n += kProducerLanes) {
-                const int tile = (int)blockIdx.x + (n / k_blocks) * (int)gridDim.x;
+                const int tile = unit0 + (n / k_blocks) * unit_step;
                 const int kb = n % k_blocks;
-                const int n0 = (tile / p.m_tiles) * kTileN;
+                const int n0 = (tile / p.m_tiles) * (kTileN * CTAS) + (int)cta_rank * kTileN;
                 const int ps = n % p.stages_p;
                 const uint32_t pph = (uint32_t)((n / p.stages_p) & 1);
                 ok = mbar_wait(smem_u32(&s_empty_p[ps]), pph ^ 1u, abort_flag, p.watchdog, kWdProducer);
@@ -464,9 +588,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     // ------------------------------------------------------------------ teardown
     tc_fence_before();
     __syncthreads();
+    if (CTAS == 2) cluster_sync_all();              // neither CTA leaves while the other may still signal it
     if (warp == 1) {
         tc_fence_after();
-        tmem_dealloc(tmem_base, (uint32_t)p.tmem_cols);
+        tmem_dealloc<CTAS>(tmem_base, (uint32_t)p.tmem_cols);
     }
 }
 
@@ -541,6 +666,31 @@ fq_status build_weight_tmap(Weights& W) {
     return FQ_OK;
 }
 
+namespace {
+
+template <int BITS, int CTAS>
+fq_status launch_variant(const CUtensorMap& map_a, const CUtensorMap& map_w, const Params& p, int grid, size_t smem,
+                         cudaStream_t stream) {
+    auto kern = gemm_tcgen05_kernel<BITS, CTAS>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+        return FQ_ERR_CUDA;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid, 1, 1);
+    cfg.blockDim = dim3(BITS == 4 ? kThreadsW4 : kThreadsW8, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = CTAS;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = CTAS == 2 ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kern, map_a, map_w, p) == cudaSuccess ? FQ_OK : FQ_ERR_CUDA;
+}
+
+}  // namespace
+
 fq_status launch_gemm_tcgen05(const int8_t* a8, int64_t M, const Weights& W, int acc_shift, const GemmOut& out,
                               cudaStream_t stream) {
     if (M == 0 || W.N == 0) return FQ_OK;
@@ -553,10 +703,12 @@ fq_status launch_gemm_tcgen05(const int8_t* a8, int64_t M, const Weights& W, int
     const int bt_max = W.bits == 4 ? 208 : 256;
     const int m_tiles = (int)((M + bt_max - 1) / bt_max);
     int bt = (int)(((M + m_tiles - 1) / m_tiles + 15) / 16 * 16);
-    if (const char* e = getenv("FQ_DEBUG_BT")) bt = atoi(e);   // TEMP experiment
     p.bt = bt;
     p.m_tiles = (int)((M + bt - 1) / bt);
-    p.n_tiles = (int)((W.N + kTileN - 1) / kTileN);
+    // CTA pairs for large 8-bit problems (measured +9 % at 8192^3; no gain for the 4-bit path, whose
+    // weights never pass through shared memory, nor for short token batches).
+    int ctas = (W.bits == 8 && W.N > kTileN && bt >= 128 && M >= 1024) ? 2 : 1;
+    p.n_tiles = (int)((W.N + kTileN * ctas - 1) / (kTileN * ctas));
     p.acc_shift = acc_shift;
     p.w_scale = W.w_scale;
     p.bias = W.bias;
@@ -570,7 +722,7 @@ fq_status launch_gemm_tcgen05(const int8_t* a8, int64_t M, const Weights& W, int
 
     const size_t epi_bytes = (size_t)kEpiWarps * kEpiStageBytes;
     const size_t budget = 227 * 1024 - 1024 /*alignment slack*/ - 1024 /*static*/ - epi_bytes;
-    const size_t a_bytes = (size_t)bt * kBlockK, w_bytes = (size_t)kTileN * kBlockK, pk_bytes = w_bytes / 2;
+    const size_t a_bytes = (size_t)(bt / ctas) * kBlockK, w_bytes = (size_t)kTileN * kBlockK, pk_bytes = w_bytes / 2;
     size_t smem;
     if (W.bits == 4) {
         p.stages_w = stages_w;
@@ -594,27 +746,23 @@ fq_status launch_gemm_tcgen05(const int8_t* a8, int64_t M, const Weights& W, int
         smem = (a_bytes + w_bytes) * stages + epi_bytes + 1024;
     }
 
+    // each CTA of a pair loads its own half of the token tile
     CUtensorMap map_a;
-    if (!encode_2d(&map_a, a8, (uint64_t)W.K, (uint64_t)M, kBlockK, (uint32_t)bt, CU_TENSOR_MAP_SWIZZLE_128B))
+    if (!encode_2d(&map_a, a8, (uint64_t)W.K, (uint64_t)M, kBlockK, (uint32_t)(bt / ctas), CU_TENSOR_MAP_SWIZZLE_128B))
         return FQ_ERR_CUDA;
 
     int dev = 0, sms = 148;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    const int num_tiles = p.m_tiles * p.n_tiles;
-    const int grid = num_tiles < sms ? num_tiles : sms;
+    const int num_units = p.m_tiles * p.n_tiles;
+    const int max_units = sms / ctas;
+    const int grid = (num_units < max_units ? num_units : max_units) * ctas;
 
-    cudaError_t e;
-    if (W.bits == 4) {
-        e = cudaFuncSetAttribute(gemm_tcgen05_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return FQ_ERR_CUDA;
-        gemm_tcgen05_kernel<4><<<grid, kThreadsW4, smem, stream>>>(map_a, W.tmap, p);
-    } else {
-        e = cudaFuncSetAttribute(gemm_tcgen05_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return FQ_ERR_CUDA;
-        gemm_tcgen05_kernel<8><<<grid, kThreadsW8, smem, stream>>>(map_a, W.tmap, p);
-    }
-    return cudaGetLastError() == cudaSuccess ? FQ_OK : FQ_ERR_CUDA;
+    if (W.bits == 4)
+        return ctas == 2 ? launch_variant<4, 2>(map_a, W.tmap, p, grid, smem, stream)
+                         : launch_variant<4, 1>(map_a, W.tmap, p, grid, smem, stream);
+    return ctas == 2 ? launch_variant<8, 2>(map_a, W.tmap, p, grid, smem, stream)
+                     : launch_variant<8, 1>(map_a, W.tmap, p, grid, smem, stream);
 }
 
 }  // namespace fq
