@@ -1,18 +1,21 @@
 // Streaming variant of the runtime prologue (Alg. 1 runtime half lines 1-2, Eq. 5) for long
 // batches: same arithmetic, bit for bit, as transform_quantize_kernel, but tokens reach the
 // SM through a TMA-fed shared-memory ring so that many rows are in flight per SM regardless
-// of register pressure.
+// of register pressure, and the floating-point work is issued as packed f32x2 instructions.
 //
-//   - One persistent CTA of 1024 threads per SM, split into row groups of `gw` warps; a
-//     group owns one token at a time, a thread owns E = 32 consecutive channels of it.
+//   - One persistent CTA of 512 threads per SM, split into row groups of `gw` warps; a
+//     group owns one token at a time, a thread owns E = 64 (or 32) consecutive channels.
 //   - A token row is fetched as a 3-D tiled TMA box {128 bytes, K*e/128, 1} with the 128-byte
-//     swizzle, which makes the per-thread 64/128-byte reads bank-conflict free.  The per-
+//     swizzle, which makes the per-thread 64..256-byte reads bank-conflict free.  The per-
 //     channel multiplier is staged once in shared memory with the same swizzle.
 //   - Each group runs `depth` slots: the group barrier that exchanges the per-warp maxima also
 //     proves that every warp has finished reading the slot, so the group's leader refills it
 //     right there -- no separate "empty" barrier.
-//   - Strides 1..16 run in registers, strides 32..block/2 by warp shuffles (2 or 3 stages for
-//     blocks of 128 / 256 channels instead of the 3 or 4 a 16-channel thread needs).
+//   - Register layout: float2 v[p] = (channel p, channel p + E/2).  Butterflies with stride
+//     below E/2 then act on both halves at once (fadd2 / ffma2 by -1: each lane of a packed
+//     instruction is one IEEE binary32 operation, so the rounding is that of the scalar
+//     network); the stride-E/2 stage works inside the pairs; strides E..block/2 go across
+//     lanes (one shuffle per value, one packed FMA per pair).
 #include <cuda_bf16.h>
 #include <float.h>
 
@@ -23,7 +26,6 @@
 namespace fq {
 namespace {
 
-constexpr int E = 32;
 constexpr int kThreads = 512;
 constexpr int kMaxSlots = 128;
 
@@ -49,11 +51,17 @@ __device__ __forceinline__ bool group_barrier_and(int id, int count, bool pred) 
         : "memory");
     return r != 0;
 }
+// A thread's slice is 64, 128 or 256 contiguous bytes of a swizzled, 1024-byte aligned region.
+// Inside one 128-byte line the swizzled address of 16-byte piece i is (address of piece 0) ^ (i << 4),
+// so one pointer per line (line0, line1 = swizzled starts of the slice's lines) is all a thread keeps.
+__device__ __forceinline__ const uint8_t* piece(const uint8_t* line0, const uint8_t* line1, int i) {
+    const uint8_t* l = i < 8 ? line0 : line1;
+    return reinterpret_cast<const uint8_t*>(reinterpret_cast<uintptr_t>(l) ^ (uintptr_t)((i & 7) << 4));
+}
 
 struct RingParams {
     int64_t rows;
     int K;
-    int block;
     float cnorm, qmax, clip_ratio;
     const float* mult;
     uint8_t* codes;
@@ -65,9 +73,10 @@ struct RingParams {
     uint32_t* watchdog;
 };
 
-template <typename XT, int FMT, bool CLAMP>
+template <typename XT, int FMT, bool CLAMP, int E, int BLOCK>
 __global__ void __launch_bounds__(kThreads, 1)
 transform_quantize_ring_kernel(const __grid_constant__ CUtensorMap map_x, const RingParams p) {
+    constexpr int H = E / 2;                       // channels per half: v[i] = (channel i, channel i + H)
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t s_full[kMaxSlots];
     __shared__ float s_part[2][32];
@@ -113,92 +122,113 @@ transform_quantize_ring_kernel(const __grid_constant__ CUtensorMap map_x, const 
             const int r = first + d * step;
             if (r < rows) {
                 mbar_arrive_expect_tx(smem_u32(&full0[d]), tx);
-                tma_load_3d(slot0 + d * p.slot_bytes, &map_x, 0, 0, (int)r, smem_u32(&full0[d]));
+                tma_load_3d(slot0 + d * p.slot_bytes, &map_x, 0, 0, r, smem_u32(&full0[d]));
                 ++issued;
             }
         }
     }
 
-    // A thread's 16-byte pieces lie in one 128-byte line, so their swizzled offsets are
-    // swz(first) ^ (i << 4): one register per operand instead of one per piece.
-    constexpr int kPieces = E * (int)sizeof(XT) / 16;      // 4 (bf16) or 8 (fp32)
-    const uint32_t xoff0 = swz128((uint32_t)col0 * (uint32_t)sizeof(XT));
-    const uint8_t* gptr = gen + swz128((uint32_t)col0 * 4u);
+    // swizzled starts of the (up to two) 128-byte lines of this thread's slices
+    const uint32_t xs0 = swz128((uint32_t)col0 * (uint32_t)sizeof(XT));
+    const uint32_t xs1 = swz128((uint32_t)col0 * (uint32_t)sizeof(XT) + 128u);
+    const uint8_t* g0 = gen + swz128((uint32_t)col0 * 4u);
+    const uint8_t* g1 = gen + swz128((uint32_t)col0 * 4u + 128u);
+    const float2 neg1 = make_float2(-1.0f, -1.0f);
 
     int n = 0, d = 0;
     uint32_t ph = 0;
     for (int row = first; row < rows; row += step, ++n) {
         bool ok = mbar_wait_warp(smem_u32(&full0[d]), ph, abort_flag, p.watchdog, 0x100u);
 
-        float v[E];
-        const uint8_t* slot = gen + slots_off + (size_t)(group * p.depth + d) * p.slot_bytes + xoff0;
+        float2 v[H];
+        const uint8_t* slot = gen + slots_off + (size_t)(group * p.depth + d) * p.slot_bytes;
+        const uint8_t* x0 = slot + xs0;
+        const uint8_t* x1 = slot + xs1;
         if (col_ok) {
             if (sizeof(XT) == 2) {
+                // bf16: 8 channels per 16-byte piece; pieces [0, H/8) are the low half, the rest the high half
 #pragma unroll
-                for (int i = 0; i < kPieces; ++i) {
-                    const uint4 q = *reinterpret_cast<const uint4*>(
-                        reinterpret_cast<const uint8_t*>(reinterpret_cast<uintptr_t>(slot) ^ (uintptr_t)(i << 4)));
-                    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+                for (int i = 0; i < H / 8; ++i) {
+                    const uint4 lo = *reinterpret_cast<const uint4*>(piece(x0, x1, i));
+                    const uint4 hi = *reinterpret_cast<const uint4*>(piece(x0, x1, i + H / 8));
+                    const uint32_t wl[4] = {lo.x, lo.y, lo.z, lo.w}, wh[4] = {hi.x, hi.y, hi.z, hi.w};
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
-                        v[8 * i + 2 * j + 0] = __uint_as_float(w[j] << 16);
-                        v[8 * i + 2 * j + 1] = __uint_as_float(w[j] & 0xffff0000u);
+                        v[8 * i + 2 * j + 0] = make_float2(__uint_as_float(wl[j] << 16), __uint_as_float(wh[j] << 16));
+                        v[8 * i + 2 * j + 1] = make_float2(__uint_as_float(wl[j] & 0xffff0000u),
+                                                           __uint_as_float(wh[j] & 0xffff0000u));
                     }
                 }
             } else {
 #pragma unroll
-                for (int i = 0; i < kPieces; ++i) {
-                    const float4 q = *reinterpret_cast<const float4*>(
-                        reinterpret_cast<const uint8_t*>(reinterpret_cast<uintptr_t>(slot) ^ (uintptr_t)(i << 4)));
-                    v[4 * i + 0] = q.x; v[4 * i + 1] = q.y; v[4 * i + 2] = q.z; v[4 * i + 3] = q.w;
+                for (int i = 0; i < H / 4; ++i) {
+                    const float4 lo = *reinterpret_cast<const float4*>(piece(x0, x1, i));
+                    const float4 hi = *reinterpret_cast<const float4*>(piece(x0, x1, i + H / 4));
+                    v[4 * i + 0] = make_float2(lo.x, hi.x);
+                    v[4 * i + 1] = make_float2(lo.y, hi.y);
+                    v[4 * i + 2] = make_float2(lo.z, hi.z);
+                    v[4 * i + 3] = make_float2(lo.w, hi.w);
                 }
             }
             if (p.mult != nullptr) {
 #pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    const float4 g4 = *reinterpret_cast<const float4*>(
-                        reinterpret_cast<const uint8_t*>(reinterpret_cast<uintptr_t>(gptr) ^ (uintptr_t)(i << 4)));
-                    v[4 * i + 0] = __fmul_rn(v[4 * i + 0], g4.x);
-                    v[4 * i + 1] = __fmul_rn(v[4 * i + 1], g4.y);
-                    v[4 * i + 2] = __fmul_rn(v[4 * i + 2], g4.z);
-                    v[4 * i + 3] = __fmul_rn(v[4 * i + 3], g4.w);
+                for (int i = 0; i < H / 4; ++i) {
+                    const float4 lo = *reinterpret_cast<const float4*>(piece(g0, g1, i));
+                    const float4 hi = *reinterpret_cast<const float4*>(piece(g0, g1, i + H / 4));
+                    v[4 * i + 0] = f2_mul(v[4 * i + 0], make_float2(lo.x, hi.x));
+                    v[4 * i + 1] = f2_mul(v[4 * i + 1], make_float2(lo.y, hi.y));
+                    v[4 * i + 2] = f2_mul(v[4 * i + 2], make_float2(lo.z, hi.z));
+                    v[4 * i + 3] = f2_mul(v[4 * i + 3], make_float2(lo.w, hi.w));
                 }
             } else {
+                const float2 c2 = make_float2(p.cnorm, p.cnorm);
 #pragma unroll
-                for (int i = 0; i < E; ++i) v[i] = __fmul_rn(v[i], p.cnorm);
+                for (int i = 0; i < H; ++i) v[i] = f2_mul(v[i], c2);
             }
         } else {
 #pragma unroll
-            for (int i = 0; i < E; ++i) v[i] = 0.0f;
+            for (int i = 0; i < H; ++i) v[i] = make_float2(0.0f, 0.0f);
         }
 
-        // strides 1..16 in registers, 32..block/2 across lanes (same network as the register-only kernel)
+        // strides 1 .. H/2: both halves at once
 #pragma unroll
-        for (int h = 1; h < E; h <<= 1) {
-            if (h < p.block) {
+        for (int h = 1; h < H; h <<= 1) {
+            if (h < BLOCK) {
 #pragma unroll
-                for (int i = 0; i < E; ++i) {
+                for (int i = 0; i < H; ++i) {
                     if ((i & h) == 0) {
-                        const float a = v[i], b = v[i + h];
-                        v[i] = __fadd_rn(a, b);
-                        v[i + h] = __fsub_rn(a, b);
+                        const float2 a = v[i], b = v[i + h];
+                        v[i] = f2_add(a, b);
+                        v[i + h] = f2_fma(b, neg1, a);       // a - b, exact product
                     }
                 }
             }
         }
-        for (int h = E; h < p.block; h <<= 1) {
-            const int lm = h / E;
-            const float sgn = (lane & lm) ? -1.0f : 1.0f;
+        // stride H: inside each pair
+        if (H < BLOCK) {
 #pragma unroll
-            for (int i = 0; i < E; ++i) {
-                const float q = __shfl_xor_sync(0xffffffffu, v[i], lm);
-                v[i] = __fmaf_rn(v[i], sgn, q);
+            for (int i = 0; i < H; ++i) {
+                const float a = v[i].x, b = v[i].y;
+                v[i] = make_float2(__fadd_rn(a, b), __fsub_rn(a, b));
+            }
+        }
+        // strides E .. BLOCK/2: partner lane = lane ^ (h / E); upper lane keeps partner - own
+#pragma unroll
+        for (int h = E; h < BLOCK; h <<= 1) {
+            const int lm = h / E;
+            const float s = (lane & lm) ? -1.0f : 1.0f;
+            const float2 s2 = make_float2(s, s);
+#pragma unroll
+            for (int i = 0; i < H; ++i) {
+                const float2 q = make_float2(__shfl_xor_sync(0xffffffffu, v[i].x, lm),
+                                             __shfl_xor_sync(0xffffffffu, v[i].y, lm));
+                v[i] = f2_fma(v[i], s2, q);
             }
         }
 
         float m = 0.0f;
 #pragma unroll
-        for (int i = 0; i < E; ++i) m = fmaxf(m, fabsf(v[i]));
+        for (int i = 0; i < H; ++i) m = fmaxf(m, fmaxf(fabsf(v[i].x), fabsf(v[i].y)));
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
         if (p.gw > 1) {
@@ -207,8 +237,6 @@ transform_quantize_ring_kernel(const __grid_constant__ CUtensorMap map_x, const 
             m = (lane < p.gw) ? s_part[n & 1][group * p.gw + lane] : 0.0f;
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-        } else {
-            ok = __all_sync(0xffffffffu, ok);
         }
         if (!ok) break;
 
@@ -218,7 +246,7 @@ transform_quantize_ring_kernel(const __grid_constant__ CUtensorMap map_x, const 
             if (nr < rows) {
                 fence_proxy_async_smem();
                 mbar_arrive_expect_tx(smem_u32(&full0[d]), tx);
-                tma_load_3d(slot0 + d * p.slot_bytes, &map_x, 0, 0, (int)nr, smem_u32(&full0[d]));
+                tma_load_3d(slot0 + d * p.slot_bytes, &map_x, 0, 0, nr, smem_u32(&full0[d]));
                 ++issued;
             }
         }
@@ -231,28 +259,38 @@ transform_quantize_ring_kernel(const __grid_constant__ CUtensorMap map_x, const 
             dl = 0.0f;
             inv = 0.0f;
         }
+        // codes: channel i from .x, channel i + H from .y
         constexpr int kPer = FMT == 0 ? 8 : 4;               // codes per 32-bit word
-        uint32_t w[E / kPer];
+        constexpr int kWords = H / kPer;                     // words per half
+        const float2 inv2 = make_float2(inv, inv);
+        uint32_t wlo[kWords], whi[kWords];
 #pragma unroll
-        for (int j = 0; j < E / kPer; ++j) {
-            uint32_t b[kPer];
+        for (int j = 0; j < kWords; ++j) {
+            uint32_t bl[kPer], bh[kPer];
 #pragma unroll
             for (int i = 0; i < kPer; ++i) {
-                float t = __fmul_rn(v[j * kPer + i], inv);
-                if (CLAMP) t = fminf(fmaxf(t, -p.qmax), p.qmax);
-                b[i] = __float_as_uint(__fadd_rn(t, 12582912.0f));
+                float2 t = f2_mul(v[j * kPer + i], inv2);
+                if (CLAMP) {
+                    t.x = fminf(fmaxf(t.x, -p.qmax), p.qmax);
+                    t.y = fminf(fmaxf(t.y, -p.qmax), p.qmax);
+                }
+                // Scalar adds on purpose: a packed multiply feeding a packed add with no other use was
+                // observed to be fused into one packed FMA by the assembler, which rounds ties differently.
+                bl[i] = __float_as_uint(__fadd_rn(t.x, 12582912.0f));
+                bh[i] = __float_as_uint(__fadd_rn(t.y, 12582912.0f));
             }
-            w[j] = pack_word<FMT>(b);
+            wlo[j] = pack_word<FMT>(bl);
+            whi[j] = pack_word<FMT>(bh);
         }
         if (col_ok) {
-            if (FMT == 0) {
-                uint4* dst = reinterpret_cast<uint4*>(p.codes + (int64_t)row * (p.K / 2) + col0 / 2);
-                dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
-            } else {
-                uint4* dst = reinterpret_cast<uint4*>(p.codes + (int64_t)row * p.K + col0);
-                dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
-                dst[1] = make_uint4(w[FMT == 0 ? 0 : 4], w[FMT == 0 ? 1 : 5], w[FMT == 0 ? 2 : 6], w[FMT == 0 ? 3 : 7]);
-            }
+            // low-half words then high-half words are consecutive channels: one contiguous store run
+            uint32_t w[2 * kWords];
+#pragma unroll
+            for (int j = 0; j < kWords; ++j) { w[j] = wlo[j]; w[kWords + j] = whi[j]; }
+            const int64_t pitch = FMT == 0 ? p.K / 2 : p.K;
+            uint4* dst = reinterpret_cast<uint4*>(p.codes + (int64_t)row * pitch + (FMT == 0 ? col0 / 2 : col0));
+#pragma unroll
+            for (int j = 0; j < 2 * kWords / 4; ++j) dst[j] = make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
             if (wg == 0 && lane == 0) p.delta[row] = dl;
         }
         if (++d == p.depth) { d = 0; ph ^= 1u; }
@@ -271,7 +309,7 @@ transform_quantize_ring_kernel(const __grid_constant__ CUtensorMap map_x, const 
     }
 }
 
-template <typename XT, int FMT>
+template <typename XT, int FMT, int E, int BLOCK>
 cudaError_t launch_ring(const CUtensorMap& map, const RingParams& p, int grid, size_t smem, cudaStream_t stream) {
     auto go = [&](auto kern) -> cudaError_t {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -279,8 +317,27 @@ cudaError_t launch_ring(const CUtensorMap& map, const RingParams& p, int grid, s
         kern<<<grid, kThreads, smem, stream>>>(map, p);
         return cudaGetLastError();
     };
-    if (p.clip_ratio < 1.0f) return go(transform_quantize_ring_kernel<XT, FMT, true>);
-    return go(transform_quantize_ring_kernel<XT, FMT, false>);
+    if (p.clip_ratio < 1.0f) return go(transform_quantize_ring_kernel<XT, FMT, true, E, BLOCK>);
+    return go(transform_quantize_ring_kernel<XT, FMT, false, E, BLOCK>);
+}
+
+template <typename XT, int FMT, int E>
+cudaError_t launch_ring_block(int block, const CUtensorMap& map, const RingParams& p, int grid, size_t smem,
+                              cudaStream_t stream) {
+    switch (block) {
+        case 32: return launch_ring<XT, FMT, E, 32>(map, p, grid, smem, stream);
+        case 64: return launch_ring<XT, FMT, E, 64>(map, p, grid, smem, stream);
+        case 128: return launch_ring<XT, FMT, E, 128>(map, p, grid, smem, stream);
+        case 256: return launch_ring<XT, FMT, E, 256>(map, p, grid, smem, stream);
+        default: return cudaErrorNotSupported;
+    }
+}
+
+template <typename XT, int FMT>
+cudaError_t launch_ring_e(int e, int block, const CUtensorMap& map, const RingParams& p, int grid, size_t smem,
+                          cudaStream_t stream) {
+    return e == 64 ? launch_ring_block<XT, FMT, 64>(block, map, p, grid, smem, stream)
+                   : launch_ring_block<XT, FMT, 32>(block, map, p, grid, smem, stream);
 }
 
 }  // namespace
@@ -290,26 +347,26 @@ cudaError_t launch_transform_quantize_ring(const void* x, fq_dtype xt, int64_t r
                                            StoreFmt fmt, void* codes, float* delta, cudaStream_t stream) {
     const size_t esz = xt == FQ_BF16 ? 2 : 4;
     const size_t row_bytes = (size_t)K * esz;
-    // shape gate: whole 128-byte lines, at most 256 of them per box, a full warp of 32-channel threads
-    if (K < 1024 || row_bytes % 128 != 0 || row_bytes / 128 > 256 || rows > 0x7fffffffll) return cudaErrorNotSupported;
+    // shape gate: whole 128-byte lines, at most 256 of them per box, blocks of 32..256 channels
+    if (K < 1024 || row_bytes % 128 != 0 || row_bytes / 128 > 256 || rows > 0x7fffffffll || block < 32)
+        return cudaErrorNotSupported;
     int dev = 0, sms = 148;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     if (rows < 2 * (int64_t)sms) return cudaErrorNotSupported;     // short batches: latency-bound, register kernel
 
+    const int e = (K >= 2048 && K % 64 == 0) ? 64 : 32;            // channels per thread
     int gw = 1;
-    while ((int64_t)gw * 32 * E < K) gw <<= 1;
-    if (gw > 32) return cudaErrorNotSupported;
+    while ((int64_t)gw * 32 * e < K) gw <<= 1;
     if (gw > kThreads / 32) return cudaErrorNotSupported;
-    int ngroups = (kThreads / 32) / gw;
+    const int ngroups = (kThreads / 32) / gw;
     const size_t slot = (row_bytes + 1023) / 1024 * 1024;
     const size_t g_bytes = mult ? ((size_t)K * 4 + 1023) / 1024 * 1024 : 0;
     const size_t budget = 227 * 1024 - 2048 - 1024;
-    if (g_bytes + 2 * slot > budget) return cudaErrorNotSupported;
+    if (g_bytes + 2 * slot * ngroups > budget) return cudaErrorNotSupported;
     int depth = (int)((budget - g_bytes) / (slot * ngroups));
     if (depth > 4) depth = 4;
-    if (depth < 2) return cudaErrorNotSupported;
-    if (ngroups * depth > kMaxSlots) return cudaErrorNotSupported;
+    if (depth < 2 || ngroups * depth > kMaxSlots) return cudaErrorNotSupported;
 
     CUtensorMap map;
     const uint64_t dims[3] = {128 / esz, row_bytes / 128, (uint64_t)rows};
@@ -320,19 +377,19 @@ cudaError_t launch_transform_quantize_ring(const void* x, fq_dtype xt, int64_t r
         return cudaErrorNotSupported;
 
     RingParams p{};
-    p.rows = rows; p.K = (int)K; p.block = block; p.cnorm = cnorm; p.qmax = (float)qmax; p.clip_ratio = clip_ratio;
+    p.rows = rows; p.K = (int)K; p.cnorm = cnorm; p.qmax = (float)qmax; p.clip_ratio = clip_ratio;
     p.mult = mult; p.codes = static_cast<uint8_t*>(codes); p.delta = delta; p.gw = gw; p.depth = depth;
     p.slot_bytes = (uint32_t)slot; p.g_bytes = (uint32_t)g_bytes;
     p.watchdog = watchdog_device_ptr();
     if (!p.watchdog) return cudaErrorUnknown;
     const size_t smem = g_bytes + slot * ngroups * depth + 1024;
-    int64_t need = (rows + ngroups - 1) / ngroups;
+    const int64_t need = (rows + ngroups - 1) / ngroups;
     const int grid = (int)(need < sms ? need : sms);
     if (xt == FQ_BF16)
-        return fmt == StoreFmt::Nibble ? launch_ring<__nv_bfloat16, 0>(map, p, grid, smem, stream)
-                                       : launch_ring<__nv_bfloat16, 1>(map, p, grid, smem, stream);
-    return fmt == StoreFmt::Nibble ? launch_ring<float, 0>(map, p, grid, smem, stream)
-                                   : launch_ring<float, 1>(map, p, grid, smem, stream);
+        return fmt == StoreFmt::Nibble ? launch_ring_e<__nv_bfloat16, 0>(e, block, map, p, grid, smem, stream)
+                                       : launch_ring_e<__nv_bfloat16, 1>(e, block, map, p, grid, smem, stream);
+    return fmt == StoreFmt::Nibble ? launch_ring_e<float, 0>(e, block, map, p, grid, smem, stream)
+                                   : launch_ring_e<float, 1>(e, block, map, p, grid, smem, stream);
 }
 
 }  // namespace fq
