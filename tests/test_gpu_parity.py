@@ -87,6 +87,32 @@ def test_quantize_act_zero_tiny_and_strided_rows(bits):
     assert (codes[M] == 0xAB).all() and delta[M] == -1.0      # nothing written past row M
 
 
+@pytest.mark.parametrize("bits", [4, 8])
+@pytest.mark.parametrize("M,K,dtype", [(40, 1024, "f32"), (600, 2048, "bf16"), (700, 4096, "f32"), (333, 1024, "bf16")])
+def test_quantize_act_exact_ties_round_to_even(bits, M, K, dtype):
+    """Every scaled value is an exact half-integer: a fused multiply-add or a different tie rule in
+    any kernel variant (register kernel for short batches, streaming kernel for long ones) shows up
+    in thousands of codes.  One-hot inputs per 32-channel block give z = +-a on the whole block; one
+    block per token carries 2q so that the step is exactly 2 and z/2 is a tie for odd a."""
+    q = 7 if bits == 4 else 127
+    rng = np.random.default_rng(M + K + bits)
+    nb = K // 32
+    a = 2 * rng.integers(0, q, size=(M, nb)) + 1                  # odd amplitudes below 2q
+    a[np.arange(M), rng.integers(0, nb, size=M)] = 2 * q          # sets max|z| = 2q  ->  step 2
+    x = np.zeros((M, K), np.float32)
+    pos = rng.integers(0, 32, size=(M, nb))
+    x[np.arange(M)[:, None], np.arange(nb)[None, :] * 32 + pos] = a
+    xs = synth.as_dtype(x, dtype)                                  # small integers: exact in bf16
+    g = np.ones(K, np.float32)
+    want_codes, want_delta = oracle.quantize_act(xs, dtype, g, 32, bits)
+    assert np.all(want_delta == 2.0)
+    c = oracle.unpack(want_codes, K, bits)
+    assert np.all((np.abs(c) % 2 == 0) | (np.abs(c) == q))        # ties went to even
+    codes, delta = fq.quantize_act(to_dev(xs, dtype), to_dev(g), 32, bits)
+    assert np.array_equal(to_np(delta), want_delta)
+    assert np.array_equal(to_np(codes), want_codes)
+
+
 def test_quantize_act_amplitude_invariance_on_device():
     x = make_x(64, 2048, "f32", seed=4)
     c0, d0 = fq.quantize_act(to_dev(x), None, 64, 4)
@@ -317,6 +343,27 @@ def test_full_size_backbone_sites_sampled_rows_and_second_witness():
         acc = fq.gemm_acc_i32(gpu["codes"], gpu["h"])
         assert np.array_equal(to_np(acc[rows]), ref["acc"]), site.name
         assert torch.equal(acc, fq.gemm_simt(gpu["codes"], None, gpu["h"], raw_acc=True)), site.name
+
+
+SWEEP_SAMPLE = [
+    # M, K=N, block, bits  (a sample of the throughput-sweep grid; outputs checked on sampled token rows)
+    (1, 1024, 32, 4), (1, 4096, 256, 8), (16, 2048, 64, 4), (64, 1024, 128, 8), (256, 4096, 32, 8),
+    (256, 2048, 256, 4), (1024, 1024, 64, 4), (1024, 4096, 128, 8), (4096, 2048, 128, 4),
+]
+
+
+@pytest.mark.parametrize("M,KN,block,bits", SWEEP_SAMPLE)
+def test_sweep_points_sampled_rows(M, KN, block, bits):
+    """Throughput-sweep shapes: prologue bit-exact on every token, accumulators bit-exact and
+    outputs within tolerance on sampled rows (first, last and tile-boundary tokens)."""
+    data = synth.make_site(synth.sweep_site(M, KN, KN, block, bits), seed=5)
+    rows = sorted({0, M - 1, min(M - 1, 207), min(M - 1, 208), M // 2, min(M - 1, 255), min(M - 1, 256)})
+    gpu, ref = run_site(data, rows=rows)
+    assert np.array_equal(to_np(gpu["codes"]), ref["codes"])
+    assert np.array_equal(to_np(gpu["delta"]).view(np.uint32), ref["delta"].view(np.uint32))
+    acc = fq.gemm_acc_i32(gpu["codes"], gpu["h"])
+    assert np.array_equal(to_np(acc[rows]), ref["acc"])
+    assert_close(to_np(gpu["y"][rows]), ref["y"], "bf16", f"sweep M={M} K=N={KN}")
 
 
 def test_calibration_helpers_match_oracle():
