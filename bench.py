@@ -265,7 +265,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     gemm_ops = 2.0 * s.M * s.K * s.N_total
     achieved = gemm_ops / (gemm_ms[dom] * 1e-3) / 1e12
     int8_peak = 2.0 * peaks["bf16_sustained"]     # dense int8 : bf16 = 2 : 1 (4.5 vs 2.25 PFLOP/s nominal)
-    roofline = {"bound": "tensor", "kernel": f"gemm_tcgen05_kernel<{s.bits}> ({s.name}: M={s.M} K={s.K} N={s.N_total})",
+    roofline = {"bound": "tensor", "kernel": f"gemm_tcgen05_kernel<{s.bits},1> ({s.name}: M={s.M} K={s.K} N={s.N_total})",
                 "achieved": round(achieved, 1), "peak": round(int8_peak, 1), "unit": "TOP/s",
                 "frac": round(achieved / int8_peak, 4),
                 "peak_source": f"{peaks['source']}: sustained bf16 cuBLAS {peaks['bf16_sustained']} TFLOP/s x 2 (int8:bf16)",
@@ -391,7 +391,7 @@ def run_reference(args):
 
 # -------------------------------------------------------------------- workloads ----
 # DRAM bytes per launch of the dominant kernel, from the ncu captures summarised under profiles/.
-TRAFFIC_BYTES = {}
+TRAFFIC_BYTES = {("backbone_layer", "gate_up"): 42319104}   # profiles/gemm_tcgen05_w4_gate_up_m816.md
 
 
 def workload_sites(name: str):

@@ -51,6 +51,12 @@ __device__ __forceinline__ bool group_barrier_and(int id, int count, bool pred) 
         : "memory");
     return r != 0;
 }
+// max(m, |x|, |y|) in one instruction (3-input max of sm_100).
+__device__ __forceinline__ float max3_abs(float m, float x, float y) {
+    float r;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(m), "f"(fabsf(x)), "f"(fabsf(y)));
+    return r;
+}
 // A thread's slice is 64, 128 or 256 contiguous bytes of a swizzled, 1024-byte aligned region.
 // Inside one 128-byte line the swizzled address of 16-byte piece i is (address of piece 0) ^ (i << 4),
 // so one pointer per line (line0, line1 = swizzled starts of the slice's lines) is all a thread keeps.
@@ -101,10 +107,13 @@ transform_quantize_ring_kernel(const __grid_constant__ CUtensorMap map_x, const 
         fence_mbarrier_init();
         fence_proxy_async_smem();
     }
-    if (p.mult != nullptr) {   // stage the multiplier, swizzled like the rows
+    if (p.mult != nullptr) {
+        // Stage the multiplier with its 16-byte pieces XOR-swizzled by the index of the thread slice
+        // (E floats) they belong to, so that the slice-per-thread reads below are bank-conflict free.
         for (int i = tid * 4; i < p.K; i += kThreads * 4) {
             const float4 g4 = __ldg(reinterpret_cast<const float4*>(p.mult + i));
-            *reinterpret_cast<float4*>(gen + swz128((uint32_t)i * 4u)) = g4;
+            const uint32_t off = (uint32_t)i * 4u;
+            *reinterpret_cast<float4*>(gen + (off ^ (((off / (E * 4u)) & 7u) << 4))) = g4;
         }
     }
     __syncthreads();
@@ -131,8 +140,9 @@ transform_quantize_ring_kernel(const __grid_constant__ CUtensorMap map_x, const 
     // swizzled starts of the (up to two) 128-byte lines of this thread's slices
     const uint32_t xs0 = swz128((uint32_t)col0 * (uint32_t)sizeof(XT));
     const uint32_t xs1 = swz128((uint32_t)col0 * (uint32_t)sizeof(XT) + 128u);
-    const uint8_t* g0 = gen + swz128((uint32_t)col0 * 4u);
-    const uint8_t* g1 = gen + swz128((uint32_t)col0 * 4u + 128u);
+    const uint32_t gkey = (uint32_t)((col0 / E) & 7) << 4;
+    const uint8_t* g0 = gen + (((uint32_t)col0 * 4u) ^ gkey);
+    const uint8_t* g1 = gen + (((uint32_t)col0 * 4u + 128u) ^ gkey);
     const float2 neg1 = make_float2(-1.0f, -1.0f);
 
     int n = 0, d = 0;
@@ -228,7 +238,7 @@ transform_quantize_ring_kernel(const __grid_constant__ CUtensorMap map_x, const 
 
         float m = 0.0f;
 #pragma unroll
-        for (int i = 0; i < H; ++i) m = fmaxf(m, fmaxf(fabsf(v[i].x), fabsf(v[i].y)));
+        for (int i = 0; i < H; ++i) m = max3_abs(m, v[i].x, v[i].y);
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
         if (p.gw > 1) {
