@@ -28,6 +28,12 @@ __device__ __forceinline__ uint32_t pack_word(const uint32_t* b) {
     }
 }
 
+// Channel (within a thread's run) that field i of 32-bit word j holds, per store format.
+template <int FMT>
+__device__ __forceinline__ constexpr int code_index(int j, int i) {
+    return FMT == 0 ? 8 * j + i : (FMT == 1 ? 4 * j + i : 8 * (j / 2) + 2 * i + (j & 1));
+}
+
 // Packed binary32 arithmetic (two independent IEEE operations per instruction).  Written as PTX
 // with an explicit rounding modifier: such instructions are never contracted into fused
 // multiply-adds by the optimizer, which the bit-exact contract of the prologue depends on.

@@ -200,7 +200,7 @@ transform_quantize_kernel(const XT* __restrict__ x, int64_t rows, int K, int64_t
             uint32_t b[kPer];
 #pragma unroll
             for (int i = 0; i < kPer; ++i) {
-                float t = __fmul_rn(v[j * kPer + i], inv);
+                float t = __fmul_rn(v[code_index<FMT>(j, i)], inv);
                 if (CLAMP) t = fminf(fmaxf(t, -qmax), qmax);
                 b[i] = __float_as_uint(__fadd_rn(t, 12582912.0f));
             }
@@ -321,7 +321,8 @@ __global__ void smooth_scale_kernel(const float* __restrict__ a, const float* __
     s[i] = (float)v;
 }
 
-// 16 packed bytes (32 codes) per thread -> 32 int8 holding 16*code, natural order.
+// 16 packed bytes (32 codes) per thread -> 32 int8 holding 16*code, each group of 8 channels in the
+// (even channels, odd channels) order of StoreFmt::Int8Perm.
 __global__ void expand_nibbles_kernel(const uint4* __restrict__ packed, int64_t n_vec, uint4* __restrict__ out) {
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n_vec) return;
@@ -332,8 +333,8 @@ __global__ void expand_nibbles_kernel(const uint4* __restrict__ packed, int64_t 
     for (int j = 0; j < 4; ++j) {
         const uint32_t lo = (w[j] << 4) & 0xF0F0F0F0u;   // even channels, code in the high nibble of each byte
         const uint32_t hi = w[j] & 0xF0F0F0F0u;          // odd channels
-        o[2 * j + 0] = __byte_perm(lo, hi, 0x5140);
-        o[2 * j + 1] = __byte_perm(lo, hi, 0x7362);
+        o[2 * j + 0] = lo;     // channels 0,2,4,6 of the group of 8
+        o[2 * j + 1] = hi;     // channels 1,3,5,7
     }
     out[2 * i + 0] = make_uint4(o[0], o[1], o[2], o[3]);
     out[2 * i + 1] = make_uint4(o[4], o[5], o[6], o[7]);
@@ -353,14 +354,14 @@ cudaError_t launch_transform_quantize(const void* x, fq_dtype xt, int64_t rows, 
     const int k = (int)K;
     if (xt == FQ_F32) {
         const float* p = static_cast<const float*>(x);
-        return fmt == StoreFmt::Nibble
-                   ? launch_t<float, 0>(p, rows, k, ldx, mult, cnorm, block, qmax, clip_ratio, codes, delta, stream)
-                   : launch_t<float, 1>(p, rows, k, ldx, mult, cnorm, block, qmax, clip_ratio, codes, delta, stream);
+            if (fmt == StoreFmt::Nibble) return launch_t<float, 0>(p, rows, k, ldx, mult, cnorm, block, qmax, clip_ratio, codes, delta, stream);
+        if (fmt == StoreFmt::Int8) return launch_t<float, 1>(p, rows, k, ldx, mult, cnorm, block, qmax, clip_ratio, codes, delta, stream);
+        return launch_t<float, 2>(p, rows, k, ldx, mult, cnorm, block, qmax, clip_ratio, codes, delta, stream);
     }
     const __nv_bfloat16* p = static_cast<const __nv_bfloat16*>(x);
-    return fmt == StoreFmt::Nibble
-               ? launch_t<__nv_bfloat16, 0>(p, rows, k, ldx, mult, cnorm, block, qmax, clip_ratio, codes, delta, stream)
-               : launch_t<__nv_bfloat16, 1>(p, rows, k, ldx, mult, cnorm, block, qmax, clip_ratio, codes, delta, stream);
+    if (fmt == StoreFmt::Nibble) return launch_t<__nv_bfloat16, 0>(p, rows, k, ldx, mult, cnorm, block, qmax, clip_ratio, codes, delta, stream);
+    if (fmt == StoreFmt::Int8) return launch_t<__nv_bfloat16, 1>(p, rows, k, ldx, mult, cnorm, block, qmax, clip_ratio, codes, delta, stream);
+    return launch_t<__nv_bfloat16, 2>(p, rows, k, ldx, mult, cnorm, block, qmax, clip_ratio, codes, delta, stream);
 }
 
 cudaError_t launch_multipliers(const float* smooth, int64_t K, float cnorm, float* mult_w, float* mult_g,

@@ -279,7 +279,7 @@ transform_quantize_ring_kernel(const __grid_constant__ CUtensorMap map_x, const 
             uint32_t bl[kPer], bh[kPer];
 #pragma unroll
             for (int i = 0; i < kPer; ++i) {
-                float2 t = f2_mul(v[j * kPer + i], inv2);
+                float2 t = f2_mul(v[code_index<FMT>(j, i)], inv2);
                 if (CLAMP) {
                     t.x = fminf(fmaxf(t.x, -p.qmax), p.qmax);
                     t.y = fminf(fmaxf(t.y, -p.qmax), p.qmax);
@@ -396,10 +396,14 @@ cudaError_t launch_transform_quantize_ring(const void* x, fq_dtype xt, int64_t r
     const int64_t need = (rows + ngroups - 1) / ngroups;
     const int grid = (int)(need < sms ? need : sms);
     if (xt == FQ_BF16)
-        return fmt == StoreFmt::Nibble ? launch_ring_e<__nv_bfloat16, 0>(e, block, map, p, grid, smem, stream)
-                                       : launch_ring_e<__nv_bfloat16, 1>(e, block, map, p, grid, smem, stream);
-    return fmt == StoreFmt::Nibble ? launch_ring_e<float, 0>(e, block, map, p, grid, smem, stream)
-                                   : launch_ring_e<float, 1>(e, block, map, p, grid, smem, stream);
+    {
+        if (fmt == StoreFmt::Nibble) return launch_ring_e<__nv_bfloat16, 0>(e, block, map, p, grid, smem, stream);
+        if (fmt == StoreFmt::Int8) return launch_ring_e<__nv_bfloat16, 1>(e, block, map, p, grid, smem, stream);
+        return launch_ring_e<__nv_bfloat16, 2>(e, block, map, p, grid, smem, stream);
+    }
+    if (fmt == StoreFmt::Nibble) return launch_ring_e<float, 0>(e, block, map, p, grid, smem, stream);
+    if (fmt == StoreFmt::Int8) return launch_ring_e<float, 1>(e, block, map, p, grid, smem, stream);
+    return launch_ring_e<float, 2>(e, block, map, p, grid, smem, stream);
 }
 
 }  // namespace fq

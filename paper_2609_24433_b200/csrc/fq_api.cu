@@ -130,10 +130,11 @@ fq_status linear_impl(const void* x, fq_dtype xt, int64_t M, int64_t ldx, const 
     st = carve(workspace, ws_bytes, M, W->K, &ws);
     if (st != FQ_OK) return st;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    // Prologue writes one int8 per code into the workspace (4-bit codes stay in [-7, 7]).
+    // Prologue writes one int8 per code into the workspace (4-bit codes stay in [-7, 7] and are laid
+    // out in the channel order the GEMM's nibble unpack gives the weights).
     const int qmax = bits == 4 ? 7 : 127;
     if (launch_transform_quantize(x, xt, M, W->K, ldx, W->mult_g, block_norm(W->block), W->block, qmax, clip_ratio,
-                                  StoreFmt::Int8, ws.a8, ws.delta, s) != cudaSuccess)
+                                  bits == 4 ? StoreFmt::Int8Perm : StoreFmt::Int8, ws.a8, ws.delta, s) != cudaSuccess)
         return FQ_ERR_CUDA;
     if (g_profile_mark != nullptr) {
         // Inside a stream capture the mark must be an external event-record node to stay readable.

@@ -27,7 +27,9 @@ struct Weights {
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 // ---- launchers (host side, defined next to their kernels) -------------------
-enum class StoreFmt : int { Nibble = 0, Int8 = 1 };
+// Int8Perm: one int8 per code, but every group of 8 channels stored as (c0,c2,c4,c6,c1,c3,c5,c7) --
+// the order in which the GEMM's nibble unpack produces the 4-bit weights without a byte permute.
+enum class StoreFmt : int { Nibble = 0, Int8 = 1, Int8Perm = 2 };
 
 // Runtime prologue / offline fold share one kernel: multiply by mult[K] (or the
 // constant `cnorm` if mult == nullptr), block FWHT, per-row absmax, quantize to

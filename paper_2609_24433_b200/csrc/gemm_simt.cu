@@ -35,10 +35,11 @@ __global__ void gemm_simt_kernel(const int8_t* __restrict__ a8, int64_t M, int64
             const uint2 w = __ldg(wrow + k);
             const uint32_t lo0 = (w.x << 4) & 0xF0F0F0F0u, hi0 = w.x & 0xF0F0F0F0u;
             const uint32_t lo1 = (w.y << 4) & 0xF0F0F0F0u, hi1 = w.y & 0xF0F0F0F0u;
-            acc = __dp4a((int)a.x, (int)__byte_perm(lo0, hi0, 0x5140), acc);
-            acc = __dp4a((int)a.y, (int)__byte_perm(lo0, hi0, 0x7362), acc);
-            acc = __dp4a((int)a.z, (int)__byte_perm(lo1, hi1, 0x5140), acc);
-            acc = __dp4a((int)a.w, (int)__byte_perm(lo1, hi1, 0x7362), acc);
+            // 4-bit activations arrive as int8 with each group of 8 channels in (even, odd) order
+            acc = __dp4a((int)a.x, (int)lo0, acc);
+            acc = __dp4a((int)a.y, (int)hi0, acc);
+            acc = __dp4a((int)a.z, (int)lo1, acc);
+            acc = __dp4a((int)a.w, (int)hi1, acc);
         }
     }
     acc >>= acc_shift;   // exact: the scaled operands make acc a multiple of 2^acc_shift

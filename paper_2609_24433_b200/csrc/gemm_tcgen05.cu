@@ -72,7 +72,7 @@ constexpr int kStagesW = 3;            // unpacked-weight stages in tensor memor
 constexpr int kColsW = kBlockK / 4;     // TMEM columns of one unpacked k-block (128 int8 per lane)
 constexpr int kMaxStages = 8;
 constexpr int kMaxStagesP = 16;
-constexpr int kProducerLanes = 1;      // threads that issue TMA copies, k-blocks dealt round-robin
+constexpr int kProducerLanes = 4;      // threads that issue TMA copies, k-blocks dealt round-robin
 
 struct Params {
     int64_t M, N, K;
@@ -490,11 +490,12 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         }
     } else if (BITS == 8) {
         // ------------------------------------------------- TMA producer, int8 weights
-        // (a thread sustains only about one bulk-tensor copy per ~400 cycles: one producer per operand)
-        if (lane == 0) {
+        // (a thread sustains only about one bulk-tensor copy per ~400 cycles: one warp per operand,
+        // k-blocks dealt round-robin to kProducerLanes lanes)
+        if (lane < kProducerLanes) {
             const int total_kb = ((num_tiles - 1 - unit0) / unit_step + 1) * k_blocks;
             bool ok = true;
-            for (int n = 0; n < total_kb; ++n) {
+            for (int n = lane; n < total_kb; n += kProducerLanes) {
                 const int tile = unit0 + (n / k_blocks) * unit_step;
                 const int kb = n % k_blocks;
                 const int n0 = (tile / p.m_tiles) * (kTileN * CTAS) + (int)cta_rank * kTileN;
@@ -550,8 +551,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                     for (int q = 0; q < 4; ++q) {
                         const uint32_t lo = (w[q] << 4) & 0xF0F0F0F0u;   // even channels, 16*code
                         const uint32_t hi = w[q] & 0xF0F0F0F0u;          // odd channels
-                        o[8 * c + 2 * q + 0] = __byte_perm(lo, hi, 0x5140);
-                        o[8 * c + 2 * q + 1] = __byte_perm(lo, hi, 0x7362);
+                        o[8 * c + 2 * q + 0] = lo;   // same (even, odd) channel order as the int8 activations
+                        o[8 * c + 2 * q + 1] = hi;
                     }
                 }
                 tmem_st32(w_tmem, o);
@@ -698,11 +699,26 @@ fq_status launch_gemm_tcgen05(const int8_t* a8, int64_t M, const Weights& W, int
 
     Params p{};
     p.M = M; p.N = W.N; p.K = W.K;
-    // Token tile: as large as TMEM allows (two accumulator stages, plus the unpacked-weight ring
-    // for 4-bit weights: 2*bt + 3*32 <= 512 columns), split evenly so ragged M wastes little.
+    int dev = 0, sms = 148;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    // Token tile.  Upper bound from TMEM: two accumulator stages, plus the unpacked-weight ring for
+    // 4-bit weights (2*bt + 3*32 <= 512 columns).  M is split evenly over m_tiles so that ragged M
+    // wastes little, and m_tiles is chosen by a small cost model: rounds of tiles over the SMs times
+    // the measured time of a 128-wide k-block, which is roughly c0 + c1*bt cycles (a large fixed part:
+    // smaller tiles are nearly as fast per k-block, so filling all SMs in one round wins).
     const int bt_max = W.bits == 4 ? 208 : 256;
-    const int m_tiles = (int)((M + bt_max - 1) / bt_max);
-    int bt = (int)(((M + m_tiles - 1) / m_tiles + 15) / 16 * 16);
+    const double c0 = W.bits == 4 ? 920.0 : 500.0, c1 = W.bits == 4 ? 1.3 : 1.8;
+    const int64_t n128 = (W.N + kTileN - 1) / kTileN;
+    int bt = 0;
+    double best = 0.0;
+    for (int mt = (int)((M + bt_max - 1) / bt_max); mt <= (int)((M + 63) / 64); ++mt) {
+        const int b = (int)(((M + mt - 1) / mt + 15) / 16 * 16);
+        if (b > bt_max) continue;
+        const int64_t tiles = n128 * ((M + b - 1) / b);
+        const double cost = (double)((tiles + sms - 1) / sms) * (c0 + c1 * b);
+        if (bt == 0 || cost < best * 0.97) { bt = b; best = cost; }   // prefer larger tiles unless clearly cheaper
+    }
     p.bt = bt;
     p.m_tiles = (int)((M + bt - 1) / bt);
     // CTA pairs for large 8-bit problems (measured +9 % at 8192^3; no gain for the 4-bit path, whose
@@ -751,9 +767,6 @@ fq_status launch_gemm_tcgen05(const int8_t* a8, int64_t M, const Weights& W, int
     if (!encode_2d(&map_a, a8, (uint64_t)W.K, (uint64_t)M, kBlockK, (uint32_t)(bt / ctas), CU_TENSOR_MAP_SWIZZLE_128B))
         return FQ_ERR_CUDA;
 
-    int dev = 0, sms = 148;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     const int num_units = p.m_tiles * p.n_tiles;
     const int max_units = sms / ctas;
     const int grid = (num_units < max_units ? num_units : max_units) * ctas;
