@@ -155,7 +155,7 @@ class LayerOnDevice:
         and a second graph per set that also carries external event-record nodes around and
         inside every site so that single-kernel durations can be read after a replay."""
         torch = self.torch
-        self.graphs, self.ev_graphs, self.ev = [], [], []
+        self.graphs, self.ev_graphs, self.ev, self.ev_empty = [], [], [], []
         for r in range(ROTATE):
             g = torch.cuda.CUDAGraph()
             with torch.cuda.graph(g):
@@ -166,25 +166,38 @@ class LayerOnDevice:
                 for e in trio:
                     e.record()          # creates the underlying event before the capture
             torch.cuda.synchronize()
+            pair = tuple(torch.cuda.Event(enable_timing=True, external=True) for _ in range(2))
+            for e in pair:
+                e.record()
+            torch.cuda.synchronize()
             g2 = torch.cuda.CUDAGraph()
             with torch.cuda.graph(g2):
                 self.step(r, evs)
+                pair[0].record()        # two event nodes with nothing between: the cost of a record node
+                pair[1].record()
             self.ev_graphs.append(g2)
             self.ev.append(evs)
+            self.ev_empty.append(pair)
         torch.cuda.synchronize()
 
     def kernel_durations(self, replays: int):
-        """Mean (prologue_ms, gemm_ms) per site over ``replays`` replays of the evented graphs."""
+        """Mean (prologue_ms, gemm_ms) per site over ``replays`` replays of the evented graphs, and
+        the mean interval between two adjacent event-record nodes (what a record node itself costs:
+        every interval between events contains one, so it is subtracted from the kernel figures)."""
         torch = self.torch
         act = [[] for _ in self.sites]
         gemm = [[] for _ in self.sites]
+        empty = []
         for k in range(replays):
             self.ev_graphs[k % ROTATE].replay()
             torch.cuda.synchronize()
             for i, (e0, mark, e1) in enumerate(self.ev[k % ROTATE]):
                 act[i].append(e0.elapsed_time(mark))
                 gemm[i].append(mark.elapsed_time(e1))
-        return [statistics.mean(a) for a in act], [statistics.mean(g) for g in gemm]
+            p0, p1 = self.ev_empty[k % ROTATE]
+            empty.append(p0.elapsed_time(p1))
+        ov = statistics.mean(empty)
+        return ([max(statistics.mean(a) - ov, 1e-6) for a in act], [max(statistics.mean(g) - ov, 1e-6) for g in gemm], ov)
 
     @property
     def launches_per_step(self) -> int:
@@ -258,7 +271,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         raise RuntimeError(f"device watchdog fired during the benchmark: {word:#x}")
 
     # per-kernel durations: the same step graphs with event-record nodes between the kernels
-    act_ms, gemm_ms = layer.kernel_durations(max(8, min(K, 40)))
+    act_ms, gemm_ms, ev_overhead_ms = layer.kernel_durations(max(8, min(K, 40)))
     peaks = read_peaks()
     dom = max(range(len(sites)), key=lambda i: gemm_ms[i])
     s = sites[dom]
@@ -270,6 +283,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
                 "frac": round(achieved / int8_peak, 4),
                 "peak_source": f"{peaks['source']}: sustained bf16 cuBLAS {peaks['bf16_sustained']} TFLOP/s x 2 (int8:bf16)",
                 "traffic": TRAFFIC_BYTES.get((args.workload, s.name)),
+                "event_node_overhead_us": round(ev_overhead_ms * 1e3, 2),
                 "per_site_us": {sites[i].name: {"prologue": round(act_ms[i] * 1e3, 2), "gemm": round(gemm_ms[i] * 1e3, 2)}
                                 for i in range(len(sites))}}
     act_i = max(range(len(sites)), key=lambda i: act_ms[i])
