@@ -28,7 +28,7 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-from paper_2609_24433_b200 import synth  # noqa: E402
+from paper_2609_24433_b200 import replicas, synth  # noqa: E402
 
 METRIC = "fused FWHT+quant+W4A4/W8A8 GEMM throughput (whole layer)"
 UNIT = "TOPS"
@@ -216,7 +216,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         dist.init_process_group("nccl", device_id=device)
 
     sites = workload_sites(args.workload)
-    layer = LayerOnDevice(sites, seed=2 + 7919 * rank, device=device)
+    layer = LayerOnDevice(sites, seed=replicas.replica_seed(2, rank), device=device)
     ops = layer_ops(sites)
     K, Wm = args.steps, max(args.warmup, 3)
 
@@ -259,12 +259,8 @@ def run_ours(args, rank: int, world: int, local_rank: int):
                     torch.cuda.synchronize()
             torch.cuda.synchronize()
         note = "sampled during an immediate untimed replay of the timed loop (timed region < NVML period)"
-    if dist is not None:
-        t = torch.tensor([ms_total], dtype=torch.float64, device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
-    ms_per_step = ms_total / K
-    value = world * ops / (ms_per_step * 1e-3) / 1e12
+    ms_per_step = replicas.max_over_ranks(ms_total, dist, device) / K
+    value = replicas.job_throughput(ops * K, ms_total * 1e-3, dist, device) / 1e12
 
     st, word = fq.device_status()
     if st != fq.OK:
@@ -346,15 +342,18 @@ def run_e2e(layer, sites, ops, world, K, Wm, dist, device):
     if dist is not None:
         dist.barrier()
     torch.cuda.synchronize()
-    t0 = time.perf_counter()
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    start.record()
     for _ in range(n):
-        step()
-    dt = (time.perf_counter() - t0) / n
+        step()                      # ends with a synchronize: host time between steps is inside the interval
+    end.record()
+    torch.cuda.synchronize()
     if dist is not None:
-        t = torch.tensor([dt], dtype=torch.float64, device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        dt = float(t.item())
-    return {"value": round(world * ops / dt / 1e12, 3), "unit": UNIT, "ms_per_step": round(dt * 1e3, 4),
+        dist.barrier()
+    seconds = start.elapsed_time(end) * 1e-3
+    dt = replicas.max_over_ranks(seconds, dist, device) / n
+    return {"value": round(replicas.job_throughput(ops * n, seconds, dist, device) / 1e12, 3), "unit": UNIT,
+            "ms_per_step": round(dt * 1e3, 4),
             "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": n}
 
 
