@@ -72,7 +72,19 @@ constexpr int kStagesW = 3;            // unpacked-weight stages in tensor memor
 constexpr int kColsW = kBlockK / 4;     // TMEM columns of one unpacked k-block (128 int8 per lane)
 constexpr int kMaxStages = 8;
 constexpr int kMaxStagesP = 16;
-constexpr int kProducerLanes = 4;      // threads that issue TMA copies, k-blocks dealt round-robin
+
+// Timeline hooks for kernel development: with -DFQ_GEMM_TRACE the first CTA records clock64() at
+// the marked points of the first 128 k-blocks (agent 0 activation producer, 2 unpack, 3 MMA
+// issuer) and fq_debug_trace() copies the table out.  Compiled out by default.
+#ifdef FQ_GEMM_TRACE
+__device__ unsigned long long g_trace[4 * 128 * 4];
+#define FQ_TRACE(agent, n, e)                                                                   \
+    do {                                                                                        \
+        if (blockIdx.x == 0 && lane == 0 && (n) < 128) g_trace[((agent) * 128 + (n)) * 4 + (e)] = clock64(); \
+    } while (0)
+#else
+#define FQ_TRACE(agent, n, e) do { } while (0)
+#endif
 
 struct Params {
     int64_t M, N, K;
@@ -181,6 +193,79 @@ __device__ __forceinline__ void mma_i8_ts(uint32_t d_tmem, uint32_t a_tmem, uint
             ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
             : "memory");
 }
+// One k-block of work for the issuing warp, as ONE block of PTX so that the two barrier tests for
+// the NEXT k-block are in flight while this k-block's four MMAs and its commits are issued (their
+// results are read only at the end; separate asm statements would stall on each test's ~100-cycle
+// latency).  Must be called by a converged warp: every lane executes the tests, and the lane that
+// elect.sync picks inside the block issues the MMAs and commits (measured: 160 cycles per k-block
+// with the election inside the block, 400 with a predicate derived from the lane index).
+//   a[4]      A operand of the four K=32 steps: TMEM addresses (TS) or shared-memory descriptors (SS)
+//   bar_stage barrier that frees the k-block's shared-memory (and TMEM weight) stage
+//   bar_acc   barrier "accumulator complete", or 0 when this is not the tile's last k-block
+// Returns 1 if both tested phases were complete (0 when `peek` is 0).
+#define FQ_ISSUE_HEAD                                                   \
+    "{\n\t"                                                             \
+    ".reg .pred pl, pacc, pt, pk, pa, pw, pc;\n\t"                       \
+    "elect.sync _|pl, 0xffffffff;\n\t"                                  \
+    "setp.ne.b32 pacc, %12, 0;\n\t"                                     \
+    "setp.eq.b32 pt, %1, %1;\n\t"                                       \
+    "setp.ne.b32 pk, %15, 0;\n\t"                                       \
+    "setp.ne.b32 pa, %1, %1;\n\t"                                       \
+    "setp.ne.b32 pw, %1, %1;\n\t"                                       \
+    "@pk mbarrier.test_wait.parity.shared::cta.b64 pa, [%16], %17;\n\t" \
+    "@pk mbarrier.test_wait.parity.shared::cta.b64 pw, [%18], %19;\n\t"
+#define FQ_ISSUE_MMAS(CG, L, R)                                                          \
+    "@pl tcgen05.mma.cta_group::" CG ".kind::i8 [%2], " L "%3" R ", %7, %11, pacc;\n\t"   \
+    "@pl tcgen05.mma.cta_group::" CG ".kind::i8 [%2], " L "%4" R ", %8, %11, pt;\n\t"     \
+    "@pl tcgen05.mma.cta_group::" CG ".kind::i8 [%2], " L "%5" R ", %9, %11, pt;\n\t"     \
+    "@pl tcgen05.mma.cta_group::" CG ".kind::i8 [%2], " L "%6" R ", %10, %11, pt;\n\t"
+#define FQ_ISSUE_COMMITS_1                                                                          \
+    "@pl tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%13];\n\t"          \
+    "setp.ne.and.b32 pc, %14, 0, pl;\n\t"                                                           \
+    "@pc tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%14];\n\t"
+#define FQ_ISSUE_COMMITS_2                                                                                          \
+    "@pl tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%13], %20;\n\t"  \
+    "setp.ne.and.b32 pc, %14, 0, pl;\n\t"                                                                           \
+    "@pc tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%14], %20;\n\t"
+#define FQ_ISSUE_TAIL            \
+    "and.pred pa, pa, pw;\n\t"   \
+    "selp.b32 %0, 1, 0, pa;\n\t" \
+    "}"
+#define FQ_ISSUE_OPERANDS(ACON)                                                                                      \
+    : "=r"(ready)                                                                                                    \
+    : "r"(issue), "r"(d_tmem), ACON(a[0]), ACON(a[1]), ACON(a[2]), ACON(a[3]), "l"(b[0]), "l"(b[1]), "l"(b[2]),      \
+      "l"(b[3]), "r"(idesc), "r"(accumulate), "r"(bar_stage), "r"(bar_acc), "r"(peek), "r"(peek_bar_a),              \
+      "r"(peek_par_a), "r"(peek_bar_w), "r"(peek_par_w), "h"(mask)                                                   \
+    : "memory"
+#define FQ_CON_R(x) "r"(x)
+#define FQ_CON_L(x) "l"(x)
+
+template <int CTAS>
+__device__ __forceinline__ uint32_t issue_kblock_ts(uint32_t issue, uint32_t d_tmem, const uint32_t* a, const uint64_t* b,
+                                                    uint32_t idesc, uint32_t accumulate, uint32_t bar_stage,
+                                                    uint32_t bar_acc, uint32_t peek, uint32_t peek_bar_a,
+                                                    uint32_t peek_par_a, uint32_t peek_bar_w, uint32_t peek_par_w) {
+    uint32_t ready;
+    const uint16_t mask = 3;
+    if (CTAS == 1)
+        asm volatile(FQ_ISSUE_HEAD FQ_ISSUE_MMAS("1", "[", "]") FQ_ISSUE_COMMITS_1 FQ_ISSUE_TAIL FQ_ISSUE_OPERANDS(FQ_CON_R));
+    else
+        asm volatile(FQ_ISSUE_HEAD FQ_ISSUE_MMAS("2", "[", "]") FQ_ISSUE_COMMITS_2 FQ_ISSUE_TAIL FQ_ISSUE_OPERANDS(FQ_CON_R));
+    return ready;
+}
+template <int CTAS>
+__device__ __forceinline__ uint32_t issue_kblock_ss(uint32_t issue, uint32_t d_tmem, const uint64_t* a, const uint64_t* b,
+                                                    uint32_t idesc, uint32_t accumulate, uint32_t bar_stage,
+                                                    uint32_t bar_acc, uint32_t peek, uint32_t peek_bar_a,
+                                                    uint32_t peek_par_a, uint32_t peek_bar_w, uint32_t peek_par_w) {
+    uint32_t ready;
+    const uint16_t mask = 3;
+    if (CTAS == 1)
+        asm volatile(FQ_ISSUE_HEAD FQ_ISSUE_MMAS("1", "", "") FQ_ISSUE_COMMITS_1 FQ_ISSUE_TAIL FQ_ISSUE_OPERANDS(FQ_CON_L));
+    else
+        asm volatile(FQ_ISSUE_HEAD FQ_ISSUE_MMAS("2", "", "") FQ_ISSUE_COMMITS_2 FQ_ISSUE_TAIL FQ_ISSUE_OPERANDS(FQ_CON_L));
+    return ready;
+}
 __device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t* r) {
     asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
                  ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
@@ -260,11 +345,11 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                     const Params p) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t s_full_tma[kMaxStages];     // activations (+ int8 weights) landed
-    __shared__ uint64_t s_empty[kMaxStages];        // ... consumed by the MMAs
+    __shared__ uint64_t s_empty[kMaxStages];        // ... consumed by the MMAs (one commit per k-block; for 4-bit
+                                                    // weights it also frees that k-block's TMEM weight slot)
     __shared__ uint64_t s_full_p[kMaxStagesP];      // packed weights landed
     __shared__ uint64_t s_empty_p[kMaxStagesP];     // ... read by the unpack warps
     __shared__ uint64_t s_full_w8[kMaxStagesW];     // unpacked weights written
-    __shared__ uint64_t s_empty_w8[kMaxStagesW];    // ... consumed by the MMAs
     __shared__ uint64_t s_acc_full[kAccStages];
     __shared__ uint64_t s_acc_empty[kAccStages];
     __shared__ uint32_t s_tmem_base;
@@ -301,7 +386,6 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             }
             for (int s = 0; s < p.stages_w; ++s) {
                 mbar_init(smem_u32(&s_full_w8[s]), 4 * CTAS);
-                mbar_init(smem_u32(&s_empty_w8[s]), 1);
             }
         }
         for (int a = 0; a < kAccStages; ++a) {
@@ -326,77 +410,113 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
-        // One thread sustains only about one bulk-tensor copy per ~400 cycles (measured), so the
-        // k-blocks are dealt round-robin to kProducerLanes lanes, each waiting on its own stages.
-        if (lane < kProducerLanes) {
+        // The whole warp runs the loop and waits; one lane issues.  (A lone lane looping while its
+        // warp-mates are parked at the final __syncthreads was measured 2-3x slower per barrier
+        // hand-off: every dependent wait/branch of the lone lane pays for the divergent warp.)
+        {
             const uint32_t tx = a_bytes;
             const int total_kb = ((num_tiles - 1 - unit0) / unit_step + 1) * k_blocks;
             bool ok = true;
-            for (int n = lane; n < total_kb; n += kProducerLanes) {
-                const int tile = unit0 + (n / k_blocks) * unit_step;
-                const int kb = n % k_blocks;
-                const int t0 = (tile % p.m_tiles) * p.bt + (int)cta_rank * bt_cta;
-                const int stage = n % p.stages;
-                const uint32_t phase = (uint32_t)((n / p.stages) & 1);
-                ok = mbar_wait(smem_u32(&s_empty[stage]), phase ^ 1u, abort_flag, p.watchdog, kWdProducer);
+            int stage = 0, kb = 0, tile = unit0;
+            uint32_t phase = 0;
+            int t0 = (tile % p.m_tiles) * p.bt + (int)cta_rank * bt_cta;
+            bool peek = false;
+            for (int n = 0; n < total_kb; ++n) {
+                ok = mbar_wait_all(smem_u32(&s_empty[stage]), phase ^ 1u, abort_flag, p.watchdog, kWdProducer, peek);
                 if (!ok) break;
-                const uint32_t bar = smem_u32(&s_full_tma[stage]);
-                if (CTAS == 1) {
-                    mbar_arrive_expect_tx(bar, tx);
-                    tma_load_2d(smem_a + stage * a_bytes, &map_a, kb * kBlockK, t0, bar);
-                } else {
-                    // the pair's bytes are all counted on the even CTA's barrier, which it arms for both
-                    if (leader) mbar_arrive_expect_tx(bar, tx * CTAS);
-                    tma_load_2d_pair(smem_a + stage * a_bytes, &map_a, kb * kBlockK, t0, bar);
+                FQ_TRACE(0, n, 0);
+                {   // look at the next stage now: the test's latency hides behind the copy issued below
+                    const int s1 = stage + 1 == p.stages ? 0 : stage + 1;
+                    const uint32_t ph1 = s1 == 0 ? phase ^ 1u : phase;
+                    peek = n + 1 < total_kb && mbar_test_wait(smem_u32(&s_empty[s1]), ph1 ^ 1u);
+                }
+                if (elect_one()) {
+                    const uint32_t bar = smem_u32(&s_full_tma[stage]);
+                    if (CTAS == 1) {
+                        mbar_arrive_expect_tx(bar, tx);
+                        tma_load_2d(smem_a + stage * a_bytes, &map_a, kb * kBlockK, t0, bar);
+                    } else {
+                        // the pair's bytes are all counted on the even CTA's barrier, which it arms for both
+                        if (leader) mbar_arrive_expect_tx(bar, tx * CTAS);
+                        tma_load_2d_pair(smem_a + stage * a_bytes, &map_a, kb * kBlockK, t0, bar);
+                    }
+                }
+                FQ_TRACE(0, n, 1);
+                if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+                if (++kb == k_blocks) {
+                    kb = 0;
+                    tile += unit_step;
+                    t0 = (tile % p.m_tiles) * p.bt + (int)cta_rank * bt_cta;
                 }
             }
-            if (!ok) drain_after_abort();
+            if (!ok && lane == 0) drain_after_abort();
         }
     } else if (warp == 1) {
         // -------------------------------------------------------------- MMA issuer
-        if (lane == 0 && leader) {
+        // All lanes of the warp run the loop and the waits (converged); lane 0 of the pair's even
+        // CTA issues the MMAs and commits.
+        if (leader) {
             const uint32_t idesc = instr_desc_i8(kTileN * CTAS, p.bt);
             int stage = 0, wstage = 0;
             uint32_t phase = 0, wphase = 0;
             int acc_stage = 0;
             uint32_t acc_phase = 0;
             bool ok = true;
+            // The barriers of the NEXT k-block are tested (without blocking) inside the block of PTX
+            // that issues the current one: a barrier test has ~100 cycles of latency, and two of them
+            // in series per k-block would otherwise sit on the issuing warp's critical path.
+            bool ready = false;
+            int left = ((num_tiles - 1 - unit0) / unit_step + 1) * k_blocks;   // k-blocks still to issue
+            [[maybe_unused]] int tn = 0;
             for (int tile = unit0; tile < num_tiles && ok; tile += unit_step) {
-                ok = mbar_wait(smem_u32(&s_acc_empty[acc_stage]), acc_phase ^ 1u, abort_flag, p.watchdog, kWdMmaAcc);
+                ok = mbar_wait_all(smem_u32(&s_acc_empty[acc_stage]), acc_phase ^ 1u, abort_flag, p.watchdog, kWdMmaAcc);
                 if (!ok) break;
-                tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc_stage * p.bt);
                 for (int kb = 0; kb < k_blocks; ++kb) {
-                    ok = mbar_wait(smem_u32(&s_full_tma[stage]), phase, abort_flag, p.watchdog, kWdMmaFull);
-                    if (ok && BITS == 4)
-                        ok = mbar_wait(smem_u32(&s_full_w8[wstage]), wphase, abort_flag, p.watchdog, kWdMmaFull);
-                    if (!ok) break;
+                    FQ_TRACE(3, tn, 0);
+                    if (!__all_sync(0xffffffffu, ready)) {
+                        ok = mbar_wait_all(smem_u32(&s_full_tma[stage]), phase, abort_flag, p.watchdog, kWdMmaFull);
+                        if (ok && BITS == 4)
+                            ok = mbar_wait_all(smem_u32(&s_full_w8[wstage]), wphase, abort_flag, p.watchdog, kWdMmaFull);
+                        if (!ok) break;
+                    }
+                    FQ_TRACE(3, tn, 2);
+                    --left;
                     tc_fence_after();
+                    const int s1 = stage + 1 == p.stages ? 0 : stage + 1;
+                    const uint32_t ph1 = s1 == 0 ? phase ^ 1u : phase;
+                    const int w1 = wstage + 1 == p.stages_w ? 0 : wstage + 1;
+                    const uint32_t wph1 = w1 == 0 ? wphase ^ 1u : wphase;
+                    const uint32_t peek_bar_a = smem_u32(&s_full_tma[s1]);
+                    const uint32_t peek_bar_w = BITS == 4 ? smem_u32(&s_full_w8[w1]) : peek_bar_a;
+                    const uint32_t peek_par_w = BITS == 4 ? wph1 : ph1;
+                    const uint32_t bar_acc = kb == k_blocks - 1 ? smem_u32(&s_acc_full[acc_stage]) : 0u;
                     const uint64_t adesc = smem_desc_sw128(smem_a + stage * a_bytes);
+                    // step 32 bytes along K inside the swizzle atom: +2 in 16-byte address units
+                    const uint64_t bd[4] = {adesc, adesc + 2, adesc + 4, adesc + 6};
+                    uint32_t r;
                     if (BITS == 4) {
+                        // 32 int8 of K = 8 TMEM columns per MMA
                         const uint32_t w_tmem = tmem_base + (uint32_t)(kAccStages * p.bt + wstage * kColsW);
-#pragma unroll
-                        for (int k = 0; k < kBlockK / kMmaK; ++k)   // 32 int8 of K = 8 TMEM columns per MMA
-                            mma_i8_ts<CTAS>(d_tmem, w_tmem + (uint32_t)(8 * k), adesc + (uint64_t)(2 * k), idesc,
-                                      (kb | k) != 0 ? 1u : 0u);
+                        const uint32_t at[4] = {w_tmem, w_tmem + 8, w_tmem + 16, w_tmem + 24};
+                        r = issue_kblock_ts<CTAS>(0u, d_tmem, at, bd, idesc, kb != 0 ? 1u : 0u,
+                                                  smem_u32(&s_empty[stage]), bar_acc, left > 0 ? 1u : 0u, peek_bar_a, ph1,
+                                                  peek_bar_w, peek_par_w);
                     } else {
                         const uint64_t wdesc = smem_desc_sw128(smem_w + stage * w_bytes);
-#pragma unroll
-                        for (int k = 0; k < kBlockK / kMmaK; ++k) {
-                            // step 32 bytes along K inside the swizzle atom: +2 in 16-byte address units
-                            mma_i8<CTAS>(d_tmem, wdesc + (uint64_t)(2 * k), adesc + (uint64_t)(2 * k), idesc,
-                                   (kb | k) != 0 ? 1u : 0u);
-                        }
+                        const uint64_t ad[4] = {wdesc, wdesc + 2, wdesc + 4, wdesc + 6};
+                        r = issue_kblock_ss<CTAS>(0u, d_tmem, ad, bd, idesc, kb != 0 ? 1u : 0u,
+                                                  smem_u32(&s_empty[stage]), bar_acc, left > 0 ? 1u : 0u, peek_bar_a, ph1,
+                                                  peek_bar_w, peek_par_w);
                     }
-                    mma_commit<CTAS>(smem_u32(&s_empty[stage]));          // frees this stage when the MMAs retire
-                    if (++stage == p.stages) { stage = 0; phase ^= 1u; }
-                    if (BITS == 4) {
-                        mma_commit<CTAS>(smem_u32(&s_empty_w8[wstage]));
-                        if (++wstage == p.stages_w) { wstage = 0; wphase ^= 1u; }
-                    }
+                    ready = r != 0;
+                    FQ_TRACE(3, tn, 3);
+                    ++tn;
+                    stage = s1;
+                    phase = ph1;
+                    if (BITS == 4) { wstage = w1; wphase = wph1; }
                 }
                 if (!ok) break;
-                mma_commit<CTAS>(smem_u32(&s_acc_full[acc_stage]));        // accumulator complete
                 if (++acc_stage == kAccStages) { acc_stage = 0; acc_phase ^= 1u; }
             }
         }
@@ -490,29 +610,40 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         }
     } else if (BITS == 8) {
         // ------------------------------------------------- TMA producer, int8 weights
-        // (a thread sustains only about one bulk-tensor copy per ~400 cycles: one warp per operand,
-        // k-blocks dealt round-robin to kProducerLanes lanes)
-        if (lane < kProducerLanes) {
+        // (converged warp, one issuing lane: see the activation producer)
+        {
             const int total_kb = ((num_tiles - 1 - unit0) / unit_step + 1) * k_blocks;
             bool ok = true;
-            for (int n = lane; n < total_kb; n += kProducerLanes) {
-                const int tile = unit0 + (n / k_blocks) * unit_step;
-                const int kb = n % k_blocks;
-                const int n0 = (tile / p.m_tiles) * (kTileN * CTAS) + (int)cta_rank * kTileN;
-                const int stage = n % p.stages;
-                const uint32_t phase = (uint32_t)((n / p.stages) & 1);
-                ok = mbar_wait(smem_u32(&s_empty[stage]), phase ^ 1u, abort_flag, p.watchdog, kWdProducer);
+            int stage = 0, kb = 0, tile = unit0;
+            uint32_t phase = 0;
+            int n0 = (tile / p.m_tiles) * (kTileN * CTAS) + (int)cta_rank * kTileN;
+            bool peek = false;
+            for (int n = 0; n < total_kb; ++n) {
+                ok = mbar_wait_all(smem_u32(&s_empty[stage]), phase ^ 1u, abort_flag, p.watchdog, kWdProducer, peek);
                 if (!ok) break;
-                const uint32_t bar = smem_u32(&s_full_tma[stage]);
-                if (CTAS == 1) {
-                    mbar_arrive_expect_tx(bar, w_bytes);
-                    tma_load_2d(smem_w + stage * w_bytes, &map_w, kb * kBlockK, n0, bar);
-                } else {
-                    if (leader) mbar_arrive_expect_tx(bar, w_bytes * CTAS);
-                    tma_load_2d_pair(smem_w + stage * w_bytes, &map_w, kb * kBlockK, n0, bar);
+                {
+                    const int s1 = stage + 1 == p.stages ? 0 : stage + 1;
+                    const uint32_t ph1 = s1 == 0 ? phase ^ 1u : phase;
+                    peek = n + 1 < total_kb && mbar_test_wait(smem_u32(&s_empty[s1]), ph1 ^ 1u);
+                }
+                if (elect_one()) {
+                    const uint32_t bar = smem_u32(&s_full_tma[stage]);
+                    if (CTAS == 1) {
+                        mbar_arrive_expect_tx(bar, w_bytes);
+                        tma_load_2d(smem_w + stage * w_bytes, &map_w, kb * kBlockK, n0, bar);
+                    } else {
+                        if (leader) mbar_arrive_expect_tx(bar, w_bytes * CTAS);
+                        tma_load_2d_pair(smem_w + stage * w_bytes, &map_w, kb * kBlockK, n0, bar);
+                    }
+                }
+                if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+                if (++kb == k_blocks) {
+                    kb = 0;
+                    tile += unit_step;
+                    n0 = (tile / p.m_tiles) * (kTileN * CTAS) + (int)cta_rank * kTileN;
                 }
             }
-            if (!ok) drain_after_abort();
+            if (!ok && lane == 0) drain_after_abort();
         }
     } else if (warp < kFirstUnpackWarp + 4 * kUnpackSets) {
         // ------------------------------------------------------------ nibble unpack
@@ -527,21 +658,31 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         const int uset = (warp - kFirstUnpackWarp) >> 2;
         const int total_kb = ((num_tiles - 1 - unit0) / unit_step + 1) * k_blocks;
         bool ok = true;
+        int ps = uset, ws = uset;                        // ring slots of k-block n, kept incrementally
+        uint32_t pph = 0, wph = 0;
+        while (ps >= p.stages_p) { ps -= p.stages_p; pph ^= 1u; }
+        while (ws >= p.stages_w) { ws -= p.stages_w; wph ^= 1u; }
+        // TMEM slot ws is free once the MMAs of k-block m = n - stages_w have retired, which is the
+        // same event that frees that k-block's activation stage: barrier s_empty[m % stages], use
+        // number m / stages (stages_w <= stages, so the barrier cannot run a phase ahead of this wait).
+        int m = uset - p.stages_w, es = 0;
+        uint32_t eph = 0;
+        if (m >= 0) es = m;
+        while (es >= p.stages) { es -= p.stages; eph ^= 1u; }
         for (int n = uset; n < total_kb && ok; n += kUnpackSets) {
             {
-                const int ps = n % p.stages_p, ws = n % p.stages_w;
-                const uint32_t pph = (uint32_t)((n / p.stages_p) & 1), wph = (uint32_t)((n / p.stages_w) & 1);
-                ok = mbar_wait(smem_u32(&s_full_p[ps]), pph, abort_flag, p.watchdog, kWdUnpackFull);
-                if (ok) ok = mbar_wait(smem_u32(&s_empty_w8[ws]), wph ^ 1u, abort_flag, p.watchdog, kWdUnpackEmpty);
-                ok = __all_sync(0xffffffffu, ok);
+                if ((warp & 3) == 0) FQ_TRACE(2, n, 0);
+                ok = mbar_wait_all(smem_u32(&s_full_p[ps]), pph, abort_flag, p.watchdog, kWdUnpackFull);
                 if (!ok) break;
-                tc_fence_after();
+                if ((warp & 3) == 0) FQ_TRACE(2, n, 1);
                 const uint8_t* src = gen_base + (smem_p - base) + ps * pk_bytes + row * 64;
                 uint4 pk[4];
 #pragma unroll
                 for (int c = 0; c < 4; ++c) pk[c] = *reinterpret_cast<const uint4*>(src + ((c ^ swz) << 4));
+                // is the TMEM slot free?  (tested now, needed only after the expansion below)
+                const bool slot_free = m < 0 || mbar_test_wait(smem_u32(&s_empty[es]), eph);
                 __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&s_empty_p[ps]));   // packed stage read: give it back
+                if (elect_one()) mbar_arrive(smem_u32(&s_empty_p[ps]));   // packed stage read: give it back
                 const uint32_t w_tmem = tmem_base + lane_addr + (uint32_t)(kAccStages * p.bt + ws * kColsW);
                 uint32_t o[32];                          // 128 codes -> 128 int8 = 32 TMEM columns
 #pragma unroll
@@ -555,34 +696,59 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                         o[8 * c + 2 * q + 1] = hi;
                     }
                 }
+                ok = mbar_wait_all(smem_u32(&s_empty[es]), eph, abort_flag, p.watchdog, kWdUnpackEmpty, slot_free);
+                if (!ok) break;
+                if ((warp & 3) == 0) FQ_TRACE(2, n, 2);
+                tc_fence_after();
                 tmem_st32(w_tmem, o);
                 tmem_st_wait();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) {
+                if (elect_one()) {
                     if (CTAS == 1) mbar_arrive(smem_u32(&s_full_w8[ws]));
                     else mbar_arrive_cta(smem_u32(&s_full_w8[ws]), 0);
                 }
+                if ((warp & 3) == 0) FQ_TRACE(2, n, 3);
+                ps += kUnpackSets;
+                while (ps >= p.stages_p) { ps -= p.stages_p; pph ^= 1u; }
+                ws += kUnpackSets;
+                while (ws >= p.stages_w) { ws -= p.stages_w; wph ^= 1u; }
+                m += kUnpackSets;
+                if (m >= kUnpackSets) es += kUnpackSets;
+                else if (m >= 0) es = m;
+                while (es >= p.stages) { es -= p.stages; eph ^= 1u; }
             }
         }
     } else if (BITS == 4) {
         // ------------------------------------------------- TMA producer, packed weights
-        if (lane < kProducerLanes) {
+        {
             const int total_kb = ((num_tiles - 1 - unit0) / unit_step + 1) * k_blocks;
             bool ok = true;
-            for (int n = lane; n < total_kb; n += kProducerLanes) {
-                const int tile = unit0 + (n / k_blocks) * unit_step;
-                const int kb = n % k_blocks;
-                const int n0 = (tile / p.m_tiles) * (kTileN * CTAS) + (int)cta_rank * kTileN;
-                const int ps = n % p.stages_p;
-                const uint32_t pph = (uint32_t)((n / p.stages_p) & 1);
-                ok = mbar_wait(smem_u32(&s_empty_p[ps]), pph ^ 1u, abort_flag, p.watchdog, kWdProducer);
+            int ps = 0, kb = 0, tile = unit0;
+            uint32_t pph = 0;
+            int n0 = (tile / p.m_tiles) * (kTileN * CTAS) + (int)cta_rank * kTileN;
+            bool peek = false;
+            for (int n = 0; n < total_kb; ++n) {
+                ok = mbar_wait_all(smem_u32(&s_empty_p[ps]), pph ^ 1u, abort_flag, p.watchdog, kWdProducer, peek);
                 if (!ok) break;
-                const uint32_t bar = smem_u32(&s_full_p[ps]);
-                mbar_arrive_expect_tx(bar, pk_bytes);
-                tma_load_2d(smem_p + ps * pk_bytes, &map_w, kb * (kBlockK / 2), n0, bar);
+                {
+                    const int s1 = ps + 1 == p.stages_p ? 0 : ps + 1;
+                    const uint32_t ph1 = s1 == 0 ? pph ^ 1u : pph;
+                    peek = n + 1 < total_kb && mbar_test_wait(smem_u32(&s_empty_p[s1]), ph1 ^ 1u);
+                }
+                if (elect_one()) {
+                    const uint32_t bar = smem_u32(&s_full_p[ps]);
+                    mbar_arrive_expect_tx(bar, pk_bytes);
+                    tma_load_2d(smem_p + ps * pk_bytes, &map_w, kb * (kBlockK / 2), n0, bar);
+                }
+                if (++ps == p.stages_p) { ps = 0; pph ^= 1u; }
+                if (++kb == k_blocks) {
+                    kb = 0;
+                    tile += unit_step;
+                    n0 = (tile / p.m_tiles) * (kTileN * CTAS) + (int)cta_rank * kTileN;
+                }
             }
-            if (!ok) drain_after_abort();
+            if (!ok && lane == 0) drain_after_abort();
         }
     }
 
@@ -749,6 +915,10 @@ fq_status launch_gemm_tcgen05(const int8_t* a8, int64_t M, const Weights& W, int
         if (sa < 2) return FQ_ERR_UNSUPPORTED;
         int sp = (int)((budget - sa * a_bytes) / pk_bytes);
         if (sp > kMaxStagesP) sp = kMaxStagesP;
+        if (stages_w > sa) {            // the unpack warps wait on the activation ring's barriers
+            stages_w = sa;
+            p.stages_w = sa;
+        }
         p.stages = sa;
         p.stages_p = sp;
         smem = sa * a_bytes + sp * pk_bytes + epi_bytes + 1024;
@@ -779,3 +949,9 @@ fq_status launch_gemm_tcgen05(const int8_t* a8, int64_t M, const Weights& W, int
 }
 
 }  // namespace fq
+
+#ifdef FQ_GEMM_TRACE
+extern "C" int fq_debug_trace(unsigned long long* out) {
+    return (int)cudaMemcpyFromSymbol(out, fq::g_trace, sizeof(fq::g_trace));
+}
+#endif
