@@ -21,6 +21,7 @@
 #include <float.h>
 
 #include "fq_common.cuh"
+#include "ptx_sm100.cuh"
 #include "act_common.cuh"
 
 namespace fq {
@@ -83,6 +84,8 @@ transform_quantize_kernel(const XT* __restrict__ x, int64_t rows, int K, int64_t
                           int tpr, int rpc) {
     __shared__ float s_part[2][32];   // per-warp partial maxima, double buffered
 
+    griddep_wait();                   // launched with programmatic serialization: see launch_pdl
+    griddep_launch_dependents();
     const int tid = threadIdx.x;
     const int lane = tid & 31;
     const int warp = tid >> 5;
@@ -249,8 +252,8 @@ cudaError_t launch_e(const XT* x, int64_t rows, int K, int64_t ldx, const float*
             resident = 1;
         int64_t grid = iters < (int64_t)sms * resident ? iters : (int64_t)sms * resident;
         if (grid < 1) grid = 1;
-        kern<<<(unsigned)grid, threads, 0, stream>>>(x, rows, K, ldx, mult, cnorm, block, (float)qmax, clip_ratio,
-                                                     static_cast<uint8_t*>(codes), delta, tpr, rpc);
+        launch_pdl(kern, (unsigned)grid, (unsigned)threads, 0, stream, 1u, x, rows, K, ldx, mult, cnorm, block, (float)qmax,
+                   clip_ratio, static_cast<uint8_t*>(codes), delta, tpr, rpc);
     };
     const bool clamp = clip_ratio < 1.0f;
     if (threads <= 512) {

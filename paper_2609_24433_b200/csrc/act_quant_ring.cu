@@ -107,6 +107,8 @@ transform_quantize_ring_kernel(const __grid_constant__ CUtensorMap map_x, const 
         fence_mbarrier_init();
         fence_proxy_async_smem();
     }
+    griddep_wait();                  // the kernel before this one may still be writing x (or reading codes)
+    griddep_launch_dependents();
     if (p.mult != nullptr) {
         // Stage the multiplier with its 16-byte pieces XOR-swizzled by the index of the thread slice
         // (E floats) they belong to, so that the slice-per-thread reads below are bank-conflict free.
@@ -324,8 +326,7 @@ cudaError_t launch_ring(const CUtensorMap& map, const RingParams& p, int grid, s
     auto go = [&](auto kern) -> cudaError_t {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        kern<<<grid, kThreads, smem, stream>>>(map, p);
-        return cudaGetLastError();
+        return launch_pdl(kern, (unsigned)grid, (unsigned)kThreads, smem, stream, 1u, map, p);
     };
     if (p.clip_ratio < 1.0f) return go(transform_quantize_ring_kernel<XT, FMT, true, E, BLOCK>);
     return go(transform_quantize_ring_kernel<XT, FMT, false, E, BLOCK>);

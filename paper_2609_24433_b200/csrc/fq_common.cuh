@@ -26,6 +26,33 @@ struct Weights {
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+// Launch with programmatic stream serialization (the kernel must call griddep_wait() before its first
+// global-memory access) and, optionally, a thread-block cluster along x.
+template <typename Kern, typename... Args>
+inline cudaError_t launch_pdl(Kern kern, unsigned grid, unsigned block, size_t smem, cudaStream_t stream,
+                              unsigned cluster_x, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid, 1, 1);
+    cfg.blockDim = dim3(block, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    unsigned n = 0;
+    attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[n].val.programmaticStreamSerializationAllowed = 1;
+    ++n;
+    if (cluster_x > 1) {
+        attr[n].id = cudaLaunchAttributeClusterDimension;
+        attr[n].val.clusterDim.x = cluster_x;
+        attr[n].val.clusterDim.y = 1;
+        attr[n].val.clusterDim.z = 1;
+        ++n;
+    }
+    cfg.attrs = attr;
+    cfg.numAttrs = n;
+    return cudaLaunchKernelEx(&cfg, kern, args...);
+}
+
 // ---- launchers (host side, defined next to their kernels) -------------------
 // Int8Perm: one int8 per code, but every group of 8 channels stored as (c0,c2,c4,c6,c1,c3,c5,c7) --
 // the order in which the GEMM's nibble unpack produces the 4-bit weights without a byte permute.

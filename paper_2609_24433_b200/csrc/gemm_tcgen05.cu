@@ -32,6 +32,9 @@
 // Every mbarrier wait is bounded by wall-clock time; on expiry the CTA records a
 // code in the watchdog word, stops issuing work, and still frees its TMEM.
 #include <cuda_bf16.h>
+#if defined(FQ_GEMM_TRACE) || defined(FQ_GEMM_DEV)
+#include <cstdlib>
+#endif
 
 #include "fq_common.cuh"
 #include "ptx_sm100.cuh"
@@ -74,13 +77,13 @@ constexpr int kMaxStages = 8;
 constexpr int kMaxStagesP = 16;
 
 // Timeline hooks for kernel development: with -DFQ_GEMM_TRACE the first CTA records clock64() at
-// the marked points of the first 128 k-blocks (agent 0 activation producer, 2 unpack, 3 MMA
+// the marked points of the first 1024 k-blocks (agent 0 activation producer, 2 unpack, 3 MMA
 // issuer) and fq_debug_trace() copies the table out.  Compiled out by default.
 #ifdef FQ_GEMM_TRACE
-__device__ unsigned long long g_trace[4 * 128 * 4];
+__device__ unsigned long long g_trace[4 * 1024 * 4];
 #define FQ_TRACE(agent, n, e)                                                                   \
     do {                                                                                        \
-        if (blockIdx.x == 0 && lane == 0 && (n) < 128) g_trace[((agent) * 128 + (n)) * 4 + (e)] = clock64(); \
+        if (blockIdx.x == 0 && lane == 0 && (n) < 1024) g_trace[((agent) * 1024 + (n)) * 4 + (e)] = clock64(); \
     } while (0)
 #else
 #define FQ_TRACE(agent, n, e) do { } while (0)
@@ -99,6 +102,9 @@ struct Params {
     const float* bias;
     GemmOut out;
     uint32_t* watchdog;
+#if defined(FQ_GEMM_TRACE) || defined(FQ_GEMM_DEV)
+    int dbg;             // development builds: switches that skip parts of the epilogue
+#endif
 };
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
@@ -401,6 +407,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     if (CTAS == 2) cluster_sync_all();              // the peer's barriers exist before anyone signals them
     tc_fence_after();
     const uint32_t tmem_base = s_tmem_base;
+    // Everything above is on-chip setup; from here on global memory is touched (activations written
+    // by the kernel before this one, outputs that it may still be reading).
+    griddep_wait();
+    griddep_launch_dependents();
 
     // work units: (super-tile of 128*CTAS channels) x (token tile); one unit per CTA or CTA pair at a time
     const int num_tiles = p.m_tiles * p.n_tiles;
@@ -548,7 +558,13 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                 const int64_t tc = t0 + c;
                 if (tc >= p.M) break;                    // tokens beyond M: nothing to store (warp-uniform)
                 uint32_t r[16];
+#if defined(FQ_GEMM_TRACE) || defined(FQ_GEMM_DEV)
+                if (p.dbg & 4) continue;
+#endif
                 tmem_ld16(taddr + (uint32_t)c, r);
+#if defined(FQ_GEMM_TRACE) || defined(FQ_GEMM_DEV)
+                if (p.dbg & 2) { tmem_ld_wait(); if (r[0] == 0x12345678u && r[7] == 0x9abcdef0u) p.watchdog[1] = 1; continue; }
+#endif
                 if (p.out.acc != nullptr) {
                     tmem_ld_wait();
 #pragma unroll
@@ -582,6 +598,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                         const int row = (lane >> 2) + 8 * k;
                         const int64_t jj = jq + (lane & 3) * 8;
                         const uint4 v = *reinterpret_cast<const uint4*>(xpose + row * 64 + (lane & 3) * 16);
+#if defined(FQ_GEMM_TRACE) || defined(FQ_GEMM_DEV)
+                        if ((p.dbg & 1) && v.x != 0x12345678u) continue;
+#endif
                         if (tc + row < p.M && jj < p.N)
                             *reinterpret_cast<uint4*>(y + (tc + row) * p.out.ldy + jj) = v;
                     }
@@ -841,19 +860,8 @@ fq_status launch_variant(const CUtensorMap& map_a, const CUtensorMap& map_w, con
     auto kern = gemm_tcgen05_kernel<BITS, CTAS>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return FQ_ERR_CUDA;
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)grid, 1, 1);
-    cfg.blockDim = dim3(BITS == 4 ? kThreadsW4 : kThreadsW8, 1, 1);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = CTAS;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = CTAS == 2 ? 1 : 0;
-    return cudaLaunchKernelEx(&cfg, kern, map_a, map_w, p) == cudaSuccess ? FQ_OK : FQ_ERR_CUDA;
+    return launch_pdl(kern, (unsigned)grid, (unsigned)(BITS == 4 ? kThreadsW4 : kThreadsW8), smem, stream, (unsigned)CTAS,
+                      map_a, map_w, p) == cudaSuccess ? FQ_OK : FQ_ERR_CUDA;
 }
 
 }  // namespace
@@ -885,11 +893,17 @@ fq_status launch_gemm_tcgen05(const int8_t* a8, int64_t M, const Weights& W, int
         const double cost = (double)((tiles + sms - 1) / sms) * (c0 + c1 * b);
         if (bt == 0 || cost < best * 0.97) { bt = b; best = cost; }   // prefer larger tiles unless clearly cheaper
     }
+#if defined(FQ_GEMM_TRACE) || defined(FQ_GEMM_DEV)
+    if (const char* e = getenv("FQ_BT")) bt = atoi(e);      // development builds: force the token tile
+#endif
     p.bt = bt;
     p.m_tiles = (int)((M + bt - 1) / bt);
     // CTA pairs for large 8-bit problems (measured +9 % at 8192^3; no gain for the 4-bit path, whose
     // weights never pass through shared memory, nor for short token batches).
     int ctas = (W.bits == 8 && W.N > kTileN && bt >= 128 && M >= 1024) ? 2 : 1;
+#if defined(FQ_GEMM_TRACE) || defined(FQ_GEMM_DEV)
+    if (const char* e = getenv("FQ_PAIR")) ctas = atoi(e);   // development builds: force single CTAs or pairs
+#endif
     p.n_tiles = (int)((W.N + kTileN * ctas - 1) / (kTileN * ctas));
     p.acc_shift = acc_shift;
     p.w_scale = W.w_scale;
@@ -897,6 +911,9 @@ fq_status launch_gemm_tcgen05(const int8_t* a8, int64_t M, const Weights& W, int
     p.out = out;
     p.watchdog = watchdog_device_ptr();
     if (!p.watchdog) return FQ_ERR_CUDA;
+#if defined(FQ_GEMM_TRACE) || defined(FQ_GEMM_DEV)
+    p.dbg = getenv("FQ_DBG") ? atoi(getenv("FQ_DBG")) : 0;
+#endif
     // 4-bit weights: every TMEM column the accumulators leave free becomes unpacked-weight ring
     int stages_w = W.bits == 4 ? (512 - kAccStages * bt) / kColsW : 0;
     if (stages_w > kMaxStagesW) stages_w = kMaxStagesW;

@@ -143,6 +143,16 @@ __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, vo
     return __shfl_sync(0xffffffffu, ok, 0) != 0;
 }
 
+// Programmatic dependent launch.  A kernel launched with the programmatic-serialization attribute
+// may start while the kernel before it in the stream is still running; griddep_wait() returns once
+// that kernel has completed and its writes are visible, so everything that touches global memory
+// comes after it and only on-chip setup (barriers, TMEM, descriptor prefetch) runs ahead.
+// griddep_launch_dependents() lets the NEXT kernel in the stream begin its own setup early.
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void griddep_launch_dependents() {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
 __device__ __forceinline__ void fence_proxy_async_smem() {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
