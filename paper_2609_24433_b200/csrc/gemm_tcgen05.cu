@@ -876,34 +876,38 @@ fq_status launch_gemm_tcgen05(const int8_t* a8, int64_t M, const Weights& W, int
     int dev = 0, sms = 148;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    // Token tile.  Upper bound from TMEM: two accumulator stages, plus the unpacked-weight ring for
-    // 4-bit weights (2*bt + 3*32 <= 512 columns).  M is split evenly over m_tiles so that ragged M
-    // wastes little, and m_tiles is chosen by a small cost model: rounds of tiles over the SMs times
-    // the measured time of a 128-wide k-block, which is roughly c0 + c1*bt cycles (a large fixed part:
-    // smaller tiles are nearly as fast per k-block, so filling all SMs in one round wins).
+    // Token tile and CTA grouping.  Upper bound of the tile from TMEM: two accumulator stages, plus the
+    // unpacked-weight ring for 4-bit weights (2*bt + 3*32 <= 512 columns).  M is split evenly over
+    // m_tiles so that ragged M wastes little.  Candidates are ranked by a cost model fitted to
+    // measured launches (cycles): rounds of work units over the SMs, each unit costing
+    //     k_blocks * per_kblock(bt) + 16*bt + 1000          (the tail: epilogue and tile hand-over)
+    //   4-bit weights:          per_kblock = 330 + bt       (issue floor, then the MMAs' 2*bt)
+    //   8-bit, one CTA:         per_kblock = 300 + 2*bt     (shared-memory bound: both operands pass through it)
+    //   8-bit, CTA pair:        per_kblock = max(545, 2.62*bt)   (each CTA stages half of the token tile)
+    // Pairs gain nothing for 4-bit weights, which never pass through shared memory unpacked.
     const int bt_max = W.bits == 4 ? 208 : 256;
-    const double c0 = W.bits == 4 ? 920.0 : 500.0, c1 = W.bits == 4 ? 1.3 : 1.8;
-    const int64_t n128 = (W.N + kTileN - 1) / kTileN;
-    int bt = 0;
+    const int64_t k_blocks_host = (W.K + kBlockK - 1) / kBlockK;
+    int bt = 0, ctas = 1;
     double best = 0.0;
-    for (int mt = (int)((M + bt_max - 1) / bt_max); mt <= (int)((M + 63) / 64); ++mt) {
-        const int b = (int)(((M + mt - 1) / mt + 15) / 16 * 16);
-        if (b > bt_max) continue;
-        const int64_t tiles = n128 * ((M + b - 1) / b);
-        const double cost = (double)((tiles + sms - 1) / sms) * (c0 + c1 * b);
-        if (bt == 0 || cost < best * 0.97) { bt = b; best = cost; }   // prefer larger tiles unless clearly cheaper
+    for (int c = 1; c <= ((W.bits == 8 && W.N > kTileN) ? 2 : 1); ++c) {
+        const int64_t n_units = (W.N + kTileN * c - 1) / (kTileN * c);
+        const int slots = sms / c;
+        for (int mt = (int)((M + bt_max - 1) / bt_max); mt <= (int)((M + 63) / 64); ++mt) {
+            const int b = (int)(((M + mt - 1) / mt + 15) / 16 * 16);
+            if (b > bt_max) continue;
+            const int64_t units = n_units * ((M + b - 1) / b);
+            const double per_kb = W.bits == 4 ? 330.0 + b
+                                  : (c == 1 ? 300.0 + 2.0 * b : (2.62 * b > 545.0 ? 2.62 * b : 545.0));
+            const double cost = (double)((units + slots - 1) / slots) * ((double)k_blocks_host * per_kb + 16.0 * b + 1000.0);
+            if (bt == 0 || cost < best * 0.98) { bt = b; ctas = c; best = cost; }   // ties: the earlier (larger) tile
+        }
     }
 #if defined(FQ_GEMM_TRACE) || defined(FQ_GEMM_DEV)
     if (const char* e = getenv("FQ_BT")) bt = atoi(e);      // development builds: force the token tile
+    if (const char* e = getenv("FQ_PAIR")) ctas = atoi(e);   // ... and single CTAs or pairs
 #endif
     p.bt = bt;
     p.m_tiles = (int)((M + bt - 1) / bt);
-    // CTA pairs for large 8-bit problems (measured +9 % at 8192^3; no gain for the 4-bit path, whose
-    // weights never pass through shared memory, nor for short token batches).
-    int ctas = (W.bits == 8 && W.N > kTileN && bt >= 128 && M >= 1024) ? 2 : 1;
-#if defined(FQ_GEMM_TRACE) || defined(FQ_GEMM_DEV)
-    if (const char* e = getenv("FQ_PAIR")) ctas = atoi(e);   // development builds: force single CTAs or pairs
-#endif
     p.n_tiles = (int)((W.N + kTileN * ctas - 1) / (kTileN * ctas));
     p.acc_shift = acc_shift;
     p.w_scale = W.w_scale;
