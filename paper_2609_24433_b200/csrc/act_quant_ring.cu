@@ -107,18 +107,9 @@ transform_quantize_ring_kernel(const __grid_constant__ CUtensorMap map_x, const 
         fence_mbarrier_init();
         fence_proxy_async_smem();
     }
+    __syncthreads();                 // barriers initialised before any copy is issued
     griddep_wait();                  // the kernel before this one may still be writing x (or reading codes)
     griddep_launch_dependents();
-    if (p.mult != nullptr) {
-        // Stage the multiplier with its 16-byte pieces XOR-swizzled by the index of the thread slice
-        // (E floats) they belong to, so that the slice-per-thread reads below are bank-conflict free.
-        for (int i = tid * 4; i < p.K; i += kThreads * 4) {
-            const float4 g4 = __ldg(reinterpret_cast<const float4*>(p.mult + i));
-            const uint32_t off = (uint32_t)i * 4u;
-            *reinterpret_cast<float4*>(gen + (off ^ (((off / (E * 4u)) & 7u) << 4))) = g4;
-        }
-    }
-    __syncthreads();
 
     const int first = (int)blockIdx.x * ngroups + group;     // rows < 2^31 (checked by the launcher)
     const int step = (int)gridDim.x * ngroups;
@@ -127,6 +118,8 @@ transform_quantize_ring_kernel(const __grid_constant__ CUtensorMap map_x, const 
     const uint32_t slot0 = base + slots_off + (uint32_t)(group * p.depth) * p.slot_bytes;
     uint64_t* full0 = &s_full[group * p.depth];
 
+    // The first rows are requested before the multiplier is staged, so that their flight time
+    // overlaps the staging loop.
     int issued = 0;          // rows requested by this group's leader
     if (leader) {
         for (int d = 0; d < p.depth; ++d) {
@@ -138,6 +131,16 @@ transform_quantize_ring_kernel(const __grid_constant__ CUtensorMap map_x, const 
             }
         }
     }
+    if (p.mult != nullptr) {
+        // Stage the multiplier with its 16-byte pieces XOR-swizzled by the index of the thread slice
+        // (E floats) they belong to, so that the slice-per-thread reads below are bank-conflict free.
+        for (int i = tid * 4; i < p.K; i += kThreads * 4) {
+            const float4 g4 = __ldg(reinterpret_cast<const float4*>(p.mult + i));
+            const uint32_t off = (uint32_t)i * 4u;
+            *reinterpret_cast<float4*>(gen + (off ^ (((off / (E * 4u)) & 7u) << 4))) = g4;
+        }
+    }
+    __syncthreads();
 
     // swizzled starts of the (up to two) 128-byte lines of this thread's slices
     const uint32_t xs0 = swz128((uint32_t)col0 * (uint32_t)sizeof(XT));
@@ -150,7 +153,7 @@ transform_quantize_ring_kernel(const __grid_constant__ CUtensorMap map_x, const 
     int n = 0, d = 0;
     uint32_t ph = 0;
     for (int row = first; row < rows; row += step, ++n) {
-        bool ok = mbar_wait_warp(smem_u32(&full0[d]), ph, abort_flag, p.watchdog, 0x100u);
+        bool ok = mbar_wait_all(smem_u32(&full0[d]), ph, abort_flag, p.watchdog, 0x100u);   // every lane polls: cheaper than one lane + broadcast
 
         float2 v[H];
         const uint8_t* slot = gen + slots_off + (size_t)(group * p.depth + d) * p.slot_bytes;
