@@ -414,10 +414,16 @@ def workload_sites(name: str):
         return synth.backbone_layer_sites(selective_int8=False)
     if name == "expert_layer":
         return synth.expert_layer_sites()
+    if name.startswith("sweep:"):        # one site of the throughput sweep: sweep:M,K,N,block,bits
+        M, K, N, beta, bits = (int(v) for v in name[6:].split(","))
+        return [synth.sweep_site(M, K, N, beta, bits)]
     raise ValueError(name)
 
 
 def workload_name(name: str) -> str:
+    if name.startswith("sweep:"):
+        M, K, N, beta, bits = (int(v) for v in name[6:].split(","))
+        return f"throughput sweep point M={M} K={K} N={N}, block {beta}, W{bits}A{bits}"
     return {"backbone_layer": "pi0.5-like backbone layer, M=816, hidden 2048, MLP 16384, o/down W8A8, rest W4A4",
             "backbone_layer_w4": "pi0.5-like backbone layer, M=816, uniform W4A4",
             "expert_layer": "action-expert layer, M=50, width 1024, MLP 4096, W4A4, block 64"}[name]

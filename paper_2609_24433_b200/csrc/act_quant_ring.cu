@@ -111,7 +111,7 @@ transform_quantize_ring_kernel(const __grid_constant__ CUtensorMap map_x, const 
     griddep_wait();                  // the kernel before this one may still be writing x (or reading codes)
     griddep_launch_dependents();
 
-    const int first = (int)blockIdx.x * ngroups + group;     // rows < 2^31 (checked by the launcher)
+    const int first = group * (int)gridDim.x + (int)blockIdx.x;   // rows < 2^31 (checked by the launcher)
     const int step = (int)gridDim.x * ngroups;
     const int rows = (int)p.rows;
     const uint32_t tx = (uint32_t)p.K * (uint32_t)sizeof(XT);
@@ -397,8 +397,9 @@ cudaError_t launch_transform_quantize_ring(const void* x, fq_dtype xt, int64_t r
     p.watchdog = watchdog_device_ptr();
     if (!p.watchdog) return cudaErrorUnknown;
     const size_t smem = g_bytes + slot * ngroups * depth + 1024;
-    const int64_t need = (rows + ngroups - 1) / ngroups;
-    const int grid = (int)(need < sms ? need : sms);
+    // Rows are dealt to the CTAs first and to a CTA's row groups second (row r -> CTA r % grid),
+    // so that a short batch spreads over all SMs instead of filling every group of a few CTAs.
+    const int grid = (int)(rows < sms ? rows : sms);
     if (xt == FQ_BF16)
     {
         if (fmt == StoreFmt::Nibble) return launch_ring_e<__nv_bfloat16, 0>(e, block, map, p, grid, smem, stream);
