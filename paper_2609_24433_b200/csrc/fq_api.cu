@@ -77,6 +77,16 @@ fq_status carve(void* workspace, size_t ws_bytes, int64_t M, int64_t K, Workspac
     return FQ_OK;
 }
 
+// Whatever the caller's workspace holds beyond the activation codes and steps serves the GEMM as
+// scratch for partial tiles (K split); without it the GEMM simply does not split.
+void* scratch_of(void* workspace, size_t ws_bytes, int64_t M, int64_t K, size_t* avail) {
+    const size_t base = ws_bytes_needed(M, K);
+    *avail = 0;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0 || ws_bytes <= base) return nullptr;
+    *avail = ws_bytes - base;
+    return static_cast<uint8_t*>(workspace) + base;
+}
+
 fq_status check_y(const void* y, fq_dtype yt, int64_t ldy, int64_t N) {
     if (!y) return FQ_ERR_INVALID_ARG;
     if (yt != FQ_F32 && yt != FQ_BF16) return FQ_ERR_INVALID_ARG;
@@ -107,7 +117,9 @@ fq_status gemm_from_codes(const void* a_codes, const float* a_delta, int64_t M, 
         shift = 8;   // both operands carry 16*code
     }
     if (simt) return launch_gemm_simt(a8, M, *W, shift, out, stream) == cudaSuccess ? FQ_OK : FQ_ERR_CUDA;
-    return launch_gemm_tcgen05(a8, M, *W, shift, out, stream);
+    size_t scratch_bytes = 0;
+    void* scratch = scratch_of(workspace, ws_bytes, M, W->K, &scratch_bytes);
+    return launch_gemm_tcgen05(a8, M, *W, shift, out, scratch, scratch_bytes, stream);
 }
 
 fq_status linear_impl(const void* x, fq_dtype xt, int64_t M, int64_t ldx, const fq_weights* Wp, int bits,
@@ -146,7 +158,9 @@ fq_status linear_impl(const void* x, fq_dtype xt, int64_t M, int64_t ldx, const 
     GemmOut out;
     out.y = y; out.yt = yt; out.ldy = ldy; out.a_delta = ws.delta;
     // 4-bit weights are expanded to 16*code on chip: accumulator = 16 * integer sum.
-    return launch_gemm_tcgen05(ws.a8, M, *W, bits == 4 ? 4 : 0, out, s);
+    size_t scratch_bytes = 0;
+    void* scratch = scratch_of(workspace, ws_bytes, M, W->K, &scratch_bytes);
+    return launch_gemm_tcgen05(ws.a8, M, *W, bits == 4 ? 4 : 0, out, scratch, scratch_bytes, s);
 }
 
 }  // namespace
@@ -354,9 +368,8 @@ fq_status fq_linear_w8a8(const void* x, fq_dtype xt, int64_t M, int64_t ldx, con
 }
 
 size_t fq_workspace_bytes(int64_t M, int64_t K, int64_t N, int bits) {
-    (void)N; (void)bits;
     if (M <= 0 || K <= 0) return 256;
-    return ws_bytes_needed(M, K);
+    return ws_bytes_needed(M, K) + align_up(gemm_scratch_bytes(M, N, K, bits == 4 ? 4 : 8), 256);
 }
 
 fq_status fq_gemm_acc_i32(const void* a_codes, int64_t M, const fq_weights* W, int32_t* acc, void* workspace,

@@ -91,9 +91,12 @@ struct GemmOut {
 cudaError_t launch_gemm_simt(const int8_t* a8, int64_t M, const Weights& W, int acc_shift, const GemmOut& out,
                              cudaStream_t stream);
 
-// tcgen05 integer GEMM; a8 = int8 activations [M, K] (pitch K), 16-byte aligned.
+// tcgen05 integer GEMM; a8 = int8 activations [M, K] (pitch K), 16-byte aligned.  `scratch` (device,
+// 256-byte aligned, may be null) holds int32 partial tiles when the launch splits K over a cluster;
+// gemm_scratch_bytes() is what the split the planner would pick for this shape needs.
 fq_status launch_gemm_tcgen05(const int8_t* a8, int64_t M, const Weights& W, int acc_shift, const GemmOut& out,
-                              cudaStream_t stream);
+                              void* scratch, size_t scratch_bytes, cudaStream_t stream);
+size_t gemm_scratch_bytes(int64_t M, int64_t N, int64_t K, int bits);
 
 // cuTensorMapEncodeTiled through the runtime's driver entry point (no link-time libcuda dependency).
 // dims/box innermost first; strides_bytes has rank-1 entries (dimension 0 is contiguous).

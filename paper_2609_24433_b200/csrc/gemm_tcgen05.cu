@@ -33,6 +33,7 @@
 // code in the watchdog word, stops issuing work, and still frees its TMEM.
 #include <cuda_bf16.h>
 #if defined(FQ_GEMM_TRACE) || defined(FQ_GEMM_DEV)
+#include <cstdio>
 #include <cstdlib>
 #endif
 
@@ -85,8 +86,13 @@ __device__ unsigned long long g_trace[4 * 1024 * 4];
     do {                                                                                        \
         if (blockIdx.x == 0 && lane == 0 && (n) < 1024) g_trace[((agent) * 1024 + (n)) * 4 + (e)] = clock64(); \
     } while (0)
+#define FQ_TRACE_B(blk, agent, n, e)                                                            \
+    do {                                                                                        \
+        if (blockIdx.x == (blk) && lane == 0 && (n) < 1024) g_trace[((agent) * 1024 + (n)) * 4 + (e)] = clock64(); \
+    } while (0)
 #else
 #define FQ_TRACE(agent, n, e) do { } while (0)
+#define FQ_TRACE_B(blk, agent, n, e) do { } while (0)
 #endif
 
 struct Params {
@@ -102,6 +108,8 @@ struct Params {
     const float* bias;
     GemmOut out;
     uint32_t* watchdog;
+    int split;           // CTAs of a cluster sharing one tile, each on its own slice of K (1 = no split)
+    int32_t* partials;   // [tile][split][bt tokens][128 channels] int32: raw sums a rank hands to the chunks' owners
 #if defined(FQ_GEMM_TRACE) || defined(FQ_GEMM_DEV)
     int dbg;             // development builds: switches that skip parts of the epilogue
 #endif
@@ -338,14 +346,14 @@ __device__ __forceinline__ void drain_after_abort() {
 
 enum : uint32_t {
     kWdProducer = 1u, kWdMmaFull = 2u, kWdMmaAcc = 4u, kWdEpilogue = 8u, kWdUnpackFull = 16u,
-    kWdUnpackEmpty = 32u, kWdDrain = 64u
+    kWdUnpackEmpty = 32u, kWdDrain = 64u, kWdPartials = 128u
 };
 
 // CTAS = 2: two CTAs of a cluster work as a pair on a 256-channel x bt-token tile (cta_group::2):
 // each loads its own 128 weight rows and HALF of the token tile, the even CTA issues the MMAs for
 // both, and every MMA reads the token halves out of both CTAs' shared memory.  This halves the
 // activation bytes each SM pulls from L2, which is what bounds the single-CTA kernel.
-template <int BITS, int CTAS>
+template <int BITS, int CTAS, bool SPLIT>
 __global__ void __launch_bounds__(BITS == 4 ? kThreadsW4 : kThreadsW8, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_w,
                     const Params p) {
@@ -358,6 +366,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     __shared__ uint64_t s_full_w8[kMaxStagesW];     // unpacked weights written
     __shared__ uint64_t s_acc_full[kAccStages];
     __shared__ uint64_t s_acc_empty[kAccStages];
+    __shared__ uint64_t s_part_full[kAccStages];    // K split: the other ranks' partial sums for this tile are written
+    __shared__ uint64_t s_part_empty[kAccStages];   // K split: the other ranks have taken my sums of the tile before last
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_abort;
 
@@ -366,6 +376,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     volatile int* abort_flag = &s_abort;
     const uint32_t cta_rank = CTAS == 2 ? cluster_ctarank() : 0u;
     const bool leader = cta_rank == 0;
+    // K split (single CTAs only): the cluster's ranks work on the same tiles, rank r on k-blocks [kb0, kb0 + k_blocks)
+    const int split = (SPLIT && CTAS == 1) ? p.split : 1;   // compile-time 1 in the common instantiation
+    const uint32_t krank = split > 1 ? cluster_ctarank() : 0u;
     const int bt_cta = p.bt / CTAS;                 // token rows this CTA loads
 
     // carve dynamic shared memory: [A8 stages][W8 stages][packed stages][epilogue transposers], 1024-byte aligned
@@ -397,6 +410,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         for (int a = 0; a < kAccStages; ++a) {
             mbar_init(smem_u32(&s_acc_full[a]), 1);
             mbar_init(smem_u32(&s_acc_empty[a]), kEpiWarps * CTAS);
+            mbar_init(smem_u32(&s_part_full[a]), (uint32_t)(kEpiWarps * (split > 1 ? split - 1 : 1)));
+            mbar_init(smem_u32(&s_part_empty[a]), (uint32_t)(kEpiWarps * (split > 1 ? split - 1 : 1)));
         }
         fence_mbarrier_init();
         fence_proxy_async_smem();
@@ -404,7 +419,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     if (warp == 1) tmem_alloc<CTAS>(smem_u32(&s_tmem_base), (uint32_t)p.tmem_cols);
     tc_fence_before();
     __syncthreads();
-    if (CTAS == 2) cluster_sync_all();              // the peer's barriers exist before anyone signals them
+    if (CTAS == 2 || split > 1) cluster_sync_all(); // the peers' barriers exist before anyone signals them
     tc_fence_after();
     const uint32_t tmem_base = s_tmem_base;
     // Everything above is on-chip setup; from here on global memory is touched (activations written
@@ -414,9 +429,13 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
 
     // work units: (super-tile of 128*CTAS channels) x (token tile); one unit per CTA or CTA pair at a time
     const int num_tiles = p.m_tiles * p.n_tiles;
-    const int unit0 = (int)blockIdx.x / CTAS;
-    const int unit_step = (int)gridDim.x / CTAS;
-    const int k_blocks = (int)((p.K + kBlockK - 1) / kBlockK);
+    const int cluster_ctas = CTAS == 2 ? 2 : split;
+    const int unit0 = (int)blockIdx.x / cluster_ctas;
+    const int unit_step = (int)gridDim.x / cluster_ctas;
+    const int k_blocks_all = (int)((p.K + kBlockK - 1) / kBlockK);
+    const int kb_per = (k_blocks_all + split - 1) / split;
+    const int kb0 = (int)krank * kb_per;                               // first k-block of this rank
+    const int k_blocks = kb0 + kb_per <= k_blocks_all ? kb_per : k_blocks_all - kb0;   // >= 1 (host check)
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
@@ -444,11 +463,11 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                     const uint32_t bar = smem_u32(&s_full_tma[stage]);
                     if (CTAS == 1) {
                         mbar_arrive_expect_tx(bar, tx);
-                        tma_load_2d(smem_a + stage * a_bytes, &map_a, kb * kBlockK, t0, bar);
+                        tma_load_2d(smem_a + stage * a_bytes, &map_a, (kb0 + kb) * kBlockK, t0, bar);
                     } else {
                         // the pair's bytes are all counted on the even CTA's barrier, which it arms for both
                         if (leader) mbar_arrive_expect_tx(bar, tx * CTAS);
-                        tma_load_2d_pair(smem_a + stage * a_bytes, &map_a, kb * kBlockK, t0, bar);
+                        tma_load_2d_pair(smem_a + stage * a_bytes, &map_a, (kb0 + kb) * kBlockK, t0, bar);
                     }
                 }
                 FQ_TRACE(0, n, 1);
@@ -552,16 +571,66 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             }
             ok = mbar_wait_warp_relaxed(smem_u32(&s_acc_full[acc_stage]), acc_phase, abort_flag, p.watchdog, kWdEpilogue);
             if (!ok) break;
-            tc_fence_after();
+            if (warp == 2) { FQ_TRACE_B(0, 2, 0, 0); FQ_TRACE_B(1, 1, 0, 0); }
+            // K split.  Every rank finishes a share of the tile: this warp's k-th chunk of 16 tokens belongs
+            // to rank k % split.  A rank first hands the raw sums of the chunks it does not own to their
+            // owners (partial blocks [tile][writer rank][bt tokens][128 channels] int32: a warp's 32
+            // channels of one token are one 128-byte line, coalesced both ways), then waits for the
+            // other ranks' blocks and finishes its own chunks.
+            int32_t* part = nullptr;
             const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc_stage * p.bt);
+            if (split > 1) {
+                tc_fence_after();
+                part = p.partials + (size_t)tile * (size_t)split * kTileN * (size_t)p.bt + (size_t)(quad * 32 + lane);
+                // flow control: the other ranks' barriers for this accumulator stage must not be signalled
+                // for a new tile before they have passed them for the previous one (phases would alias)
+                ok = mbar_wait_warp_relaxed(smem_u32(&s_part_empty[acc_stage]), acc_phase ^ 1u, abort_flag, p.watchdog,
+                                            kWdPartials);
+                if (!ok) break;
+                int32_t* mine = part + (size_t)krank * kTileN * (size_t)p.bt;
+                for (int c = half * 16; c < p.bt; c += 32) {
+                    if (t0 + c >= p.M) break;
+                    if ((uint32_t)((c >> 5) % split) == krank) continue;
+                    uint32_t r[16];
+                    tmem_ld16(taddr + (uint32_t)c, r);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) __stcg(mine + (size_t)(c + i) * kTileN, (int)r[i]);
+                }
+                __threadfence();                 // partial sums visible before the owners are told
+                __syncwarp();
+                if (lane == 0)
+                    for (uint32_t rk = 0; rk < (uint32_t)split; ++rk)
+                        if (rk != krank) mbar_arrive_cta(smem_u32(&s_part_full[acc_stage]), rk);
+                ok = mbar_wait_warp_relaxed(smem_u32(&s_part_full[acc_stage]), acc_phase, abort_flag, p.watchdog, kWdPartials);
+                if (!ok) break;
+                __threadfence();
+            }
+            tc_fence_after();
+            if (warp == 2) { FQ_TRACE_B(0, 2, 0, 1); FQ_TRACE_B(1, 1, 0, 1); }
             for (int c = half * 16; c < p.bt; c += 32) {
                 const int64_t tc = t0 + c;
                 if (tc >= p.M) break;                    // tokens beyond M: nothing to store (warp-uniform)
+                if (split > 1 && (uint32_t)((c >> 5) % split) != krank) continue;   // another rank finishes this chunk
                 uint32_t r[16];
 #if defined(FQ_GEMM_TRACE) || defined(FQ_GEMM_DEV)
                 if (p.dbg & 4) continue;
 #endif
                 tmem_ld16(taddr + (uint32_t)c, r);
+                if (split > 1) {
+                    int32_t pv[16];
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) pv[i] = 0;
+                    for (uint32_t rk = 0; rk < (uint32_t)split; ++rk) {
+                        if (rk == krank) continue;
+                        const int32_t* src = part + ((size_t)rk * (size_t)p.bt + (size_t)c) * kTileN;
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) pv[i] += __ldcg(src + (size_t)i * kTileN);
+                    }
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) r[i] += (uint32_t)pv[i];
+                }
 #if defined(FQ_GEMM_TRACE) || defined(FQ_GEMM_DEV)
                 if (p.dbg & 2) { tmem_ld_wait(); if (r[0] == 0x12345678u && r[7] == 0x9abcdef0u) p.watchdog[1] = 1; continue; }
 #endif
@@ -619,6 +688,14 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                     }
                 }
             }
+            if (warp == 2) { FQ_TRACE_B(0, 2, 0, 2); FQ_TRACE_B(1, 1, 0, 2); }
+            if (split > 1) {
+                __syncwarp();
+                if (lane == 0)
+                    for (uint32_t rk = 0; rk < (uint32_t)split; ++rk)
+                        if (rk != krank) mbar_arrive_cta(smem_u32(&s_part_empty[acc_stage]), rk);
+            }
+            if (warp == 2) { FQ_TRACE_B(0, 2, 0, 3); FQ_TRACE_B(1, 1, 0, 3); }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) {
@@ -649,10 +726,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                     const uint32_t bar = smem_u32(&s_full_tma[stage]);
                     if (CTAS == 1) {
                         mbar_arrive_expect_tx(bar, w_bytes);
-                        tma_load_2d(smem_w + stage * w_bytes, &map_w, kb * kBlockK, n0, bar);
+                        tma_load_2d(smem_w + stage * w_bytes, &map_w, (kb0 + kb) * kBlockK, n0, bar);
                     } else {
                         if (leader) mbar_arrive_expect_tx(bar, w_bytes * CTAS);
-                        tma_load_2d_pair(smem_w + stage * w_bytes, &map_w, kb * kBlockK, n0, bar);
+                        tma_load_2d_pair(smem_w + stage * w_bytes, &map_w, (kb0 + kb) * kBlockK, n0, bar);
                     }
                 }
                 if (++stage == p.stages) { stage = 0; phase ^= 1u; }
@@ -758,7 +835,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                 if (elect_one()) {
                     const uint32_t bar = smem_u32(&s_full_p[ps]);
                     mbar_arrive_expect_tx(bar, pk_bytes);
-                    tma_load_2d(smem_p + ps * pk_bytes, &map_w, kb * (kBlockK / 2), n0, bar);
+                    tma_load_2d(smem_p + ps * pk_bytes, &map_w, (kb0 + kb) * (kBlockK / 2), n0, bar);
                 }
                 if (++ps == p.stages_p) { ps = 0; pph ^= 1u; }
                 if (++kb == k_blocks) {
@@ -774,7 +851,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     // ------------------------------------------------------------------ teardown
     tc_fence_before();
     __syncthreads();
-    if (CTAS == 2) cluster_sync_all();              // neither CTA leaves while the other may still signal it
+    if (CTAS == 2 || split > 1) cluster_sync_all(); // no CTA leaves while another may still signal it
     if (warp == 1) {
         tc_fence_after();
         tmem_dealloc<CTAS>(tmem_base, (uint32_t)p.tmem_cols);
@@ -854,58 +931,105 @@ fq_status build_weight_tmap(Weights& W) {
 
 namespace {
 
-template <int BITS, int CTAS>
+template <int BITS, int CTAS, bool SPLIT>
 fq_status launch_variant(const CUtensorMap& map_a, const CUtensorMap& map_w, const Params& p, int grid, size_t smem,
-                         cudaStream_t stream) {
-    auto kern = gemm_tcgen05_kernel<BITS, CTAS>;
+                         int cluster, cudaStream_t stream) {
+    auto kern = gemm_tcgen05_kernel<BITS, CTAS, SPLIT>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return FQ_ERR_CUDA;
-    return launch_pdl(kern, (unsigned)grid, (unsigned)(BITS == 4 ? kThreadsW4 : kThreadsW8), smem, stream, (unsigned)CTAS,
+    return launch_pdl(kern, (unsigned)grid, (unsigned)(BITS == 4 ? kThreadsW4 : kThreadsW8), smem, stream, (unsigned)cluster,
                       map_a, map_w, p) == cudaSuccess ? FQ_OK : FQ_ERR_CUDA;
 }
 
 }  // namespace
 
+namespace {
+
+struct Plan {
+    int bt = 0;       // tokens per tile
+    int ctas = 1;     // 2: CTA pairs on 256-channel tiles (cta_group::2)
+    int split = 1;    // >1: that many CTAs of a cluster share a tile, each taking a slice of K
+    size_t scratch = 0;   // bytes of int32 partial tiles the split needs
+};
+
+// Token tile, CTA grouping and K split.  Upper bound of the tile from TMEM: two accumulator stages,
+// plus the unpacked-weight ring for 4-bit weights (2*bt + 3*32 <= 512 columns).  M is split evenly
+// over m_tiles so that ragged M wastes little.  Candidates are ranked by a cost model fitted to
+// measured launches (cycles): rounds of work units over the SMs, each unit costing
+//     k_blocks * per_kblock(bt) + 16*bt + 1000          (the tail: epilogue and tile hand-over)
+//   4-bit weights:          per_kblock = 330 + bt       (issue floor, then the MMAs' 2*bt)
+//   8-bit, one CTA:         per_kblock = max(350 + 0.8*bt, 230 + 2*bt)   (issue floor, then shared memory:
+//                                        both operands pass through it)
+//   8-bit, CTA pair:        per_kblock = max(545, 2.62*bt)   (each CTA stages half of the token tile)
+// Pairs gain nothing for 4-bit weights, which never pass through shared memory unpacked.
+// K split (single CTAs only): problems with fewer tiles than SMs and a long K (down_proj at M = 816:
+// 64 tiles of 128 k-blocks) can run `split` CTAs per tile; the ranks exchange int32 partial sums through
+// scratch and each finishes a share of the tile (measured cost of the exchange: about 6000 + 40*bt
+// cycles, + 1500 per extra rank, so the split pays only for long K and few tiles).
+Plan plan_gemm(int64_t M, int64_t N, int64_t K, int bits, int sms, size_t scratch_avail) {
+    const int bt_max = bits == 4 ? 208 : 256;
+    const int64_t kb = (K + kBlockK - 1) / kBlockK;
+    Plan best;
+    double best_cost = 0.0;
+    for (int c = 1; c <= ((bits == 8 && N > kTileN) ? 2 : 1); ++c) {
+        const int64_t n_units = (N + kTileN * c - 1) / (kTileN * c);
+        for (int mt = (int)((M + bt_max - 1) / bt_max); mt <= (int)((M + 63) / 64); ++mt) {
+            const int b = (int)(((M + mt - 1) / mt + 15) / 16 * 16);
+            if (b > bt_max) continue;
+            const int64_t units = n_units * ((M + b - 1) / b);
+            const double w8_single = 350.0 + 0.8 * b > 230.0 + 2.0 * b ? 350.0 + 0.8 * b : 230.0 + 2.0 * b;
+            const double per_kb = bits == 4 ? 330.0 + b : (c == 1 ? w8_single : (2.62 * b > 545.0 ? 2.62 * b : 545.0));
+            for (int sp = 1; sp <= (c == 1 ? 8 : 1); sp *= 2) {
+                const int64_t kb_per = (kb + sp - 1) / sp;
+                if (sp > 1 && (kb_per * (sp - 1) >= kb || kb_per < 4 || units * sp > 2 * (int64_t)sms)) continue;
+                const size_t scratch = sp > 1 ? (size_t)units * sp * kTileN * b * sizeof(int32_t) : 0;
+                if (scratch > scratch_avail) continue;
+                const int slots = sms / (c * sp);
+                if (slots < 1) continue;
+                const double unit_cost = (double)kb_per * per_kb + 16.0 * b + 1000.0 + (sp > 1 ? 6000.0 + 40.0 * b + 1500.0 * (sp - 1) : 0.0);
+                const double cost = (double)((units + slots - 1) / slots) * unit_cost;
+                if (best.bt == 0 || cost < best_cost * 0.98) {   // ties: the earlier candidate (larger tile, no split)
+                    best.bt = b; best.ctas = c; best.split = sp; best.scratch = scratch;
+                    best_cost = cost;
+                }
+            }
+        }
+    }
+    return best;
+}
+
+int device_sms() {
+    int dev = 0, sms = 148;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    else (void)cudaGetLastError();
+    return sms > 0 ? sms : 148;
+}
+
+}  // namespace
+
+size_t gemm_scratch_bytes(int64_t M, int64_t N, int64_t K, int bits) {
+    if (M <= 0 || N <= 0 || K <= 0) return 0;
+    return plan_gemm(M, N, K, bits, device_sms(), (size_t)-1).scratch;
+}
+
 fq_status launch_gemm_tcgen05(const int8_t* a8, int64_t M, const Weights& W, int acc_shift, const GemmOut& out,
-                              cudaStream_t stream) {
+                              void* scratch, size_t scratch_bytes, cudaStream_t stream) {
     if (M == 0 || W.N == 0) return FQ_OK;
     if (!W.tmap_valid) return FQ_ERR_CUDA;
 
     Params p{};
     p.M = M; p.N = W.N; p.K = W.K;
-    int dev = 0, sms = 148;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    // Token tile and CTA grouping.  Upper bound of the tile from TMEM: two accumulator stages, plus the
-    // unpacked-weight ring for 4-bit weights (2*bt + 3*32 <= 512 columns).  M is split evenly over
-    // m_tiles so that ragged M wastes little.  Candidates are ranked by a cost model fitted to
-    // measured launches (cycles): rounds of work units over the SMs, each unit costing
-    //     k_blocks * per_kblock(bt) + 16*bt + 1000          (the tail: epilogue and tile hand-over)
-    //   4-bit weights:          per_kblock = 330 + bt       (issue floor, then the MMAs' 2*bt)
-    //   8-bit, one CTA:         per_kblock = 300 + 2*bt     (shared-memory bound: both operands pass through it)
-    //   8-bit, CTA pair:        per_kblock = max(545, 2.62*bt)   (each CTA stages half of the token tile)
-    // Pairs gain nothing for 4-bit weights, which never pass through shared memory unpacked.
-    const int bt_max = W.bits == 4 ? 208 : 256;
-    const int64_t k_blocks_host = (W.K + kBlockK - 1) / kBlockK;
-    int bt = 0, ctas = 1;
-    double best = 0.0;
-    for (int c = 1; c <= ((W.bits == 8 && W.N > kTileN) ? 2 : 1); ++c) {
-        const int64_t n_units = (W.N + kTileN * c - 1) / (kTileN * c);
-        const int slots = sms / c;
-        for (int mt = (int)((M + bt_max - 1) / bt_max); mt <= (int)((M + 63) / 64); ++mt) {
-            const int b = (int)(((M + mt - 1) / mt + 15) / 16 * 16);
-            if (b > bt_max) continue;
-            const int64_t units = n_units * ((M + b - 1) / b);
-            const double per_kb = W.bits == 4 ? 330.0 + b
-                                  : (c == 1 ? 300.0 + 2.0 * b : (2.62 * b > 545.0 ? 2.62 * b : 545.0));
-            const double cost = (double)((units + slots - 1) / slots) * ((double)k_blocks_host * per_kb + 16.0 * b + 1000.0);
-            if (bt == 0 || cost < best * 0.98) { bt = b; ctas = c; best = cost; }   // ties: the earlier (larger) tile
-        }
-    }
+    const int sms = device_sms();
+    Plan plan = plan_gemm(M, W.N, W.K, W.bits, sms, scratch ? scratch_bytes : 0);
+    int bt = plan.bt, ctas = plan.ctas, split = plan.split;
 #if defined(FQ_GEMM_TRACE) || defined(FQ_GEMM_DEV)
-    if (const char* e = getenv("FQ_BT")) bt = atoi(e);      // development builds: force the token tile
-    if (const char* e = getenv("FQ_PAIR")) ctas = atoi(e);   // ... and single CTAs or pairs
+    if (const char* e = getenv("FQ_BT")) { bt = atoi(e); split = 1; }       // development builds: force the token tile
+    if (const char* e = getenv("FQ_PAIR")) { ctas = atoi(e); split = 1; }   // ... and single CTAs or pairs
+    if (const char* e = getenv("FQ_SPLIT")) split = atoi(e);                // ... and the K split
+    if (getenv("FQ_PLAN_PRINT")) fprintf(stderr, "plan: M=%lld N=%lld K=%lld bits=%d -> bt=%d ctas=%d split=%d\n", (long long)M, (long long)W.N, (long long)W.K, W.bits, bt, ctas, split);
 #endif
+    p.split = split;
+    p.partials = static_cast<int32_t*>(scratch);
     p.bt = bt;
     p.m_tiles = (int)((M + bt - 1) / bt);
     p.n_tiles = (int)((W.N + kTileN * ctas - 1) / (kTileN * ctas));
@@ -959,14 +1083,18 @@ fq_status launch_gemm_tcgen05(const int8_t* a8, int64_t M, const Weights& W, int
         return FQ_ERR_CUDA;
 
     const int num_units = p.m_tiles * p.n_tiles;
-    const int max_units = sms / ctas;
-    const int grid = (num_units < max_units ? num_units : max_units) * ctas;
+    const int group = ctas * split;                  // CTAs of one cluster: a pair, or the ranks of a K split
+    const int max_units = sms / group;
+    const int grid = (num_units < max_units ? num_units : max_units) * group;
 
-    if (W.bits == 4)
-        return ctas == 2 ? launch_variant<4, 2>(map_a, W.tmap, p, grid, smem, stream)
-                         : launch_variant<4, 1>(map_a, W.tmap, p, grid, smem, stream);
-    return ctas == 2 ? launch_variant<8, 2>(map_a, W.tmap, p, grid, smem, stream)
-                     : launch_variant<8, 1>(map_a, W.tmap, p, grid, smem, stream);
+    if (W.bits == 4) {
+        if (ctas == 2) return launch_variant<4, 2, false>(map_a, W.tmap, p, grid, smem, 2, stream);
+        return split > 1 ? launch_variant<4, 1, true>(map_a, W.tmap, p, grid, smem, split, stream)
+                         : launch_variant<4, 1, false>(map_a, W.tmap, p, grid, smem, 1, stream);
+    }
+    if (ctas == 2) return launch_variant<8, 2, false>(map_a, W.tmap, p, grid, smem, 2, stream);
+    return split > 1 ? launch_variant<8, 1, true>(map_a, W.tmap, p, grid, smem, split, stream)
+                     : launch_variant<8, 1, false>(map_a, W.tmap, p, grid, smem, 1, stream);
 }
 
 }  // namespace fq
