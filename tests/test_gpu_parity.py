@@ -223,6 +223,34 @@ def test_accumulator_extremes_and_one_hot(bits):
     assert np.array_equal(to_np(got), wi.T)
 
 
+@pytest.mark.parametrize("M,N,K,bits", [(64, 256, 8192, 4), (208, 384, 16384, 8), (50, 128, 16384, 4)])
+def test_k_split_equals_unsplit_and_oracle(M, N, K, bits):
+    """Few tiles and a long K: the planner splits K over a CTA cluster when the workspace has room
+    for the partial sums.  With a workspace that holds only the activation codes and steps the same
+    call runs unsplit; both must give the oracle's integer sums exactly."""
+    rng = np.random.default_rng(M + N + K + bits)
+    a, w = random_codes(rng, M, K, bits), random_codes(rng, N, K, bits)
+    want = oracle.gemm_i32(a, w, K, bits)
+    h = import_codes(w, K, bits)
+    base = (M * K + 255) // 256 * 256 + (4 * M + 255) // 256 * 256
+    full = fq.workspace_bytes(M, K, N, bits)
+    assert full > base, "the planner was expected to ask for split scratch on this shape"
+    split = fq.gemm_acc_i32(to_dev(a), h, workspace=torch.empty(full, dtype=torch.uint8, device="cuda"))
+    unsplit = fq.gemm_acc_i32(to_dev(a), h, workspace=torch.empty(base, dtype=torch.uint8, device="cuda"))
+    assert np.array_equal(to_np(split), want)
+    assert np.array_equal(to_np(unsplit), want)
+    # and through the scaled epilogue (bf16 output, ragged token tail)
+    delta = torch.rand(M, device="cuda") + 0.5
+    y1 = fq.gemm_w4a4(to_dev(a), delta, h, out_dtype=torch.bfloat16) if bits == 4 else \
+        fq.gemm_w8a8(to_dev(a), delta, h, out_dtype=torch.bfloat16)
+    ws = torch.empty(base, dtype=torch.uint8, device="cuda")
+    y2 = fq.gemm_w4a4(to_dev(a), delta, h, out_dtype=torch.bfloat16, workspace=ws) if bits == 4 else \
+        fq.gemm_w8a8(to_dev(a), delta, h, out_dtype=torch.bfloat16, workspace=ws)
+    assert torch.equal(y1, y2)
+    st, word = fq.device_status()
+    assert st == fq.OK and word == 0
+
+
 def test_gemm_is_deterministic_run_to_run():
     rng = np.random.default_rng(5)
     a, w = random_codes(rng, 333, 2048, 4), random_codes(rng, 520, 2048, 4)
