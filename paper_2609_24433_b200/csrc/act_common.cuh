@@ -21,10 +21,14 @@ __device__ __forceinline__ uint32_t pack_word(const uint32_t* b) {
         for (int i = 6; i >= 0; --i) w = (w << 4) + b[i];
         return (w + (0x88888888u - kMagicBits * 0x11111111u)) ^ 0x88888888u;
     } else {
-        uint32_t w = b[3];
-#pragma unroll
-        for (int i = 2; i >= 0; --i) w = (w << 8) + b[i];
-        return (w + (0x80808080u - kMagicBits * 0x01010101u)) ^ 0x80808080u;
+        // 8-bit codes: the low byte of every raw pattern already is the two's-complement code
+        // (0x4B400000 + code has the code's low 8 bits in its lowest byte), so three byte permutes
+        // gather the four bytes.
+        uint32_t lo, hi, w;
+        asm("prmt.b32 %0, %1, %2, 0x0040;" : "=r"(lo) : "r"(b[0]), "r"(b[1]));
+        asm("prmt.b32 %0, %1, %2, 0x0040;" : "=r"(hi) : "r"(b[2]), "r"(b[3]));
+        asm("prmt.b32 %0, %1, %2, 0x5410;" : "=r"(w) : "r"(lo), "r"(hi));
+        return w;
     }
 }
 

@@ -59,10 +59,21 @@ __device__ __forceinline__ float max3_abs(float m, float x, float y) {
 }
 // A thread's slice is 64, 128 or 256 contiguous bytes of a swizzled, 1024-byte aligned region.
 // Inside one 128-byte line the swizzled address of 16-byte piece i is (address of piece 0) ^ (i << 4),
-// so one pointer per line (line0, line1 = swizzled starts of the slice's lines) is all a thread keeps.
-__device__ __forceinline__ const uint8_t* piece(const uint8_t* line0, const uint8_t* line1, int i) {
-    const uint8_t* l = i < 8 ? line0 : line1;
-    return reinterpret_cast<const uint8_t*>(reinterpret_cast<uintptr_t>(l) ^ (uintptr_t)((i & 7) << 4));
+// so one address per line (line0, line1 = swizzled starts of the slice's lines) is all a thread keeps.
+// Addresses are 32-bit shared-window addresses and the loads explicit ld.shared: through generic
+// pointers the same reads cost 64-bit address arithmetic (about one extra instruction per element).
+__device__ __forceinline__ uint32_t piece(uint32_t line0, uint32_t line1, int i) {
+    return (i < 8 ? line0 : line1) ^ (uint32_t)((i & 7) << 4);
+}
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ float4 lds128f(uint32_t addr) {
+    float4 v;
+    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
+    return v;
 }
 
 struct RingParams {
@@ -146,8 +157,9 @@ transform_quantize_ring_kernel(const __grid_constant__ CUtensorMap map_x, const 
     const uint32_t xs0 = swz128((uint32_t)col0 * (uint32_t)sizeof(XT));
     const uint32_t xs1 = swz128((uint32_t)col0 * (uint32_t)sizeof(XT) + 128u);
     const uint32_t gkey = (uint32_t)((col0 / E) & 7) << 4;
-    const uint8_t* g0 = gen + (((uint32_t)col0 * 4u) ^ gkey);
-    const uint8_t* g1 = gen + (((uint32_t)col0 * 4u + 128u) ^ gkey);
+    const uint32_t g0 = base + (((uint32_t)col0 * 4u) ^ gkey);
+    const uint32_t g1 = base + (((uint32_t)col0 * 4u + 128u) ^ gkey);
+    const bool warp_ok = __all_sync(0xffffffffu, col_ok);   // the usual case: no lane of the warp is past K
     const float2 neg1 = make_float2(-1.0f, -1.0f);
 
     int n = 0, d = 0;
@@ -156,16 +168,16 @@ transform_quantize_ring_kernel(const __grid_constant__ CUtensorMap map_x, const 
         bool ok = mbar_wait_all(smem_u32(&full0[d]), ph, abort_flag, p.watchdog, 0x100u);   // every lane polls: cheaper than one lane + broadcast
 
         float2 v[H];
-        const uint8_t* slot = gen + slots_off + (size_t)(group * p.depth + d) * p.slot_bytes;
-        const uint8_t* x0 = slot + xs0;
-        const uint8_t* x1 = slot + xs1;
-        if (col_ok) {
+        const uint32_t slot = base + slots_off + (uint32_t)(group * p.depth + d) * p.slot_bytes;
+        const uint32_t x0 = slot + xs0;
+        const uint32_t x1 = slot + xs1;
+        auto load_row = [&]() {
             if (sizeof(XT) == 2) {
                 // bf16: 8 channels per 16-byte piece; pieces [0, H/8) are the low half, the rest the high half
 #pragma unroll
                 for (int i = 0; i < H / 8; ++i) {
-                    const uint4 lo = *reinterpret_cast<const uint4*>(piece(x0, x1, i));
-                    const uint4 hi = *reinterpret_cast<const uint4*>(piece(x0, x1, i + H / 8));
+                    const uint4 lo = lds128(piece(x0, x1, i));
+                    const uint4 hi = lds128(piece(x0, x1, i + H / 8));
                     const uint32_t wl[4] = {lo.x, lo.y, lo.z, lo.w}, wh[4] = {hi.x, hi.y, hi.z, hi.w};
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
@@ -177,8 +189,8 @@ transform_quantize_ring_kernel(const __grid_constant__ CUtensorMap map_x, const 
             } else {
 #pragma unroll
                 for (int i = 0; i < H / 4; ++i) {
-                    const float4 lo = *reinterpret_cast<const float4*>(piece(x0, x1, i));
-                    const float4 hi = *reinterpret_cast<const float4*>(piece(x0, x1, i + H / 4));
+                    const float4 lo = lds128f(piece(x0, x1, i));
+                    const float4 hi = lds128f(piece(x0, x1, i + H / 4));
                     v[4 * i + 0] = make_float2(lo.x, hi.x);
                     v[4 * i + 1] = make_float2(lo.y, hi.y);
                     v[4 * i + 2] = make_float2(lo.z, hi.z);
@@ -188,8 +200,8 @@ transform_quantize_ring_kernel(const __grid_constant__ CUtensorMap map_x, const 
             if (p.mult != nullptr) {
 #pragma unroll
                 for (int i = 0; i < H / 4; ++i) {
-                    const float4 lo = *reinterpret_cast<const float4*>(piece(g0, g1, i));
-                    const float4 hi = *reinterpret_cast<const float4*>(piece(g0, g1, i + H / 4));
+                    const float4 lo = lds128f(piece(g0, g1, i));
+                    const float4 hi = lds128f(piece(g0, g1, i + H / 4));
                     v[4 * i + 0] = f2_mul(v[4 * i + 0], make_float2(lo.x, hi.x));
                     v[4 * i + 1] = f2_mul(v[4 * i + 1], make_float2(lo.y, hi.y));
                     v[4 * i + 2] = f2_mul(v[4 * i + 2], make_float2(lo.z, hi.z));
@@ -200,6 +212,13 @@ transform_quantize_ring_kernel(const __grid_constant__ CUtensorMap map_x, const 
 #pragma unroll
                 for (int i = 0; i < H; ++i) v[i] = f2_mul(v[i], c2);
             }
+        };
+        // Warp-uniform fast path: with a per-lane `col_ok` the zero fill below is compiled into
+        // predicated instructions that every row pays for (half an instruction per element).
+        if (warp_ok) {
+            load_row();
+        } else if (col_ok) {
+            load_row();
         } else {
 #pragma unroll
             for (int i = 0; i < H; ++i) v[i] = make_float2(0.0f, 0.0f);
