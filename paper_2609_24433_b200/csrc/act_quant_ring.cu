@@ -308,10 +308,12 @@ transform_quantize_ring_kernel(const __grid_constant__ CUtensorMap map_x, const 
                     t.x = fminf(fmaxf(t.x, -p.qmax), p.qmax);
                     t.y = fminf(fmaxf(t.y, -p.qmax), p.qmax);
                 }
-                // Scalar adds on purpose: a packed multiply feeding a packed add with no other use was
-                // observed to be fused into one packed FMA by the assembler, which rounds ties differently.
-                bl[i] = __float_as_uint(__fadd_rn(t.x, 12582912.0f));
-                bh[i] = __float_as_uint(__fadd_rn(t.y, 12582912.0f));
+                // t * 1 + magic as an explicit packed FMA (exact product, so it rounds like the add).  A
+                // packed multiply feeding a packed ADD was observed to be fused into one packed FMA by the
+                // assembler, which rounds exact ties differently.
+                t = f2_fma(t, make_float2(1.0f, 1.0f), make_float2(12582912.0f, 12582912.0f));
+                bl[i] = __float_as_uint(t.x);
+                bh[i] = __float_as_uint(t.y);
             }
             wlo[j] = pack_word<FMT>(bl);
             whi[j] = pack_word<FMT>(bh);
