@@ -39,6 +39,7 @@
 
 #include "fq_common.cuh"
 #include "ptx_sm100.cuh"
+#include "act_common.cuh"
 
 namespace fq {
 
@@ -654,24 +655,40 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                 }
                 tmem_ld_wait();
                 if (staged) {
-                    // transpose 32 channels x 16 tokens through shared memory, then 16-byte stores
+                    // Transpose 32 channels x 16 tokens through shared memory, then 16-byte stores.  Tokens
+                    // go in pairs: packed multiply, packed FMA and one two-way bf16 conversion per pair, the
+                    // pair's word (token 2k low, token 2k+1 high) stored at [pair k][channel].  A lane then
+                    // reads 8 channels of one pair (32 bytes), splits the two tokens with byte permutes and
+                    // writes 8 consecutive channels of each token.
+                    uint32_t* xw = reinterpret_cast<uint32_t*>(xpose);
+                    const float2 sw2 = make_float2(sw, sw), bj2 = make_float2(bj, bj);
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) {
-                        const float v = fmaf((float)(int)r[i], d[i] * sw, bj);
-                        *reinterpret_cast<__nv_bfloat16*>(xpose + i * 64 + lane * 2) = __float2bfloat16_rn(v);
+                    for (int k = 0; k < 8; ++k) {
+                        const float2 a2 = make_float2((float)(int)r[2 * k], (float)(int)r[2 * k + 1]);
+                        const float2 v2 = f2_fma(a2, f2_mul(make_float2(d[2 * k], d[2 * k + 1]), sw2), bj2);
+                        uint32_t w;
+                        asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(w) : "f"(v2.y), "f"(v2.x));
+                        xw[k * 32 + lane] = w;
                     }
                     __syncwarp();
                     __nv_bfloat16* y = static_cast<__nv_bfloat16*>(p.out.y);
-#pragma unroll
-                    for (int k = 0; k < 2; ++k) {
-                        const int row = (lane >> 2) + 8 * k;
+                    {
+                        const int k = lane >> 2;
                         const int64_t jj = jq + (lane & 3) * 8;
-                        const uint4 v = *reinterpret_cast<const uint4*>(xpose + row * 64 + (lane & 3) * 16);
+                        const uint4 q0 = *reinterpret_cast<const uint4*>(xw + k * 32 + (lane & 3) * 8);
+                        const uint4 q1 = *reinterpret_cast<const uint4*>(xw + k * 32 + (lane & 3) * 8 + 4);
+                        uint4 lo, hi;     // token 2k and token 2k + 1, channels jj .. jj + 7
+                        lo.x = __byte_perm(q0.x, q0.y, 0x5410); hi.x = __byte_perm(q0.x, q0.y, 0x7632);
+                        lo.y = __byte_perm(q0.z, q0.w, 0x5410); hi.y = __byte_perm(q0.z, q0.w, 0x7632);
+                        lo.z = __byte_perm(q1.x, q1.y, 0x5410); hi.z = __byte_perm(q1.x, q1.y, 0x7632);
+                        lo.w = __byte_perm(q1.z, q1.w, 0x5410); hi.w = __byte_perm(q1.z, q1.w, 0x7632);
 #if defined(FQ_GEMM_TRACE) || defined(FQ_GEMM_DEV)
-                        if ((p.dbg & 1) && v.x != 0x12345678u) continue;
+                        if ((p.dbg & 1) && lo.x != 0x12345678u) continue;
 #endif
-                        if (tc + row < p.M && jj < p.N)
-                            *reinterpret_cast<uint4*>(y + (tc + row) * p.out.ldy + jj) = v;
+                        if (jj < p.N) {
+                            if (tc + 2 * k < p.M) *reinterpret_cast<uint4*>(y + (tc + 2 * k) * p.out.ldy + jj) = lo;
+                            if (tc + 2 * k + 1 < p.M) *reinterpret_cast<uint4*>(y + (tc + 2 * k + 1) * p.out.ldy + jj) = hi;
+                        }
                     }
                     __syncwarp();
                 } else {
