@@ -328,12 +328,26 @@ def run_e2e(layer, sites, ops, world, K, Wm, dist, device):
     h2d = sum(t.numel() * t.element_size() for t in host_x)
     d2h = sum(t.numel() * t.element_size() for t in host_y)
 
+    # Copies in, kernels and copies out run on three streams chained by events, so that a site's
+    # result travels to the host while the next site's input travels to the device (PCIe is full
+    # duplex) and its kernels run; every step still moves all inputs and all outputs.
+    s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
+    s_run = torch.cuda.current_stream()
+    ev_in = [torch.cuda.Event() for _ in entry]
+    ev_done = [torch.cuda.Event() for _ in entry]
+
     def step():
-        for e, hx, hy in zip(entry, host_x, host_y):
+        for i, (e, hx, hy) in enumerate(zip(entry, host_x, host_y)):
             dst = e["x"].view(torch.int16) if e["x"].dtype == torch.bfloat16 else e["x"]
-            dst.copy_(hx, non_blocking=True)
+            with torch.cuda.stream(s_in):
+                dst.copy_(hx, non_blocking=True)
+                ev_in[i].record(s_in)
+            s_run.wait_event(ev_in[i])
             layer.fq.linear(e["x"], e["h"], 1.0, y=e["y"], workspace=e["ws"])
-            hy.copy_(e["y"], non_blocking=True)
+            ev_done[i].record(s_run)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(ev_done[i])
+                hy.copy_(e["y"], non_blocking=True)
         torch.cuda.synchronize()
 
     n = max(3, min(K, 20))
