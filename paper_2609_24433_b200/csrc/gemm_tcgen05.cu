@@ -23,10 +23,16 @@
 //   warp 0       TMA producer          warp 1  MMA issuer + TMEM allocator
 //   warps 2-9    epilogue (two warps per TMEM lane quadrant, alternating 16-token chunks)
 //   warps 10-17  nibble unpack (two sets of four, alternating k-blocks), warp 18 TMA producer
-//                of packed weights (4-bit weights only)
-// With 4-bit weights three rings are decoupled: activations (TMA -> MMA), packed weights
-// (TMA -> unpack, deep and cheap: 8 KB a stage) and unpacked weights (unpack -> MMA, 3 stages
-// of 32 TMEM columns), so the unpack latency sits beside, not inside, the TMA round trip.
+//                of packed weights (4-bit weights); warp 10 TMA producer of int8 weights (8-bit)
+// Every role runs its loop with the whole warp converged and elects one lane (elect.sync) for
+// the issue itself; a k-block of the MMA warp is one block of PTX that also tests the next
+// k-block's barriers (see issue_kblock_*).  With 4-bit weights three rings are decoupled:
+// activations (TMA -> MMA), packed weights (TMA -> unpack, deep and cheap: 8 KB a stage) and
+// unpacked weights (unpack -> MMA, 32 TMEM columns a stage); one tcgen05.commit per k-block
+// frees both the activation stage and the k-block's TMEM slot.
+// Variants: CTAS = 2 runs CTA pairs (cta_group::2, 256 channels per MMA, each CTA staging half
+// of the token tile); SPLIT lets the CTAs of a cluster share a tile along K and exchange int32
+// partial sums through global scratch.
 // bf16 outputs leave through a per-warp 1 KB shared-memory transposer so that global
 // stores are 16-byte vectors of 8 consecutive channels; fp32/raw outputs store directly.
 // Every mbarrier wait is bounded by wall-clock time; on expiry the CTA records a
@@ -64,7 +70,6 @@ namespace {
 
 constexpr int kTileN = 128;          // output channels per tile (MMA M)
 constexpr int kBlockK = 128;         // int8 elements (= bytes) of K per pipeline stage
-constexpr int kMmaK = 32;            // K per tcgen05.mma.kind::i8
 constexpr int kAccStages = 2;
 constexpr int kEpiWarps = 8;
 constexpr int kEpiStageBytes = 16 * 64;   // 16 tokens x 32 channels of bf16 per epilogue warp
@@ -73,7 +78,6 @@ constexpr int kFirstUnpackWarp = 2 + kEpiWarps;
 constexpr int kUnpackSets = 2;          // sets of four unpack warps, one TMEM lane quadrant each
 constexpr int kThreadsW4 = 32 * (2 + kEpiWarps) + kUnpackSets * 128 + 32;
 constexpr int kMaxStagesW = 8;
-constexpr int kStagesW = 3;            // unpacked-weight stages in tensor memory (4-bit weights)
 constexpr int kColsW = kBlockK / 4;     // TMEM columns of one unpacked k-block (128 int8 per lane)
 constexpr int kMaxStages = 8;
 constexpr int kMaxStagesP = 16;
@@ -171,43 +175,6 @@ __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
     else
         asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
 }
-template <int CTAS>
-__device__ __forceinline__ void mma_i8(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                       uint32_t accumulate) {
-    if (CTAS == 1)
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t"
-            "setp.ne.b32 p, %4, 0;\n\t"
-            "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
-            ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-            : "memory");
-    else
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t"
-            "setp.ne.b32 p, %4, 0;\n\t"
-            "tcgen05.mma.cta_group::2.kind::i8 [%0], %1, %2, %3, p;\n\t}"
-            ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-            : "memory");
-}
-// A operand from tensor memory (lane = row, 4 int8 per 32-bit column), B from shared memory.
-template <int CTAS>
-__device__ __forceinline__ void mma_i8_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
-                                          uint32_t accumulate) {
-    if (CTAS == 1)
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t"
-            "setp.ne.b32 p, %4, 0;\n\t"
-            "tcgen05.mma.cta_group::1.kind::i8 [%0], [%1], %2, %3, p;\n\t}"
-            ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
-            : "memory");
-    else
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t"
-            "setp.ne.b32 p, %4, 0;\n\t"
-            "tcgen05.mma.cta_group::2.kind::i8 [%0], [%1], %2, %3, p;\n\t}"
-            ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
-            : "memory");
-}
 // One k-block of work for the issuing warp, as ONE block of PTX so that the two barrier tests for
 // the NEXT k-block are in flight while this k-block's four MMAs and its commits are issued (their
 // results are read only at the end; separate asm statements would stall on each test's ~100-cycle
@@ -281,11 +248,6 @@ __device__ __forceinline__ uint32_t issue_kblock_ss(uint32_t issue, uint32_t d_t
         asm volatile(FQ_ISSUE_HEAD FQ_ISSUE_MMAS("2", "", "") FQ_ISSUE_COMMITS_2 FQ_ISSUE_TAIL FQ_ISSUE_OPERANDS(FQ_CON_L));
     return ready;
 }
-__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t* r) {
-    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
-                 ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
-                 : "memory");
-}
 __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
     asm volatile(
         "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
@@ -297,21 +259,6 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
         : "memory");
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
-// Arrive on `bar` once every MMA issued so far by this thread has retired; for a CTA pair the
-// arrival is delivered to the barrier at that offset in BOTH CTAs.
-template <int CTAS>
-__device__ __forceinline__ void mma_commit(uint32_t bar) {
-    if (CTAS == 1) {
-        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
-                     : "memory");
-    } else {
-        const uint16_t mask = 3;
-        asm volatile(
-            "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
-            ::"r"(bar), "h"(mask)
-            : "memory");
-    }
-}
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* r) {
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
