@@ -289,6 +289,9 @@ fq_status fq_weights_import(const void* codes, const float* w_scale, const float
         ok = ok && cudaMemcpyAsync(w->mult_g, mult_g, sizeof(float) * (size_t)K, cudaMemcpyDeviceToDevice, s) == cudaSuccess;
     else
         ok = ok && launch_multipliers(nullptr, K, block_norm(hadamard_block), nullptr, w->mult_g, s) == cudaSuccess;
+    // A handle is complete when it is returned (as after fq_fold_weights): the GEMM's weight
+    // producers start reading it before the kernels ahead of them in the stream have finished.
+    ok = ok && cudaStreamSynchronize(s) == cudaSuccess;
     if (ok) ok = build_weight_tmap(*w) == FQ_OK;
     if (!ok) {
         fq_weights_destroy(reinterpret_cast<fq_weights*>(w));

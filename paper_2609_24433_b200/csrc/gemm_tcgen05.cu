@@ -113,6 +113,11 @@ struct Params {
     const float* bias;
     GemmOut out;
     uint32_t* watchdog;
+    // index arithmetic done once on the host (integer divisions cost the short launches ~0.3 us)
+    int cluster_shift;   // log2 of the CTAs per cluster (pair or K split)
+    int unit_step;       // clusters in the grid
+    int tiles_q, tiles_rem;   // tiles per cluster: tiles_q, one more for the first tiles_rem clusters
+    int k_blocks_all, kb_per; // k-blocks of the problem, and per rank of a K split
     int split;           // CTAs of a cluster sharing one tile, each on its own slice of K (1 = no split)
     int32_t* partials;   // [tile][split][bt tokens][128 channels] int32: raw sums a rank hands to the chunks' owners
 #if defined(FQ_GEMM_TRACE) || defined(FQ_GEMM_DEV)
@@ -322,6 +327,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     volatile int* abort_flag = &s_abort;
+    if (warp == 1) FQ_TRACE(3, 1023, 0);             // kernel entry
     const uint32_t cta_rank = CTAS == 2 ? cluster_ctarank() : 0u;
     const bool leader = cta_rank == 0;
     // K split (single CTAs only): the cluster's ranks work on the same tiles, rank r on k-blocks [kb0, kb0 + k_blocks)
@@ -340,26 +346,26 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     const uint32_t smem_e = smem_p + (BITS == 4 ? (uint32_t)p.stages_p * pk_bytes : 0u);
     uint8_t* gen_base = smem_raw + (base - smem_u32(smem_raw));   // generic pointer to `base`
 
-    if (threadIdx.x == 0) {
-        s_abort = 0;
-        for (int s = 0; s < p.stages; ++s) {
-            mbar_init(smem_u32(&s_full_tma[s]), BITS == 8 ? 2 : 1);   // 8-bit: activation and weight producers
-            mbar_init(smem_u32(&s_empty[s]), 1);
+    if (threadIdx.x == 0) s_abort = 0;
+    if (warp == 2) {
+        // one lane per ring slot: the ~40 barrier initialisations run side by side (and beside the
+        // TMEM allocation in warp 1) instead of one after the other in a single thread
+        if (lane < p.stages) {
+            mbar_init(smem_u32(&s_full_tma[lane]), BITS == 8 ? 2 : 1);   // 8-bit: activation and weight producers
+            mbar_init(smem_u32(&s_empty[lane]), 1);
         }
         if (BITS == 4) {
-            for (int s = 0; s < p.stages_p; ++s) {
-                mbar_init(smem_u32(&s_full_p[s]), 1);
-                mbar_init(smem_u32(&s_empty_p[s]), 4);
+            if (lane < p.stages_p) {
+                mbar_init(smem_u32(&s_full_p[lane]), 1);
+                mbar_init(smem_u32(&s_empty_p[lane]), 4);
             }
-            for (int s = 0; s < p.stages_w; ++s) {
-                mbar_init(smem_u32(&s_full_w8[s]), 4 * CTAS);
-            }
+            if (lane < p.stages_w) mbar_init(smem_u32(&s_full_w8[lane]), 4 * CTAS);
         }
-        for (int a = 0; a < kAccStages; ++a) {
-            mbar_init(smem_u32(&s_acc_full[a]), 1);
-            mbar_init(smem_u32(&s_acc_empty[a]), kEpiWarps * CTAS);
-            mbar_init(smem_u32(&s_part_full[a]), (uint32_t)(kEpiWarps * (split > 1 ? split - 1 : 1)));
-            mbar_init(smem_u32(&s_part_empty[a]), (uint32_t)(kEpiWarps * (split > 1 ? split - 1 : 1)));
+        if (lane < kAccStages) {
+            mbar_init(smem_u32(&s_acc_full[lane]), 1);
+            mbar_init(smem_u32(&s_acc_empty[lane]), kEpiWarps * CTAS);
+            mbar_init(smem_u32(&s_part_full[lane]), (uint32_t)(kEpiWarps * (split > 1 ? split - 1 : 1)));
+            mbar_init(smem_u32(&s_part_empty[lane]), (uint32_t)(kEpiWarps * (split > 1 ? split - 1 : 1)));
         }
         fence_mbarrier_init();
         fence_proxy_async_smem();
@@ -372,16 +378,21 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     const uint32_t tmem_base = s_tmem_base;
     // Everything above is on-chip setup; from here on global memory is touched (activations written
     // by the kernel before this one, outputs that it may still be reading).
-    griddep_wait();
+    if (warp == 1) FQ_TRACE(3, 1023, 1);             // set-up done
+    // The weight producers do not wait: a weight handle is complete before any call that uses it
+    // is enqueued, so its tiles can stream in while the kernel ahead (the prologue) still runs.
+    const bool weight_producer = BITS == 8 ? warp == kFirstUnpackWarp : warp == kFirstUnpackWarp + 4 * kUnpackSets;
+    if (!weight_producer) griddep_wait();
+    if (warp == 1) FQ_TRACE(3, 1023, 2);             // previous kernel complete
     griddep_launch_dependents();
 
     // work units: (super-tile of 128*CTAS channels) x (token tile); one unit per CTA or CTA pair at a time
     const int num_tiles = p.m_tiles * p.n_tiles;
-    const int cluster_ctas = CTAS == 2 ? 2 : split;
-    const int unit0 = (int)blockIdx.x / cluster_ctas;
-    const int unit_step = (int)gridDim.x / cluster_ctas;
-    const int k_blocks_all = (int)((p.K + kBlockK - 1) / kBlockK);
-    const int kb_per = (k_blocks_all + split - 1) / split;
+    const int unit0 = (int)blockIdx.x >> p.cluster_shift;
+    const int unit_step = p.unit_step;
+    const int my_tiles = p.tiles_q + (unit0 < p.tiles_rem ? 1 : 0);
+    const int k_blocks_all = p.k_blocks_all;
+    const int kb_per = (SPLIT && CTAS == 1) ? p.kb_per : k_blocks_all;
     const int kb0 = (int)krank * kb_per;                               // first k-block of this rank
     const int k_blocks = kb0 + kb_per <= k_blocks_all ? kb_per : k_blocks_all - kb0;   // >= 1 (host check)
 
@@ -392,7 +403,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         // hand-off: every dependent wait/branch of the lone lane pays for the divergent warp.)
         {
             const uint32_t tx = a_bytes;
-            const int total_kb = ((num_tiles - 1 - unit0) / unit_step + 1) * k_blocks;
+            const int total_kb = my_tiles * k_blocks;
             bool ok = true;
             int stage = 0, kb = 0, tile = unit0;
             uint32_t phase = 0;
@@ -443,7 +454,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             // that issues the current one: a barrier test has ~100 cycles of latency, and two of them
             // in series per k-block would otherwise sit on the issuing warp's critical path.
             bool ready = false;
-            int left = ((num_tiles - 1 - unit0) / unit_step + 1) * k_blocks;   // k-blocks still to issue
+            int left = my_tiles * k_blocks;   // k-blocks still to issue
             [[maybe_unused]] int tn = 0;
             for (int tile = unit0; tile < num_tiles && ok; tile += unit_step) {
                 ok = mbar_wait_all(smem_u32(&s_acc_empty[acc_stage]), acc_phase ^ 1u, abort_flag, p.watchdog, kWdMmaAcc);
@@ -672,7 +683,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         // ------------------------------------------------- TMA producer, int8 weights
         // (converged warp, one issuing lane: see the activation producer)
         {
-            const int total_kb = ((num_tiles - 1 - unit0) / unit_step + 1) * k_blocks;
+            const int total_kb = my_tiles * k_blocks;
             bool ok = true;
             int stage = 0, kb = 0, tile = unit0;
             uint32_t phase = 0;
@@ -716,7 +727,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         // Set `uset` takes the k-blocks whose running index n is congruent to it modulo kUnpackSets,
         // so two k-blocks are in flight per quadrant and one set's store latency hides behind the other.
         const int uset = (warp - kFirstUnpackWarp) >> 2;
-        const int total_kb = ((num_tiles - 1 - unit0) / unit_step + 1) * k_blocks;
+        const int total_kb = my_tiles * k_blocks;
         bool ok = true;
         int ps = uset, ws = uset;                        // ring slots of k-block n, kept incrementally
         uint32_t pph = 0, wph = 0;
@@ -782,7 +793,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     } else if (BITS == 4) {
         // ------------------------------------------------- TMA producer, packed weights
         {
-            const int total_kb = ((num_tiles - 1 - unit0) / unit_step + 1) * k_blocks;
+            const int total_kb = my_tiles * k_blocks;
             bool ok = true;
             int ps = 0, kb = 0, tile = unit0;
             uint32_t pph = 0;
@@ -815,6 +826,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     // ------------------------------------------------------------------ teardown
     tc_fence_before();
     __syncthreads();
+    if (warp == 1) FQ_TRACE(3, 1023, 3);             // all roles done
     if (CTAS == 2 || split > 1) cluster_sync_all(); // no CTA leaves while another may still signal it
     if (warp == 1) {
         tc_fence_after();
@@ -1049,7 +1061,14 @@ fq_status launch_gemm_tcgen05(const int8_t* a8, int64_t M, const Weights& W, int
     const int num_units = p.m_tiles * p.n_tiles;
     const int group = ctas * split;                  // CTAs of one cluster: a pair, or the ranks of a K split
     const int max_units = sms / group;
-    const int grid = (num_units < max_units ? num_units : max_units) * group;
+    const int clusters = num_units < max_units ? num_units : max_units;
+    const int grid = clusters * group;
+    p.cluster_shift = group == 1 ? 0 : (group == 2 ? 1 : (group == 4 ? 2 : 3));
+    p.unit_step = clusters;
+    p.tiles_q = num_units / clusters;
+    p.tiles_rem = num_units % clusters;
+    p.k_blocks_all = (int)((W.K + kBlockK - 1) / kBlockK);
+    p.kb_per = (p.k_blocks_all + split - 1) / split;
 
     if (W.bits == 4) {
         if (ctas == 2) return launch_variant<4, 2, false>(map_a, W.tmap, p, grid, smem, 2, stream);
