@@ -65,14 +65,26 @@ __device__ __forceinline__ float max3_abs(float m, float x, float y) {
 __device__ __forceinline__ uint32_t piece(uint32_t line0, uint32_t line1, int i) {
     return (i < 8 ? line0 : line1) ^ (uint32_t)((i & 7) << 4);
 }
+// (Not volatile, so that the compiler may batch and hoist them; the caller pins their addresses
+// behind the barrier wait that makes the data valid, see `pin_after_wait`.)
 __device__ __forceinline__ uint4 lds128(uint32_t addr) {
     uint4 v;
-    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    asm("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+// An empty volatile statement that "rewrites" an address: loads through that address cannot be
+// moved above it, and it cannot be moved above the (volatile) barrier wait before it.
+__device__ __forceinline__ void pin_after_wait(uint32_t& addr) { asm volatile("" : "+r"(addr) : : "memory"); }
+// Volatile variant for the multiplier: kept in program order, interleaved with the multiplies that
+// consume it (hoisting all of them too would not fit the register file).
+__device__ __forceinline__ float4 lds128f_ordered(uint32_t addr) {
+    float4 v;
+    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
     return v;
 }
 __device__ __forceinline__ float4 lds128f(uint32_t addr) {
     float4 v;
-    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
+    asm("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
     return v;
 }
 
@@ -169,8 +181,9 @@ transform_quantize_ring_kernel(const __grid_constant__ CUtensorMap map_x, const 
 
         float2 v[H];
         const uint32_t slot = base + slots_off + (uint32_t)(group * p.depth + d) * p.slot_bytes;
-        const uint32_t x0 = slot + xs0;
-        const uint32_t x1 = slot + xs1;
+        uint32_t x0 = slot + xs0, x1 = slot + xs1;
+        pin_after_wait(x0);
+        pin_after_wait(x1);
         auto load_row = [&]() {
             if (sizeof(XT) == 2) {
                 // bf16: 8 channels per 16-byte piece; pieces [0, H/8) are the low half, the rest the high half
@@ -200,8 +213,8 @@ transform_quantize_ring_kernel(const __grid_constant__ CUtensorMap map_x, const 
             if (p.mult != nullptr) {
 #pragma unroll
                 for (int i = 0; i < H / 4; ++i) {
-                    const float4 lo = lds128f(piece(g0, g1, i));
-                    const float4 hi = lds128f(piece(g0, g1, i + H / 4));
+                    const float4 lo = lds128f_ordered(piece(g0, g1, i));
+                    const float4 hi = lds128f_ordered(piece(g0, g1, i + H / 4));
                     v[4 * i + 0] = f2_mul(v[4 * i + 0], make_float2(lo.x, hi.x));
                     v[4 * i + 1] = f2_mul(v[4 * i + 1], make_float2(lo.y, hi.y));
                     v[4 * i + 2] = f2_mul(v[4 * i + 2], make_float2(lo.z, hi.z));
