@@ -251,6 +251,41 @@ def test_k_split_equals_unsplit_and_oracle(M, N, K, bits):
     assert st == fq.OK and word == 0
 
 
+def test_back_to_back_calls_share_a_workspace_without_syncs():
+    """The kernels are launched with programmatic stream serialization (each may start its on-chip
+    set-up, and the GEMM its weight loads, before the kernel ahead has finished).  A chain of calls
+    on one stream that reuse ONE workspace and feed each other must give exactly what the same
+    calls give when the device is synchronised after every call."""
+    torch.manual_seed(7)
+    dev = "cuda"
+    K0, N0, N1 = 2048, 1024, 768
+    M = 300
+    hs = []
+    for (n, k, bits) in [(N0, K0, 4), (N1, N0, 8), (N0, N1, 4)]:
+        w = (torch.randn((n, k), device=dev) * 0.02)
+        hs.append(fq.fold_weights(w, None, torch.randn(n, device=dev) * 0.02, 128 if k % 128 == 0 else 32, bits))
+    x0 = torch.randn((M, K0), device=dev).to(torch.bfloat16)
+    ws = torch.empty(max(fq.workspace_bytes(M, h.K, h.N, h.bits) for h in hs), dtype=torch.uint8, device=dev)
+
+    def chain(sync):
+        outs, x = [], x0
+        for rep in range(3):
+            for h in hs:
+                y = fq.linear(x, h, 1.0, out_dtype=torch.bfloat16, workspace=ws)
+                if sync:
+                    torch.cuda.synchronize()
+                outs.append(y)
+                x = y if h is not hs[-1] else x0      # the next call reads this call's output
+        torch.cuda.synchronize()
+        return outs
+
+    want = chain(sync=True)
+    for _ in range(3):
+        got = chain(sync=False)
+        for a, b in zip(got, want):
+            assert torch.equal(a, b)
+
+
 def test_gemm_is_deterministic_run_to_run():
     rng = np.random.default_rng(5)
     a, w = random_codes(rng, 333, 2048, 4), random_codes(rng, 520, 2048, 4)
