@@ -173,15 +173,13 @@ transform_quantize_kernel(const XT* __restrict__ x, int64_t rows, int K, int64_t
         float m = 0.0f;
 #pragma unroll
         for (int i = 0; i < E; ++i) m = fmaxf(m, fabsf(v[i]));
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+        m = warp_max_nonneg(m);
         if (wpr > 1) {
             if (lane == 0) s_part[buf][warp] = m;
             __syncthreads();
             const int w0 = r_in_cta * wpr;
             m = (lane < wpr) ? s_part[buf][w0 + lane] : 0.0f;
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+            m = warp_max_nonneg(m);
         }
 
         // Eq. 5 step; a token whose step is below the smallest normal float is the zero token

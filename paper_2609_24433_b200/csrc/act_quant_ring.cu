@@ -276,14 +276,12 @@ transform_quantize_ring_kernel(const __grid_constant__ CUtensorMap map_x, const 
         float m = 0.0f;
 #pragma unroll
         for (int i = 0; i < H; ++i) m = max3_abs(m, v[i].x, v[i].y);
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+        m = warp_max_nonneg(m);
         if (p.gw > 1) {
             if (lane == 0) s_part[n & 1][warp] = m;
             ok = group_barrier_and(1 + group, p.gw * 32, ok);
             m = (lane < p.gw) ? s_part[n & 1][group * p.gw + lane] : 0.0f;
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+            m = warp_max_nonneg(m);
         }
         if (!ok) break;
 
