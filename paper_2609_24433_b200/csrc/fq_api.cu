@@ -47,9 +47,12 @@ fq_status alloc_handle(int64_t N, int64_t K, int block, int bits, Weights** out)
     ok = ok && cudaMalloc(&w->w_scale, sizeof(float) * (size_t)(N > 0 ? N : 4)) == cudaSuccess;
     ok = ok && cudaMalloc(&w->bias, sizeof(float) * (size_t)(N > 0 ? N : 4)) == cudaSuccess;
     ok = ok && cudaMalloc(&w->mult_g, sizeof(float) * (size_t)K) == cudaSuccess;
+    // counters of the GEMM's K split (slices of a tile finished): zero whenever no launch is in flight
+    ok = ok && cudaMalloc(&w->tile_counters, sizeof(uint32_t) * 1024) == cudaSuccess;
+    ok = ok && cudaMemset(w->tile_counters, 0, sizeof(uint32_t) * 1024) == cudaSuccess;
     if (!ok) {
         cudaGetLastError();
-        cudaFree(w->codes); cudaFree(w->w_scale); cudaFree(w->bias); cudaFree(w->mult_g);
+        cudaFree(w->codes); cudaFree(w->w_scale); cudaFree(w->bias); cudaFree(w->mult_g); cudaFree(w->tile_counters);
         delete w;
         return FQ_ERR_NOMEM;
     }
@@ -228,7 +231,7 @@ fq_status fq_fold_weights(const void* Wsrc, fq_dtype wt, int64_t N, int64_t K, i
 fq_status fq_weights_destroy(fq_weights* wp) {
     Weights* w = reinterpret_cast<Weights*>(wp);
     if (!w) return FQ_OK;
-    cudaFree(w->codes); cudaFree(w->w_scale); cudaFree(w->bias); cudaFree(w->mult_g);
+    cudaFree(w->codes); cudaFree(w->w_scale); cudaFree(w->bias); cudaFree(w->mult_g); cudaFree(w->tile_counters);
     delete w;
     return FQ_OK;
 }

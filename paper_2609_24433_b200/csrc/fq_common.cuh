@@ -20,6 +20,7 @@ struct Weights {
     float* w_scale = nullptr;   // [N]
     float* bias = nullptr;      // [N]
     float* mult_g = nullptr;    // [K] runtime multiplier (1/s_c) * block^-1/2
+    uint32_t* tile_counters = nullptr;   // [1024] zero between launches: slices of a tile finished (K split)
     CUtensorMap tmap;           // TMA view of `codes` for the GEMM's weight operand
     bool tmap_valid = false;
 };

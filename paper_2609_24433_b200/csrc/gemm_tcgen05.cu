@@ -81,6 +81,8 @@ constexpr int kMaxStagesW = 8;
 constexpr int kColsW = kBlockK / 4;     // TMEM columns of one unpacked k-block (128 int8 per lane)
 constexpr int kMaxStages = 8;
 constexpr int kMaxStagesP = 16;
+constexpr int kMaxSplit = 16;          // K slices per tile, at most
+constexpr int kMaxSplitTiles = 1024;   // tiles of a launch that splits K (one counter each in the weight handle)
 
 // Timeline hooks for kernel development: with -DFQ_GEMM_TRACE the first CTA records clock64() at
 // the marked points of the first 1024 k-blocks (agent 0 activation producer, 2 unpack, 3 MMA
@@ -91,13 +93,8 @@ __device__ unsigned long long g_trace[4 * 1024 * 4];
     do {                                                                                        \
         if (blockIdx.x == 0 && lane == 0 && (n) < 1024) g_trace[((agent) * 1024 + (n)) * 4 + (e)] = clock64(); \
     } while (0)
-#define FQ_TRACE_B(blk, agent, n, e)                                                            \
-    do {                                                                                        \
-        if (blockIdx.x == (blk) && lane == 0 && (n) < 1024) g_trace[((agent) * 1024 + (n)) * 4 + (e)] = clock64(); \
-    } while (0)
 #else
 #define FQ_TRACE(agent, n, e) do { } while (0)
-#define FQ_TRACE_B(blk, agent, n, e) do { } while (0)
 #endif
 
 struct Params {
@@ -114,12 +111,13 @@ struct Params {
     GemmOut out;
     uint32_t* watchdog;
     // index arithmetic done once on the host (integer divisions cost the short launches ~0.3 us)
-    int cluster_shift;   // log2 of the CTAs per cluster (pair or K split)
-    int unit_step;       // clusters in the grid
-    int tiles_q, tiles_rem;   // tiles per cluster: tiles_q, one more for the first tiles_rem clusters
-    int k_blocks_all, kb_per; // k-blocks of the problem, and per rank of a K split
-    int split;           // CTAs of a cluster sharing one tile, each on its own slice of K (1 = no split)
-    int32_t* partials;   // [tile][split][bt tokens][128 channels] int32: raw sums a rank hands to the chunks' owners
+    int cluster_shift;   // log2 of the CTAs per cluster (1 for CTA pairs)
+    int unit_step;       // CTAs (or pairs) in the grid
+    int units_q, units_rem;   // work units per CTA: units_q, one more for the first units_rem CTAs
+    int kb_per;          // k-blocks of one work unit (all of K, or K / split)
+    int split, split_shift;   // K split: a tile is `split` (power of two) work units, each on a slice of K
+    int32_t* partials;   // [tile][slice][bt tokens][128 channels] int32 raw sums of the slices (K split)
+    uint32_t* counters;  // [tile] slices finished so far; zero between launches (K split)
 #if defined(FQ_GEMM_TRACE) || defined(FQ_GEMM_DEV)
     int dbg;             // development builds: switches that skip parts of the epilogue
 #endif
@@ -319,8 +317,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     __shared__ uint64_t s_full_w8[kMaxStagesW];     // unpacked weights written
     __shared__ uint64_t s_acc_full[kAccStages];
     __shared__ uint64_t s_acc_empty[kAccStages];
-    __shared__ uint64_t s_part_full[kAccStages];    // K split: the other ranks' partial sums for this tile are written
-    __shared__ uint64_t s_part_empty[kAccStages];   // K split: the other ranks have taken my sums of the tile before last
+    __shared__ uint64_t s_epi_sync;                 // K split: rendezvous of the eight epilogue warps (bounded, unlike bar.sync)
+    __shared__ int s_last[2];                       // K split: this CTA counted the last slice of its tile (alternating slots)
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_abort;
 
@@ -330,9 +328,11 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     if (warp == 1) FQ_TRACE(3, 1023, 0);             // kernel entry
     const uint32_t cta_rank = CTAS == 2 ? cluster_ctarank() : 0u;
     const bool leader = cta_rank == 0;
-    // K split (single CTAs only): the cluster's ranks work on the same tiles, rank r on k-blocks [kb0, kb0 + k_blocks)
+    // K split (single CTAs only): a tile is `split` work units, unit = tile * split + slice, slice s
+    // covering k-blocks [s * k_blocks, (s + 1) * k_blocks).  Any CTA takes any unit; the CTA that
+    // finishes a tile's last slice adds up the slices' partial sums and runs the epilogue.
     const int split = (SPLIT && CTAS == 1) ? p.split : 1;   // compile-time 1 in the common instantiation
-    const uint32_t krank = split > 1 ? cluster_ctarank() : 0u;
+    const int split_shift = (SPLIT && CTAS == 1) ? p.split_shift : 0;
     const int bt_cta = p.bt / CTAS;                 // token rows this CTA loads
 
     // carve dynamic shared memory: [A8 stages][W8 stages][packed stages][epilogue transposers], 1024-byte aligned
@@ -346,34 +346,33 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     const uint32_t smem_e = smem_p + (BITS == 4 ? (uint32_t)p.stages_p * pk_bytes : 0u);
     uint8_t* gen_base = smem_raw + (base - smem_u32(smem_raw));   // generic pointer to `base`
 
-    if (threadIdx.x == 0) s_abort = 0;
-    if (warp == 2) {
-        // one lane per ring slot: the ~40 barrier initialisations run side by side (and beside the
-        // TMEM allocation in warp 1) instead of one after the other in a single thread
-        if (lane < p.stages) {
-            mbar_init(smem_u32(&s_full_tma[lane]), BITS == 8 ? 2 : 1);   // 8-bit: activation and weight producers
-            mbar_init(smem_u32(&s_empty[lane]), 1);
+    if (threadIdx.x == 0) {
+        // (One thread on purpose: spreading these initialisations over the lanes of a warp, one ring
+        // slot per lane, shortened the set-up by 0.3 us but made the 8-bit main loop 10 % slower.)
+        s_abort = 0;
+        for (int s = 0; s < p.stages; ++s) {
+            mbar_init(smem_u32(&s_full_tma[s]), BITS == 8 ? 2 : 1);   // 8-bit: activation and weight producers
+            mbar_init(smem_u32(&s_empty[s]), 1);
         }
         if (BITS == 4) {
-            if (lane < p.stages_p) {
-                mbar_init(smem_u32(&s_full_p[lane]), 1);
-                mbar_init(smem_u32(&s_empty_p[lane]), 4);
+            for (int s = 0; s < p.stages_p; ++s) {
+                mbar_init(smem_u32(&s_full_p[s]), 1);
+                mbar_init(smem_u32(&s_empty_p[s]), 4);
             }
-            if (lane < p.stages_w) mbar_init(smem_u32(&s_full_w8[lane]), 4 * CTAS);
+            for (int s = 0; s < p.stages_w; ++s) mbar_init(smem_u32(&s_full_w8[s]), 4 * CTAS);
         }
-        if (lane < kAccStages) {
-            mbar_init(smem_u32(&s_acc_full[lane]), 1);
-            mbar_init(smem_u32(&s_acc_empty[lane]), kEpiWarps * CTAS);
-            mbar_init(smem_u32(&s_part_full[lane]), (uint32_t)(kEpiWarps * (split > 1 ? split - 1 : 1)));
-            mbar_init(smem_u32(&s_part_empty[lane]), (uint32_t)(kEpiWarps * (split > 1 ? split - 1 : 1)));
+        for (int a = 0; a < kAccStages; ++a) {
+            mbar_init(smem_u32(&s_acc_full[a]), 1);
+            mbar_init(smem_u32(&s_acc_empty[a]), kEpiWarps * CTAS);
         }
+        mbar_init(smem_u32(&s_epi_sync), kEpiWarps);
         fence_mbarrier_init();
         fence_proxy_async_smem();
     }
     if (warp == 1) tmem_alloc<CTAS>(smem_u32(&s_tmem_base), (uint32_t)p.tmem_cols);
     tc_fence_before();
     __syncthreads();
-    if (CTAS == 2 || split > 1) cluster_sync_all(); // the peers' barriers exist before anyone signals them
+    if (CTAS == 2) cluster_sync_all();              // the peer's barriers exist before anyone signals them
     tc_fence_after();
     const uint32_t tmem_base = s_tmem_base;
     // Everything above is on-chip setup; from here on global memory is touched (activations written
@@ -382,19 +381,23 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     // The weight producers do not wait: a weight handle is complete before any call that uses it
     // is enqueued, so its tiles can stream in while the kernel ahead (the prologue) still runs.
     const bool weight_producer = BITS == 8 ? warp == kFirstUnpackWarp : warp == kFirstUnpackWarp + 4 * kUnpackSets;
+#if defined(FQ_GEMM_TRACE) || defined(FQ_GEMM_DEV)
+    if (!weight_producer || (p.dbg & 8)) griddep_wait();
+#else
     if (!weight_producer) griddep_wait();
+#endif
     if (warp == 1) FQ_TRACE(3, 1023, 2);             // previous kernel complete
     griddep_launch_dependents();
 
-    // work units: (super-tile of 128*CTAS channels) x (token tile); one unit per CTA or CTA pair at a time
-    const int num_tiles = p.m_tiles * p.n_tiles;
+    // work units: (super-tile of 128*CTAS channels) x (token tile) [x K slice]; one unit per CTA or
+    // CTA pair at a time
+    const int num_units = (p.m_tiles * p.n_tiles) << split_shift;
     const int unit0 = (int)blockIdx.x >> p.cluster_shift;
     const int unit_step = p.unit_step;
-    const int my_tiles = p.tiles_q + (unit0 < p.tiles_rem ? 1 : 0);
-    const int k_blocks_all = p.k_blocks_all;
-    const int kb_per = (SPLIT && CTAS == 1) ? p.kb_per : k_blocks_all;
-    const int kb0 = (int)krank * kb_per;                               // first k-block of this rank
-    const int k_blocks = kb0 + kb_per <= k_blocks_all ? kb_per : k_blocks_all - kb0;   // >= 1 (host check)
+    const int my_units = p.units_q + (unit0 < p.units_rem ? 1 : 0);
+    const int k_blocks = p.kb_per;
+    auto tile_of = [&](int unit) { return unit >> split_shift; };
+    auto kb0_of = [&](int unit) { return (unit & (split - 1)) * k_blocks; };   // first k-block of the unit's slice
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
@@ -403,11 +406,12 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         // hand-off: every dependent wait/branch of the lone lane pays for the divergent warp.)
         {
             const uint32_t tx = a_bytes;
-            const int total_kb = my_tiles * k_blocks;
+            const int total_kb = my_units * k_blocks;
             bool ok = true;
-            int stage = 0, kb = 0, tile = unit0;
+            int stage = 0, kb = 0, unit = unit0;
             uint32_t phase = 0;
-            int t0 = (tile % p.m_tiles) * p.bt + (int)cta_rank * bt_cta;
+            int t0 = (tile_of(unit) % p.m_tiles) * p.bt + (int)cta_rank * bt_cta;
+            int kb0 = kb0_of(unit);
             bool peek = false;
             for (int n = 0; n < total_kb; ++n) {
                 ok = mbar_wait_all(smem_u32(&s_empty[stage]), phase ^ 1u, abort_flag, p.watchdog, kWdProducer, peek);
@@ -433,8 +437,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                 if (++stage == p.stages) { stage = 0; phase ^= 1u; }
                 if (++kb == k_blocks) {
                     kb = 0;
-                    tile += unit_step;
-                    t0 = (tile % p.m_tiles) * p.bt + (int)cta_rank * bt_cta;
+                    unit += unit_step;
+                    t0 = (tile_of(unit) % p.m_tiles) * p.bt + (int)cta_rank * bt_cta;
+                    kb0 = kb0_of(unit);
                 }
             }
             if (!ok && lane == 0) drain_after_abort();
@@ -454,9 +459,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             // that issues the current one: a barrier test has ~100 cycles of latency, and two of them
             // in series per k-block would otherwise sit on the issuing warp's critical path.
             bool ready = false;
-            int left = my_tiles * k_blocks;   // k-blocks still to issue
+            int left = my_units * k_blocks;   // k-blocks still to issue
             [[maybe_unused]] int tn = 0;
-            for (int tile = unit0; tile < num_tiles && ok; tile += unit_step) {
+            for (int unit = unit0; unit < num_units && ok; unit += unit_step) {
                 ok = mbar_wait_all(smem_u32(&s_acc_empty[acc_stage]), acc_phase ^ 1u, abort_flag, p.watchdog, kWdMmaAcc);
                 if (!ok) break;
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc_stage * p.bt);
@@ -517,8 +522,11 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         const float unshift = 1.0f / (float)(1 << p.acc_shift);   // exact power of two
         int acc_stage = 0;
         uint32_t acc_phase = 0;
+        [[maybe_unused]] uint32_t epi_phase = 0;
+        [[maybe_unused]] int epi_use = 0;
         bool ok = true;
-        for (int tile = unit0; tile < num_tiles && ok; tile += unit_step) {
+        for (int unit = unit0; unit < num_units && ok; unit += unit_step) {
+            const int tile = tile_of(unit);
             const int64_t jq = (int64_t)(tile / p.m_tiles) * (kTileN * CTAS) + (int64_t)cta_rank * kTileN + quad * 32;   // first channel of this warp
             const int64_t j = jq + lane;
             const int64_t t0 = (int64_t)(tile % p.m_tiles) * p.bt;
@@ -530,47 +538,61 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             }
             ok = mbar_wait_warp_relaxed(smem_u32(&s_acc_full[acc_stage]), acc_phase, abort_flag, p.watchdog, kWdEpilogue);
             if (!ok) break;
-            if (warp == 2) { FQ_TRACE_B(0, 2, 0, 0); FQ_TRACE_B(1, 1, 0, 0); }
-            // K split.  Every rank finishes a share of the tile: this warp's k-th chunk of 16 tokens belongs
-            // to rank k % split.  A rank first hands the raw sums of the chunks it does not own to their
-            // owners (partial blocks [tile][writer rank][bt tokens][128 channels] int32: a warp's 32
-            // channels of one token are one 128-byte line, coalesced both ways), then waits for the
-            // other ranks' blocks and finishes its own chunks.
-            int32_t* part = nullptr;
+            // K split.  Every slice writes its raw int32 sums to its own block of scratch
+            // ([tile][slice][bt tokens][128 channels]: a warp's 32 channels of one token are one 128-byte
+            // line, coalesced both ways) and then counts itself in; the CTA that counts last adds the other
+            // slices to its own accumulator (still in TMEM) and runs the epilogue.  Nobody waits for anybody.
+            const int32_t* part = nullptr;
             const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc_stage * p.bt);
+            const int slice = unit & (split - 1);
             if (split > 1) {
                 tc_fence_after();
-                part = p.partials + (size_t)tile * (size_t)split * kTileN * (size_t)p.bt + (size_t)(quad * 32 + lane);
-                // flow control: the other ranks' barriers for this accumulator stage must not be signalled
-                // for a new tile before they have passed them for the previous one (phases would alias)
-                ok = mbar_wait_warp_relaxed(smem_u32(&s_part_empty[acc_stage]), acc_phase ^ 1u, abort_flag, p.watchdog,
-                                            kWdPartials);
-                if (!ok) break;
-                int32_t* mine = part + (size_t)krank * kTileN * (size_t)p.bt;
+                int32_t* tile_part = p.partials + (size_t)tile * (size_t)split * kTileN * (size_t)p.bt + (size_t)(quad * 32 + lane);
+                int32_t* mine = tile_part + (size_t)slice * kTileN * (size_t)p.bt;
                 for (int c = half * 16; c < p.bt; c += 32) {
                     if (t0 + c >= p.M) break;
-                    if ((uint32_t)((c >> 5) % split) == krank) continue;
                     uint32_t r[16];
                     tmem_ld16(taddr + (uint32_t)c, r);
                     tmem_ld_wait();
 #pragma unroll
                     for (int i = 0; i < 16; ++i) __stcg(mine + (size_t)(c + i) * kTileN, (int)r[i]);
                 }
-                __threadfence();                 // partial sums visible before the owners are told
+                __threadfence();                 // this slice's sums are visible before it is counted
+                // rendezvous 1: every epilogue warp has written and fenced its part
                 __syncwarp();
-                if (lane == 0)
-                    for (uint32_t rk = 0; rk < (uint32_t)split; ++rk)
-                        if (rk != krank) mbar_arrive_cta(smem_u32(&s_part_full[acc_stage]), rk);
-                ok = mbar_wait_warp_relaxed(smem_u32(&s_part_full[acc_stage]), acc_phase, abort_flag, p.watchdog, kWdPartials);
+                if (lane == 0) mbar_arrive(smem_u32(&s_epi_sync));
+                ok = mbar_wait_all(smem_u32(&s_epi_sync), epi_phase, abort_flag, p.watchdog, kWdPartials);
+                epi_phase ^= 1u;
                 if (!ok) break;
-                __threadfence();
+                int* last_slot = &s_last[epi_use & 1];
+                if (warp == 2 && lane == 0) {
+                    const uint32_t done = atomicAdd(p.counters + tile, 1u);
+                    *last_slot = done == (uint32_t)(split - 1) ? 1 : 0;
+                    if (*last_slot) p.counters[tile] = 0u;   // every slice has been counted: ready for the next launch
+                }
+                // rendezvous 2: the verdict is written (its slot is reused two tiles later, after both
+                // rendezvous of the next tile)
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&s_epi_sync));
+                ok = mbar_wait_all(smem_u32(&s_epi_sync), epi_phase, abort_flag, p.watchdog, kWdPartials);
+                epi_phase ^= 1u;
+                if (!ok) break;
+                const bool last = *reinterpret_cast<volatile int*>(last_slot) != 0;
+                ++epi_use;
+                if (!last) {
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&s_acc_empty[acc_stage]));
+                    if (++acc_stage == kAccStages) { acc_stage = 0; acc_phase ^= 1u; }
+                    continue;
+                }
+                __threadfence();                 // the other slices' sums, written through L2
+                part = tile_part;
             }
             tc_fence_after();
-            if (warp == 2) { FQ_TRACE_B(0, 2, 0, 1); FQ_TRACE_B(1, 1, 0, 1); }
             for (int c = half * 16; c < p.bt; c += 32) {
                 const int64_t tc = t0 + c;
                 if (tc >= p.M) break;                    // tokens beyond M: nothing to store (warp-uniform)
-                if (split > 1 && (uint32_t)((c >> 5) % split) != krank) continue;   // another rank finishes this chunk
                 uint32_t r[16];
 #if defined(FQ_GEMM_TRACE) || defined(FQ_GEMM_DEV)
                 if (p.dbg & 4) continue;
@@ -580,8 +602,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                     int32_t pv[16];
 #pragma unroll
                     for (int i = 0; i < 16; ++i) pv[i] = 0;
-                    for (uint32_t rk = 0; rk < (uint32_t)split; ++rk) {
-                        if (rk == krank) continue;
+                    for (int rk = 0; rk < split; ++rk) {
+                        if (rk == slice) continue;
                         const int32_t* src = part + ((size_t)rk * (size_t)p.bt + (size_t)c) * kTileN;
 #pragma unroll
                         for (int i = 0; i < 16; ++i) pv[i] += __ldcg(src + (size_t)i * kTileN);
@@ -663,14 +685,6 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                     }
                 }
             }
-            if (warp == 2) { FQ_TRACE_B(0, 2, 0, 2); FQ_TRACE_B(1, 1, 0, 2); }
-            if (split > 1) {
-                __syncwarp();
-                if (lane == 0)
-                    for (uint32_t rk = 0; rk < (uint32_t)split; ++rk)
-                        if (rk != krank) mbar_arrive_cta(smem_u32(&s_part_empty[acc_stage]), rk);
-            }
-            if (warp == 2) { FQ_TRACE_B(0, 2, 0, 3); FQ_TRACE_B(1, 1, 0, 3); }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) {
@@ -683,11 +697,12 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         // ------------------------------------------------- TMA producer, int8 weights
         // (converged warp, one issuing lane: see the activation producer)
         {
-            const int total_kb = my_tiles * k_blocks;
+            const int total_kb = my_units * k_blocks;
             bool ok = true;
-            int stage = 0, kb = 0, tile = unit0;
+            int stage = 0, kb = 0, unit = unit0;
             uint32_t phase = 0;
-            int n0 = (tile / p.m_tiles) * (kTileN * CTAS) + (int)cta_rank * kTileN;
+            int n0 = (tile_of(unit) / p.m_tiles) * (kTileN * CTAS) + (int)cta_rank * kTileN;
+            int kb0 = kb0_of(unit);
             bool peek = false;
             for (int n = 0; n < total_kb; ++n) {
                 ok = mbar_wait_all(smem_u32(&s_empty[stage]), phase ^ 1u, abort_flag, p.watchdog, kWdProducer, peek);
@@ -710,8 +725,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                 if (++stage == p.stages) { stage = 0; phase ^= 1u; }
                 if (++kb == k_blocks) {
                     kb = 0;
-                    tile += unit_step;
-                    n0 = (tile / p.m_tiles) * (kTileN * CTAS) + (int)cta_rank * kTileN;
+                    unit += unit_step;
+                    n0 = (tile_of(unit) / p.m_tiles) * (kTileN * CTAS) + (int)cta_rank * kTileN;
+                    kb0 = kb0_of(unit);
                 }
             }
             if (!ok && lane == 0) drain_after_abort();
@@ -727,7 +743,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         // Set `uset` takes the k-blocks whose running index n is congruent to it modulo kUnpackSets,
         // so two k-blocks are in flight per quadrant and one set's store latency hides behind the other.
         const int uset = (warp - kFirstUnpackWarp) >> 2;
-        const int total_kb = my_tiles * k_blocks;
+        const int total_kb = my_units * k_blocks;
         bool ok = true;
         int ps = uset, ws = uset;                        // ring slots of k-block n, kept incrementally
         uint32_t pph = 0, wph = 0;
@@ -793,11 +809,12 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     } else if (BITS == 4) {
         // ------------------------------------------------- TMA producer, packed weights
         {
-            const int total_kb = my_tiles * k_blocks;
+            const int total_kb = my_units * k_blocks;
             bool ok = true;
-            int ps = 0, kb = 0, tile = unit0;
+            int ps = 0, kb = 0, unit = unit0;
             uint32_t pph = 0;
-            int n0 = (tile / p.m_tiles) * (kTileN * CTAS) + (int)cta_rank * kTileN;
+            int n0 = (tile_of(unit) / p.m_tiles) * (kTileN * CTAS) + (int)cta_rank * kTileN;
+            int kb0 = kb0_of(unit);
             bool peek = false;
             for (int n = 0; n < total_kb; ++n) {
                 ok = mbar_wait_all(smem_u32(&s_empty_p[ps]), pph ^ 1u, abort_flag, p.watchdog, kWdProducer, peek);
@@ -815,8 +832,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                 if (++ps == p.stages_p) { ps = 0; pph ^= 1u; }
                 if (++kb == k_blocks) {
                     kb = 0;
-                    tile += unit_step;
-                    n0 = (tile / p.m_tiles) * (kTileN * CTAS) + (int)cta_rank * kTileN;
+                    unit += unit_step;
+                    n0 = (tile_of(unit) / p.m_tiles) * (kTileN * CTAS) + (int)cta_rank * kTileN;
+                    kb0 = kb0_of(unit);
                 }
             }
             if (!ok && lane == 0) drain_after_abort();
@@ -827,7 +845,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     tc_fence_before();
     __syncthreads();
     if (warp == 1) FQ_TRACE(3, 1023, 3);             // all roles done
-    if (CTAS == 2 || split > 1) cluster_sync_all(); // no CTA leaves while another may still signal it
+    if (CTAS == 2) cluster_sync_all();              // neither CTA leaves while the other may still signal it
     if (warp == 1) {
         tc_fence_after();
         tmem_dealloc<CTAS>(tmem_base, (uint32_t)p.tmem_cols);
@@ -924,7 +942,7 @@ namespace {
 struct Plan {
     int bt = 0;       // tokens per tile
     int ctas = 1;     // 2: CTA pairs on 256-channel tiles (cta_group::2)
-    int split = 1;    // >1: that many CTAs of a cluster share a tile, each taking a slice of K
+    int split = 1;    // >1: every tile is that many work units, each on a slice of K
     size_t scratch = 0;   // bytes of int32 partial tiles the split needs
 };
 
@@ -938,10 +956,10 @@ struct Plan {
 //                                        both operands pass through it)
 //   8-bit, CTA pair:        per_kblock = max(545, 2.62*bt)   (each CTA stages half of the token tile)
 // Pairs gain nothing for 4-bit weights, which never pass through shared memory unpacked.
-// K split (single CTAs only): problems with fewer tiles than SMs and a long K (down_proj at M = 816:
-// 64 tiles of 128 k-blocks) can run `split` CTAs per tile; the ranks exchange int32 partial sums through
-// scratch and each finishes a share of the tile (measured cost of the exchange: about 6000 + 40*bt
-// cycles, + 1500 per extra rank, so the split pays only for long K and few tiles).
+// K split (single CTAs only): problems with fewer tiles than SMs and a long K (every short batch; down_proj
+// at M = 816: 64 tiles of 128 k-blocks) make `split` work units of every tile, each on a slice of K; the
+// slices leave int32 partial sums in scratch and the one that finishes last adds them up (fitted cost per
+// unit: 1500 + 70*bt cycles, plus 8*bt per extra slice).
 Plan plan_gemm(int64_t M, int64_t N, int64_t K, int bits, int sms, size_t scratch_avail) {
     const int bt_max = bits == 4 ? 208 : 256;
     const int64_t kb = (K + kBlockK - 1) / kBlockK;
@@ -955,15 +973,14 @@ Plan plan_gemm(int64_t M, int64_t N, int64_t K, int bits, int sms, size_t scratc
             const int64_t units = n_units * ((M + b - 1) / b);
             const double w8_single = 350.0 + 0.8 * b > 230.0 + 2.0 * b ? 350.0 + 0.8 * b : 230.0 + 2.0 * b;
             const double per_kb = bits == 4 ? 330.0 + b : (c == 1 ? w8_single : (2.62 * b > 545.0 ? 2.62 * b : 545.0));
-            for (int sp = 1; sp <= (c == 1 ? 8 : 1); sp *= 2) {
-                const int64_t kb_per = (kb + sp - 1) / sp;
-                if (sp > 1 && (kb_per * (sp - 1) >= kb || kb_per < 4 || units * sp > 2 * (int64_t)sms)) continue;
+            for (int sp = 1; sp <= (c == 1 ? kMaxSplit : 1); sp *= 2) {
+                if (sp > 1 && (kb % sp != 0 || kb / sp < 2 || units > kMaxSplitTiles || units * sp > 4 * (int64_t)sms)) continue;
+                const int64_t kb_per = kb / sp;
                 const size_t scratch = sp > 1 ? (size_t)units * sp * kTileN * b * sizeof(int32_t) : 0;
                 if (scratch > scratch_avail) continue;
-                const int slots = sms / (c * sp);
-                if (slots < 1) continue;
-                const double unit_cost = (double)kb_per * per_kb + 16.0 * b + 1000.0 + (sp > 1 ? 6000.0 + 40.0 * b + 1500.0 * (sp - 1) : 0.0);
-                const double cost = (double)((units + slots - 1) / slots) * unit_cost;
+                const int slots = sms / c;
+                const double unit_cost = (double)kb_per * per_kb + 16.0 * b + 1000.0 + (sp > 1 ? 1500.0 + 70.0 * b + 8.0 * b * (sp - 1) : 0.0);
+                const double cost = (double)((units * sp + slots - 1) / slots) * unit_cost;
                 if (best.bt == 0 || cost < best_cost * 0.98) {   // ties: the earlier candidate (larger tile, no split)
                     best.bt = b; best.ctas = c; best.split = sp; best.scratch = scratch;
                     best_cost = cost;
@@ -1001,7 +1018,15 @@ fq_status launch_gemm_tcgen05(const int8_t* a8, int64_t M, const Weights& W, int
 #if defined(FQ_GEMM_TRACE) || defined(FQ_GEMM_DEV)
     if (const char* e = getenv("FQ_BT")) { bt = atoi(e); split = 1; }       // development builds: force the token tile
     if (const char* e = getenv("FQ_PAIR")) { ctas = atoi(e); split = 1; }   // ... and single CTAs or pairs
-    if (const char* e = getenv("FQ_SPLIT")) split = atoi(e);                // ... and the K split
+    if (const char* e = getenv("FQ_SPLIT")) {                               // ... and the K split, if it is a legal one
+        const int sp = atoi(e);
+        const int64_t kb = (W.K + kBlockK - 1) / kBlockK;
+        const int64_t tiles = ((W.N + kTileN - 1) / kTileN) * ((M + bt - 1) / bt);
+        const bool legal = ctas == 1 && sp >= 1 && sp <= kMaxSplit && (sp & (sp - 1)) == 0 && kb % sp == 0 && kb / sp >= 2 &&
+                           tiles <= kMaxSplitTiles && scratch != nullptr &&
+                           (size_t)tiles * sp * kTileN * bt * sizeof(int32_t) <= scratch_bytes;
+        split = legal ? sp : 1;
+    }
     if (getenv("FQ_PLAN_PRINT")) fprintf(stderr, "plan: M=%lld N=%lld K=%lld bits=%d -> bt=%d ctas=%d split=%d\n", (long long)M, (long long)W.N, (long long)W.K, W.bits, bt, ctas, split);
 #endif
     p.split = split;
@@ -1058,25 +1083,25 @@ fq_status launch_gemm_tcgen05(const int8_t* a8, int64_t M, const Weights& W, int
     if (!encode_2d(&map_a, a8, (uint64_t)W.K, (uint64_t)M, kBlockK, (uint32_t)(bt / ctas), CU_TENSOR_MAP_SWIZZLE_128B))
         return FQ_ERR_CUDA;
 
-    const int num_units = p.m_tiles * p.n_tiles;
-    const int group = ctas * split;                  // CTAs of one cluster: a pair, or the ranks of a K split
-    const int max_units = sms / group;
+    const int num_units = p.m_tiles * p.n_tiles * split;       // a K split makes `split` units of every tile
+    const int max_units = sms / ctas;
     const int clusters = num_units < max_units ? num_units : max_units;
-    const int grid = clusters * group;
-    p.cluster_shift = group == 1 ? 0 : (group == 2 ? 1 : (group == 4 ? 2 : 3));
+    const int grid = clusters * ctas;
+    p.cluster_shift = ctas == 2 ? 1 : 0;
     p.unit_step = clusters;
-    p.tiles_q = num_units / clusters;
-    p.tiles_rem = num_units % clusters;
-    p.k_blocks_all = (int)((W.K + kBlockK - 1) / kBlockK);
-    p.kb_per = (p.k_blocks_all + split - 1) / split;
+    p.units_q = num_units / clusters;
+    p.units_rem = num_units % clusters;
+    p.kb_per = (int)((W.K + kBlockK - 1) / kBlockK) / split;    // the planner only picks splits that divide it
+    p.split_shift = split == 1 ? 0 : (split == 2 ? 1 : (split == 4 ? 2 : (split == 8 ? 3 : 4)));
+    p.counters = W.tile_counters;
 
     if (W.bits == 4) {
         if (ctas == 2) return launch_variant<4, 2, false>(map_a, W.tmap, p, grid, smem, 2, stream);
-        return split > 1 ? launch_variant<4, 1, true>(map_a, W.tmap, p, grid, smem, split, stream)
+        return split > 1 ? launch_variant<4, 1, true>(map_a, W.tmap, p, grid, smem, 1, stream)
                          : launch_variant<4, 1, false>(map_a, W.tmap, p, grid, smem, 1, stream);
     }
     if (ctas == 2) return launch_variant<8, 2, false>(map_a, W.tmap, p, grid, smem, 2, stream);
-    return split > 1 ? launch_variant<8, 1, true>(map_a, W.tmap, p, grid, smem, split, stream)
+    return split > 1 ? launch_variant<8, 1, true>(map_a, W.tmap, p, grid, smem, 1, stream)
                      : launch_variant<8, 1, false>(map_a, W.tmap, p, grid, smem, 1, stream);
 }
 

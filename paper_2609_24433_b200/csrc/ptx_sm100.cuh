@@ -121,7 +121,7 @@ __device__ __forceinline__ bool mbar_wait_warp_relaxed(uint32_t bar, uint32_t pa
     if ((threadIdx.x & 31) == 0) {
         const uint64_t t0 = global_timer_ns();
         for (uint32_t spin = 1; !mbar_try_wait(bar, parity); ++spin) {
-            __nanosleep(100);
+            __nanosleep(200);
             if ((spin & 0x3f) == 0) {
                 if (*abort_flag) { ok = 0; break; }
                 if (global_timer_ns() - t0 > kWaitLimitNs) {
