@@ -153,7 +153,9 @@ fq_status fq_linear_w4a4_static(const void* x, fq_dtype xt, int64_t M, int64_t l
 /* Bytes of workspace that fq_gemm_* / fq_linear_* want for this shape (host computation): the int8
  * activation codes and steps (M*K + 4*M bytes, each rounded up to 256), plus scratch for int32 partial
  * tiles on shapes with few output tiles and a long K, which the GEMM then splits along K.  A workspace
- * that holds only the first part is accepted; the GEMM then runs without the split. */
+ * that holds only the first part is accepted; the GEMM then runs without the split.  A split launch
+ * keeps per-tile counters in the weight handle: calls that may split K on the same handle must be
+ * ordered on one stream (or pass workspaces without the scratch part). */
 size_t fq_workspace_bytes(int64_t M, int64_t K, int64_t N, int bits);
 
 /* Parity/debug: raw int32 accumulators acc[M, N] (device, pitch N) of Eq. 8's integer sum. */
