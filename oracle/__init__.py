@@ -159,6 +159,43 @@ def fold_weights(W: np.ndarray, dtype: str, smooth, beta: int, bits: int, return
     return (codes, w_scale, g, wt) if return_wt else (codes, w_scale, g)
 
 
+def transform_quantize(x: np.ndarray, dtype: str, pre, post, beta: int, bits: int, clip_ratio: float = 1.0,
+                       return_z: bool = False):
+    """z = D^o (R (D^i x)) then Eq. 5, for the whole family T = D^o R D^i: ``pre`` = d^i * beta^-1/2 per
+    channel (None: the constant beta^-1/2), ``post`` = d^o per channel (None: 1).
+    Returns (codes, delta[, z])."""
+    x = _mat(x, dtype)
+    M, K = x.shape
+    codes = np.zeros((M, K * bits // 8), dtype=np.uint8)
+    delta = np.zeros(M, dtype=np.float32)
+    z = np.zeros((M, K), dtype=np.float32) if return_z else None
+    _check(_load().fqo_transform_quantize(_p(x), ctypes.c_int(_dt(dtype)), ctypes.c_int64(M), ctypes.c_int64(K),
+                                          ctypes.c_int64(K), _p(_f32(pre)), _p(_f32(post)), ctypes.c_int(beta),
+                                          ctypes.c_int(bits), ctypes.c_float(clip_ratio), _p(codes), _p(delta),
+                                          _p(z)), "transform_quantize")
+    return (codes, delta, z) if return_z else (codes, delta)
+
+
+def quantize_act_after(x: np.ndarray, dtype: str, g_post, beta: int, bits: int, clip_ratio: float = 1.0,
+                       return_z: bool = False):
+    """Runtime prologue of a fold-after site: z = P^-1 R x with g_post = 1/p."""
+    return transform_quantize(x, dtype, None, g_post, beta, bits, clip_ratio, return_z)
+
+
+def fold_weights_after(W: np.ndarray, dtype: str, p, beta: int, bits: int, return_wt: bool = False):
+    """Fold-after, offline: W~ = W R^T P, RTN, pack.  Returns (codes, w_scale[N], g_post[K] = 1/p[, W~])."""
+    W = _mat(W, dtype)
+    N, K = W.shape
+    codes = np.zeros((N, K * bits // 8), dtype=np.uint8)
+    w_scale = np.zeros(N, dtype=np.float32)
+    g = np.zeros(K, dtype=np.float32)
+    wt = np.zeros((N, K), dtype=np.float32) if return_wt else None
+    _check(_load().fqo_fold_weights_after(_p(W), ctypes.c_int(_dt(dtype)), ctypes.c_int64(N), ctypes.c_int64(K),
+                                          ctypes.c_int64(K), _p(_f32(p)), ctypes.c_int(beta), ctypes.c_int(bits),
+                                          _p(codes), _p(w_scale), _p(g), _p(wt)), "fold_weights_after")
+    return (codes, w_scale, g, wt) if return_wt else (codes, w_scale, g)
+
+
 def gemm_i32(a_codes: np.ndarray, w_codes: np.ndarray, K: int, bits: int) -> np.ndarray:
     a = np.ascontiguousarray(a_codes).view(np.uint8)
     w = np.ascontiguousarray(w_codes).view(np.uint8)

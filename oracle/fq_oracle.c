@@ -242,6 +242,58 @@ int fqo_quantize_act(const void* x, int dtype, int64_t M, int64_t K, int64_t ldx
     return 0;
 }
 
+/* The whole transform family of the section "Transforms supported by the runtime":
+ * T = D^o R D^i with positive diagonals, z = D^o (R (D^i x)), followed by Eq. 5.
+ *   pre  (optional) = d^i_c * beta^(-1/2) per channel, applied before the butterflies
+ *                     (NULL: the constant beta^(-1/2), i.e. D^i = I);
+ *   post (optional) = d^o_c per channel, applied after them (NULL: D^o = I).
+ * Fold-before is (pre, NULL), fold-after is (NULL, post).  With post == NULL this is
+ * fqo_quantize_act operation for operation.  z_out (optional) receives z [M, K]. */
+int fqo_transform_quantize(const void* x, int dtype, int64_t M, int64_t K, int64_t ldx, const float* pre,
+                           const float* post, int beta, int bits, float clip_ratio, uint8_t* codes,
+                           float* delta, float* z_out) {
+    if (!valid_block(beta, K) || (bits != 4 && bits != 8)) return 1;
+    if (!(clip_ratio > 0.0f && clip_ratio <= 1.0f)) return 1;
+    if (M < 0 || ldx < K || (M > 0 && (!x || !codes || !delta))) return 1;
+    float c = (float)(1.0 / sqrt((double)beta));
+    int64_t pitch = K * bits / 8;
+#pragma omp parallel
+    {
+        float* v = (float*)malloc(sizeof(float) * (size_t)K);
+        int* code = (int*)malloc(sizeof(int) * (size_t)K);
+#pragma omp for schedule(static)
+        for (int64_t t = 0; t < M; ++t) {
+            for (int64_t i = 0; i < K; ++i) {
+                float xv = load_elem(x, dtype, t * ldx + i);
+                float gi = pre ? pre[i] : c;
+                v[i] = xv * gi;
+            }
+            fqo_fwht_row(v, K, beta);
+            if (post)
+                for (int64_t i = 0; i < K; ++i) v[i] = v[i] * post[i];
+            if (z_out) memcpy(z_out + t * K, v, sizeof(float) * (size_t)K);
+            delta[t] = quantize_row(v, K, bits, clip_ratio, code);
+            pack_row(code, K, bits, codes + t * pitch);
+        }
+        free(v);
+        free(code);
+    }
+    return 0;
+}
+
+/* Fold-after, offline half: W~ = W R^T P, row j = (R w_j) (.) p (the block Hadamard matrix is
+ * symmetric), then RTN as in fqo_fold_weights.  mult_post (optional) receives the RUNTIME
+ * post-rotation multiplier 1/p_c (one binary32 division per channel); at run time the
+ * pre-rotation factor is the constant beta^(-1/2).  wt_out (optional) receives W~. */
+int fqo_fold_weights_after(const void* W, int dtype, int64_t N, int64_t K, int64_t ldw, const float* p,
+                           int beta, int bits, uint8_t* codes, float* w_scale, float* mult_post,
+                           float* wt_out) {
+    if (!p) return 1;
+    if (mult_post)
+        for (int64_t i = 0; i < K; ++i) mult_post[i] = 1.0f / p[i];
+    return fqo_transform_quantize(W, dtype, N, K, ldw, NULL, p, beta, bits, 1.0f, codes, w_scale, wt_out);
+}
+
 /* Offline half of Alg. 1 for one consumer with round-to-nearest:
  * row j of W~ = W S R^T is R (s (.) w_j) because the block Hadamard matrix is
  * symmetric.  Per-output-channel step s^W_j = max|W~_j| / q, no clipping.

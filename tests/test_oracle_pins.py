@@ -370,3 +370,90 @@ def test_bf16_helpers_match_torch():
     assert np.array_equal(synth.f32_to_bf16_bits(x), want)
     assert np.array_equal(synth.bf16_bits_to_f32(want),
                           torch.from_numpy(x).to(torch.bfloat16).float().numpy())
+
+
+# ------------------------------------- transform family T = D^o R D^i, fold-after ----
+def dense_rotation(K: int, beta: int) -> np.ndarray:
+    """R = I (x) beta^(-1/2) H_beta as a dense float64 matrix, built independently of the oracle."""
+    H = sylvester(beta).astype(np.float64) / np.sqrt(beta)
+    return np.kron(np.eye(K // beta), H)
+
+
+def test_transform_family_reduces_to_fold_before():
+    rng = np.random.default_rng(11)
+    x = rng.standard_normal((9, 256)).astype(np.float32)
+    g = (rng.random(256).astype(np.float32) + 0.5) / np.float32(8.0)
+    for bits in (4, 8):
+        a = oracle.quantize_act(x, "f32", g, 64, bits, 0.9)
+        b = oracle.transform_quantize(x, "f32", g, None, 64, bits, 0.9)
+        assert np.array_equal(a[0], b[0]) and np.array_equal(a[1].view(np.uint32), b[1].view(np.uint32))
+        # D^o = I written out as a vector of ones changes nothing (x * 1.0 is exact)
+        c = oracle.transform_quantize(x, "f32", g, np.ones(256, np.float32), 64, bits, 0.9)
+        assert np.array_equal(a[0], c[0]) and np.array_equal(a[1].view(np.uint32), c[1].view(np.uint32))
+
+
+def test_fold_after_hand_case():
+    """beta = K = 4: x = (1,1,1,1) -> R x = (2,0,0,0); p = (4,1,1,1) -> z = (0.5,0,0,0), delta = 0.5/7.
+    w = (2,2,2,2) -> R w = (4,0,0,0), times p = (16,0,0,0), s^W = 16/7.  codes (7,0,0,0) on both
+    sides, acc = 49, y = (0.5/7)(16/7) 49 = 8 = w . x."""
+    x = np.ones((1, 4), np.float32)
+    w = np.full((1, 4), 2.0, np.float32)
+    p = np.array([4, 1, 1, 1], np.float32)
+    wc, ws, gpost, wt = oracle.fold_weights_after(w, "f32", p, 4, 4, return_wt=True)
+    assert np.array_equal(wt, [[16, 0, 0, 0]]) and np.array_equal(gpost, [0.25, 1, 1, 1])
+    assert ws[0] == np.float32(16.0) / np.float32(7.0)
+    assert np.array_equal(oracle.unpack(wc, 4, 4), [[7, 0, 0, 0]])
+    ac, ad, z = oracle.quantize_act_after(x, "f32", gpost, 4, 4, return_z=True)
+    assert np.array_equal(z, [[0.5, 0, 0, 0]]) and ad[0] == np.float32(0.5) / np.float32(7.0)
+    assert np.array_equal(oracle.unpack(ac, 4, 4), [[7, 0, 0, 0]])
+    acc = oracle.gemm_i32(ac, wc, 4, 4)
+    assert acc[0, 0] == 49
+    y = oracle.epilogue(acc, ad, ws, np.zeros(1, np.float32))
+    assert abs(float(y[0, 0]) - 8.0) < 1e-5
+
+
+@pytest.mark.parametrize("beta", [4, 64, 256])
+def test_fold_after_matches_dense_matrices_and_preserves_the_projection(beta):
+    """z = P^-1 R x and W~ = W R^T P against dense float64 matrices (the diagonal sits AFTER the rotation on
+    the activation side and multiplies the rotated weight columns), and W~ z = W x before rounding."""
+    rng = np.random.default_rng(beta)
+    K, N, M = 2 * beta, 6, 5
+    x = rng.standard_normal((M, K)).astype(np.float32)
+    W = (rng.standard_normal((N, K)) * 0.1).astype(np.float32)
+    p = (rng.random(K) * 3 + 0.25).astype(np.float32)
+    R = dense_rotation(K, beta)
+    _, _, gpost, wt = oracle.fold_weights_after(W, "f32", p, beta, 8, return_wt=True)
+    _, _, z = oracle.quantize_act_after(x, "f32", gpost, beta, 8, return_z=True)
+    z_ref = (x.astype(np.float64) @ R.T) / p.astype(np.float64)
+    wt_ref = (W.astype(np.float64) @ R.T) * p.astype(np.float64)
+    assert np.allclose(z, z_ref, rtol=1e-5, atol=1e-6)
+    assert np.allclose(wt, wt_ref, rtol=1e-5, atol=1e-6)
+    assert np.allclose(wt.astype(np.float64) @ z.astype(np.float64).T, W.astype(np.float64) @ x.astype(np.float64).T,
+                       rtol=1e-4, atol=1e-5)
+    # fold-before with the same vector is a DIFFERENT transform (R S R^T is dense): the two must not coincide
+    _, _, g_before = oracle.fold_weights(W, "f32", p, beta, 8)
+    _, _, z_before = oracle.quantize_act(x, "f32", g_before, beta, 8, return_z=True)
+    assert not np.allclose(z_before, z, rtol=1e-3, atol=1e-4)
+
+
+def test_fold_after_end_to_end_accuracy_is_that_of_the_quantizer():
+    """Eq. 8 on a fold-after site: the output error stays at the level the code width allows."""
+    rng = np.random.default_rng(3)
+    M, K, N, beta = 32, 512, 48, 128
+    x = rng.standard_normal((M, K)).astype(np.float32)
+    x[:, :4] *= 30.0                                    # outlier channels
+    W = (rng.standard_normal((N, K)) * 0.02).astype(np.float32)
+    b = (rng.standard_normal(N) * 0.02).astype(np.float32)
+    R = dense_rotation(K, beta)
+    # P calibrated after rotation, in the coordinates where it is applied (SmoothQuant rule, alpha = 0.5)
+    a_rot = np.abs(x.astype(np.float64) @ R.T).max(0).astype(np.float32)
+    w_rot = np.abs(W.astype(np.float64) @ R.T).max(0).astype(np.float32)
+    p = oracle.smooth_scale(a_rot, w_rot, 0.5)
+    y_ref = x.astype(np.float64) @ W.astype(np.float64).T + b
+    errs = {}
+    for bits in (4, 8):
+        wc, ws, gpost = oracle.fold_weights_after(W, "f32", p, beta, bits)
+        ac, ad = oracle.quantize_act_after(x, "f32", gpost, beta, bits)
+        y = oracle.epilogue(oracle.gemm_i32(ac, wc, K, bits), ad, ws, b)
+        errs[bits] = np.linalg.norm(y - y_ref) / np.linalg.norm(y_ref)
+    assert errs[8] < 0.02 and errs[4] < 0.25 and errs[8] < errs[4] / 5
