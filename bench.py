@@ -120,7 +120,11 @@ class LayerOnDevice:
                 if site.alpha is not None:      # SmoothQuant scale from the calibration batch, on the device
                     a = fq.col_absmax(torch.from_numpy(data.calib).to(device))
                     smooth = fq.smooth_scale(a, fq.col_absmax(W), site.alpha)
-                h = fq.fold_weights(W, smooth, b, site.beta, site.bits)
+                if site.fold_after:
+                    pscale = torch.from_numpy(synth.post_scale(site, seed + 1000 * r + i)).to(device)
+                    h = fq.fold_weights_after(W, pscale, b, site.beta, site.bits)
+                else:
+                    h = fq.fold_weights(W, smooth, b, site.beta, site.bits)
                 ydt = torch.float32 if site.y_dtype == "f32" else torch.bfloat16
                 y = torch.empty((site.M, site.N_total), dtype=ydt, device=device)
                 ws = torch.empty(fq.workspace_bytes(site.M, site.K, site.N_total, site.bits), dtype=torch.uint8,
@@ -385,13 +389,20 @@ def cpu_baseline(workload: str, steps: int):
         smooth = None
         if site.alpha is not None:
             smooth = oracle.smooth_scale(oracle.col_absmax(data.calib), oracle.col_absmax(W), site.alpha)
-        wc, ws, g = oracle.fold_weights(W, "f32", smooth, site.beta, site.bits)      # offline, untimed
+        if site.fold_after:
+            wc, ws, g = oracle.fold_weights_after(W, "f32", synth.post_scale(site, 2 + i), site.beta, site.bits)
+        else:
+            wc, ws, g = oracle.fold_weights(W, "f32", smooth, site.beta, site.bits)      # offline, untimed
         prepared.append((site, np.ascontiguousarray(data.x[:rows]), g, wc, ws, b))
     times = []
     for _ in range(steps):
         t0 = time.perf_counter()
         for site, x, g, wc, ws, b in prepared:
-            oracle.linear(x, site.x_dtype, g, site.beta, site.bits, 1.0, wc, ws, b, site.y_dtype)
+            if site.fold_after:
+                ac, ad = oracle.quantize_act_after(x, site.x_dtype, g, site.beta, site.bits)
+                oracle.epilogue(oracle.gemm_i32(ac, wc, site.K, site.bits), ad, ws, b, site.y_dtype)
+            else:
+                oracle.linear(x, site.x_dtype, g, site.beta, site.bits, 1.0, wc, ws, b, site.y_dtype)
         times.append(time.perf_counter() - t0)
     ops = sum(2.0 * rows * s.K * s.N_total for s in sites)
     dt = statistics.mean(times)
@@ -428,16 +439,19 @@ def workload_sites(name: str):
         return synth.backbone_layer_sites(selective_int8=False)
     if name == "expert_layer":
         return synth.expert_layer_sites()
-    if name.startswith("sweep:"):        # one site of the throughput sweep: sweep:M,K,N,block,bits
-        M, K, N, beta, bits = (int(v) for v in name[6:].split(","))
-        return [synth.sweep_site(M, K, N, beta, bits)]
+    if name.startswith("sweep:"):        # one site of the throughput sweep: sweep:M,K,N,block,bits[,after]
+        f = name[6:].split(",")
+        M, K, N, beta, bits = (int(v) for v in f[:5])
+        return [synth.sweep_site(M, K, N, beta, bits, fold_after=len(f) > 5 and f[5] == "after")]
     raise ValueError(name)
 
 
 def workload_name(name: str) -> str:
     if name.startswith("sweep:"):
-        M, K, N, beta, bits = (int(v) for v in name[6:].split(","))
-        return f"throughput sweep point M={M} K={K} N={N}, block {beta}, W{bits}A{bits}"
+        f = name[6:].split(",")
+        M, K, N, beta, bits = (int(v) for v in f[:5])
+        return f"throughput sweep point M={M} K={K} N={N}, block {beta}, W{bits}A{bits}" + \
+               (", fold-after" if len(f) > 5 and f[5] == "after" else "")
     return {"backbone_layer": "pi0.5-like backbone layer, M=816, hidden 2048, MLP 16384, o/down W8A8, rest W4A4",
             "backbone_layer_w4": "pi0.5-like backbone layer, M=816, uniform W4A4",
             "expert_layer": "action-expert layer, M=50, width 1024, MLP 4096, W4A4, block 64"}[name]

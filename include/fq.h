@@ -70,6 +70,20 @@ fq_status fq_fold_weights(const void* W, fq_dtype wt, int64_t N, int64_t K, int6
                           const float* smooth, const float* bias, int hadamard_block, int bits,
                           void* stream, fq_weights** out);
 
+/* ---- offline, fold-after variant (section "Transforms supported by the runtime", Eq. 2 with
+ * (D^i, D^o) = (I, P^-1)): W~ = W R^T P, row j = (R w_j) (.) p, then RTN and packing as above.
+ * post_scale device float[K], the positive diagonal P calibrated AFTER rotation (statistics of R x and
+ * of W R^T; fq_col_absmax / fq_smooth_scale work on such rotated tensors like on any other).
+ * The handle's runtime multiplier is 1/p_c and is applied behind the rotation: z = P^-1 R x, with the
+ * constant block^-1/2 ahead of it (the paper's "extra pass" costs one multiply per element in the same
+ * kernel).  Every other call takes such a handle like a fold-before one. */
+fq_status fq_fold_weights_after(const void* W, fq_dtype wt, int64_t N, int64_t K, int64_t ldw,
+                                const float* post_scale, const float* bias, int hadamard_block, int bits,
+                                void* stream, fq_weights** out);
+
+/* 1 if the handle was folded after the rotation (its multiplier is the post-rotation 1/p), else 0. */
+int fq_weights_fold_after(const fq_weights* w);
+
 /* Frees the handle's device memory (cudaFree synchronises the device). NULL is accepted. */
 fq_status fq_weights_destroy(fq_weights* w);
 
@@ -88,6 +102,11 @@ fq_status fq_weights_import(const void* codes, const float* w_scale, const float
                             const float* bias, int64_t N, int64_t K, int hadamard_block, int bits,
                             void* stream, fq_weights** out);
 
+/* Import of a fold-after pack: mult_post device float[K] = 1/p (required). */
+fq_status fq_weights_import_after(const void* codes, const float* w_scale, const float* mult_post,
+                                  const float* bias, int64_t N, int64_t K, int hadamard_block, int bits,
+                                  void* stream, fq_weights** out);
+
 /* ---- calibration support (section "Transforms supported by the runtime", SmoothQuant scale) --
  * fq_col_absmax: out[c] = max(out[c] if accumulate else 0, max_t |x[t][c]|); x device [M, K].
  * fq_smooth_scale: s_c = clamp(max(a_c,1e-5)^alpha / max(w_c,1e-5)^(1-alpha), 1e-5, 1e5) in
@@ -105,6 +124,12 @@ fq_status fq_smooth_scale(const float* a, const float* w, int64_t K, double alph
 fq_status fq_quantize_act(const void* x, fq_dtype xt, int64_t M, int64_t K, int64_t ldx,
                           const float* mult_g, int hadamard_block, int bits, float clip_ratio,
                           void* codes_out, float* delta_out, void* stream);
+
+/* Runtime prologue of a fold-after site: z = P^-1 R x (mult_post = fq_weights_multiplier of a consumer
+ * folded with fq_fold_weights_after), then Eq. 5 as above. */
+fq_status fq_quantize_act_after(const void* x, fq_dtype xt, int64_t M, int64_t K, int64_t ldx,
+                                const float* mult_post, int hadamard_block, int bits, float clip_ratio,
+                                void* codes_out, float* delta_out, void* stream);
 
 /* ---- integer GEMM + rescale/bias epilogue on pre-quantized activations (Eq. 8) -----------------
  * a_codes device, canonical codes from fq_quantize_act with the same bit width as W.

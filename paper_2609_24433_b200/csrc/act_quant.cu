@@ -81,7 +81,7 @@ __global__ void __launch_bounds__(CACHE ? 512 : kMaxThreads)
 transform_quantize_kernel(const XT* __restrict__ x, int64_t rows, int K, int64_t ldx,
                           const float* __restrict__ mult, float cnorm, int block, float qmax,
                           float clip_ratio, uint8_t* __restrict__ codes, float* __restrict__ delta,
-                          int tpr, int rpc) {
+                          int tpr, int rpc, int mult_after) {
     __shared__ float s_part[2][32];   // per-warp partial maxima, double buffered
 
     griddep_wait();                   // launched with programmatic serialization: see launch_pdl
@@ -125,11 +125,11 @@ transform_quantize_kernel(const XT* __restrict__ x, int64_t rows, int K, int64_t
             const int64_t nrow = row + row_step;
             raw.load(x + nrow * ldx + col0, col_ok && nrow < rows);
 #pragma unroll
-            for (int i = 0; i < E; ++i) v[i] = __fmul_rn(v[i], g[i % (CACHE ? E : 1)]);
+            for (int i = 0; i < E; ++i) v[i] = __fmul_rn(v[i], mult_after ? cnorm : g[i % (CACHE ? E : 1)]);
         } else {
             raw.load(x + row * ldx + col0, row_ok);
             raw.widen(v);
-            if (mult != nullptr && col_ok) {
+            if (mult != nullptr && col_ok && !mult_after) {
 #pragma unroll
                 for (int i = 0; i < E / 4; ++i) {
                     const float4 t = __ldg(reinterpret_cast<const float4*>(mult + col0) + i);
@@ -166,6 +166,22 @@ transform_quantize_kernel(const XT* __restrict__ x, int64_t rows, int K, int64_t
             for (int i = 0; i < E; ++i) {
                 const float p = __shfl_xor_sync(0xffffffffu, v[i], lm);
                 v[i] = __fmaf_rn(v[i], sgn, p);
+            }
+        }
+        // fold-after sites: the diagonal sits behind the rotation (z = D^o R x)
+        if (mult_after) {
+            if (CACHE) {
+#pragma unroll
+                for (int i = 0; i < E; ++i) v[i] = __fmul_rn(v[i], g[i % (CACHE ? E : 1)]);
+            } else if (col_ok) {
+#pragma unroll
+                for (int i = 0; i < E / 4; ++i) {
+                    const float4 t = __ldg(reinterpret_cast<const float4*>(mult + col0) + i);
+                    v[4 * i + 0] = __fmul_rn(v[4 * i + 0], t.x);
+                    v[4 * i + 1] = __fmul_rn(v[4 * i + 1], t.y);
+                    v[4 * i + 2] = __fmul_rn(v[4 * i + 2], t.z);
+                    v[4 * i + 3] = __fmul_rn(v[4 * i + 3], t.w);
+                }
             }
         }
 
@@ -233,7 +249,7 @@ transform_quantize_kernel(const XT* __restrict__ x, int64_t rows, int K, int64_t
 }
 
 template <typename XT, int E, int FMT>
-cudaError_t launch_e(const XT* x, int64_t rows, int K, int64_t ldx, const float* mult, float cnorm,
+cudaError_t launch_e(const XT* x, int64_t rows, int K, int64_t ldx, const float* mult, float cnorm, int mult_after,
                      int block, int qmax, float clip_ratio, void* codes, float* delta, cudaStream_t stream) {
     const int tpr = ((K / E) + 31) / 32 * 32;
     if (tpr > kMaxThreads) return cudaErrorInvalidConfiguration;
@@ -251,7 +267,7 @@ cudaError_t launch_e(const XT* x, int64_t rows, int K, int64_t ldx, const float*
         int64_t grid = iters < (int64_t)sms * resident ? iters : (int64_t)sms * resident;
         if (grid < 1) grid = 1;
         launch_pdl(kern, (unsigned)grid, (unsigned)threads, 0, stream, 1u, x, rows, K, ldx, mult, cnorm, block, (float)qmax,
-                   clip_ratio, static_cast<uint8_t*>(codes), delta, tpr, rpc);
+                   clip_ratio, static_cast<uint8_t*>(codes), delta, tpr, rpc, mult_after);
     };
     const bool clamp = clip_ratio < 1.0f;
     if (threads <= 512) {
@@ -265,15 +281,15 @@ cudaError_t launch_e(const XT* x, int64_t rows, int K, int64_t ldx, const float*
 }
 
 template <typename XT, int FMT>
-cudaError_t launch_t(const XT* x, int64_t rows, int K, int64_t ldx, const float* mult, float cnorm, int block,
-                     int qmax, float clip_ratio, void* codes, float* delta, cudaStream_t stream) {
+cudaError_t launch_t(const XT* x, int64_t rows, int K, int64_t ldx, const float* mult, float cnorm, int mult_after,
+                     int block, int qmax, float clip_ratio, void* codes, float* delta, cudaStream_t stream) {
     // E = 8 keeps short rows spread over a full warp; E = 16 is the streaming default;
     // E = 32 holds K = 16384 in 512 threads (cached variant) and reaches K = 32768 in 1024.
     if (K % 16 != 0 || K <= 256)
-        return launch_e<XT, 8, FMT>(x, rows, K, ldx, mult, cnorm, block, qmax, clip_ratio, codes, delta, stream);
+        return launch_e<XT, 8, FMT>(x, rows, K, ldx, mult, cnorm, mult_after, block, qmax, clip_ratio, codes, delta, stream);
     if (K <= 8192)
-        return launch_e<XT, 16, FMT>(x, rows, K, ldx, mult, cnorm, block, qmax, clip_ratio, codes, delta, stream);
-    return launch_e<XT, 32, FMT>(x, rows, K, ldx, mult, cnorm, block, qmax, clip_ratio, codes, delta, stream);
+        return launch_e<XT, 16, FMT>(x, rows, K, ldx, mult, cnorm, mult_after, block, qmax, clip_ratio, codes, delta, stream);
+    return launch_e<XT, 32, FMT>(x, rows, K, ldx, mult, cnorm, mult_after, block, qmax, clip_ratio, codes, delta, stream);
 }
 
 __global__ void multipliers_kernel(const float* __restrict__ smooth, int K, float cnorm,
@@ -344,25 +360,26 @@ __global__ void expand_nibbles_kernel(const uint4* __restrict__ packed, int64_t 
 }  // namespace
 
 cudaError_t launch_transform_quantize(const void* x, fq_dtype xt, int64_t rows, int64_t K, int64_t ldx,
-                                      const float* mult, float cnorm, int block, int qmax, float clip_ratio,
-                                      StoreFmt fmt, void* codes, float* delta, cudaStream_t stream) {
+                                      const float* mult, float cnorm, bool mult_after_rotation, int block, int qmax,
+                                      float clip_ratio, StoreFmt fmt, void* codes, float* delta, cudaStream_t stream) {
     if (rows == 0) return cudaSuccess;
+    const int mult_after = (mult != nullptr && mult_after_rotation) ? 1 : 0;
     {   // long batches stream through the TMA-fed ring; everything else stays in registers
-        const cudaError_t e = launch_transform_quantize_ring(x, xt, rows, K, ldx, mult, cnorm, block, qmax, clip_ratio,
-                                                             fmt, codes, delta, stream);
+        const cudaError_t e = launch_transform_quantize_ring(x, xt, rows, K, ldx, mult, cnorm, mult_after != 0, block, qmax,
+                                                             clip_ratio, fmt, codes, delta, stream);
         if (e != cudaErrorNotSupported) return e;
     }
     const int k = (int)K;
     if (xt == FQ_F32) {
         const float* p = static_cast<const float*>(x);
-            if (fmt == StoreFmt::Nibble) return launch_t<float, 0>(p, rows, k, ldx, mult, cnorm, block, qmax, clip_ratio, codes, delta, stream);
-        if (fmt == StoreFmt::Int8) return launch_t<float, 1>(p, rows, k, ldx, mult, cnorm, block, qmax, clip_ratio, codes, delta, stream);
-        return launch_t<float, 2>(p, rows, k, ldx, mult, cnorm, block, qmax, clip_ratio, codes, delta, stream);
+            if (fmt == StoreFmt::Nibble) return launch_t<float, 0>(p, rows, k, ldx, mult, cnorm, mult_after, block, qmax, clip_ratio, codes, delta, stream);
+        if (fmt == StoreFmt::Int8) return launch_t<float, 1>(p, rows, k, ldx, mult, cnorm, mult_after, block, qmax, clip_ratio, codes, delta, stream);
+        return launch_t<float, 2>(p, rows, k, ldx, mult, cnorm, mult_after, block, qmax, clip_ratio, codes, delta, stream);
     }
     const __nv_bfloat16* p = static_cast<const __nv_bfloat16*>(x);
-    if (fmt == StoreFmt::Nibble) return launch_t<__nv_bfloat16, 0>(p, rows, k, ldx, mult, cnorm, block, qmax, clip_ratio, codes, delta, stream);
-    if (fmt == StoreFmt::Int8) return launch_t<__nv_bfloat16, 1>(p, rows, k, ldx, mult, cnorm, block, qmax, clip_ratio, codes, delta, stream);
-    return launch_t<__nv_bfloat16, 2>(p, rows, k, ldx, mult, cnorm, block, qmax, clip_ratio, codes, delta, stream);
+    if (fmt == StoreFmt::Nibble) return launch_t<__nv_bfloat16, 0>(p, rows, k, ldx, mult, cnorm, mult_after, block, qmax, clip_ratio, codes, delta, stream);
+    if (fmt == StoreFmt::Int8) return launch_t<__nv_bfloat16, 1>(p, rows, k, ldx, mult, cnorm, mult_after, block, qmax, clip_ratio, codes, delta, stream);
+    return launch_t<__nv_bfloat16, 2>(p, rows, k, ldx, mult, cnorm, mult_after, block, qmax, clip_ratio, codes, delta, stream);
 }
 
 cudaError_t launch_multipliers(const float* smooth, int64_t K, float cnorm, float* mult_w, float* mult_g,

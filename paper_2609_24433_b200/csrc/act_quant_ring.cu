@@ -93,6 +93,7 @@ struct RingParams {
     int K;
     float cnorm, qmax, clip_ratio;
     const float* mult;
+    int mult_after;    // 1: multiply by cnorm before the butterflies and by mult after them (fold-after sites)
     uint8_t* codes;
     float* delta;
     int gw;            // warps per row group (power of two)
@@ -210,7 +211,7 @@ transform_quantize_ring_kernel(const __grid_constant__ CUtensorMap map_x, const 
                     v[4 * i + 3] = make_float2(lo.w, hi.w);
                 }
             }
-            if (p.mult != nullptr) {
+            if (p.mult != nullptr && !p.mult_after) {
 #pragma unroll
                 for (int i = 0; i < H / 4; ++i) {
                     const float4 lo = lds128f_ordered(piece(g0, g1, i));
@@ -270,6 +271,19 @@ transform_quantize_ring_kernel(const __grid_constant__ CUtensorMap map_x, const 
                 const float2 q = make_float2(__shfl_xor_sync(0xffffffffu, v[i].x, lm),
                                              __shfl_xor_sync(0xffffffffu, v[i].y, lm));
                 v[i] = f2_fma(v[i], s2, q);
+            }
+        }
+
+        // fold-after sites: the diagonal sits behind the rotation (z = D^o R x)
+        if (p.mult_after && col_ok) {
+#pragma unroll
+            for (int i = 0; i < H / 4; ++i) {
+                const float4 lo = lds128f_ordered(piece(g0, g1, i));
+                const float4 hi = lds128f_ordered(piece(g0, g1, i + H / 4));
+                v[4 * i + 0] = f2_mul(v[4 * i + 0], make_float2(lo.x, hi.x));
+                v[4 * i + 1] = f2_mul(v[4 * i + 1], make_float2(lo.y, hi.y));
+                v[4 * i + 2] = f2_mul(v[4 * i + 2], make_float2(lo.z, hi.z));
+                v[4 * i + 3] = f2_mul(v[4 * i + 3], make_float2(lo.w, hi.w));
             }
         }
 
@@ -389,8 +403,9 @@ cudaError_t launch_ring_e(int e, int block, const CUtensorMap& map, const RingPa
 }  // namespace
 
 cudaError_t launch_transform_quantize_ring(const void* x, fq_dtype xt, int64_t rows, int64_t K, int64_t ldx,
-                                           const float* mult, float cnorm, int block, int qmax, float clip_ratio,
-                                           StoreFmt fmt, void* codes, float* delta, cudaStream_t stream) {
+                                           const float* mult, float cnorm, bool mult_after_rotation, int block,
+                                           int qmax, float clip_ratio, StoreFmt fmt, void* codes, float* delta,
+                                           cudaStream_t stream) {
     const size_t esz = xt == FQ_BF16 ? 2 : 4;
     const size_t row_bytes = (size_t)K * esz;
     // shape gate: whole 128-byte lines, at most 256 of them per box, blocks of 32..256 channels
@@ -424,7 +439,7 @@ cudaError_t launch_transform_quantize_ring(const void* x, fq_dtype xt, int64_t r
 
     RingParams p{};
     p.rows = rows; p.K = (int)K; p.cnorm = cnorm; p.qmax = (float)qmax; p.clip_ratio = clip_ratio;
-    p.mult = mult; p.codes = static_cast<uint8_t*>(codes); p.delta = delta; p.gw = gw; p.depth = depth;
+    p.mult = mult; p.mult_after = (mult != nullptr && mult_after_rotation) ? 1 : 0; p.codes = static_cast<uint8_t*>(codes); p.delta = delta; p.gw = gw; p.depth = depth;
     p.slot_bytes = (uint32_t)slot; p.g_bytes = (uint32_t)g_bytes;
     p.watchdog = watchdog_device_ptr();
     if (!p.watchdog) return cudaErrorUnknown;

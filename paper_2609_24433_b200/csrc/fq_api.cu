@@ -148,8 +148,9 @@ fq_status linear_impl(const void* x, fq_dtype xt, int64_t M, int64_t ldx, const 
     // Prologue writes one int8 per code into the workspace (4-bit codes stay in [-7, 7] and are laid
     // out in the channel order the GEMM's nibble unpack gives the weights).
     const int qmax = bits == 4 ? 7 : 127;
-    if (launch_transform_quantize(x, xt, M, W->K, ldx, W->mult_g, block_norm(W->block), W->block, qmax, clip_ratio,
-                                  bits == 4 ? StoreFmt::Int8Perm : StoreFmt::Int8, ws.a8, ws.delta, s) != cudaSuccess)
+    if (launch_transform_quantize(x, xt, M, W->K, ldx, W->mult_g, block_norm(W->block), W->fold_after, W->block, qmax,
+                                  clip_ratio, bits == 4 ? StoreFmt::Int8Perm : StoreFmt::Int8, ws.a8, ws.delta,
+                                  s) != cudaSuccess)
         return FQ_ERR_CUDA;
     if (g_profile_mark != nullptr) {
         // Inside a stream capture the mark must be an external event-record node to stay readable.
@@ -184,8 +185,11 @@ const char* fq_status_string(fq_status s) {
     return "unknown status";
 }
 
-fq_status fq_fold_weights(const void* Wsrc, fq_dtype wt, int64_t N, int64_t K, int64_t ldw, const float* smooth,
-                          const float* bias, int hadamard_block, int bits, void* stream, fq_weights** out) {
+namespace {
+// fold-before (after == false): diag = s, W~ = W S R^T, runtime multiplier (1/s) * block^-1/2 ahead of the rotation.
+// fold-after  (after == true):  diag = p, W~ = W R^T P, runtime multiplier 1/p behind the rotation.
+fq_status fold_impl(const void* Wsrc, fq_dtype wt, int64_t N, int64_t K, int64_t ldw, const float* smooth, bool after,
+                    const float* bias, int hadamard_block, int bits, void* stream, fq_weights** out) {
     if (!out) return FQ_ERR_INVALID_ARG;
     *out = nullptr;
     fq_status st = check_shape(N, K, hadamard_block, bits);
@@ -207,9 +211,11 @@ fq_status fq_fold_weights(const void* Wsrc, fq_dtype wt, int64_t N, int64_t K, i
         return FQ_ERR_NOMEM;
     }
     const float cn = block_norm(hadamard_block);
-    bool ok = launch_multipliers(smooth, K, cn, mult_w, w->mult_g, s) == cudaSuccess;
-    ok = ok && launch_transform_quantize(Wsrc, wt, N, K, ldw, mult_w, cn, hadamard_block, bits == 4 ? 7 : 127, 1.0f,
-                                         bits == 4 ? StoreFmt::Nibble : StoreFmt::Int8, w->codes, w->w_scale,
+    w->fold_after = after;
+    // fold-after: the two vectors are p itself (offline side) and 1/p (runtime side), without the block norm
+    bool ok = launch_multipliers(smooth, K, after ? 1.0f : cn, mult_w, w->mult_g, s) == cudaSuccess;
+    ok = ok && launch_transform_quantize(Wsrc, wt, N, K, ldw, mult_w, cn, after, hadamard_block, bits == 4 ? 7 : 127,
+                                         1.0f, bits == 4 ? StoreFmt::Nibble : StoreFmt::Int8, w->codes, w->w_scale,
                                          s) == cudaSuccess;
     if (N > 0) {
         if (bias)
@@ -226,6 +232,24 @@ fq_status fq_fold_weights(const void* Wsrc, fq_dtype wt, int64_t N, int64_t K, i
     }
     *out = reinterpret_cast<fq_weights*>(w);
     return FQ_OK;
+}
+
+}  // namespace
+
+fq_status fq_fold_weights(const void* Wsrc, fq_dtype wt, int64_t N, int64_t K, int64_t ldw, const float* smooth,
+                          const float* bias, int hadamard_block, int bits, void* stream, fq_weights** out) {
+    return fold_impl(Wsrc, wt, N, K, ldw, smooth, false, bias, hadamard_block, bits, stream, out);
+}
+
+fq_status fq_fold_weights_after(const void* Wsrc, fq_dtype wt, int64_t N, int64_t K, int64_t ldw, const float* post_scale,
+                                const float* bias, int hadamard_block, int bits, void* stream, fq_weights** out) {
+    if (!post_scale) return FQ_ERR_INVALID_ARG;
+    return fold_impl(Wsrc, wt, N, K, ldw, post_scale, true, bias, hadamard_block, bits, stream, out);
+}
+
+int fq_weights_fold_after(const fq_weights* wp) {
+    const Weights* w = reinterpret_cast<const Weights*>(wp);
+    return (w && w->fold_after) ? 1 : 0;
 }
 
 fq_status fq_weights_destroy(fq_weights* wp) {
@@ -265,8 +289,9 @@ fq_status fq_weights_export(const fq_weights* wp, void* codes, float* w_scale, f
     return ok ? FQ_OK : FQ_ERR_CUDA;
 }
 
-fq_status fq_weights_import(const void* codes, const float* w_scale, const float* mult_g, const float* bias,
-                            int64_t N, int64_t K, int hadamard_block, int bits, void* stream, fq_weights** out) {
+namespace {
+fq_status import_impl(const void* codes, const float* w_scale, const float* mult_g, bool after, const float* bias,
+                      int64_t N, int64_t K, int hadamard_block, int bits, void* stream, fq_weights** out) {
     if (!out) return FQ_ERR_INVALID_ARG;
     *out = nullptr;
     fq_status st = check_shape(N, K, hadamard_block, bits);
@@ -279,6 +304,7 @@ fq_status fq_weights_import(const void* codes, const float* w_scale, const float
     if (st != FQ_OK) return st;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const size_t code_bytes = (size_t)N * (size_t)K * bits / 8;
+    w->fold_after = after && mult_g != nullptr;
     bool ok = true;
     if (N > 0) {
         ok = ok && cudaMemcpyAsync(w->codes, codes, code_bytes, cudaMemcpyDeviceToDevice, s) == cudaSuccess;
@@ -303,6 +329,18 @@ fq_status fq_weights_import(const void* codes, const float* w_scale, const float
     *out = reinterpret_cast<fq_weights*>(w);
     return FQ_OK;
 }
+}  // namespace
+
+fq_status fq_weights_import(const void* codes, const float* w_scale, const float* mult_g, const float* bias,
+                            int64_t N, int64_t K, int hadamard_block, int bits, void* stream, fq_weights** out) {
+    return import_impl(codes, w_scale, mult_g, false, bias, N, K, hadamard_block, bits, stream, out);
+}
+
+fq_status fq_weights_import_after(const void* codes, const float* w_scale, const float* mult_post, const float* bias,
+                                  int64_t N, int64_t K, int hadamard_block, int bits, void* stream, fq_weights** out) {
+    if (!mult_post) return FQ_ERR_INVALID_ARG;
+    return import_impl(codes, w_scale, mult_post, true, bias, N, K, hadamard_block, bits, stream, out);
+}
 
 fq_status fq_col_absmax(const void* x, fq_dtype xt, int64_t M, int64_t K, int64_t ldx, int accumulate, float* out,
                         void* stream) {
@@ -318,9 +356,10 @@ fq_status fq_smooth_scale(const float* a, const float* w, int64_t K, double alph
                                                                                                      : FQ_ERR_CUDA;
 }
 
-fq_status fq_quantize_act(const void* x, fq_dtype xt, int64_t M, int64_t K, int64_t ldx, const float* mult_g,
-                          int hadamard_block, int bits, float clip_ratio, void* codes_out, float* delta_out,
-                          void* stream) {
+namespace {
+fq_status quantize_impl(const void* x, fq_dtype xt, int64_t M, int64_t K, int64_t ldx, const float* mult_g, bool after,
+                        int hadamard_block, int bits, float clip_ratio, void* codes_out, float* delta_out,
+                        void* stream) {
     if (M < 0 || K <= 0) return FQ_ERR_INVALID_ARG;
     if (bits != 4 && bits != 8) return FQ_ERR_INVALID_ARG;
     if (!(clip_ratio > 0.0f && clip_ratio <= 1.0f)) return FQ_ERR_INVALID_ARG;
@@ -332,11 +371,25 @@ fq_status fq_quantize_act(const void* x, fq_dtype xt, int64_t M, int64_t K, int6
         return FQ_ERR_ALIGNMENT;
     fq_status st = check_arch();
     if (st != FQ_OK) return st;
-    cudaError_t e = launch_transform_quantize(x, xt, M, K, ldx, mult_g, block_norm(hadamard_block), hadamard_block,
-                                              bits == 4 ? 7 : 127, clip_ratio,
+    cudaError_t e = launch_transform_quantize(x, xt, M, K, ldx, mult_g, block_norm(hadamard_block), after,
+                                              hadamard_block, bits == 4 ? 7 : 127, clip_ratio,
                                               bits == 4 ? StoreFmt::Nibble : StoreFmt::Int8, codes_out, delta_out,
                                               static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? FQ_OK : FQ_ERR_CUDA;
+}
+}  // namespace
+
+fq_status fq_quantize_act(const void* x, fq_dtype xt, int64_t M, int64_t K, int64_t ldx, const float* mult_g,
+                          int hadamard_block, int bits, float clip_ratio, void* codes_out, float* delta_out,
+                          void* stream) {
+    return quantize_impl(x, xt, M, K, ldx, mult_g, false, hadamard_block, bits, clip_ratio, codes_out, delta_out, stream);
+}
+
+fq_status fq_quantize_act_after(const void* x, fq_dtype xt, int64_t M, int64_t K, int64_t ldx, const float* mult_post,
+                                int hadamard_block, int bits, float clip_ratio, void* codes_out, float* delta_out,
+                                void* stream) {
+    if (!mult_post) return FQ_ERR_INVALID_ARG;
+    return quantize_impl(x, xt, M, K, ldx, mult_post, true, hadamard_block, bits, clip_ratio, codes_out, delta_out, stream);
 }
 
 fq_status fq_gemm_w4a4(const void* a_codes, const float* a_delta, int64_t M, const fq_weights* W, void* y,

@@ -20,6 +20,7 @@ struct Weights {
     float* w_scale = nullptr;   // [N]
     float* bias = nullptr;      // [N]
     float* mult_g = nullptr;    // [K] runtime multiplier (1/s_c) * block^-1/2
+    bool fold_after = false;    // mult_g is the post-rotation multiplier 1/p (T = P^-1 R) instead of (1/s) block^-1/2
     uint32_t* tile_counters = nullptr;   // [1024] zero between launches: slices of a tile finished (K split)
     CUtensorMap tmap;           // TMA view of `codes` for the GEMM's weight operand
     bool tmap_valid = false;
@@ -62,9 +63,11 @@ enum class StoreFmt : int { Nibble = 0, Int8 = 1, Int8Perm = 2 };
 // Runtime prologue / offline fold share one kernel: multiply by mult[K] (or the
 // constant `cnorm` if mult == nullptr), block FWHT, per-row absmax, quantize to
 // +-qmax, store codes in `fmt`, store per-row step to delta.
+// mult_after_rotation (fold-after sites, T = D^o R): multiply by `cnorm` before the butterflies
+// and by mult[K] after them instead.
 cudaError_t launch_transform_quantize(const void* x, fq_dtype xt, int64_t rows, int64_t K, int64_t ldx,
-                                      const float* mult, float cnorm, int block, int qmax,
-                                      float clip_ratio, StoreFmt fmt, void* codes, float* delta,
+                                      const float* mult, float cnorm, bool mult_after_rotation, int block,
+                                      int qmax, float clip_ratio, StoreFmt fmt, void* codes, float* delta,
                                       cudaStream_t stream);
 
 // mult_w[c] = s_c * cnorm, mult_g[c] = (1/s_c) * cnorm (smooth == nullptr: both = cnorm).
@@ -107,8 +110,9 @@ bool encode_tiled(CUtensorMap* map, CUtensorMapDataType dt, uint32_t rank, const
 // Streaming variant of the prologue (TMA-fed shared-memory ring). Returns cudaErrorNotSupported
 // when the shape does not fit it; the caller then uses the register-only kernel.
 cudaError_t launch_transform_quantize_ring(const void* x, fq_dtype xt, int64_t rows, int64_t K, int64_t ldx,
-                                           const float* mult, float cnorm, int block, int qmax, float clip_ratio,
-                                           StoreFmt fmt, void* codes, float* delta, cudaStream_t stream);
+                                           const float* mult, float cnorm, bool mult_after_rotation, int block,
+                                           int qmax, float clip_ratio, StoreFmt fmt, void* codes, float* delta,
+                                           cudaStream_t stream);
 
 // Builds the weight-operand tensor map of a handle (after `codes` is allocated).
 fq_status build_weight_tmap(Weights& W);

@@ -80,7 +80,7 @@ extern "C" fq_status fq_linear_w4a4_static(const void* x, fq_dtype xt, int64_t M
     float* delta = reinterpret_cast<float*>(scratch + kCodeBytes);   // [M] steps,    rows < M rewritten below
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const float cnorm = (float)(1.0 / sqrt((double)W->block));
-    if (launch_transform_quantize(x, xt, M, W->K, ldx, W->mult_g, cnorm, W->block, 7, clip_ratio, StoreFmt::Int8Perm, a8,
+    if (launch_transform_quantize(x, xt, M, W->K, ldx, W->mult_g, cnorm, W->fold_after, W->block, 7, clip_ratio, StoreFmt::Int8Perm, a8,
                                   delta, s) != cudaSuccess)
         return FQ_ERR_CUDA;
     GemmOut out;

@@ -24,6 +24,7 @@ EXPORTS = [
     "fq_weights_export", "fq_weights_import", "fq_col_absmax", "fq_smooth_scale", "fq_quantize_act",
     "fq_gemm_w4a4", "fq_gemm_w8a8", "fq_linear_w4a4", "fq_linear_w8a8", "fq_workspace_bytes",
     "fq_gemm_acc_i32", "fq_gemm_simt", "fq_device_status", "fq_profile_mark", "fq_linear_w4a4_static",
+    "fq_fold_weights_after", "fq_weights_fold_after", "fq_weights_import_after", "fq_quantize_act_after",
 ]
 
 _lib = None
@@ -47,6 +48,8 @@ def lib() -> ctypes.CDLL:
         L.fq_status_string.argtypes = [ctypes.c_int]
         L.fq_weights_multiplier.restype = ctypes.c_void_p
         L.fq_weights_multiplier.argtypes = [ctypes.c_void_p]
+        L.fq_weights_fold_after.restype = ctypes.c_int
+        L.fq_weights_fold_after.argtypes = [ctypes.c_void_p]
         L.fq_workspace_bytes.restype = ctypes.c_size_t
         L.fq_workspace_bytes.argtypes = [ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, ctypes.c_int]
         _lib = L
@@ -98,6 +101,7 @@ class Weights:
         _check(lib().fq_weights_info(self._h, ctypes.byref(n), ctypes.byref(k), ctypes.byref(blk),
                                      ctypes.byref(bits)), "fq_weights_info")
         self.N, self.K, self.block, self.bits = n.value, k.value, blk.value, bits.value
+        self.fold_after = bool(lib().fq_weights_fold_after(self._h))
 
     @property
     def handle(self) -> ctypes.c_void_p:
@@ -142,13 +146,27 @@ def fold_weights(W: torch.Tensor, smooth: Optional[torch.Tensor], bias: Optional
     return Weights(out.value)
 
 
-def weights_import(codes: torch.Tensor, w_scale: torch.Tensor, mult_g: Optional[torch.Tensor],
-                   bias: Optional[torch.Tensor], K: int, hadamard_block: int, bits: int) -> Weights:
+def fold_weights_after(W: torch.Tensor, post_scale: torch.Tensor, bias: Optional[torch.Tensor],
+                       hadamard_block: int, bits: int) -> Weights:
+    """Fold-after variant: W~ = W R^T P; the handle's multiplier 1/p is applied behind the rotation."""
+    W = _rowmajor(W)
     out = ctypes.c_void_p()
-    _check(lib().fq_weights_import(_ptr(codes), _ptr(w_scale), _ptr(mult_g), _ptr(bias),
+    _check(lib().fq_fold_weights_after(_ptr(W), _dt(W), ctypes.c_int64(W.shape[0]), ctypes.c_int64(W.shape[1]),
+                                       ctypes.c_int64(W.stride(0)), _ptr(post_scale), _ptr(bias),
+                                       ctypes.c_int(hadamard_block), ctypes.c_int(bits), _stream(),
+                                       ctypes.byref(out)), "fq_fold_weights_after")
+    return Weights(out.value)
+
+
+def weights_import(codes: torch.Tensor, w_scale: torch.Tensor, mult_g: Optional[torch.Tensor],
+                   bias: Optional[torch.Tensor], K: int, hadamard_block: int, bits: int,
+                   fold_after: bool = False) -> Weights:
+    out = ctypes.c_void_p()
+    fn_name = "fq_weights_import_after" if fold_after else "fq_weights_import"
+    _check(getattr(lib(), fn_name)(_ptr(codes), _ptr(w_scale), _ptr(mult_g), _ptr(bias),
                                    ctypes.c_int64(codes.shape[0]), ctypes.c_int64(K),
                                    ctypes.c_int(hadamard_block), ctypes.c_int(bits), _stream(), ctypes.byref(out)),
-           "fq_weights_import")
+           fn_name)
     return Weights(out.value)
 
 
@@ -172,8 +190,10 @@ def smooth_scale(a: torch.Tensor, w: torch.Tensor, alpha: float) -> torch.Tensor
 
 
 def quantize_act(x: torch.Tensor, mult_g, hadamard_block: int, bits: int, clip_ratio: float = 1.0,
-                 codes: Optional[torch.Tensor] = None, delta: Optional[torch.Tensor] = None):
-    """Runtime prologue. ``mult_g``: device float tensor, a Weights (its multiplier) or None."""
+                 codes: Optional[torch.Tensor] = None, delta: Optional[torch.Tensor] = None,
+                 fold_after: Optional[bool] = None):
+    """Runtime prologue. ``mult_g``: device float tensor, a Weights (its multiplier) or None.
+    ``fold_after``: the multiplier is the post-rotation 1/p (default: what the Weights says, else False)."""
     x = _rowmajor(x)
     M, K = x.shape
     if codes is None:
@@ -182,11 +202,14 @@ def quantize_act(x: torch.Tensor, mult_g, hadamard_block: int, bits: int, clip_r
         delta = torch.empty(M, dtype=torch.float32, device=x.device)
     if isinstance(mult_g, Weights):
         g = ctypes.c_void_p(mult_g.multiplier_ptr())
+        if fold_after is None:
+            fold_after = mult_g.fold_after
     else:
         g = _ptr(mult_g)
-    _check(lib().fq_quantize_act(_ptr(x), _dt(x), ctypes.c_int64(M), ctypes.c_int64(K), ctypes.c_int64(x.stride(0)),
-                                 g, ctypes.c_int(hadamard_block), ctypes.c_int(bits), ctypes.c_float(clip_ratio),
-                                 _ptr(codes), _ptr(delta), _stream()), "fq_quantize_act")
+    fn_name = "fq_quantize_act_after" if fold_after else "fq_quantize_act"
+    _check(getattr(lib(), fn_name)(_ptr(x), _dt(x), ctypes.c_int64(M), ctypes.c_int64(K), ctypes.c_int64(x.stride(0)),
+                                   g, ctypes.c_int(hadamard_block), ctypes.c_int(bits), ctypes.c_float(clip_ratio),
+                                   _ptr(codes), _ptr(delta), _stream()), fn_name)
     return codes, delta
 
 

@@ -62,6 +62,7 @@ class Site:
     outlier_kind: str = "student_t"           # 'student_t' | 'scale'
     outlier_gain: float = 30.0
     sigma: float = 1.0
+    fold_after: bool = False                  # the site's diagonal sits behind the rotation (T = P^-1 R)
 
     @property
     def N_total(self) -> int:
@@ -159,9 +160,17 @@ def expert_layer_sites(M: int = 50, width: int = 1024, mlp: int = 4096, sigma: f
     ]
 
 
-def sweep_site(M: int, K: int, N: int, beta: int, bits: int) -> Site:
-    return Site(f"sweep_m{M}_k{K}_n{N}_b{beta}_w{bits}", M, K, [("proj", N)], beta=beta, bits=bits,
-                alpha=None, outlier_frac=0.005, outlier_kind="scale", outlier_gain=30.0)
+def sweep_site(M: int, K: int, N: int, beta: int, bits: int, fold_after: bool = False) -> Site:
+    return Site(f"sweep_m{M}_k{K}_n{N}_b{beta}_w{bits}" + ("_after" if fold_after else ""), M, K, [("proj", N)],
+                beta=beta, bits=bits, alpha=None, outlier_frac=0.005, outlier_kind="scale", outlier_gain=30.0,
+                fold_after=fold_after)
+
+
+def post_scale(site: Site, seed: int) -> np.ndarray:
+    """Positive post-rotation diagonal P of a fold-after site: log-uniform in [1/e, e] (stands in for a
+    calibrated one; the kernels do not care where it came from)."""
+    rng = np.random.default_rng(seed + 424243)
+    return np.exp(rng.uniform(-1.0, 1.0, site.K)).astype(np.float32)
 
 
 def expert_step_sigma(step: int, steps: int = 10) -> float:

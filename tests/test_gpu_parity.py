@@ -162,6 +162,68 @@ def test_fold_weights_bit_exact(N, K, block, bits, wdtype, smooth):
     assert torch.equal(c2, codes) and torch.equal(s2, scale) and torch.equal(g2, g) and torch.equal(b2, b)
 
 
+# ------------------------------------------------- fold-after variant (T = P^-1 R) ----
+AFTER_CASES = [
+    # M, K, block, bits, dtype, clip      (register kernel: short batches / small K; ring kernel: the rest)
+    (50, 1024, 64, 4, "bf16", 1.0),
+    (64, 1024, 128, 4, "f32", 1.0),
+    (9, 96, 32, 8, "bf16", 0.9),
+    (33, 512, 8, 8, "f32", 1.0),
+    (131, 16384, 256, 4, "f32", 0.8),
+    (816, 2048, 128, 4, "bf16", 1.0),
+    (816, 2048, 128, 8, "bf16", 1.0),
+    (600, 4096, 64, 8, "f32", 1.0),
+    (1000, 16384, 256, 8, "bf16", 1.0),
+    (700, 8192, 32, 4, "bf16", 0.6),
+    (333, 3072, 128, 4, "bf16", 1.0),
+]
+
+
+@pytest.mark.parametrize("M,K,block,bits,dtype,clip", AFTER_CASES)
+def test_quantize_act_after_bit_exact(M, K, block, bits, dtype, clip):
+    x = make_x(M, K, dtype, seed=M + K + block + 1)
+    rng = np.random.default_rng(K + 1)
+    gpost = (np.float32(1.0) / np.exp(rng.uniform(-2, 2, K)).astype(np.float32)).astype(np.float32)
+    want_codes, want_delta = oracle.quantize_act_after(x, dtype, gpost, block, bits, clip)
+    codes, delta = fq.quantize_act(to_dev(x, dtype), to_dev(gpost), block, bits, clip, fold_after=True)
+    assert np.array_equal(to_np(delta).view(np.uint32), want_delta.view(np.uint32))
+    assert np.array_equal(to_np(codes), want_codes)
+    # the same vector ahead of the rotation is a different transform: the flag must matter
+    other, _ = fq.quantize_act(to_dev(x, dtype), to_dev(gpost), block, bits, clip, fold_after=False)
+    assert not torch.equal(other, codes)
+
+
+@pytest.mark.parametrize("N,K,block,bits,wdtype", [(40, 1024, 128, 4, "f32"), (136, 2048, 64, 8, "bf16"),
+                                                    (304, 4096, 256, 4, "f32"), (24, 96, 32, 8, "f32")])
+def test_fold_weights_after_bit_exact_and_linear(N, K, block, bits, wdtype):
+    rng = np.random.default_rng(N + K)
+    W = (rng.standard_normal((N, K)) * 0.02).astype(np.float32)
+    if wdtype == "bf16":
+        W = synth.f32_to_bf16_bits(W)
+    bias = (rng.standard_normal(N) * 0.02).astype(np.float32)
+    p = np.exp(rng.uniform(-1.5, 1.5, K)).astype(np.float32)
+    want_codes, want_scale, want_g = oracle.fold_weights_after(W, wdtype, p, block, bits)
+    h = fq.fold_weights_after(to_dev(W, wdtype), to_dev(p), to_dev(bias), block, bits)
+    assert h.fold_after and (h.N, h.K, h.block, h.bits) == (N, K, block, bits)
+    codes, scale, g, b = h.export()
+    assert np.array_equal(to_np(g).view(np.uint32), want_g.view(np.uint32))
+    assert np.array_equal(to_np(scale).view(np.uint32), want_scale.view(np.uint32))
+    assert np.array_equal(to_np(codes), want_codes)
+    # whole runtime path on that handle (prologue behind the rotation, GEMM, epilogue) against the oracle
+    M = 70
+    x = make_x(M, K, "bf16", seed=5)
+    ac, ad = oracle.quantize_act_after(x, "bf16", want_g, block, bits)
+    want_y = oracle.epilogue(oracle.gemm_i32(ac, want_codes, K, bits), ad, want_scale, bias, "f32")
+    y = fq.linear(to_dev(x, "bf16"), h, 1.0)
+    assert_close(to_np(y), want_y, "f32", "fold-after linear")
+    gc, gd = fq.quantize_act(to_dev(x, "bf16"), h, block, bits)          # picks the mode up from the handle
+    assert np.array_equal(to_np(gc), ac) and np.array_equal(to_np(gd).view(np.uint32), ad.view(np.uint32))
+    # an imported copy keeps the mode
+    h2 = fq.weights_import(codes, scale, g, b, K, block, bits, fold_after=True)
+    assert h2.fold_after
+    assert torch.equal(fq.linear(to_dev(x, "bf16"), h2, 1.0), y)
+
+
 # ------------------------------------------------------------ integer GEMM ----
 def random_codes(rng, rows, K, bits):
     q = 7 if bits == 4 else 127
