@@ -54,7 +54,8 @@ typedef enum {
 typedef enum { FQ_F32 = 0, FQ_BF16 = 1 } fq_dtype;
 
 /* Opaque folded-weight pack of one consumer projection (or several consumers of one
- * site concatenated along N).  Owns device memory; immutable after creation. */
+ * site concatenated along N).  Owns device memory; changed only by the offline calls
+ * fq_weights_set_multiplier / fq_weights_scale_outputs. */
 typedef struct fq_weights fq_weights;
 
 const char* fq_status_string(fq_status s);
@@ -101,6 +102,19 @@ fq_status fq_weights_export(const fq_weights* w, void* codes, float* w_scale, fl
 fq_status fq_weights_import(const void* codes, const float* w_scale, const float* mult_g,
                             const float* bias, int64_t N, int64_t K, int hadamard_block, int bits,
                             void* stream, fq_weights** out);
+
+/* ---- exact folds into neighbouring operators (section "Normalization gains", Eq. 4) --------------
+ * fq_weights_set_multiplier replaces the handle's runtime multiplier (offline; the stream is synchronised).
+ *   mult device float[K]: e.g. gamma_c * (1/s_c) * block^-1/2 for a projection that follows an RMS
+ *   normalisation whose learned gain gamma is absorbed here (the product D^i Gamma of Eq. 4: the input is
+ *   then the gain-free normalised activation), or NULL: the constant block^-1/2, for a site whose diagonal
+ *   1/s has been absorbed by its producer.
+ * fq_weights_scale_outputs multiplies output channels [first, first + count) of a handle by d_j > 0
+ *   (d device float[count]): s^W_j *= d_j and b_j *= d_j, one binary32 multiply each; codes unchanged.  This
+ *   is how a diagonal 1/s ahead of down_proj is absorbed into the linear up branch of a gated MLP (d = 1/s on
+ *   the up rows of the gate/up handle) without crossing the gate non-linearity. */
+fq_status fq_weights_set_multiplier(fq_weights* w, const float* mult, void* stream);
+fq_status fq_weights_scale_outputs(fq_weights* w, int64_t first, int64_t count, const float* d, void* stream);
 
 /* Import of a fold-after pack: mult_post device float[K] = 1/p (required). */
 fq_status fq_weights_import_after(const void* codes, const float* w_scale, const float* mult_post,

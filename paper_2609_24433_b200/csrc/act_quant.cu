@@ -306,6 +306,15 @@ __global__ void multipliers_kernel(const float* __restrict__ smooth, int K, floa
     if (mult_g) mult_g[i] = mg;
 }
 
+// s^W_j *= d_j, b_j *= d_j for a run of output channels (one binary32 multiply each).
+__global__ void scale_outputs_kernel(float* __restrict__ w_scale, float* __restrict__ bias,
+                                     const float* __restrict__ d, int64_t count) {
+    const int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= count) return;
+    w_scale[j] = __fmul_rn(w_scale[j], d[j]);
+    bias[j] = __fmul_rn(bias[j], d[j]);
+}
+
 template <typename XT>
 __global__ void col_absmax_kernel(const XT* __restrict__ x, int64_t M, int K, int64_t ldx, int accumulate,
                                   float* __restrict__ out, int rows_per_block) {
@@ -385,6 +394,12 @@ cudaError_t launch_transform_quantize(const void* x, fq_dtype xt, int64_t rows, 
 cudaError_t launch_multipliers(const float* smooth, int64_t K, float cnorm, float* mult_w, float* mult_g,
                                cudaStream_t stream) {
     multipliers_kernel<<<(unsigned)((K + 255) / 256), 256, 0, stream>>>(smooth, (int)K, cnorm, mult_w, mult_g);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_scale_outputs(float* w_scale, float* bias, const float* d, int64_t count, cudaStream_t stream) {
+    if (count == 0) return cudaSuccess;
+    scale_outputs_kernel<<<(unsigned)((count + 255) / 256), 256, 0, stream>>>(w_scale, bias, d, count);
     return cudaGetLastError();
 }
 

@@ -342,6 +342,30 @@ fq_status fq_weights_import_after(const void* codes, const float* w_scale, const
     return import_impl(codes, w_scale, mult_post, true, bias, N, K, hadamard_block, bits, stream, out);
 }
 
+fq_status fq_weights_set_multiplier(fq_weights* wp, const float* mult, void* stream) {
+    Weights* w = reinterpret_cast<Weights*>(wp);
+    if (!w) return FQ_ERR_INVALID_ARG;
+    if (mult && !aligned16(mult)) return FQ_ERR_ALIGNMENT;
+    if (w->fold_after && !mult) return FQ_ERR_INVALID_ARG;     // a fold-after handle keeps a post-rotation vector
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    bool ok;
+    if (mult)
+        ok = cudaMemcpyAsync(w->mult_g, mult, sizeof(float) * (size_t)w->K, cudaMemcpyDeviceToDevice, s) == cudaSuccess;
+    else
+        ok = launch_multipliers(nullptr, w->K, block_norm(w->block), nullptr, w->mult_g, s) == cudaSuccess;
+    ok = ok && cudaStreamSynchronize(s) == cudaSuccess;        // the handle is complete when the call returns
+    return ok ? FQ_OK : FQ_ERR_CUDA;
+}
+
+fq_status fq_weights_scale_outputs(fq_weights* wp, int64_t first, int64_t count, const float* d, void* stream) {
+    Weights* w = reinterpret_cast<Weights*>(wp);
+    if (!w || !d || first < 0 || count < 0 || first + count > w->N) return FQ_ERR_INVALID_ARG;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    bool ok = launch_scale_outputs(w->w_scale + first, w->bias + first, d, count, s) == cudaSuccess;
+    ok = ok && cudaStreamSynchronize(s) == cudaSuccess;
+    return ok ? FQ_OK : FQ_ERR_CUDA;
+}
+
 fq_status fq_col_absmax(const void* x, fq_dtype xt, int64_t M, int64_t K, int64_t ldx, int accumulate, float* out,
                         void* stream) {
     if (M < 0 || K <= 0 || !out || (M > 0 && (!x || ldx < K))) return FQ_ERR_INVALID_ARG;

@@ -74,6 +74,9 @@ cudaError_t launch_transform_quantize(const void* x, fq_dtype xt, int64_t rows, 
 cudaError_t launch_multipliers(const float* smooth, int64_t K, float cnorm, float* mult_w, float* mult_g,
                                cudaStream_t stream);
 
+// w_scale[j] *= d[j], bias[j] *= d[j] for j < count (pointers already offset to the first channel).
+cudaError_t launch_scale_outputs(float* w_scale, float* bias, const float* d, int64_t count, cudaStream_t stream);
+
 cudaError_t launch_col_absmax(const void* x, fq_dtype xt, int64_t M, int64_t K, int64_t ldx, int accumulate,
                               float* out, cudaStream_t stream);
 cudaError_t launch_smooth_scale(const float* a, const float* w, int64_t K, double alpha, float* s,

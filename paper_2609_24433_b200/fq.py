@@ -25,6 +25,7 @@ EXPORTS = [
     "fq_gemm_w4a4", "fq_gemm_w8a8", "fq_linear_w4a4", "fq_linear_w8a8", "fq_workspace_bytes",
     "fq_gemm_acc_i32", "fq_gemm_simt", "fq_device_status", "fq_profile_mark", "fq_linear_w4a4_static",
     "fq_fold_weights_after", "fq_weights_fold_after", "fq_weights_import_after", "fq_quantize_act_after",
+    "fq_weights_set_multiplier", "fq_weights_scale_outputs",
 ]
 
 _lib = None
@@ -122,6 +123,15 @@ class Weights:
         _check(lib().fq_weights_export(self.handle, _ptr(codes), _ptr(ws), _ptr(g), _ptr(b), _stream()),
                "fq_weights_export")
         return codes, ws, g, b
+
+    def set_multiplier(self, mult: Optional[torch.Tensor]):
+        """Replace the runtime multiplier (None: the constant block^-1/2); offline."""
+        _check(lib().fq_weights_set_multiplier(self.handle, _ptr(mult), _stream()), "fq_weights_set_multiplier")
+
+    def scale_outputs(self, first: int, d: torch.Tensor):
+        """s^W_j *= d_j, b_j *= d_j for output channels first .. first + len(d); offline."""
+        _check(lib().fq_weights_scale_outputs(self.handle, ctypes.c_int64(first), ctypes.c_int64(d.numel()),
+                                              _ptr(d), _stream()), "fq_weights_scale_outputs")
 
     def destroy(self):
         if self._h is not None:

@@ -224,6 +224,43 @@ def test_fold_weights_after_bit_exact_and_linear(N, K, block, bits, wdtype):
     assert torch.equal(fq.linear(to_dev(x, "bf16"), h2, 1.0), y)
 
 
+def test_exact_folds_set_multiplier_and_scale_outputs():
+    """Eq. 4 helpers: a replaced runtime multiplier (RMS gain absorbed: gamma * g) and scaled output channels
+    (1/s absorbed by the up rows of a gate/up handle) against the oracle with the same vectors."""
+    rng = np.random.default_rng(31)
+    M, K, N, block = 120, 1024, 256, 64
+    x = make_x(M, K, "bf16", seed=9)
+    W = (rng.standard_normal((N, K)) * 0.02).astype(np.float32)
+    bias = (rng.standard_normal(N) * 0.02).astype(np.float32)
+    s = np.exp(rng.uniform(-1, 1, K)).astype(np.float32)
+    gamma = (rng.random(K) + 0.5).astype(np.float32)
+    wc, wsc, g = oracle.fold_weights(W, "f32", s, block, 4)
+    h = fq.fold_weights(to_dev(W), to_dev(s), to_dev(bias), block, 4)
+    # (1) gain absorbed by the multiplier
+    g2 = gamma * g
+    h.set_multiplier(to_dev(g2))
+    want = oracle.linear(x, "bf16", g2, block, 4, 1.0, wc, wsc, bias, "f32")
+    y = fq.linear(to_dev(x, "bf16"), h, 1.0)
+    assert_close(to_np(y), want[0], "f32", "replaced multiplier")
+    codes, delta = fq.quantize_act(to_dev(x, "bf16"), h, block, 4)
+    assert np.array_equal(to_np(codes), want[1]) and np.array_equal(to_np(delta).view(np.uint32), want[2].view(np.uint32))
+    # (2) constant multiplier (diagonal absorbed upstream)
+    h.set_multiplier(None)
+    want = oracle.linear(x, "bf16", None, block, 4, 1.0, wc, wsc, bias, "f32")
+    assert_close(to_np(fq.linear(to_dev(x, "bf16"), h, 1.0)), want[0], "f32", "constant multiplier")
+    # (3) output channels 64..191 scaled by d
+    d = np.exp(rng.uniform(-1, 1, 128)).astype(np.float32)
+    h.scale_outputs(64, to_dev(d))
+    _, sc, _, b = h.export()
+    wsc2, bias2 = wsc.copy(), bias.copy()
+    wsc2[64:192] *= d
+    bias2[64:192] *= d
+    assert np.array_equal(to_np(sc).view(np.uint32), wsc2.view(np.uint32))
+    assert np.array_equal(to_np(b).view(np.uint32), bias2.view(np.uint32))
+    want = oracle.linear(x, "bf16", None, block, 4, 1.0, wc, wsc2, bias2, "f32")
+    assert_close(to_np(fq.linear(to_dev(x, "bf16"), h, 1.0)), want[0], "f32", "scaled outputs")
+
+
 # ------------------------------------------------------------ integer GEMM ----
 def random_codes(rng, rows, K, bits):
     q = 7 if bits == 4 else 127

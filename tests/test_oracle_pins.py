@@ -457,3 +457,43 @@ def test_fold_after_end_to_end_accuracy_is_that_of_the_quantizer():
         y = oracle.epilogue(oracle.gemm_i32(ac, wc, K, bits), ad, ws, b)
         errs[bits] = np.linalg.norm(y - y_ref) / np.linalg.norm(y_ref)
     assert errs[8] < 0.02 and errs[4] < 0.25 and errs[8] < errs[4] / 5
+
+
+# ------------------------------------------ exact folds into neighbouring operators (Eq. 4) ----
+def test_rms_gain_is_absorbed_by_the_runtime_multiplier():
+    """x = Gamma h: R S^-1 (Gamma h) with the multiplier (gamma/s) beta^-1/2 on the gain-free input equals
+    the same transform of x with (1/s) beta^-1/2, up to the single rounding of gamma * h."""
+    rng = np.random.default_rng(21)
+    K, beta = 512, 64
+    h = rng.standard_normal((7, K)).astype(np.float32)
+    gamma = (rng.random(K) + 0.5).astype(np.float32)
+    s = np.exp(rng.uniform(-1, 1, K)).astype(np.float32)
+    g = oracle.multiplier(s, K, beta, False)
+    _, _, z_plain = oracle.quantize_act(gamma * h, "f32", g, beta, 8, return_z=True)
+    _, _, z_fold = oracle.quantize_act(h, "f32", gamma * g, beta, 8, return_z=True)
+    assert np.allclose(z_plain, z_fold, rtol=1e-5, atol=1e-6)
+
+
+def test_input_diagonal_is_absorbed_by_the_linear_up_branch():
+    """x_down = act(gate) * up.  Scaling the up branch's output channel c by 1/s_c (its s^W and bias) makes the
+    producer emit x/s, so down_proj's runtime multiplier becomes the constant beta^-1/2; Eq. 8 of down_proj on
+    the absorbed pair equals Eq. 8 on the plain pair up to rounding of the intermediate activation."""
+    rng = np.random.default_rng(22)
+    M, D, I, beta = 24, 128, 256, 64
+    x = rng.standard_normal((M, D)).astype(np.float32)
+    Wg, Wu = (rng.standard_normal((2, I, D)) * 0.1).astype(np.float32)
+    bu = (rng.standard_normal(I) * 0.1).astype(np.float32)
+    Wd = (rng.standard_normal((16, I)) * 0.1).astype(np.float32)
+    s = np.exp(rng.uniform(-1, 1, I)).astype(np.float32)
+    # up branch through the quantized path (8 bits), gate kept in floating point for the test
+    uc, us, ug = oracle.fold_weights(Wu, "f32", None, beta, 8)
+    ac, ad = oracle.quantize_act(x, "f32", ug, beta, 8)
+    acc = oracle.gemm_i32(ac, uc, D, 8)
+    up = oracle.epilogue(acc, ad, us, bu)
+    up_abs = oracle.epilogue(acc, ad, us * (np.float32(1) / s), bu * (np.float32(1) / s))   # absorbed: same codes
+    gate = np.tanh(x.astype(np.float64) @ Wg.astype(np.float64).T).astype(np.float32)
+    dc, ds, dg = oracle.fold_weights(Wd, "f32", s, beta, 8)
+    y_plain = oracle.linear(gate * up, "f32", dg, beta, 8, 1.0, dc, ds, None)[0]
+    y_abs = oracle.linear(gate * up_abs, "f32", None, beta, 8, 1.0, dc, ds, None)[0]
+    assert np.allclose(up_abs, up / s, rtol=1e-5, atol=1e-6)
+    assert np.linalg.norm(y_abs - y_plain) < 2e-2 * np.linalg.norm(y_plain)
