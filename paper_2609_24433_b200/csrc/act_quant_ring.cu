@@ -103,7 +103,7 @@ struct RingParams {
     uint32_t* watchdog;
 };
 
-template <typename XT, int FMT, bool CLAMP, int E, int BLOCK>
+template <typename XT, int FMT, bool CLAMP, int E, int BLOCK, bool AFTER>
 __global__ void __launch_bounds__(kThreads, 1)
 transform_quantize_ring_kernel(const __grid_constant__ CUtensorMap map_x, const RingParams p) {
     constexpr int H = E / 2;                       // channels per half: v[i] = (channel i, channel i + H)
@@ -211,7 +211,7 @@ transform_quantize_ring_kernel(const __grid_constant__ CUtensorMap map_x, const 
                     v[4 * i + 3] = make_float2(lo.w, hi.w);
                 }
             }
-            if (p.mult != nullptr && !p.mult_after) {
+            if (!AFTER && p.mult != nullptr) {
 #pragma unroll
                 for (int i = 0; i < H / 4; ++i) {
                     const float4 lo = lds128f_ordered(piece(g0, g1, i));
@@ -275,7 +275,7 @@ transform_quantize_ring_kernel(const __grid_constant__ CUtensorMap map_x, const 
         }
 
         // fold-after sites: the diagonal sits behind the rotation (z = D^o R x)
-        if (p.mult_after && col_ok) {
+        if (AFTER && col_ok) {
 #pragma unroll
             for (int i = 0; i < H / 4; ++i) {
                 const float4 lo = lds128f_ordered(piece(g0, g1, i));
@@ -377,8 +377,14 @@ cudaError_t launch_ring(const CUtensorMap& map, const RingParams& p, int grid, s
         if (e != cudaSuccess) return e;
         return launch_pdl(kern, (unsigned)grid, (unsigned)kThreads, smem, stream, 1u, map, p);
     };
-    if (p.clip_ratio < 1.0f) return go(transform_quantize_ring_kernel<XT, FMT, true, E, BLOCK>);
-    return go(transform_quantize_ring_kernel<XT, FMT, false, E, BLOCK>);
+    // (the fold-after variant is its own instantiation: as a run-time branch it cost the default
+    // path registers, and spills, in the 64-channels-per-thread kernels)
+    if (p.mult_after) {
+        if (p.clip_ratio < 1.0f) return go(transform_quantize_ring_kernel<XT, FMT, true, E, BLOCK, true>);
+        return go(transform_quantize_ring_kernel<XT, FMT, false, E, BLOCK, true>);
+    }
+    if (p.clip_ratio < 1.0f) return go(transform_quantize_ring_kernel<XT, FMT, true, E, BLOCK, false>);
+    return go(transform_quantize_ring_kernel<XT, FMT, false, E, BLOCK, false>);
 }
 
 template <typename XT, int FMT, int E>
@@ -416,7 +422,8 @@ cudaError_t launch_transform_quantize_ring(const void* x, fq_dtype xt, int64_t r
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     if (rows < 2 * (int64_t)sms) return cudaErrorNotSupported;     // short batches: latency-bound, register kernel
 
-    const int e = (K >= 2048 && K % 64 == 0) ? 64 : 32;            // channels per thread
+    // channels per thread (the fold-after variant with shuffle stages does not fit 64 without spills)
+    const int e = (K >= 2048 && K % 64 == 0 && !(mult != nullptr && mult_after_rotation && block >= 128)) ? 64 : 32;
     int gw = 1;
     while ((int64_t)gw * 32 * e < K) gw <<= 1;
     if (gw > kThreads / 32) return cudaErrorNotSupported;
