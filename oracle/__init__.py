@@ -238,3 +238,18 @@ def linear(x: np.ndarray, xdtype: str, g, beta: int, bits: int, clip_ratio: floa
                               _p(y), ctypes.c_int(_dt(out_dtype)), ctypes.c_int64(N), _p(codes),
                               _p(delta), _p(acc)), "linear")
     return y, codes, delta, acc
+
+
+def linear_wonly(x: np.ndarray, xdtype: str, w_codes: np.ndarray, w_scale, bias, bits: int = 4,
+                 out_dtype: str = "f32") -> np.ndarray:
+    """Weight-only projection with floating-point activations: y = s^W (qW x) + b in binary64."""
+    x = _mat(x, xdtype)
+    M, K = x.shape
+    w = np.ascontiguousarray(w_codes).view(np.uint8)
+    N = w.shape[0]
+    y = np.zeros((M, N), dtype=np.float32 if _dt(out_dtype) == F32 else np.uint16)
+    _check(_load().fqo_linear_wonly(_p(x), ctypes.c_int(_dt(xdtype)), ctypes.c_int64(M), ctypes.c_int64(K),
+                                    ctypes.c_int64(K), _p(w), _p(_f32(w_scale)), _p(_f32(bias)),
+                                    ctypes.c_int64(N), ctypes.c_int(bits), _p(y), ctypes.c_int(_dt(out_dtype)),
+                                    ctypes.c_int64(N)), "linear_wonly")
+    return y

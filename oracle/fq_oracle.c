@@ -65,8 +65,10 @@ static float load_elem(const void* base, int dtype, int64_t idx) {
     return ((const float*)base)[idx];
 }
 
+/* beta = 1 is the identity rotation (R = I: sites that are only scaled, and the identity transforms at
+ * graph and engine boundaries); the butterfly loops below then have no stage and beta^(-1/2) = 1. */
 static int valid_block(int beta, int64_t K) {
-    if (beta < 2 || beta > 256 || (beta & (beta - 1)) != 0) return 0;
+    if (beta < 1 || beta > 256 || (beta & (beta - 1)) != 0) return 0;
     return K > 0 && K % beta == 0;
 }
 
@@ -363,6 +365,34 @@ int fqo_epilogue(const int32_t* acc, const float* delta, const float* w_scale, c
         for (int64_t j = 0; j < N; ++j) {
             double v = (double)w_scale[j] * (double)delta[t] * (double)acc[t * N + j] +
                        (bias ? (double)bias[j] : 0.0);
+            float f = (float)v;
+            if (ydtype == FQO_BF16)
+                ((uint16_t*)y)[t * ldy + j] = f32_to_bf16(f);
+            else
+                ((float*)y)[t * ldy + j] = f;
+        }
+    }
+    return 0;
+}
+
+/* Weight-only low-bit projection with floating-point activations (section "Problem statement": in
+ * the W4A4 engines the adaptive layer-normalisation modulation keeps its activations in floating
+ * point and only its weights are 4-bit).  With the weight reconstruction W^_jc = s^W_j qW_jc of Eq. 8:
+ *   y[t][j] = s^W_j * sum_c qW[j][c] * x[t][c] + b_j,
+ * products and sum in binary64 in channel order, rounded once to the output type. */
+int fqo_linear_wonly(const void* x, int xdtype, int64_t M, int64_t K, int64_t ldx, const uint8_t* w_codes,
+                     const float* w_scale, const float* bias, int64_t N, int bits, void* y, int ydtype,
+                     int64_t ldy) {
+    if ((bits != 4 && bits != 8) || (K & 1) || ldx < K || ldy < N) return 1;
+    int64_t pitch = K * bits / 8;
+#pragma omp parallel for schedule(static)
+    for (int64_t t = 0; t < M; ++t) {
+        for (int64_t j = 0; j < N; ++j) {
+            const uint8_t* wrow = w_codes + j * pitch;
+            double s = 0.0;
+            for (int64_t c = 0; c < K; ++c)
+                s += (double)code_at(wrow, c, bits) * (double)load_elem(x, xdtype, t * ldx + c);
+            double v = (double)w_scale[j] * s + (bias ? (double)bias[j] : 0.0);
             float f = (float)v;
             if (ydtype == FQO_BF16)
                 ((uint16_t*)y)[t * ldy + j] = f32_to_bf16(f);

@@ -497,3 +497,86 @@ def test_input_diagonal_is_absorbed_by_the_linear_up_branch():
     y_abs = oracle.linear(gate * up_abs, "f32", None, beta, 8, 1.0, dc, ds, None)[0]
     assert np.allclose(up_abs, up / s, rtol=1e-5, atol=1e-6)
     assert np.linalg.norm(y_abs - y_plain) < 2e-2 * np.linalg.norm(y_plain)
+
+
+# ---------------------------------------------- identity rotation (beta = 1) ----
+def test_identity_rotation_hand_case():
+    """beta = 1 is R = I: the fold rounds the scaled weights themselves and the prologue quantizes
+    x (.) g.  Hand-worked: W row (7, -3.5, 1.75, 0) has s^W = 1, codes (7, -4, 2, 0) (ties to even);
+    the token (0.5, -1.5, 3.5, 0.25) at 4 bits has delta = 0.5, codes (1, -3, 7, 0) (0.5 is a tie -> 0)."""
+    W = np.zeros((8, 32), np.float32)
+    W[0, :4] = [7.0, -3.5, 1.75, 0.0]
+    wc, ws, g = oracle.fold_weights(W, "f32", None, 1, 4)
+    assert ws[0] == np.float32(1.0) and np.all(g == np.float32(1.0))
+    assert np.array_equal(oracle.unpack(wc, 32, 4)[0, :4], [7, -4, 2, 0])
+    x = np.zeros((1, 32), np.float32)
+    x[0, :4] = [0.5, -1.5, 3.5, 0.25]
+    codes, delta, z = oracle.quantize_act(x, "f32", None, 1, 4, 1.0, return_z=True)
+    assert np.array_equal(z, x)                            # no rotation, unit multiplier
+    assert delta[0] == np.float32(0.5)
+    assert np.array_equal(oracle.unpack(codes, 32, 4)[0, :4], [1, -3, 7, 0])
+
+
+def test_identity_rotation_with_smoothing_keeps_the_projection():
+    """W~ z = (W S)(S^-1 x) = W x before rounding, with no rotation in between."""
+    rng = np.random.default_rng(5)
+    W = rng.standard_normal((8, 64)).astype(np.float32)
+    x = rng.standard_normal((3, 64)).astype(np.float32)
+    s = np.exp2(rng.integers(-2, 3, size=64)).astype(np.float32)      # powers of two: exact scaling
+    _, _, g, wt = oracle.fold_weights(W, "f32", s, 1, 8, return_wt=True)
+    _, _, z = oracle.quantize_act(x, "f32", g, 1, 8, 1.0, return_z=True)
+    assert np.array_equal(wt, W * s) and np.array_equal(z, x / s)
+    assert np.allclose(z.astype(np.float64) @ wt.astype(np.float64).T, x.astype(np.float64) @ W.astype(np.float64).T,
+                       rtol=1e-12, atol=1e-12)
+
+
+# ------------------------------------- weight-only projection, float activations ----
+def test_weight_only_linear_hand_case():
+    """y = s^W (q . x) + b: q = (3, -8, 7, 1), x = (0.5, 0.25, -1, 2), s^W = 0.5, b = 1
+    -> q.x = 1.5 - 2 - 7 + 2 = -5.5, y = -1.75."""
+    K = 32
+    q = np.zeros((8, K), np.int32)
+    q[0, :4] = [3, -8, 7, 1]
+    x = np.zeros((2, K), np.float32)
+    x[0, :4] = [0.5, 0.25, -1.0, 2.0]
+    ws = np.full(8, 0.5, np.float32)
+    b = np.full(8, 1.0, np.float32)
+    y = oracle.linear_wonly(x, "f32", oracle.pack(q, 4), ws, b)
+    assert y[0, 0] == np.float32(-1.75)
+    assert np.all(y[1] == 1.0) and np.all(y[0, 1:] == 1.0)     # zero token / zero rows give the bias
+
+
+@pytest.mark.parametrize("bits", [4, 8])
+def test_weight_only_linear_on_integer_activations_equals_eq8(bits):
+    """With activations that are themselves integer codes, the weight-only product is Eq. 8 with
+    delta = 1: the brute-force-pinned integer product and epilogue give the same numbers."""
+    qm = 7 if bits == 4 else 127
+    rng = np.random.default_rng(10 + bits)
+    M, N, K = 5, 16, 96
+    a = rng.integers(-qm, qm + 1, size=(M, K)).astype(np.int32)
+    w = rng.integers(-qm, qm + 1, size=(N, K)).astype(np.int32)
+    ws = rng.uniform(0.01, 0.1, N).astype(np.float32)
+    b = rng.standard_normal(N).astype(np.float32)
+    wc = oracle.pack(w, bits)
+    want = oracle.epilogue(oracle.gemm_i32(oracle.pack(a, bits), wc, K, bits), np.ones(M, np.float32), ws, b)
+    got = oracle.linear_wonly(a.astype(np.float32), "f32", wc, ws, b, bits)
+    assert np.array_equal(got, want)
+    assert got.shape == (M, N)
+
+
+def test_weight_only_linear_one_hot_bf16_and_linearity():
+    rng = np.random.default_rng(12)
+    N, K = 16, 64
+    w = rng.integers(-8, 8, size=(N, K)).astype(np.int32)          # the full two's-complement nibble range
+    ws = np.exp2(rng.integers(-6, -2, size=N)).astype(np.float32)
+    wc = oracle.pack(w, 4)
+    eye = np.eye(K, dtype=np.float32)
+    y = oracle.linear_wonly(synth.f32_to_bf16_bits(eye), "bf16", wc, ws, None)
+    assert np.array_equal(y, (w.T * ws).astype(np.float32))          # one-hot tokens read the dequantised columns
+    x1 = rng.integers(-64, 64, size=(4, K)).astype(np.float32) / 16  # dyadic: sums are exact
+    x2 = rng.integers(-64, 64, size=(4, K)).astype(np.float32) / 16
+    y12 = oracle.linear_wonly(x1 + x2, "f32", wc, ws, None)
+    assert np.array_equal(y12, oracle.linear_wonly(x1, "f32", wc, ws, None) + oracle.linear_wonly(x2, "f32", wc, ws, None))
+    # bf16 output: one rounding of the binary64 result
+    yb = oracle.linear_wonly(x1, "f32", wc, ws, None, out_dtype="bf16")
+    assert np.array_equal(yb, synth.f32_to_bf16_bits(oracle.linear_wonly(x1, "f32", wc, ws, None)))
