@@ -66,7 +66,9 @@ const char* fq_status_string(fq_status s);
  * bias   device float[N] or NULL (= 0); copied into the handle unchanged (output transform is I).
  * Creates *out holding: packed codes [N, K*bits/8], s^W[N], bias[N] and the runtime multiplier
  * g[K] = (1/s_c) * block^-1/2.  Allocates with cudaMalloc (this call only); work is async on stream.
- * Row j of W~ is FWHT(s (.) w_j * block^-1/2); s^W_j = max|W~_j| / q; no weight clipping. */
+ * Row j of W~ is FWHT(s (.) w_j * block^-1/2); s^W_j = max|W~_j| / q; no weight clipping.
+ * hadamard_block is a power of two in [1, 256] dividing K; 1 is the identity rotation (R = I: a site that is
+ * only scaled, or -- with smooth = NULL -- plain RTN of W, the identity transform of a graph boundary). */
 fq_status fq_fold_weights(const void* W, fq_dtype wt, int64_t N, int64_t K, int64_t ldw,
                           const float* smooth, const float* bias, int hadamard_block, int bits,
                           void* stream, fq_weights** out);
@@ -165,6 +167,19 @@ fq_status fq_linear_w4a4(const void* x, fq_dtype xt, int64_t M, int64_t ldx, con
 fq_status fq_linear_w8a8(const void* x, fq_dtype xt, int64_t M, int64_t ldx, const fq_weights* W,
                          float clip_ratio, void* y, fq_dtype yt, int64_t ldy, void* workspace,
                          size_t ws_bytes, void* stream);
+
+/* ---- weight-only 4-bit projection with floating-point activations ------------------------------
+ * (Section "Problem statement": in the W4A4 engines the adaptive layer-normalisation modulation keeps
+ * floating-point activations and only its weights are INT4.)  With the reconstruction W^_jc = s^W_j qW_jc
+ * of Eq. 8:   y[t][j] = s^W_j * sum_c qW[j][c] * x[t][c] + b_j.
+ * W is any 4-bit handle; its codes multiply x as given, so a handle meant for this call is made with the
+ * identity transform (fq_fold_weights with hadamard_block = 1 and smooth = NULL: plain per-output-channel
+ * RTN of W), or x must already be in the handle's transformed coordinates.  No quantization of x, no
+ * workspace.  x device [M, K] of dtype xt (FQ_F32 or FQ_BF16); binary32 accumulation.  These projections see
+ * one conditioning vector per sample: the kernel streams the weights once per four tokens and is meant for
+ * short batches (any M is accepted).  Errors as for fq_linear_w4a4; FQ_ERR_UNSUPPORTED for 8-bit handles. */
+fq_status fq_linear_w4a16(const void* x, fq_dtype xt, int64_t M, int64_t ldx, const fq_weights* W, void* y,
+                          fq_dtype yt, int64_t ldy, void* stream);
 
 /* ---- fused W4A4 linear without a workspace, for callers that cannot allocate ------------------
  * (The paper has no counterpart: this is a deployment convenience of this library.)

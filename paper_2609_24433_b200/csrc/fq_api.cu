@@ -16,7 +16,8 @@ constexpr int64_t kMaxPrologueK = 32768; // one token must fit the registers of 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 bool valid_block(int block, int64_t K) {
-    return block >= 2 && block <= 256 && (block & (block - 1)) == 0 && K > 0 && K % block == 0;
+    // block 1 is the identity rotation (R = I: scale-only sites, weight-only handles)
+    return block >= 1 && block <= 256 && (block & (block - 1)) == 0 && K > 0 && K % block == 0;
 }
 
 float block_norm(int block) { return (float)(1.0 / sqrt((double)block)); }
@@ -448,6 +449,23 @@ fq_status fq_linear_w4a4(const void* x, fq_dtype xt, int64_t M, int64_t ldx, con
 fq_status fq_linear_w8a8(const void* x, fq_dtype xt, int64_t M, int64_t ldx, const fq_weights* W, float clip_ratio,
                          void* y, fq_dtype yt, int64_t ldy, void* workspace, size_t ws_bytes, void* stream) {
     return linear_impl(x, xt, M, ldx, W, 8, clip_ratio, y, yt, ldy, workspace, ws_bytes, stream);
+}
+
+fq_status fq_linear_w4a16(const void* x, fq_dtype xt, int64_t M, int64_t ldx, const fq_weights* Wp, void* y,
+                          fq_dtype yt, int64_t ldy, void* stream) {
+    const Weights* W = reinterpret_cast<const Weights*>(Wp);
+    if (!W || M < 0) return FQ_ERR_INVALID_ARG;
+    if (W->bits != 4) return FQ_ERR_UNSUPPORTED;
+    if (xt != FQ_F32 && xt != FQ_BF16) return FQ_ERR_INVALID_ARG;
+    if (M == 0 || W->N == 0) return FQ_OK;
+    if (!x || ldx < W->K) return FQ_ERR_INVALID_ARG;
+    if (!aligned16(x) || ldx % 8 != 0) return FQ_ERR_ALIGNMENT;
+    fq_status st = check_y(y, yt, ldy, W->N);
+    if (st != FQ_OK) return st;
+    st = check_arch();
+    if (st != FQ_OK) return st;
+    return launch_linear_wonly4(x, xt, M, ldx, *W, y, yt, ldy, static_cast<cudaStream_t>(stream)) == cudaSuccess
+               ? FQ_OK : FQ_ERR_CUDA;
 }
 
 size_t fq_workspace_bytes(int64_t M, int64_t K, int64_t N, int bits) {

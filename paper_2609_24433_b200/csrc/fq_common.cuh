@@ -98,6 +98,10 @@ struct GemmOut {
 cudaError_t launch_gemm_simt(const int8_t* a8, int64_t M, const Weights& W, int acc_shift, const GemmOut& out,
                              cudaStream_t stream);
 
+// Weight-only 4-bit projection with float activations (CUDA cores; short batches): y = s^W (qW x) + b.
+cudaError_t launch_linear_wonly4(const void* x, fq_dtype xt, int64_t M, int64_t ldx, const Weights& W, void* y,
+                                 fq_dtype yt, int64_t ldy, cudaStream_t stream);
+
 // tcgen05 integer GEMM; a8 = int8 activations [M, K] (pitch K), 16-byte aligned.  `scratch` (device,
 // 256-byte aligned, may be null) holds int32 partial tiles when the launch splits K over a cluster;
 // gemm_scratch_bytes() is what the split the planner would pick for this shape needs.

@@ -79,7 +79,7 @@ constexpr int kUnpackSets = 2;          // sets of four unpack warps, one TMEM l
 constexpr int kThreadsW4 = 32 * (2 + kEpiWarps) + kUnpackSets * 128 + 32;
 constexpr int kMaxStagesW = 8;
 constexpr int kColsW = kBlockK / 4;     // TMEM columns of one unpacked k-block (128 int8 per lane)
-constexpr int kMaxStages = 8;
+constexpr int kMaxStages = 16;
 constexpr int kMaxStagesP = 16;
 constexpr int kMaxSplit = 16;          // K slices per tile, at most
 constexpr int kMaxSplitTiles = 1024;   // tiles of a launch that splits K (one counter each in the weight handle)

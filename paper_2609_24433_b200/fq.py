@@ -25,7 +25,7 @@ EXPORTS = [
     "fq_gemm_w4a4", "fq_gemm_w8a8", "fq_linear_w4a4", "fq_linear_w8a8", "fq_workspace_bytes",
     "fq_gemm_acc_i32", "fq_gemm_simt", "fq_device_status", "fq_profile_mark", "fq_linear_w4a4_static",
     "fq_fold_weights_after", "fq_weights_fold_after", "fq_weights_import_after", "fq_quantize_act_after",
-    "fq_weights_set_multiplier", "fq_weights_scale_outputs",
+    "fq_weights_set_multiplier", "fq_weights_scale_outputs", "fq_linear_w4a16",
 ]
 
 _lib = None
@@ -289,6 +289,17 @@ def linear_w4a4_static(x, W: Weights, clip_ratio: float = 1.0, out_dtype=torch.f
     _check(lib().fq_linear_w4a4_static(_ptr(x), _dt(x), ctypes.c_int64(M), ctypes.c_int64(x.stride(0)), W.handle,
                                        ctypes.c_float(clip_ratio), _ptr(y), _out_dt(y.dtype),
                                        ctypes.c_int64(y.stride(0)), _stream()), "fq_linear_w4a4_static")
+    return y
+
+
+def linear_w4a16(x, W: Weights, out_dtype=torch.float32, y=None):
+    """Weight-only 4-bit projection of float activations: y = s^W (qW x) + b (no quantization of x)."""
+    x = _rowmajor(x)
+    M = x.shape[0]
+    if y is None:
+        y = torch.empty((M, W.N), dtype=out_dtype, device=x.device)
+    _check(lib().fq_linear_w4a16(_ptr(x), _dt(x), ctypes.c_int64(M), ctypes.c_int64(x.stride(0)), W.handle,
+                                 _ptr(y), _out_dt(y.dtype), ctypes.c_int64(y.stride(0)), _stream()), "fq_linear_w4a16")
     return y
 
 

@@ -7,7 +7,7 @@ import pytest
 import torch
 
 import oracle
-from helpers import assert_close, concat_consumers, oracle_smooth, to_dev, to_np
+from helpers import as_f64, assert_close, concat_consumers, oracle_smooth, to_dev, to_np
 from paper_2609_24433_b200 import fq, synth
 
 pytestmark = pytest.mark.gpu
@@ -53,6 +53,11 @@ ACT_CASES = [
     (333, 3072, 128, 4, "bf16", True, 1.0),
     (1000, 16384, 256, 4, "bf16", True, 1.0),
     (700, 8192, 32, 8, "bf16", False, 0.6),
+    # identity rotation (block 1): scale-only sites
+    (64, 1024, 1, 4, "f32", True, 1.0),
+    (816, 2048, 1, 8, "bf16", False, 1.0),
+    (300, 8192, 1, 4, "bf16", True, 0.8),
+    (2500, 1024, 1, 4, "bf16", False, 1.0),
 ]
 
 
@@ -137,6 +142,8 @@ FOLD_CASES = [
     (24, 16384, 256, 8, "bf16", False),
     (16, 16384, 256, 4, "f32", True),
     (40, 96, 32, 8, "f32", True),
+    (264, 1536, 1, 4, "bf16", False),       # identity transform: plain RTN of W
+    (64, 2048, 1, 8, "f32", True),
 ]
 
 
@@ -539,6 +546,82 @@ def test_calibration_helpers_match_oracle():
                                                 oracle.col_absmax(2 * data.W["proj"][:100])))
     s = fq.smooth_scale(a, w, 0.5)
     assert np.allclose(to_np(s), oracle.smooth_scale(to_np(a), to_np(w), 0.5), rtol=1e-6)
+
+
+# ------------------------------- weight-only 4-bit projection, float activations ----
+W4A16_CASES = [
+    # M, N, K, xdtype, ydtype          (adaptive layer-norm modulation: one conditioning vector per sample)
+    (1, 3072, 1536, "bf16", "bf16"),
+    (1, 3072, 1536, "f32", "f32"),
+    (2, 512, 2048, "bf16", "f32"),
+    (4, 3072, 1536, "bf16", "bf16"),
+    (7, 264, 96, "f32", "f32"),
+    (16, 1024, 1024, "bf16", "bf16"),
+    (50, 4096, 1024, "bf16", "f32"),
+    (3, 8, 32, "f32", "bf16"),
+    (5, 6144, 4096, "f32", "f32"),
+    (300, 72, 544, "bf16", "f32"),      # more token groups than the grid's second dimension
+]
+
+
+@pytest.mark.parametrize("M,N,K,xdtype,ydtype", W4A16_CASES)
+def test_linear_w4a16_matches_oracle(M, N, K, xdtype, ydtype):
+    rng = np.random.default_rng(M + 3 * N + 7 * K)
+    W = synth.draw_weights(rng, N, K)
+    bias = rng.standard_normal(N).astype(np.float32)
+    x = synth.as_dtype(rng.standard_normal((M, K)).astype(np.float32), xdtype)
+    wc, ws, _ = oracle.fold_weights(W, "f32", None, 1, 4)           # identity transform: RTN of W itself
+    h = fq.fold_weights(to_dev(W), None, to_dev(bias), 1, 4)
+    hc, hs, _, _ = h.export()
+    assert np.array_equal(to_np(hc), wc) and np.array_equal(to_np(hs).view(np.uint32), ws.view(np.uint32))
+    want = oracle.linear_wonly(x, xdtype, wc, ws, bias, 4, ydtype)
+    ydt = torch.float32 if ydtype == "f32" else torch.bfloat16
+    y = fq.linear_w4a16(to_dev(x, xdtype), h, ydt)
+    assert_close(to_np(y), want, ydtype, f"w4a16 {M}x{N}x{K}")
+    # it does what it is for: the 4-bit weights reproduce the float projection to RTN accuracy
+    ref = synth.to_f32(x, xdtype).astype(np.float64) @ W.astype(np.float64).T + bias
+    assert np.linalg.norm(as_f64(to_np(y)) - ref) / np.linalg.norm(ref) < 0.2
+
+
+def test_linear_w4a16_exact_on_integer_activations_and_edges():
+    """Integer activations make every binary32 partial sum exact, whatever the order of the additions:
+    the kernel must then equal the oracle bit for bit (any indexing slip shows).  Plus the edges: zero
+    tokens give the bias, rows beyond M and columns beyond N of a wider output stay untouched."""
+    rng = np.random.default_rng(77)
+    M, N, K = 6, 136, 1120
+    q = rng.integers(-8, 8, size=(N, K)).astype(np.int32)
+    wc = oracle.pack(q, 4)
+    ws = np.exp2(rng.integers(-8, -3, size=N)).astype(np.float32)
+    bias = (rng.integers(-64, 64, size=N) / 8).astype(np.float32)
+    x = rng.integers(-31, 32, size=(M, K)).astype(np.float32)
+    x[2] = 0
+    h = fq.weights_import(to_dev(wc), to_dev(ws), None, to_dev(bias), K, 1, 4)
+    want = oracle.linear_wonly(x, "f32", wc, ws, bias)
+    ybuf = torch.full((M + 2, N + 8), -7.0, dtype=torch.float32, device="cuda")
+    fq.linear_w4a16(to_dev(x), h, y=ybuf[:M, :N])
+    got = to_np(ybuf)
+    assert np.array_equal(got[:M, :N], want)
+    assert np.array_equal(got[2, :N], bias)
+    assert np.all(got[M:] == -7.0) and np.all(got[:, N:] == -7.0)
+    xb = synth.as_dtype(x, "bf16")                                   # small integers are exact in bf16 too
+    assert np.array_equal(to_np(fq.linear_w4a16(to_dev(xb, "bf16"), h)), want)
+    assert fq.linear_w4a16(to_dev(x[:0]), h).shape == (0, N)
+    h8 = fq.weights_import(to_dev(oracle.pack(q, 8)), to_dev(ws), None, None, K, 1, 8)
+    with pytest.raises(fq.FqError) as e:
+        fq.linear_w4a16(to_dev(x), h8)
+    assert e.value.status == fq.ERR_UNSUPPORTED
+
+
+def test_identity_rotation_linear_end_to_end():
+    """block 1 through the whole W4A4 / W8A8 path: smoothing only, no rotation."""
+    for bits, M, K, N in [(4, 70, 1024, 256), (8, 33, 544, 72)]:
+        site = synth.Site("scale_only", M, K, [("p", N)], beta=1, bits=bits, x_dtype="bf16", y_dtype="f32", alpha=0.5)
+        data = synth.make_site(site, seed=bits, calib_tokens=128)
+        gpu, ref = run_site(data)
+        assert np.array_equal(to_np(gpu["codes"]), ref["codes"])
+        assert np.array_equal(to_np(gpu["delta"]).view(np.uint32), ref["delta"].view(np.uint32))
+        assert np.array_equal(to_np(fq.gemm_acc_i32(gpu["codes"], gpu["h"])), ref["acc"])
+        assert_close(to_np(gpu["y"]), ref["y"], "f32", f"identity rotation W{bits}")
 
 
 def test_error_codes_on_device_arguments():
