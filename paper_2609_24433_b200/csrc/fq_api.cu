@@ -123,7 +123,7 @@ fq_status gemm_from_codes(const void* a_codes, const float* a_delta, int64_t M, 
     if (simt) return launch_gemm_simt(a8, M, *W, shift, out, stream) == cudaSuccess ? FQ_OK : FQ_ERR_CUDA;
     size_t scratch_bytes = 0;
     void* scratch = scratch_of(workspace, ws_bytes, M, W->K, &scratch_bytes);
-    return launch_gemm_tcgen05(a8, M, *W, shift, out, scratch, scratch_bytes, stream);
+    return launch_gemm(a8, M, *W, shift, out, scratch, scratch_bytes, stream);
 }
 
 fq_status linear_impl(const void* x, fq_dtype xt, int64_t M, int64_t ldx, const fq_weights* Wp, int bits,
@@ -165,7 +165,7 @@ fq_status linear_impl(const void* x, fq_dtype xt, int64_t M, int64_t ldx, const 
     // 4-bit weights are expanded to 16*code on chip: accumulator = 16 * integer sum.
     size_t scratch_bytes = 0;
     void* scratch = scratch_of(workspace, ws_bytes, M, W->K, &scratch_bytes);
-    return launch_gemm_tcgen05(ws.a8, M, *W, bits == 4 ? 4 : 0, out, scratch, scratch_bytes, s);
+    return launch_gemm(ws.a8, M, *W, bits == 4 ? 4 : 0, out, scratch, scratch_bytes, s);
 }
 
 }  // namespace

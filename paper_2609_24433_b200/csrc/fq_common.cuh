@@ -24,6 +24,8 @@ struct Weights {
     uint32_t* tile_counters = nullptr;   // [1024] zero between launches: slices of a tile finished (K split)
     CUtensorMap tmap;           // TMA view of `codes` for the GEMM's weight operand
     bool tmap_valid = false;
+    CUtensorMap tmap_stream;    // 4-bit weights: view for the short-batch streaming kernel (32 rows x 128 bytes)
+    bool tmap_stream_valid = false;
 };
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -98,7 +100,13 @@ struct GemmOut {
 cudaError_t launch_gemm_simt(const int8_t* a8, int64_t M, const Weights& W, int acc_shift, const GemmOut& out,
                              cudaStream_t stream);
 
-// Weight-only 4-bit projection with float activations (CUDA cores; short batches): y = s^W (qW x) + b.
+// Short-batch weight streaming (4-bit weights, warp-level MMAs fed by a TMA ring).
+//  - launch_linear_wonly4: weight-only projection of float activations, y = s^W (qW x) + b;
+//  - launch_gemm_stream: the integer product + epilogue of the GEMM for batches gemm_stream_applies() accepts.
+bool build_stream_tmap(Weights& W);
+bool gemm_stream_applies(int64_t M, const Weights& W);
+cudaError_t launch_gemm_stream(const int8_t* a8, int64_t M, const Weights& W, int acc_shift, const GemmOut& out,
+                               cudaStream_t stream);
 cudaError_t launch_linear_wonly4(const void* x, fq_dtype xt, int64_t M, int64_t ldx, const Weights& W, void* y,
                                  fq_dtype yt, int64_t ldy, cudaStream_t stream);
 
@@ -107,6 +115,9 @@ cudaError_t launch_linear_wonly4(const void* x, fq_dtype xt, int64_t M, int64_t 
 // gemm_scratch_bytes() is what the split the planner would pick for this shape needs.
 fq_status launch_gemm_tcgen05(const int8_t* a8, int64_t M, const Weights& W, int acc_shift, const GemmOut& out,
                               void* scratch, size_t scratch_bytes, cudaStream_t stream);
+// The GEMM of the runtime path: the streaming kernel for short batches on 4-bit weights, else the tcgen05 kernel.
+fq_status launch_gemm(const int8_t* a8, int64_t M, const Weights& W, int acc_shift, const GemmOut& out,
+                      void* scratch, size_t scratch_bytes, cudaStream_t stream);
 size_t gemm_scratch_bytes(int64_t M, int64_t N, int64_t K, int bits);
 
 // cuTensorMapEncodeTiled through the runtime's driver entry point (no link-time libcuda dependency).

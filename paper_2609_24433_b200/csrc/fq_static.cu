@@ -85,5 +85,5 @@ extern "C" fq_status fq_linear_w4a4_static(const void* x, fq_dtype xt, int64_t M
         return FQ_ERR_CUDA;
     GemmOut out;
     out.y = y; out.yt = yt; out.ldy = ldy; out.a_delta = delta;
-    return launch_gemm_tcgen05(a8, M, *W, 4, out, nullptr, 0, s);   // no scratch: the GEMM does not split K
+    return launch_gemm(a8, M, *W, 4, out, nullptr, 0, s);   // no scratch: the GEMM does not split K
 }

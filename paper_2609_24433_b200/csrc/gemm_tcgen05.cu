@@ -920,6 +920,7 @@ fq_status build_weight_tmap(Weights& W) {
                                     CU_TENSOR_MAP_SWIZZLE_128B);
     if (!ok) return FQ_ERR_CUDA;
     W.tmap_valid = true;
+    build_stream_tmap(W);       // optional second view (short batches); shapes it does not fit go without
     return FQ_OK;
 }
 
@@ -999,6 +1000,14 @@ int device_sms() {
 }
 
 }  // namespace
+
+fq_status launch_gemm(const int8_t* a8, int64_t M, const Weights& W, int acc_shift, const GemmOut& out, void* scratch,
+                      size_t scratch_bytes, cudaStream_t stream) {
+    if (M == 0 || W.N == 0) return FQ_OK;
+    if (gemm_stream_applies(M, W))
+        return launch_gemm_stream(a8, M, W, acc_shift, out, stream) == cudaSuccess ? FQ_OK : FQ_ERR_CUDA;
+    return launch_gemm_tcgen05(a8, M, W, acc_shift, out, scratch, scratch_bytes, stream);
+}
 
 size_t gemm_scratch_bytes(int64_t M, int64_t N, int64_t K, int bits) {
     if (M <= 0 || N <= 0 || K <= 0) return 0;

@@ -1,10 +1,28 @@
-// Weight-only 4-bit projection with floating-point activations (the adaptive layer-normalisation
-// modulation of the W4A4 engines keeps its activations in floating point):
-//   y[t][j] = s^W_j * sum_c qW[j][c] * x[t][c] + b_j
-// These projections see one conditioning vector per sample (M = batch, a handful of tokens), so the
-// operation is a matrix-vector product bound by the weight bytes: CUDA cores, each warp streaming
-// eight weight rows with 8-byte loads per lane while the activations of its 16 channels stay in
-// registers; binary32 accumulation, one fused multiply-add for the rescale and bias.
+// Short-batch weight streaming for 4-bit weights: the projection of a handful of tokens is a
+// matrix-vector product bound by the weight bytes, which must cross HBM once.  Two users:
+//   * the W4A4 integer product of Eq. 8 for batches of at most 32 tokens (the iterative action expert,
+//     the short end of the throughput sweep), where the TMA/TMEM pipeline of the big GEMM cannot be fed
+//     at HBM rate by so thin a tile;
+//   * the weight-only projection with floating-point activations (the adaptive layer-normalisation
+//     modulation of the W4A4 engines):  y[t][j] = s^W_j * sum_c qW[j][c] * x[t][c] + b_j.
+// One persistent CTA per SM walks groups of 32 weight rows.  A producer warp streams the packed rows
+// through a ring of 32 KB stages (32 rows x 2048 channels, ONE 128-byte-swizzled TMA box each: an
+// issuing warp gets out one tensor copy per ~260 cycles whatever its size, so a stage must not be
+// several) that holds ~160 KB in flight per SM; 16 consumer warps each take one 16-row tile x 256 channels of a stage,
+// expand the codes in registers and multiply with warp-level MMAs (m16n8k32 s8 -> s32, or m16n8k16
+// bf16 -> f32 after an exact code -> bf16 expansion); tokens ride along 8 per MMA at no extra weight
+// traffic.  The warps' partial sums meet in shared memory, are added in a fixed order, rescaled and
+// stored.  binary32 activations are split into three bf16 terms (exactly), so both float input types
+// see exact products and binary32 sums.
+//
+// Operand layout.  Lane (g = lane / 4, t = lane % 4) reads 16 bytes = 32 codes of rows g and g + 8 at
+// channel 32 t of the warp's chunk, and the activations of token g at the same channels.  A sum over
+// channels may run in any order as long as both operands agree on it, so the k index of the MMA is
+// mapped to channels the way the codes unpack cheapest:
+//   int8:  (w << 4) & 0xF0F0F0F0 holds 16 x the codes of channels 0,2,4,6 of a word and w & 0xF0F0F0F0
+//          those of channels 1,3,5,7 -- the order in which the prologue stores its int8 codes;
+//   bf16:  one mask of the word shifted by 4 j isolates the codes of channels j and j + 4 in the two
+//          halves of a register, and the B fragment pairs the activations of those channels.
 #include <cuda_bf16.h>
 
 #include "fq_common.cuh"
@@ -13,133 +31,422 @@
 namespace fq {
 namespace {
 
-constexpr int kRows = 8;          // weight rows per warp
-constexpr int kWarps = 8;
-constexpr int kChunk = 16;        // channels per lane and step (one 8-byte load of packed weights)
+constexpr int kConsumers = 16;                  // consumer warps: (row tile, 128-channel slot of a stage)
+constexpr int kThreads = 32 * (kConsumers + 1); // + one producer warp
+constexpr int kRowsCta = 32;                    // two 16-row MMA tiles
+constexpr int kStageCh = 2048;                  // channels per stage
+constexpr int kLines = kStageCh / 256;          // 128-byte lines (256 channels) per row and stage
+constexpr int kStageBytes = kRowsCta * kStageCh / 2;   // one TMA box: 32 rows x 8 lines of 128 bytes (32 KB)
+constexpr int kMaxDepth = 6;
+enum : int { kModeInt = 0, kModeBf16 = 1, kModeF32 = 2 };
 
-// Eight 4-bit two's-complement codes of a word -> binary32, exactly: (n & 15) ^ 8 = n + 8, placed in
-// the mantissa of 2^23, minus (2^23 + 8).
-__device__ __forceinline__ void decode8(uint32_t w, float* q) {
-#pragma unroll
-    for (int i = 0; i < 8; ++i)
-        q[i] = __uint_as_float(((w >> (4 * i)) & 0xFu) ^ 0x4B000008u) - 8388616.0f;
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(c2), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ void mma_bf16(float* d, const uint32_t* a, uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void mma_s8(int* d, const uint32_t* a, uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
 }
 
-template <typename XT>
-__device__ __forceinline__ void load_x16(const XT* p, bool ok, float* v);
-template <>
-__device__ __forceinline__ void load_x16<float>(const float* p, bool ok, float* v) {
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const float4 t = ok ? __ldg(reinterpret_cast<const float4*>(p) + i) : make_float4(0.f, 0.f, 0.f, 0.f);
-        v[4 * i + 0] = t.x; v[4 * i + 1] = t.y; v[4 * i + 2] = t.z; v[4 * i + 3] = t.w;
-    }
+// Codes of channels j and j + 4 of a packed word (eight two's-complement nibbles, channel i at bits
+// 4 i) as two bf16: (n & 15) ^ 8 = n + 8 goes into the mantissa of 128 (0x4300), then 136 comes off.
+// Both steps are exact.
+__device__ __forceinline__ uint32_t codes_bf16x2(uint32_t w, int j) {
+    const uint32_t biased = ((w >> (4 * j)) & 0x000F000Fu) ^ 0x43084308u;
+    uint32_t r;
+    asm("sub.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(biased), "r"(0x43084308u));
+    return r;
 }
+
+// The activations of one token at a lane's 32 channels as B-fragment registers.
+template <int MODE>
+struct XFrag;
+// int8 codes as the prologue stores them: 8 channels = (c0,c2,c4,c6) (c1,c3,c5,c7); word w -> b[2w], b[2w+1]
 template <>
-__device__ __forceinline__ void load_x16<__nv_bfloat16>(const __nv_bfloat16* p, bool ok, float* v) {
+struct XFrag<kModeInt> {
+    typedef int8_t elem;
+    static constexpr int kTerms = 1;
+    uint32_t b[1][8];
+    __device__ __forceinline__ void load(const int8_t* p, bool ok) {
 #pragma unroll
-    for (int i = 0; i < 2; ++i) {
-        const uint4 t = ok ? __ldg(reinterpret_cast<const uint4*>(p) + i) : make_uint4(0u, 0u, 0u, 0u);
-        const uint32_t w[4] = {t.x, t.y, t.z, t.w};
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            v[8 * i + 2 * k + 0] = __uint_as_float(w[k] << 16);
-            v[8 * i + 2 * k + 1] = __uint_as_float(w[k] & 0xFFFF0000u);
+        for (int h = 0; h < 2; ++h) {
+            const uint4 n = ok ? __ldg(reinterpret_cast<const uint4*>(p) + h) : make_uint4(0u, 0u, 0u, 0u);
+            b[0][4 * h + 0] = n.x; b[0][4 * h + 1] = n.y; b[0][4 * h + 2] = n.z; b[0][4 * h + 3] = n.w;
         }
     }
+};
+// bf16: for word w, b[4w + j] = (channel j, channel j + 4), j = 0..3
+template <>
+struct XFrag<kModeBf16> {
+    typedef __nv_bfloat16 elem;
+    static constexpr int kTerms = 1;
+    uint32_t b[1][16];
+    __device__ __forceinline__ void load(const __nv_bfloat16* p, bool ok) {
+#pragma unroll
+        for (int w = 0; w < 4; ++w) {
+            const uint4 n = ok ? __ldg(reinterpret_cast<const uint4*>(p) + w) : make_uint4(0u, 0u, 0u, 0u);
+            b[0][4 * w + 0] = __byte_perm(n.x, n.z, 0x5410);   // (c0, c4)
+            b[0][4 * w + 1] = __byte_perm(n.x, n.z, 0x7632);   // (c1, c5)
+            b[0][4 * w + 2] = __byte_perm(n.y, n.w, 0x5410);   // (c2, c6)
+            b[0][4 * w + 3] = __byte_perm(n.y, n.w, 0x7632);   // (c3, c7)
+        }
+    }
+};
+// binary32, split into three bf16 terms that add up to it exactly (8 + 8 + 8 significant bits, by truncation)
+template <>
+struct XFrag<kModeF32> {
+    typedef float elem;
+    static constexpr int kTerms = 3;
+    uint32_t b[3][16];
+    __device__ __forceinline__ void load(const float* p, bool ok) {
+#pragma unroll
+        for (int w = 0; w < 4; ++w) {
+            const float4 lo4 = ok ? __ldg(reinterpret_cast<const float4*>(p) + 2 * w) : make_float4(0.f, 0.f, 0.f, 0.f);
+            const float4 hi4 = ok ? __ldg(reinterpret_cast<const float4*>(p) + 2 * w + 1) : make_float4(0.f, 0.f, 0.f, 0.f);
+            float r[8] = {lo4.x, lo4.y, lo4.z, lo4.w, hi4.x, hi4.y, hi4.z, hi4.w};
+#pragma unroll
+            for (int s = 0; s < 3; ++s) {
+                uint32_t top[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    top[i] = __float_as_uint(r[i]) & 0xFFFF0000u;            // leading 8 significant bits
+                    r[i] = __fsub_rn(r[i], __uint_as_float(top[i]));        // exact remainder
+                }
+#pragma unroll
+                for (int j = 0; j < 4; ++j) b[s][4 * w + j] = __byte_perm(top[j], top[j + 4], 0x7632);
+            }
+        }
+    }
+};
+
+struct StreamParams {
+    const void* x;            // activations [M, K]: int8 codes (pitch K) or bf16 / binary32 (pitch ldx)
+    int64_t ldx;
+    int64_t M, N;
+    int K;
+    int depth;                // ring stages
+    int acc_shift;            // int8: the integer sum carries a factor 2^acc_shift
+    const float* a_delta;     // int8: per-token steps
+    const float* w_scale;
+    const float* bias;
+    void* y;
+    fq_dtype yt;
+    int64_t ldy;
+    int32_t* acc_out;         // int8: raw sums instead of y (parity/debug)
+    uint32_t* watchdog;
+};
+
+enum : uint32_t { kWdStreamFull = 0x400u, kWdStreamEmpty = 0x800u, kWdStreamSync = 0x1000u };
+
+// GROUPS token groups of 8 per pass over the weights.
+template <int MODE, int GROUPS>
+__global__ void __launch_bounds__(kThreads, 1)
+weight_stream_kernel(const __grid_constant__ CUtensorMap map_w, const StreamParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    typedef typename XFrag<MODE>::elem XT;
+    typedef typename std::conditional<MODE == kModeInt, int, float>::type AccT;
+    constexpr int kTerms = XFrag<MODE>::kTerms;
+    constexpr int kTok = 8 * GROUPS;
+    __shared__ uint64_t s_full[kMaxDepth], s_empty[kMaxDepth];
+    __shared__ uint64_t s_sync;                       // rendezvous of the consumer warps (bounded, unlike bar.sync)
+    __shared__ int s_abort;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    volatile int* abort_flag = &s_abort;
+    const uint32_t ring = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    AccT* s_part = reinterpret_cast<AccT*>(smem_raw + (ring - smem_u32(smem_raw)) + (size_t)p.depth * kStageBytes);
+    // s_part[k slot 0..7][row 0..31][token, padded to kTok + 1]
+
+    if (threadIdx.x == 0) {
+        s_abort = 0;
+        for (int s = 0; s < p.depth; ++s) {
+            mbar_init(smem_u32(&s_full[s]), 1);
+            mbar_init(smem_u32(&s_empty[s]), kConsumers);
+        }
+        mbar_init(smem_u32(&s_sync), kConsumers);
+        fence_mbarrier_init();
+        fence_proxy_async_smem();
+    }
+    __syncthreads();
+    const int row_groups = (int)((p.N + kRowsCta - 1) / kRowsCta);
+    const int stages_k = (p.K + kStageCh - 1) / kStageCh;
+    const int passes = (int)((p.M + kTok - 1) / kTok);
+
+    if (warp == kConsumers) {
+        // ------------------------------------------------------------------ producer
+        // The weights are complete before any call that uses them is enqueued: no need to wait for
+        // the kernel ahead in the stream.
+        griddep_launch_dependents();
+        int slot = 0;
+        uint32_t ph = 0;
+        bool ok = true;
+        for (int rg = blockIdx.x; rg < row_groups && ok; rg += gridDim.x)
+            for (int pass = 0; pass < passes && ok; ++pass)
+                for (int s = 0; s < stages_k; ++s) {
+                    ok = mbar_wait_all(smem_u32(&s_empty[slot]), ph ^ 1u, abort_flag, p.watchdog, kWdStreamEmpty);
+                    if (!ok) break;
+                    if (elect_one()) {
+                        // the weights as [row][128-byte line][byte]: lines past the row's end and rows past N
+                        // are out of bounds and arrive as zeros (the whole box always counts as transferred)
+                        const uint32_t bar = smem_u32(&s_full[slot]);
+                        mbar_arrive_expect_tx(bar, (uint32_t)kStageBytes);
+                        tma_load_3d(ring + slot * kStageBytes, &map_w, 0, s * kLines, rg * kRowsCta, bar);
+                    }
+                    __syncwarp();
+                    if (++slot == p.depth) { slot = 0; ph ^= 1u; }
+                }
+        if (!ok && lane == 0) {               // let the copies already issued land before the CTA gives its memory back
+            const uint64_t t0 = global_timer_ns();
+            while (global_timer_ns() - t0 < 100000ull) __nanosleep(1000);
+        }
+    } else {
+        // ----------------------------------------------------------------- consumers
+        griddep_wait();                       // activations come from the kernel ahead in the stream
+        griddep_launch_dependents();
+        const int g = lane >> 2, t = lane & 3;
+        const int rt = warp & 1, kq = warp >> 1;            // row tile, 128-channel slot of the stage
+        // Stage layout: [row 0..31][line 0..7][128 bytes], line = 256 channels; the 128-byte swizzle XORs the
+        // 16-byte unit index with the low three bits of (8 row + line) = line.  This warp reads line kq of
+        // rows 16 rt + g and 16 rt + 8 + g; lane t takes units 2t and 2t + 1 (64 channels), one after the other.
+        // (All rows of an MMA must use the same channels for a given lane t, so the two rows that share a
+        // shared-memory phase read the same unit: a two-way bank conflict that cannot be swizzled away here.)
+        const int line = kq;
+        const uint32_t unit_off0 = (uint32_t)(((2 * t) ^ line) << 4), unit_off1 = (uint32_t)(((2 * t + 1) ^ line) << 4);
+        int slot = 0;
+        uint32_t ph = 0, sync_ph = 0;
+        bool ok = true;
+        const XT* xp = static_cast<const XT*>(p.x);
+        for (int rg = blockIdx.x; rg < row_groups && ok; rg += gridDim.x) {
+            const int64_t j0 = (int64_t)rg * kRowsCta;
+            for (int pass = 0; pass < passes && ok; ++pass) {
+                const int64_t t0 = (int64_t)pass * kTok;
+                AccT acc[GROUPS][4];
+#pragma unroll
+                for (int q = 0; q < GROUPS; ++q)
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) acc[q][i] = 0;
+                XFrag<MODE> xf[GROUPS];
+                // step = 2 * stage + unit: the lane's 32 channels of that unit
+                auto load_x = [&](int step) {
+                    const int c = (step >> 1) * kStageCh + kq * 256 + 64 * t + 32 * (step & 1);
+#pragma unroll
+                    for (int q = 0; q < GROUPS; ++q) {
+                        const int64_t tok = t0 + 8 * q + g;
+                        xf[q].load(xp + tok * p.ldx + c, tok < p.M && c < p.K);
+                    }
+                };
+                load_x(0);
+                for (int s = 0; s < stages_k; ++s) {
+                    ok = mbar_wait_all(smem_u32(&s_full[slot]), ph, abort_flag, p.watchdog, kWdStreamFull);
+                    if (!ok) break;
+                    const uint32_t rowa = ring + slot * kStageBytes + (uint32_t)(((16 * rt + g) * kLines + line) * 128);
+                    const uint32_t rowb = rowa + 8 * kLines * 128;
+                    const uint4 wq[2][2] = {{lds128(rowa + unit_off0), lds128(rowb + unit_off0)},
+                                            {lds128(rowa + unit_off1), lds128(rowb + unit_off1)}};
+                    __syncwarp();
+                    if (elect_one()) mbar_arrive(smem_u32(&s_empty[slot]));
+                    if (++slot == p.depth) { slot = 0; ph ^= 1u; }
+                    const bool exists = s * kStageCh + kq * 256 < p.K;     // (warp-uniform) the line is inside the row
+#pragma unroll
+                    for (int u = 0; u < 2; ++u) {
+                        const uint32_t w0[4] = {wq[u][0].x, wq[u][0].y, wq[u][0].z, wq[u][0].w};   // row g
+                        const uint32_t w1[4] = {wq[u][1].x, wq[u][1].y, wq[u][1].z, wq[u][1].w};   // row g + 8
+                        if (exists) {
+                            if (MODE == kModeInt) {
+#pragma unroll
+                                for (int w = 0; w < 4; ++w) {
+                                    const uint32_t a[4] = {(w0[w] << 4) & 0xF0F0F0F0u, (w1[w] << 4) & 0xF0F0F0F0u,
+                                                           w0[w] & 0xF0F0F0F0u, w1[w] & 0xF0F0F0F0u};
+#pragma unroll
+                                    for (int q = 0; q < GROUPS; ++q)
+                                        mma_s8(reinterpret_cast<int*>(acc[q]), a, xf[q].b[0][2 * w], xf[q].b[0][2 * w + 1]);
+                                }
+                            } else {
+#pragma unroll
+                                for (int w = 0; w < 4; ++w)
+#pragma unroll
+                                    for (int m = 0; m < 2; ++m) {      // channels (2m, 2m+4 | 2m+1, 2m+5) of the word
+                                        const uint32_t a[4] = {codes_bf16x2(w0[w], 2 * m), codes_bf16x2(w1[w], 2 * m),
+                                                               codes_bf16x2(w0[w], 2 * m + 1), codes_bf16x2(w1[w], 2 * m + 1)};
+#pragma unroll
+                                        for (int q = 0; q < GROUPS; ++q)
+#pragma unroll
+                                            for (int tm = 0; tm < kTerms; ++tm)
+                                                mma_bf16(reinterpret_cast<float*>(acc[q]), a, xf[q].b[tm][4 * w + 2 * m],
+                                                         xf[q].b[tm][4 * w + 2 * m + 1]);
+                                    }
+                            }
+                        }
+                        // the next unit's activations: in flight while this one's MMAs (or the barrier wait) run
+                        if (2 * s + u + 1 < 2 * stages_k) load_x(2 * s + u + 1);
+                    }
+                }
+                if (!ok) break;
+                // C fragment: [0..1] = row g, tokens 2t, 2t+1; [2..3] = row g + 8
+                AccT* part = s_part + (size_t)kq * kRowsCta * (kTok + 1);
+#pragma unroll
+                for (int q = 0; q < GROUPS; ++q) {
+                    part[(16 * rt + g) * (kTok + 1) + 8 * q + 2 * t] = acc[q][0];
+                    part[(16 * rt + g) * (kTok + 1) + 8 * q + 2 * t + 1] = acc[q][1];
+                    part[(16 * rt + g + 8) * (kTok + 1) + 8 * q + 2 * t] = acc[q][2];
+                    part[(16 * rt + g + 8) * (kTok + 1) + 8 * q + 2 * t + 1] = acc[q][3];
+                }
+                __syncwarp();
+                if (elect_one()) mbar_arrive(smem_u32(&s_sync));
+                ok = mbar_wait_all(smem_u32(&s_sync), sync_ph, abort_flag, p.watchdog, kWdStreamSync);
+                sync_ph ^= 1u;
+                if (!ok) break;
+                for (int o = threadIdx.x; o < kRowsCta * kTok; o += kConsumers * 32) {
+                    const int row = o % kRowsCta, tok = o / kRowsCta;    // consecutive threads: consecutive channels
+                    AccT sum = 0;
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) sum += s_part[((size_t)k * kRowsCta + row) * (kTok + 1) + tok];
+                    const int64_t j = j0 + row, tt = t0 + tok;
+                    if (j < p.N && tt < p.M) {
+                        if (MODE == kModeInt && p.acc_out != nullptr) {
+                            p.acc_out[tt * p.N + j] = (int)sum >> p.acc_shift;
+                        } else {
+                            float v;
+                            if (MODE == kModeInt) {
+                                // (float)sum * 2^-shift is exact: the shift is folded into the channel scale
+                                const float sw = __ldg(p.w_scale + j) * (1.0f / (float)(1 << p.acc_shift));
+                                v = fmaf((float)sum, __ldg(p.a_delta + tt) * sw, __ldg(p.bias + j));
+                            } else {
+                                v = fmaf((float)sum, __ldg(p.w_scale + j), __ldg(p.bias + j));
+                            }
+                            if (p.yt == FQ_F32) static_cast<float*>(p.y)[tt * p.ldy + j] = v;
+                            else static_cast<__nv_bfloat16*>(p.y)[tt * p.ldy + j] = __float2bfloat16_rn(v);
+                        }
+                    }
+                }
+                // the partial sums are rewritten by the next pass / row group
+                __syncwarp();
+                if (elect_one()) mbar_arrive(smem_u32(&s_sync));
+                ok = mbar_wait_all(smem_u32(&s_sync), sync_ph, abort_flag, p.watchdog, kWdStreamSync);
+                sync_ph ^= 1u;
+            }
+        }
+    }
+    __syncthreads();
 }
 
-// MT tokens per pass over the weights (their activations live in registers).
-template <typename XT, int MT>
-__global__ void __launch_bounds__(kWarps * 32)
-linear_wonly4_kernel(const XT* __restrict__ x, int64_t M, int K, int64_t ldx, const uint8_t* __restrict__ wcodes,
-                     const float* __restrict__ w_scale, const float* __restrict__ bias, int64_t N, void* __restrict__ y,
-                     fq_dtype yt, int64_t ldy) {
-    griddep_wait();                   // launched with programmatic serialization
+template <int MODE, int GROUPS>
+cudaError_t launch_stream(const CUtensorMap& map, StreamParams p, cudaStream_t stream) {
+    typedef typename std::conditional<MODE == kModeInt, int, float>::type AccT;
+    int dev = 0, sms = 148;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const size_t part_bytes = (size_t)8 * kRowsCta * (8 * GROUPS + 1) * sizeof(AccT);
+    const size_t budget = 227 * 1024 - 1024 /*alignment*/ - 1024 /*static*/ - part_bytes;
+    int depth = (int)(budget / kStageBytes);
+    if (depth > kMaxDepth) depth = kMaxDepth;
+    if (depth < 2) return cudaErrorInvalidConfiguration;
+    p.depth = depth;
+    p.watchdog = watchdog_device_ptr();
+    if (!p.watchdog) return cudaErrorUnknown;
+    const size_t smem = (size_t)depth * kStageBytes + part_bytes + 1024;
+    auto kern = weight_stream_kernel<MODE, GROUPS>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    const int64_t row_groups = (p.N + kRowsCta - 1) / kRowsCta;
+    const unsigned grid = (unsigned)(row_groups < sms ? row_groups : sms);
+    return launch_pdl(kern, grid, (unsigned)kThreads, smem, stream, 1u, map, p);
+}
+
+// Rows shorter than one TMA box (K < 256): one thread per output, plain loops.  Such projections are a
+// few kilobytes; nothing about them is worth tuning.
+template <typename XT>
+__global__ void linear_wonly4_small_kernel(const XT* __restrict__ x, int64_t M, int K, int64_t ldx,
+                                           const uint8_t* __restrict__ wcodes, const float* __restrict__ w_scale,
+                                           const float* __restrict__ bias, int64_t N, void* __restrict__ y, fq_dtype yt,
+                                           int64_t ldy) {
+    griddep_wait();
     griddep_launch_dependents();
-    const int lane = threadIdx.x & 31;
-    const int64_t j0 = ((int64_t)blockIdx.x * kWarps + (threadIdx.x >> 5)) * kRows;
-    if (j0 >= N) return;              // N is a multiple of 8: a warp has all of its rows or none
-    const int64_t pitch = K / 2;
-    for (int64_t t0 = (int64_t)blockIdx.y * MT; t0 < M; t0 += (int64_t)gridDim.y * MT) {
-        float acc[kRows][MT];
-#pragma unroll
-        for (int r = 0; r < kRows; ++r)
-#pragma unroll
-            for (int t = 0; t < MT; ++t) acc[r][t] = 0.0f;
-        for (int c0 = lane * kChunk; c0 < K; c0 += 32 * kChunk) {
-            float xv[MT][kChunk];
-#pragma unroll
-            for (int t = 0; t < MT; ++t) load_x16<XT>(x + (t0 + t) * ldx + c0, t0 + t < M, xv[t]);
-            uint2 w[kRows];
-#pragma unroll
-            for (int r = 0; r < kRows; ++r) w[r] = __ldg(reinterpret_cast<const uint2*>(wcodes + (j0 + r) * pitch + c0 / 2));
-#pragma unroll
-            for (int r = 0; r < kRows; ++r) {
-                float q[kChunk];
-                decode8(w[r].x, q);
-                decode8(w[r].y, q + 8);
-#pragma unroll
-                for (int t = 0; t < MT; ++t)
-#pragma unroll
-                    for (int i = 0; i < kChunk; ++i) acc[r][t] = fmaf(q[i], xv[t][i], acc[r][t]);
-            }
+    const int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x, t = blockIdx.y;
+    if (j >= N || t >= M) return;
+    const uint8_t* wrow = wcodes + j * (K / 2);
+    float acc = 0.0f;
+    for (int c = 0; c < K; c += 2) {
+        const int byte = wrow[c / 2];
+        const float q0 = (float)(((byte & 15) ^ 8) - 8), q1 = (float)(((byte >> 4) ^ 8) - 8);
+        float x0, x1;
+        if (sizeof(XT) == 4) {
+            x0 = reinterpret_cast<const float*>(x)[t * ldx + c];
+            x1 = reinterpret_cast<const float*>(x)[t * ldx + c + 1];
+        } else {
+            x0 = __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(x)[t * ldx + c]);
+            x1 = __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(x)[t * ldx + c + 1]);
         }
-        // lanes hold partial sums over their channels: butterfly reduction, then lane r*MT + t stores
-        float mine = 0.0f;
-#pragma unroll
-        for (int r = 0; r < kRows; ++r)
-#pragma unroll
-            for (int t = 0; t < MT; ++t) {
-                float v = acc[r][t];
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-                if (lane == r * MT + t) mine = v;
-            }
-        if (lane < kRows * MT) {
-            const int r = lane / MT, t = lane % MT;
-            const int64_t j = j0 + r, tt = t0 + t;
-            if (tt < M) {
-                const float v = fmaf(mine, __ldg(w_scale + j), __ldg(bias + j));
-                if (yt == FQ_F32) static_cast<float*>(y)[tt * ldy + j] = v;
-                else static_cast<__nv_bfloat16*>(y)[tt * ldy + j] = __float2bfloat16_rn(v);
-            }
-        }
+        acc = fmaf(q0, x0, acc);
+        acc = fmaf(q1, x1, acc);
     }
-}
-
-template <typename XT>
-cudaError_t launch_xt(const XT* x, int64_t M, const Weights& W, int64_t ldx, void* y, fq_dtype yt, int64_t ldy,
-                      cudaStream_t stream) {
-    const unsigned gx = (unsigned)((W.N / kRows + kWarps - 1) / kWarps);
-    const int K = (int)W.K;
-    auto go = [&](auto kern, int mt) {
-        int64_t groups = (M + mt - 1) / mt;
-        if (groups > 64) groups = 64;               // beyond that a CTA walks several token groups
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(gx, (unsigned)groups, 1);
-        cfg.blockDim = dim3(kWarps * 32, 1, 1);
-        cfg.stream = stream;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[0].val.programmaticStreamSerializationAllowed = 1;
-        cfg.attrs = attr;
-        cfg.numAttrs = 1;
-        return cudaLaunchKernelEx(&cfg, kern, x, M, K, ldx, (const uint8_t*)W.codes, (const float*)W.w_scale,
-                                  (const float*)W.bias, W.N, y, yt, ldy);
-    };
-    if (M == 1) return go(linear_wonly4_kernel<XT, 1>, 1);
-    if (M == 2) return go(linear_wonly4_kernel<XT, 2>, 2);
-    return go(linear_wonly4_kernel<XT, 4>, 4);
+    const float v = fmaf(acc, w_scale[j], bias[j]);
+    if (yt == FQ_F32) static_cast<float*>(y)[t * ldy + j] = v;
+    else static_cast<__nv_bfloat16*>(y)[t * ldy + j] = __float2bfloat16_rn(v);
 }
 
 }  // namespace
 
+bool build_stream_tmap(Weights& W) {
+    W.tmap_stream_valid = false;
+    // rows of whole 128-byte lines only (K a multiple of 256); other widths take the general kernels
+    if (W.bits != 4 || W.N == 0 || W.K % 256 != 0) return true;
+    const uint64_t dims[3] = {128, (uint64_t)W.K / 256, (uint64_t)W.N};
+    const uint64_t strides[2] = {128, (uint64_t)W.K / 2};
+    const uint32_t box[3] = {128, (uint32_t)kLines, (uint32_t)kRowsCta};
+    W.tmap_stream_valid = encode_tiled(&W.tmap_stream, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, W.codes, dims, strides, box, true);
+    return W.tmap_stream_valid;
+}
+
+bool gemm_stream_applies(int64_t M, const Weights& W) {
+    // measured against the tcgen05 kernel: ahead for at most 16 tokens on matrices up to 32 Mi weights
+    return W.bits == 4 && W.tmap_stream_valid && M >= 1 && M <= 16 && W.N * W.K <= (1ll << 25);
+}
+
+cudaError_t launch_gemm_stream(const int8_t* a8, int64_t M, const Weights& W, int acc_shift, const GemmOut& out,
+                               cudaStream_t stream) {
+    StreamParams p{};
+    p.x = a8; p.ldx = W.K; p.M = M; p.N = W.N; p.K = (int)W.K; p.acc_shift = acc_shift;
+    p.a_delta = out.a_delta; p.w_scale = W.w_scale; p.bias = W.bias;
+    p.y = out.y; p.yt = out.yt; p.ldy = out.ldy; p.acc_out = out.acc;
+    if (M <= 8) return launch_stream<kModeInt, 1>(W.tmap_stream, p, stream);
+    return launch_stream<kModeInt, 2>(W.tmap_stream, p, stream);
+}
+
 cudaError_t launch_linear_wonly4(const void* x, fq_dtype xt, int64_t M, int64_t ldx, const Weights& W, void* y,
                                  fq_dtype yt, int64_t ldy, cudaStream_t stream) {
     if (M == 0 || W.N == 0) return cudaSuccess;
-    if (xt == FQ_F32) return launch_xt(static_cast<const float*>(x), M, W, ldx, y, yt, ldy, stream);
-    return launch_xt(static_cast<const __nv_bfloat16*>(x), M, W, ldx, y, yt, ldy, stream);
+    if (!W.tmap_stream_valid) {
+        if (M > 65535) return cudaErrorInvalidConfiguration;
+        const dim3 grid((unsigned)((W.N + 127) / 128), (unsigned)M);
+        if (xt == FQ_F32)
+            linear_wonly4_small_kernel<float><<<grid, 128, 0, stream>>>(static_cast<const float*>(x), M, (int)W.K, ldx, W.codes,
+                                                                        W.w_scale, W.bias, W.N, y, yt, ldy);
+        else
+            linear_wonly4_small_kernel<__nv_bfloat16><<<grid, 128, 0, stream>>>(static_cast<const __nv_bfloat16*>(x), M,
+                                                                                (int)W.K, ldx, W.codes, W.w_scale, W.bias,
+                                                                                W.N, y, yt, ldy);
+        return cudaGetLastError();
+    }
+    StreamParams p{};
+    p.x = x; p.ldx = ldx; p.M = M; p.N = W.N; p.K = (int)W.K;
+    p.w_scale = W.w_scale; p.bias = W.bias; p.y = y; p.yt = yt; p.ldy = ldy;
+    if (xt == FQ_F32) return launch_stream<kModeF32, 1>(W.tmap_stream, p, stream);
+    if (M <= 8) return launch_stream<kModeBf16, 1>(W.tmap_stream, p, stream);
+    return launch_stream<kModeBf16, 2>(W.tmap_stream, p, stream);
 }
 
 }  // namespace fq
