@@ -8,7 +8,7 @@ one batch: per site the prologue kernel (scale + FWHT + per-token quantization) 
 tcgen05 integer GEMM with its dequant/bias epilogue.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
-                    [--workload backbone_layer|expert_loop|sweep]
+                    [--workload backbone_layer|backbone_layer_w4|expert_layer|sweep:M,K,N,block,bits[,after]|w4a16:M,K,N]
 
 Prints ONE JSON line (rank 0).  ``--impl reference`` times the CPU oracle on host cores.
 """
@@ -375,6 +375,138 @@ def run_e2e(layer, sites, ops, world, K, Wm, dist, device):
             "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": n}
 
 
+# --------------------------------------- weight-only W4A16 projection (its own workload) ----
+def w4a16_shape(name: str):
+    M, K, N = (int(v) for v in name[len("w4a16:"):].split(","))
+    return M, K, N
+
+
+def w4a16_inputs(M: int, K: int, N: int, seed: int):
+    rng = np.random.default_rng(seed)
+    W = synth.draw_weights(rng, N, K)
+    b = rng.standard_normal(N).astype(np.float32)
+    x = synth.as_dtype(rng.standard_normal((M, K)).astype(np.float32), "bf16")
+    return W, b, x
+
+
+def w4a16_cpu_baseline(M: int, K: int, N: int, steps: int):
+    import oracle
+    W, b, x = w4a16_inputs(M, K, N, 2)
+    rows = min(N, max(8, (1 << 28) // max(1, M * K) // 8 * 8))     # bound the sample to ~2.7e8 multiply-adds
+    wc, ws, _ = oracle.fold_weights(W[:rows], "f32", None, 1, 4)     # offline, untimed
+    times = []
+    for _ in range(steps):
+        t0 = time.perf_counter()
+        oracle.linear_wonly(x, "bf16", wc, ws, b[:rows], 4, "bf16")
+        times.append(time.perf_counter() - t0)
+    dt = statistics.mean(times)
+    return {"value": round(2.0 * M * K * rows / dt / 1e12, 6), "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"{rows} of {N} output channels, all {M} tokens (binary64 products and sums), {dt:.2f} s per step",
+            "seconds_per_step": round(dt, 3)}
+
+
+def run_w4a16(args, rank: int, world: int, local_rank: int):
+    """fq_linear_w4a16 alone: y = s^W (qW x) + b on bf16 activations, weights rotating through enough
+    handles that every call streams its 4-bit codes from HBM.  The bound is HBM (weight bytes)."""
+    import torch
+    from paper_2609_24433_b200 import fq
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=device)
+    M, K, N = w4a16_shape(args.workload)
+    sets = max(ROTATE, min(64, -(-300_000_000 // (N * K // 2))))      # > 2 x L2 of packed weights in rotation
+    hs, xs = [], []
+    for r in range(sets):
+        W, b, x = w4a16_inputs(M, K, N, replicas.replica_seed(2, rank) + r)
+        hs.append(fq.fold_weights(torch.from_numpy(W).to(device), None, torch.from_numpy(b).to(device), 1, 4))
+        xs.append(torch.from_numpy(x.view(np.int16)).to(device).view(torch.bfloat16))
+    y = torch.empty((M, N), dtype=torch.bfloat16, device=device)
+    steps, Wm = args.steps, max(args.warmup, 3)
+    for k in range(Wm):
+        fq.linear_w4a16(xs[k % sets], hs[k % sets], y=y)
+    torch.cuda.synchronize()
+    # the K timed steps are ONE captured graph (K kernel nodes, handles rotating): a replay per step would
+    # time the graph launch (4-5 us) rather than this microsecond-scale kernel
+    timed = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(timed):
+        for k in range(steps):
+            fq.linear_w4a16(xs[(Wm + k) % sets], hs[(Wm + k) % sets], y=y)
+    timed.replay()                      # untimed: every handle touched once more before the timed replay
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(local_rank)
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    with sampler:
+        start.record()
+        timed.replay()
+        end.record()
+        torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    ms_total = start.elapsed_time(end)
+    note = ""
+    if len(sampler.samples) < 5:
+        sampler = ClockSampler(local_rank)
+        t_end = time.time() + 0.5
+        with sampler:
+            while time.time() < t_end:
+                timed.replay()
+                torch.cuda.synchronize()
+        note = "sampled during an immediate untimed replay of the timed loop (timed region < NVML period)"
+    st, word = fq.device_status()
+    if st != fq.OK:
+        raise RuntimeError(f"device watchdog fired during the benchmark: {word:#x}")
+    ops = 2.0 * M * K * N
+    ms_per_step = replicas.max_over_ranks(ms_total, dist, device) / steps
+    value = replicas.job_throughput(ops * steps, ms_total * 1e-3, dist, device) / 1e12
+    peaks = read_peaks()
+    alg_bytes = N * K // 2 + 8 * N + 2 * M * K + 2 * M * N          # codes + scale/bias + x + y
+    gbs = alg_bytes / (ms_total / steps * 1e-3) / 1e9
+    # end to end: x from pinned host memory, y back to pinned host memory, every step
+    hx = torch.from_numpy(w4a16_inputs(M, K, N, 2)[2].view(np.int16)).pin_memory()
+    hy = torch.empty((M, N), dtype=torch.bfloat16).pin_memory()
+    n = max(3, min(steps, 50))
+
+    def e2e_step(k):
+        xs[k % sets].view(torch.int16).copy_(hx, non_blocking=True)
+        fq.linear_w4a16(xs[k % sets], hs[k % sets], y=y)
+        hy.copy_(y, non_blocking=True)
+        torch.cuda.synchronize()
+    for k in range(3):
+        e2e_step(k)
+    start.record()
+    for k in range(n):
+        e2e_step(k)
+    end.record()
+    torch.cuda.synchronize()
+    sec = start.elapsed_time(end) * 1e-3
+    e2e = {"value": round(replicas.job_throughput(ops * n, sec, dist, device) / 1e12, 4), "unit": UNIT,
+           "ms_per_step": round(replicas.max_over_ranks(sec, dist, device) / n * 1e3, 4),
+           "h2d_bytes_per_step": 2 * M * K, "d2h_bytes_per_step": 2 * M * N, "steps": n}
+    out = {"metric": "weight-only W4A16 projection (fq_linear_w4a16)", "value": round(value, 3), "unit": UNIT,
+           "n_gpus": world, "steps": steps, "warmup": Wm, "ms_per_step": round(ms_per_step, 5),
+           "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+           "dtype": "int4 codes expanded to bf16 (exact), bf16 activations, f32 accumulate", "data": "synthetic", "impl": "ours",
+           "config": {"workload": f"weight-only INT4 projection, M={M} tokens, K={K}, N={N}, bf16 in/out",
+                      "l2": f"{sets} rotating weight handles ({sets * N * K // 2 >> 20} MiB of codes), no flush kernel",
+                      "launch": "the K steps are one CUDA graph of K kernel nodes", "parallelism": "replicas only"},
+           "clocks": sampler.summary(note), "e2e": e2e, "gpu_launches": steps,
+           "roofline": {"bound": "hbm", "kernel": "weight_stream_kernel<bf16>", "achieved": round(gbs, 1),
+                        "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": round(gbs / peaks["hbm_gbs"], 4),
+                        "bytes": alg_bytes, "traffic": None, "peak_source": f"{peaks['source']}: copy rate"}}
+    if rank == 0:
+        if world == 1 and not args.no_cpu_baseline:
+            out["cpu_baseline"] = w4a16_cpu_baseline(M, K, N, steps=1)
+        print(json.dumps(out), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
 # ------------------------------------------------------------------- oracle arm ----
 def cpu_baseline(workload: str, steps: int):
     """The CPU oracle, as it stands, on a bounded sample of the same workload."""
@@ -413,6 +545,19 @@ def cpu_baseline(workload: str, steps: int):
 
 
 def run_reference(args):
+    if args.workload.startswith("w4a16:"):
+        M, K, N = w4a16_shape(args.workload)
+        steps = max(1, min(args.steps, 5))
+        base = w4a16_cpu_baseline(M, K, N, steps)
+        print(json.dumps({"metric": "weight-only W4A16 projection (fq_linear_w4a16)", "value": base["value"], "unit": UNIT,
+                          "n_gpus": args.gpus, "steps": steps, "warmup": 0,
+                          "ms_per_step": round(base["seconds_per_step"] * 1e3, 2), "higher_is_better": True,
+                          "scaling": "weak", "vs_baseline": None, "dtype": "binary64 products and sums", "data": "synthetic",
+                          "impl": "reference", "config": {"workload": f"weight-only INT4 projection, M={M}, K={K}, N={N}"},
+                          "cpu_baseline": base,
+                          "e2e": {"value": base["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}),
+              flush=True)
+        return
     sites = workload_sites(args.workload)
     steps = max(1, min(args.steps, 5))
     base = cpu_baseline(args.workload, steps=steps)
@@ -472,6 +617,9 @@ def main():
     if args.impl == "reference":
         if rank == 0:
             run_reference(args)
+        return
+    if args.workload.startswith("w4a16:"):
+        run_w4a16(args, rank, world, local_rank)
         return
     run_ours(args, rank, world, local_rank)
 
