@@ -253,3 +253,33 @@ def linear_wonly(x: np.ndarray, xdtype: str, w_codes: np.ndarray, w_scale, bias,
                                     ctypes.c_int64(N), ctypes.c_int(bits), _p(y), ctypes.c_int(_dt(out_dtype)),
                                     ctypes.c_int64(N)), "linear_wonly")
     return y
+
+
+def composite_quantize(x: np.ndarray, dtype: str, pre, perm, blocks, bits: int, clip_ratio: float = 1.0,
+                       return_z: bool = False):
+    """Stored composite rotation R = blockdiag(B_b) Pi: z = R (pre (.) x), then Eq. 5.  ``blocks`` is
+    [K/beta, beta, beta]; ``perm[c]`` the source channel of position c.  Returns (codes, delta[, z])."""
+    x = _mat(x, dtype)
+    M, K = x.shape
+    blocks = np.ascontiguousarray(blocks, dtype=np.float32)
+    beta = blocks.shape[1]
+    assert blocks.shape == (K // beta, beta, beta)
+    perm = np.ascontiguousarray(perm, dtype=np.int32)
+    codes = np.zeros((M, K * bits // 8), dtype=np.uint8)
+    delta = np.zeros(M, dtype=np.float32)
+    z = np.zeros((M, K), dtype=np.float32) if return_z else None
+    _check(_load().fqo_composite_quantize(_p(x), ctypes.c_int(_dt(dtype)), ctypes.c_int64(M), ctypes.c_int64(K),
+                                          ctypes.c_int64(K), _p(_f32(pre)), _p(perm), _p(blocks), ctypes.c_int(beta),
+                                          ctypes.c_int(bits), ctypes.c_float(clip_ratio), _p(codes), _p(delta), _p(z)),
+           "composite_quantize")
+    return (codes, delta, z) if return_z else (codes, delta)
+
+
+def fold_weights_composite(W: np.ndarray, dtype: str, smooth, perm, blocks, bits: int, return_wt: bool = False):
+    """Offline fold for a composite rotation: row j of W~ = R (s (.) w_j), RTN, pack.  Returns
+    (codes, w_scale[N], mult_g[K] = 1/s (ones without smoothing)[, W~])."""
+    K = W.shape[1]
+    s = None if smooth is None else _f32(smooth)
+    out = composite_quantize(W, dtype, s, perm, blocks, bits, 1.0, return_z=return_wt)
+    g = np.ones(K, np.float32) if s is None else (np.float32(1.0) / s).astype(np.float32)
+    return (out[0], out[1], g, out[2]) if return_wt else (out[0], out[1], g)

@@ -283,6 +283,55 @@ int fqo_transform_quantize(const void* x, int dtype, int64_t M, int64_t K, int64
     return 0;
 }
 
+/* Stored composite rotation (section "Transforms supported by the runtime": optional for the action
+ * expert -- a channel permutation followed by one stored dense matrix per block of beta channels):
+ *   R = blockdiag(B_0 .. B_{K/beta-1}) Pi,   z = R (d (.) x),   then Eq. 5.
+ *   pre  (optional) = the input diagonal d (1/s at run time, s when folding weights); NULL = 1;
+ *   perm[c]         = source channel of position c: p_c = v[perm[c]];
+ *   blocks          = [K/beta][beta][beta] row-major, u[b*beta + i] = sum_j B_b[i][j] * p[b*beta + j].
+ * The normalisation lives inside the stored matrices (no beta^(-1/2) factor here).  binary32: one
+ * multiply for the diagonal, then one fused multiply-add per term in ascending j, starting from 0.
+ * Applied to weight rows with pre = s this is the offline fold: row j of W~ = W S R^T is R (s (.) w_j)
+ * for any real R.  z_out (optional) receives z [M, K]. */
+int fqo_composite_quantize(const void* x, int dtype, int64_t M, int64_t K, int64_t ldx, const float* pre,
+                           const int32_t* perm, const float* blocks, int beta, int bits, float clip_ratio,
+                           uint8_t* codes, float* delta, float* z_out) {
+    if (beta < 1 || beta > 256 || K <= 0 || K % beta != 0 || (bits != 4 && bits != 8)) return 1;
+    if (!(clip_ratio > 0.0f && clip_ratio <= 1.0f) || !perm || !blocks) return 1;
+    if (M < 0 || ldx < K || (M > 0 && (!x || !codes || !delta))) return 1;
+    for (int64_t c = 0; c < K; ++c)
+        if (perm[c] < 0 || perm[c] >= K) return 1;
+    int64_t pitch = K * bits / 8;
+#pragma omp parallel
+    {
+        float* v = (float*)malloc(sizeof(float) * (size_t)K);
+        float* u = (float*)malloc(sizeof(float) * (size_t)K);
+        int* code = (int*)malloc(sizeof(int) * (size_t)K);
+#pragma omp for schedule(static)
+        for (int64_t t = 0; t < M; ++t) {
+            for (int64_t c = 0; c < K; ++c) {
+                float xv = load_elem(x, dtype, t * ldx + c);
+                v[c] = pre ? xv * pre[c] : xv;
+            }
+            for (int64_t b = 0; b < K / beta; ++b) {
+                const float* B = blocks + b * (int64_t)beta * beta;
+                for (int i = 0; i < beta; ++i) {
+                    float acc = 0.0f;
+                    for (int j = 0; j < beta; ++j) acc = fmaf(B[i * beta + j], v[perm[b * beta + j]], acc);
+                    u[b * beta + i] = acc;
+                }
+            }
+            if (z_out) memcpy(z_out + t * K, u, sizeof(float) * (size_t)K);
+            delta[t] = quantize_row(u, K, bits, clip_ratio, code);
+            pack_row(code, K, bits, codes + t * pitch);
+        }
+        free(v);
+        free(u);
+        free(code);
+    }
+    return 0;
+}
+
 /* Fold-after, offline half: W~ = W R^T P, row j = (R w_j) (.) p (the block Hadamard matrix is
  * symmetric), then RTN as in fqo_fold_weights.  mult_post (optional) receives the RUNTIME
  * post-rotation multiplier 1/p_c (one binary32 division per channel); at run time the

@@ -580,3 +580,75 @@ def test_weight_only_linear_one_hot_bf16_and_linearity():
     # bf16 output: one rounding of the binary64 result
     yb = oracle.linear_wonly(x1, "f32", wc, ws, None, out_dtype="bf16")
     assert np.array_equal(yb, synth.f32_to_bf16_bits(oracle.linear_wonly(x1, "f32", wc, ws, None)))
+
+
+# ----------------------------------------------- stored composite rotation ----
+def _random_rotation(rng, K, beta):
+    """Random permutation and per-block orthogonal matrices (QR of Gaussians), float32."""
+    perm = rng.permutation(K).astype(np.int32)
+    blocks = np.stack([np.linalg.qr(rng.standard_normal((beta, beta)))[0] for _ in range(K // beta)]).astype(np.float32)
+    return perm, blocks
+
+
+def test_composite_rotation_hand_case():
+    """beta = 2, K = 4 (padded to 32 with identity blocks): perm = (1, 0, 3, 2), B_0 = [[1, 2], [3, 4]],
+    B_1 = [[0.5, -0.5], [0.25, 1]], pre = (2, 1, 1, 0.5), x = (1, 2, 3, 4):
+    v = (2, 2, 3, 2); p = (2, 2, 2, 3); u = (1*2 + 2*2, 3*2 + 4*2, 0.5*2 - 0.5*3, 0.25*2 + 3) = (6, 14, -0.5, 3.5)."""
+    K, beta = 32, 2
+    perm = np.arange(K, dtype=np.int32)
+    perm[:4] = [1, 0, 3, 2]
+    blocks = np.tile(np.eye(2, dtype=np.float32), (K // beta, 1, 1))
+    blocks[0] = [[1, 2], [3, 4]]
+    blocks[1] = [[0.5, -0.5], [0.25, 1]]
+    pre = np.ones(K, np.float32)
+    pre[:4] = [2, 1, 1, 0.5]
+    x = np.zeros((1, K), np.float32)
+    x[0, :4] = [1, 2, 3, 4]
+    codes, delta, z = oracle.composite_quantize(x, "f32", pre, perm, blocks, 8, 1.0, return_z=True)
+    assert np.array_equal(z[0, :4], [6, 14, -0.5, 3.5]) and not z[0, 4:].any()
+    assert delta[0] == np.float32(14.0) / np.float32(127.0)
+    assert np.array_equal(oracle.unpack(codes, K, 8)[0, :4], [54, 127, -5, 32])     # rint(u * 127 / 14), -4.54 -> -5
+
+
+@pytest.mark.parametrize("beta", [16, 64])
+def test_composite_rotation_with_hadamard_blocks_is_the_fwht_path(beta):
+    """Identity permutation and B_b = beta^-1/2 H_beta (entries +-2^-k, exact) on integer inputs: every
+    operation of both routes is exact, so the stored-matrix route must reproduce the butterflies."""
+    rng = np.random.default_rng(beta)
+    K = 4 * beta
+    x = rng.integers(-50, 51, size=(6, K)).astype(np.float32)
+    H = (sylvester(beta) / np.sqrt(beta)).astype(np.float32)
+    blocks = np.tile(H, (K // beta, 1, 1))
+    c1, d1, z1 = oracle.composite_quantize(x, "f32", None, np.arange(K), blocks, 4, 1.0, return_z=True)
+    c2, d2, z2 = oracle.quantize_act(x, "f32", None, beta, 4, 1.0, return_z=True)
+    assert np.array_equal(z1, z2) and np.array_equal(d1, d2) and np.array_equal(c1, c2)
+
+
+def test_composite_rotation_matches_dense_matrices_and_keeps_the_projection():
+    rng = np.random.default_rng(21)
+    K, beta, N = 128, 32, 24
+    perm, blocks = _random_rotation(rng, K, beta)
+    x = rng.standard_normal((5, K)).astype(np.float32)
+    W = rng.standard_normal((N, K)).astype(np.float32)
+    s = np.exp(rng.uniform(-1, 1, K)).astype(np.float32)
+    # dense R = blockdiag(B) Pi, built independently in float64
+    Pi = np.zeros((K, K))
+    Pi[np.arange(K), perm] = 1.0
+    Bd = np.zeros((K, K))
+    for b in range(K // beta):
+        Bd[b * beta:(b + 1) * beta, b * beta:(b + 1) * beta] = blocks[b]
+    R = Bd @ Pi
+    _, _, g, wt = oracle.fold_weights_composite(W, "f32", s, perm, blocks, 8, return_wt=True)
+    _, _, z = oracle.composite_quantize(x, "f32", g, perm, blocks, 8, 1.0, return_z=True)
+    assert np.allclose(z, (R @ (x / s).T.astype(np.float64)).T, rtol=1e-5, atol=1e-5)
+    assert np.allclose(wt, (R @ (W * s).T.astype(np.float64)).T, rtol=1e-5, atol=1e-5)
+    # R is orthogonal (to float32 accuracy of the stored blocks): the unquantized projection is preserved
+    want = x.astype(np.float64) @ W.astype(np.float64).T
+    assert np.allclose(z.astype(np.float64) @ wt.astype(np.float64).T, want, rtol=1e-4, atol=1e-4)
+    # a transposed block or an inverted permutation would not preserve it
+    wrong = np.transpose(blocks, (0, 2, 1)).copy()
+    _, _, zbad = oracle.composite_quantize(x, "f32", g, perm, wrong, 8, 1.0, return_z=True)
+    assert not np.allclose(zbad.astype(np.float64) @ wt.astype(np.float64).T, want, rtol=1e-2, atol=1e-2)
+    inv = np.argsort(perm).astype(np.int32)
+    _, _, zbad = oracle.composite_quantize(x, "f32", g, inv, blocks, 8, 1.0, return_z=True)
+    assert not np.allclose(zbad.astype(np.float64) @ wt.astype(np.float64).T, want, rtol=1e-2, atol=1e-2)
