@@ -123,6 +123,32 @@ fq_status fq_weights_import_after(const void* codes, const float* w_scale, const
                                   const float* bias, int64_t N, int64_t K, int hadamard_block, int bits,
                                   void* stream, fq_weights** out);
 
+/* ---- stored composite rotation (section "Transforms supported by the runtime": optional for the action
+ * expert; the design ablation "butterfly vs. composite rotation") ------------------------------------------
+ * R = blockdiag(B_0 .. B_{K/block-1}) Pi: a channel permutation, then one stored dense block x block matrix per
+ * block of channels.   z[b*block + i] = sum_j B_b[i][j] * v[perm[b*block + j]],  v = x (.) (1/s).
+ *   perm   device int32[K]: perm[c] = source channel of position c (a permutation of 0..K-1);
+ *   blocks device float[K/block][block][block], row-major; orthogonal matrices that carry their own
+ *          normalisation (e.g. block^-1/2 H U^T of an SVD basis U) -- the library does not check orthogonality:
+ *          the fold W~ = W S R^T computed here is row j = R (s (.) w_j), which equals W S R^-1 only if R^T R = I;
+ *   block  in {16, 32, 64, 128, 256}.
+ * Arithmetic: binary32, one multiply for the diagonal, then one fused multiply-add per term in ascending j.
+ * fq_fold_weights_composite: as fq_fold_weights (RTN per output channel, packing, allocation, offline
+ *   synchronisation); FQ_ERR_INVALID_ARG if perm has an entry outside [0, K).  The handle's runtime multiplier is
+ *   1/s_c (ones without smoothing).  The handle does not keep perm and blocks.
+ * fq_quantize_act_composite: the runtime prologue of such a site (rotation, then Eq. 5); workspace device, at least
+ *   4*M*K bytes, 16-byte aligned (the rotated rows in binary32; two kernels).  Entries of perm outside [0, K) are
+ *   clamped.  Then fq_gemm_w4a4 / fq_gemm_w8a8 per consumer; the one-call fq_linear_* entry points return
+ *   FQ_ERR_UNSUPPORTED for a composite handle. */
+fq_status fq_fold_weights_composite(const void* W, fq_dtype wt, int64_t N, int64_t K, int64_t ldw, const float* smooth,
+                                    const float* bias, const int32_t* perm, const float* blocks, int block, int bits,
+                                    void* stream, fq_weights** out);
+fq_status fq_quantize_act_composite(const void* x, fq_dtype xt, int64_t M, int64_t K, int64_t ldx, const float* mult_g,
+                                    const int32_t* perm, const float* blocks, int block, int bits, float clip_ratio,
+                                    void* codes_out, float* delta_out, void* workspace, size_t ws_bytes, void* stream);
+/* 1 if the handle was folded with a stored composite rotation, else 0. */
+int fq_weights_composite(const fq_weights* w);
+
 /* ---- calibration support (section "Transforms supported by the runtime", SmoothQuant scale) --
  * fq_col_absmax: out[c] = max(out[c] if accumulate else 0, max_t |x[t][c]|); x device [M, K].
  * fq_smooth_scale: s_c = clamp(max(a_c,1e-5)^alpha / max(w_c,1e-5)^(1-alpha), 1e-5, 1e5) in

@@ -132,6 +132,7 @@ fq_status linear_impl(const void* x, fq_dtype xt, int64_t M, int64_t ldx, const 
     const Weights* W = reinterpret_cast<const Weights*>(Wp);
     if (!W || M < 0) return FQ_ERR_INVALID_ARG;
     if (W->bits != bits) return FQ_ERR_UNSUPPORTED;
+    if (W->composite) return FQ_ERR_UNSUPPORTED;   // two calls: fq_quantize_act_composite, then fq_gemm_*
     if (!(clip_ratio > 0.0f && clip_ratio <= 1.0f)) return FQ_ERR_INVALID_ARG;
     if (xt != FQ_F32 && xt != FQ_BF16) return FQ_ERR_INVALID_ARG;
     if (M == 0 || W->N == 0) return FQ_OK;
@@ -246,6 +247,89 @@ fq_status fq_fold_weights_after(const void* Wsrc, fq_dtype wt, int64_t N, int64_
                                 const float* bias, int hadamard_block, int bits, void* stream, fq_weights** out) {
     if (!post_scale) return FQ_ERR_INVALID_ARG;
     return fold_impl(Wsrc, wt, N, K, ldw, post_scale, true, bias, hadamard_block, bits, stream, out);
+}
+
+fq_status fq_fold_weights_composite(const void* Wsrc, fq_dtype wt, int64_t N, int64_t K, int64_t ldw, const float* smooth,
+                                    const float* bias, const int32_t* perm, const float* blocks, int block, int bits,
+                                    void* stream, fq_weights** out) {
+    if (!out) return FQ_ERR_INVALID_ARG;
+    *out = nullptr;
+    fq_status st = check_shape(N, K, block, bits);
+    if (st != FQ_OK) return st;
+    if (block < 16) return FQ_ERR_UNSUPPORTED;
+    if (wt != FQ_F32 && wt != FQ_BF16) return FQ_ERR_INVALID_ARG;
+    if (!perm || !blocks || K > kMaxPrologueK) return !perm || !blocks ? FQ_ERR_INVALID_ARG : FQ_ERR_UNSUPPORTED;
+    if (N > 0 && (!Wsrc || ldw < K)) return FQ_ERR_INVALID_ARG;
+    if ((smooth && !aligned16(smooth)) || (bias && !aligned16(bias))) return FQ_ERR_ALIGNMENT;
+    st = check_arch();
+    if (st != FQ_OK) return st;
+    Weights* w = nullptr;
+    st = alloc_handle(N, K, block, bits, &w);
+    if (st != FQ_OK) return st;
+    w->composite = true;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    float* mult_w = nullptr;   // s_c, only needed while folding
+    float* u = nullptr;        // rotated rows before rounding
+    int* bad = nullptr;
+    bool ok = cudaMalloc(&mult_w, sizeof(float) * (size_t)K) == cudaSuccess &&
+              cudaMalloc(&u, sizeof(float) * (size_t)(N > 0 ? N : 1) * (size_t)K) == cudaSuccess &&
+              cudaMalloc(&bad, sizeof(int)) == cudaSuccess;
+    if (!ok) {
+        cudaFree(mult_w); cudaFree(u); cudaFree(bad);
+        fq_weights_destroy(reinterpret_cast<fq_weights*>(w));
+        return FQ_ERR_NOMEM;
+    }
+    // the normalisation lives in the stored matrices: both vectors carry the diagonal only (s and 1/s)
+    ok = cudaMemsetAsync(bad, 0, sizeof(int), s) == cudaSuccess;
+    ok = ok && launch_perm_check(perm, K, bad, s) == cudaSuccess;
+    ok = ok && launch_multipliers(smooth, K, 1.0f, mult_w, w->mult_g, s) == cudaSuccess;
+    ok = ok && launch_composite_rotate(Wsrc, wt, N, K, ldw, smooth ? mult_w : nullptr, perm, blocks, block, u, s) == cudaSuccess;
+    ok = ok && launch_transform_quantize(u, FQ_F32, N, K, K, nullptr, 1.0f, false, 1, bits == 4 ? 7 : 127, 1.0f,
+                                         bits == 4 ? StoreFmt::Nibble : StoreFmt::Int8, w->codes, w->w_scale, s) == cudaSuccess;
+    if (N > 0) {
+        if (bias)
+            ok = ok && cudaMemcpyAsync(w->bias, bias, sizeof(float) * (size_t)N, cudaMemcpyDeviceToDevice, s) == cudaSuccess;
+        else
+            ok = ok && cudaMemsetAsync(w->bias, 0, sizeof(float) * (size_t)N, s) == cudaSuccess;
+    }
+    int bad_host = 0;
+    ok = ok && cudaMemcpyAsync(&bad_host, bad, sizeof(int), cudaMemcpyDeviceToHost, s) == cudaSuccess;
+    ok = ok && cudaStreamSynchronize(s) == cudaSuccess;   // the temporaries are freed below; folding is offline
+    cudaFree(mult_w); cudaFree(u); cudaFree(bad);
+    if (ok && !bad_host) ok = build_weight_tmap(*w) == FQ_OK;
+    if (!ok || bad_host) {
+        fq_weights_destroy(reinterpret_cast<fq_weights*>(w));
+        return bad_host ? FQ_ERR_INVALID_ARG : FQ_ERR_CUDA;
+    }
+    *out = reinterpret_cast<fq_weights*>(w);
+    return FQ_OK;
+}
+
+int fq_weights_composite(const fq_weights* wp) {
+    const Weights* w = reinterpret_cast<const Weights*>(wp);
+    return (w && w->composite) ? 1 : 0;
+}
+
+fq_status fq_quantize_act_composite(const void* x, fq_dtype xt, int64_t M, int64_t K, int64_t ldx, const float* mult_g,
+                                    const int32_t* perm, const float* blocks, int block, int bits, float clip_ratio,
+                                    void* codes_out, float* delta_out, void* workspace, size_t ws_bytes, void* stream) {
+    if (M < 0 || (bits != 4 && bits != 8)) return FQ_ERR_INVALID_ARG;
+    if (xt != FQ_F32 && xt != FQ_BF16) return FQ_ERR_INVALID_ARG;
+    if (!(clip_ratio > 0.0f && clip_ratio <= 1.0f)) return FQ_ERR_INVALID_ARG;
+    if (!valid_block(block, K) || block < 16 || K % 32 != 0 || K > kMaxPrologueK) return FQ_ERR_UNSUPPORTED;
+    if (M == 0) return FQ_OK;
+    if (!x || !codes_out || !delta_out || !perm || !blocks || ldx < K) return FQ_ERR_INVALID_ARG;
+    if (!aligned16(codes_out) || (mult_g && !aligned16(mult_g))) return FQ_ERR_ALIGNMENT;
+    if (!workspace || ws_bytes < sizeof(float) * (size_t)M * (size_t)K) return FQ_ERR_NOMEM;
+    if (!aligned16(workspace)) return FQ_ERR_ALIGNMENT;
+    fq_status st = check_arch();
+    if (st != FQ_OK) return st;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    float* u = static_cast<float*>(workspace);
+    if (launch_composite_rotate(x, xt, M, K, ldx, mult_g, perm, blocks, block, u, s) != cudaSuccess) return FQ_ERR_CUDA;
+    return launch_transform_quantize(u, FQ_F32, M, K, K, nullptr, 1.0f, false, 1, bits == 4 ? 7 : 127, clip_ratio,
+                                     bits == 4 ? StoreFmt::Nibble : StoreFmt::Int8, codes_out, delta_out, s) == cudaSuccess
+               ? FQ_OK : FQ_ERR_CUDA;
 }
 
 int fq_weights_fold_after(const fq_weights* wp) {

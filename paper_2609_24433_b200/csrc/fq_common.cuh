@@ -21,6 +21,7 @@ struct Weights {
     float* bias = nullptr;      // [N]
     float* mult_g = nullptr;    // [K] runtime multiplier (1/s_c) * block^-1/2
     bool fold_after = false;    // mult_g is the post-rotation multiplier 1/p (T = P^-1 R) instead of (1/s) block^-1/2
+    bool composite = false;     // folded with a stored composite rotation: the prologue is fq_quantize_act_composite
     uint32_t* tile_counters = nullptr;   // [1024] zero between launches: slices of a tile finished (K split)
     CUtensorMap tmap;           // TMA view of `codes` for the GEMM's weight operand
     bool tmap_valid = false;
@@ -131,6 +132,13 @@ cudaError_t launch_transform_quantize_ring(const void* x, fq_dtype xt, int64_t r
                                            const float* mult, float cnorm, bool mult_after_rotation, int block,
                                            int qmax, float clip_ratio, StoreFmt fmt, void* codes, float* delta,
                                            cudaStream_t stream);
+
+// Stored composite rotation: u[t][b*beta + i] = sum_j B_b[i][j] * (x (.) diag)[t][perm[b*beta + j]] in binary32,
+// u [rows, K] (pitch K).  beta in {16, 32, 64, 128, 256}; diag may be null.
+cudaError_t launch_composite_rotate(const void* x, fq_dtype xt, int64_t rows, int64_t K, int64_t ldx, const float* diag,
+                                    const int32_t* perm, const float* blocks, int beta, float* u, cudaStream_t stream);
+// *bad_flag (device int) is set to 1 if an entry of perm[K] lies outside [0, K).
+cudaError_t launch_perm_check(const int32_t* perm, int64_t K, int* bad_flag, cudaStream_t stream);
 
 // Builds the weight-operand tensor map of a handle (after `codes` is allocated).
 fq_status build_weight_tmap(Weights& W);

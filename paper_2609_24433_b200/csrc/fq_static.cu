@@ -57,7 +57,7 @@ extern "C" fq_status fq_linear_w4a4_static(const void* x, fq_dtype xt, int64_t M
     using namespace fq;
     const Weights* W = reinterpret_cast<const Weights*>(Wp);
     if (!W || M < 0) return FQ_ERR_INVALID_ARG;
-    if (W->bits != 4) return FQ_ERR_UNSUPPORTED;
+    if (W->bits != 4 || W->composite) return FQ_ERR_UNSUPPORTED;
     if (!(clip_ratio > 0.0f && clip_ratio <= 1.0f)) return FQ_ERR_INVALID_ARG;
     if ((xt != FQ_F32 && xt != FQ_BF16) || (yt != FQ_F32 && yt != FQ_BF16)) return FQ_ERR_INVALID_ARG;
     if (M == 0 || W->N == 0) return FQ_OK;

@@ -26,6 +26,7 @@ EXPORTS = [
     "fq_gemm_acc_i32", "fq_gemm_simt", "fq_device_status", "fq_profile_mark", "fq_linear_w4a4_static",
     "fq_fold_weights_after", "fq_weights_fold_after", "fq_weights_import_after", "fq_quantize_act_after",
     "fq_weights_set_multiplier", "fq_weights_scale_outputs", "fq_linear_w4a16",
+    "fq_fold_weights_composite", "fq_quantize_act_composite", "fq_weights_composite",
 ]
 
 _lib = None
@@ -51,6 +52,8 @@ def lib() -> ctypes.CDLL:
         L.fq_weights_multiplier.argtypes = [ctypes.c_void_p]
         L.fq_weights_fold_after.restype = ctypes.c_int
         L.fq_weights_fold_after.argtypes = [ctypes.c_void_p]
+        L.fq_weights_composite.restype = ctypes.c_int
+        L.fq_weights_composite.argtypes = [ctypes.c_void_p]
         L.fq_workspace_bytes.restype = ctypes.c_size_t
         L.fq_workspace_bytes.argtypes = [ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, ctypes.c_int]
         _lib = L
@@ -166,6 +169,42 @@ def fold_weights_after(W: torch.Tensor, post_scale: torch.Tensor, bias: Optional
                                        ctypes.c_int(hadamard_block), ctypes.c_int(bits), _stream(),
                                        ctypes.byref(out)), "fq_fold_weights_after")
     return Weights(out.value)
+
+
+def fold_weights_composite(W: torch.Tensor, smooth: Optional[torch.Tensor], bias: Optional[torch.Tensor],
+                           perm: torch.Tensor, blocks: torch.Tensor, bits: int) -> Weights:
+    """Fold with a stored composite rotation R = blockdiag(B_b) Pi: rows R (s (.) w_j), RTN, pack.
+    ``perm``: int32[K] source channels; ``blocks``: float32[K/beta, beta, beta]."""
+    W = _rowmajor(W)
+    assert perm.dtype == torch.int32 and blocks.dtype == torch.float32 and blocks.is_contiguous()
+    out = ctypes.c_void_p()
+    _check(lib().fq_fold_weights_composite(_ptr(W), _dt(W), ctypes.c_int64(W.shape[0]), ctypes.c_int64(W.shape[1]),
+                                           ctypes.c_int64(W.stride(0)), _ptr(smooth), _ptr(bias), _ptr(perm), _ptr(blocks),
+                                           ctypes.c_int(blocks.shape[1]), ctypes.c_int(bits), _stream(),
+                                           ctypes.byref(out)), "fq_fold_weights_composite")
+    return Weights(out.value)
+
+
+def quantize_act_composite(x: torch.Tensor, mult_g, perm: torch.Tensor, blocks: torch.Tensor, bits: int,
+                           clip_ratio: float = 1.0, codes: Optional[torch.Tensor] = None,
+                           delta: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None):
+    """Runtime prologue of a composite-rotation site: z = R ((1/s) (.) x), then Eq. 5.  ``mult_g``: device
+    float tensor, a Weights (its multiplier) or None.  ``workspace``: uint8 tensor of at least 4*M*K bytes."""
+    x = _rowmajor(x)
+    M, K = x.shape
+    assert perm.dtype == torch.int32 and blocks.dtype == torch.float32 and blocks.is_contiguous()
+    if codes is None:
+        codes = torch.empty((M, K * bits // 8), dtype=torch.uint8, device=x.device)
+    if delta is None:
+        delta = torch.empty(M, dtype=torch.float32, device=x.device)
+    if workspace is None:
+        workspace = torch.empty(max(16, 4 * M * K), dtype=torch.uint8, device=x.device)
+    g = ctypes.c_void_p(mult_g.multiplier_ptr()) if isinstance(mult_g, Weights) else _ptr(mult_g)
+    _check(lib().fq_quantize_act_composite(_ptr(x), _dt(x), ctypes.c_int64(M), ctypes.c_int64(K), ctypes.c_int64(x.stride(0)),
+                                           g, _ptr(perm), _ptr(blocks), ctypes.c_int(blocks.shape[1]), ctypes.c_int(bits),
+                                           ctypes.c_float(clip_ratio), _ptr(codes), _ptr(delta), _ptr(workspace),
+                                           ctypes.c_size_t(workspace.numel()), _stream()), "fq_quantize_act_composite")
+    return codes, delta
 
 
 def weights_import(codes: torch.Tensor, w_scale: torch.Tensor, mult_g: Optional[torch.Tensor],

@@ -178,3 +178,39 @@ def expert_step_sigma(step: int, steps: int = 10) -> float:
     if steps <= 1:
         return 1.0
     return 1.0 - 0.9 * step / (steps - 1)
+
+
+# ----------------------------------------------------------------------------
+# stored composite rotation: a stand-in for the calibration that produces it
+# ----------------------------------------------------------------------------
+def composite_rotation(K: int, beta: int, seed: int, calib: Optional[np.ndarray] = None):
+    """A permutation and per-block orthogonal matrices shaped like the paper's stored composite
+    rotation: channels ranked by calibrated magnitude are dealt to the blocks in zigzag order
+    (0, 1, .., B-1, B-1, .., 1, 0, 0, 1, ..) so that every block receives a mix of large and small
+    channels, and each block's matrix is a normalised Hadamard matrix applied after the block's
+    principal axes (beta^-1/2 H U^T, U from an SVD of the block's calibration columns).  Without a
+    calibration batch the ranking is random and U is a random orthogonal matrix.
+    Returns (perm int32[K], blocks float32[K/beta, beta, beta])."""
+    rng = np.random.default_rng(seed)
+    nb = K // beta
+    order = np.argsort(-np.abs(calib).max(axis=0), kind="stable") if calib is not None else rng.permutation(K)
+    perm = np.empty(K, dtype=np.int32)
+    fill = np.zeros(nb, dtype=np.int64)
+    for rank, c in enumerate(order):
+        r, pos = divmod(rank, nb)
+        b = pos if r % 2 == 0 else nb - 1 - pos
+        perm[b * beta + fill[b]] = c
+        fill[b] += 1
+    H = np.array([[1.0]])
+    while H.shape[0] < beta:
+        H = np.block([[H, H], [H, -H]])
+    H = H / np.sqrt(beta)
+    blocks = np.empty((nb, beta, beta), dtype=np.float32)
+    for b in range(nb):
+        if calib is not None and calib.shape[0] >= beta:
+            cols = calib[:, perm[b * beta:(b + 1) * beta]].astype(np.float64)
+            U = np.linalg.svd(cols.T @ cols)[0]
+        else:
+            U = np.linalg.qr(rng.standard_normal((beta, beta)))[0]
+        blocks[b] = (H @ U.T).astype(np.float32)
+    return perm, blocks

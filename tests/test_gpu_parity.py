@@ -624,6 +624,69 @@ def test_identity_rotation_linear_end_to_end():
         assert_close(to_np(gpu["y"]), ref["y"], "f32", f"identity rotation W{bits}")
 
 
+# ----------------------------------------------------- stored composite rotation ----
+COMPOSITE_CASES = [
+    # M, K, beta, bits, dtype, smooth, clip
+    (50, 1024, 64, 4, "bf16", True, 1.0),
+    (50, 4096, 64, 4, "bf16", False, 1.0),
+    (7, 96, 32, 8, "f32", True, 0.9),
+    (33, 512, 16, 4, "f32", False, 1.0),
+    (131, 2048, 128, 8, "bf16", True, 1.0),
+    (20, 1024, 256, 4, "f32", True, 0.8),
+    (816, 2048, 64, 4, "bf16", True, 1.0),
+]
+
+
+@pytest.mark.parametrize("M,K,beta,bits,dtype,smooth,clip", COMPOSITE_CASES)
+def test_quantize_act_composite_bit_exact(M, K, beta, bits, dtype, smooth, clip):
+    x = make_x(M, K, dtype, seed=M + K + beta)
+    rng = np.random.default_rng(K + beta)
+    calib = rng.standard_normal((256, K)).astype(np.float32) * np.exp(rng.uniform(-1, 2, K)).astype(np.float32)
+    perm, blocks = synth.composite_rotation(K, beta, seed=3, calib=calib if beta <= 64 else None)
+    g = (1.0 / np.exp(rng.uniform(-2, 2, K))).astype(np.float32) if smooth else None
+    want_codes, want_delta = oracle.composite_quantize(x, dtype, g, perm, blocks, bits, clip)
+    codes, delta = fq.quantize_act_composite(to_dev(x, dtype), to_dev(g), to_dev(perm), to_dev(blocks), bits, clip)
+    assert np.array_equal(to_np(delta).view(np.uint32), want_delta.view(np.uint32))
+    assert np.array_equal(to_np(codes), want_codes)
+
+
+def test_composite_rotation_fold_and_two_call_linear():
+    """Offline fold bit-exact; runtime = fq_quantize_act_composite + fq_gemm_*; the result tracks the float
+    projection as well as the butterfly rotation does (the paper's ablation finds them equivalent)."""
+    site = synth.Site("expert_qkv", 50, 1024, [("qkv", 3072)], beta=64, bits=4, x_dtype="bf16", y_dtype="f32", alpha=0.5)
+    data = synth.make_site(site, seed=11, calib_tokens=256)
+    W, b = concat_consumers(data)
+    s = oracle_smooth(data)
+    perm, blocks = synth.composite_rotation(site.K, site.beta, seed=5, calib=data.calib / s)
+    wc, ws, g = oracle.fold_weights_composite(W, "f32", s, perm, blocks, 4)
+    ac, ad = oracle.composite_quantize(data.x, "bf16", g, perm, blocks, 4, 1.0)
+    want = oracle.epilogue(oracle.gemm_i32(ac, wc, site.K, 4), ad, ws, b, "f32")
+    dperm, dblocks = to_dev(perm), to_dev(blocks)
+    h = fq.fold_weights_composite(to_dev(W), to_dev(s), to_dev(b), dperm, dblocks, 4)
+    hc, hs, hg, _ = h.export()
+    assert np.array_equal(to_np(hc), wc) and np.array_equal(to_np(hs).view(np.uint32), ws.view(np.uint32))
+    assert np.array_equal(to_np(hg).view(np.uint32), g.view(np.uint32))
+    x_dev = to_dev(data.x, "bf16")
+    codes, delta = fq.quantize_act_composite(x_dev, h, dperm, dblocks, 4)
+    assert np.array_equal(to_np(codes), ac) and np.array_equal(to_np(delta).view(np.uint32), ad.view(np.uint32))
+    y = fq.gemm_w4a4(codes, delta, h, torch.float32)
+    assert_close(to_np(y), want, "f32", "composite rotation, two calls")
+    ref = synth.to_f32(data.x, "bf16").astype(np.float64) @ W.astype(np.float64).T + b
+    err_c = np.linalg.norm(to_np(y) - ref) / np.linalg.norm(ref)
+    gpu_b, _ = run_site(data)
+    err_b = np.linalg.norm(to_np(gpu_b["y"]) - ref) / np.linalg.norm(ref)
+    assert err_c < 0.35 and err_c < 1.5 * err_b, (err_c, err_b)
+    # the one-call entry points refuse a composite handle, and a bad permutation is refused at fold time
+    with pytest.raises(fq.FqError) as e:
+        fq.linear_w4a4(x_dev, h)
+    assert e.value.status == fq.ERR_UNSUPPORTED
+    bad = perm.copy()
+    bad[3] = site.K
+    with pytest.raises(fq.FqError) as e:
+        fq.fold_weights_composite(to_dev(W), None, None, to_dev(bad), dblocks, 4)
+    assert e.value.status == fq.ERR_INVALID_ARG
+
+
 def test_error_codes_on_device_arguments():
     x = torch.zeros((8, 1024), dtype=torch.float32, device="cuda")
     W = torch.zeros((16, 1024), dtype=torch.float32, device="cuda")
