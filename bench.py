@@ -8,7 +8,7 @@ one batch: per site the prologue kernel (scale + FWHT + per-token quantization) 
 tcgen05 integer GEMM with its dequant/bias epilogue.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
-                    [--workload backbone_layer|backbone_layer_w4|expert_layer|sweep:M,K,N,block,bits[,after]|w4a16:M,K,N]
+                    [--workload backbone_layer|backbone_layer_w4|expert_layer|sweep:M,K,N,block,bits[,after|composite]|w4a16:M,K,N]
 
 Prints ONE JSON line (rank 0).  ``--impl reference`` times the CPU oracle on host cores.
 """
@@ -120,7 +120,15 @@ class LayerOnDevice:
                 if site.alpha is not None:      # SmoothQuant scale from the calibration batch, on the device
                     a = fq.col_absmax(torch.from_numpy(data.calib).to(device))
                     smooth = fq.smooth_scale(a, fq.col_absmax(W), site.alpha)
-                if site.fold_after:
+                rot = None
+                if site.composite:      # stored rotation: permutation + per-block matrices (synthetic stand-ins)
+                    perm, blocks = synth.composite_rotation(site.K, site.beta, seed + 1000 * r + i)
+                    rot = (torch.from_numpy(perm).to(device), torch.from_numpy(blocks).to(device),
+                           torch.empty(4 * site.M * site.K, dtype=torch.uint8, device=device),
+                           torch.empty((site.M, site.K * site.bits // 8), dtype=torch.uint8, device=device),
+                           torch.empty(site.M, dtype=torch.float32, device=device))
+                    h = fq.fold_weights_composite(W, smooth, b, rot[0], rot[1], site.bits)
+                elif site.fold_after:
                     pscale = torch.from_numpy(synth.post_scale(site, seed + 1000 * r + i)).to(device)
                     h = fq.fold_weights_after(W, pscale, b, site.beta, site.bits)
                 else:
@@ -129,7 +137,7 @@ class LayerOnDevice:
                 y = torch.empty((site.M, site.N_total), dtype=ydt, device=device)
                 ws = torch.empty(fq.workspace_bytes(site.M, site.K, site.N_total, site.bits), dtype=torch.uint8,
                                  device=device)
-                entry.append(dict(x=x, h=h, y=y, ws=ws, host_x=data.x, site=site))
+                entry.append(dict(x=x, h=h, y=y, ws=ws, host_x=data.x, site=site, rot=rot))
                 del W, data
             self.sets.append(entry)
         torch.cuda.synchronize()
@@ -149,10 +157,23 @@ class LayerOnDevice:
                 e0, mark, e1 = events[i]
                 e0.record()
                 fq.profile_mark(mark)
-            fq.linear(e["x"], e["h"], 1.0, y=e["y"], workspace=e["ws"])
+            self.run_site(e, None if events is None else events[i][1])
             if events is not None:
                 fq.profile_mark(None)
                 e1.record()
+
+    def run_site(self, e, mark=None):
+        """Prologue + GEMM of one site: one call, or two for a stored composite rotation."""
+        fq = self.fq
+        if e["rot"] is None:
+            fq.linear(e["x"], e["h"], 1.0, y=e["y"], workspace=e["ws"])
+            return
+        perm, blocks, scratch, codes, delta = e["rot"]
+        fq.quantize_act_composite(e["x"], e["h"], perm, blocks, e["site"].bits, 1.0, codes=codes, delta=delta,
+                                  workspace=scratch)
+        if mark is not None:
+            mark.record()
+        (fq.gemm_w4a4 if e["site"].bits == 4 else fq.gemm_w8a8)(codes, delta, e["h"], y=e["y"], workspace=e["ws"])
 
     def capture(self):
         """One CUDA graph per rotating set (the step's kernels back to back, no host launch gaps),
@@ -347,7 +368,7 @@ def run_e2e(layer, sites, ops, world, K, Wm, dist, device):
                 dst.copy_(hx, non_blocking=True)
                 ev_in[i].record(s_in)
             s_run.wait_event(ev_in[i])
-            layer.fq.linear(e["x"], e["h"], 1.0, y=e["y"], workspace=e["ws"])
+            layer.run_site(e)
             ev_done[i].record(s_run)
             with torch.cuda.stream(s_out):
                 s_out.wait_event(ev_done[i])
@@ -521,16 +542,23 @@ def cpu_baseline(workload: str, steps: int):
         smooth = None
         if site.alpha is not None:
             smooth = oracle.smooth_scale(oracle.col_absmax(data.calib), oracle.col_absmax(W), site.alpha)
-        if site.fold_after:
+        rot = None
+        if site.composite:
+            rot = synth.composite_rotation(site.K, site.beta, 2 + i)
+            wc, ws, g = oracle.fold_weights_composite(W, "f32", smooth, rot[0], rot[1], site.bits)
+        elif site.fold_after:
             wc, ws, g = oracle.fold_weights_after(W, "f32", synth.post_scale(site, 2 + i), site.beta, site.bits)
         else:
             wc, ws, g = oracle.fold_weights(W, "f32", smooth, site.beta, site.bits)      # offline, untimed
-        prepared.append((site, np.ascontiguousarray(data.x[:rows]), g, wc, ws, b))
+        prepared.append((site, np.ascontiguousarray(data.x[:rows]), g, wc, ws, b, rot))
     times = []
     for _ in range(steps):
         t0 = time.perf_counter()
-        for site, x, g, wc, ws, b in prepared:
-            if site.fold_after:
+        for site, x, g, wc, ws, b, rot in prepared:
+            if site.composite:
+                ac, ad = oracle.composite_quantize(x, site.x_dtype, g, rot[0], rot[1], site.bits)
+                oracle.epilogue(oracle.gemm_i32(ac, wc, site.K, site.bits), ad, ws, b, site.y_dtype)
+            elif site.fold_after:
                 ac, ad = oracle.quantize_act_after(x, site.x_dtype, g, site.beta, site.bits)
                 oracle.epilogue(oracle.gemm_i32(ac, wc, site.K, site.bits), ad, ws, b, site.y_dtype)
             else:
@@ -587,7 +615,8 @@ def workload_sites(name: str):
     if name.startswith("sweep:"):        # one site of the throughput sweep: sweep:M,K,N,block,bits[,after]
         f = name[6:].split(",")
         M, K, N, beta, bits = (int(v) for v in f[:5])
-        return [synth.sweep_site(M, K, N, beta, bits, fold_after=len(f) > 5 and f[5] == "after")]
+        return [synth.sweep_site(M, K, N, beta, bits, fold_after=len(f) > 5 and f[5] == "after",
+                                 composite=len(f) > 5 and f[5] == "composite")]
     raise ValueError(name)
 
 
@@ -596,7 +625,8 @@ def workload_name(name: str) -> str:
         f = name[6:].split(",")
         M, K, N, beta, bits = (int(v) for v in f[:5])
         return f"throughput sweep point M={M} K={K} N={N}, block {beta}, W{bits}A{bits}" + \
-               (", fold-after" if len(f) > 5 and f[5] == "after" else "")
+               (", fold-after" if len(f) > 5 and f[5] == "after" else "") + \
+               (", stored composite rotation" if len(f) > 5 and f[5] == "composite" else "")
     return {"backbone_layer": "pi0.5-like backbone layer, M=816, hidden 2048, MLP 16384, o/down W8A8, rest W4A4",
             "backbone_layer_w4": "pi0.5-like backbone layer, M=816, uniform W4A4",
             "expert_layer": "action-expert layer, M=50, width 1024, MLP 4096, W4A4, block 64"}[name]

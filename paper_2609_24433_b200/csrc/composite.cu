@@ -30,15 +30,16 @@ __device__ __forceinline__ float load_as_float<__nv_bfloat16>(const __nv_bfloat1
 }
 
 // BETA in {16, 32, 64, 128, 256}.  Thread (group = tid / BETA, i = tid % BETA) computes output i of
-// R = max(1, BETA / 32) tokens; a CTA covers (256 / BETA) * R tokens of one block.
+// R = 8 tokens (one shared-memory read of the matrix entry and two 16-byte reads of the inputs feed eight
+// multiply-adds); a CTA covers (256 / BETA) * 8 tokens of one block.
 template <typename XT, int BETA>
 __global__ void __launch_bounds__(kThreads)
 composite_rotate_kernel(const XT* __restrict__ x, int64_t rows, int K, int64_t ldx, const float* __restrict__ diag,
                         const int32_t* __restrict__ perm, const float* __restrict__ blocks, float* __restrict__ u) {
     constexpr int G = kThreads / BETA;
-    constexpr int R = BETA >= 32 ? BETA / 32 : 1;
+    constexpr int R = 8;
     constexpr int TOK = G * R;
-    __shared__ float s_p[TOK][BETA];                 // permuted, scaled inputs of the tile
+    __shared__ __align__(16) float s_p[BETA][TOK];   // permuted, scaled inputs of the tile, token-minor
     __shared__ float s_b[kChunkJ][BETA + 1];         // B_b[.][j0 .. j0+31], transposed: s_b[jj][i]
     griddep_wait();
     griddep_launch_dependents();
@@ -55,7 +56,7 @@ composite_rotate_kernel(const XT* __restrict__ x, int64_t rows, int K, int64_t l
             v = load_as_float<XT>(x + (tile0 + tok) * ldx + src);
             if (diag != nullptr) v = __fmul_rn(v, __ldg(diag + src));
         }
-        s_p[tok][j] = v;
+        s_p[j][tok] = v;
     }
     const int grp = tid / BETA, i = tid % BETA;
     float acc[R];
@@ -73,8 +74,12 @@ composite_rotate_kernel(const XT* __restrict__ x, int64_t rows, int K, int64_t l
 #pragma unroll 8
         for (int jj = 0; jj < CJ; ++jj) {
             const float bv = s_b[jj][i];
-#pragma unroll
-            for (int r = 0; r < R; ++r) acc[r] = __fmaf_rn(bv, s_p[grp * R + r][j0 + jj], acc[r]);
+            const float4 pa = *reinterpret_cast<const float4*>(&s_p[j0 + jj][grp * R]);
+            const float4 pb = *reinterpret_cast<const float4*>(&s_p[j0 + jj][grp * R + 4]);
+            acc[0] = __fmaf_rn(bv, pa.x, acc[0]); acc[1] = __fmaf_rn(bv, pa.y, acc[1]);
+            acc[2] = __fmaf_rn(bv, pa.z, acc[2]); acc[3] = __fmaf_rn(bv, pa.w, acc[3]);
+            acc[4] = __fmaf_rn(bv, pb.x, acc[4]); acc[5] = __fmaf_rn(bv, pb.y, acc[5]);
+            acc[6] = __fmaf_rn(bv, pb.z, acc[6]); acc[7] = __fmaf_rn(bv, pb.w, acc[7]);
         }
     }
 #pragma unroll
@@ -87,7 +92,7 @@ composite_rotate_kernel(const XT* __restrict__ x, int64_t rows, int K, int64_t l
 template <typename XT, int BETA>
 cudaError_t launch_beta(const XT* x, int64_t rows, int K, int64_t ldx, const float* diag, const int32_t* perm,
                         const float* blocks, float* u, cudaStream_t stream) {
-    constexpr int TOK = (kThreads / BETA) * (BETA >= 32 ? BETA / 32 : 1);
+    constexpr int TOK = (kThreads / BETA) * 8;
     const int64_t tiles = (rows + TOK - 1) / TOK;
     if (tiles > 65535) return cudaErrorInvalidConfiguration;
     cudaLaunchConfig_t cfg = {};

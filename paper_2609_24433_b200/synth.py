@@ -63,6 +63,7 @@ class Site:
     outlier_gain: float = 30.0
     sigma: float = 1.0
     fold_after: bool = False                  # the site's diagonal sits behind the rotation (T = P^-1 R)
+    composite: bool = False                   # stored composite rotation instead of the butterflies
 
     @property
     def N_total(self) -> int:
@@ -160,10 +161,11 @@ def expert_layer_sites(M: int = 50, width: int = 1024, mlp: int = 4096, sigma: f
     ]
 
 
-def sweep_site(M: int, K: int, N: int, beta: int, bits: int, fold_after: bool = False) -> Site:
-    return Site(f"sweep_m{M}_k{K}_n{N}_b{beta}_w{bits}" + ("_after" if fold_after else ""), M, K, [("proj", N)],
+def sweep_site(M: int, K: int, N: int, beta: int, bits: int, fold_after: bool = False, composite: bool = False) -> Site:
+    tag = "_after" if fold_after else ("_composite" if composite else "")
+    return Site(f"sweep_m{M}_k{K}_n{N}_b{beta}_w{bits}" + tag, M, K, [("proj", N)],
                 beta=beta, bits=bits, alpha=None, outlier_frac=0.005, outlier_kind="scale", outlier_gain=30.0,
-                fold_after=fold_after)
+                fold_after=fold_after, composite=composite)
 
 
 def post_scale(site: Site, seed: int) -> np.ndarray:
