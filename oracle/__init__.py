@@ -283,3 +283,38 @@ def fold_weights_composite(W: np.ndarray, dtype: str, smooth, perm, blocks, bits
     out = composite_quantize(W, dtype, s, perm, blocks, bits, 1.0, return_z=return_wt)
     g = np.ones(K, np.float32) if s is None else (np.float32(1.0) / s).astype(np.float32)
     return (out[0], out[1], g, out[2]) if return_wt else (out[0], out[1], g)
+
+
+def gptq_factor(z: np.ndarray, damp: float = 0.01):
+    """Upper Cholesky factor U of (Z^T Z + lambda I)^-1 (rows of z are transformed calibration tokens) and the
+    dead-channel mask, in binary32 as the device computes them.  Returns (U[K, K], dead[K] bool)."""
+    z = np.ascontiguousarray(z, dtype=np.float32)
+    Mc, K = z.shape
+    U = np.zeros((K, K), dtype=np.float32)
+    dead = np.zeros(K, dtype=np.uint8)
+    _check(_load().fqo_gptq_factor(_p(z), ctypes.c_int64(Mc), ctypes.c_int64(K), ctypes.c_float(damp), _p(U), _p(dead)),
+           "gptq_factor")
+    return U, dead.astype(bool)
+
+
+def gptq_round(wt: np.ndarray, U: np.ndarray, dead: np.ndarray, w_scale: np.ndarray, bits: int = 4) -> np.ndarray:
+    """The GPTQ sweep over the transformed weights W~ [N, K]; returns int codes [N, K]."""
+    w = np.array(wt, dtype=np.float32, order="C", copy=True)
+    N, K = w.shape
+    codes = np.zeros((N, K), dtype=np.int32)
+    _check(_load().fqo_gptq_round(_p(w), ctypes.c_int64(N), ctypes.c_int64(K), _p(np.ascontiguousarray(U, dtype=np.float32)),
+                                  _p(np.ascontiguousarray(dead, dtype=np.uint8)), _p(_f32(w_scale)),
+                                  ctypes.c_int(7 if bits == 4 else 127), _p(codes)), "gptq_round")
+    return codes
+
+
+def fold_weights_gptq(W: np.ndarray, dtype: str, smooth, beta: int, calib: np.ndarray, calib_dtype: str = "f32",
+                      damp: float = 0.01, bits: int = 4, return_all: bool = False):
+    """Offline fold with GPTQ rounding (Eq. 7): W~ = W S R^T, Z = T(calibration tokens), sweep, pack.
+    Per-output-channel steps are those of the RTN fold (max|W~_j| / q).  Returns (codes, w_scale, mult_g)."""
+    _, w_scale, g, wt = fold_weights(W, dtype, smooth, beta, bits, return_wt=True)
+    _, _, z = quantize_act(calib, calib_dtype, g, beta, bits, 1.0, return_z=True)
+    U, dead = gptq_factor(z, damp)
+    q = gptq_round(wt, U, dead, w_scale, bits)
+    out = (pack(q, bits), w_scale, g)
+    return out + (wt, z, U, dead) if return_all else out

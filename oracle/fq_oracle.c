@@ -452,6 +452,96 @@ int fqo_linear_wonly(const void* x, int xdtype, int64_t M, int64_t K, int64_t ld
     return 0;
 }
 
+/* ---- GPTQ rounding in transformed coordinates (section "Rounding and native execution", Eq. 7) ----
+ * min_Q ||(W~ - Q) Z||_F^2 with G = Z Z^T (Z: transformed calibration tokens as columns; here the tokens
+ * are the ROWS of z[Mc][K]) and diagonal damping, solved approximately by the published GPTQ sweep:
+ * channels are rounded one after the other and each rounding error is spread over the channels not yet
+ * rounded, along the rows of the upper Cholesky factor U of H^-1 (H^-1 = U^T U), H = G + lambda I.
+ * All arithmetic is binary32 in a fixed order (fused multiply-add chains in ascending index), because it
+ * decides integer codes: the device path takes the same steps in the same order.
+ *
+ * fqo_gptq_factor:  G[a][b] = sum_t z[t][a] z[t][b];  lambda = damp * mean(diag G);
+ *   a channel with G[a][a] = 0 is dead (never active in calibration): H[a][a] = 1, reported in dead[a];
+ *   H = M M^T with M upper triangular (columns from the last to the first), U = M^-1 (upper triangular),
+ *   so that H^-1 = U^T U.  U is written row-major [K][K] (zeros below the diagonal).  Returns 3 if H is
+ *   not positive definite in binary32. */
+int fqo_gptq_factor(const float* z, int64_t Mc, int64_t K, float damp, float* U, uint8_t* dead) {
+    if (!z || !U || !dead || Mc < 0 || K <= 0 || !(damp >= 0.0f)) return 1;
+    float* H = (float*)malloc(sizeof(float) * (size_t)K * (size_t)K);
+    float* Mu = (float*)malloc(sizeof(float) * (size_t)K * (size_t)K);   /* Mu[i][k], k >= i */
+    if (!H || !Mu) { free(H); free(Mu); return 1; }
+#pragma omp parallel for schedule(static)
+    for (int64_t a = 0; a < K; ++a)
+        for (int64_t b = 0; b < K; ++b) {
+            float acc = 0.0f;
+            for (int64_t t = 0; t < Mc; ++t) acc = fmaf(z[t * K + a], z[t * K + b], acc);
+            H[a * K + b] = acc;
+        }
+    float sum = 0.0f;
+    for (int64_t a = 0; a < K; ++a) sum = sum + H[a * K + a];
+    float lambda = damp * (sum / (float)K);
+    for (int64_t a = 0; a < K; ++a) {
+        dead[a] = H[a * K + a] == 0.0f;
+        if (dead[a]) H[a * K + a] = 1.0f;
+        H[a * K + a] = H[a * K + a] + lambda;
+    }
+    memset(Mu, 0, sizeof(float) * (size_t)K * (size_t)K);
+    int bad = 0;
+    for (int64_t j = K - 1; j >= 0; --j) {
+        float acc = H[j * K + j];
+        for (int64_t k = j + 1; k < K; ++k) acc = fmaf(-Mu[j * K + k], Mu[j * K + k], acc);
+        if (!(acc > 0.0f)) { bad = 1; break; }
+        float d = sqrtf(acc);
+        Mu[j * K + j] = d;
+#pragma omp parallel for schedule(static)
+        for (int64_t i = 0; i < j; ++i) {
+            float a2 = H[i * K + j];
+            for (int64_t k = j + 1; k < K; ++k) a2 = fmaf(-Mu[i * K + k], Mu[j * K + k], a2);
+            Mu[i * K + j] = a2 / d;
+        }
+    }
+    if (!bad) {
+        memset(U, 0, sizeof(float) * (size_t)K * (size_t)K);
+#pragma omp parallel for schedule(dynamic, 8)
+        for (int64_t c = 0; c < K; ++c) {           /* column c of U: M U = I, from row c upwards */
+            U[c * K + c] = 1.0f / Mu[c * K + c];
+            for (int64_t i = c - 1; i >= 0; --i) {
+                float acc = 0.0f;
+                for (int64_t k = i + 1; k <= c; ++k) acc = fmaf(Mu[i * K + k], U[k * K + c], acc);
+                U[i * K + c] = -acc / Mu[i * K + i];
+            }
+        }
+    }
+    free(H);
+    free(Mu);
+    return bad ? 3 : 0;
+}
+
+/* fqo_gptq_round: the sweep.  Wt [N][K] (modified in place), per-output-channel steps w_scale[N] taken
+ * from the unmodified W~ (max|row| / q), codes[N][K] as ints.  For channel i = 0 .. K-1 and every row r:
+ *   w = Wt[r][i] (0 if the channel is dead);  code = clip(rint(w * (1 / s_r)), -q, q);  e = (w - code * s_r) / U[i][i];
+ *   Wt[r][j] = fma(-e, U[i][j], Wt[r][j]) for j > i.        A row with s_r = 0 gets zero codes. */
+int fqo_gptq_round(float* Wt, int64_t N, int64_t K, const float* U, const uint8_t* dead, const float* w_scale,
+                   int q, int* codes) {
+    if (!Wt || !U || !dead || !w_scale || !codes || N < 0 || K <= 0) return 1;
+#pragma omp parallel for schedule(static)
+    for (int64_t r = 0; r < N; ++r) {
+        float s = w_scale[r];
+        float inv = s >= FLT_MIN ? 1.0f / s : 0.0f;
+        float* w = Wt + r * K;
+        for (int64_t i = 0; i < K; ++i) {
+            float wi = dead[i] ? 0.0f : w[i];
+            int v = (int)rintf(wi * inv);
+            if (v > q) v = q;
+            if (v < -q) v = -q;
+            codes[r * K + i] = v;
+            float e = (wi - (float)v * s) / U[i * K + i];
+            for (int64_t j = i + 1; j < K; ++j) w[j] = fmaf(-e, U[i * K + j], w[j]);
+        }
+    }
+    return 0;
+}
+
 /* Whole runtime path for one consumer: prologue, integer product, epilogue.
  * rows_sel (optional, n_sel entries) restricts the integer product and the
  * epilogue to those token rows (output then has n_sel rows); the prologue

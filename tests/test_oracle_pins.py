@@ -652,3 +652,78 @@ def test_composite_rotation_matches_dense_matrices_and_keeps_the_projection():
     inv = np.argsort(perm).astype(np.int32)
     _, _, zbad = oracle.composite_quantize(x, "f32", g, inv, blocks, 8, 1.0, return_z=True)
     assert not np.allclose(zbad.astype(np.float64) @ wt.astype(np.float64).T, want, rtol=1e-2, atol=1e-2)
+
+
+# ------------------------------------- GPTQ rounding in transformed coordinates ----
+def _gptq_inputs(seed, N=24, K=64, Mc=160, beta=32, corr=0.9):
+    """Weights and strongly correlated calibration tokens (GPTQ only differs from RTN when G is not diagonal)."""
+    rng = np.random.default_rng(seed)
+    W = (0.02 * rng.standard_normal((N, K))).astype(np.float32)
+    base = rng.standard_normal((Mc, 8)).astype(np.float32)
+    mix = rng.standard_normal((8, K)).astype(np.float32)
+    calib = (corr * base @ mix + (1 - corr) * rng.standard_normal((Mc, K))).astype(np.float32)
+    return W, calib, beta
+
+
+def test_gptq_factor_is_the_upper_cholesky_factor_of_the_inverse():
+    W, calib, beta = _gptq_inputs(1)
+    _, _, z = oracle.quantize_act(calib, "f32", None, beta, 4, 1.0, return_z=True)
+    U, dead = oracle.gptq_factor(z, damp=0.01)
+    assert not dead.any() and np.allclose(np.tril(U, -1), 0)
+    z64 = z.astype(np.float64)
+    G = z64.T @ z64
+    H = G + 0.01 * np.mean(np.diag(G)) * np.eye(G.shape[0])
+    want = np.linalg.cholesky(np.linalg.inv(H)).T           # unique upper factor with positive diagonal
+    assert np.allclose(U, want, rtol=2e-3, atol=2e-3 * np.abs(want).max())
+    assert np.allclose(U.T.astype(np.float64) @ U.astype(np.float64) @ H, np.eye(H.shape[0]), atol=5e-3)
+
+
+def test_gptq_with_uncorrelated_channels_is_rtn():
+    """A diagonal second moment leaves nothing to compensate: U is diagonal and the sweep is RTN."""
+    rng = np.random.default_rng(2)
+    N, K = 16, 32
+    wt = rng.standard_normal((N, K)).astype(np.float32)
+    z = np.zeros((K, K), np.float32)
+    z[np.arange(K), np.arange(K)] = np.exp2(rng.integers(-2, 3, size=K)).astype(np.float32)   # one token per channel
+    U, dead = oracle.gptq_factor(z, damp=0.0)
+    assert np.count_nonzero(U - np.diag(np.diag(U))) == 0
+    s = (np.abs(wt).max(axis=1) / np.float32(7)).astype(np.float32)
+    codes = oracle.gptq_round(wt, U, dead, s, 4)
+    rtn = np.clip(np.rint(wt * (np.float32(1) / s)[:, None]), -7, 7).astype(np.int32)
+    assert np.array_equal(codes, rtn)
+
+
+def test_gptq_hand_case_two_channels():
+    """K = 2 worked by hand.  z rows (1, 1) and (1, -0.5): G = [[2, 0.5], [0.5, 1.25]], no damping.
+    H = M M^T with M = [[m00, m01], [0, m11]]: m11 = sqrt(1.25), m01 = 0.5 / m11, m00 = sqrt(2 - m01^2);
+    U = M^-1 = [[1/m00, -m01 / (m00 m11)], [0, 1/m11]].  Row w = (0.9, 0.2), step 0.25 (q irrelevant):
+    code0 = rint(3.6) = 4, e = (0.9 - 1.0) / U00 = -0.1 m00; w1 <- 0.2 - e U01 = 0.2 - 0.1 m01 / m11 = 0.2 - 0.04 = 0.16;
+    code1 = rint(0.64) = 1.  RTN would give rint(0.8) = 1 too; with w = (0.9, 0.14): RTN (4, 1), GPTQ (4, 0) since 0.10 / 0.25 = 0.4."""
+    z = np.zeros((2, 32), np.float32)        # pad to 32 channels with dead ones
+    z[0, :2] = [1.0, 1.0]
+    z[1, :2] = [1.0, -0.5]
+    U, dead = oracle.gptq_factor(z, damp=0.0)
+    assert dead[2:].all() and not dead[:2].any()
+    m11 = np.sqrt(1.25); m01 = 0.5 / m11; m00 = np.sqrt(2 - m01 ** 2)
+    assert np.allclose(U[:2, :2], [[1 / m00, -m01 / (m00 * m11)], [0, 1 / m11]], rtol=1e-6)
+    wt = np.zeros((8, 32), np.float32)
+    wt[0, :2] = [0.9, 0.2]
+    wt[1, :2] = [0.9, 0.14]
+    wt[:, 31] = 1.75                             # fixes the row step at 1.75 / 7 = 0.25 (a dead channel: code 0)
+    s = np.full(8, 0.25, np.float32)
+    codes = oracle.gptq_round(wt, U, dead, s, 4)
+    assert list(codes[0, :2]) == [4, 1] and list(codes[1, :2]) == [4, 0]
+    assert not codes[:, 2:].any()               # dead channels get zero codes
+
+
+def test_gptq_lowers_the_objective_of_eq7_against_rtn():
+    W, calib, beta = _gptq_inputs(3)
+    wc, ws, g, wt, z, U, dead = oracle.fold_weights_gptq(W, "f32", None, beta, calib, return_all=True)
+    rtn_codes, ws2, _ = oracle.fold_weights(W, "f32", None, beta, 4)
+    assert np.array_equal(ws, ws2)               # same per-output-channel steps as the RTN fold
+    q_g = oracle.unpack(wc, W.shape[1], 4).astype(np.float64) * ws[:, None]
+    q_r = oracle.unpack(rtn_codes, W.shape[1], 4).astype(np.float64) * ws[:, None]
+    z64, w64 = z.astype(np.float64), wt.astype(np.float64)
+    obj = lambda q: np.linalg.norm((w64 - q) @ z64.T) ** 2
+    assert obj(q_g) < 0.7 * obj(q_r)
+    assert np.abs(oracle.unpack(wc, W.shape[1], 4)).max() <= 7
