@@ -123,6 +123,23 @@ fq_status fq_weights_import_after(const void* codes, const float* w_scale, const
                                   const float* bias, int64_t N, int64_t K, int hadamard_block, int bits,
                                   void* stream, fq_weights** out);
 
+/* ---- offline fold with GPTQ rounding in transformed coordinates (section "Rounding and native execution",
+ * Eq. 7: min_Q ||(W~ - Q) Z||_F^2 with G = Z Z^T and diagonal damping; the paper's rounding at four bits) ------
+ * As fq_fold_weights (fold-before), but the codes come from the GPTQ sweep instead of round-to-nearest:
+ *   calib  device [Mc, K] of dtype ct, leading dimension ldc: calibration tokens of the site in ORIGINAL
+ *          coordinates; they are transformed with the handle's own runtime multiplier, Z = T calib;
+ *   damp   lambda = damp * mean(diag G) is added to the diagonal (0.01 is customary); a channel that is never
+ *          active in calibration (G_cc = 0) gets zero codes;
+ *   the per-output-channel steps are those of the round-to-nearest fold (max|W~_j| / q).
+ * Channels are rounded in index order; each rounding error (w - q s)/U_ii is spread over the channels still to
+ * come along row i of the upper Cholesky factor U of (G + lambda I)^-1.  All of it runs in binary32 in a fixed
+ * order, so the codes are reproducible bit for bit.  K <= 4096 (FQ_ERR_UNSUPPORTED beyond); FQ_ERR_INVALID_ARG if
+ * the damped second moment is not positive definite in binary32.  Offline: allocates (about 3 K^2 + (N + Mc) K
+ * floats of temporaries) and synchronises the stream. */
+fq_status fq_fold_weights_gptq(const void* W, fq_dtype wt, int64_t N, int64_t K, int64_t ldw, const float* smooth,
+                               const float* bias, const void* calib, fq_dtype ct, int64_t Mc, int64_t ldc,
+                               int hadamard_block, int bits, float damp, void* stream, fq_weights** out);
+
 /* ---- stored composite rotation (section "Transforms supported by the runtime": optional for the action
  * expert; the design ablation "butterfly vs. composite rotation") ------------------------------------------
  * R = blockdiag(B_0 .. B_{K/block-1}) Pi: a channel permutation, then one stored dense block x block matrix per

@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libfq_b200.so")
-SOURCES = ["fq_api.cu", "act_quant.cu", "act_quant_ring.cu", "gemm_simt.cu", "gemm_tcgen05.cu", "fq_static.cu", "linear_wonly.cu", "composite.cu"]
+SOURCES = ["fq_api.cu", "act_quant.cu", "act_quant_ring.cu", "gemm_simt.cu", "gemm_tcgen05.cu", "fq_static.cu", "linear_wonly.cu", "composite.cu", "gptq.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
 

@@ -305,6 +305,72 @@ fq_status fq_fold_weights_composite(const void* Wsrc, fq_dtype wt, int64_t N, in
     return FQ_OK;
 }
 
+fq_status fq_fold_weights_gptq(const void* Wsrc, fq_dtype wt, int64_t N, int64_t K, int64_t ldw, const float* smooth,
+                               const float* bias, const void* calib, fq_dtype ct, int64_t Mc, int64_t ldc,
+                               int hadamard_block, int bits, float damp, void* stream, fq_weights** out) {
+    if (!out) return FQ_ERR_INVALID_ARG;
+    *out = nullptr;
+    fq_status st = check_shape(N, K, hadamard_block, bits);
+    if (st != FQ_OK) return st;
+    if (K > 4096) return FQ_ERR_UNSUPPORTED;          // K x K factorisation in shared-nothing column steps
+    if ((wt != FQ_F32 && wt != FQ_BF16) || (ct != FQ_F32 && ct != FQ_BF16)) return FQ_ERR_INVALID_ARG;
+    if (!calib || Mc < 1 || ldc < K || !(damp >= 0.0f)) return FQ_ERR_INVALID_ARG;
+    if (N > 0 && (!Wsrc || ldw < K)) return FQ_ERR_INVALID_ARG;
+    if (N > 0 && (!aligned16(Wsrc) || ldw % 8 != 0)) return FQ_ERR_ALIGNMENT;
+    if ((smooth && !aligned16(smooth)) || (bias && !aligned16(bias))) return FQ_ERR_ALIGNMENT;
+    st = check_arch();
+    if (st != FQ_OK) return st;
+    Weights* w = nullptr;
+    st = alloc_handle(N, K, hadamard_block, bits, &w);
+    if (st != FQ_OK) return st;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t kk = sizeof(float) * (size_t)K * (size_t)K;
+    float *mult_w = nullptr, *Wt = nullptr, *Z = nullptr, *H = nullptr, *Mt = nullptr, *U = nullptr;
+    uint8_t* dead = nullptr;
+    int* bad = nullptr;
+    bool ok = cudaMalloc(&mult_w, sizeof(float) * (size_t)K) == cudaSuccess &&
+              cudaMalloc(&Wt, sizeof(float) * (size_t)(N > 0 ? N : 1) * (size_t)K) == cudaSuccess &&
+              cudaMalloc(&Z, sizeof(float) * (size_t)Mc * (size_t)K) == cudaSuccess &&
+              cudaMalloc(&H, kk) == cudaSuccess && cudaMalloc(&Mt, kk) == cudaSuccess && cudaMalloc(&U, kk) == cudaSuccess &&
+              cudaMalloc(&dead, (size_t)K) == cudaSuccess && cudaMalloc(&bad, sizeof(int)) == cudaSuccess;
+    auto release = [&]() {
+        cudaFree(mult_w); cudaFree(Wt); cudaFree(Z); cudaFree(H); cudaFree(Mt); cudaFree(U); cudaFree(dead); cudaFree(bad);
+    };
+    if (!ok) {
+        release();
+        fq_weights_destroy(reinterpret_cast<fq_weights*>(w));
+        return FQ_ERR_NOMEM;
+    }
+    const float cn = block_norm(hadamard_block);
+    const int qmax = bits == 4 ? 7 : 127;
+    ok = cudaMemsetAsync(bad, 0, sizeof(int), s) == cudaSuccess;
+    ok = ok && launch_multipliers(smooth, K, cn, mult_w, w->mult_g, s) == cudaSuccess;
+    // per-output-channel steps: those of the round-to-nearest fold (its codes are overwritten by the sweep)
+    ok = ok && launch_transform_quantize(Wsrc, wt, N, K, ldw, mult_w, cn, false, hadamard_block, qmax, 1.0f,
+                                         bits == 4 ? StoreFmt::Nibble : StoreFmt::Int8, w->codes, w->w_scale, s) == cudaSuccess;
+    ok = ok && launch_transform_rows(Wsrc, wt, N, K, ldw, mult_w, cn, hadamard_block, Wt, s) == cudaSuccess;
+    ok = ok && launch_transform_rows(calib, ct, Mc, K, ldc, w->mult_g, cn, hadamard_block, Z, s) == cudaSuccess;
+    ok = ok && launch_gptq_factor(Z, Mc, K, damp, H, Mt, U, dead, bad, s) == cudaSuccess;
+    ok = ok && launch_gptq_sweep(Wt, N, K, U, dead, w->w_scale, bits, w->codes, s) == cudaSuccess;
+    if (N > 0) {
+        if (bias)
+            ok = ok && cudaMemcpyAsync(w->bias, bias, sizeof(float) * (size_t)N, cudaMemcpyDeviceToDevice, s) == cudaSuccess;
+        else
+            ok = ok && cudaMemsetAsync(w->bias, 0, sizeof(float) * (size_t)N, s) == cudaSuccess;
+    }
+    int bad_host = 0;
+    ok = ok && cudaMemcpyAsync(&bad_host, bad, sizeof(int), cudaMemcpyDeviceToHost, s) == cudaSuccess;
+    ok = ok && cudaStreamSynchronize(s) == cudaSuccess;   // offline: the temporaries are freed below
+    release();
+    if (ok && !bad_host) ok = build_weight_tmap(*w) == FQ_OK;
+    if (!ok || bad_host) {
+        fq_weights_destroy(reinterpret_cast<fq_weights*>(w));
+        return bad_host ? FQ_ERR_INVALID_ARG : FQ_ERR_CUDA;
+    }
+    *out = reinterpret_cast<fq_weights*>(w);
+    return FQ_OK;
+}
+
 int fq_weights_composite(const fq_weights* wp) {
     const Weights* w = reinterpret_cast<const Weights*>(wp);
     return (w && w->composite) ? 1 : 0;

@@ -140,6 +140,15 @@ cudaError_t launch_composite_rotate(const void* x, fq_dtype xt, int64_t rows, in
 // *bad_flag (device int) is set to 1 if an entry of perm[K] lies outside [0, K).
 cudaError_t launch_perm_check(const int32_t* perm, int64_t K, int* bad_flag, cudaStream_t stream);
 
+// GPTQ rounding (offline): the transform without its quantizer, the damped second moment and the upper factor U
+// of its inverse (H, Mt: K x K scratch; *bad set if not positive definite), and the sweep that writes the codes.
+cudaError_t launch_transform_rows(const void* x, fq_dtype xt, int64_t rows, int64_t K, int64_t ldx, const float* mult,
+                                  float cnorm, int block, float* z, cudaStream_t stream);
+cudaError_t launch_gptq_factor(const float* z, int64_t Mc, int64_t K, float damp, float* H, float* Mt, float* U,
+                               uint8_t* dead, int* bad, cudaStream_t stream);
+cudaError_t launch_gptq_sweep(const float* Wt, int64_t N, int64_t K, const float* U, const uint8_t* dead,
+                              const float* w_scale, int bits, uint8_t* codes, cudaStream_t stream);
+
 // Builds the weight-operand tensor map of a handle (after `codes` is allocated).
 fq_status build_weight_tmap(Weights& W);
 

@@ -26,7 +26,7 @@ EXPORTS = [
     "fq_gemm_acc_i32", "fq_gemm_simt", "fq_device_status", "fq_profile_mark", "fq_linear_w4a4_static",
     "fq_fold_weights_after", "fq_weights_fold_after", "fq_weights_import_after", "fq_quantize_act_after",
     "fq_weights_set_multiplier", "fq_weights_scale_outputs", "fq_linear_w4a16",
-    "fq_fold_weights_composite", "fq_quantize_act_composite", "fq_weights_composite",
+    "fq_fold_weights_composite", "fq_quantize_act_composite", "fq_weights_composite", "fq_fold_weights_gptq",
 ]
 
 _lib = None
@@ -168,6 +168,20 @@ def fold_weights_after(W: torch.Tensor, post_scale: torch.Tensor, bias: Optional
                                        ctypes.c_int64(W.stride(0)), _ptr(post_scale), _ptr(bias),
                                        ctypes.c_int(hadamard_block), ctypes.c_int(bits), _stream(),
                                        ctypes.byref(out)), "fq_fold_weights_after")
+    return Weights(out.value)
+
+
+def fold_weights_gptq(W: torch.Tensor, smooth: Optional[torch.Tensor], bias: Optional[torch.Tensor], calib: torch.Tensor,
+                      hadamard_block: int, bits: int = 4, damp: float = 0.01) -> Weights:
+    """Fold-before with GPTQ rounding in transformed coordinates (Eq. 7); ``calib``: [Mc, K] calibration tokens of
+    the site in original coordinates."""
+    W, calib = _rowmajor(W), _rowmajor(calib)
+    out = ctypes.c_void_p()
+    _check(lib().fq_fold_weights_gptq(_ptr(W), _dt(W), ctypes.c_int64(W.shape[0]), ctypes.c_int64(W.shape[1]),
+                                      ctypes.c_int64(W.stride(0)), _ptr(smooth), _ptr(bias), _ptr(calib), _dt(calib),
+                                      ctypes.c_int64(calib.shape[0]), ctypes.c_int64(calib.stride(0)),
+                                      ctypes.c_int(hadamard_block), ctypes.c_int(bits), ctypes.c_float(damp), _stream(),
+                                      ctypes.byref(out)), "fq_fold_weights_gptq")
     return Weights(out.value)
 
 

@@ -687,6 +687,80 @@ def test_composite_rotation_fold_and_two_call_linear():
     assert e.value.status == fq.ERR_INVALID_ARG
 
 
+# ------------------------------------------- GPTQ rounding in transformed coordinates ----
+def _correlated_calib(rng, Mc, K, rank=16, corr=0.85):
+    base = rng.standard_normal((Mc, rank)).astype(np.float32)
+    mix = rng.standard_normal((rank, K)).astype(np.float32)
+    return (corr * base @ mix + (1 - corr) * rng.standard_normal((Mc, K))).astype(np.float32)
+
+
+GPTQ_CASES = [
+    # N, K, Mc, block, bits, smooth, wdtype, cdtype
+    (24, 64, 160, 32, 4, False, "f32", "f32"),
+    (72, 256, 300, 64, 4, True, "f32", "bf16"),
+    (40, 96, 50, 32, 4, False, "bf16", "f32"),       # fewer tokens than channels: the damping carries the rank deficit
+    (136, 512, 700, 128, 4, True, "f32", "f32"),
+    (16, 128, 200, 1, 8, False, "f32", "f32"),       # identity rotation, 8-bit codes
+]
+
+
+@pytest.mark.parametrize("N,K,Mc,block,bits,smooth,wdtype,cdtype", GPTQ_CASES)
+def test_fold_weights_gptq_bit_exact(N, K, Mc, block, bits, smooth, wdtype, cdtype):
+    rng = np.random.default_rng(N + K + Mc)
+    W = synth.as_dtype(synth.draw_weights(rng, N, K), wdtype)
+    W_f = synth.to_f32(W, wdtype)
+    calib = synth.as_dtype(_correlated_calib(rng, Mc, K), cdtype)
+    if block == 1:
+        calib[:, 5] = 0                                    # a dead channel (no rotation: channel 5 itself never fires)
+    bias = rng.standard_normal(N).astype(np.float32)
+    s = np.exp(rng.uniform(-1, 1, K)).astype(np.float32) if smooth else None
+    wc, ws, g, wt, z, U, dead = oracle.fold_weights_gptq(W, wdtype, s, block, calib, cdtype, 0.01, bits, return_all=True)
+    h = fq.fold_weights_gptq(to_dev(W, wdtype), to_dev(s), to_dev(bias), to_dev(calib, cdtype), block, bits, 0.01)
+    hc, hs, hg, hb = h.export()
+    assert np.array_equal(to_np(hs).view(np.uint32), ws.view(np.uint32))
+    assert np.array_equal(to_np(hg).view(np.uint32), g.view(np.uint32))
+    got, want = oracle.unpack(to_np(hc), K, bits), oracle.unpack(wc, K, bits)
+    assert np.array_equal(got, want), f"{(got != want).sum()} of {got.size} codes differ"
+    if block == 1:
+        assert dead[5] and not got[:, 5].any()
+    # the handle runs like any other, and on the calibration tokens it beats the RTN fold (the objective of Eq. 7)
+    h_rtn = fq.fold_weights(to_dev(W, wdtype), to_dev(s), to_dev(bias), block, bits)
+    rtn = oracle.unpack(to_np(h_rtn.export()[0]), K, bits)
+    z64, w64 = z.astype(np.float64), wt.astype(np.float64)
+    obj = lambda q: np.linalg.norm((w64 - q * ws[:, None].astype(np.float64)) @ z64.T) ** 2
+    assert obj(got) < obj(rtn)
+    x = to_dev(calib[: min(Mc, 64)], cdtype)
+    y = fq.linear(x, h, 1.0, torch.float32)
+    ac, ad = oracle.quantize_act(calib[: min(Mc, 64)], cdtype, g, block, bits)
+    want_y = oracle.epilogue(oracle.gemm_i32(ac, wc, K, bits), ad, ws, bias, "f32")
+    assert_close(to_np(y), want_y, "f32", "gptq handle through the runtime path")
+
+
+def test_fold_weights_gptq_backbone_width_sampled_and_errors():
+    """K = 2048 (the backbone's 4-bit sites): the oracle's factorisation takes seconds, so it runs once and
+    all codes are compared; then the argument checks."""
+    rng = np.random.default_rng(9)
+    N, K, Mc, block = 64, 2048, 1024, 128
+    W = synth.draw_weights(rng, N, K)
+    calib = _correlated_calib(rng, Mc, K, rank=64)
+    wc, ws, g = oracle.fold_weights_gptq(W, "f32", None, block, calib, "f32", 0.01, 4)
+    h = fq.fold_weights_gptq(to_dev(W), None, None, to_dev(calib), block, 4, 0.01)
+    hc, hs, _, _ = h.export()
+    assert np.array_equal(to_np(hs).view(np.uint32), ws.view(np.uint32))
+    assert np.array_equal(to_np(hc), wc)
+    with pytest.raises(fq.FqError) as e:
+        fq.fold_weights_gptq(torch.zeros((8, 8192), device="cuda"), None, None, torch.zeros((4, 8192), device="cuda"), 64, 4)
+    assert e.value.status == fq.ERR_UNSUPPORTED
+    # two channels that always fire together and no damping: the second moment is exactly singular
+    twin = 2.0 * np.eye(32, dtype=np.float32)
+    twin[:, 1] = twin[:, 0]
+    with pytest.raises(fq.FqError) as e:
+        fq.fold_weights_gptq(to_dev(W[:, :32].copy()), None, None, to_dev(twin), 1, 4, 0.0)
+    assert e.value.status == fq.ERR_INVALID_ARG
+    with pytest.raises(RuntimeError):
+        oracle.gptq_factor(twin, 0.0)
+
+
 def test_error_codes_on_device_arguments():
     x = torch.zeros((8, 1024), dtype=torch.float32, device="cuda")
     W = torch.zeros((16, 1024), dtype=torch.float32, device="cuda")
