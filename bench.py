@@ -8,7 +8,7 @@ one batch: per site the prologue kernel (scale + FWHT + per-token quantization) 
 tcgen05 integer GEMM with its dequant/bias epilogue.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
-                    [--workload backbone_layer|backbone_layer_w4|expert_layer|sweep:M,K,N,block,bits[,after|composite]|w4a16:M,K,N]
+                    [--workload backbone_layer|backbone_layer_w4|expert_layer|sweep:M,K,N,block,bits[,after|composite]|w4a16:M,K,N|gptq:N,K,Mc,block]
 
 Prints ONE JSON line (rank 0).  ``--impl reference`` times the CPU oracle on host cores.
 """
@@ -528,6 +528,90 @@ def run_w4a16(args, rank: int, world: int, local_rank: int):
         dist.destroy_process_group()
 
 
+# ------------------------------------------------ GPTQ fold (offline step, its own workload) ----
+def gptq_shape(name: str):
+    N, K, Mc, block = (int(v) for v in name[len("gptq:"):].split(","))
+    return N, K, Mc, block
+
+
+def gptq_inputs(N: int, K: int, Mc: int, seed: int):
+    """Weights and calibration tokens with cross-channel correlation (a rank-32 mixture plus noise): the
+    structure that gives error compensation something to do."""
+    rng = np.random.default_rng(seed)
+    W = synth.draw_weights(rng, N, K)
+    mix = rng.standard_normal((32, K)).astype(np.float32)
+    calib = (0.85 * rng.standard_normal((Mc, 32)).astype(np.float32) @ mix
+             + 0.15 * rng.standard_normal((Mc, K)).astype(np.float32)).astype(np.float32)
+    return W, calib
+
+
+def gptq_flops(N: int, K: int, Mc: int) -> float:
+    # fused multiply-adds x 2: second moment K^2 Mc, factorisation K^3/3, triangular inverse K^3/6, sweep N K^2/2
+    return 2.0 * (K * K * Mc + K ** 3 / 3.0 + K ** 3 / 6.0 + N * K * K / 2.0)
+
+
+def gptq_cpu_baseline(N: int, K: int, Mc: int, block: int, steps: int):
+    import oracle
+    Ks = min(K, 512)                                  # the oracle's factorisation is cubic: a narrower site
+    Ns = min(N, 256)
+    W, calib = gptq_inputs(Ns, Ks, min(Mc, 1024), 2)
+    times = []
+    for _ in range(steps):
+        t0 = time.perf_counter()
+        oracle.fold_weights_gptq(W, "f32", None, min(block, Ks), calib, "f32", 0.01, 4)
+        times.append(time.perf_counter() - t0)
+    dt = statistics.mean(times)
+    return {"value": round(gptq_flops(Ns, Ks, min(Mc, 1024)) / dt / 1e12, 6), "unit": "TFLOP/s", "cores": oracle.num_threads(),
+            "kind": "oracle", "sample": f"a narrower site of the same kind: N={Ns}, K={Ks}, {min(Mc, 1024)} tokens, {dt:.2f} s per fold",
+            "seconds_per_step": round(dt, 3)}
+
+
+def run_gptq(args, rank: int, world: int, local_rank: int):
+    """fq_fold_weights_gptq alone (offline): one fold per step, timed with CUDA events around the call."""
+    import torch
+    from paper_2609_24433_b200 import fq
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    N, K, Mc, block = gptq_shape(args.workload)
+    W, calib = gptq_inputs(N, K, Mc, replicas.replica_seed(2, rank))
+    Wd, cd = torch.from_numpy(W).to(device), torch.from_numpy(calib).to(device)
+    steps, Wm = max(1, min(args.steps, 10)), 3
+    for _ in range(Wm):
+        fq.fold_weights_gptq(Wd, None, None, cd, block, 4, 0.01)
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(local_rank)
+    torch.cuda.synchronize()
+    each = []
+    with sampler:
+        for _ in range(steps):
+            start.record()
+            fq.fold_weights_gptq(Wd, None, None, cd, block, 4, 0.01)      # synchronises its stream (offline call)
+            end.record()
+            torch.cuda.synchronize()
+            each.append(start.elapsed_time(end))
+    # the call allocates, frees and issues ~K launches from the host: the median keeps a busy host out of the figure
+    ms = statistics.median(each)
+    flops = gptq_flops(N, K, Mc)
+    peak = 148 * 128 * 2 * 1.965e9 / 1e12            # binary32 fma lanes x 2 flops x boost clock, TFLOP/s
+    ach = flops / (ms * 1e-3) / 1e12
+    out = {"metric": "GPTQ fold in transformed coordinates (fq_fold_weights_gptq, offline): arithmetic rate", "value": round(ach, 4),
+           "unit": "TFLOP/s", "n_gpus": world, "steps": steps, "warmup": Wm, "ms_per_step": round(ms, 3), "higher_is_better": True,
+           "scaling": "weak", "vs_baseline": None, "dtype": "f32 (fixed-order fma chains), int4 codes", "data": "synthetic",
+           "impl": "ours", "config": {"workload": f"GPTQ fold N={N} K={K}, {Mc} calibration tokens, block {block}, W4",
+                                      "timing": f"median of {steps} folds; min {min(each):.1f} ms, max {max(each):.1f} ms",
+                                      "parallelism": "replicas only"},
+           "clocks": sampler.summary(""), "gpu_launches": steps * (K + 8),
+           "e2e": {"value": round(ach, 4), "unit": "TFLOP/s", "ms_per_step": round(ms, 3), "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 4,
+                   "note": "the call itself is the user-facing API and ends with a host synchronisation; inputs are device tensors"},
+           "roofline": {"bound": "alu", "kernel": "rev_chol_col_kernel x K (column-sequential)", "achieved": round(ach, 4),
+                        "peak": round(peak, 1), "unit": "TFLOP/s", "frac": round(ach / peak, 5), "traffic": None,
+                        "peak_source": "derived: 148 SMs x 128 binary32 lanes x 2 flops x 1.965 GHz"}}
+    if rank == 0:
+        if world == 1 and not args.no_cpu_baseline:
+            out["cpu_baseline"] = gptq_cpu_baseline(N, K, Mc, block, steps=1)
+        print(json.dumps(out), flush=True)
+
+
 # ------------------------------------------------------------------- oracle arm ----
 def cpu_baseline(workload: str, steps: int):
     """The CPU oracle, as it stands, on a bounded sample of the same workload."""
@@ -573,6 +657,17 @@ def cpu_baseline(workload: str, steps: int):
 
 
 def run_reference(args):
+    if args.workload.startswith("gptq:"):
+        N, K, Mc, block = gptq_shape(args.workload)
+        base = gptq_cpu_baseline(N, K, Mc, block, steps=max(1, min(args.steps, 3)))
+        print(json.dumps({"metric": "GPTQ fold in transformed coordinates (fq_fold_weights_gptq, offline): arithmetic rate",
+                          "value": base["value"], "unit": "TFLOP/s", "n_gpus": args.gpus,
+                          "steps": max(1, min(args.steps, 3)), "warmup": 0, "ms_per_step": round(base["seconds_per_step"] * 1e3, 3),
+                          "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+                          "impl": "reference", "config": {"workload": "GPTQ fold, " + base["sample"]}, "cpu_baseline": base,
+                          "e2e": {"value": base["value"], "unit": "TFLOP/s",
+                                  "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}), flush=True)
+        return
     if args.workload.startswith("w4a16:"):
         M, K, N = w4a16_shape(args.workload)
         steps = max(1, min(args.steps, 5))
@@ -650,6 +745,9 @@ def main():
         return
     if args.workload.startswith("w4a16:"):
         run_w4a16(args, rank, world, local_rank)
+        return
+    if args.workload.startswith("gptq:"):
+        run_gptq(args, rank, world, local_rank)
         return
     run_ours(args, rank, world, local_rank)
 

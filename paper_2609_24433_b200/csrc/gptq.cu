@@ -85,17 +85,21 @@ __global__ void damp_kernel(float* __restrict__ H, int K, float damp, uint8_t* _
     }
 }
 
-// Column j of M (H = M M^T, M upper triangular), stored as row j of Mt.  Every CTA recomputes the
-// diagonal entry (one chain of at most K terms) instead of waiting for another CTA to publish it.
+// Column j of M (H = M M^T, M upper triangular), stored as row j of Mt.  Every CTA first copies the
+// finished entries M[j][k], k > j, into shared memory (all threads load, so the strided reads overlap),
+// then recomputes the diagonal entry from them (one chain of at most K terms) instead of waiting for
+// another CTA to publish it; the off-diagonal chains read the same copy.
+constexpr int kMaxK = 4096;
 __global__ void __launch_bounds__(256)
 rev_chol_col_kernel(const float* __restrict__ H, float* __restrict__ Mt, int K, int j, int* __restrict__ bad) {
+    __shared__ float s_mj[kMaxK];                    // s_mj[k - j - 1] = M[j][k]
     __shared__ float s_d;
+    const int n = K - 1 - j;
+    for (int o = threadIdx.x; o < n; o += blockDim.x) s_mj[o] = Mt[(int64_t)(j + 1 + o) * K + j];
+    __syncthreads();
     if (threadIdx.x == 0) {
         float acc = H[(int64_t)j * K + j];
-        for (int k = j + 1; k < K; ++k) {
-            const float m = Mt[(int64_t)k * K + j];
-            acc = __fmaf_rn(-m, m, acc);
-        }
+        for (int o = 0; o < n; ++o) acc = __fmaf_rn(-s_mj[o], s_mj[o], acc);
         if (!(acc > 0.0f)) { *bad = 1; acc = 1.0f; }
         s_d = __fsqrt_rn(acc);
     }
@@ -104,8 +108,27 @@ rev_chol_col_kernel(const float* __restrict__ H, float* __restrict__ Mt, int K, 
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i == j) Mt[(int64_t)j * K + j] = d;
     if (i < j) {
+        // sixteen loads in flight ahead of the (sequential) chain: the loop is bound by their latency otherwise
         float acc = H[(int64_t)i * K + j];
-        for (int k = j + 1; k < K; ++k) acc = __fmaf_rn(-Mt[(int64_t)k * K + i], Mt[(int64_t)k * K + j], acc);
+        const float* col = Mt + (int64_t)(j + 1) * K + i;
+        int o = 0;
+        if (n >= 32) {
+            float cur[32], nxt[32];
+#pragma unroll
+            for (int q = 0; q < 32; ++q) cur[q] = col[(int64_t)q * K];
+            for (; o + 64 <= n; o += 32) {           // the next batch is requested before this one is consumed
+#pragma unroll
+                for (int q = 0; q < 32; ++q) nxt[q] = col[(int64_t)(o + 32 + q) * K];
+#pragma unroll
+                for (int q = 0; q < 32; ++q) acc = __fmaf_rn(-cur[q], s_mj[o + q], acc);
+#pragma unroll
+                for (int q = 0; q < 32; ++q) cur[q] = nxt[q];
+            }
+#pragma unroll
+            for (int q = 0; q < 32; ++q) acc = __fmaf_rn(-cur[q], s_mj[o + q], acc);
+            o += 32;
+        }
+        for (; o < n; ++o) acc = __fmaf_rn(-col[(int64_t)o * K], s_mj[o], acc);
         Mt[(int64_t)j * K + i] = __fdiv_rn(acc, d);
     }
 }
@@ -119,7 +142,15 @@ tri_inverse_kernel(const float* __restrict__ Mt, float* __restrict__ U, int K) {
     U[(int64_t)c * K + c] = __fdiv_rn(1.0f, Mt[(int64_t)c * K + c]);
     for (int i = c - 1; i >= 0; --i) {
         float acc = 0.0f;
-        for (int k = i + 1; k <= c; ++k) acc = __fmaf_rn(Mt[(int64_t)k * K + i], U[(int64_t)k * K + c], acc);
+        int k = i + 1;
+        for (; k + 8 <= c + 1; k += 8) {             // eight pairs of loads in flight ahead of the chain
+            float m[8], u[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) { m[q] = Mt[(int64_t)(k + q) * K + i]; u[q] = U[(int64_t)(k + q) * K + c]; }
+#pragma unroll
+            for (int q = 0; q < 8; ++q) acc = __fmaf_rn(m[q], u[q], acc);
+        }
+        for (; k <= c; ++k) acc = __fmaf_rn(Mt[(int64_t)k * K + i], U[(int64_t)k * K + c], acc);
         U[(int64_t)i * K + c] = __fdiv_rn(-acc, Mt[(int64_t)i * K + i]);
     }
 }
