@@ -81,6 +81,62 @@ def test_argument_checks_run_before_any_device_work(lib):
     assert lib.fq_weights_destroy(null) == fq.OK
 
 
+def test_argument_checks_of_the_widened_entry_points(lib):
+    out = ctypes.c_void_p()
+    null = ctypes.c_void_p(0)
+    i64 = ctypes.c_int64
+    f32 = ctypes.c_float
+    # weight-only projection: a NULL handle, a negative batch
+    assert lib.fq_linear_w4a16(null, 0, i64(1), i64(1024), null, null, 0, i64(8), null) == fq.ERR_INVALID_ARG
+    # block 1 is the identity rotation and a legal block everywhere (NULL data is what is refused here)
+    assert lib.fq_fold_weights(null, 0, i64(8), i64(1024), i64(1024), null, null, 1, 4, null, ctypes.byref(out)) == fq.ERR_INVALID_ARG
+    assert lib.fq_quantize_act(null, 0, i64(0), i64(1024), i64(1024), null, 1, 4, f32(1.0), null, null, null) == fq.OK
+
+    def fold_c(K, block, perm, blocks):
+        return lib.fq_fold_weights_composite(null, 0, i64(8), i64(K), i64(K), null, null, perm, blocks, block, 4, null,
+                                             ctypes.byref(out))
+
+    one = ctypes.c_void_p(16)           # any non-NULL address: the checks below return before it is touched
+    assert fold_c(1024, 8, one, one) == fq.ERR_UNSUPPORTED           # stored blocks below 16 channels
+    assert fold_c(1024, 48, one, one) == fq.ERR_UNSUPPORTED
+    assert fold_c(1024, 64, null, one) == fq.ERR_INVALID_ARG         # no permutation
+    assert fold_c(1024, 64, one, null) == fq.ERR_INVALID_ARG         # no matrices
+
+    def quant_c(M, K, block, ws_bytes):
+        return lib.fq_quantize_act_composite(one, 0, i64(M), i64(K), i64(K), null, one, one, block, 4, f32(1.0), one, one,
+                                             one, ctypes.c_size_t(ws_bytes), null)
+
+    assert quant_c(0, 1024, 64, 0) == fq.OK                          # empty batch
+    assert quant_c(4, 1024, 8, 1 << 20) == fq.ERR_UNSUPPORTED
+    assert quant_c(4, 1024, 64, 4 * 4 * 1024 - 1) == fq.ERR_NOMEM     # scratch for the rotated rows too small
+
+    def gptq(K, Mc, calib, damp):
+        return lib.fq_fold_weights_gptq(one, 0, i64(8), i64(K), i64(K), null, null, calib, 0, i64(Mc), i64(K), 64, 4,
+                                        f32(damp), null, ctypes.byref(out))
+
+    assert gptq(8192, 16, one, 0.01) == fq.ERR_UNSUPPORTED            # K beyond the factorisation's limit
+    assert gptq(1024, 16, null, 0.01) == fq.ERR_INVALID_ARG           # no calibration tokens
+    assert gptq(1024, 0, one, 0.01) == fq.ERR_INVALID_ARG
+    assert gptq(1024, 16, one, -1.0) == fq.ERR_INVALID_ARG
+    assert lib.fq_weights_composite(null) == 0
+
+
+def test_reference_arm_lines_of_the_extra_workloads():
+    """`bench.py --impl reference` runs on the host alone; its JSON line keeps the contract's keys."""
+    import json
+    import subprocess
+    import sys
+    for workload in ("w4a16:1,256,64", "gptq:16,128,64,32"):
+        r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--workload", workload,
+                            "--steps", "1"], capture_output=True, text=True, timeout=300)
+        assert r.returncode == 0, r.stderr[-500:]
+        line = json.loads(r.stdout.strip().splitlines()[-1])
+        for key in ("metric", "value", "unit", "n_gpus", "steps", "warmup", "ms_per_step", "higher_is_better", "scaling",
+                    "vs_baseline", "dtype", "data", "config", "e2e", "cpu_baseline", "impl"):
+            assert key in line, (workload, key)
+        assert line["impl"] == "reference" and line["cpu_baseline"]["kind"] == "oracle" and line["value"] > 0
+
+
 def test_missing_library_fails_loudly(monkeypatch):
     monkeypatch.setattr(fq, "_lib", None)
     monkeypatch.setattr(fq, "LIB_PATH", "/nonexistent/libfq_b200.so")
