@@ -318,3 +318,29 @@ def fold_weights_gptq(W: np.ndarray, dtype: str, smooth, beta: int, calib: np.nd
     q = gptq_round(wt, U, dead, w_scale, bits)
     out = (pack(q, bits), w_scale, g)
     return out + (wt, z, U, dead) if return_all else out
+
+
+SILU, GELU_TANH = 0, 1
+
+
+def gate_act(x, act: int) -> np.ndarray:
+    """act(x) = x * sigmoid(k(x)) in the fixed binary32 arithmetic of the gated product (elementwise)."""
+    lib = _load()
+    lib.fqo_gate_act.restype = ctypes.c_float
+    xs = np.asarray(x, dtype=np.float32).ravel()
+    return np.array([lib.fqo_gate_act(ctypes.c_float(float(v)), ctypes.c_int(act)) for v in xs], dtype=np.float32).reshape(np.shape(x))
+
+
+def gated_product(gate_up: np.ndarray, dtype: str, act: int) -> np.ndarray:
+    """h = act(gate) * up for gate_up [M, 2K] (gate first); binary32 [M, K]."""
+    gu = _mat(gate_up, dtype)
+    M, K2 = gu.shape
+    h = np.zeros((M, K2 // 2), dtype=np.float32)
+    _check(_load().fqo_gated_product(_p(gu), ctypes.c_int(_dt(dtype)), ctypes.c_int64(M), ctypes.c_int64(K2 // 2),
+                                     ctypes.c_int64(K2), ctypes.c_int(act), _p(h)), "gated_product")
+    return h
+
+
+def quantize_act_gated(gate_up: np.ndarray, dtype: str, act: int, g, beta: int, bits: int, clip_ratio: float = 1.0):
+    """Runtime prologue of the site behind a gated MLP: Eq. 5 on T (act(gate) * up)."""
+    return quantize_act(gated_product(gate_up, dtype, act), "f32", g, beta, bits, clip_ratio)

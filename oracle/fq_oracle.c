@@ -452,6 +452,59 @@ int fqo_linear_wonly(const void* x, int xdtype, int64_t M, int64_t K, int64_t ld
     return 0;
 }
 
+/* ---- gated-MLP product ahead of down_proj's quantizer ---------------------------------------------
+ * The site feeding down_proj holds h = act(gate) (.) up (section "Normalization gains" names the gated
+ * MLP and its gate non-linearity without fixing it; the two in use by the policies' language models are
+ * SiLU and the tanh form of GELU).  Both are x * sigmoid(k): k = x for SiLU, k = 2 sqrt(2/pi) (x + 0.044715 x^3)
+ * for GELU-tanh (0.5 (1 + tanh u) = sigmoid(2u)).  Because h feeds a quantizer, its arithmetic is fixed in
+ * binary32 and the device takes the same steps:
+ *   e = exp(-k): argument clamped to [-87, 88]; n = rint(a * log2e); r = fma(n, -ln2_hi, a); r = fma(n, -ln2_lo, r);
+ *       degree-6 Taylor polynomial in Horner form with fused multiply-adds; times 2^n built from its exponent bits;
+ *   act = x / (1 + e);   h = act * up.
+ * gate_up [M][2K]: gate in columns [0, K), up in [K, 2K) (the layout of a fused gate/up projection). */
+static float exp_fixed(float a) {
+    if (a < -87.0f) a = -87.0f;
+    if (a > 88.0f) a = 88.0f;
+    float n = rintf(a * 1.44269504f);
+    float r = fmaf(n, -0.693145752f, a);
+    r = fmaf(n, -1.42860677e-06f, r);
+    float p = 1.38888892e-03f;
+    p = fmaf(p, r, 8.33333377e-03f);
+    p = fmaf(p, r, 4.16666679e-02f);
+    p = fmaf(p, r, 1.66666672e-01f);
+    p = fmaf(p, r, 0.5f);
+    p = fmaf(p, r, 1.0f);
+    p = fmaf(p, r, 1.0f);
+    int32_t bits = ((int32_t)n + 127) << 23;
+    float s;
+    memcpy(&s, &bits, 4);
+    return p * s;
+}
+
+float fqo_gate_act(float x, int act) {
+    float k = x;
+    if (act == 1) {                                  /* GELU, tanh form */
+        float x2 = x * x;
+        float x3 = x2 * x;
+        float inner = fmaf(0.044715f, x3, x);
+        k = 1.59576917f * inner;
+    }
+    float e = exp_fixed(-k);
+    return x / (1.0f + e);
+}
+
+int fqo_gated_product(const void* gate_up, int dtype, int64_t M, int64_t K, int64_t ld, int act, float* h) {
+    if (!gate_up || !h || M < 0 || K <= 0 || ld < 2 * K || (act != 0 && act != 1)) return 1;
+#pragma omp parallel for schedule(static)
+    for (int64_t t = 0; t < M; ++t)
+        for (int64_t c = 0; c < K; ++c) {
+            float g = load_elem(gate_up, dtype, t * ld + c);
+            float u = load_elem(gate_up, dtype, t * ld + K + c);
+            h[t * K + c] = fqo_gate_act(g, act) * u;
+        }
+    return 0;
+}
+
 /* ---- GPTQ rounding in transformed coordinates (section "Rounding and native execution", Eq. 7) ----
  * min_Q ||(W~ - Q) Z||_F^2 with G = Z Z^T (Z: transformed calibration tokens as columns; here the tokens
  * are the ROWS of z[Mc][K]) and diagonal damping, solved approximately by the published GPTQ sweep:

@@ -727,3 +727,41 @@ def test_gptq_lowers_the_objective_of_eq7_against_rtn():
     obj = lambda q: np.linalg.norm((w64 - q) @ z64.T) ** 2
     assert obj(q_g) < 0.7 * obj(q_r)
     assert np.abs(oracle.unpack(wc, W.shape[1], 4)).max() <= 7
+
+
+# ---------------------------------------------- gated-MLP product (SiLU / GELU-tanh) ----
+def test_gate_activations_against_float64_and_special_values():
+    x = np.concatenate([np.linspace(-30, 30, 2001), [-100.0, -88.5, 100.0, 0.0, 1e-6, -1e-6]]).astype(np.float32)
+    x64 = x.astype(np.float64)
+    silu = x64 / (1.0 + np.exp(-x64))
+    gelu = 0.5 * x64 * (1.0 + np.tanh(np.sqrt(2.0 / np.pi) * (x64 + 0.044715 * x64 ** 3)))
+    got_s, got_g = oracle.gate_act(x, oracle.SILU), oracle.gate_act(x, oracle.GELU_TANH)
+    # relative to the magnitude of the result, with an absolute floor in the far negative tail
+    assert np.all(np.abs(got_s - silu) <= 2e-6 * np.abs(silu) + 1e-30 + 1e-6 * np.exp(-np.abs(x64)))
+    assert np.all(np.abs(got_g - gelu) <= 3e-6 * np.abs(gelu) + 1e-30 + 1e-6 * np.exp(-np.abs(x64)))
+    assert oracle.gate_act(0.0, oracle.SILU) == 0.0 and oracle.gate_act(0.0, oracle.GELU_TANH) == 0.0
+    assert oracle.gate_act(50.0, oracle.SILU) == np.float32(50.0)          # sigmoid saturates to 1
+    assert oracle.gate_act(10.0, oracle.GELU_TANH) == np.float32(10.0)
+    assert abs(float(oracle.gate_act(-50.0, oracle.SILU))) < 1e-19       # and to 0
+    assert oracle.gate_act(1.0, oracle.SILU) == pytest.approx(0.7310585786300049, rel=2e-7)
+    assert oracle.gate_act(1.0, oracle.GELU_TANH) == pytest.approx(0.8411919906082768, rel=3e-7)
+
+
+def test_gated_product_layout_and_composition():
+    rng = np.random.default_rng(30)
+    M, K = 3, 64
+    gu = rng.standard_normal((M, 2 * K)).astype(np.float32)
+    h = oracle.gated_product(gu, "f32", oracle.SILU)
+    assert h.shape == (M, K)
+    # gate is the first half, up the second: swapping them changes the result; a unit up branch returns act(gate)
+    assert np.array_equal(h, oracle.gate_act(gu[:, :K], oracle.SILU) * gu[:, K:])
+    ones = gu.copy()
+    ones[:, K:] = 1.0
+    assert np.array_equal(oracle.gated_product(ones, "f32", oracle.GELU_TANH), oracle.gate_act(gu[:, :K], oracle.GELU_TANH))
+    # bf16 inputs are widened exactly; the quantizer then sees the product
+    gb = synth.f32_to_bf16_bits(gu)
+    hb = oracle.gated_product(gb, "bf16", oracle.SILU)
+    assert np.array_equal(hb, oracle.gated_product(synth.bf16_bits_to_f32(gb), "f32", oracle.SILU))
+    c1, d1 = oracle.quantize_act_gated(gb, "bf16", oracle.SILU, None, 32, 4)
+    c2, d2 = oracle.quantize_act(hb, "f32", None, 32, 4)
+    assert np.array_equal(c1, c2) and np.array_equal(d1, d2)
