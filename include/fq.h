@@ -224,6 +224,24 @@ fq_status fq_linear_w8a8(const void* x, fq_dtype xt, int64_t M, int64_t ldx, con
 fq_status fq_linear_w4a16(const void* x, fq_dtype xt, int64_t M, int64_t ldx, const fq_weights* W, void* y,
                           fq_dtype yt, int64_t ldy, void* stream);
 
+/* ---- the site behind a gated MLP: gate product fused into down_proj's prologue -------------------------
+ * (Section "Normalization gains" names the gated MLP and its gate non-linearity; the paper fixes neither the
+ * function nor a fused kernel -- this removes the round trip of the widest activation of a layer through HBM.)
+ * gate_up device [M, 2K] of dtype xt, leading dimension ld >= 2K: gate in columns [0, K), up in [K, 2K), as a fused
+ * gate/up projection writes them.  The quantizer's input is h = act(gate) (.) up, never stored:
+ *   act(x) = x * sigmoid(k),  k = x (FQ_GATE_SILU)  or  k = 2 sqrt(2/pi) (x + 0.044715 x^3) (FQ_GATE_GELU_TANH),
+ * in fixed binary32 arithmetic (the exponential is a range reduction, a degree-6 polynomial in Horner form with
+ * fused multiply-adds and a scaling by exponent bits: h decides integer codes, so the oracle and the device take
+ * the same steps).  Then as fq_quantize_act / fq_linear_* with K = the handle's (intermediate) width.
+ * fq_linear_gated dispatches on the handle's bit width; fold-after handles work, composite ones do not. */
+typedef enum { FQ_GATE_SILU = 0, FQ_GATE_GELU_TANH = 1 } fq_gate_act;
+fq_status fq_quantize_act_gated(const void* gate_up, fq_dtype xt, int64_t M, int64_t K, int64_t ld, fq_gate_act act,
+                                const float* mult_g, int hadamard_block, int bits, float clip_ratio, void* codes_out,
+                                float* delta_out, void* stream);
+fq_status fq_linear_gated(const void* gate_up, fq_dtype xt, int64_t M, int64_t ld, fq_gate_act act, const fq_weights* W,
+                          float clip_ratio, void* y, fq_dtype yt, int64_t ldy, void* workspace, size_t ws_bytes,
+                          void* stream);
+
 /* ---- fused W4A4 linear without a workspace, for callers that cannot allocate ------------------
  * (The paper has no counterpart: this is a deployment convenience of this library.)
  * Same result as fq_linear_w4a4, but the quantized activations and per-token steps that sit

@@ -72,16 +72,45 @@ struct RawRow<__nv_bfloat16, E> {
     }
 };
 
+// Gate non-linearity of a gated MLP in fixed binary32 arithmetic: act(x) = x * sigmoid(k), k = x (SiLU) or
+// k = 2 sqrt(2/pi) (x + 0.044715 x^3) (GELU, tanh form).  exp(-k): argument clamped to [-87, 88], n = rint(a log2e),
+// two-step reduction by ln2, degree-6 Taylor polynomial in Horner form, times 2^n from its exponent bits.  The
+// product act(gate) * up feeds a quantizer, so every operation and its order are part of the definition.
+__device__ __forceinline__ float exp_fixed(float a) {
+    a = fminf(fmaxf(a, -87.0f), 88.0f);
+    const float n = rintf(__fmul_rn(a, 1.44269504f));
+    float r = __fmaf_rn(n, -0.693145752f, a);
+    r = __fmaf_rn(n, -1.42860677e-06f, r);
+    float p = 1.38888892e-03f;
+    p = __fmaf_rn(p, r, 8.33333377e-03f);
+    p = __fmaf_rn(p, r, 4.16666679e-02f);
+    p = __fmaf_rn(p, r, 1.66666672e-01f);
+    p = __fmaf_rn(p, r, 0.5f);
+    p = __fmaf_rn(p, r, 1.0f);
+    p = __fmaf_rn(p, r, 1.0f);
+    return __fmul_rn(p, __int_as_float(((int)n + 127) << 23));
+}
+__device__ __forceinline__ float gate_act(float x, int kind) {
+    float k = x;
+    if (kind == 1) {
+        const float x3 = __fmul_rn(__fmul_rn(x, x), x);
+        k = __fmul_rn(1.59576917f, __fmaf_rn(0.044715f, x3, x));
+    }
+    return __fdiv_rn(x, __fadd_rn(1.0f, exp_fixed(-k)));
+}
+
 // FMT: 0 = two 4-bit codes per byte, 1 = one int8 per code.  CLAMP: clip_ratio < 1.
+// GATED (lean variant only): the row is [gate | up] with 2K columns and the kernel's input is
+// act(gate) * up (the site behind a gated MLP), gate_kind 0 = SiLU, 1 = GELU-tanh.
 // CACHE: keep the multiplier slice in registers across tokens and prefetch the next
 // token (thread blocks of at most 512 threads); otherwise a lean variant for up to
 // 1024 threads that re-reads the multiplier (L1/L2 resident) for every token.
-template <typename XT, int E, int FMT, bool CLAMP, bool CACHE>
+template <typename XT, int E, int FMT, bool CLAMP, bool CACHE, bool GATED = false>
 __global__ void __launch_bounds__(CACHE ? 512 : kMaxThreads)
 transform_quantize_kernel(const XT* __restrict__ x, int64_t rows, int K, int64_t ldx,
                           const float* __restrict__ mult, float cnorm, int block, float qmax,
                           float clip_ratio, uint8_t* __restrict__ codes, float* __restrict__ delta,
-                          int tpr, int rpc, int mult_after) {
+                          int tpr, int rpc, int mult_after, int gate_kind) {
     __shared__ float s_part[2][32];   // per-warp partial maxima, double buffered
 
     griddep_wait();                   // launched with programmatic serialization: see launch_pdl
@@ -129,6 +158,14 @@ transform_quantize_kernel(const XT* __restrict__ x, int64_t rows, int K, int64_t
         } else {
             raw.load(x + row * ldx + col0, row_ok);
             raw.widen(v);
+            if (GATED) {
+                RawRow<XT, E> up;
+                up.load(x + row * ldx + K + col0, row_ok);
+                float u[E];
+                up.widen(u);
+#pragma unroll
+                for (int i = 0; i < E; ++i) v[i] = __fmul_rn(gate_act(v[i], gate_kind), u[i]);
+            }
             if (mult != nullptr && col_ok && !mult_after) {
 #pragma unroll
                 for (int i = 0; i < E / 4; ++i) {
@@ -250,7 +287,7 @@ transform_quantize_kernel(const XT* __restrict__ x, int64_t rows, int K, int64_t
 
 template <typename XT, int E, int FMT>
 cudaError_t launch_e(const XT* x, int64_t rows, int K, int64_t ldx, const float* mult, float cnorm, int mult_after,
-                     int block, int qmax, float clip_ratio, void* codes, float* delta, cudaStream_t stream) {
+                     int block, int qmax, float clip_ratio, void* codes, float* delta, cudaStream_t stream, int gate = -1) {
     const int tpr = ((K / E) + 31) / 32 * 32;
     if (tpr > kMaxThreads) return cudaErrorInvalidConfiguration;
     int rpc = 256 / tpr;
@@ -267,10 +304,13 @@ cudaError_t launch_e(const XT* x, int64_t rows, int K, int64_t ldx, const float*
         int64_t grid = iters < (int64_t)sms * resident ? iters : (int64_t)sms * resident;
         if (grid < 1) grid = 1;
         launch_pdl(kern, (unsigned)grid, (unsigned)threads, 0, stream, 1u, x, rows, K, ldx, mult, cnorm, block, (float)qmax,
-                   clip_ratio, static_cast<uint8_t*>(codes), delta, tpr, rpc, mult_after);
+                   clip_ratio, static_cast<uint8_t*>(codes), delta, tpr, rpc, mult_after, gate);
     };
     const bool clamp = clip_ratio < 1.0f;
-    if (threads <= 512) {
+    if (gate >= 0) {
+        if (clamp) args(transform_quantize_kernel<XT, E, FMT, true, false, true>);
+        else args(transform_quantize_kernel<XT, E, FMT, false, false, true>);
+    } else if (threads <= 512) {
         if (clamp) args(transform_quantize_kernel<XT, E, FMT, true, true>);
         else args(transform_quantize_kernel<XT, E, FMT, false, true>);
     } else {
@@ -282,14 +322,14 @@ cudaError_t launch_e(const XT* x, int64_t rows, int K, int64_t ldx, const float*
 
 template <typename XT, int FMT>
 cudaError_t launch_t(const XT* x, int64_t rows, int K, int64_t ldx, const float* mult, float cnorm, int mult_after,
-                     int block, int qmax, float clip_ratio, void* codes, float* delta, cudaStream_t stream) {
+                     int block, int qmax, float clip_ratio, void* codes, float* delta, cudaStream_t stream, int gate = -1) {
     // E = 8 keeps short rows spread over a full warp; E = 16 is the streaming default;
     // E = 32 holds K = 16384 in 512 threads (cached variant) and reaches K = 32768 in 1024.
     if (K % 16 != 0 || K <= 256)
-        return launch_e<XT, 8, FMT>(x, rows, K, ldx, mult, cnorm, mult_after, block, qmax, clip_ratio, codes, delta, stream);
+        return launch_e<XT, 8, FMT>(x, rows, K, ldx, mult, cnorm, mult_after, block, qmax, clip_ratio, codes, delta, stream, gate);
     if (K <= 8192)
-        return launch_e<XT, 16, FMT>(x, rows, K, ldx, mult, cnorm, mult_after, block, qmax, clip_ratio, codes, delta, stream);
-    return launch_e<XT, 32, FMT>(x, rows, K, ldx, mult, cnorm, mult_after, block, qmax, clip_ratio, codes, delta, stream);
+        return launch_e<XT, 16, FMT>(x, rows, K, ldx, mult, cnorm, mult_after, block, qmax, clip_ratio, codes, delta, stream, gate);
+    return launch_e<XT, 32, FMT>(x, rows, K, ldx, mult, cnorm, mult_after, block, qmax, clip_ratio, codes, delta, stream, gate);
 }
 
 __global__ void multipliers_kernel(const float* __restrict__ smooth, int K, float cnorm,
@@ -389,6 +429,26 @@ cudaError_t launch_transform_quantize(const void* x, fq_dtype xt, int64_t rows, 
     if (fmt == StoreFmt::Nibble) return launch_t<__nv_bfloat16, 0>(p, rows, k, ldx, mult, cnorm, mult_after, block, qmax, clip_ratio, codes, delta, stream);
     if (fmt == StoreFmt::Int8) return launch_t<__nv_bfloat16, 1>(p, rows, k, ldx, mult, cnorm, mult_after, block, qmax, clip_ratio, codes, delta, stream);
     return launch_t<__nv_bfloat16, 2>(p, rows, k, ldx, mult, cnorm, mult_after, block, qmax, clip_ratio, codes, delta, stream);
+}
+
+// The site behind a gated MLP: x is [rows, 2K] = [gate | up], the quantizer's input is act(gate) * up.
+// Always the register kernel's lean variant (the streaming kernel has no gated form).
+cudaError_t launch_gated_transform_quantize(const void* x, fq_dtype xt, int64_t rows, int64_t K, int64_t ldx, int gate_kind,
+                                            const float* mult, float cnorm, bool mult_after_rotation, int block, int qmax,
+                                            float clip_ratio, StoreFmt fmt, void* codes, float* delta, cudaStream_t stream) {
+    if (rows == 0) return cudaSuccess;
+    const int k = (int)K;
+    const int after = mult_after_rotation ? 1 : 0;
+    if (xt == FQ_F32) {
+        const float* p = static_cast<const float*>(x);
+        if (fmt == StoreFmt::Nibble) return launch_t<float, 0>(p, rows, k, ldx, mult, cnorm, after, block, qmax, clip_ratio, codes, delta, stream, gate_kind);
+        if (fmt == StoreFmt::Int8) return launch_t<float, 1>(p, rows, k, ldx, mult, cnorm, after, block, qmax, clip_ratio, codes, delta, stream, gate_kind);
+        return launch_t<float, 2>(p, rows, k, ldx, mult, cnorm, after, block, qmax, clip_ratio, codes, delta, stream, gate_kind);
+    }
+    const __nv_bfloat16* p = static_cast<const __nv_bfloat16*>(x);
+    if (fmt == StoreFmt::Nibble) return launch_t<__nv_bfloat16, 0>(p, rows, k, ldx, mult, cnorm, after, block, qmax, clip_ratio, codes, delta, stream, gate_kind);
+    if (fmt == StoreFmt::Int8) return launch_t<__nv_bfloat16, 1>(p, rows, k, ldx, mult, cnorm, after, block, qmax, clip_ratio, codes, delta, stream, gate_kind);
+    return launch_t<__nv_bfloat16, 2>(p, rows, k, ldx, mult, cnorm, after, block, qmax, clip_ratio, codes, delta, stream, gate_kind);
 }
 
 cudaError_t launch_multipliers(const float* smooth, int64_t K, float cnorm, float* mult_w, float* mult_g,

@@ -128,7 +128,7 @@ fq_status gemm_from_codes(const void* a_codes, const float* a_delta, int64_t M, 
 
 fq_status linear_impl(const void* x, fq_dtype xt, int64_t M, int64_t ldx, const fq_weights* Wp, int bits,
                       float clip_ratio, void* y, fq_dtype yt, int64_t ldy, void* workspace, size_t ws_bytes,
-                      void* stream) {
+                      void* stream, int gate = -1) {
     const Weights* W = reinterpret_cast<const Weights*>(Wp);
     if (!W || M < 0) return FQ_ERR_INVALID_ARG;
     if (W->bits != bits) return FQ_ERR_UNSUPPORTED;
@@ -136,7 +136,7 @@ fq_status linear_impl(const void* x, fq_dtype xt, int64_t M, int64_t ldx, const 
     if (!(clip_ratio > 0.0f && clip_ratio <= 1.0f)) return FQ_ERR_INVALID_ARG;
     if (xt != FQ_F32 && xt != FQ_BF16) return FQ_ERR_INVALID_ARG;
     if (M == 0 || W->N == 0) return FQ_OK;
-    if (!x || ldx < W->K) return FQ_ERR_INVALID_ARG;
+    if (!x || ldx < (gate >= 0 ? 2 * W->K : W->K)) return FQ_ERR_INVALID_ARG;
     if (!aligned16(x) || ldx % 8 != 0) return FQ_ERR_ALIGNMENT;
     if (W->K > kMaxPrologueK) return FQ_ERR_UNSUPPORTED;
     fq_status st = check_y(y, yt, ldy, W->N);
@@ -150,10 +150,13 @@ fq_status linear_impl(const void* x, fq_dtype xt, int64_t M, int64_t ldx, const 
     // Prologue writes one int8 per code into the workspace (4-bit codes stay in [-7, 7] and are laid
     // out in the channel order the GEMM's nibble unpack gives the weights).
     const int qmax = bits == 4 ? 7 : 127;
-    if (launch_transform_quantize(x, xt, M, W->K, ldx, W->mult_g, block_norm(W->block), W->fold_after, W->block, qmax,
-                                  clip_ratio, bits == 4 ? StoreFmt::Int8Perm : StoreFmt::Int8, ws.a8, ws.delta,
-                                  s) != cudaSuccess)
-        return FQ_ERR_CUDA;
+    const StoreFmt fmt = bits == 4 ? StoreFmt::Int8Perm : StoreFmt::Int8;
+    const cudaError_t pe =
+        gate >= 0 ? launch_gated_transform_quantize(x, xt, M, W->K, ldx, gate, W->mult_g, block_norm(W->block), W->fold_after,
+                                                    W->block, qmax, clip_ratio, fmt, ws.a8, ws.delta, s)
+                  : launch_transform_quantize(x, xt, M, W->K, ldx, W->mult_g, block_norm(W->block), W->fold_after, W->block,
+                                              qmax, clip_ratio, fmt, ws.a8, ws.delta, s);
+    if (pe != cudaSuccess) return FQ_ERR_CUDA;
     if (g_profile_mark != nullptr) {
         // Inside a stream capture the mark must be an external event-record node to stay readable.
         cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
@@ -369,6 +372,36 @@ fq_status fq_fold_weights_gptq(const void* Wsrc, fq_dtype wt, int64_t N, int64_t
     }
     *out = reinterpret_cast<fq_weights*>(w);
     return FQ_OK;
+}
+
+fq_status fq_quantize_act_gated(const void* gate_up, fq_dtype xt, int64_t M, int64_t K, int64_t ld, fq_gate_act act,
+                                const float* mult_g, int hadamard_block, int bits, float clip_ratio, void* codes_out,
+                                float* delta_out, void* stream) {
+    if (M < 0 || (bits != 4 && bits != 8)) return FQ_ERR_INVALID_ARG;
+    if (xt != FQ_F32 && xt != FQ_BF16) return FQ_ERR_INVALID_ARG;
+    if (act != FQ_GATE_SILU && act != FQ_GATE_GELU_TANH) return FQ_ERR_INVALID_ARG;
+    if (!(clip_ratio > 0.0f && clip_ratio <= 1.0f)) return FQ_ERR_INVALID_ARG;
+    if (!valid_block(hadamard_block, K) || K % 32 != 0 || K > kMaxPrologueK) return FQ_ERR_UNSUPPORTED;
+    if (M == 0) return FQ_OK;
+    if (!gate_up || !codes_out || !delta_out || ld < 2 * K) return FQ_ERR_INVALID_ARG;
+    if (!aligned16(gate_up) || !aligned16(codes_out) || ld % 8 != 0 || (mult_g && !aligned16(mult_g)))
+        return FQ_ERR_ALIGNMENT;
+    fq_status st = check_arch();
+    if (st != FQ_OK) return st;
+    return launch_gated_transform_quantize(gate_up, xt, M, K, ld, (int)act, mult_g, block_norm(hadamard_block), false,
+                                           hadamard_block, bits == 4 ? 7 : 127, clip_ratio,
+                                           bits == 4 ? StoreFmt::Nibble : StoreFmt::Int8, codes_out, delta_out,
+                                           static_cast<cudaStream_t>(stream)) == cudaSuccess
+               ? FQ_OK : FQ_ERR_CUDA;
+}
+
+fq_status fq_linear_gated(const void* gate_up, fq_dtype xt, int64_t M, int64_t ld, fq_gate_act act, const fq_weights* W,
+                          float clip_ratio, void* y, fq_dtype yt, int64_t ldy, void* workspace, size_t ws_bytes,
+                          void* stream) {
+    const Weights* w = reinterpret_cast<const Weights*>(W);
+    if (!w) return FQ_ERR_INVALID_ARG;
+    if (act != FQ_GATE_SILU && act != FQ_GATE_GELU_TANH) return FQ_ERR_INVALID_ARG;
+    return linear_impl(gate_up, xt, M, ld, W, w->bits, clip_ratio, y, yt, ldy, workspace, ws_bytes, stream, (int)act);
 }
 
 int fq_weights_composite(const fq_weights* wp) {

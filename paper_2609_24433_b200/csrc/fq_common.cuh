@@ -73,6 +73,12 @@ cudaError_t launch_transform_quantize(const void* x, fq_dtype xt, int64_t rows, 
                                       int qmax, float clip_ratio, StoreFmt fmt, void* codes, float* delta,
                                       cudaStream_t stream);
 
+// Same, for the site behind a gated MLP: x is [rows, 2K] = [gate | up] and the input is act(gate) * up
+// (gate_kind 0 = SiLU, 1 = GELU-tanh, fixed binary32 arithmetic).
+cudaError_t launch_gated_transform_quantize(const void* x, fq_dtype xt, int64_t rows, int64_t K, int64_t ldx, int gate_kind,
+                                            const float* mult, float cnorm, bool mult_after_rotation, int block, int qmax,
+                                            float clip_ratio, StoreFmt fmt, void* codes, float* delta, cudaStream_t stream);
+
 // mult_w[c] = s_c * cnorm, mult_g[c] = (1/s_c) * cnorm (smooth == nullptr: both = cnorm).
 cudaError_t launch_multipliers(const float* smooth, int64_t K, float cnorm, float* mult_w, float* mult_g,
                                cudaStream_t stream);

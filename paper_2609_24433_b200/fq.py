@@ -27,6 +27,7 @@ EXPORTS = [
     "fq_fold_weights_after", "fq_weights_fold_after", "fq_weights_import_after", "fq_quantize_act_after",
     "fq_weights_set_multiplier", "fq_weights_scale_outputs", "fq_linear_w4a16",
     "fq_fold_weights_composite", "fq_quantize_act_composite", "fq_weights_composite", "fq_fold_weights_gptq",
+    "fq_quantize_act_gated", "fq_linear_gated",
 ]
 
 _lib = None
@@ -342,6 +343,38 @@ def linear_w4a4_static(x, W: Weights, clip_ratio: float = 1.0, out_dtype=torch.f
     _check(lib().fq_linear_w4a4_static(_ptr(x), _dt(x), ctypes.c_int64(M), ctypes.c_int64(x.stride(0)), W.handle,
                                        ctypes.c_float(clip_ratio), _ptr(y), _out_dt(y.dtype),
                                        ctypes.c_int64(y.stride(0)), _stream()), "fq_linear_w4a4_static")
+    return y
+
+
+GATE_SILU, GATE_GELU_TANH = 0, 1
+
+
+def quantize_act_gated(gate_up: torch.Tensor, act: int, mult_g, hadamard_block: int, bits: int, clip_ratio: float = 1.0):
+    """Prologue of the site behind a gated MLP: Eq. 5 on T (act(gate) * up); gate_up is [M, 2K], gate first."""
+    gate_up = _rowmajor(gate_up)
+    M, K = gate_up.shape[0], gate_up.shape[1] // 2
+    codes = torch.empty((M, K * bits // 8), dtype=torch.uint8, device=gate_up.device)
+    delta = torch.empty(M, dtype=torch.float32, device=gate_up.device)
+    g = ctypes.c_void_p(mult_g.multiplier_ptr()) if isinstance(mult_g, Weights) else _ptr(mult_g)
+    _check(lib().fq_quantize_act_gated(_ptr(gate_up), _dt(gate_up), ctypes.c_int64(M), ctypes.c_int64(K),
+                                       ctypes.c_int64(gate_up.stride(0)), ctypes.c_int(act), g, ctypes.c_int(hadamard_block),
+                                       ctypes.c_int(bits), ctypes.c_float(clip_ratio), _ptr(codes), _ptr(delta), _stream()),
+           "fq_quantize_act_gated")
+    return codes, delta
+
+
+def linear_gated(gate_up: torch.Tensor, act: int, W: Weights, clip_ratio: float = 1.0, out_dtype=torch.float32, y=None,
+                 workspace=None):
+    """down_proj with the gate product fused into its prologue: y = linear(act(gate) * up)."""
+    gate_up = _rowmajor(gate_up)
+    M = gate_up.shape[0]
+    if y is None:
+        y = torch.empty((M, W.N), dtype=out_dtype, device=gate_up.device)
+    ws = _workspace(M, W, workspace, gate_up.device)
+    _check(lib().fq_linear_gated(_ptr(gate_up), _dt(gate_up), ctypes.c_int64(M), ctypes.c_int64(gate_up.stride(0)),
+                                 ctypes.c_int(act), W.handle, ctypes.c_float(clip_ratio), _ptr(y), _out_dt(y.dtype),
+                                 ctypes.c_int64(y.stride(0)), _ptr(ws), ctypes.c_size_t(ws.numel()), _stream()),
+           "fq_linear_gated")
     return y
 
 

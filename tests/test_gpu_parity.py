@@ -761,6 +761,64 @@ def test_fold_weights_gptq_backbone_width_sampled_and_errors():
         oracle.gptq_factor(twin, 0.0)
 
 
+# ------------------------------------------------- gate product fused into the prologue ----
+GATED_CASES = [
+    # M, K, block, bits, dtype, act, smooth, clip
+    (50, 4096, 64, 4, "bf16", oracle.SILU, False, 1.0),
+    (816, 16384, 256, 8, "bf16", oracle.GELU_TANH, False, 1.0),
+    (7, 96, 32, 8, "f32", oracle.SILU, True, 0.9),
+    (300, 2048, 128, 4, "f32", oracle.GELU_TANH, True, 1.0),
+    (33, 512, 1, 4, "bf16", oracle.GELU_TANH, False, 1.0),
+    (131, 8192, 128, 4, "bf16", oracle.SILU, True, 0.8),
+]
+
+
+def _gate_up(rng, M, K, dtype):
+    gu = rng.standard_normal((M, 2 * K)).astype(np.float32)
+    gu[:, :K] *= 3.0                                          # gates reach both saturated ends
+    gu[0, :8] = [0.0, -0.0, 100.0, -100.0, 88.5, -87.5, 1e-6, -1e-6]
+    if M > 1:
+        gu[1] = 0                                             # a zero token
+    return synth.as_dtype(gu, dtype)
+
+
+@pytest.mark.parametrize("M,K,block,bits,dtype,act,smooth,clip", GATED_CASES)
+def test_quantize_act_gated_bit_exact(M, K, block, bits, dtype, act, smooth, clip):
+    rng = np.random.default_rng(M + K + act)
+    gu = _gate_up(rng, M, K, dtype)
+    g = None
+    if smooth:
+        g = ((1.0 / np.exp(rng.uniform(-2, 2, K))) * (1.0 / np.sqrt(block))).astype(np.float32)
+    want_codes, want_delta = oracle.quantize_act_gated(gu, dtype, act, g, block, bits, clip)
+    codes, delta = fq.quantize_act_gated(to_dev(gu, dtype), act, to_dev(g), block, bits, clip)
+    assert np.array_equal(to_np(delta).view(np.uint32), want_delta.view(np.uint32))
+    assert np.array_equal(to_np(codes), want_codes)
+    if M > 1:
+        assert to_np(delta)[1] == 0 and not to_np(codes)[1].any()
+
+
+@pytest.mark.parametrize("bits,act", [(8, oracle.GELU_TANH), (4, oracle.SILU)])
+def test_linear_gated_is_down_proj_on_the_gate_product(bits, act):
+    rng = np.random.default_rng(40 + bits)
+    M, K, N, block = 70, 4096, 1024, 128
+    gu = _gate_up(rng, M, K, "bf16")
+    W = synth.draw_weights(rng, N, K)
+    b = rng.standard_normal(N).astype(np.float32)
+    wc, ws, g = oracle.fold_weights(W, "f32", None, block, bits)
+    ac, ad = oracle.quantize_act_gated(gu, "bf16", act, g, block, bits)
+    want = oracle.epilogue(oracle.gemm_i32(ac, wc, K, bits), ad, ws, b, "bf16")
+    h = fq.fold_weights(to_dev(W), None, to_dev(b), block, bits)
+    y = fq.linear_gated(to_dev(gu, "bf16"), act, h, 1.0, torch.bfloat16)
+    assert_close(to_np(y), want, "bf16", "gated down_proj")
+    # and it is the projection of the float gate product, to quantization accuracy
+    hf = oracle.gated_product(gu, "bf16", act).astype(np.float64)
+    ref = hf @ W.astype(np.float64).T + b
+    assert np.linalg.norm(as_f64(to_np(y)) - ref) / np.linalg.norm(ref) < (0.05 if bits == 8 else 0.35)
+    with pytest.raises(fq.FqError) as e:
+        fq.linear_gated(to_dev(gu, "bf16")[:, :K].contiguous(), act, h)  # only K columns: no up branch
+    assert e.value.status == fq.ERR_INVALID_ARG
+
+
 def test_error_codes_on_device_arguments():
     x = torch.zeros((8, 1024), dtype=torch.float32, device="cuda")
     W = torch.zeros((16, 1024), dtype=torch.float32, device="cuda")
