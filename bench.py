@@ -8,7 +8,7 @@ one batch: per site the prologue kernel (scale + FWHT + per-token quantization) 
 tcgen05 integer GEMM with its dequant/bias epilogue.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
-                    [--workload backbone_layer|backbone_layer_w4|expert_layer|sweep:M,K,N,block,bits[,after|composite]|w4a16:M,K,N|gptq:N,K,Mc,block]
+                    [--workload backbone_layer|backbone_layer_w4|backbone_forward|backbone_forward_w4|expert_layer|expert_loop|sweep:M,K,N,block,bits[,after|composite]|w4a16:M,K,N|gptq:N,K,Mc,block]
 
 Prints ONE JSON line (rank 0).  ``--impl reference`` times the CPU oracle on host cores.
 """
@@ -111,7 +111,16 @@ class LayerOnDevice:
         self.sets = []
         for r in range(ROTATE):
             entry = []
+            shared = {}          # expert loop: the 18 layers' handles serve all 10 denoising steps
             for i, site in enumerate(sites):
+                wkey = site.name.split(".", 1)[1] if site.name.startswith("S") and "." in site.name else None
+                if wkey is not None and wkey in shared:
+                    # same weights as step 0 of this layer; only the activations (their scale drifts) are new
+                    h0, y0, ws0 = shared[wkey]
+                    data = synth.make_site(site, seed + 1000 * r + i, with_weights=False)
+                    x = self._dev(data.x, site.x_dtype, device)
+                    entry.append(dict(x=x, h=h0, y=y0, ws=ws0, host_x=data.x, site=site, rot=None))
+                    continue
                 data = synth.make_site(site, seed + 1000 * r + i)
                 x = self._dev(data.x, site.x_dtype, device)
                 W = torch.from_numpy(np.concatenate([data.W[n] for n, _ in site.consumers], 0)).to(device)
@@ -138,6 +147,8 @@ class LayerOnDevice:
                 ws = torch.empty(fq.workspace_bytes(site.M, site.K, site.N_total, site.bits), dtype=torch.uint8,
                                  device=device)
                 entry.append(dict(x=x, h=h, y=y, ws=ws, host_x=data.x, site=site, rot=rot))
+                if wkey is not None:
+                    shared[wkey] = (h, y, ws)
                 del W, data
             self.sets.append(entry)
         torch.cuda.synchronize()
@@ -240,6 +251,10 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         dist = dist_mod
         dist.init_process_group("nccl", device_id=device)
 
+    global ROTATE, CPU_SAMPLE_ROWS
+    if args.workload in ("backbone_forward", "backbone_forward_w4", "expert_loop"):
+        ROTATE = 1              # a step already walks far more weight bytes than L2 holds
+        CPU_SAMPLE_ROWS = 32    # keeps the oracle arm's sample to tens of seconds
     sites = workload_sites(args.workload)
     layer = LayerOnDevice(sites, seed=replicas.replica_seed(2, rank), device=device)
     ops = layer_ops(sites)
@@ -306,7 +321,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
                 "traffic": TRAFFIC_BYTES.get((args.workload, s.name)),
                 "event_node_overhead_us": round(ev_overhead_ms * 1e3, 2),
                 "per_site_us": {sites[i].name: {"prologue": round(act_ms[i] * 1e3, 2), "gemm": round(gemm_ms[i] * 1e3, 2)}
-                                for i in range(len(sites))}}
+                                for i in range(min(len(sites), 8))}}
     act_i = max(range(len(sites)), key=lambda i: act_ms[i])
     sa = sites[act_i]
     act_bytes = sa.M * sa.K * (2 if sa.x_dtype == "bf16" else 4) + sa.M * sa.K + 4 * sa.M
@@ -324,8 +339,8 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int8/int4 codes, int32 accumulate, f32 transform",
         "data": "synthetic", "impl": "ours",
         "config": {"workload": workload_name(args.workload), "M": sites[0].M,
-                   "sites": {s.name: {"K": s.K, "N": s.N_total, "bits": s.bits, "block": s.beta} for s in sites},
-                   "ops_per_step": ops, "parallelism": "replicas only (one batch per GPU, no collective)",
+                   "sites": {s.name: {"K": s.K, "N": s.N_total, "bits": s.bits, "block": s.beta} for s in sites[:8]},
+                   "n_sites": len(sites), "ops_per_step": ops, "parallelism": "replicas only (one batch per GPU, no collective)",
                    "l2": f"{ROTATE} rotating weight+activation sets (> 126 MB L2 in total), no flush kernel",
                    "launch": "one CUDA-graph replay per step"},
         "clocks": sampler.summary(note), "e2e": e2e, "gpu_launches": layer.launches_per_step * K,
@@ -657,6 +672,9 @@ def cpu_baseline(workload: str, steps: int):
 
 
 def run_reference(args):
+    global CPU_SAMPLE_ROWS
+    if args.workload in ("backbone_forward", "backbone_forward_w4", "expert_loop"):
+        CPU_SAMPLE_ROWS = 32
     if args.workload.startswith("gptq:"):
         N, K, Mc, block = gptq_shape(args.workload)
         base = gptq_cpu_baseline(N, K, Mc, block, steps=max(1, min(args.steps, 3)))
@@ -689,7 +707,8 @@ def run_reference(args):
            "scaling": "weak", "vs_baseline": None, "dtype": "int8/int4 codes, int32 accumulate, f32 transform",
            "data": "synthetic", "impl": "reference",
            "config": {"workload": workload_name(args.workload), "M": sites[0].M,
-                      "sites": {s.name: {"K": s.K, "N": s.N_total, "bits": s.bits, "block": s.beta} for s in sites}},
+                      "sites": {s.name: {"K": s.K, "N": s.N_total, "bits": s.bits, "block": s.beta} for s in sites[:8]},
+                      "n_sites": len(sites)},
            "cpu_baseline": base,
            "e2e": {"value": base["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(out), flush=True)
@@ -707,6 +726,15 @@ def workload_sites(name: str):
         return synth.backbone_layer_sites(selective_int8=False)
     if name == "expert_layer":
         return synth.expert_layer_sites()
+    if name in ("backbone_forward", "backbone_forward_w4"):   # 18 layers with distinct weights: one forward per step
+        import dataclasses
+        return [dataclasses.replace(s, name=f"L{layer:02d}.{s.name}")
+                for layer in range(18) for s in synth.backbone_layer_sites(selective_int8=name == "backbone_forward")]
+    if name == "expert_loop":                                  # 18 layers x 10 denoising steps, activation scale drifting
+        import dataclasses
+        return [dataclasses.replace(s, name=f"S{step}.L{layer:02d}.{s.name}")
+                for step in range(10) for layer in range(18)
+                for s in synth.expert_layer_sites(sigma=synth.expert_step_sigma(step))]
     if name.startswith("sweep:"):        # one site of the throughput sweep: sweep:M,K,N,block,bits[,after]
         f = name[6:].split(",")
         M, K, N, beta, bits = (int(v) for v in f[:5])
@@ -722,7 +750,11 @@ def workload_name(name: str) -> str:
         return f"throughput sweep point M={M} K={K} N={N}, block {beta}, W{bits}A{bits}" + \
                (", fold-after" if len(f) > 5 and f[5] == "after" else "") + \
                (", stored composite rotation" if len(f) > 5 and f[5] == "composite" else "")
-    return {"backbone_layer": "pi0.5-like backbone layer, M=816, hidden 2048, MLP 16384, o/down W8A8, rest W4A4",
+    return {"backbone_forward": "18-layer pi0.5-like backbone forward (distinct weights per layer), M=816, o/down W8A8, rest W4A4",
+            "backbone_forward_w4": "18-layer pi0.5-like backbone forward (distinct weights per layer), M=816, uniform W4A4",
+            "expert_loop": "action-expert denoising loop: 10 steps x 18 layers (one set of layer weights serves all steps), M=50, "
+                           "width 1024, MLP 4096, W4A4, block 64, activation scale drifting 1.0 -> 0.1",
+            "backbone_layer": "pi0.5-like backbone layer, M=816, hidden 2048, MLP 16384, o/down W8A8, rest W4A4",
             "backbone_layer_w4": "pi0.5-like backbone layer, M=816, uniform W4A4",
             "expert_layer": "action-expert layer, M=50, width 1024, MLP 4096, W4A4, block 64"}[name]
 
