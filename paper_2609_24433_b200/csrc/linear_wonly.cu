@@ -1,8 +1,8 @@
 // Short-batch weight streaming for 4-bit weights: the projection of a handful of tokens is a
 // matrix-vector product bound by the weight bytes, which must cross HBM once.  Two users:
-//   * the W4A4 integer product of Eq. 8 for batches of at most 32 tokens (the iterative action expert,
-//     the short end of the throughput sweep), where the TMA/TMEM pipeline of the big GEMM cannot be fed
-//     at HBM rate by so thin a tile;
+//   * the W4A4 integer product of Eq. 8 for batches of at most 16 tokens on matrices of up to 32 Mi weights
+//     (the short end of the throughput sweep), where it measured faster than the TMA/TMEM pipeline of the
+//     big GEMM, whose per-k-block hand-overs cannot be fed at HBM rate by so thin a tile;
 //   * the weight-only projection with floating-point activations (the adaptive layer-normalisation
 //     modulation of the W4A4 engines):  y[t][j] = s^W_j * sum_c qW[j][c] * x[t][c] + b_j.
 // One persistent CTA per SM walks groups of 32 weight rows.  A producer warp streams the packed rows
