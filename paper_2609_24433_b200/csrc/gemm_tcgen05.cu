@@ -414,7 +414,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             int kb0 = kb0_of(unit);
             bool peek = false;
             for (int n = 0; n < total_kb; ++n) {
-                ok = mbar_wait_all(smem_u32(&s_empty[stage]), phase ^ 1u, abort_flag, p.watchdog, kWdProducer, peek);
+                ok = mbar_wait_all_lazy(smem_u32(&s_empty[stage]), phase ^ 1u, abort_flag, p.watchdog, kWdProducer, peek);
                 if (!ok) break;
                 FQ_TRACE(0, n, 0);
                 {   // look at the next stage now: the test's latency hides behind the copy issued below
@@ -705,7 +705,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             int kb0 = kb0_of(unit);
             bool peek = false;
             for (int n = 0; n < total_kb; ++n) {
-                ok = mbar_wait_all(smem_u32(&s_empty[stage]), phase ^ 1u, abort_flag, p.watchdog, kWdProducer, peek);
+                ok = mbar_wait_all_lazy(smem_u32(&s_empty[stage]), phase ^ 1u, abort_flag, p.watchdog, kWdProducer, peek);
                 if (!ok) break;
                 {
                     const int s1 = stage + 1 == p.stages ? 0 : stage + 1;
@@ -817,7 +817,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             int kb0 = kb0_of(unit);
             bool peek = false;
             for (int n = 0; n < total_kb; ++n) {
-                ok = mbar_wait_all(smem_u32(&s_empty_p[ps]), pph ^ 1u, abort_flag, p.watchdog, kWdProducer, peek);
+                ok = mbar_wait_all_lazy(smem_u32(&s_empty_p[ps]), pph ^ 1u, abort_flag, p.watchdog, kWdProducer, peek);
                 if (!ok) break;
                 {
                     const int s1 = ps + 1 == p.stages_p ? 0 : ps + 1;

@@ -113,6 +113,29 @@ __device__ __forceinline__ bool mbar_wait_all(uint32_t bar, uint32_t parity, vol
     const bool ok = mbar_wait(bar, parity, abort_flag, watchdog, code);
     return __all_sync(0xffffffffu, ok);
 }
+// Converged wait for roles that run far ahead of their consumer (TMA producers behind a full ring): between
+// tries the warp sleeps, so that it does not take issue slots from the warps on the critical path.
+__device__ __forceinline__ bool mbar_wait_all_lazy(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                                   uint32_t* watchdog, uint32_t code, bool peeked = false) {
+    if (__all_sync(0xffffffffu, peeked)) return true;
+    bool ok = true;
+    if (!mbar_try_wait(bar, parity)) {
+        const uint64_t t0 = global_timer_ns();
+        for (uint32_t spin = 1; !mbar_try_wait(bar, parity); ++spin) {
+            __nanosleep(100);
+            if ((spin & 0x3ff) == 0) {
+                if (*abort_flag) { ok = false; break; }
+                if (global_timer_ns() - t0 > kWaitLimitNs) {
+                    *abort_flag = 1;
+                    atomicOr(watchdog, code);
+                    ok = false;
+                    break;
+                }
+            }
+        }
+    }
+    return __all_sync(0xffffffffu, ok);
+}
 // Wait for latency-tolerant roles (epilogue): lane 0 polls with a short sleep between tries so that
 // an idle warp does not compete for issue slots with the warps feeding the tensor core.
 __device__ __forceinline__ bool mbar_wait_warp_relaxed(uint32_t bar, uint32_t parity, volatile int* abort_flag,
