@@ -536,6 +536,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                 sw = __ldg(p.w_scale + j) * unshift;     // (float)acc * 2^-shift is exact: fold the shift here
                 bj = __ldg(p.bias + j);
             }
+            // a tile takes at least ~0.2 us per k-block: sleep through a quarter of that before the first look,
+            // so that eight idle warps do not spend issue slots polling while a long tile is being accumulated
+            if (k_blocks >= 32) __nanosleep(k_blocks >= 400 ? 20000u : (unsigned)k_blocks * 50u);
             ok = mbar_wait_warp_relaxed(smem_u32(&s_acc_full[acc_stage]), acc_phase, abort_flag, p.watchdog, kWdEpilogue);
             if (!ok) break;
             // K split.  Every slice writes its raw int32 sums to its own block of scratch
