@@ -261,6 +261,11 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
           "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
         : "memory");
 }
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
+    return v;
+}
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* r) {
     asm volatile(
@@ -743,15 +748,18 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         const int row = (warp & 3) * 32 + lane;
         const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
         const int swz = (row >> 1) & 3;
+        uint32_t row_off[4];                             // this lane's four 16-byte chunks inside a packed stage
+#pragma unroll
+        for (int c = 0; c < 4; ++c) row_off[c] = (uint32_t)(row * 64 + ((c ^ swz) << 4));
         // Set `uset` takes the k-blocks whose running index n is congruent to it modulo kUnpackSets,
         // so two k-blocks are in flight per quadrant and one set's store latency hides behind the other.
         const int uset = (warp - kFirstUnpackWarp) >> 2;
         const int total_kb = my_units * k_blocks;
         bool ok = true;
         int ps = uset, ws = uset;                        // ring slots of k-block n, kept incrementally
-        uint32_t pph = 0, wph = 0;
+        uint32_t pph = 0;
         while (ps >= p.stages_p) { ps -= p.stages_p; pph ^= 1u; }
-        while (ws >= p.stages_w) { ws -= p.stages_w; wph ^= 1u; }
+        while (ws >= p.stages_w) ws -= p.stages_w;
         // TMEM slot ws is free once the MMAs of k-block m = n - stages_w have retired, which is the
         // same event that frees that k-block's activation stage: barrier s_empty[m % stages], use
         // number m / stages (stages_w <= stages, so the barrier cannot run a phase ahead of this wait).
@@ -765,10 +773,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                 ok = mbar_wait_all(smem_u32(&s_full_p[ps]), pph, abort_flag, p.watchdog, kWdUnpackFull);
                 if (!ok) break;
                 if ((warp & 3) == 0) FQ_TRACE(2, n, 1);
-                const uint8_t* src = gen_base + (smem_p - base) + ps * pk_bytes + row * 64;
+                const uint32_t src = smem_p + (uint32_t)ps * pk_bytes;     // shared-space address of the stage
                 uint4 pk[4];
 #pragma unroll
-                for (int c = 0; c < 4; ++c) pk[c] = *reinterpret_cast<const uint4*>(src + ((c ^ swz) << 4));
+                for (int c = 0; c < 4; ++c) pk[c] = lds128(src + row_off[c]);
                 // is the TMEM slot free?  (tested now, needed only after the expansion below)
                 const bool slot_free = m < 0 || mbar_test_wait(smem_u32(&s_empty[es]), eph);
                 __syncwarp();
@@ -799,14 +807,15 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                     else mbar_arrive_cta(smem_u32(&s_full_w8[ws]), 0);
                 }
                 if ((warp & 3) == 0) FQ_TRACE(2, n, 3);
+                // (every ring has at least kUnpackSets slots: one subtraction brings an index back into range)
                 ps += kUnpackSets;
-                while (ps >= p.stages_p) { ps -= p.stages_p; pph ^= 1u; }
+                if (ps >= p.stages_p) { ps -= p.stages_p; pph ^= 1u; }
                 ws += kUnpackSets;
-                while (ws >= p.stages_w) { ws -= p.stages_w; wph ^= 1u; }
+                if (ws >= p.stages_w) ws -= p.stages_w;
                 m += kUnpackSets;
                 if (m >= kUnpackSets) es += kUnpackSets;
                 else if (m >= 0) es = m;
-                while (es >= p.stages) { es -= p.stages; eph ^= 1u; }
+                if (es >= p.stages) { es -= p.stages; eph ^= 1u; }
             }
         }
     } else if (BITS == 4) {
