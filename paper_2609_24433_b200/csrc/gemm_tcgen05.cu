@@ -578,7 +578,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                     *last_slot = done == (uint32_t)(split - 1) ? 1 : 0;
                     if (*last_slot) p.counters[tile] = 0u;   // every slice has been counted: ready for the next launch
                 }
-                // rendezvous 2: the verdict is written (its slot is reused two tiles later, after both
+                // rendezvous 2: the outcome is written (its slot is reused two tiles later, after both
                 // rendezvous of the next tile)
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&s_epi_sync));

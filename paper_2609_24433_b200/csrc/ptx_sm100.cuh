@@ -101,7 +101,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     if (mbar_try_wait(bar, parity)) return true;
     return mbar_wait_slow(bar, parity, abort_flag, watchdog, code);
 }
-// Warp-converged wait: every lane polls the same barrier, the verdict is made warp-uniform.
+// Warp-converged wait: every lane polls the same barrier, the result is made warp-uniform.
 // Roles that hand work over through barriers run their loops with the whole warp converged and
 // elect a lane only for the issue itself: a lone lane looping while its warp-mates are parked at a
 // CTA barrier was measured 2-3x slower per dependent wait/arrive pair.
