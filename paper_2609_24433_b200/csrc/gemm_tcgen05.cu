@@ -261,6 +261,25 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
           "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
         : "memory");
 }
+// Four TS-form MMAs (one K = 128 atom) from the lane elect.sync picks; no commit: the stage's last atom,
+// issued by issue_kblock_ts right after, commits for both.
+__device__ __forceinline__ void issue_mmas_ts(uint32_t d_tmem, const uint32_t* a, const uint64_t* b, uint32_t idesc,
+                                              uint32_t accumulate) {
+    asm volatile(
+        "{\n\t"
+        ".reg .pred pl, pacc, pt;\n\t"
+        "elect.sync _|pl, 0xffffffff;\n\t"
+        "setp.ne.b32 pacc, %10, 0;\n\t"
+        "setp.eq.b32 pt, %0, %0;\n\t"
+        "@pl tcgen05.mma.cta_group::1.kind::i8 [%0], [%1], %5, %9, pacc;\n\t"
+        "@pl tcgen05.mma.cta_group::1.kind::i8 [%0], [%2], %6, %9, pt;\n\t"
+        "@pl tcgen05.mma.cta_group::1.kind::i8 [%0], [%3], %7, %9, pt;\n\t"
+        "@pl tcgen05.mma.cta_group::1.kind::i8 [%0], [%4], %8, %9, pt;\n\t"
+        "}"
+        ::"r"(d_tmem), "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "l"(b[0]), "l"(b[1]), "l"(b[2]), "l"(b[3]), "r"(idesc),
+          "r"(accumulate)
+        : "memory");
+}
 __device__ __forceinline__ uint4 lds128(uint32_t addr) {
     uint4 v;
     asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
@@ -309,7 +328,11 @@ enum : uint32_t {
 // each loads its own 128 weight rows and HALF of the token tile, the even CTA issues the MMAs for
 // both, and every MMA reads the token halves out of both CTAs' shared memory.  This halves the
 // activation bytes each SM pulls from L2, which is what bounds the single-CTA kernel.
-template <int BITS, int CTAS, bool SPLIT>
+// ATOMS (4-bit weights, single CTAs, token tiles of at most 128): a pipeline stage holds ATOMS k-blocks of 128
+// channels (two 128-byte swizzle atoms side by side).  The kernel is bound by instruction issue, and the waits,
+// arrivals, fences and ring arithmetic of every role are paid per stage: twice the channels per stage take a
+// third off the instructions per channel.  (Longer token tiles have no TMEM left for slots twice as wide.)
+template <int BITS, int CTAS, bool SPLIT, int ATOMS = 1>
 __global__ void __launch_bounds__(BITS == 4 ? kThreadsW4 : kThreadsW8, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_w,
                     const Params p) {
@@ -342,9 +365,12 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
 
     // carve dynamic shared memory: [A8 stages][W8 stages][packed stages][epilogue transposers], 1024-byte aligned
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t a_bytes = (uint32_t)bt_cta * kBlockK;
+    const uint32_t a_atom = (uint32_t)bt_cta * kBlockK;        // one 128-channel atom of the token tile
+    const uint32_t a_bytes = a_atom * ATOMS;
     const uint32_t w_bytes = kTileN * kBlockK;
-    const uint32_t pk_bytes = kTileN * kBlockK / 2;
+    const uint32_t pk_atom = kTileN * kBlockK / 2;
+    const uint32_t pk_bytes = pk_atom * ATOMS;
+    constexpr int kSlotCols = kColsW * ATOMS;                   // TMEM columns of one unpacked stage
     const uint32_t smem_a = base;
     const uint32_t smem_w = smem_a + (uint32_t)p.stages * a_bytes;
     const uint32_t smem_p = smem_w + (BITS == 4 ? 0u : (uint32_t)p.stages * w_bytes);
@@ -431,7 +457,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                     const uint32_t bar = smem_u32(&s_full_tma[stage]);
                     if (CTAS == 1) {
                         mbar_arrive_expect_tx(bar, tx);
-                        tma_load_2d(smem_a + stage * a_bytes, &map_a, (kb0 + kb) * kBlockK, t0, bar);
+#pragma unroll
+                        for (int h = 0; h < ATOMS; ++h)     // channels past K arrive as zeros
+                            tma_load_2d(smem_a + stage * a_bytes + h * a_atom, &map_a, ((kb0 + kb) * ATOMS + h) * kBlockK, t0, bar);
                     } else {
                         // the pair's bytes are all counted on the even CTA's barrier, which it arms for both
                         if (leader) mbar_arrive_expect_tx(bar, tx * CTAS);
@@ -489,15 +517,24 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                     const uint32_t peek_bar_w = BITS == 4 ? smem_u32(&s_full_w8[w1]) : peek_bar_a;
                     const uint32_t peek_par_w = BITS == 4 ? wph1 : ph1;
                     const uint32_t bar_acc = kb == k_blocks - 1 ? smem_u32(&s_acc_full[acc_stage]) : 0u;
-                    const uint64_t adesc = smem_desc_sw128(smem_a + stage * a_bytes);
+                    uint32_t accumulate = kb != 0 ? 1u : 0u;
+                    if (BITS == 4 && ATOMS == 2) {       // the stage's first atom: four MMAs, no commit yet
+                        const uint64_t adesc0 = smem_desc_sw128(smem_a + stage * a_bytes);
+                        const uint64_t bd0[4] = {adesc0, adesc0 + 2, adesc0 + 4, adesc0 + 6};
+                        const uint32_t w0 = tmem_base + (uint32_t)(kAccStages * p.bt + wstage * kSlotCols);
+                        const uint32_t at0[4] = {w0, w0 + 8, w0 + 16, w0 + 24};
+                        issue_mmas_ts(d_tmem, at0, bd0, idesc, accumulate);
+                        accumulate = 1u;
+                    }
+                    const uint64_t adesc = smem_desc_sw128(smem_a + stage * a_bytes + (ATOMS - 1) * a_atom);
                     // step 32 bytes along K inside the swizzle atom: +2 in 16-byte address units
                     const uint64_t bd[4] = {adesc, adesc + 2, adesc + 4, adesc + 6};
                     uint32_t r;
                     if (BITS == 4) {
                         // 32 int8 of K = 8 TMEM columns per MMA
-                        const uint32_t w_tmem = tmem_base + (uint32_t)(kAccStages * p.bt + wstage * kColsW);
+                        const uint32_t w_tmem = tmem_base + (uint32_t)(kAccStages * p.bt + wstage * kSlotCols + (ATOMS - 1) * kColsW);
                         const uint32_t at[4] = {w_tmem, w_tmem + 8, w_tmem + 16, w_tmem + 24};
-                        r = issue_kblock_ts<CTAS>(0u, d_tmem, at, bd, idesc, kb != 0 ? 1u : 0u,
+                        r = issue_kblock_ts<CTAS>(0u, d_tmem, at, bd, idesc, accumulate,
                                                   smem_u32(&s_empty[stage]), bar_acc, left > 0 ? 1u : 0u, peek_bar_a, ph1,
                                                   peek_bar_w, peek_par_w);
                     } else {
@@ -543,7 +580,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             }
             // a tile takes at least ~0.2 us per k-block: sleep through a quarter of that before the first look,
             // so that eight idle warps do not spend issue slots polling while a long tile is being accumulated
-            if (k_blocks >= 32) __nanosleep(k_blocks >= 400 ? 20000u : (unsigned)k_blocks * 50u);
+            if (k_blocks * ATOMS >= 32) __nanosleep(k_blocks * ATOMS >= 400 ? 20000u : (unsigned)(k_blocks * ATOMS) * 50u);
             ok = mbar_wait_warp_relaxed(smem_u32(&s_acc_full[acc_stage]), acc_phase, abort_flag, p.watchdog, kWdEpilogue);
             if (!ok) break;
             // K split.  Every slice writes its raw int32 sums to its own block of scratch
@@ -774,31 +811,42 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                 if (!ok) break;
                 if ((warp & 3) == 0) FQ_TRACE(2, n, 1);
                 const uint32_t src = smem_p + (uint32_t)ps * pk_bytes;     // shared-space address of the stage
-                uint4 pk[4];
+                const uint32_t w_tmem = tmem_base + lane_addr + (uint32_t)(kAccStages * p.bt + ws * kSlotCols);
+                bool slot_free = false;
 #pragma unroll
-                for (int c = 0; c < 4; ++c) pk[c] = lds128(src + row_off[c]);
-                // is the TMEM slot free?  (tested now, needed only after the expansion below)
-                const bool slot_free = m < 0 || mbar_test_wait(smem_u32(&s_empty[es]), eph);
-                __syncwarp();
-                if (elect_one()) mbar_arrive(smem_u32(&s_empty_p[ps]));   // packed stage read: give it back
-                const uint32_t w_tmem = tmem_base + lane_addr + (uint32_t)(kAccStages * p.bt + ws * kColsW);
-                uint32_t o[32];                          // 128 codes -> 128 int8 = 32 TMEM columns
+                for (int h = 0; h < ATOMS; ++h) {
+                    uint4 pk[4];
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    const uint32_t w[4] = {pk[c].x, pk[c].y, pk[c].z, pk[c].w};
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        const uint32_t lo = (w[q] << 4) & 0xF0F0F0F0u;   // even channels, 16*code
-                        const uint32_t hi = w[q] & 0xF0F0F0F0u;          // odd channels
-                        o[8 * c + 2 * q + 0] = lo;   // same (even, odd) channel order as the int8 activations
-                        o[8 * c + 2 * q + 1] = hi;
+                    for (int c = 0; c < 4; ++c) pk[c] = lds128(src + h * pk_atom + row_off[c]);
+                    if (h == 0) {
+                        // is the TMEM slot free?  (tested now, needed only after the expansion below)
+                        slot_free = m < 0 || mbar_test_wait(smem_u32(&s_empty[es]), eph);
                     }
+                    if (h == ATOMS - 1) {
+                        __syncwarp();
+                        if (elect_one()) mbar_arrive(smem_u32(&s_empty_p[ps]));   // packed stage read: give it back
+                    }
+                    uint32_t o[32];                          // 128 codes -> 128 int8 = 32 TMEM columns
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        const uint32_t w[4] = {pk[c].x, pk[c].y, pk[c].z, pk[c].w};
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            const uint32_t lo = (w[q] << 4) & 0xF0F0F0F0u;   // even channels, 16*code
+                            const uint32_t hi = w[q] & 0xF0F0F0F0u;          // odd channels
+                            o[8 * c + 2 * q + 0] = lo;   // same (even, odd) channel order as the int8 activations
+                            o[8 * c + 2 * q + 1] = hi;
+                        }
+                    }
+                    if (h == 0) {
+                        ok = mbar_wait_all(smem_u32(&s_empty[es]), eph, abort_flag, p.watchdog, kWdUnpackEmpty, slot_free);
+                        if (!ok) break;
+                        if ((warp & 3) == 0) FQ_TRACE(2, n, 2);
+                        tc_fence_after();
+                    }
+                    tmem_st32(w_tmem + h * kColsW, o);
                 }
-                ok = mbar_wait_all(smem_u32(&s_empty[es]), eph, abort_flag, p.watchdog, kWdUnpackEmpty, slot_free);
                 if (!ok) break;
-                if ((warp & 3) == 0) FQ_TRACE(2, n, 2);
-                tc_fence_after();
-                tmem_st32(w_tmem, o);
                 tmem_st_wait();
                 tc_fence_before();
                 __syncwarp();
@@ -839,7 +887,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                 if (elect_one()) {
                     const uint32_t bar = smem_u32(&s_full_p[ps]);
                     mbar_arrive_expect_tx(bar, pk_bytes);
-                    tma_load_2d(smem_p + ps * pk_bytes, &map_w, (kb0 + kb) * (kBlockK / 2), n0, bar);
+#pragma unroll
+                    for (int h = 0; h < ATOMS; ++h)
+                        tma_load_2d(smem_p + ps * pk_bytes + h * pk_atom, &map_w, ((kb0 + kb) * ATOMS + h) * (kBlockK / 2), n0, bar);
                 }
                 if (++ps == p.stages_p) { ps = 0; pph ^= 1u; }
                 if (++kb == k_blocks) {
@@ -938,10 +988,10 @@ fq_status build_weight_tmap(Weights& W) {
 
 namespace {
 
-template <int BITS, int CTAS, bool SPLIT>
+template <int BITS, int CTAS, bool SPLIT, int ATOMS = 1>
 fq_status launch_variant(const CUtensorMap& map_a, const CUtensorMap& map_w, const Params& p, int grid, size_t smem,
                          int cluster, cudaStream_t stream) {
-    auto kern = gemm_tcgen05_kernel<BITS, CTAS, SPLIT>;
+    auto kern = gemm_tcgen05_kernel<BITS, CTAS, SPLIT, ATOMS>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return FQ_ERR_CUDA;
     return launch_pdl(kern, (unsigned)grid, (unsigned)(BITS == 4 ? kThreadsW4 : kThreadsW8), smem, stream, (unsigned)cluster,
@@ -1064,14 +1114,23 @@ fq_status launch_gemm_tcgen05(const int8_t* a8, int64_t M, const Weights& W, int
 #if defined(FQ_GEMM_TRACE) || defined(FQ_GEMM_DEV)
     p.dbg = getenv("FQ_DBG") ? atoi(getenv("FQ_DBG")) : 0;
 #endif
+    // 4-bit weights, single CTAs, token tiles of at most 128: two 128-channel atoms per pipeline stage (the
+    // accumulators of longer tiles leave no room for TMEM slots twice as wide).  Needs whole atoms (K a multiple
+    // of 128) and, with a K split, slices of whole stages.
+    const int64_t kb128 = (W.K + kBlockK - 1) / kBlockK;
+    int atoms = (W.bits == 4 && ctas == 1 && bt <= 128 && W.K % kBlockK == 0 && (split == 1 || kb128 % (2 * split) == 0)) ? 2 : 1;
+#if defined(FQ_GEMM_TRACE) || defined(FQ_GEMM_DEV)
+    if (getenv("FQ_ATOMS") && atoi(getenv("FQ_ATOMS")) == 1) atoms = 1;
+#endif
     // 4-bit weights: every TMEM column the accumulators leave free becomes unpacked-weight ring
-    int stages_w = W.bits == 4 ? (512 - kAccStages * bt) / kColsW : 0;
+    int stages_w = W.bits == 4 ? (512 - kAccStages * bt) / (kColsW * atoms) : 0;
     if (stages_w > kMaxStagesW) stages_w = kMaxStagesW;
-    p.tmem_cols = next_pow2(kAccStages * bt + stages_w * kColsW);
+    p.tmem_cols = next_pow2(kAccStages * bt + stages_w * kColsW * atoms);
 
     const size_t epi_bytes = (size_t)kEpiWarps * kEpiStageBytes;
     const size_t budget = 227 * 1024 - 1024 /*alignment slack*/ - 1024 /*static*/ - epi_bytes;
-    const size_t a_bytes = (size_t)(bt / ctas) * kBlockK, w_bytes = (size_t)kTileN * kBlockK, pk_bytes = w_bytes / 2;
+    const size_t a_bytes = (size_t)(bt / ctas) * kBlockK * atoms, w_bytes = (size_t)kTileN * kBlockK,
+                 pk_bytes = w_bytes / 2 * atoms;
     size_t smem;
     if (W.bits == 4) {
         p.stages_w = stages_w;
@@ -1112,12 +1171,15 @@ fq_status launch_gemm_tcgen05(const int8_t* a8, int64_t M, const Weights& W, int
     p.unit_step = clusters;
     p.units_q = num_units / clusters;
     p.units_rem = num_units % clusters;
-    p.kb_per = (int)((W.K + kBlockK - 1) / kBlockK) / split;    // the planner only picks splits that divide it
+    p.kb_per = (int)((kb128 + atoms - 1) / atoms) / split;      // stages per unit; the planner only picks splits that divide it
     p.split_shift = split == 1 ? 0 : (split == 2 ? 1 : (split == 4 ? 2 : (split == 8 ? 3 : 4)));
     p.counters = W.tile_counters;
 
     if (W.bits == 4) {
         if (ctas == 2) return launch_variant<4, 2, false>(map_a, W.tmap, p, grid, smem, 2, stream);
+        if (atoms == 2)
+            return split > 1 ? launch_variant<4, 1, true, 2>(map_a, W.tmap, p, grid, smem, 1, stream)
+                             : launch_variant<4, 1, false, 2>(map_a, W.tmap, p, grid, smem, 1, stream);
         return split > 1 ? launch_variant<4, 1, true>(map_a, W.tmap, p, grid, smem, 1, stream)
                          : launch_variant<4, 1, false>(map_a, W.tmap, p, grid, smem, 1, stream);
     }
