@@ -1014,7 +1014,8 @@ struct Plan {
 // over m_tiles so that ragged M wastes little.  Candidates are ranked by a cost model fitted to
 // measured launches (cycles): rounds of work units over the SMs, each unit costing
 //     k_blocks * per_kblock(bt) + 16*bt + 1000          (the tail: epilogue and tile hand-over)
-//   4-bit weights:          per_kblock = 330 + bt       (issue floor, then the MMAs' 2*bt)
+//   4-bit weights:          per_kblock = 330 + bt       (issue floor, then the MMAs' 2*bt); 235 + bt for tiles of at
+//                                        most 128 tokens, whose stages hold two k-blocks
 //   8-bit, one CTA:         per_kblock = max(350 + 0.8*bt, 230 + 2*bt)   (issue floor, then shared memory:
 //                                        both operands pass through it)
 //   8-bit, CTA pair:        per_kblock = max(545, 2.62*bt)   (each CTA stages half of the token tile)
@@ -1035,7 +1036,9 @@ Plan plan_gemm(int64_t M, int64_t N, int64_t K, int bits, int sms, size_t scratc
             if (b > bt_max) continue;
             const int64_t units = n_units * ((M + b - 1) / b);
             const double w8_single = 350.0 + 0.8 * b > 230.0 + 2.0 * b ? 350.0 + 0.8 * b : 230.0 + 2.0 * b;
-            const double per_kb = bits == 4 ? 330.0 + b : (c == 1 ? w8_single : (2.62 * b > 545.0 ? 2.62 * b : 545.0));
+            // 4-bit, tiles of at most 128 tokens: two-atom stages (see the kernel) cost less per 128 channels
+            const double w4 = (c == 1 && b <= 128 && K % kBlockK == 0) ? 235.0 + b : 330.0 + b;
+            const double per_kb = bits == 4 ? w4 : (c == 1 ? w8_single : (2.62 * b > 545.0 ? 2.62 * b : 545.0));
             for (int sp = 1; sp <= (c == 1 ? kMaxSplit : 1); sp *= 2) {
                 if (sp > 1 && (kb % sp != 0 || kb / sp < 2 || units > kMaxSplitTiles || units * sp > 4 * (int64_t)sms)) continue;
                 const int64_t kb_per = kb / sp;
