@@ -1,6 +1,6 @@
 // Short-batch weight streaming for 4-bit weights: the projection of a handful of tokens is a
 // matrix-vector product bound by the weight bytes, which must cross HBM once.  Two users:
-//   * the W4A4 integer product of Eq. 8 for batches of at most 16 tokens on matrices of up to 32 Mi weights
+//   * the W4A4 integer product of Eq. 8 for batches of at most 16 tokens on matrices of up to 16-32 Mi weights
 //     (the short end of the throughput sweep), where it measured faster than the TMA/TMEM pipeline of the
 //     big GEMM, whose per-k-block hand-overs cannot be fed at HBM rate by so thin a tile;
 //   * the weight-only projection with floating-point activations (the adaptive layer-normalisation
@@ -24,6 +24,7 @@
 //   bf16:  one mask of the word shifted by 4 j isolates the codes of channels j and j + 4 in the two
 //          halves of a register, and the B fragment pairs the activations of those channels.
 #include <cuda_bf16.h>
+#include <stdlib.h>
 
 #include "fq_common.cuh"
 #include "ptx_sm100.cuh"
@@ -412,8 +413,13 @@ bool build_stream_tmap(Weights& W) {
 }
 
 bool gemm_stream_applies(int64_t M, const Weights& W) {
-    // measured against the tcgen05 kernel: ahead for at most 16 tokens on matrices up to 32 Mi weights
-    return W.bits == 4 && W.tmap_stream_valid && M >= 1 && M <= 16 && W.N * W.K <= (1ll << 25);
+#if defined(FQ_GEMM_TRACE) || defined(FQ_GEMM_DEV)
+    if (getenv("FQ_NO_STREAM")) return false;      // development builds: compare against the tcgen05 kernel
+#endif
+    // measured against the tcgen05 kernel: ahead for at most 8 tokens on matrices up to 32 Mi weights and for at
+    // most 16 tokens up to 16 Mi
+    if (W.bits != 4 || !W.tmap_stream_valid || M < 1 || M > 16) return false;
+    return W.N * W.K <= (M <= 8 ? (1ll << 25) : (1ll << 24));
 }
 
 cudaError_t launch_gemm_stream(const int8_t* a8, int64_t M, const Weights& W, int acc_shift, const GemmOut& out,
