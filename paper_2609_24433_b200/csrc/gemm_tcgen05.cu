@@ -518,13 +518,16 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                     const uint32_t peek_par_w = BITS == 4 ? wph1 : ph1;
                     const uint32_t bar_acc = kb == k_blocks - 1 ? smem_u32(&s_acc_full[acc_stage]) : 0u;
                     uint32_t accumulate = kb != 0 ? 1u : 0u;
-                    if (BITS == 4 && ATOMS == 2) {       // the stage's first atom: four MMAs, no commit yet
-                        const uint64_t adesc0 = smem_desc_sw128(smem_a + stage * a_bytes);
-                        const uint64_t bd0[4] = {adesc0, adesc0 + 2, adesc0 + 4, adesc0 + 6};
-                        const uint32_t w0 = tmem_base + (uint32_t)(kAccStages * p.bt + wstage * kSlotCols);
-                        const uint32_t at0[4] = {w0, w0 + 8, w0 + 16, w0 + 24};
-                        issue_mmas_ts(d_tmem, at0, bd0, idesc, accumulate);
-                        accumulate = 1u;
+                    if (BITS == 4 && ATOMS > 1) {        // all atoms of the stage but the last: four MMAs each, no commit yet
+#pragma unroll
+                        for (int h = 0; h < ATOMS - 1; ++h) {
+                            const uint64_t adesc0 = smem_desc_sw128(smem_a + stage * a_bytes + h * a_atom);
+                            const uint64_t bd0[4] = {adesc0, adesc0 + 2, adesc0 + 4, adesc0 + 6};
+                            const uint32_t w0 = tmem_base + (uint32_t)(kAccStages * p.bt + wstage * kSlotCols + h * kColsW);
+                            const uint32_t at0[4] = {w0, w0 + 8, w0 + 16, w0 + 24};
+                            issue_mmas_ts(d_tmem, at0, bd0, idesc, accumulate);
+                            accumulate = 1u;
+                        }
                     }
                     const uint64_t adesc = smem_desc_sw128(smem_a + stage * a_bytes + (ATOMS - 1) * a_atom);
                     // step 32 bytes along K inside the swizzle atom: +2 in 16-byte address units
@@ -1122,6 +1125,7 @@ fq_status launch_gemm_tcgen05(const int8_t* a8, int64_t M, const Weights& W, int
     // of 128) and, with a K split, slices of whole stages.
     const int64_t kb128 = (W.K + kBlockK - 1) / kBlockK;
     int atoms = (W.bits == 4 && ctas == 1 && bt <= 128 && W.K % kBlockK == 0 && (split == 1 || kb128 % (2 * split) == 0)) ? 2 : 1;
+    if (atoms == 2 && bt <= 64 && kb128 >= 4 * split && (split == 1 || kb128 % (4 * split) == 0)) atoms = 4;   // four for the shortest tiles
 #if defined(FQ_GEMM_TRACE) || defined(FQ_GEMM_DEV)
     if (getenv("FQ_ATOMS") && atoi(getenv("FQ_ATOMS")) == 1) atoms = 1;
 #endif
@@ -1180,6 +1184,9 @@ fq_status launch_gemm_tcgen05(const int8_t* a8, int64_t M, const Weights& W, int
 
     if (W.bits == 4) {
         if (ctas == 2) return launch_variant<4, 2, false>(map_a, W.tmap, p, grid, smem, 2, stream);
+        if (atoms == 4)
+            return split > 1 ? launch_variant<4, 1, true, 4>(map_a, W.tmap, p, grid, smem, 1, stream)
+                             : launch_variant<4, 1, false, 4>(map_a, W.tmap, p, grid, smem, 1, stream);
         if (atoms == 2)
             return split > 1 ? launch_variant<4, 1, true, 2>(map_a, W.tmap, p, grid, smem, 1, stream)
                              : launch_variant<4, 1, false, 2>(map_a, W.tmap, p, grid, smem, 1, stream);
