@@ -392,6 +392,58 @@ def test_back_to_back_calls_share_a_workspace_without_syncs():
             assert torch.equal(a, b)
 
 
+def _pack_dev(c: torch.Tensor, bits: int) -> torch.Tensor:
+    if bits == 8:
+        return c.view(torch.uint8)
+    u = c.to(torch.int16) & 15
+    return (u[:, 0::2] | (u[:, 1::2] << 4)).to(torch.uint8)
+
+
+def test_random_shapes_against_the_second_witness():
+    """Seeded random (M, N, K, bits): every launch configuration the planner can pick (token tiles of 16..208,
+    one-, two- and four-atom stages, K splits, CTA pairs, the streaming kernel) must give the dp4a witness's
+    accumulators bit for bit and its outputs, with no bounded wait expiring."""
+    rng = np.random.default_rng(2024)
+    done = 0
+    while done < 48:
+        bits = int(rng.choice([4, 4, 4, 8]))
+        M = int(rng.choice([1, 3, 8, 16, 17, 33, 50, 64, 65, 100, 128, 129, 200, 256, 300, 520, 816]))
+        N = int(rng.choice([8, 72, 128, 136, 1024, 3072, 4096, 8192]))
+        K = int(rng.choice([32, 96, 128, 256, 384, 512, 640, 1024, 1536, 2048, 4096, 8192, 16384]))
+        if N * K > 1 << 26 or M * N > 1 << 22:
+            continue
+        done += 1
+        q = 7 if bits == 4 else 127
+        gen = torch.Generator(device="cuda").manual_seed(done)
+        wc = torch.randint(-q, q + 1, (N, K), dtype=torch.int8, device="cuda", generator=gen)
+        ac = torch.randint(-q, q + 1, (M, K), dtype=torch.int8, device="cuda", generator=gen)
+        h = fq.weights_import(_pack_dev(wc, bits), torch.ones(N, device="cuda"), None, None, K, 32, bits)
+        a = _pack_dev(ac, bits)
+        assert torch.equal(fq.gemm_acc_i32(a, h), fq.gemm_simt(a, None, h, raw_acc=True)), (M, N, K, bits)
+        d = torch.rand(M, device="cuda", generator=gen) + 0.5
+        y = (fq.gemm_w4a4 if bits == 4 else fq.gemm_w8a8)(a, d, h, torch.float32)
+        assert torch.allclose(y, fq.gemm_simt(a, d, h, torch.float32), rtol=1e-5, atol=1e-5), (M, N, K, bits)
+        st, word = fq.device_status()
+        assert st == fq.OK, (M, N, K, bits, hex(word))
+
+
+@pytest.mark.parametrize("M", [1, 16, 64])
+def test_short_batch_on_a_large_matrix(M):
+    """Long K loops on many tiles (128 stages of four atoms, or a K split): the regime where a pipeline that
+    loses a barrier phase would stall rather than miscompute."""
+    N, K = 8192, 16384
+    gen = torch.Generator(device="cuda").manual_seed(M)
+    wc = torch.randint(-7, 8, (N, K), dtype=torch.int8, device="cuda", generator=gen)
+    ac = torch.randint(-7, 8, (M, K), dtype=torch.int8, device="cuda", generator=gen)
+    h = fq.weights_import(_pack_dev(wc, 4), torch.ones(N, device="cuda"), None, None, K, 32, 4)
+    a = _pack_dev(ac, 4)
+    for _ in range(3):                                        # back to back: ring phases carry over nothing
+        acc = fq.gemm_acc_i32(a, h)
+    assert torch.equal(acc, fq.gemm_simt(a, None, h, raw_acc=True))
+    st, word = fq.device_status()
+    assert st == fq.OK, hex(word)
+
+
 def test_gemm_is_deterministic_run_to_run():
     rng = np.random.default_rng(5)
     a, w = random_codes(rng, 333, 2048, 4), random_codes(rng, 520, 2048, 4)
