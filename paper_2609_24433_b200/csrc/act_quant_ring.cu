@@ -420,7 +420,10 @@ cudaError_t launch_transform_quantize_ring(const void* x, fq_dtype xt, int64_t r
     int dev = 0, sms = 148;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    if (rows < 2 * (int64_t)sms) return cudaErrorNotSupported;     // short batches: latency-bound, register kernel
+    // Short batches are latency-bound and go to the register kernel, which spreads a row over more threads: fewer
+    // than 8 rows per SM, unless the rows are long (measured at M = 816: K = 2048 6.4 us there against 7.1-7.9 us
+    // here, K = 16384 24.3 us there against 21.2 us here).
+    if (rows < 2 * (int64_t)sms || (rows < 8 * (int64_t)sms && K < 8192)) return cudaErrorNotSupported;
 
     // channels per thread (the fold-after variant with shuffle stages does not fit 64 without spills)
     const int e = (K >= 2048 && K % 64 == 0 && !(mult != nullptr && mult_after_rotation && block >= 128)) ? 64 : 32;
