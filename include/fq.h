@@ -20,7 +20,7 @@
  *   - Errors are return codes.  Nothing aborts, throws or traps.  Argument checks run
  *     on the host before any launch; a failed check launches nothing.
  *   - Inputs must be finite; NaN/Inf give unspecified codes (never a fault).
- *   - Supported sizes: hadamard_block a power of two in [2, 256] dividing K;
+ *   - Supported sizes: hadamard_block a power of two in [1, 256] dividing K (1 = identity rotation);
  *     K a multiple of 32 and <= 131072 (int32 accumulator bound; the prologue and the fold
  *     keep a whole token in one thread block and accept K <= 32768); N a multiple of 8;
  *     bits 4 or 8; clip_ratio in (0, 1].  M = 0 or N = 0 succeeds and does nothing.
@@ -192,7 +192,9 @@ fq_status fq_quantize_act_after(const void* x, fq_dtype xt, int64_t M, int64_t K
 
 /* ---- integer GEMM + rescale/bias epilogue on pre-quantized activations (Eq. 8) -----------------
  * a_codes device, canonical codes from fq_quantize_act with the same bit width as W.
- * a_delta device float[M].   y device [M, N] of dtype yt, leading dimension ldy.
+ * a_delta device float[M]; any 4-byte aligned address is accepted (a slice delta + t0 of a longer vector is
+ * fine: the epilogue then reads the steps one by one instead of four at a time).
+ * y device [M, N] of dtype yt, leading dimension ldy.
  * workspace device, at least fq_workspace_bytes(M, K, N, bits) bytes, 256-byte aligned; contents
  * are scratch (calls sharing a workspace must be stream-ordered).
  * Shared sites: quantize once, then call this once per consumer handle. */
@@ -255,7 +257,11 @@ fq_status fq_linear_gated(const void* gate_up, fq_dtype xt, int64_t M, int64_t l
  *   anything larger returns FQ_ERR_NOMEM and launches nothing.  The scratch (4 MiB + 64 KiB) is
  *   held by every GPU that loads the library until the process exits.
  *   The first call on each device looks up the scratch's device address (once, with that device
- *   current); make that first call before any stream capture.
+ *   current).  That look-up is also what makes the CUDA runtime load the part of the library image
+ *   that holds the scratch onto the device, so this ONE call may itself reserve device memory, may
+ *   synchronise, and can fail with FQ_ERR_CUDA on a device that has no room left: make it at
+ *   start-up, before any stream capture and before the phase in which allocation is forbidden.  A
+ *   call with M = 0 performs just this set-up and launches nothing, so it serves as the warm-up.
  *   All calls on a device share the one scratch.  Nothing in it needs clearing -- each call
  *   rewrites every row it later reads -- but it keeps the previous call's contents, and two calls
  *   whose kernels may overlap on the GPU (different streams without an ordering between them)
@@ -268,9 +274,10 @@ fq_status fq_linear_w4a4_static(const void* x, fq_dtype xt, int64_t M, int64_t l
 /* Bytes of workspace that fq_gemm_* / fq_linear_* want for this shape (host computation): the int8
  * activation codes and steps (M*K + 4*M bytes, each rounded up to 256), plus scratch for int32 partial
  * tiles on shapes with few output tiles and a long K, which the GEMM then splits along K.  A workspace
- * that holds only the first part is accepted; the GEMM then runs without the split.  A split launch
- * keeps per-tile counters in the weight handle: calls that may split K on the same handle must be
- * ordered on one stream (or pass workspaces without the scratch part). */
+ * that holds only the first part is accepted; the GEMM then runs without the split.  Everything a call
+ * scribbles on lives in the workspace it was given (the split's tile counters included, cleared by a
+ * memset node at the head of the call): a weight handle is read-only at run time, so calls on the same
+ * handle may run concurrently on different streams as long as each has its own workspace. */
 size_t fq_workspace_bytes(int64_t M, int64_t K, int64_t N, int bits);
 
 /* Parity/debug: raw int32 accumulators acc[M, N] (device, pitch N) of Eq. 8's integer sum. */
@@ -289,6 +296,13 @@ fq_status fq_gemm_simt(const void* a_codes, const float* a_delta, int64_t M, con
  * events of its own obtains the two kernel durations of that very launch.  During a stream capture
  * the mark becomes an external event-record node of the graph.  NULL switches it off. */
 fq_status fq_profile_mark(void* event);
+
+/* Self-test of the watchdog below: enqueues a one-warp kernel whose only action is a bounded wait, with the
+ * library's own wait routine and a limit of limit_ns nanoseconds (clamped to [1 us, 100 ms]), on a barrier that
+ * nothing ever signals.  The wait gives up, the kernel ends normally, and the next fq_device_status() returns
+ * FQ_ERR_TIMEOUT (detail bit 0x400) and clears the record; the device stays fully usable.  Lets a deployment
+ * (and this library's tests) check the time-out plumbing without any faulting or hanging kernel. */
+fq_status fq_watchdog_selftest(uint64_t limit_ns, void* stream);
 
 /* Device-side wait watchdog.  Every spin on an mbarrier inside the kernels is bounded; a wait
  * that expires records a code in a device word and the kernel winds down normally.  This call

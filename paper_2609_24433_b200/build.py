@@ -27,15 +27,19 @@ def build(force: bool = False, verbose: bool = False) -> str:
     headers.append(os.path.join(ROOT, "include", "fq.h"))
     objs = []
     relink = force
+    jobs = []
     for src in SOURCES:
         s = os.path.join(CSRC, src)
         o = os.path.join(CSRC, src.replace(".cu", ".o"))
         objs.append(o)
         if force or _stale(o, [s] + headers):
-            extra = os.environ.get("FQ_NVCC_EXTRA", "").split()      # e.g. -DFQ_GEMM_TRACE (development)
-            cmd = [nvcc] + NVCC_FLAGS + extra + (["-Xptxas", "-v"] if verbose else []) + ["-c", s, "-o", o]
-            subprocess.run(cmd, check=True)
+            jobs.append([nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-c", s, "-o", o])
             relink = True
+    if jobs:      # the translation units are independent: compile them side by side
+        from concurrent.futures import ThreadPoolExecutor
+        with ThreadPoolExecutor(max_workers=min(len(jobs), os.cpu_count() or 1)) as pool:
+            for done in pool.map(lambda cmd: subprocess.run(cmd, check=True), jobs):
+                pass
     if relink or _stale(LIB, objs):
         subprocess.run([nvcc, "-shared", "-o", LIB] + objs, check=True)
     return LIB

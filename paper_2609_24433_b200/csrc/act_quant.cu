@@ -293,14 +293,10 @@ cudaError_t launch_e(const XT* x, int64_t rows, int K, int64_t ldx, const float*
     int rpc = 256 / tpr;
     if (rpc < 1) rpc = 1;
     const int threads = tpr * rpc;
-    int dev = 0, sms = 148;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int sms = device_sm_count();
     const int64_t iters = (rows + rpc - 1) / rpc;
     auto args = [&](auto kern) {
-        int resident = 1;
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&resident, kern, threads, 0) != cudaSuccess || resident < 1)
-            resident = 1;
+        const int resident = max_resident_blocks(reinterpret_cast<const void*>(kern), threads);
         int64_t grid = iters < (int64_t)sms * resident ? iters : (int64_t)sms * resident;
         if (grid < 1) grid = 1;
         launch_pdl(kern, (unsigned)grid, (unsigned)threads, 0, stream, 1u, x, rows, K, ldx, mult, cnorm, block, (float)qmax,

@@ -373,7 +373,7 @@ transform_quantize_ring_kernel(const __grid_constant__ CUtensorMap map_x, const 
 template <typename XT, int FMT, int E, int BLOCK>
 cudaError_t launch_ring(const CUtensorMap& map, const RingParams& p, int grid, size_t smem, cudaStream_t stream) {
     auto go = [&](auto kern) -> cudaError_t {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), smem);
         if (e != cudaSuccess) return e;
         return launch_pdl(kern, (unsigned)grid, (unsigned)kThreads, smem, stream, 1u, map, p);
     };
@@ -417,9 +417,7 @@ cudaError_t launch_transform_quantize_ring(const void* x, fq_dtype xt, int64_t r
     // shape gate: whole 128-byte lines, at most 256 of them per box, blocks of 32..256 channels
     if (K < 1024 || row_bytes % 128 != 0 || row_bytes / 128 > 256 || rows > 0x7fffffffll || block < 32)
         return cudaErrorNotSupported;
-    int dev = 0, sms = 148;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int sms = device_sm_count();
     // Short batches are latency-bound and go to the register kernel, which spreads a row over more threads: fewer
     // than 8 rows per SM, unless the rows are long (measured at M = 816: K = 2048 6.4 us there against 7.1-7.9 us
     // here, K = 16384 24.3 us there against 21.2 us here).

@@ -2,11 +2,90 @@
 // management and stream-ordered dispatch.  No entry point below touches data on
 // the host; every step of the path runs in the kernels of this library.
 #include <math.h>
+#include <mutex>
 #include <new>
+#include <unordered_map>
 
 #include "fq_common.cuh"
 
 using namespace fq;
+
+namespace fq {
+
+namespace {
+constexpr int kMaxDevices = 64;
+struct DeviceFacts { int sms = 0, major = -1; };
+std::mutex g_facts_mutex;
+DeviceFacts g_facts[kMaxDevices];
+std::unordered_map<const void*, size_t> g_smem_opt_in[kMaxDevices];
+std::unordered_map<const void*, std::unordered_map<int, int>> g_resident[kMaxDevices];
+
+DeviceFacts device_facts() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) { (void)cudaGetLastError(); return DeviceFacts(); }
+    const bool cached = dev >= 0 && dev < kMaxDevices;
+    std::lock_guard<std::mutex> lock(g_facts_mutex);
+    if (cached && g_facts[dev].sms > 0) return g_facts[dev];
+    DeviceFacts f;
+    if (cudaDeviceGetAttribute(&f.sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&f.major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return DeviceFacts();
+    }
+    if (cached) g_facts[dev] = f;
+    return f;
+}
+}  // namespace
+
+int device_sm_count() {
+    const int sms = device_facts().sms;
+    return sms > 0 ? sms : 148;
+}
+
+int device_cc_major() { return device_facts().major; }
+
+cudaError_t ensure_dynamic_smem(const void* kernel, size_t bytes) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return cudaGetLastError();
+    const bool cached = dev >= 0 && dev < kMaxDevices;
+    if (cached) {
+        std::lock_guard<std::mutex> lock(g_facts_mutex);
+        auto it = g_smem_opt_in[dev].find(kernel);
+        if (it != g_smem_opt_in[dev].end() && it->second >= bytes) return cudaSuccess;
+    }
+    const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+    if (e == cudaSuccess && cached) {
+        std::lock_guard<std::mutex> lock(g_facts_mutex);
+        g_smem_opt_in[dev][kernel] = bytes;
+    }
+    return e;
+}
+
+int max_resident_blocks(const void* kernel, int threads) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) { (void)cudaGetLastError(); return 1; }
+    const bool cached = dev >= 0 && dev < kMaxDevices;
+    if (cached) {
+        std::lock_guard<std::mutex> lock(g_facts_mutex);
+        auto it = g_resident[dev].find(kernel);
+        if (it != g_resident[dev].end()) {
+            auto jt = it->second.find(threads);
+            if (jt != it->second.end()) return jt->second;
+        }
+    }
+    int resident = 1;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&resident, kernel, threads, 0) != cudaSuccess || resident < 1) {
+        (void)cudaGetLastError();
+        return 1;
+    }
+    if (cached) {
+        std::lock_guard<std::mutex> lock(g_facts_mutex);
+        g_resident[dev][kernel][threads] = resident;
+    }
+    return resident;
+}
+
+}  // namespace fq
 
 namespace {
 
@@ -23,10 +102,8 @@ bool valid_block(int block, int64_t K) {
 float block_norm(int block) { return (float)(1.0 / sqrt((double)block)); }
 
 fq_status check_arch() {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return FQ_ERR_CUDA;
-    int major = 0;
-    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return FQ_ERR_CUDA;
+    const int major = device_cc_major();
+    if (major < 0) return FQ_ERR_CUDA;
     return major == 10 ? FQ_OK : FQ_ERR_ARCH;
 }
 
@@ -48,12 +125,9 @@ fq_status alloc_handle(int64_t N, int64_t K, int block, int bits, Weights** out)
     ok = ok && cudaMalloc(&w->w_scale, sizeof(float) * (size_t)(N > 0 ? N : 4)) == cudaSuccess;
     ok = ok && cudaMalloc(&w->bias, sizeof(float) * (size_t)(N > 0 ? N : 4)) == cudaSuccess;
     ok = ok && cudaMalloc(&w->mult_g, sizeof(float) * (size_t)K) == cudaSuccess;
-    // counters of the GEMM's K split (slices of a tile finished): zero whenever no launch is in flight
-    ok = ok && cudaMalloc(&w->tile_counters, sizeof(uint32_t) * 1024) == cudaSuccess;
-    ok = ok && cudaMemset(w->tile_counters, 0, sizeof(uint32_t) * 1024) == cudaSuccess;
     if (!ok) {
         cudaGetLastError();
-        cudaFree(w->codes); cudaFree(w->w_scale); cudaFree(w->bias); cudaFree(w->mult_g); cudaFree(w->tile_counters);
+        cudaFree(w->codes); cudaFree(w->w_scale); cudaFree(w->bias); cudaFree(w->mult_g);
         delete w;
         return FQ_ERR_NOMEM;
     }
@@ -112,6 +186,12 @@ fq_status gemm_from_codes(const void* a_codes, const float* a_delta, int64_t M, 
     if (st != FQ_OK) return st;
     const int8_t* a8 = static_cast<const int8_t*>(a_codes);
     int shift = 0;
+    size_t scratch_bytes = 0;
+    void* scratch = scratch_of(workspace, ws_bytes, M, W->K, &scratch_bytes);
+    if (!simt) {
+        st = gemm_prepare(M, *W, scratch, scratch_bytes, stream);
+        if (st != FQ_OK) return st;
+    }
     if (bits == 4) {
         Workspace ws;
         st = carve(workspace, ws_bytes, M, W->K, &ws);
@@ -121,8 +201,6 @@ fq_status gemm_from_codes(const void* a_codes, const float* a_delta, int64_t M, 
         shift = 8;   // both operands carry 16*code
     }
     if (simt) return launch_gemm_simt(a8, M, *W, shift, out, stream) == cudaSuccess ? FQ_OK : FQ_ERR_CUDA;
-    size_t scratch_bytes = 0;
-    void* scratch = scratch_of(workspace, ws_bytes, M, W->K, &scratch_bytes);
     return launch_gemm(a8, M, *W, shift, out, scratch, scratch_bytes, stream);
 }
 
@@ -147,14 +225,20 @@ fq_status linear_impl(const void* x, fq_dtype xt, int64_t M, int64_t ldx, const 
     st = carve(workspace, ws_bytes, M, W->K, &ws);
     if (st != FQ_OK) return st;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    size_t scratch_bytes = 0;
+    void* scratch = scratch_of(workspace, ws_bytes, M, W->K, &scratch_bytes);
+    st = gemm_prepare(M, *W, scratch, scratch_bytes, s);       // ahead of the prologue: see gemm_prepare
+    if (st != FQ_OK) return st;
     // Prologue writes one int8 per code into the workspace (4-bit codes stay in [-7, 7] and are laid
     // out in the channel order the GEMM's nibble unpack gives the weights).
     const int qmax = bits == 4 ? 7 : 127;
     const StoreFmt fmt = bits == 4 ? StoreFmt::Int8Perm : StoreFmt::Int8;
+    // a multiplier that is block^-1/2 in every channel is passed as "none": same products, no vector to stage
+    const float* mult = W->mult_const ? nullptr : W->mult_g;
     const cudaError_t pe =
-        gate >= 0 ? launch_gated_transform_quantize(x, xt, M, W->K, ldx, gate, W->mult_g, block_norm(W->block), W->fold_after,
+        gate >= 0 ? launch_gated_transform_quantize(x, xt, M, W->K, ldx, gate, mult, block_norm(W->block), W->fold_after,
                                                     W->block, qmax, clip_ratio, fmt, ws.a8, ws.delta, s)
-                  : launch_transform_quantize(x, xt, M, W->K, ldx, W->mult_g, block_norm(W->block), W->fold_after, W->block,
+                  : launch_transform_quantize(x, xt, M, W->K, ldx, mult, block_norm(W->block), W->fold_after, W->block,
                                               qmax, clip_ratio, fmt, ws.a8, ws.delta, s);
     if (pe != cudaSuccess) return FQ_ERR_CUDA;
     if (g_profile_mark != nullptr) {
@@ -167,8 +251,6 @@ fq_status linear_impl(const void* x, fq_dtype xt, int64_t M, int64_t ldx, const 
     GemmOut out;
     out.y = y; out.yt = yt; out.ldy = ldy; out.a_delta = ws.delta;
     // 4-bit weights are expanded to 16*code on chip: accumulator = 16 * integer sum.
-    size_t scratch_bytes = 0;
-    void* scratch = scratch_of(workspace, ws_bytes, M, W->K, &scratch_bytes);
     return launch_gemm(ws.a8, M, *W, bits == 4 ? 4 : 0, out, scratch, scratch_bytes, s);
 }
 
@@ -217,6 +299,7 @@ fq_status fold_impl(const void* Wsrc, fq_dtype wt, int64_t N, int64_t K, int64_t
     }
     const float cn = block_norm(hadamard_block);
     w->fold_after = after;
+    w->mult_const = smooth == nullptr;
     // fold-after: the two vectors are p itself (offline side) and 1/p (runtime side), without the block norm
     bool ok = launch_multipliers(smooth, K, after ? 1.0f : cn, mult_w, w->mult_g, s) == cudaSuccess;
     ok = ok && launch_transform_quantize(Wsrc, wt, N, K, ldw, mult_w, cn, after, hadamard_block, bits == 4 ? 7 : 127,
@@ -346,6 +429,7 @@ fq_status fq_fold_weights_gptq(const void* Wsrc, fq_dtype wt, int64_t N, int64_t
     }
     const float cn = block_norm(hadamard_block);
     const int qmax = bits == 4 ? 7 : 127;
+    w->mult_const = smooth == nullptr;
     ok = cudaMemsetAsync(bad, 0, sizeof(int), s) == cudaSuccess;
     ok = ok && launch_multipliers(smooth, K, cn, mult_w, w->mult_g, s) == cudaSuccess;
     // per-output-channel steps: those of the round-to-nearest fold (its codes are overwritten by the sweep)
@@ -439,7 +523,7 @@ int fq_weights_fold_after(const fq_weights* wp) {
 fq_status fq_weights_destroy(fq_weights* wp) {
     Weights* w = reinterpret_cast<Weights*>(wp);
     if (!w) return FQ_OK;
-    cudaFree(w->codes); cudaFree(w->w_scale); cudaFree(w->bias); cudaFree(w->mult_g); cudaFree(w->tile_counters);
+    cudaFree(w->codes); cudaFree(w->w_scale); cudaFree(w->bias); cudaFree(w->mult_g);
     delete w;
     return FQ_OK;
 }
@@ -489,6 +573,7 @@ fq_status import_impl(const void* codes, const float* w_scale, const float* mult
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const size_t code_bytes = (size_t)N * (size_t)K * bits / 8;
     w->fold_after = after && mult_g != nullptr;
+    w->mult_const = mult_g == nullptr;
     bool ok = true;
     if (N > 0) {
         ok = ok && cudaMemcpyAsync(w->codes, codes, code_bytes, cudaMemcpyDeviceToDevice, s) == cudaSuccess;
@@ -538,6 +623,7 @@ fq_status fq_weights_set_multiplier(fq_weights* wp, const float* mult, void* str
     else
         ok = launch_multipliers(nullptr, w->K, block_norm(w->block), nullptr, w->mult_g, s) == cudaSuccess;
     ok = ok && cudaStreamSynchronize(s) == cudaSuccess;        // the handle is complete when the call returns
+    if (ok) w->mult_const = mult == nullptr;
     return ok ? FQ_OK : FQ_ERR_CUDA;
 }
 
@@ -686,6 +772,14 @@ fq_status fq_gemm_simt(const void* a_codes, const float* a_delta, int64_t M, con
 fq_status fq_profile_mark(void* event) {
     g_profile_mark = static_cast<cudaEvent_t>(event);
     return FQ_OK;
+}
+
+fq_status fq_watchdog_selftest(uint64_t limit_ns, void* stream) {
+    fq_status st = check_arch();
+    if (st != FQ_OK) return st;
+    if (limit_ns < 1000ull) limit_ns = 1000ull;
+    if (limit_ns > 100000000ull) limit_ns = 100000000ull;
+    return launch_watchdog_selftest(limit_ns, static_cast<cudaStream_t>(stream)) == cudaSuccess ? FQ_OK : FQ_ERR_CUDA;
 }
 
 fq_status fq_device_status(uint32_t* detail) {

@@ -22,7 +22,8 @@ struct Weights {
     float* mult_g = nullptr;    // [K] runtime multiplier (1/s_c) * block^-1/2
     bool fold_after = false;    // mult_g is the post-rotation multiplier 1/p (T = P^-1 R) instead of (1/s) block^-1/2
     bool composite = false;     // folded with a stored composite rotation: the prologue is fq_quantize_act_composite
-    uint32_t* tile_counters = nullptr;   // [1024] zero between launches: slices of a tile finished (K split)
+    bool mult_const = false;    // mult_g holds the constant block^-1/2 in every entry (no smoothing, or the diagonal absorbed
+                                // upstream): the fused calls then run the prologue without the per-channel vector
     CUtensorMap tmap;           // TMA view of `codes` for the GEMM's weight operand
     bool tmap_valid = false;
     CUtensorMap tmap_stream;    // 4-bit weights: view for the short-batch streaming kernel (32 rows x 128 bytes)
@@ -30,6 +31,13 @@ struct Weights {
 };
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// Facts about the current device and per-kernel launch set-up, looked up once and remembered (an eager call
+// otherwise pays several runtime queries per launch).
+int device_sm_count();                                              // multiprocessors of the current device
+int device_cc_major();                                              // compute-capability major, -1 on error
+cudaError_t ensure_dynamic_smem(const void* kernel, size_t bytes);  // opt a kernel in to `bytes` of dynamic shared memory
+int max_resident_blocks(const void* kernel, int threads);           // thread blocks of a kernel one SM holds (no dynamic smem)
 
 // Launch with programmatic stream serialization (the kernel must call griddep_wait() before its first
 // global-memory access) and, optionally, a thread-block cluster along x.
@@ -126,6 +134,9 @@ fq_status launch_gemm_tcgen05(const int8_t* a8, int64_t M, const Weights& W, int
 fq_status launch_gemm(const int8_t* a8, int64_t M, const Weights& W, int acc_shift, const GemmOut& out,
                       void* scratch, size_t scratch_bytes, cudaStream_t stream);
 size_t gemm_scratch_bytes(int64_t M, int64_t N, int64_t K, int bits);
+// Enqueue whatever the GEMM of this shape needs cleared in `scratch` (the K split's tile counters).  Called by every
+// entry point ahead of the call's first kernel; a launch_gemm on the same scratch must follow on the same stream.
+fq_status gemm_prepare(int64_t M, const Weights& W, void* scratch, size_t scratch_bytes, cudaStream_t stream);
 
 // cuTensorMapEncodeTiled through the runtime's driver entry point (no link-time libcuda dependency).
 // dims/box innermost first; strides_bytes has rank-1 entries (dimension 0 is contiguous).
@@ -161,5 +172,7 @@ fq_status build_weight_tmap(Weights& W);
 // Device watchdog word (see fq_device_status).
 cudaError_t read_and_clear_watchdog(uint32_t* word);
 uint32_t* watchdog_device_ptr();
+// One-warp kernel whose bounded wait is certain to expire after limit_ns (see fq_watchdog_selftest).
+cudaError_t launch_watchdog_selftest(uint64_t limit_ns, cudaStream_t stream);
 
 }  // namespace fq

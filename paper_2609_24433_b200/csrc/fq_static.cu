@@ -60,17 +60,20 @@ extern "C" fq_status fq_linear_w4a4_static(const void* x, fq_dtype xt, int64_t M
     if (W->bits != 4 || W->composite) return FQ_ERR_UNSUPPORTED;
     if (!(clip_ratio > 0.0f && clip_ratio <= 1.0f)) return FQ_ERR_INVALID_ARG;
     if ((xt != FQ_F32 && xt != FQ_BF16) || (yt != FQ_F32 && yt != FQ_BF16)) return FQ_ERR_INVALID_ARG;
-    if (M == 0 || W->N == 0) return FQ_OK;
+    if (M == 0 || W->N == 0) {
+        // A call without tokens still performs the one-time set-up for the current device (it loads the
+        // module that holds the scratch and looks the address up), so it can serve as the start-up call.
+        unsigned char* warm = nullptr;
+        return device_cc_major() == 10 ? scratch_on_current_device(&warm) : FQ_OK;
+    }
     // The built-in scratch is fixed: refuse anything that does not fit instead of overrunning it.
     if (M > FQ_STATIC_MAX_TOKENS_ || (size_t)M * (size_t)W->K > kCodeBytes) return FQ_ERR_NOMEM;
     if (!x || !y || ldx < W->K || ldy < W->N) return FQ_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(x) & 15u) || (reinterpret_cast<uintptr_t>(y) & 15u) || ldx % 8 != 0 || ldy % 8 != 0)
         return FQ_ERR_ALIGNMENT;
     if (W->K > 32768) return FQ_ERR_UNSUPPORTED;
-    int dev = 0, major = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess ||
-        cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess)
-        return FQ_ERR_CUDA;
+    const int major = device_cc_major();
+    if (major < 0) return FQ_ERR_CUDA;
     if (major != 10) return FQ_ERR_ARCH;
 
     unsigned char* scratch = nullptr;
@@ -80,7 +83,7 @@ extern "C" fq_status fq_linear_w4a4_static(const void* x, fq_dtype xt, int64_t M
     float* delta = reinterpret_cast<float*>(scratch + kCodeBytes);   // [M] steps,    rows < M rewritten below
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const float cnorm = (float)(1.0 / sqrt((double)W->block));
-    if (launch_transform_quantize(x, xt, M, W->K, ldx, W->mult_g, cnorm, W->fold_after, W->block, 7, clip_ratio, StoreFmt::Int8Perm, a8,
+    if (launch_transform_quantize(x, xt, M, W->K, ldx, W->mult_const ? nullptr : W->mult_g, cnorm, W->fold_after, W->block, 7, clip_ratio, StoreFmt::Int8Perm, a8,
                                   delta, s) != cudaSuccess)
         return FQ_ERR_CUDA;
     GemmOut out;

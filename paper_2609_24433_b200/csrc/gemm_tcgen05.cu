@@ -38,10 +38,8 @@
 // Every mbarrier wait is bounded by wall-clock time; on expiry the CTA records a
 // code in the watchdog word, stops issuing work, and still frees its TMEM.
 #include <cuda_bf16.h>
-#if defined(FQ_GEMM_TRACE) || defined(FQ_GEMM_DEV)
-#include <cstdio>
-#include <cstdlib>
-#endif
+
+#include <mutex>
 
 #include "fq_common.cuh"
 #include "ptx_sm100.cuh"
@@ -52,9 +50,40 @@ namespace fq {
 __device__ uint32_t g_watchdog_word = 0;
 
 uint32_t* watchdog_device_ptr() {
+    // the symbol's address differs per device: looked up once for each
+    static std::mutex mutex;
+    static uint32_t* addr[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return nullptr;
+    const bool cached = dev >= 0 && dev < 64;
+    std::lock_guard<std::mutex> lock(mutex);
+    if (cached && addr[dev] != nullptr) return addr[dev];
     uint32_t* p = nullptr;
     if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_watchdog_word) != cudaSuccess) return nullptr;
+    if (cached) addr[dev] = p;
     return p;
+}
+
+// Self-test of the bounded-wait machinery: one warp waits, with the ordinary wait routine and a caller-chosen
+// limit, on a barrier that nobody ever arrives at.  The wait must give up, record its code in the watchdog word
+// and let the kernel end normally.
+__global__ void watchdog_selftest_kernel(uint32_t* watchdog, uint64_t limit_ns) {
+    __shared__ uint64_t s_bar;
+    __shared__ int s_abort;
+    if (threadIdx.x == 0) {
+        s_abort = 0;
+        mbar_init(smem_u32(&s_bar), 1);
+        fence_mbarrier_init();
+    }
+    __syncthreads();
+    mbar_wait_all(smem_u32(&s_bar), 0u, &s_abort, watchdog, 0x400u, false, limit_ns);
+}
+
+cudaError_t launch_watchdog_selftest(uint64_t limit_ns, cudaStream_t stream) {
+    uint32_t* wd = watchdog_device_ptr();
+    if (!wd) return cudaErrorUnknown;
+    watchdog_selftest_kernel<<<1, 32, 0, stream>>>(wd, limit_ns);
+    return cudaGetLastError();
 }
 
 cudaError_t read_and_clear_watchdog(uint32_t* word) {
@@ -82,20 +111,8 @@ constexpr int kColsW = kBlockK / 4;     // TMEM columns of one unpacked k-block 
 constexpr int kMaxStages = 16;
 constexpr int kMaxStagesP = 16;
 constexpr int kMaxSplit = 16;          // K slices per tile, at most
-constexpr int kMaxSplitTiles = 1024;   // tiles of a launch that splits K (one counter each in the weight handle)
-
-// Timeline hooks for kernel development: with -DFQ_GEMM_TRACE the first CTA records clock64() at
-// the marked points of the first 1024 k-blocks (agent 0 activation producer, 2 unpack, 3 MMA
-// issuer) and fq_debug_trace() copies the table out.  Compiled out by default.
-#ifdef FQ_GEMM_TRACE
-__device__ unsigned long long g_trace[4 * 1024 * 4];
-#define FQ_TRACE(agent, n, e)                                                                   \
-    do {                                                                                        \
-        if (blockIdx.x == 0 && lane == 0 && (n) < 1024) g_trace[((agent) * 1024 + (n)) * 4 + (e)] = clock64(); \
-    } while (0)
-#else
-#define FQ_TRACE(agent, n, e) do { } while (0)
-#endif
+constexpr int kMaxSplitTiles = 1024;   // tiles of a launch that splits K (one counter each, ahead of the partial sums)
+constexpr size_t kCounterBytes = kMaxSplitTiles * sizeof(uint32_t);
 
 struct Params {
     int64_t M, N, K;
@@ -117,10 +134,8 @@ struct Params {
     int kb_per;          // k-blocks of one work unit (all of K, or K / split)
     int split, split_shift;   // K split: a tile is `split` (power of two) work units, each on a slice of K
     int32_t* partials;   // [tile][slice][bt tokens][128 channels] int32 raw sums of the slices (K split)
-    uint32_t* counters;  // [tile] slices finished so far; zero between launches (K split)
-#if defined(FQ_GEMM_TRACE) || defined(FQ_GEMM_DEV)
-    int dbg;             // development builds: switches that skip parts of the epilogue
-#endif
+    uint32_t* counters;  // [tile] slices finished so far; zeroed by the host before the launch (K split)
+    int delta_vec;       // a_delta is 16-byte aligned: the epilogue may read four steps per load
 };
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
@@ -353,7 +368,6 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     volatile int* abort_flag = &s_abort;
-    if (warp == 1) FQ_TRACE(3, 1023, 0);             // kernel entry
     const uint32_t cta_rank = CTAS == 2 ? cluster_ctarank() : 0u;
     const bool leader = cta_rank == 0;
     // K split (single CTAs only): a tile is `split` work units, unit = tile * split + slice, slice s
@@ -408,16 +422,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     const uint32_t tmem_base = s_tmem_base;
     // Everything above is on-chip setup; from here on global memory is touched (activations written
     // by the kernel before this one, outputs that it may still be reading).
-    if (warp == 1) FQ_TRACE(3, 1023, 1);             // set-up done
     // The weight producers do not wait: a weight handle is complete before any call that uses it
     // is enqueued, so its tiles can stream in while the kernel ahead (the prologue) still runs.
     const bool weight_producer = BITS == 8 ? warp == kFirstUnpackWarp : warp == kFirstUnpackWarp + 4 * kUnpackSets;
-#if defined(FQ_GEMM_TRACE) || defined(FQ_GEMM_DEV)
-    if (!weight_producer || (p.dbg & 8)) griddep_wait();
-#else
     if (!weight_producer) griddep_wait();
-#endif
-    if (warp == 1) FQ_TRACE(3, 1023, 2);             // previous kernel complete
     griddep_launch_dependents();
 
     // work units: (super-tile of 128*CTAS channels) x (token tile) [x K slice]; one unit per CTA or
@@ -447,7 +455,6 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             for (int n = 0; n < total_kb; ++n) {
                 ok = mbar_wait_all_lazy(smem_u32(&s_empty[stage]), phase ^ 1u, abort_flag, p.watchdog, kWdProducer, peek);
                 if (!ok) break;
-                FQ_TRACE(0, n, 0);
                 {   // look at the next stage now: the test's latency hides behind the copy issued below
                     const int s1 = stage + 1 == p.stages ? 0 : stage + 1;
                     const uint32_t ph1 = s1 == 0 ? phase ^ 1u : phase;
@@ -466,7 +473,6 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                         tma_load_2d_pair(smem_a + stage * a_bytes, &map_a, (kb0 + kb) * kBlockK, t0, bar);
                     }
                 }
-                FQ_TRACE(0, n, 1);
                 if (++stage == p.stages) { stage = 0; phase ^= 1u; }
                 if (++kb == k_blocks) {
                     kb = 0;
@@ -493,20 +499,17 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             // in series per k-block would otherwise sit on the issuing warp's critical path.
             bool ready = false;
             int left = my_units * k_blocks;   // k-blocks still to issue
-            [[maybe_unused]] int tn = 0;
             for (int unit = unit0; unit < num_units && ok; unit += unit_step) {
                 ok = mbar_wait_all(smem_u32(&s_acc_empty[acc_stage]), acc_phase ^ 1u, abort_flag, p.watchdog, kWdMmaAcc);
                 if (!ok) break;
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc_stage * p.bt);
                 for (int kb = 0; kb < k_blocks; ++kb) {
-                    FQ_TRACE(3, tn, 0);
                     if (!__all_sync(0xffffffffu, ready)) {
                         ok = mbar_wait_all(smem_u32(&s_full_tma[stage]), phase, abort_flag, p.watchdog, kWdMmaFull);
                         if (ok && BITS == 4)
                             ok = mbar_wait_all(smem_u32(&s_full_w8[wstage]), wphase, abort_flag, p.watchdog, kWdMmaFull);
                         if (!ok) break;
                     }
-                    FQ_TRACE(3, tn, 2);
                     --left;
                     tc_fence_after();
                     const int s1 = stage + 1 == p.stages ? 0 : stage + 1;
@@ -548,8 +551,6 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                                                   peek_bar_w, peek_par_w);
                     }
                     ready = r != 0;
-                    FQ_TRACE(3, tn, 3);
-                    ++tn;
                     stage = s1;
                     phase = ph1;
                     if (BITS == 4) { wstage = w1; wphase = wph1; }
@@ -616,7 +617,6 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                 if (warp == 2 && lane == 0) {
                     const uint32_t done = atomicAdd(p.counters + tile, 1u);
                     *last_slot = done == (uint32_t)(split - 1) ? 1 : 0;
-                    if (*last_slot) p.counters[tile] = 0u;   // every slice has been counted: ready for the next launch
                 }
                 // rendezvous 2: the outcome is written (its slot is reused two tiles later, after both
                 // rendezvous of the next tile)
@@ -642,9 +642,6 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                 const int64_t tc = t0 + c;
                 if (tc >= p.M) break;                    // tokens beyond M: nothing to store (warp-uniform)
                 uint32_t r[16];
-#if defined(FQ_GEMM_TRACE) || defined(FQ_GEMM_DEV)
-                if (p.dbg & 4) continue;
-#endif
                 tmem_ld16(taddr + (uint32_t)c, r);
                 if (split > 1) {
                     int32_t pv[16];
@@ -660,9 +657,6 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
 #pragma unroll
                     for (int i = 0; i < 16; ++i) r[i] += (uint32_t)pv[i];
                 }
-#if defined(FQ_GEMM_TRACE) || defined(FQ_GEMM_DEV)
-                if (p.dbg & 2) { tmem_ld_wait(); if (r[0] == 0x12345678u && r[7] == 0x9abcdef0u) p.watchdog[1] = 1; continue; }
-#endif
                 if (p.out.acc != nullptr) {
                     tmem_ld_wait();
 #pragma unroll
@@ -671,7 +665,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                     continue;
                 }
                 float d[16];
-                if (tc + 16 <= p.M) {
+                if (tc + 16 <= p.M && p.delta_vec) {
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
                         const float4 q = __ldg(reinterpret_cast<const float4*>(p.out.a_delta + tc) + i);
@@ -710,9 +704,6 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                         lo.y = __byte_perm(q0.z, q0.w, 0x5410); hi.y = __byte_perm(q0.z, q0.w, 0x7632);
                         lo.z = __byte_perm(q1.x, q1.y, 0x5410); hi.z = __byte_perm(q1.x, q1.y, 0x7632);
                         lo.w = __byte_perm(q1.z, q1.w, 0x5410); hi.w = __byte_perm(q1.z, q1.w, 0x7632);
-#if defined(FQ_GEMM_TRACE) || defined(FQ_GEMM_DEV)
-                        if ((p.dbg & 1) && lo.x != 0x12345678u) continue;
-#endif
                         if (jj < p.N) {
                             if (tc + 2 * k < p.M) *reinterpret_cast<uint4*>(y + (tc + 2 * k) * p.out.ldy + jj) = lo;
                             if (tc + 2 * k + 1 < p.M) *reinterpret_cast<uint4*>(y + (tc + 2 * k + 1) * p.out.ldy + jj) = hi;
@@ -809,10 +800,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         while (es >= p.stages) { es -= p.stages; eph ^= 1u; }
         for (int n = uset; n < total_kb && ok; n += kUnpackSets) {
             {
-                if ((warp & 3) == 0) FQ_TRACE(2, n, 0);
                 ok = mbar_wait_all(smem_u32(&s_full_p[ps]), pph, abort_flag, p.watchdog, kWdUnpackFull);
                 if (!ok) break;
-                if ((warp & 3) == 0) FQ_TRACE(2, n, 1);
                 const uint32_t src = smem_p + (uint32_t)ps * pk_bytes;     // shared-space address of the stage
                 const uint32_t w_tmem = tmem_base + lane_addr + (uint32_t)(kAccStages * p.bt + ws * kSlotCols);
                 bool slot_free = false;
@@ -844,7 +833,6 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                     if (h == 0) {
                         ok = mbar_wait_all(smem_u32(&s_empty[es]), eph, abort_flag, p.watchdog, kWdUnpackEmpty, slot_free);
                         if (!ok) break;
-                        if ((warp & 3) == 0) FQ_TRACE(2, n, 2);
                         tc_fence_after();
                     }
                     tmem_st32(w_tmem + h * kColsW, o);
@@ -857,7 +845,6 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                     if (CTAS == 1) mbar_arrive(smem_u32(&s_full_w8[ws]));
                     else mbar_arrive_cta(smem_u32(&s_full_w8[ws]), 0);
                 }
-                if ((warp & 3) == 0) FQ_TRACE(2, n, 3);
                 // (every ring has at least kUnpackSets slots: one subtraction brings an index back into range)
                 ps += kUnpackSets;
                 if (ps >= p.stages_p) { ps -= p.stages_p; pph ^= 1u; }
@@ -909,7 +896,6 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     // ------------------------------------------------------------------ teardown
     tc_fence_before();
     __syncthreads();
-    if (warp == 1) FQ_TRACE(3, 1023, 3);             // all roles done
     if (CTAS == 2) cluster_sync_all();              // neither CTA leaves while the other may still signal it
     if (warp == 1) {
         tc_fence_after();
@@ -995,8 +981,7 @@ template <int BITS, int CTAS, bool SPLIT, int ATOMS = 1>
 fq_status launch_variant(const CUtensorMap& map_a, const CUtensorMap& map_w, const Params& p, int grid, size_t smem,
                          int cluster, cudaStream_t stream) {
     auto kern = gemm_tcgen05_kernel<BITS, CTAS, SPLIT, ATOMS>;
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-        return FQ_ERR_CUDA;
+    if (ensure_dynamic_smem(reinterpret_cast<const void*>(kern), smem) != cudaSuccess) return FQ_ERR_CUDA;
     return launch_pdl(kern, (unsigned)grid, (unsigned)(BITS == 4 ? kThreadsW4 : kThreadsW8), smem, stream, (unsigned)cluster,
                       map_a, map_w, p) == cudaSuccess ? FQ_OK : FQ_ERR_CUDA;
 }
@@ -1009,7 +994,7 @@ struct Plan {
     int bt = 0;       // tokens per tile
     int ctas = 1;     // 2: CTA pairs on 256-channel tiles (cta_group::2)
     int split = 1;    // >1: every tile is that many work units, each on a slice of K
-    size_t scratch = 0;   // bytes of int32 partial tiles the split needs
+    size_t scratch = 0;   // bytes of scratch the split needs: the tile counters, then the int32 partial tiles
 };
 
 // Token tile, CTA grouping and K split.  Upper bound of the tile from TMEM: two accumulator stages,
@@ -1045,7 +1030,7 @@ Plan plan_gemm(int64_t M, int64_t N, int64_t K, int bits, int sms, size_t scratc
             for (int sp = 1; sp <= (c == 1 ? kMaxSplit : 1); sp *= 2) {
                 if (sp > 1 && (kb % sp != 0 || kb / sp < 2 || units > kMaxSplitTiles || units * sp > 4 * (int64_t)sms)) continue;
                 const int64_t kb_per = kb / sp;
-                const size_t scratch = sp > 1 ? (size_t)units * sp * kTileN * b * sizeof(int32_t) : 0;
+                const size_t scratch = sp > 1 ? kCounterBytes + (size_t)units * sp * kTileN * b * sizeof(int32_t) : 0;
                 if (scratch > scratch_avail) continue;
                 const int slots = sms / c;
                 const double unit_cost = (double)kb_per * per_kb + 16.0 * b + 1000.0 + (sp > 1 ? 1500.0 + 70.0 * b + 8.0 * b * (sp - 1) : 0.0);
@@ -1060,14 +1045,19 @@ Plan plan_gemm(int64_t M, int64_t N, int64_t K, int bits, int sms, size_t scratc
     return best;
 }
 
-int device_sms() {
-    int dev = 0, sms = 148;
-    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    else (void)cudaGetLastError();
-    return sms > 0 ? sms : 148;
-}
-
 }  // namespace
+
+// A launch that splits K counts the finished slices of every tile in counters at the head of the scratch.
+// They are cleared here, by a memset node enqueued AHEAD of the call's first kernel (between the prologue
+// and the GEMM it would break the programmatic overlap of the two): each call starts from zero whatever an
+// earlier call -- even one that gave up on an expired wait -- left there, and nothing in the weight handle
+// changes at run time.
+fq_status gemm_prepare(int64_t M, const Weights& W, void* scratch, size_t scratch_bytes, cudaStream_t stream) {
+    if (M <= 0 || W.N == 0 || scratch == nullptr || gemm_stream_applies(M, W)) return FQ_OK;
+    const Plan plan = plan_gemm(M, W.N, W.K, W.bits, device_sm_count(), scratch_bytes);
+    if (plan.split <= 1) return FQ_OK;
+    return cudaMemsetAsync(scratch, 0, kCounterBytes, stream) == cudaSuccess ? FQ_OK : FQ_ERR_CUDA;
+}
 
 fq_status launch_gemm(const int8_t* a8, int64_t M, const Weights& W, int acc_shift, const GemmOut& out, void* scratch,
                       size_t scratch_bytes, cudaStream_t stream) {
@@ -1079,7 +1069,7 @@ fq_status launch_gemm(const int8_t* a8, int64_t M, const Weights& W, int acc_shi
 
 size_t gemm_scratch_bytes(int64_t M, int64_t N, int64_t K, int bits) {
     if (M <= 0 || N <= 0 || K <= 0) return 0;
-    return plan_gemm(M, N, K, bits, device_sms(), (size_t)-1).scratch;
+    return plan_gemm(M, N, K, bits, device_sm_count(), (size_t)-1).scratch;
 }
 
 fq_status launch_gemm_tcgen05(const int8_t* a8, int64_t M, const Weights& W, int acc_shift, const GemmOut& out,
@@ -1089,25 +1079,13 @@ fq_status launch_gemm_tcgen05(const int8_t* a8, int64_t M, const Weights& W, int
 
     Params p{};
     p.M = M; p.N = W.N; p.K = W.K;
-    const int sms = device_sms();
-    Plan plan = plan_gemm(M, W.N, W.K, W.bits, sms, scratch ? scratch_bytes : 0);
-    int bt = plan.bt, ctas = plan.ctas, split = plan.split;
-#if defined(FQ_GEMM_TRACE) || defined(FQ_GEMM_DEV)
-    if (const char* e = getenv("FQ_BT")) { bt = atoi(e); split = 1; }       // development builds: force the token tile
-    if (const char* e = getenv("FQ_PAIR")) { ctas = atoi(e); split = 1; }   // ... and single CTAs or pairs
-    if (const char* e = getenv("FQ_SPLIT")) {                               // ... and the K split, if it is a legal one
-        const int sp = atoi(e);
-        const int64_t kb = (W.K + kBlockK - 1) / kBlockK;
-        const int64_t tiles = ((W.N + kTileN - 1) / kTileN) * ((M + bt - 1) / bt);
-        const bool legal = ctas == 1 && sp >= 1 && sp <= kMaxSplit && (sp & (sp - 1)) == 0 && kb % sp == 0 && kb / sp >= 2 &&
-                           tiles <= kMaxSplitTiles && scratch != nullptr &&
-                           (size_t)tiles * sp * kTileN * bt * sizeof(int32_t) <= scratch_bytes;
-        split = legal ? sp : 1;
-    }
-    if (getenv("FQ_PLAN_PRINT")) fprintf(stderr, "plan: M=%lld N=%lld K=%lld bits=%d -> bt=%d ctas=%d split=%d\n", (long long)M, (long long)W.N, (long long)W.K, W.bits, bt, ctas, split);
-#endif
+    const int sms = device_sm_count();
+    const Plan plan = plan_gemm(M, W.N, W.K, W.bits, sms, scratch ? scratch_bytes : 0);
+    const int bt = plan.bt, ctas = plan.ctas, split = plan.split;
     p.split = split;
-    p.partials = static_cast<int32_t*>(scratch);
+    p.counters = static_cast<uint32_t*>(scratch);            // cleared by gemm_prepare()
+    p.partials = reinterpret_cast<int32_t*>(static_cast<uint8_t*>(scratch) + kCounterBytes);
+    p.delta_vec = (reinterpret_cast<uintptr_t>(out.a_delta) & 15u) == 0 ? 1 : 0;
     p.bt = bt;
     p.m_tiles = (int)((M + bt - 1) / bt);
     p.n_tiles = (int)((W.N + kTileN * ctas - 1) / (kTileN * ctas));
@@ -1117,18 +1095,12 @@ fq_status launch_gemm_tcgen05(const int8_t* a8, int64_t M, const Weights& W, int
     p.out = out;
     p.watchdog = watchdog_device_ptr();
     if (!p.watchdog) return FQ_ERR_CUDA;
-#if defined(FQ_GEMM_TRACE) || defined(FQ_GEMM_DEV)
-    p.dbg = getenv("FQ_DBG") ? atoi(getenv("FQ_DBG")) : 0;
-#endif
     // 4-bit weights, single CTAs, token tiles of at most 128: two 128-channel atoms per pipeline stage (the
     // accumulators of longer tiles leave no room for TMEM slots twice as wide).  Needs whole atoms (K a multiple
     // of 128) and, with a K split, slices of whole stages.
     const int64_t kb128 = (W.K + kBlockK - 1) / kBlockK;
     int atoms = (W.bits == 4 && ctas == 1 && bt <= 128 && W.K % kBlockK == 0 && (split == 1 || kb128 % (2 * split) == 0)) ? 2 : 1;
     if (atoms == 2 && bt <= 64 && kb128 >= 4 * split && (split == 1 || kb128 % (4 * split) == 0)) atoms = 4;   // four for the shortest tiles
-#if defined(FQ_GEMM_TRACE) || defined(FQ_GEMM_DEV)
-    if (getenv("FQ_ATOMS") && atoi(getenv("FQ_ATOMS")) == 1) atoms = 1;
-#endif
     // 4-bit weights: every TMEM column the accumulators leave free becomes unpacked-weight ring
     int stages_w = W.bits == 4 ? (512 - kAccStages * bt) / (kColsW * atoms) : 0;
     if (stages_w > kMaxStagesW) stages_w = kMaxStagesW;
@@ -1180,7 +1152,6 @@ fq_status launch_gemm_tcgen05(const int8_t* a8, int64_t M, const Weights& W, int
     p.units_rem = num_units % clusters;
     p.kb_per = (int)((kb128 + atoms - 1) / atoms) / split;      // stages per unit; the planner only picks splits that divide it
     p.split_shift = split == 1 ? 0 : (split == 2 ? 1 : (split == 4 ? 2 : (split == 8 ? 3 : 4)));
-    p.counters = W.tile_counters;
 
     if (W.bits == 4) {
         if (ctas == 2) return launch_variant<4, 2, false>(map_a, W.tmap, p, grid, smem, 2, stream);
@@ -1199,9 +1170,3 @@ fq_status launch_gemm_tcgen05(const int8_t* a8, int64_t M, const Weights& W, int
 }
 
 }  // namespace fq
-
-#ifdef FQ_GEMM_TRACE
-extern "C" int fq_debug_trace(unsigned long long* out) {
-    return (int)cudaMemcpyFromSymbol(out, fq::g_trace, sizeof(fq::g_trace));
-}
-#endif

@@ -347,9 +347,7 @@ weight_stream_kernel(const __grid_constant__ CUtensorMap map_w, const StreamPara
 template <int MODE, int GROUPS>
 cudaError_t launch_stream(const CUtensorMap& map, StreamParams p, cudaStream_t stream) {
     typedef typename std::conditional<MODE == kModeInt, int, float>::type AccT;
-    int dev = 0, sms = 148;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int sms = device_sm_count();
     const size_t part_bytes = (size_t)8 * kRowsCta * (8 * GROUPS + 1) * sizeof(AccT);
     const size_t budget = 227 * 1024 - 1024 /*alignment*/ - 1024 /*static*/ - part_bytes;
     int depth = (int)(budget / kStageBytes);
@@ -360,7 +358,7 @@ cudaError_t launch_stream(const CUtensorMap& map, StreamParams p, cudaStream_t s
     if (!p.watchdog) return cudaErrorUnknown;
     const size_t smem = (size_t)depth * kStageBytes + part_bytes + 1024;
     auto kern = weight_stream_kernel<MODE, GROUPS>;
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), smem);
     if (e != cudaSuccess) return e;
     const int64_t row_groups = (p.N + kRowsCta - 1) / kRowsCta;
     const unsigned grid = (unsigned)(row_groups < sms ? row_groups : sms);
@@ -413,9 +411,6 @@ bool build_stream_tmap(Weights& W) {
 }
 
 bool gemm_stream_applies(int64_t M, const Weights& W) {
-#if defined(FQ_GEMM_TRACE) || defined(FQ_GEMM_DEV)
-    if (getenv("FQ_NO_STREAM")) return false;      // development builds: compare against the tcgen05 kernel
-#endif
     // measured against the tcgen05 kernel: ahead for at most 8 tokens on matrices up to 32 Mi weights and for at
     // most 16 tokens up to 16 Mi
     if (W.bits != 4 || !W.tmap_stream_valid || M < 1 || M > 16) return false;

@@ -79,7 +79,7 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
 // few thousand failed tries (each try may itself suspend the thread for a while), so that the
 // common short wait pays for nothing but the tries.
 static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                            uint32_t* watchdog, uint32_t code) {
+                                            uint32_t* watchdog, uint32_t code, uint64_t limit_ns = kWaitLimitNs) {
     uint64_t t0 = 0;
     for (uint32_t spin = 1;; ++spin) {
         if (mbar_try_wait(bar, parity)) return true;
@@ -87,7 +87,7 @@ static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity
             if (*abort_flag) return false;
             const uint64_t now = global_timer_ns();
             if (t0 == 0) t0 = now;
-            if (now - t0 > kWaitLimitNs) {
+            if (now - t0 > limit_ns) {
                 *abort_flag = 1;
                 atomicOr(watchdog, code);
                 return false;
@@ -96,10 +96,10 @@ static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity
     }
 }
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                          uint32_t* watchdog, uint32_t code) {
+                                          uint32_t* watchdog, uint32_t code, uint64_t limit_ns = kWaitLimitNs) {
     if (mbar_try_wait(bar, parity)) return true;
     if (mbar_try_wait(bar, parity)) return true;
-    return mbar_wait_slow(bar, parity, abort_flag, watchdog, code);
+    return mbar_wait_slow(bar, parity, abort_flag, watchdog, code, limit_ns);
 }
 // Warp-converged wait: every lane polls the same barrier, the result is made warp-uniform.
 // Roles that hand work over through barriers run their loops with the whole warp converged and
@@ -108,9 +108,10 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
 // `peeked` is the result of an earlier mbar_test_wait on the same phase: when it was already true
 // the wait costs nothing.
 __device__ __forceinline__ bool mbar_wait_all(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                              uint32_t* watchdog, uint32_t code, bool peeked = false) {
+                                              uint32_t* watchdog, uint32_t code, bool peeked = false,
+                                              uint64_t limit_ns = kWaitLimitNs) {
     if (__all_sync(0xffffffffu, peeked)) return true;
-    const bool ok = mbar_wait(bar, parity, abort_flag, watchdog, code);
+    const bool ok = mbar_wait(bar, parity, abort_flag, watchdog, code, limit_ns);
     return __all_sync(0xffffffffu, ok);
 }
 // Converged wait for roles that run far ahead of their consumer (TMA producers behind a full ring): between

@@ -27,7 +27,7 @@ EXPORTS = [
     "fq_fold_weights_after", "fq_weights_fold_after", "fq_weights_import_after", "fq_quantize_act_after",
     "fq_weights_set_multiplier", "fq_weights_scale_outputs", "fq_linear_w4a16",
     "fq_fold_weights_composite", "fq_quantize_act_composite", "fq_weights_composite", "fq_fold_weights_gptq",
-    "fq_quantize_act_gated", "fq_linear_gated",
+    "fq_quantize_act_gated", "fq_linear_gated", "fq_watchdog_selftest",
 ]
 
 _lib = None
@@ -423,6 +423,12 @@ def profile_mark(event: Optional[torch.cuda.Event]):
     if event is not None and not event.cuda_event:
         event.record()      # torch creates the underlying cudaEvent_t lazily, on its first record
     _check(lib().fq_profile_mark(ctypes.c_void_p(0 if event is None else event.cuda_event)), "fq_profile_mark")
+
+
+def watchdog_selftest(limit_ns: int = 2_000_000):
+    """Enqueue the one-warp kernel whose bounded wait is certain to expire after ``limit_ns``; the next
+    device_status() then reports ERR_TIMEOUT once."""
+    _check(lib().fq_watchdog_selftest(ctypes.c_uint64(limit_ns), _stream()), "fq_watchdog_selftest")
 
 
 def device_status() -> Tuple[int, int]:

@@ -20,6 +20,39 @@ def _watchdog_clean():
     assert st == fq.OK, f"device wait watchdog fired: {word:#x}"
 
 
+def fused_workspace(ws: torch.Tensor, M: int, K: int, bits: int):
+    """What the one-call entry points leave in the caller's workspace between their two kernels: the
+    activation codes as one int8 per code ([M, K]; at 4 bits every group of 8 channels is stored even
+    channels first: c0 c2 c4 c6 c1 c3 c5 c7) and, 256-byte aligned behind them, the per-token steps.
+    Returns (codes [M, K] int32 in natural channel order, steps as uint32 bit patterns)."""
+    raw = ws[:M * K].view(torch.int8).view(M, K).cpu().numpy().astype(np.int32)
+    if bits == 4:
+        g = raw.reshape(M, K // 8, 8)
+        nat = np.empty_like(g)
+        nat[:, :, 0::2] = g[:, :, 0:4]
+        nat[:, :, 1::2] = g[:, :, 4:8]
+        raw = nat.reshape(M, K)
+    off = (M * K + 255) // 256 * 256
+    delta = ws[off:off + 4 * M].view(torch.float32).cpu().numpy()
+    return raw, delta.view(np.uint32)
+
+
+def assert_fused_stages(x_dev, h, clip, ydt, want_codes, want_delta, what=""):
+    """The one-call path (its own prologue instantiations: int8 codes in the GEMM's channel order) against the
+    oracle's codes and steps bit for bit, and its output against the two-call route bit for bit: the same
+    integer sums scaled by an exact power of two, so nothing may differ."""
+    M, K = x_dev.shape
+    ws = torch.zeros(fq.workspace_bytes(M, h.K, h.N, h.bits), dtype=torch.uint8, device="cuda")
+    y = fq.linear(x_dev, h, clip, ydt, workspace=ws)
+    codes, delta = fused_workspace(ws, M, K, h.bits)
+    assert np.array_equal(delta, want_delta.view(np.uint32)), f"{what}: fused steps differ"
+    assert np.array_equal(codes, oracle.unpack(want_codes, K, h.bits)), f"{what}: fused codes differ"
+    c2, d2 = fq.quantize_act(x_dev, h, h.block, h.bits, clip)
+    y2 = (fq.gemm_w4a4 if h.bits == 4 else fq.gemm_w8a8)(c2, d2, h, ydt)
+    assert torch.equal(y, y2), f"{what}: one-call and two-call outputs differ"
+    return y
+
+
 def make_x(M, K, dtype, seed, frac=0.01):
     site = synth.Site("t", M, K, [("p", 8)], beta=32, bits=4, x_dtype=dtype, outlier_frac=frac)
     return synth.make_site(site, seed, with_weights=False).x
@@ -93,7 +126,8 @@ def test_quantize_act_zero_tiny_and_strided_rows(bits):
 
 
 @pytest.mark.parametrize("bits", [4, 8])
-@pytest.mark.parametrize("M,K,dtype", [(40, 1024, "f32"), (600, 2048, "bf16"), (700, 4096, "f32"), (333, 1024, "bf16")])
+@pytest.mark.parametrize("M,K,dtype", [(40, 1024, "f32"), (600, 2048, "bf16"), (700, 4096, "f32"), (333, 1024, "bf16"),
+                                       (1200, 2048, "bf16"), (1300, 4096, "f32"), (300, 8192, "bf16")])
 def test_quantize_act_exact_ties_round_to_even(bits, M, K, dtype):
     """Every scaled value is an exact half-integer: a fused multiply-add or a different tie rule in
     any kernel variant (register kernel for short batches, streaming kernel for long ones) shows up
@@ -116,6 +150,11 @@ def test_quantize_act_exact_ties_round_to_even(bits, M, K, dtype):
     codes, delta = fq.quantize_act(to_dev(xs, dtype), to_dev(g), 32, bits)
     assert np.array_equal(to_np(delta), want_delta)
     assert np.array_equal(to_np(codes), want_codes)
+    # the same ties through the one-call path, whose prologue instantiations (int8 codes in the GEMM's channel
+    # order) are compiled separately from the canonical-format ones above
+    wq = rng.integers(-q, q + 1, size=(8, K)).astype(np.int32)
+    h = fq.weights_import(to_dev(oracle.pack(wq, bits)), to_dev(np.ones(8, np.float32)), to_dev(g), None, K, 32, bits)
+    assert_fused_stages(to_dev(xs, dtype), h, 1.0, torch.float32, want_codes, want_delta, "exact ties")
 
 
 def test_quantize_act_amplitude_invariance_on_device():
@@ -465,7 +504,7 @@ def run_site(data: synth.SiteData, rows=None, clip=1.0):
     h = fq.fold_weights(to_dev(W), to_dev(s), to_dev(b), site.beta, site.bits)
     ydt = torch.float32 if site.y_dtype == "f32" else torch.bfloat16
     x_dev = to_dev(data.x, site.x_dtype)
-    y = fq.linear(x_dev, h, clip, ydt)
+    y = assert_fused_stages(x_dev, h, clip, ydt, codes_ref, delta_ref, site.name)
     codes, delta = fq.quantize_act(x_dev, h, site.beta, site.bits, clip)
     return dict(h=h, y=y, codes=codes, delta=delta, x=x_dev), dict(y=y_ref, codes=codes_ref, delta=delta_ref,
                                                                   acc=acc_ref, wc=wc, ws=ws, g=g)
@@ -555,7 +594,9 @@ def test_full_size_backbone_sites_sampled_rows_and_second_witness():
     """Full-size backbone layer (gate/up N = 32768, down K = 16384): prologue checked in full,
     outputs checked on sampled token rows, accumulators checked against the dp4a kernel."""
     rows = [0, 1, 127, 128, 207, 208, 415, 500, 623, 624, 799, 815]
-    for site in synth.backbone_layer_sites(True):
+    # selective INT8 layer, then the two sites that differ in the uniform W4A4 layer (o_proj and down_proj at 4 bits:
+    # the latter is the K split on a 128-k-block tile with multi-atom stages)
+    for site in synth.backbone_layer_sites(True) + synth.backbone_layer_sites(False)[1::2]:
         data = synth.make_site(site, seed=2)
         gpu, ref = run_site(data, rows=rows)
         assert np.array_equal(to_np(gpu["codes"]), ref["codes"]), site.name
@@ -585,6 +626,106 @@ def test_sweep_points_sampled_rows(M, KN, block, bits):
     acc = fq.gemm_acc_i32(gpu["codes"], gpu["h"])
     assert np.array_equal(to_np(acc[rows]), ref["acc"])
     assert_close(to_np(gpu["y"][rows]), ref["y"], "bf16", f"sweep M={M} K=N={KN}")
+
+
+@pytest.mark.parametrize("M,KN,block,bits", [(16384, 4096, 64, 4), (4096, 8192, 128, 8)])
+def test_sweep_corners_sampled_rows(M, KN, block, bits):
+    """Two large points of the throughput sweep (the streaming prologue on long batches; CTA pairs at 8 bits):
+    every token's codes and steps, of the canonical call and of the one-call path, against the oracle; accumulators
+    and outputs on sampled rows."""
+    data = synth.make_site(synth.sweep_site(M, KN, KN, block, bits), seed=5)
+    rows = sorted({0, 1, 207, 208, 255, 256, M // 2 + 3, M - 209, M - 2, M - 1})
+    gpu, ref = run_site(data, rows=rows)
+    assert np.array_equal(to_np(gpu["codes"]), ref["codes"])
+    assert np.array_equal(to_np(gpu["delta"]).view(np.uint32), ref["delta"].view(np.uint32))
+    acc = fq.gemm_acc_i32(gpu["codes"], gpu["h"])
+    assert np.array_equal(to_np(acc[rows]), ref["acc"])
+    assert_close(to_np(gpu["y"][rows]), ref["y"], "bf16", f"sweep corner M={M} K=N={KN}")
+
+
+@pytest.mark.parametrize("clip", [1.0, 0.7])
+@pytest.mark.parametrize("M,K,block,bits,dtype", [
+    (64, 2048, 128, 4, "bf16"), (816, 2048, 128, 4, "f32"),            # register kernel
+    (1184, 2048, 128, 4, "bf16"), (1500, 4096, 64, 4, "f32"),          # streaming kernel, 8 rows per SM and more
+    (296, 8192, 256, 4, "bf16"), (400, 16384, 256, 8, "bf16"),         # streaming kernel on long rows
+    (2000, 1024, 32, 8, "bf16"),
+])
+def test_fused_call_integer_stages_both_prologue_kernels(M, K, block, bits, dtype, clip):
+    """The codes and steps that fq_linear_* hands from its prologue to its GEMM, read back from the workspace."""
+    x = make_x(M, K, dtype, seed=M + K)
+    rng = np.random.default_rng(M + K + bits)
+    s = np.exp(rng.uniform(-1, 1, K)).astype(np.float32)
+    W = synth.draw_weights(rng, 72, K)
+    wc, ws, g = oracle.fold_weights(W, "f32", s, block, bits)
+    want_codes, want_delta = oracle.quantize_act(x, dtype, g, block, bits, clip)
+    h = fq.fold_weights(to_dev(W), to_dev(s), None, block, bits)
+    y = assert_fused_stages(to_dev(x, dtype), h, clip, torch.float32, want_codes, want_delta, "fused stages")
+    rows = [0, M // 2, M - 1]
+    sub = oracle.pack(oracle.unpack(want_codes, K, bits)[rows], bits)
+    want_y = oracle.epilogue(oracle.gemm_i32(sub, wc, K, bits), want_delta[rows], ws, np.zeros(72, np.float32), "f32")
+    assert_close(to_np(y[rows]), want_y, "f32", "fused stages")
+    # and without smoothing: the handle's multiplier is the constant block^-1/2, which the one-call path applies
+    # without reading a per-channel vector
+    wc0, ws0, g0 = oracle.fold_weights(W, "f32", None, block, bits)
+    c0, d0 = oracle.quantize_act(x, dtype, g0, block, bits, clip)
+    h0 = fq.fold_weights(to_dev(W), None, None, block, bits)
+    assert_fused_stages(to_dev(x, dtype), h0, clip, torch.bfloat16, c0, d0, "fused stages, constant multiplier")
+
+
+def test_one_handle_three_streams_three_workspaces():
+    """A weight handle is read-only at run time: consumers of one handle on three streams, each with its own
+    workspace (K split included), give what the same calls give one after the other."""
+    rng = np.random.default_rng(12)
+    M, K, N = 64, 8192, 256                     # few tiles, long K: the planner splits K when scratch is there
+    W = synth.draw_weights(rng, N, K)
+    h = fq.fold_weights(to_dev(W), None, None, 128, 4)
+    need = fq.workspace_bytes(M, K, N, 4)
+    assert need > (M * K + 255) // 256 * 256 + 256, "expected split scratch for this shape"
+    xs = [to_dev(make_x(M, K, "bf16", seed=20 + i), "bf16") for i in range(3)]
+    want = [fq.linear(x, h, 1.0, torch.bfloat16) for x in xs]
+    torch.cuda.synchronize()
+    streams = [torch.cuda.Stream() for _ in range(3)]
+    wss = [torch.empty(need, dtype=torch.uint8, device="cuda") for _ in range(3)]
+    for rep in range(5):
+        got = []
+        for x, st, ws in zip(xs, streams, wss):
+            with torch.cuda.stream(st):
+                for _ in range(4):
+                    y = fq.linear(x, h, 1.0, torch.bfloat16, workspace=ws)
+                got.append(y)
+        torch.cuda.synchronize()
+        for a, b in zip(got, want):
+            assert torch.equal(a, b)
+
+
+def test_gemm_accepts_a_step_vector_at_any_float_offset():
+    """a_delta need only be 4-byte aligned: a slice of a longer vector of steps gives what a copy of it gives."""
+    rng = np.random.default_rng(8)
+    M, K, N = 70, 1024, 136
+    h = import_codes(random_codes(rng, N, K, 4), K, 4)
+    a = to_dev(random_codes(rng, M, K, 4))
+    long = torch.rand(M + 8, device="cuda") + 0.5
+    for off in (1, 2, 3, 4):
+        d = long[off:off + M]
+        assert d.data_ptr() % 16 != 0 or off == 4
+        for ydt in (torch.float32, torch.bfloat16):
+            assert torch.equal(fq.gemm_w4a4(a, d, h, ydt), fq.gemm_w4a4(a, d.clone(), h, ydt))
+
+
+def test_bounded_wait_expires_into_the_watchdog_and_the_device_stays_usable():
+    """fq_watchdog_selftest: a wait nobody ends must give up after its limit, surface once as FQ_ERR_TIMEOUT
+    through fq_device_status, and leave the context usable."""
+    assert fq.device_status()[0] == fq.OK
+    fq.watchdog_selftest(2_000_000)                         # 2 ms
+    st, word = fq.device_status()
+    assert st == fq.ERR_TIMEOUT and word == 0x400, (st, hex(word))
+    assert fq.device_status() == (fq.OK, 0)                 # the record was cleared by the read
+    x = to_dev(make_x(50, 1024, "bf16", seed=1), "bf16")
+    h = fq.fold_weights(torch.randn((264, 1024), device="cuda") * 0.02, None, None, 64, 4)
+    y = fq.linear(x, h, 1.0, torch.bfloat16)
+    c, d = fq.quantize_act(x, h, 64, 4)
+    assert torch.equal(y, fq.gemm_w4a4(c, d, h, torch.bfloat16))
+    assert fq.device_status() == (fq.OK, 0)
 
 
 def test_calibration_helpers_match_oracle():
