@@ -7,17 +7,20 @@ o_proj/down_proj at W8A8 and the rest W4A4.  A step is one pass of the whole hot
 one batch: per site the prologue kernel (scale + FWHT + per-token quantization) and the
 tcgen05 integer GEMM with its dequant/bias epilogue.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--no-large-m] [--no-cpu-baseline]
                     [--workload backbone_layer|backbone_layer_w4|backbone_forward|backbone_forward_w4|expert_layer|expert_loop|sweep:M,K,N,block,bits[,after|composite]|w4a16:M,K,N|gptq:N,K,Mc,block]
 
 Prints ONE JSON line (rank 0).  ``--impl reference`` times the CPU oracle on host cores.
+``--gpus N`` without a torchrun environment starts the N ranks itself (one process per GPU).
 """
 from __future__ import annotations
 
 import argparse
 import json
 import os
+import socket
 import statistics
+import subprocess
 import sys
 import threading
 import time
@@ -34,6 +37,8 @@ METRIC = "fused FWHT+quant+W4A4/W8A8 GEMM throughput (whole layer)"
 UNIT = "TOPS"
 ROTATE = 4            # distinct weight/activation sets cycled so that no step finds its operands in L2
 CPU_SAMPLE_ROWS = 512  # token rows the oracle arm processes per step (about 10 s on 8 cores)
+INT8_DATASHEET_TOPS = 4500.0   # dense INT8 tensor rate of the B200 data sheet
+LARGE_M_POINT = (16384, 8192, 8192, 128, 4)   # M, K, N, block, bits of the long-batch record in the default line
 
 
 def layer_ops(sites) -> float:
@@ -104,12 +109,13 @@ class ClockSampler:
 class LayerOnDevice:
     """Folded weights, inputs, outputs and workspace of ROTATE copies of one layer."""
 
-    def __init__(self, sites, seed: int, device):
+    def __init__(self, sites, seed: int, device, rotate: int = 0):
         import torch
         from paper_2609_24433_b200 import fq
         self.sites, self.fq, self.torch = sites, fq, torch
+        self.rotate = rotate if rotate > 0 else ROTATE
         self.sets = []
-        for r in range(ROTATE):
+        for r in range(self.rotate):
             entry = []
             shared = {}          # expert loop: the 18 layers' handles serve all 10 denoising steps
             for i, site in enumerate(sites):
@@ -163,7 +169,7 @@ class LayerOnDevice:
     def step(self, k: int, events=None):
         """One pass of the layer. ``events``: optional list of (e0, mark, e1) per site."""
         fq = self.fq
-        for i, e in enumerate(self.sets[k % ROTATE]):
+        for i, e in enumerate(self.sets[k % self.rotate]):
             if events is not None:
                 e0, mark, e1 = events[i]
                 e0.record()
@@ -192,7 +198,7 @@ class LayerOnDevice:
         inside every site so that single-kernel durations can be read after a replay."""
         torch = self.torch
         self.graphs, self.ev_graphs, self.ev, self.ev_empty = [], [], [], []
-        for r in range(ROTATE):
+        for r in range(self.rotate):
             g = torch.cuda.CUDAGraph()
             with torch.cuda.graph(g):
                 self.step(r)
@@ -225,19 +231,92 @@ class LayerOnDevice:
         gemm = [[] for _ in self.sites]
         empty = []
         for k in range(replays):
-            self.ev_graphs[k % ROTATE].replay()
+            self.ev_graphs[k % self.rotate].replay()
             torch.cuda.synchronize()
-            for i, (e0, mark, e1) in enumerate(self.ev[k % ROTATE]):
+            for i, (e0, mark, e1) in enumerate(self.ev[k % self.rotate]):
                 act[i].append(e0.elapsed_time(mark))
                 gemm[i].append(mark.elapsed_time(e1))
-            p0, p1 = self.ev_empty[k % ROTATE]
+            p0, p1 = self.ev_empty[k % self.rotate]
             empty.append(p0.elapsed_time(p1))
         ov = statistics.mean(empty)
         return ([max(statistics.mean(a) - ov, 1e-6) for a in act], [max(statistics.mean(g) - ov, 1e-6) for g in gemm], ov)
 
+    def site_pair_us(self, i: int, calls: int = 8, replays: int = 5) -> float:
+        """Microseconds per call of site i alone: ``calls`` back-to-back calls (rotating sets) captured as one
+        graph with nothing between the prologue and the GEMM, so the two kernels overlap as they do in a step."""
+        torch = self.torch
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            for c in range(calls):
+                self.run_site(self.sets[c % self.rotate][i])
+        g.replay()
+        torch.cuda.synchronize()
+        start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        start.record()
+        for _ in range(replays):
+            g.replay()
+        end.record()
+        torch.cuda.synchronize()
+        return start.elapsed_time(end) * 1e3 / (calls * replays)
+
     @property
     def launches_per_step(self) -> int:
         return 2 * len(self.sites)
+
+
+def tensor_fractions(tops: float, peaks) -> dict:
+    """One achieved INT8 rate against the three denominators in use: twice the measured bf16 cuBLAS rate, as a
+    burst (a kernel timed alone or in a short region) and sustained (seconds under the power cap) -- dense int8 is
+    nominally 2 x bf16 -- and the data-sheet dense INT8 figure."""
+    return {"frac_burst": round(tops / (2.0 * peaks["bf16_burst"]), 4),
+            "frac_sustained": round(tops / (2.0 * peaks["bf16_sustained"]), 4),
+            "frac_datasheet_4500": round(tops / INT8_DATASHEET_TOPS, 4)}
+
+
+def large_m_record(device, local_rank: int, peaks, seed: int):
+    """The long-batch point of the throughput sweep, measured in the same process as the default step: the
+    integer GEMM against the tensor peak and the prologue against the copy rate, with the clocks seen meanwhile."""
+    import torch
+    M, K, N, beta, bits = LARGE_M_POINT
+    site = synth.sweep_site(M, K, N, beta, bits)
+    layer = LayerOnDevice([site], seed=seed, device=device, rotate=1)     # 268 MB of activations per step: beyond L2
+    for k in range(3):
+        layer.step(k)
+    torch.cuda.synchronize()
+    layer.capture()
+    for _ in range(3):
+        layer.graphs[0].replay()
+    steps = 12
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(local_rank)
+    torch.cuda.synchronize()
+    with sampler:
+        start.record()
+        for _ in range(steps):
+            layer.graphs[0].replay()
+        end.record()
+        torch.cuda.synchronize()
+        t_end = time.time() + 0.4          # keep the same load up long enough for NVML to see it
+        while time.time() < t_end:
+            layer.graphs[0].replay()
+            torch.cuda.synchronize()
+    ms_step = start.elapsed_time(end) / steps
+    act_ms, gemm_ms, ov = layer.kernel_durations(8)
+    ops = 2.0 * M * K * N
+    gemm_tops = ops / (gemm_ms[0] * 1e-3) / 1e12
+    act_bytes = M * K * 2 + M * K + 4 * M
+    act_gbs = act_bytes / (act_ms[0] * 1e-3) / 1e9
+    rec = {"workload": workload_name(f"sweep:{M},{K},{N},{beta},{bits}"), "steps": steps,
+           "us_per_step": round(ms_step * 1e3, 1), "tops_per_step": round(ops / (ms_step * 1e-3) / 1e12, 1),
+           "l2": "268 MB of activations and 268 MB of outputs per step (beyond the 126 MB L2); 32 MB of weights stay resident",
+           "gemm": dict({"us": round(gemm_ms[0] * 1e3, 1), "achieved_tops": round(gemm_tops, 1)}, **tensor_fractions(gemm_tops, peaks)),
+           "prologue": {"us": round(act_ms[0] * 1e3, 1), "bytes": act_bytes, "achieved_gbs": round(act_gbs, 1),
+                        "peak_gbs": peaks["hbm_gbs"], "frac": round(act_gbs / peaks["hbm_gbs"], 4)},
+           "timing": "kernel figures from event-record nodes inside the step graph (they serialise the two kernels)",
+           "clocks": sampler.summary()}
+    del layer
+    torch.cuda.empty_cache()
+    return rec
 
 
 def run_ours(args, rank: int, world: int, local_rank: int):
@@ -313,15 +392,29 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     s = sites[dom]
     gemm_ops = 2.0 * s.M * s.K * s.N_total
     achieved = gemm_ops / (gemm_ms[dom] * 1e-3) / 1e12
-    int8_peak = 2.0 * peaks["bf16_sustained"]     # dense int8 : bf16 = 2 : 1 (4.5 vs 2.25 PFLOP/s nominal)
+    # dense int8 : bf16 = 2 : 1 (4.5 vs 2.25 PFLOP/s nominal).  A timed region of well under a second runs at boost
+    # clocks: the burst figure is its denominator; a region of seconds under the power cap takes the sustained one.
+    short_region = ms_total < 1000.0
+    which = "bf16_burst" if short_region else "bf16_sustained"
+    int8_peak = 2.0 * peaks[which]
     roofline = {"bound": "tensor", "kernel": f"gemm_tcgen05_kernel<{s.bits},1> ({s.name}: M={s.M} K={s.K} N={s.N_total})",
                 "achieved": round(achieved, 1), "peak": round(int8_peak, 1), "unit": "TOP/s",
                 "frac": round(achieved / int8_peak, 4),
-                "peak_source": f"{peaks['source']}: sustained bf16 cuBLAS {peaks['bf16_sustained']} TFLOP/s x 2 (int8:bf16)",
+                "peak_source": f"{peaks['source']}: {'burst' if short_region else 'sustained'} bf16 cuBLAS {peaks[which]} TFLOP/s x 2 "
+                               f"(int8:bf16), chosen because the timed region lasted {ms_total:.1f} ms",
                 "traffic": TRAFFIC_BYTES.get((args.workload, s.name)),
+                "traffic_source": "dram__bytes_read.sum + dram__bytes_write.sum of one launch in an ncu capture of this workload, "
+                                  "taken separately (not re-measured by this run)" if (args.workload, s.name) in TRAFFIC_BYTES else None,
                 "event_node_overhead_us": round(ev_overhead_ms * 1e3, 2),
                 "per_site_us": {sites[i].name: {"prologue": round(act_ms[i] * 1e3, 2), "gemm": round(gemm_ms[i] * 1e3, 2)}
-                                for i in range(min(len(sites), 8))}}
+                                for i in range(min(len(sites), 8))},
+                "per_site_us_note": "from event-record nodes between the kernels of the step graph: the nodes serialise kernels "
+                                    "that otherwise overlap (programmatic dependent launch), so these durations are upper bounds, "
+                                    "`achieved` is a lower bound, and their sum exceeds the step"}
+    roofline.update(tensor_fractions(achieved, peaks))
+    if len(sites) <= 8:
+        roofline["site_us_alone"] = {sites[i].name: round(layer.site_pair_us(i), 2) for i in range(len(sites))}
+        roofline["site_us_alone_note"] = "each site's two kernels replayed back to back on rotating sets, no event nodes"
     act_i = max(range(len(sites)), key=lambda i: act_ms[i])
     sa = sites[act_i]
     act_bytes = sa.M * sa.K * (2 if sa.x_dtype == "bf16" else 4) + sa.M * sa.K + 4 * sa.M
@@ -338,14 +431,14 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         "ms_per_step": round(ms_per_step, 5), "us_per_layer": round(ms_per_step * 1e3, 2),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int8/int4 codes, int32 accumulate, f32 transform",
         "data": "synthetic", "impl": "ours",
-        "config": {"workload": workload_name(args.workload), "M": sites[0].M,
-                   "sites": {s.name: {"K": s.K, "N": s.N_total, "bits": s.bits, "block": s.beta} for s in sites[:8]},
-                   "n_sites": len(sites), "ops_per_step": ops, "parallelism": "replicas only (one batch per GPU, no collective)",
-                   "l2": f"{ROTATE} rotating weight+activation sets (> 126 MB L2 in total), no flush kernel",
-                   "launch": "one CUDA-graph replay per step"},
+        "config": bench_config(args.workload, sites),
         "clocks": sampler.summary(note), "e2e": e2e, "gpu_launches": layer.launches_per_step * K,
         "roofline": roofline,
     }
+    if world == 1 and args.workload == "backbone_layer" and not args.no_large_m:
+        del layer
+        torch.cuda.empty_cache()
+        out["large_m"] = large_m_record(device, local_rank, peaks, seed=5)
     if rank == 0:
         if world == 1 and not args.no_cpu_baseline:
             out["cpu_baseline"] = cpu_baseline(args.workload, steps=1)
@@ -628,7 +721,7 @@ def run_gptq(args, rank: int, world: int, local_rank: int):
 
 
 # ------------------------------------------------------------------- oracle arm ----
-def cpu_baseline(workload: str, steps: int):
+def cpu_baseline(workload: str, steps: int, warmup: int = 0):
     """The CPU oracle, as it stands, on a bounded sample of the same workload."""
     import oracle
     sites = workload_sites(workload)
@@ -651,7 +744,7 @@ def cpu_baseline(workload: str, steps: int):
             wc, ws, g = oracle.fold_weights(W, "f32", smooth, site.beta, site.bits)      # offline, untimed
         prepared.append((site, np.ascontiguousarray(data.x[:rows]), g, wc, ws, b, rot))
     times = []
-    for _ in range(steps):
+    for it in range(warmup + steps):
         t0 = time.perf_counter()
         for site, x, g, wc, ws, b, rot in prepared:
             if site.composite:
@@ -662,13 +755,27 @@ def cpu_baseline(workload: str, steps: int):
                 oracle.epilogue(oracle.gemm_i32(ac, wc, site.K, site.bits), ad, ws, b, site.y_dtype)
             else:
                 oracle.linear(x, site.x_dtype, g, site.beta, site.bits, 1.0, wc, ws, b, site.y_dtype)
-        times.append(time.perf_counter() - t0)
+        if it >= warmup:
+            times.append(time.perf_counter() - t0)
     ops = sum(2.0 * rows * s.K * s.N_total for s in sites)
     dt = statistics.mean(times)
     return {"value": round(ops / dt / 1e12, 6), "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
             "sample": f"{rows} of {sites[0].M} token rows through all {len(sites)} sites "
                       f"(prologue + integer GEMM + epilogue, all N), {dt:.2f} s per step",
             "seconds_per_step": round(dt, 3)}
+
+
+def bench_config(workload: str, sites) -> dict:
+    """The `config` object of the JSON line: the workload and how the GPU arm stages and launches it.  Both arms
+    print the same object (the oracle arm runs a bounded sample of this workload; its `cpu_baseline.sample` says
+    which)."""
+    rotate = 1 if workload in ("backbone_forward", "backbone_forward_w4", "expert_loop") else ROTATE
+    return {"workload": workload_name(workload), "M": sites[0].M,
+            "sites": {s.name: {"K": s.K, "N": s.N_total, "bits": s.bits, "block": s.beta} for s in sites[:8]},
+            "n_sites": len(sites), "ops_per_step": layer_ops(sites),
+            "parallelism": "replicas only (one batch per GPU, no collective)",
+            "l2": f"{rotate} rotating weight+activation sets (> 126 MB L2 in total), no flush kernel",
+            "launch": "one CUDA-graph replay per step"}
 
 
 def run_reference(args):
@@ -700,23 +807,24 @@ def run_reference(args):
               flush=True)
         return
     sites = workload_sites(args.workload)
-    steps = max(1, min(args.steps, 5))
-    base = cpu_baseline(args.workload, steps=steps)
+    # Exactly --steps timed steps after --warmup untimed ones, like the GPU arm; the per-step sample of token rows
+    # shrinks with the number of steps so that the whole run stays within about two minutes of host time.
+    steps, warm = max(1, args.steps), max(0, args.warmup)
+    CPU_SAMPLE_ROWS = max(16, min(CPU_SAMPLE_ROWS, sites[0].M, CPU_SAMPLE_ROWS * 12 // (steps + warm) // 16 * 16))
+    base = cpu_baseline(args.workload, steps=steps, warmup=warm)
     out = {"metric": METRIC, "value": base["value"], "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
-           "warmup": 0, "ms_per_step": round(base["seconds_per_step"] * 1e3, 2), "higher_is_better": True,
+           "warmup": warm, "ms_per_step": round(base["seconds_per_step"] * 1e3, 2), "higher_is_better": True,
            "scaling": "weak", "vs_baseline": None, "dtype": "int8/int4 codes, int32 accumulate, f32 transform",
            "data": "synthetic", "impl": "reference",
-           "config": {"workload": workload_name(args.workload), "M": sites[0].M,
-                      "sites": {s.name: {"K": s.K, "N": s.N_total, "bits": s.bits, "block": s.beta} for s in sites[:8]},
-                      "n_sites": len(sites)},
+           "config": bench_config(args.workload, sites),
            "cpu_baseline": base,
            "e2e": {"value": base["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(out), flush=True)
 
 
 # -------------------------------------------------------------------- workloads ----
-# DRAM bytes per launch of the dominant kernel, from the ncu captures summarised under profiles/.
-TRAFFIC_BYTES = {("backbone_layer", "gate_up"): 41771776}   # profiles/gemm_tcgen05_w4_gate_up_m816.md
+# DRAM bytes per launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture).
+TRAFFIC_BYTES = {("backbone_layer", "gate_up"): 41771776}
 
 
 def workload_sites(name: str):
@@ -759,6 +867,44 @@ def workload_name(name: str) -> str:
             "expert_layer": "action-expert layer, M=50, width 1024, MLP 4096, W4A4, block 64"}[name]
 
 
+def spawn_ranks(args) -> int:
+    """`--gpus N` outside a torchrun environment: start the N ranks here, one process per GPU, the way a launcher
+    would (rendezvous on 127.0.0.1).  Refuses loudly when the machine does not have N GPUs."""
+    if not args.dry_run and args.impl == "ours":
+        import torch
+        have = torch.cuda.device_count() if torch.cuda.is_available() else 0
+        if have < args.gpus:
+            print(f"bench.py: --gpus {args.gpus} needs {args.gpus} CUDA devices, this machine shows {have}", file=sys.stderr)
+            return 2
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    env = dict(os.environ)
+    env.setdefault("NCCL_DEBUG", "INFO")            # the communicator's own log (one line per rank) stays on
+    env.setdefault("NCCL_DEBUG_SUBSYS", "INIT")
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd, env=env)
+
+
+def run_dry(args, rank: int, world: int):
+    """The multi-rank bookkeeping of the benchmark without any GPU: every rank reports a made-up duration of
+    (rank + 1) ms for 10 units of work, and rank 0 prints the line that MAX-over-ranks timing gives."""
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("gloo")
+    ms = float(rank + 1)
+    slowest = replicas.max_over_ranks(ms, dist)
+    rate = replicas.job_throughput(10.0, ms * 1e-3, dist)
+    if rank == 0:
+        print(json.dumps({"dry_run": True, "n_gpus": world, "ms_per_step": slowest, "value": rate,
+                          "seed_of_last_rank": replicas.replica_seed(2, world - 1)}), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -767,10 +913,20 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="backbone_layer")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-large-m", action="store_true", help="skip the long-batch record of the default workload")
+    ap.add_argument("--dry-run", action="store_true",
+                    help="rank plumbing only: CPU ranks (gloo) exchange a per-rank duration; used by the CPU tests")
     args = ap.parse_args()
+    if "WORLD_SIZE" not in os.environ and args.gpus > 1:
+        sys.exit(spawn_ranks(args))
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if world != args.gpus:
+        sys.exit(f"bench.py: --gpus {args.gpus} but the launcher started {world} rank(s): start one rank per GPU")
+    if args.dry_run:
+        run_dry(args, rank, world)
+        return
     if args.impl == "reference":
         if rank == 0:
             run_reference(args)

@@ -70,3 +70,34 @@ def test_single_process_is_identity():
     assert [len(replicas.split_batches(10, 4, r)) for r in range(4)] == [2, 3, 2, 3]
     with pytest.raises(ValueError):
         replicas.split_batches(4, 2, 2)
+
+
+def _bench(*args, timeout=150):
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    return subprocess.run([sys.executable, os.path.join(root, "bench.py"), *args], capture_output=True, text=True,
+                          timeout=timeout, env=env, cwd=root)
+
+
+@pytest.mark.timeout(200)
+def test_bench_starts_its_own_ranks_when_no_launcher_did():
+    """`bench.py --gpus 2` outside torchrun starts two ranks itself; with --dry-run they are CPU ranks (gloo) that
+    run only the MAX-over-ranks bookkeeping, and rank 0 alone prints the line."""
+    import json
+    r = _bench("--gpus", "2", "--dry-run")
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [ln for ln in r.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1, r.stdout
+    out = json.loads(lines[0])
+    assert out["n_gpus"] == 2 and out["ms_per_step"] == 2.0            # the slower of the two made-up ranks
+    assert out["value"] == pytest.approx(20.0 / 2e-3)                  # both ranks' units over the slowest duration
+    assert out["seed_of_last_rank"] == replicas.replica_seed(2, 1)
+
+
+@pytest.mark.skipif(torch.cuda.is_available() and torch.cuda.device_count() >= 2, reason="needs a machine with fewer than 2 GPUs")
+def test_bench_refuses_more_gpus_than_the_machine_has():
+    r = _bench("--gpus", "2", "--steps", "1", "--warmup", "1")
+    assert r.returncode != 0 and "needs 2 CUDA devices" in r.stderr
+    assert not [ln for ln in r.stdout.splitlines() if ln.startswith("{")]   # and prints no result line
