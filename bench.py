@@ -264,6 +264,44 @@ class LayerOnDevice:
         return 2 * len(self.sites)
 
 
+def measure_int8_library_rate(device, local_rank: int) -> dict:
+    """A yardstick, not part of the path: the INT8 rate a vendor-library GEMM (torch._int_mm, 8192^3) reaches on this
+    very GPU, as a burst (best of 10) and sustained for two seconds under the power cap, with the clocks seen."""
+    import torch
+    n = 8192
+    a = torch.randint(-127, 128, (n, n), dtype=torch.int8, device=device)
+    b = torch.randint(-127, 128, (n, n), dtype=torch.int8, device=device).t()      # column-major second operand
+    try:
+        for _ in range(3):
+            torch._int_mm(a, b)
+    except Exception as exc:                                                         # not available in this build
+        return {"unavailable": str(exc)[:120]}
+    torch.cuda.synchronize()
+    ops = 2.0 * n ** 3
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    best = float("inf")
+    for _ in range(10):
+        start.record()
+        torch._int_mm(a, b)
+        end.record()
+        torch.cuda.synchronize()
+        best = min(best, start.elapsed_time(end))
+    sampler = ClockSampler(local_rank)
+    with sampler:
+        reps, t_end = 0, time.time() + 2.0
+        start.record()
+        while time.time() < t_end:
+            for _ in range(20):
+                torch._int_mm(a, b)
+            reps += 20
+            torch.cuda.synchronize()
+        end.record()
+        torch.cuda.synchronize()
+    sustained_ms = start.elapsed_time(end) / reps
+    return {"kernel": "torch._int_mm 8192^3 (vendor library; yardstick only)", "burst_tops": round(ops / (best * 1e-3) / 1e12, 1),
+            "sustained_tops": round(ops / (sustained_ms * 1e-3) / 1e12, 1), "clocks_sustained": sampler.summary()}
+
+
 def tensor_fractions(tops: float, peaks) -> dict:
     """One achieved INT8 rate against the three denominators in use: twice the measured bf16 cuBLAS rate, as a
     burst (a kernel timed alone or in a short region) and sustained (seconds under the power cap) -- dense int8 is
@@ -439,6 +477,12 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         del layer
         torch.cuda.empty_cache()
         out["large_m"] = large_m_record(device, local_rank, peaks, seed=5)
+        # last, so that its two seconds of full load do not heat the measurements above
+        lib = measure_int8_library_rate(device, local_rank)
+        out["int8_library_rate"] = lib
+        if "burst_tops" in lib:
+            out["roofline"]["frac_int8_library_burst"] = round(achieved / lib["burst_tops"], 4)
+            out["large_m"]["gemm"]["frac_int8_library_sustained"] = round(out["large_m"]["gemm"]["achieved_tops"] / lib["sustained_tops"], 4)
     if rank == 0:
         if world == 1 and not args.no_cpu_baseline:
             out["cpu_baseline"] = cpu_baseline(args.workload, steps=1)

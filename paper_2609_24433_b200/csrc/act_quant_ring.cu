@@ -27,6 +27,11 @@ namespace fq {
 namespace {
 
 constexpr int kThreads = 512;
+#ifndef FQ_RING_T32
+#define FQ_RING_T32 512
+#endif
+// Threads of a CTA by channels per thread.
+constexpr int threads_for(int e) { return e == 32 ? FQ_RING_T32 : kThreads; }
 constexpr int kMaxSlots = 128;
 
 // 128-byte swizzle of a byte offset inside a 1024-byte aligned region.
@@ -103,8 +108,8 @@ struct RingParams {
     uint32_t* watchdog;
 };
 
-template <typename XT, int FMT, bool CLAMP, int E, int BLOCK, bool AFTER>
-__global__ void __launch_bounds__(kThreads, 1)
+template <typename XT, int FMT, bool CLAMP, int E, int BLOCK, bool AFTER, int THREADS = kThreads>
+__global__ void __launch_bounds__(THREADS, 1)
 transform_quantize_ring_kernel(const __grid_constant__ CUtensorMap map_x, const RingParams p) {
     constexpr int H = E / 2;                       // channels per half: v[i] = (channel i, channel i + H)
     extern __shared__ uint8_t smem_raw[];
@@ -113,7 +118,7 @@ transform_quantize_ring_kernel(const __grid_constant__ CUtensorMap map_x, const 
     __shared__ int s_abort;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int ngroups = (kThreads / 32) / p.gw;
+    const int ngroups = (THREADS / 32) / p.gw;
     const int group = warp / p.gw;
     const int wg = warp - group * p.gw;
     const int col0 = (wg * 32 + lane) * E;
@@ -156,12 +161,21 @@ transform_quantize_ring_kernel(const __grid_constant__ CUtensorMap map_x, const 
         }
     }
     if (p.mult != nullptr) {
-        // Stage the multiplier with its 16-byte pieces XOR-swizzled by the index of the thread slice
-        // (E floats) they belong to, so that the slice-per-thread reads below are bank-conflict free.
-        for (int i = tid * 4; i < p.K; i += kThreads * 4) {
+        // Stage the multiplier in the order the registers hold a slice: inside every thread slice (E floats)
+        // the entries are interleaved as (g[q], g[q + H]) pairs, so that one 16-byte read yields two ready
+        // operands of the packed multiply (no register moves to pair them up), and the 16-byte pieces are
+        // XOR-swizzled by the slice index, so that the slice-per-thread reads are bank-conflict free.
+        for (int i = tid * 4; i < p.K; i += THREADS * 4) {
             const float4 g4 = __ldg(reinterpret_cast<const float4*>(p.mult + i));
-            const uint32_t off = (uint32_t)i * 4u;
-            *reinterpret_cast<float4*>(gen + (off ^ (((off / (E * 4u)) & 7u) << 4))) = g4;
+            const float gv[4] = {g4.x, g4.y, g4.z, g4.w};
+            const uint32_t slice = (uint32_t)i / E;
+            const uint32_t key = (slice & 7u) << 4;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const uint32_t q = ((uint32_t)i % E) + k;                       // position inside the slice
+                const uint32_t off = q < H ? q * 8u : (q - H) * 8u + 4u;         // pair q (low half) or q - H (high half)
+                *reinterpret_cast<float*>(gen + ((slice * (E * 4u) + off) ^ key)) = gv[k];
+            }
         }
     }
     __syncthreads();
@@ -213,13 +227,10 @@ transform_quantize_ring_kernel(const __grid_constant__ CUtensorMap map_x, const 
             }
             if (!AFTER && p.mult != nullptr) {
 #pragma unroll
-                for (int i = 0; i < H / 4; ++i) {
-                    const float4 lo = lds128f_ordered(piece(g0, g1, i));
-                    const float4 hi = lds128f_ordered(piece(g0, g1, i + H / 4));
-                    v[4 * i + 0] = f2_mul(v[4 * i + 0], make_float2(lo.x, hi.x));
-                    v[4 * i + 1] = f2_mul(v[4 * i + 1], make_float2(lo.y, hi.y));
-                    v[4 * i + 2] = f2_mul(v[4 * i + 2], make_float2(lo.z, hi.z));
-                    v[4 * i + 3] = f2_mul(v[4 * i + 3], make_float2(lo.w, hi.w));
+                for (int i = 0; i < H / 2; ++i) {           // one piece = the multipliers of pairs 2i and 2i + 1
+                    const float4 q = lds128f_ordered(piece(g0, g1, i));
+                    v[2 * i + 0] = f2_mul(v[2 * i + 0], make_float2(q.x, q.y));
+                    v[2 * i + 1] = f2_mul(v[2 * i + 1], make_float2(q.z, q.w));
                 }
             } else {
                 const float2 c2 = make_float2(p.cnorm, p.cnorm);
@@ -277,13 +288,10 @@ transform_quantize_ring_kernel(const __grid_constant__ CUtensorMap map_x, const 
         // fold-after sites: the diagonal sits behind the rotation (z = D^o R x)
         if (AFTER && col_ok) {
 #pragma unroll
-            for (int i = 0; i < H / 4; ++i) {
-                const float4 lo = lds128f_ordered(piece(g0, g1, i));
-                const float4 hi = lds128f_ordered(piece(g0, g1, i + H / 4));
-                v[4 * i + 0] = f2_mul(v[4 * i + 0], make_float2(lo.x, hi.x));
-                v[4 * i + 1] = f2_mul(v[4 * i + 1], make_float2(lo.y, hi.y));
-                v[4 * i + 2] = f2_mul(v[4 * i + 2], make_float2(lo.z, hi.z));
-                v[4 * i + 3] = f2_mul(v[4 * i + 3], make_float2(lo.w, hi.w));
+            for (int i = 0; i < H / 2; ++i) {
+                const float4 q = lds128f_ordered(piece(g0, g1, i));
+                v[2 * i + 0] = f2_mul(v[2 * i + 0], make_float2(q.x, q.y));
+                v[2 * i + 1] = f2_mul(v[2 * i + 1], make_float2(q.z, q.w));
             }
         }
 
@@ -372,19 +380,20 @@ transform_quantize_ring_kernel(const __grid_constant__ CUtensorMap map_x, const 
 
 template <typename XT, int FMT, int E, int BLOCK>
 cudaError_t launch_ring(const CUtensorMap& map, const RingParams& p, int grid, size_t smem, cudaStream_t stream) {
+    constexpr int THREADS = threads_for(E);
     auto go = [&](auto kern) -> cudaError_t {
         cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), smem);
         if (e != cudaSuccess) return e;
-        return launch_pdl(kern, (unsigned)grid, (unsigned)kThreads, smem, stream, 1u, map, p);
+        return launch_pdl(kern, (unsigned)grid, (unsigned)THREADS, smem, stream, 1u, map, p);
     };
     // (the fold-after variant is its own instantiation: as a run-time branch it cost the default
     // path registers, and spills, in the 64-channels-per-thread kernels)
     if (p.mult_after) {
-        if (p.clip_ratio < 1.0f) return go(transform_quantize_ring_kernel<XT, FMT, true, E, BLOCK, true>);
-        return go(transform_quantize_ring_kernel<XT, FMT, false, E, BLOCK, true>);
+        if (p.clip_ratio < 1.0f) return go(transform_quantize_ring_kernel<XT, FMT, true, E, BLOCK, true, THREADS>);
+        return go(transform_quantize_ring_kernel<XT, FMT, false, E, BLOCK, true, THREADS>);
     }
-    if (p.clip_ratio < 1.0f) return go(transform_quantize_ring_kernel<XT, FMT, true, E, BLOCK, false>);
-    return go(transform_quantize_ring_kernel<XT, FMT, false, E, BLOCK, false>);
+    if (p.clip_ratio < 1.0f) return go(transform_quantize_ring_kernel<XT, FMT, true, E, BLOCK, false, THREADS>);
+    return go(transform_quantize_ring_kernel<XT, FMT, false, E, BLOCK, false, THREADS>);
 }
 
 template <typename XT, int FMT, int E>
@@ -424,11 +433,17 @@ cudaError_t launch_transform_quantize_ring(const void* x, fq_dtype xt, int64_t r
     if (rows < 2 * (int64_t)sms || (rows < 8 * (int64_t)sms && K < 8192)) return cudaErrorNotSupported;
 
     // channels per thread (the fold-after variant with shuffle stages does not fit 64 without spills)
+#ifdef FQ_RING_FORCE_E
+    const int e = FQ_RING_FORCE_E;
+#else
     const int e = (K >= 2048 && K % 64 == 0 && !(mult != nullptr && mult_after_rotation && block >= 128)) ? 64 : 32;
+#endif
+    const int threads = threads_for(e);
     int gw = 1;
     while ((int64_t)gw * 32 * e < K) gw <<= 1;
-    if (gw > kThreads / 32) return cudaErrorNotSupported;
-    const int ngroups = (kThreads / 32) / gw;
+    if (gw > threads / 32) return cudaErrorNotSupported;
+    const int ngroups = (threads / 32) / gw;
+    if (gw > 1 && ngroups > 15) return cudaErrorNotSupported;      // one named barrier per group
     const size_t slot = (row_bytes + 1023) / 1024 * 1024;
     const size_t g_bytes = mult ? ((size_t)K * 4 + 1023) / 1024 * 1024 : 0;
     const size_t budget = 227 * 1024 - 2048 - 1024;

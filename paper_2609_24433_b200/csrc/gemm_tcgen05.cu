@@ -39,6 +39,8 @@
 // code in the watchdog word, stops issuing work, and still frees its TMEM.
 #include <cuda_bf16.h>
 
+#include <string.h>
+
 #include <mutex>
 
 #include "fq_common.cuh"
@@ -101,7 +103,7 @@ constexpr int kTileN = 128;          // output channels per tile (MMA M)
 constexpr int kBlockK = 128;         // int8 elements (= bytes) of K per pipeline stage
 constexpr int kAccStages = 2;
 constexpr int kEpiWarps = 8;
-constexpr int kEpiStageBytes = 16 * 64;   // 16 tokens x 32 channels of bf16 per epilogue warp
+constexpr int kEpiStageBytes = 2 * 16 * 64;   // per epilogue warp: two buffers of 16 tokens x 32 channels of bf16
 constexpr int kThreadsW8 = 32 * (2 + kEpiWarps + 1);   // + one warp: TMA producer of int8 weights
 constexpr int kFirstUnpackWarp = 2 + kEpiWarps;
 constexpr int kUnpackSets = 2;          // sets of four unpack warps, one TMEM lane quadrant each
@@ -121,6 +123,7 @@ struct Params {
     int stages_p;        // packed-weight ring (4-bit weights)
     int stages_w;        // unpacked-weight ring (4-bit weights)
     int m_tiles, n_tiles;
+    int band;            // token tiles per band of the tile order (see tile_coords); m_tiles = one band = channel-major order
     int tmem_cols;
     int acc_shift;
     const float* w_scale;
@@ -310,6 +313,43 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* r) {
         : "memory");
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+// 16 TMEM lanes x 16 columns in the layout of a warp-level MMA accumulator: thread T holds, for column groups n = 0, 1,
+//   r[4n + 0], r[4n + 1] = lane T/4,     columns 8n + 2(T%4), 8n + 2(T%4) + 1
+//   r[4n + 2], r[4n + 3] = lane T/4 + 8, the same two columns.
+// With channels on the lanes and tokens on the columns, a register pair is one channel at two adjacent tokens --
+// the fragment that stmatrix stores transposed, i.e. token-major.
+__device__ __forceinline__ void tmem_ld_16x256b_x2(uint32_t taddr, uint32_t* r) {
+    asm volatile("tcgen05.ld.sync.aligned.16x256b.x2.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                 : "r"(taddr)
+                 : "memory");
+}
+// Four 8x8 matrices of 16-bit elements, each thread's register i a fragment (row T/4, columns 2(T%4), 2(T%4)+1) of
+// matrix i, stored TRANSPOSED: the 16 bytes at the address given by thread 8i + r receive column r of matrix i.
+__device__ __forceinline__ void stmatrix_x4_trans(uint32_t addr, uint32_t r0, uint32_t r1, uint32_t r2, uint32_t r3) {
+    asm volatile("stmatrix.sync.aligned.m8n8.x4.trans.shared.b16 [%0], {%1, %2, %3, %4};"
+                 ::"r"(addr), "r"(r0), "r"(r1), "r"(r2), "r"(r3)
+                 : "memory");
+}
+// Tiled bulk STORE shared -> global (a store, never a multicast load); rows and columns beyond the tensor's extent
+// are clipped by the copy engine.  Completion is tracked per issuing thread in bulk groups.
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, int c0, int c1, uint32_t src) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+                 ::"l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(src)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// At most one (zero) of this thread's bulk groups still reads its shared-memory source.
+__device__ __forceinline__ void bulk_wait_read_1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+// One channel at two adjacent tokens: y = acc * (delta_t * s_j) + b_j, rounded to bf16, token 2k in the low half.
+__device__ __forceinline__ uint32_t scale_pair_bf16(uint32_t a0, uint32_t a1, float2 d, float2 sw2, float2 bj2) {
+    const float2 a2 = make_float2((float)(int)a0, (float)(int)a1);
+    const float2 v2 = f2_fma(a2, f2_mul(d, sw2), bj2);
+    uint32_t w;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(w) : "f"(v2.y), "f"(v2.x));
+    return w;
+}
 
 // Shared-memory matrix descriptor: K-major operand, 128-byte rows, 128B swizzle,
 // 8-row groups 1024 bytes apart.
@@ -350,7 +390,7 @@ enum : uint32_t {
 template <int BITS, int CTAS, bool SPLIT, int ATOMS = 1>
 __global__ void __launch_bounds__(BITS == 4 ? kThreadsW4 : kThreadsW8, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_w,
-                    const Params p) {
+                    const __grid_constant__ CUtensorMap map_y, const Params p) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t s_full_tma[kMaxStages];     // activations (+ int8 weights) landed
     __shared__ uint64_t s_empty[kMaxStages];        // ... consumed by the MMAs (one commit per k-block; for 4-bit
@@ -436,6 +476,24 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     const int my_units = p.units_q + (unit0 < p.units_rem ? 1 : 0);
     const int k_blocks = p.kb_per;
     auto tile_of = [&](int unit) { return unit >> split_shift; };
+    // Tile order.  Consecutive tile numbers -- the tiles the SMs work on at the same time -- cover a compact block of
+    // the output: the token tiles are cut into bands of p.band, a band is walked channel tile by channel tile with
+    // its token tiles fastest.  What one wave of CTAs pulls through L2 is then band activation tiles plus SMs/band
+    // weight tiles instead of every activation tile of the batch (long batches: the int8 activations alone exceed
+    // L2, and in channel-major order every wave streamed all of them from HBM again).
+    auto m_of = [&](int tile) {
+        if (p.band >= p.m_tiles) return tile % p.m_tiles;
+        const int b = tile / (p.band * p.n_tiles);
+        const int r = tile - b * (p.band * p.n_tiles);
+        const int rows = max(1, min(p.band, p.m_tiles - b * p.band));   // (a producer also maps the unit past its last one)
+        return b * p.band + r % rows;
+    };
+    auto n_of = [&](int tile) {
+        if (p.band >= p.m_tiles) return tile / p.m_tiles;
+        const int b = tile / (p.band * p.n_tiles);
+        const int r = tile - b * (p.band * p.n_tiles);
+        return r / max(1, min(p.band, p.m_tiles - b * p.band));
+    };
     auto kb0_of = [&](int unit) { return (unit & (split - 1)) * k_blocks; };   // first k-block of the unit's slice
 
     if (warp == 0) {
@@ -449,7 +507,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             bool ok = true;
             int stage = 0, kb = 0, unit = unit0;
             uint32_t phase = 0;
-            int t0 = (tile_of(unit) % p.m_tiles) * p.bt + (int)cta_rank * bt_cta;
+            int t0 = m_of(tile_of(unit)) * p.bt + (int)cta_rank * bt_cta;
             int kb0 = kb0_of(unit);
             bool peek = false;
             for (int n = 0; n < total_kb; ++n) {
@@ -477,7 +535,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                 if (++kb == k_blocks) {
                     kb = 0;
                     unit += unit_step;
-                    t0 = (tile_of(unit) % p.m_tiles) * p.bt + (int)cta_rank * bt_cta;
+                    t0 = m_of(tile_of(unit)) * p.bt + (int)cta_rank * bt_cta;
                     kb0 = kb0_of(unit);
                 }
             }
@@ -570,12 +628,13 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         uint32_t acc_phase = 0;
         [[maybe_unused]] uint32_t epi_phase = 0;
         [[maybe_unused]] int epi_use = 0;
+        [[maybe_unused]] int store_use = 0;             // bulk stores issued by this warp so far (buffer = parity)
         bool ok = true;
         for (int unit = unit0; unit < num_units && ok; unit += unit_step) {
             const int tile = tile_of(unit);
-            const int64_t jq = (int64_t)(tile / p.m_tiles) * (kTileN * CTAS) + (int64_t)cta_rank * kTileN + quad * 32;   // first channel of this warp
+            const int64_t jq = (int64_t)n_of(tile) * (kTileN * CTAS) + (int64_t)cta_rank * kTileN + quad * 32;   // first channel of this warp
             const int64_t j = jq + lane;
-            const int64_t t0 = (int64_t)(tile % p.m_tiles) * p.bt;
+            const int64_t t0 = (int64_t)m_of(tile) * p.bt;
             const bool j_ok = j < p.N;
             float sw = 0.0f, bj = 0.0f;
             if (j_ok && p.out.acc == nullptr) {
@@ -638,6 +697,66 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                 part = tile_part;
             }
             tc_fence_after();
+            if (!SPLIT && staged) {
+                // bf16 outputs.  The accumulators are read as MMA-style fragments (a thread: four channels, two adjacent
+                // tokens of each 8-token group), scaled in packed pairs, stored token-major into a 1 KB buffer of
+                // [16 tokens][32 channels] with two transposing matrix stores, and leave as one tiled bulk store; two
+                // buffers alternate so that a chunk is written while the previous one is on its way out.
+                const int g = lane >> 2, q = lane & 3;
+                float2 sw4[4], bj4[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int64_t ji = jq + g + 8 * i;
+                    float swv = 0.0f, bv = 0.0f;
+                    if (ji < p.N) { swv = __ldg(p.w_scale + ji) * unshift; bv = __ldg(p.bias + ji); }
+                    sw4[i] = make_float2(swv, swv);
+                    bj4[i] = make_float2(bv, bv);
+                }
+                // address of "matrix lane>>3, row lane&7" inside a buffer: token (lane>>4)*8 + (lane&7), 16-byte
+                // chunk ((lane>>3)&1) [+2 for channels 16..31], chunk index XORed with (token>>1)&3 (64-byte swizzle)
+                const uint32_t tok = (uint32_t)((lane >> 4) * 8 + (lane & 7));
+                const uint32_t ch = (uint32_t)((lane >> 3) & 1);
+                const uint32_t off_a = tok * 64u + ((ch ^ ((tok >> 1) & 3u)) << 4);
+                const uint32_t off_b = tok * 64u + (((ch + 2u) ^ ((tok >> 1) & 3u)) << 4);
+                const uint32_t buf0 = smem_e + (uint32_t)(warp - 2) * kEpiStageBytes;
+                const bool any_channel = jq < p.N;        // warp-uniform
+                for (int c = half * 16; c < p.bt; c += 32) {
+                    const int64_t tc = t0 + c;
+                    if (tc >= p.M) break;                // tokens beyond M: nothing to store (warp-uniform)
+                    uint32_t ra[8], rb[8];
+                    tmem_ld_16x256b_x2(taddr + (uint32_t)c, ra);                    // channels 0..15 of the quadrant
+                    tmem_ld_16x256b_x2(taddr + (16u << 16) + (uint32_t)c, rb);      // channels 16..31
+                    const int64_t ta = tc + 2 * q, tb = ta + 8;
+                    float2 d0, d1;
+                    d0.x = ta < p.M ? __ldg(p.out.a_delta + ta) : 0.0f;
+                    d0.y = ta + 1 < p.M ? __ldg(p.out.a_delta + ta + 1) : 0.0f;
+                    d1.x = tb < p.M ? __ldg(p.out.a_delta + tb) : 0.0f;
+                    d1.y = tb + 1 < p.M ? __ldg(p.out.a_delta + tb + 1) : 0.0f;
+                    const uint32_t buf = buf0 + (uint32_t)(store_use & 1) * 1024u;
+                    if (store_use >= 2) {                // the store that last used this buffer has read it
+                        if (lane == 0) bulk_wait_read_1();
+                        __syncwarp();
+                    }
+                    tmem_ld_wait();
+                    const uint32_t wa0 = scale_pair_bf16(ra[0], ra[1], d0, sw4[0], bj4[0]);
+                    const uint32_t wa1 = scale_pair_bf16(ra[2], ra[3], d0, sw4[1], bj4[1]);
+                    const uint32_t wa2 = scale_pair_bf16(ra[4], ra[5], d1, sw4[0], bj4[0]);
+                    const uint32_t wa3 = scale_pair_bf16(ra[6], ra[7], d1, sw4[1], bj4[1]);
+                    stmatrix_x4_trans(buf + off_a, wa0, wa1, wa2, wa3);
+                    const uint32_t wb0 = scale_pair_bf16(rb[0], rb[1], d0, sw4[2], bj4[2]);
+                    const uint32_t wb1 = scale_pair_bf16(rb[2], rb[3], d0, sw4[3], bj4[3]);
+                    const uint32_t wb2 = scale_pair_bf16(rb[4], rb[5], d1, sw4[2], bj4[2]);
+                    const uint32_t wb3 = scale_pair_bf16(rb[6], rb[7], d1, sw4[3], bj4[3]);
+                    stmatrix_x4_trans(buf + off_b, wb0, wb1, wb2, wb3);
+                    fence_proxy_async_smem();            // the buffer, written through the generic proxy, is read by the copy engine
+                    __syncwarp();
+                    if (lane == 0 && any_channel) {
+                        tma_store_2d(&map_y, (int)jq * 2, (int)tc, buf);   // the output map counts bytes along a row
+                        bulk_commit();
+                    }
+                    ++store_use;
+                }
+            } else
             for (int c = half * 16; c < p.bt; c += 32) {
                 const int64_t tc = t0 + c;
                 if (tc >= p.M) break;                    // tokens beyond M: nothing to store (warp-uniform)
@@ -732,6 +851,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             }
             if (++acc_stage == kAccStages) { acc_stage = 0; acc_phase ^= 1u; }
         }
+        if (!SPLIT && staged && lane == 0) bulk_wait_all();   // this warp's stores have left before the CTA gives up its shared memory
     } else if (BITS == 8) {
         // ------------------------------------------------- TMA producer, int8 weights
         // (converged warp, one issuing lane: see the activation producer)
@@ -740,7 +860,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             bool ok = true;
             int stage = 0, kb = 0, unit = unit0;
             uint32_t phase = 0;
-            int n0 = (tile_of(unit) / p.m_tiles) * (kTileN * CTAS) + (int)cta_rank * kTileN;
+            int n0 = n_of(tile_of(unit)) * (kTileN * CTAS) + (int)cta_rank * kTileN;
             int kb0 = kb0_of(unit);
             bool peek = false;
             for (int n = 0; n < total_kb; ++n) {
@@ -765,7 +885,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                 if (++kb == k_blocks) {
                     kb = 0;
                     unit += unit_step;
-                    n0 = (tile_of(unit) / p.m_tiles) * (kTileN * CTAS) + (int)cta_rank * kTileN;
+                    n0 = n_of(tile_of(unit)) * (kTileN * CTAS) + (int)cta_rank * kTileN;
                     kb0 = kb0_of(unit);
                 }
             }
@@ -863,7 +983,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             bool ok = true;
             int ps = 0, kb = 0, unit = unit0;
             uint32_t pph = 0;
-            int n0 = (tile_of(unit) / p.m_tiles) * (kTileN * CTAS) + (int)cta_rank * kTileN;
+            int n0 = n_of(tile_of(unit)) * (kTileN * CTAS) + (int)cta_rank * kTileN;
             int kb0 = kb0_of(unit);
             bool peek = false;
             for (int n = 0; n < total_kb; ++n) {
@@ -885,7 +1005,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                 if (++kb == k_blocks) {
                     kb = 0;
                     unit += unit_step;
-                    n0 = (tile_of(unit) / p.m_tiles) * (kTileN * CTAS) + (int)cta_rank * kTileN;
+                    n0 = n_of(tile_of(unit)) * (kTileN * CTAS) + (int)cta_rank * kTileN;
                     kb0 = kb0_of(unit);
                 }
             }
@@ -922,13 +1042,13 @@ EncodeTiledFn encode_fn() {
     return fn;
 }
 
-// 2-D byte tensor [rows, row_bytes] (row pitch = row_bytes), box [box_rows, box_bytes].
+// 2-D byte tensor [rows, row_bytes] (row pitch = pitch_bytes, 0 = row_bytes), box [box_rows, box_bytes].
 bool encode_2d(CUtensorMap* map, const void* ptr, uint64_t row_bytes, uint64_t rows, uint32_t box_bytes,
-               uint32_t box_rows, CUtensorMapSwizzle swizzle) {
+               uint32_t box_rows, CUtensorMapSwizzle swizzle, uint64_t pitch_bytes = 0) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
     const cuuint64_t dims[2] = {row_bytes, rows};
-    const cuuint64_t strides[1] = {row_bytes};
+    const cuuint64_t strides[1] = {pitch_bytes ? pitch_bytes : row_bytes};
     const cuuint32_t box[2] = {box_bytes, box_rows};
     const cuuint32_t estr[2] = {1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(ptr), dims, strides, box, estr,
@@ -978,12 +1098,12 @@ fq_status build_weight_tmap(Weights& W) {
 namespace {
 
 template <int BITS, int CTAS, bool SPLIT, int ATOMS = 1>
-fq_status launch_variant(const CUtensorMap& map_a, const CUtensorMap& map_w, const Params& p, int grid, size_t smem,
-                         int cluster, cudaStream_t stream) {
+fq_status launch_variant(const CUtensorMap& map_a, const CUtensorMap& map_w, const CUtensorMap& map_y, const Params& p,
+                         int grid, size_t smem, int cluster, cudaStream_t stream) {
     auto kern = gemm_tcgen05_kernel<BITS, CTAS, SPLIT, ATOMS>;
     if (ensure_dynamic_smem(reinterpret_cast<const void*>(kern), smem) != cudaSuccess) return FQ_ERR_CUDA;
     return launch_pdl(kern, (unsigned)grid, (unsigned)(BITS == 4 ? kThreadsW4 : kThreadsW8), smem, stream, (unsigned)cluster,
-                      map_a, map_w, p) == cudaSuccess ? FQ_OK : FQ_ERR_CUDA;
+                      map_a, map_w, map_y, p) == cudaSuccess ? FQ_OK : FQ_ERR_CUDA;
 }
 
 }  // namespace
@@ -1017,7 +1137,12 @@ Plan plan_gemm(int64_t M, int64_t N, int64_t K, int bits, int sms, size_t scratc
     const int64_t kb = (K + kBlockK - 1) / kBlockK;
     Plan best;
     double best_cost = 0.0;
+#ifdef FQ_DEV_W4_PAIRS     // working builds only: force CTA pairs on 4-bit weights for batches of FQ_DEV_W4_PAIRS tokens or more
+    const int c_first = (bits == 4 && N > kTileN && M >= FQ_DEV_W4_PAIRS) ? 2 : 1;
+    for (int c = c_first; c <= (((bits == 8 || c_first == 2) && N > kTileN) ? 2 : 1); ++c) {
+#else
     for (int c = 1; c <= ((bits == 8 && N > kTileN) ? 2 : 1); ++c) {
+#endif
         const int64_t n_units = (N + kTileN * c - 1) / (kTileN * c);
         for (int mt = (int)((M + bt_max - 1) / bt_max); mt <= (int)((M + 63) / 64); ++mt) {
             const int b = (int)(((M + mt - 1) / mt + 15) / 16 * 16);
@@ -1089,6 +1214,9 @@ fq_status launch_gemm_tcgen05(const int8_t* a8, int64_t M, const Weights& W, int
     p.bt = bt;
     p.m_tiles = (int)((M + bt - 1) / bt);
     p.n_tiles = (int)((W.N + kTileN * ctas - 1) / (kTileN * ctas));
+    // Bands of 8 token tiles once the batch is long enough for the order to matter: a wave of 148 CTAs (74 pairs)
+    // then covers 8 token tiles x 18 (9) channel tiles, close to the square that minimises the bytes it shares.
+    p.band = p.m_tiles >= 16 ? 8 : p.m_tiles;
     p.acc_shift = acc_shift;
     p.w_scale = W.w_scale;
     p.bias = W.bias;
@@ -1142,6 +1270,14 @@ fq_status launch_gemm_tcgen05(const int8_t* a8, int64_t M, const Weights& W, int
     if (!encode_2d(&map_a, a8, (uint64_t)W.K, (uint64_t)M, kBlockK, (uint32_t)(bt / ctas), CU_TENSOR_MAP_SWIZZLE_128B))
         return FQ_ERR_CUDA;
 
+    // bf16 outputs of an unsplit launch leave through tiled bulk stores of [16 tokens x 32 channels] (64-byte rows,
+    // 64-byte swizzle in shared memory); the copy engine clips what lies beyond M tokens or N channels
+    CUtensorMap map_y;
+    memset(&map_y, 0, sizeof(map_y));
+    if (out.acc == nullptr && out.yt == FQ_BF16 && split == 1 &&
+        !encode_2d(&map_y, out.y, (uint64_t)W.N * 2, (uint64_t)M, 64, 16, CU_TENSOR_MAP_SWIZZLE_64B, (uint64_t)out.ldy * 2))
+        return FQ_ERR_CUDA;
+
     const int num_units = p.m_tiles * p.n_tiles * split;       // a K split makes `split` units of every tile
     const int max_units = sms / ctas;
     const int clusters = num_units < max_units ? num_units : max_units;
@@ -1154,19 +1290,19 @@ fq_status launch_gemm_tcgen05(const int8_t* a8, int64_t M, const Weights& W, int
     p.split_shift = split == 1 ? 0 : (split == 2 ? 1 : (split == 4 ? 2 : (split == 8 ? 3 : 4)));
 
     if (W.bits == 4) {
-        if (ctas == 2) return launch_variant<4, 2, false>(map_a, W.tmap, p, grid, smem, 2, stream);
+        if (ctas == 2) return launch_variant<4, 2, false>(map_a, W.tmap, map_y, p, grid, smem, 2, stream);
         if (atoms == 4)
-            return split > 1 ? launch_variant<4, 1, true, 4>(map_a, W.tmap, p, grid, smem, 1, stream)
-                             : launch_variant<4, 1, false, 4>(map_a, W.tmap, p, grid, smem, 1, stream);
+            return split > 1 ? launch_variant<4, 1, true, 4>(map_a, W.tmap, map_y, p, grid, smem, 1, stream)
+                             : launch_variant<4, 1, false, 4>(map_a, W.tmap, map_y, p, grid, smem, 1, stream);
         if (atoms == 2)
-            return split > 1 ? launch_variant<4, 1, true, 2>(map_a, W.tmap, p, grid, smem, 1, stream)
-                             : launch_variant<4, 1, false, 2>(map_a, W.tmap, p, grid, smem, 1, stream);
-        return split > 1 ? launch_variant<4, 1, true>(map_a, W.tmap, p, grid, smem, 1, stream)
-                         : launch_variant<4, 1, false>(map_a, W.tmap, p, grid, smem, 1, stream);
+            return split > 1 ? launch_variant<4, 1, true, 2>(map_a, W.tmap, map_y, p, grid, smem, 1, stream)
+                             : launch_variant<4, 1, false, 2>(map_a, W.tmap, map_y, p, grid, smem, 1, stream);
+        return split > 1 ? launch_variant<4, 1, true>(map_a, W.tmap, map_y, p, grid, smem, 1, stream)
+                         : launch_variant<4, 1, false>(map_a, W.tmap, map_y, p, grid, smem, 1, stream);
     }
-    if (ctas == 2) return launch_variant<8, 2, false>(map_a, W.tmap, p, grid, smem, 2, stream);
-    return split > 1 ? launch_variant<8, 1, true>(map_a, W.tmap, p, grid, smem, 1, stream)
-                     : launch_variant<8, 1, false>(map_a, W.tmap, p, grid, smem, 1, stream);
+    if (ctas == 2) return launch_variant<8, 2, false>(map_a, W.tmap, map_y, p, grid, smem, 2, stream);
+    return split > 1 ? launch_variant<8, 1, true>(map_a, W.tmap, map_y, p, grid, smem, 1, stream)
+                     : launch_variant<8, 1, false>(map_a, W.tmap, map_y, p, grid, smem, 1, stream);
 }
 
 }  // namespace fq
