@@ -27,11 +27,10 @@ namespace fq {
 namespace {
 
 constexpr int kThreads = 512;
-#ifndef FQ_RING_T32
-#define FQ_RING_T32 512
-#endif
-// Threads of a CTA by channels per thread.
-constexpr int threads_for(int e) { return e == 32 ? FQ_RING_T32 : kThreads; }
+// Threads of a CTA by channels per thread.  (1024 threads of 32 channels -- twice the warps at 64 registers -- measured
+// slower than 512 threads of 64 channels for 4-bit output: 0.65 against 0.75 of the copy rate at K = 8192, block 128;
+// the extra cross-lane butterfly stage costs more than the occupancy returns.)
+constexpr int threads_for(int) { return kThreads; }
 constexpr int kMaxSlots = 128;
 
 // 128-byte swizzle of a byte offset inside a 1024-byte aligned region.
@@ -433,11 +432,7 @@ cudaError_t launch_transform_quantize_ring(const void* x, fq_dtype xt, int64_t r
     if (rows < 2 * (int64_t)sms || (rows < 8 * (int64_t)sms && K < 8192)) return cudaErrorNotSupported;
 
     // channels per thread (the fold-after variant with shuffle stages does not fit 64 without spills)
-#ifdef FQ_RING_FORCE_E
-    const int e = FQ_RING_FORCE_E;
-#else
     const int e = (K >= 2048 && K % 64 == 0 && !(mult != nullptr && mult_after_rotation && block >= 128)) ? 64 : 32;
-#endif
     const int threads = threads_for(e);
     int gw = 1;
     while ((int64_t)gw * 32 * e < K) gw <<= 1;

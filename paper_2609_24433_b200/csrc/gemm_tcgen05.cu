@@ -410,11 +410,11 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     volatile int* abort_flag = &s_abort;
     const uint32_t cta_rank = CTAS == 2 ? cluster_ctarank() : 0u;
     const bool leader = cta_rank == 0;
-    // K split (single CTAs only): a tile is `split` work units, unit = tile * split + slice, slice s
+    // K split: a tile is `split` work units, unit = tile * split + slice, slice s
     // covering k-blocks [s * k_blocks, (s + 1) * k_blocks).  Any CTA takes any unit; the CTA that
     // finishes a tile's last slice adds up the slices' partial sums and runs the epilogue.
-    const int split = (SPLIT && CTAS == 1) ? p.split : 1;   // compile-time 1 in the common instantiation
-    const int split_shift = (SPLIT && CTAS == 1) ? p.split_shift : 0;
+    const int split = SPLIT ? p.split : 1;   // compile-time 1 in the common instantiation
+    const int split_shift = SPLIT ? p.split_shift : 0;
     const int bt_cta = p.bt / CTAS;                 // token rows this CTA loads
 
     // carve dynamic shared memory: [A8 stages][W8 stages][packed stages][epilogue transposers], 1024-byte aligned
@@ -655,7 +655,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             const int slice = unit & (split - 1);
             if (split > 1) {
                 tc_fence_after();
-                int32_t* tile_part = p.partials + (size_t)tile * (size_t)split * kTileN * (size_t)p.bt + (size_t)(quad * 32 + lane);
+                // (in a CTA pair each CTA exchanges and counts its own 128 channels of the tile)
+                const int ctile = tile * CTAS + (int)cta_rank;
+                int32_t* tile_part = p.partials + (size_t)ctile * (size_t)split * kTileN * (size_t)p.bt + (size_t)(quad * 32 + lane);
                 int32_t* mine = tile_part + (size_t)slice * kTileN * (size_t)p.bt;
                 for (int c = half * 16; c < p.bt; c += 32) {
                     if (t0 + c >= p.M) break;
@@ -674,7 +676,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                 if (!ok) break;
                 int* last_slot = &s_last[epi_use & 1];
                 if (warp == 2 && lane == 0) {
-                    const uint32_t done = atomicAdd(p.counters + tile, 1u);
+                    const uint32_t done = atomicAdd(p.counters + ctile, 1u);
                     *last_slot = done == (uint32_t)(split - 1) ? 1 : 0;
                 }
                 // rendezvous 2: the outcome is written (its slot is reused two tiles later, after both
@@ -689,7 +691,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                 if (!last) {
                     tc_fence_before();
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(smem_u32(&s_acc_empty[acc_stage]));
+                    if (lane == 0) {
+                        if (CTAS == 1) mbar_arrive(smem_u32(&s_acc_empty[acc_stage]));
+                        else mbar_arrive_cta(smem_u32(&s_acc_empty[acc_stage]), 0);
+                    }
                     if (++acc_stage == kAccStages) { acc_stage = 0; acc_phase ^= 1u; }
                     continue;
                 }
@@ -756,7 +761,21 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                     }
                     ++store_use;
                 }
-            } else
+            } else {
+            // K split: the other slices' sums of a chunk are requested one chunk ahead of their use, so that their
+            // trip through L2 overlaps the arithmetic and stores of the chunk before.
+            [[maybe_unused]] int32_t pv_next[16];
+            auto fetch_partials = [&](int c) {
+#pragma unroll
+                for (int i = 0; i < 16; ++i) pv_next[i] = 0;
+                for (int rk = 0; rk < split; ++rk) {
+                    if (rk == slice) continue;
+                    const int32_t* src = part + ((size_t)rk * (size_t)p.bt + (size_t)c) * kTileN;
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) pv_next[i] += __ldcg(src + (size_t)i * kTileN);
+                }
+            };
+            if (split > 1 && t0 + half * 16 < p.M) fetch_partials(half * 16);
             for (int c = half * 16; c < p.bt; c += 32) {
                 const int64_t tc = t0 + c;
                 if (tc >= p.M) break;                    // tokens beyond M: nothing to store (warp-uniform)
@@ -765,13 +784,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                 if (split > 1) {
                     int32_t pv[16];
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) pv[i] = 0;
-                    for (int rk = 0; rk < split; ++rk) {
-                        if (rk == slice) continue;
-                        const int32_t* src = part + ((size_t)rk * (size_t)p.bt + (size_t)c) * kTileN;
-#pragma unroll
-                        for (int i = 0; i < 16; ++i) pv[i] += __ldcg(src + (size_t)i * kTileN);
-                    }
+                    for (int i = 0; i < 16; ++i) pv[i] = pv_next[i];
+                    if (c + 32 < p.bt && tc + 32 < p.M) fetch_partials(c + 32);
                     tmem_ld_wait();
 #pragma unroll
                     for (int i = 0; i < 16; ++i) r[i] += (uint32_t)pv[i];
@@ -842,6 +856,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                         }
                     }
                 }
+            }
             }
             tc_fence_before();
             __syncwarp();
@@ -1128,7 +1143,7 @@ struct Plan {
 //                                        both operands pass through it)
 //   8-bit, CTA pair:        per_kblock = max(545, 2.62*bt)   (each CTA stages half of the token tile)
 // Pairs gain nothing for 4-bit weights, which never pass through shared memory unpacked.
-// K split (single CTAs only): problems with fewer tiles than SMs and a long K (every short batch; down_proj
+// K split (single CTAs, and CTA pairs on 8-bit weights): problems with fewer tiles than SMs and a long K (every short batch; down_proj
 // at M = 816: 64 tiles of 128 k-blocks) make `split` work units of every tile, each on a slice of K; the
 // slices leave int32 partial sums in scratch and the one that finishes last adds them up (fitted cost per
 // unit: 1500 + 70*bt cycles, plus 8*bt per extra slice).
@@ -1137,12 +1152,7 @@ Plan plan_gemm(int64_t M, int64_t N, int64_t K, int bits, int sms, size_t scratc
     const int64_t kb = (K + kBlockK - 1) / kBlockK;
     Plan best;
     double best_cost = 0.0;
-#ifdef FQ_DEV_W4_PAIRS     // working builds only: force CTA pairs on 4-bit weights for batches of FQ_DEV_W4_PAIRS tokens or more
-    const int c_first = (bits == 4 && N > kTileN && M >= FQ_DEV_W4_PAIRS) ? 2 : 1;
-    for (int c = c_first; c <= (((bits == 8 || c_first == 2) && N > kTileN) ? 2 : 1); ++c) {
-#else
     for (int c = 1; c <= ((bits == 8 && N > kTileN) ? 2 : 1); ++c) {
-#endif
         const int64_t n_units = (N + kTileN * c - 1) / (kTileN * c);
         for (int mt = (int)((M + bt_max - 1) / bt_max); mt <= (int)((M + 63) / 64); ++mt) {
             const int b = (int)(((M + mt - 1) / mt + 15) / 16 * 16);
@@ -1152,10 +1162,10 @@ Plan plan_gemm(int64_t M, int64_t N, int64_t K, int bits, int sms, size_t scratc
             // 4-bit, tiles of at most 128 tokens: two-atom stages (see the kernel) cost less per 128 channels
             const double w4 = (c == 1 && b <= 128 && K % kBlockK == 0) ? 235.0 + b : 330.0 + b;
             const double per_kb = bits == 4 ? w4 : (c == 1 ? w8_single : (2.62 * b > 545.0 ? 2.62 * b : 545.0));
-            for (int sp = 1; sp <= (c == 1 ? kMaxSplit : 1); sp *= 2) {
-                if (sp > 1 && (kb % sp != 0 || kb / sp < 2 || units > kMaxSplitTiles || units * sp > 4 * (int64_t)sms)) continue;
+            for (int sp = 1; sp <= ((c == 1 || bits == 8) ? kMaxSplit : 1); sp *= 2) {
+                if (sp > 1 && (kb % sp != 0 || kb / sp < 2 || units * c > kMaxSplitTiles || units * c * sp > 4 * (int64_t)sms)) continue;
                 const int64_t kb_per = kb / sp;
-                const size_t scratch = sp > 1 ? kCounterBytes + (size_t)units * sp * kTileN * b * sizeof(int32_t) : 0;
+                const size_t scratch = sp > 1 ? kCounterBytes + (size_t)units * c * sp * kTileN * b * sizeof(int32_t) : 0;
                 if (scratch > scratch_avail) continue;
                 const int slots = sms / c;
                 const double unit_cost = (double)kb_per * per_kb + 16.0 * b + 1000.0 + (sp > 1 ? 1500.0 + 70.0 * b + 8.0 * b * (sp - 1) : 0.0);
@@ -1300,7 +1310,9 @@ fq_status launch_gemm_tcgen05(const int8_t* a8, int64_t M, const Weights& W, int
         return split > 1 ? launch_variant<4, 1, true>(map_a, W.tmap, map_y, p, grid, smem, 1, stream)
                          : launch_variant<4, 1, false>(map_a, W.tmap, map_y, p, grid, smem, 1, stream);
     }
-    if (ctas == 2) return launch_variant<8, 2, false>(map_a, W.tmap, map_y, p, grid, smem, 2, stream);
+    if (ctas == 2)
+        return split > 1 ? launch_variant<8, 2, true>(map_a, W.tmap, map_y, p, grid, smem, 2, stream)
+                         : launch_variant<8, 2, false>(map_a, W.tmap, map_y, p, grid, smem, 2, stream);
     return split > 1 ? launch_variant<8, 1, true>(map_a, W.tmap, map_y, p, grid, smem, 1, stream)
                      : launch_variant<8, 1, false>(map_a, W.tmap, map_y, p, grid, smem, 1, stream);
 }
