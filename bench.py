@@ -373,6 +373,8 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         ROTATE = 1              # a step already walks far more weight bytes than L2 holds
         CPU_SAMPLE_ROWS = 32    # keeps the oracle arm's sample to tens of seconds
     sites = workload_sites(args.workload)
+    if args.workload.startswith("sweep:") and sites[0].M * sites[0].K >= (1 << 26):
+        ROTATE = 1              # one step's activations and outputs alone are several times L2
     layer = LayerOnDevice(sites, seed=replicas.replica_seed(2, rank), device=device)
     ops = layer_ops(sites)
     K, Wm = args.steps, max(args.warmup, 3)
@@ -813,7 +815,8 @@ def bench_config(workload: str, sites) -> dict:
     """The `config` object of the JSON line: the workload and how the GPU arm stages and launches it.  Both arms
     print the same object (the oracle arm runs a bounded sample of this workload; its `cpu_baseline.sample` says
     which)."""
-    rotate = 1 if workload in ("backbone_forward", "backbone_forward_w4", "expert_loop") else ROTATE
+    rotate = 1 if workload in ("backbone_forward", "backbone_forward_w4", "expert_loop") or \
+        (workload.startswith("sweep:") and sites[0].M * sites[0].K >= (1 << 26)) else ROTATE
     return {"workload": workload_name(workload), "M": sites[0].M,
             "sites": {s.name: {"K": s.K, "N": s.N_total, "bits": s.bits, "block": s.beta} for s in sites[:8]},
             "n_sites": len(sites), "ops_per_step": layer_ops(sites),
