@@ -343,7 +343,6 @@ __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.comm
 // At most N of this thread's bulk groups still read their shared-memory source.
 template <int N>
 __device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
-__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 // One channel at two adjacent tokens: y = acc * (delta_t * s_j) + b_j, rounded to bf16, token 2k in the low half.
 __device__ __forceinline__ uint32_t scale_pair_bf16(uint32_t a0, uint32_t a1, float2 d, float2 sw2, float2 bj2) {
     const float2 a2 = make_float2((float)(int)a0, (float)(int)a1);
@@ -410,6 +409,13 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     volatile int* abort_flag = &s_abort;
+    if (threadIdx.x == 32) {
+        // the three copy descriptors are kernel parameters: fetching them now takes their first-use latency (a few
+        // hundred nanoseconds each) off the path between the end of the kernel ahead and this kernel's first copy
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_a)) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_w)) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_y)) : "memory");
+    }
     const uint32_t cta_rank = CTAS == 2 ? cluster_ctarank() : 0u;
     const bool leader = cta_rank == 0;
     // K split: a tile is `split` work units, unit = tile * split + slice, slice s
@@ -881,7 +887,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             }
             if (++acc_stage == kAccStages) { acc_stage = 0; acc_phase ^= 1u; }
         }
-        if (!SPLIT && staged && lane == 0) bulk_wait_all();   // this warp's stores have left before the CTA gives up its shared memory
+        // this warp's stores have read their buffers before the CTA gives up its shared memory (the writes themselves
+        // are complete when the grid is: no need to wait for them here, which would add their latency to the tail)
+        if (!SPLIT && staged && lane == 0) bulk_wait_read<0>();
     } else if (BITS == 8) {
         // ------------------------------------------------- TMA producer, int8 weights
         // (converged warp, one issuing lane: see the activation producer)
