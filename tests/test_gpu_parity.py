@@ -698,6 +698,41 @@ def test_one_handle_three_streams_three_workspaces():
             assert torch.equal(a, b)
 
 
+@pytest.mark.parametrize("M,K,N,bits", [(50, 1024, 3072, 4), (50, 4096, 1024, 4), (16, 8192, 8192, 4), (64, 8192, 8192, 4),
+                                        (256, 4096, 4096, 4), (816, 2048, 2560, 4), (64, 8192, 2048, 8), (816, 2048, 2048, 8)])
+def test_linear_replayed_in_a_cuda_graph_equals_the_eager_call(M, K, N, bits):
+    """The benchmark and any latency-minded caller replay the one-call path from CUDA graphs, where the prologue, the
+    GEMM (programmatic dependent launch) and the K split's counter memset really overlap and follow each other
+    without host gaps: two rotating operand sets, one step per graph, replayed back to back, must reproduce the
+    eager results bit for bit with no bounded wait expiring."""
+    gen = torch.Generator(device="cuda").manual_seed(M + K + N)
+    sets = []
+    for r in range(2):
+        W = torch.randn((N, K), device="cuda", generator=gen) * 0.02
+        b = torch.randn(N, device="cuda", generator=gen) * 0.02
+        h = fq.fold_weights(W, None, b, 64, bits)
+        x = (torch.randn((M, K), device="cuda", generator=gen) * 2).to(torch.bfloat16)
+        ws = torch.empty(fq.workspace_bytes(M, K, N, bits), dtype=torch.uint8, device="cuda")
+        y = torch.zeros((M, N), dtype=torch.bfloat16, device="cuda")
+        sets.append((x, h, ws, y))
+    want = [fq.linear(x, h, 1.0, torch.bfloat16, workspace=ws).clone() for x, h, ws, _ in sets]
+    torch.cuda.synchronize()
+    graphs = []
+    for x, h, ws, y in sets:
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            fq.linear(x, h, 1.0, y=y, workspace=ws)
+        graphs.append(g)
+    for rep in range(6):
+        for g in graphs:
+            g.replay()
+    torch.cuda.synchronize()
+    for (_, _, _, y), w in zip(sets, want):
+        assert torch.equal(y, w)
+    st, word = fq.device_status()
+    assert st == fq.OK, hex(word)
+
+
 def test_gemm_accepts_a_step_vector_at_any_float_offset():
     """a_delta need only be 4-byte aligned: a slice of a longer vector of steps gives what a copy of it gives."""
     rng = np.random.default_rng(8)
