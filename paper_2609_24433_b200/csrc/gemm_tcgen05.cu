@@ -470,10 +470,11 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     const uint32_t tmem_base = s_tmem_base;
     // Everything above is on-chip setup; from here on global memory is touched (activations written
     // by the kernel before this one, outputs that it may still be reading).
-    // The weight producers do not wait: a weight handle is complete before any call that uses it
-    // is enqueued, so its tiles can stream in while the kernel ahead (the prologue) still runs.
-    const bool weight_producer = BITS == 8 ? warp == kFirstUnpackWarp : warp == kFirstUnpackWarp + 4 * kUnpackSets;
-    if (!weight_producer) griddep_wait();
+    // Only the warps that touch what the kernel ahead writes (or may still read) wait for it: the activation
+    // producer, and the epilogue warps (per-token steps, K-split scratch, the output).  A weight handle is
+    // complete before any call that uses it is enqueued, so the weight producer streams tiles in, the unpack
+    // warps fill their TMEM slots, and the MMA warp parks on its barriers while the prologue still runs.
+    if (warp == 0 || (warp >= 2 && warp < 2 + kEpiWarps)) griddep_wait();
     griddep_launch_dependents();
 
     // work units: (super-tile of 128*CTAS channels) x (token tile) [x K slice]; one unit per CTA or
