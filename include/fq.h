@@ -221,7 +221,7 @@ fq_status fq_linear_w8a8(const void* x, fq_dtype xt, int64_t M, int64_t ldx, con
  * identity transform (fq_fold_weights with hadamard_block = 1 and smooth = NULL: plain per-output-channel
  * RTN of W), or x must already be in the handle's transformed coordinates.  No quantization of x, no
  * workspace.  x device [M, K] of dtype xt (FQ_F32 or FQ_BF16); binary32 accumulation.  These projections see
- * one conditioning vector per sample: the kernel streams the weights once per four tokens and is meant for
+ * one conditioning vector per sample: the kernel streams the weights once per eight tokens and is meant for
  * short batches (any M is accepted).  Errors as for fq_linear_w4a4; FQ_ERR_UNSUPPORTED for 8-bit handles. */
 fq_status fq_linear_w4a16(const void* x, fq_dtype xt, int64_t M, int64_t ldx, const fq_weights* W, void* y,
                           fq_dtype yt, int64_t ldy, void* stream);

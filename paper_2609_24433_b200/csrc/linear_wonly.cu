@@ -1,28 +1,33 @@
 // Short-batch weight streaming for 4-bit weights: the projection of a handful of tokens is a
 // matrix-vector product bound by the weight bytes, which must cross HBM once.  Two users:
-//   * the W4A4 integer product of Eq. 8 for batches of at most 16 tokens on matrices of up to 16-32 Mi weights
-//     (the short end of the throughput sweep), where it measured faster than the TMA/TMEM pipeline of the
-//     big GEMM, whose per-k-block hand-overs cannot be fed at HBM rate by so thin a tile;
+//   * the W4A4 integer product of Eq. 8 for batches of at most 16 tokens where it measured faster than the
+//     TMA/TMEM pipeline of the big GEMM (see gemm_stream_applies), whose per-k-block hand-overs cannot be fed
+//     at HBM rate by so thin a tile;
 //   * the weight-only projection with floating-point activations (the adaptive layer-normalisation
 //     modulation of the W4A4 engines):  y[t][j] = s^W_j * sum_c qW[j][c] * x[t][c] + b_j.
 // One persistent CTA per SM walks groups of 32 weight rows.  A producer warp streams the packed rows
 // through a ring of 32 KB stages (32 rows x 2048 channels, ONE 128-byte-swizzled TMA box each: an
 // issuing warp gets out one tensor copy per ~260 cycles whatever its size, so a stage must not be
-// several) that holds ~160 KB in flight per SM; 16 consumer warps each take one 16-row tile x 256 channels of a stage,
-// expand the codes in registers and multiply with warp-level MMAs (m16n8k32 s8 -> s32, or m16n8k16
-// bf16 -> f32 after an exact code -> bf16 expansion); tokens ride along 8 per MMA at no extra weight
-// traffic.  The warps' partial sums meet in shared memory, are added in a fixed order, rescaled and
-// stored.  binary32 activations are split into three bf16 terms (exactly), so both float input types
-// see exact products and binary32 sums.
+// several) that holds ~190 KB in flight per SM.  Each of the 16 consumer warps takes, of every stage, one
+// 256-channel line of all 32 rows and in it every other 32-channel unit: both 16-row MMA tiles share one B
+// fragment, so a token's activations are fetched and permuted once per 32 rows.  The codes are expanded in
+// registers and multiplied with warp-level MMAs (m16n8k32 s8 -> s32, or m16n8k16 bf16 -> f32); tokens ride
+// along 8 per MMA at no extra weight traffic.  The warps' partial sums meet in shared memory, are added in a
+// fixed order, rescaled and stored.  binary32 activations are split into three bf16 terms (exactly), so both
+// float input types see exact products and binary32 sums.
 //
-// Operand layout.  Lane (g = lane / 4, t = lane % 4) reads 16 bytes = 32 codes of rows g and g + 8 at
-// channel 32 t of the warp's chunk, and the activations of token g at the same channels.  A sum over
+// Operand layout.  Lane (g = lane / 4, t = lane % 4) reads 16 bytes = 32 codes of rows g, g + 8, g + 16 and
+// g + 24 at unit 2t + h of the warp's line, and the activations of token g at the same channels.  A sum over
 // channels may run in any order as long as both operands agree on it, so the k index of the MMA is
 // mapped to channels the way the codes unpack cheapest:
 //   int8:  (w << 4) & 0xF0F0F0F0 holds 16 x the codes of channels 0,2,4,6 of a word and w & 0xF0F0F0F0
 //          those of channels 1,3,5,7 -- the order in which the prologue stores its int8 codes;
 //   bf16:  one mask of the word shifted by 4 j isolates the codes of channels j and j + 4 in the two
 //          halves of a register, and the B fragment pairs the activations of those channels.
+// What bounds the float path is the integer pipe (shift + mask per pair of codes, half the rate of the
+// other pipes): the codes enter the MMAs 136 too large (see codes_plus136_bf16x2) because taking the offset
+// off each pair cost another instruction, and the activations' loads are issued a stage ahead of the byte
+// permutes that consume them.
 #include <cuda_bf16.h>
 #include <stdlib.h>
 
@@ -64,16 +69,18 @@ __device__ __forceinline__ uint4 lds128(uint32_t addr) {
 }
 
 // Codes of channels j and j + 4 of a packed word (eight two's-complement nibbles, channel i at bits
-// 4 i) as two bf16: (n & 15) ^ 8 = n + 8 goes into the mantissa of 128 (0x4300), then 136 comes off.
-// Both steps are exact.
-__device__ __forceinline__ uint32_t codes_bf16x2(uint32_t w, int j) {
-    const uint32_t biased = ((w >> (4 * j)) & 0x000F000Fu) ^ 0x43084308u;
-    uint32_t r;
-    asm("sub.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(biased), "r"(0x43084308u));
-    return r;
+// 4 i) as two bf16, each 136 too large: (n & 15) ^ 8 = n + 8 goes into the mantissa of 128 (0x4300).
+// The exact value 136 + n is what the MMAs multiply; 136 times the sum of the token's activations --
+// accumulated beside the products by MMAs against a matrix of ones -- comes off once per output.  (Taking
+// 136 off every pair with a packed subtract cost a third of the kernel's integer instructions.)
+__device__ __forceinline__ uint32_t codes_plus136_bf16x2(uint32_t w, int j) {
+    return ((w >> (4 * j)) & 0x000F000Fu) ^ 0x43084308u;
 }
+constexpr float kCodeOffset = 136.0f;
 
-// The activations of one token at a lane's 32 channels as B-fragment registers.
+// The activations of one token at a lane's 32 channels: fetch() issues the loads into raw registers, permute() --
+// called a stage later, when they have long arrived -- forms the B-fragment registers.  (With the byte permutes right
+// behind the loads a warp sat out the loads' latency in every stage.)
 template <int MODE>
 struct XFrag;
 // int8 codes as the prologue stores them: 8 channels = (c0,c2,c4,c6) (c1,c3,c5,c7); word w -> b[2w], b[2w+1]
@@ -81,12 +88,16 @@ template <>
 struct XFrag<kModeInt> {
     typedef int8_t elem;
     static constexpr int kTerms = 1;
+    uint4 raw[2];
     uint32_t b[1][8];
-    __device__ __forceinline__ void load(const int8_t* p, bool ok) {
+    __device__ __forceinline__ void fetch(const int8_t* p, bool ok) {
+#pragma unroll
+        for (int h = 0; h < 2; ++h) raw[h] = ok ? __ldg(reinterpret_cast<const uint4*>(p) + h) : make_uint4(0u, 0u, 0u, 0u);
+    }
+    __device__ __forceinline__ void permute() {
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
-            const uint4 n = ok ? __ldg(reinterpret_cast<const uint4*>(p) + h) : make_uint4(0u, 0u, 0u, 0u);
-            b[0][4 * h + 0] = n.x; b[0][4 * h + 1] = n.y; b[0][4 * h + 2] = n.z; b[0][4 * h + 3] = n.w;
+            b[0][4 * h + 0] = raw[h].x; b[0][4 * h + 1] = raw[h].y; b[0][4 * h + 2] = raw[h].z; b[0][4 * h + 3] = raw[h].w;
         }
     }
 };
@@ -95,11 +106,16 @@ template <>
 struct XFrag<kModeBf16> {
     typedef __nv_bfloat16 elem;
     static constexpr int kTerms = 1;
+    uint4 raw[4];
     uint32_t b[1][16];
-    __device__ __forceinline__ void load(const __nv_bfloat16* p, bool ok) {
+    __device__ __forceinline__ void fetch(const __nv_bfloat16* p, bool ok) {
+#pragma unroll
+        for (int w = 0; w < 4; ++w) raw[w] = ok ? __ldg(reinterpret_cast<const uint4*>(p) + w) : make_uint4(0u, 0u, 0u, 0u);
+    }
+    __device__ __forceinline__ void permute() {
 #pragma unroll
         for (int w = 0; w < 4; ++w) {
-            const uint4 n = ok ? __ldg(reinterpret_cast<const uint4*>(p) + w) : make_uint4(0u, 0u, 0u, 0u);
+            const uint4 n = raw[w];
             b[0][4 * w + 0] = __byte_perm(n.x, n.z, 0x5410);   // (c0, c4)
             b[0][4 * w + 1] = __byte_perm(n.x, n.z, 0x7632);   // (c1, c5)
             b[0][4 * w + 2] = __byte_perm(n.y, n.w, 0x5410);   // (c2, c6)
@@ -112,12 +128,16 @@ template <>
 struct XFrag<kModeF32> {
     typedef float elem;
     static constexpr int kTerms = 3;
+    float4 raw[8];
     uint32_t b[3][16];
-    __device__ __forceinline__ void load(const float* p, bool ok) {
+    __device__ __forceinline__ void fetch(const float* p, bool ok) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) raw[i] = ok ? __ldg(reinterpret_cast<const float4*>(p) + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    __device__ __forceinline__ void permute() {
 #pragma unroll
         for (int w = 0; w < 4; ++w) {
-            const float4 lo4 = ok ? __ldg(reinterpret_cast<const float4*>(p) + 2 * w) : make_float4(0.f, 0.f, 0.f, 0.f);
-            const float4 hi4 = ok ? __ldg(reinterpret_cast<const float4*>(p) + 2 * w + 1) : make_float4(0.f, 0.f, 0.f, 0.f);
+            const float4 lo4 = raw[2 * w], hi4 = raw[2 * w + 1];
             float r[8] = {lo4.x, lo4.y, lo4.z, lo4.w, hi4.x, hi4.y, hi4.z, hi4.w};
 #pragma unroll
             for (int s = 0; s < 3; ++s) {
@@ -169,7 +189,8 @@ weight_stream_kernel(const __grid_constant__ CUtensorMap map_w, const StreamPara
     volatile int* abort_flag = &s_abort;
     const uint32_t ring = (smem_u32(smem_raw) + 1023u) & ~1023u;
     AccT* s_part = reinterpret_cast<AccT*>(smem_raw + (ring - smem_u32(smem_raw)) + (size_t)p.depth * kStageBytes);
-    // s_part[k slot 0..7][row 0..31][token, padded to kTok + 1]
+    // s_part[consumer warp][row 0..31][token, padded to kTok + 1]
+    [[maybe_unused]] float* s_xsum = reinterpret_cast<float*>(s_part + (size_t)kConsumers * kRowsCta * (kTok + 1));   // [consumer warp][token]
 
     if (threadIdx.x == 0) {
         s_abort = 0;
@@ -218,14 +239,15 @@ weight_stream_kernel(const __grid_constant__ CUtensorMap map_w, const StreamPara
         griddep_wait();                       // activations come from the kernel ahead in the stream
         griddep_launch_dependents();
         const int g = lane >> 2, t = lane & 3;
-        const int rt = warp & 1, kq = warp >> 1;            // row tile, 128-channel slot of the stage
+        const int h = warp & 1, kq = warp >> 1;            // unit parity, 256-channel line of the stage
         // Stage layout: [row 0..31][line 0..7][128 bytes], line = 256 channels; the 128-byte swizzle XORs the
-        // 16-byte unit index with the low three bits of (8 row + line) = line.  This warp reads line kq of
-        // rows 16 rt + g and 16 rt + 8 + g; lane t takes units 2t and 2t + 1 (64 channels), one after the other.
-        // (All rows of an MMA must use the same channels for a given lane t, so the two rows that share a
-        // shared-memory phase read the same unit: a two-way bank conflict that cannot be swizzled away here.)
+        // 16-byte unit index with the low three bits of (8 row + line) = line.  This warp reads line kq of all 32
+        // rows -- lane (g, t): rows g, g + 8, g + 16, g + 24 -- and of each row the 16-byte unit 2t + h (32 channels):
+        // both 16-row MMA tiles of the stage share one B fragment, so the activations are fetched and permuted
+        // once per 32 rows.  (All rows of an MMA must use the same channels for a given lane t, so the two rows that
+        // share a shared-memory phase read the same unit: a two-way bank conflict that cannot be swizzled away here.)
         const int line = kq;
-        const uint32_t unit_off0 = (uint32_t)(((2 * t) ^ line) << 4), unit_off1 = (uint32_t)(((2 * t + 1) ^ line) << 4);
+        const uint32_t unit_off = (uint32_t)(((2 * t + h) ^ line) << 4);
         int slot = 0;
         uint32_t ph = 0, sync_ph = 0;
         bool ok = true;
@@ -234,38 +256,56 @@ weight_stream_kernel(const __grid_constant__ CUtensorMap map_w, const StreamPara
             const int64_t j0 = (int64_t)rg * kRowsCta;
             for (int pass = 0; pass < passes && ok; ++pass) {
                 const int64_t t0 = (int64_t)pass * kTok;
-                AccT acc[GROUPS][4];
+                AccT acc[2][GROUPS][4];                      // [row tile][token group][C fragment]
+#pragma unroll
+                for (int r = 0; r < 2; ++r)
+#pragma unroll
+                    for (int q = 0; q < GROUPS; ++q)
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) acc[r][q][i] = 0;
+                // float modes: sum of the tokens' activations over this warp's channels (see codes_plus136_bf16x2).  It does
+                // not depend on the rows: with one pass per row group the CTA's first row group computes it for all
+                [[maybe_unused]] const bool do_sum = MODE != kModeInt && (passes > 1 || rg == (int)blockIdx.x);
+                [[maybe_unused]] float acc_s[GROUPS][4];
 #pragma unroll
                 for (int q = 0; q < GROUPS; ++q)
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) acc[q][i] = 0;
+                    for (int i = 0; i < 4; ++i) acc_s[q][i] = 0.0f;
                 XFrag<MODE> xf[GROUPS];
-                // step = 2 * stage + unit: the lane's 32 channels of that unit
-                auto load_x = [&](int step) {
-                    const int c = (step >> 1) * kStageCh + kq * 256 + 64 * t + 32 * (step & 1);
+                // the lane's 32 channels of stage s
+                auto load_x = [&](int s) {
+                    const int c = s * kStageCh + kq * 256 + 32 * (2 * t + h);
 #pragma unroll
                     for (int q = 0; q < GROUPS; ++q) {
                         const int64_t tok = t0 + 8 * q + g;
-                        xf[q].load(xp + tok * p.ldx + c, tok < p.M && c < p.K);
+                        xf[q].fetch(xp + tok * p.ldx + c, tok < p.M && c < p.K);
                     }
                 };
                 load_x(0);
                 for (int s = 0; s < stages_k; ++s) {
                     ok = mbar_wait_all(smem_u32(&s_full[slot]), ph, abort_flag, p.watchdog, kWdStreamFull);
                     if (!ok) break;
-                    const uint32_t rowa = ring + slot * kStageBytes + (uint32_t)(((16 * rt + g) * kLines + line) * 128);
-                    const uint32_t rowb = rowa + 8 * kLines * 128;
-                    const uint4 wq[2][2] = {{lds128(rowa + unit_off0), lds128(rowb + unit_off0)},
-                                            {lds128(rowa + unit_off1), lds128(rowb + unit_off1)}};
+                    const uint32_t row0 = ring + slot * kStageBytes + (uint32_t)((g * kLines + line) * 128) + unit_off;
+                    uint4 wq[4];                             // rows g, g + 8, g + 16, g + 24
+#pragma unroll
+                    for (int r = 0; r < 4; ++r) wq[r] = lds128(row0 + (uint32_t)(r * 8 * kLines * 128));
                     __syncwarp();
                     if (elect_one()) mbar_arrive(smem_u32(&s_empty[slot]));
                     if (++slot == p.depth) { slot = 0; ph ^= 1u; }
                     const bool exists = s * kStageCh + kq * 256 < p.K;     // (warp-uniform) the line is inside the row
+                    // this stage's activations arrived a stage ago: form the fragments, then put the next stage's loads in
+                    // flight behind this stage's MMAs (after them for binary32 activations, whose three fragments per token
+                    // leave no registers for both)
+                    constexpr bool kAhead = MODE != kModeF32;
 #pragma unroll
-                    for (int u = 0; u < 2; ++u) {
-                        const uint32_t w0[4] = {wq[u][0].x, wq[u][0].y, wq[u][0].z, wq[u][0].w};   // row g
-                        const uint32_t w1[4] = {wq[u][1].x, wq[u][1].y, wq[u][1].z, wq[u][1].w};   // row g + 8
-                        if (exists) {
+                    for (int q = 0; q < GROUPS; ++q) xf[q].permute();
+                    if (kAhead && s + 1 < stages_k) load_x(s + 1);
+                    XFrag<MODE>* xc = xf;
+                    if (exists) {
+#pragma unroll
+                        for (int r = 0; r < 2; ++r) {
+                            const uint32_t w0[4] = {wq[2 * r].x, wq[2 * r].y, wq[2 * r].z, wq[2 * r].w};                   // row 16 r + g
+                            const uint32_t w1[4] = {wq[2 * r + 1].x, wq[2 * r + 1].y, wq[2 * r + 1].z, wq[2 * r + 1].w};   // row 16 r + g + 8
                             if (MODE == kModeInt) {
 #pragma unroll
                                 for (int w = 0; w < 4; ++w) {
@@ -273,37 +313,55 @@ weight_stream_kernel(const __grid_constant__ CUtensorMap map_w, const StreamPara
                                                            w0[w] & 0xF0F0F0F0u, w1[w] & 0xF0F0F0F0u};
 #pragma unroll
                                     for (int q = 0; q < GROUPS; ++q)
-                                        mma_s8(reinterpret_cast<int*>(acc[q]), a, xf[q].b[0][2 * w], xf[q].b[0][2 * w + 1]);
+                                        mma_s8(reinterpret_cast<int*>(acc[r][q]), a, xc[q].b[0][2 * w], xc[q].b[0][2 * w + 1]);
                                 }
                             } else {
 #pragma unroll
                                 for (int w = 0; w < 4; ++w)
 #pragma unroll
                                     for (int m = 0; m < 2; ++m) {      // channels (2m, 2m+4 | 2m+1, 2m+5) of the word
-                                        const uint32_t a[4] = {codes_bf16x2(w0[w], 2 * m), codes_bf16x2(w1[w], 2 * m),
-                                                               codes_bf16x2(w0[w], 2 * m + 1), codes_bf16x2(w1[w], 2 * m + 1)};
+                                        const uint32_t a[4] = {codes_plus136_bf16x2(w0[w], 2 * m), codes_plus136_bf16x2(w1[w], 2 * m),
+                                                               codes_plus136_bf16x2(w0[w], 2 * m + 1), codes_plus136_bf16x2(w1[w], 2 * m + 1)};
 #pragma unroll
                                         for (int q = 0; q < GROUPS; ++q)
 #pragma unroll
                                             for (int tm = 0; tm < kTerms; ++tm)
-                                                mma_bf16(reinterpret_cast<float*>(acc[q]), a, xf[q].b[tm][4 * w + 2 * m],
-                                                         xf[q].b[tm][4 * w + 2 * m + 1]);
+                                                mma_bf16(reinterpret_cast<float*>(acc[r][q]), a, xc[q].b[tm][4 * w + 2 * m],
+                                                         xc[q].b[tm][4 * w + 2 * m + 1]);
                                     }
                             }
                         }
-                        // the next unit's activations: in flight while this one's MMAs (or the barrier wait) run
-                        if (2 * s + u + 1 < 2 * stages_k) load_x(2 * s + u + 1);
+                        if (MODE != kModeInt && do_sum) {
+                            const uint32_t ones[4] = {0x3F803F80u, 0x3F803F80u, 0x3F803F80u, 0x3F803F80u};   // bf16 1.0
+#pragma unroll
+                            for (int i = 0; i < 8; ++i)
+#pragma unroll
+                                for (int q = 0; q < GROUPS; ++q)
+#pragma unroll
+                                    for (int tm = 0; tm < kTerms; ++tm)
+                                        mma_bf16(acc_s[q], ones, xc[q].b[tm][2 * i], xc[q].b[tm][2 * i + 1]);
+                        }
                     }
+                    if (!kAhead && s + 1 < stages_k) load_x(s + 1);
                 }
                 if (!ok) break;
                 // C fragment: [0..1] = row g, tokens 2t, 2t+1; [2..3] = row g + 8
-                AccT* part = s_part + (size_t)kq * kRowsCta * (kTok + 1);
+                AccT* part = s_part + (size_t)warp * kRowsCta * (kTok + 1);
 #pragma unroll
-                for (int q = 0; q < GROUPS; ++q) {
-                    part[(16 * rt + g) * (kTok + 1) + 8 * q + 2 * t] = acc[q][0];
-                    part[(16 * rt + g) * (kTok + 1) + 8 * q + 2 * t + 1] = acc[q][1];
-                    part[(16 * rt + g + 8) * (kTok + 1) + 8 * q + 2 * t] = acc[q][2];
-                    part[(16 * rt + g + 8) * (kTok + 1) + 8 * q + 2 * t + 1] = acc[q][3];
+                for (int r = 0; r < 2; ++r)
+#pragma unroll
+                    for (int q = 0; q < GROUPS; ++q) {
+                        part[(16 * r + g) * (kTok + 1) + 8 * q + 2 * t] = acc[r][q][0];
+                        part[(16 * r + g) * (kTok + 1) + 8 * q + 2 * t + 1] = acc[r][q][1];
+                        part[(16 * r + g + 8) * (kTok + 1) + 8 * q + 2 * t] = acc[r][q][2];
+                        part[(16 * r + g + 8) * (kTok + 1) + 8 * q + 2 * t + 1] = acc[r][q][3];
+                    }
+                if (MODE != kModeInt && do_sum && g == 0) {      // every row of the ones product holds the same sums: row 0
+#pragma unroll
+                    for (int q = 0; q < GROUPS; ++q) {
+                        s_xsum[warp * kTok + 8 * q + 2 * t] = acc_s[q][0];
+                        s_xsum[warp * kTok + 8 * q + 2 * t + 1] = acc_s[q][1];
+                    }
                 }
                 __syncwarp();
                 if (elect_one()) mbar_arrive(smem_u32(&s_sync));
@@ -314,7 +372,13 @@ weight_stream_kernel(const __grid_constant__ CUtensorMap map_w, const StreamPara
                     const int row = o % kRowsCta, tok = o / kRowsCta;    // consecutive threads: consecutive channels
                     AccT sum = 0;
 #pragma unroll
-                    for (int k = 0; k < 8; ++k) sum += s_part[((size_t)k * kRowsCta + row) * (kTok + 1) + tok];
+                    for (int k = 0; k < kConsumers; ++k) sum += s_part[((size_t)k * kRowsCta + row) * (kTok + 1) + tok];
+                    if (MODE != kModeInt) {
+                        float xs = 0.0f;
+#pragma unroll
+                        for (int k = 0; k < kConsumers; ++k) xs += s_xsum[k * kTok + tok];
+                        sum = (AccT)fmaf(-kCodeOffset, xs, (float)sum);
+                    }
                     const int64_t j = j0 + row, tt = t0 + tok;
                     if (j < p.N && tt < p.M) {
                         if (MODE == kModeInt && p.acc_out != nullptr) {
@@ -348,7 +412,7 @@ template <int MODE, int GROUPS>
 cudaError_t launch_stream(const CUtensorMap& map, StreamParams p, cudaStream_t stream) {
     typedef typename std::conditional<MODE == kModeInt, int, float>::type AccT;
     const int sms = device_sm_count();
-    const size_t part_bytes = (size_t)8 * kRowsCta * (8 * GROUPS + 1) * sizeof(AccT);
+    const size_t part_bytes = (size_t)kConsumers * kRowsCta * (8 * GROUPS + 1) * sizeof(AccT) + (size_t)kConsumers * 8 * GROUPS * sizeof(float);
     const size_t budget = 227 * 1024 - 1024 /*alignment*/ - 1024 /*static*/ - part_bytes;
     int depth = (int)(budget / kStageBytes);
     if (depth > kMaxDepth) depth = kMaxDepth;
@@ -411,10 +475,13 @@ bool build_stream_tmap(Weights& W) {
 }
 
 bool gemm_stream_applies(int64_t M, const Weights& W) {
-    // measured against the tcgen05 kernel: ahead for at most 8 tokens on matrices up to 32 Mi weights and for at
-    // most 16 tokens up to 16 Mi
+    // Measured against the tcgen05 kernel over M in {1, 8, 16} x K, N in {4096, 8192, 16384}: ahead (or level) wherever the
+    // row groups make at most two rounds over the SMs (N <= 64 x SMs: 4096 and 8192 rows) -- every row group ends with a
+    // rendezvous and a reduction, which four rounds of short rows (K = 4096, N = 16384: 19 us against 10 us) do not amortise --
+    // up to 128 Mi weights for at most 8 tokens and 64 Mi for at most 16 (16 x 16384 x 8192: 23 us against 21 us).
     if (W.bits != 4 || !W.tmap_stream_valid || M < 1 || M > 16) return false;
-    return W.N * W.K <= (M <= 8 ? (1ll << 25) : (1ll << 24));
+    if (W.N > 64ll * device_sm_count()) return false;
+    return W.N * W.K <= (M <= 8 ? (1ll << 27) : (1ll << 26));
 }
 
 cudaError_t launch_gemm_stream(const int8_t* a8, int64_t M, const Weights& W, int acc_shift, const GemmOut& out,
@@ -445,9 +512,10 @@ cudaError_t launch_linear_wonly4(const void* x, fq_dtype xt, int64_t M, int64_t 
     StreamParams p{};
     p.x = x; p.ldx = ldx; p.M = M; p.N = W.N; p.K = (int)W.K;
     p.w_scale = W.w_scale; p.bias = W.bias; p.y = y; p.yt = yt; p.ldy = ldy;
+    // eight tokens per pass over the weights: two token groups at a time need more registers than a thread has
+    // (16 tokens measured 130 us against 2 x 59 us at 16384 x 16384)
     if (xt == FQ_F32) return launch_stream<kModeF32, 1>(W.tmap_stream, p, stream);
-    if (M <= 8) return launch_stream<kModeBf16, 1>(W.tmap_stream, p, stream);
-    return launch_stream<kModeBf16, 2>(W.tmap_stream, p, stream);
+    return launch_stream<kModeBf16, 1>(W.tmap_stream, p, stream);
 }
 
 }  // namespace fq

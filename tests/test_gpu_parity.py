@@ -611,6 +611,7 @@ SWEEP_SAMPLE = [
     # M, K=N, block, bits  (a sample of the throughput-sweep grid; outputs checked on sampled token rows)
     (1, 1024, 32, 4), (1, 4096, 256, 8), (16, 2048, 64, 4), (64, 1024, 128, 8), (256, 4096, 32, 8),
     (256, 2048, 256, 4), (1024, 1024, 64, 4), (1024, 4096, 128, 8), (4096, 2048, 128, 4),
+    (8, 8192, 128, 4), (16, 8192, 64, 4),      # the weight-streaming kernel at its largest square (64 Mi weights)
 ]
 
 
@@ -809,6 +810,23 @@ def test_linear_w4a16_matches_oracle(M, N, K, xdtype, ydtype):
     # it does what it is for: the 4-bit weights reproduce the float projection to RTN accuracy
     ref = synth.to_f32(x, xdtype).astype(np.float64) @ W.astype(np.float64).T + bias
     assert np.linalg.norm(as_f64(to_np(y)) - ref) / np.linalg.norm(ref) < 0.2
+
+
+@pytest.mark.parametrize("M,N,K,xdtype,mean", [(9, 512, 8192, "f32", 4.0), (1, 8192, 8192, "bf16", 0.0), (8, 1024, 16384, "bf16", -2.0)])
+def test_linear_w4a16_long_rows_and_activations_with_a_mean(M, N, K, xdtype, mean):
+    """The kernel multiplies the codes 136 too large and takes 136 x (sum of the token's activations) off each output:
+    activations whose sum is far from zero (mean / sigma up to 4, K up to 16384) are where that cancellation costs the
+    most binary32 digits.  Same tolerance as everywhere; also the largest rows the streaming ring sees here."""
+    rng = np.random.default_rng(M + N + K)
+    q = rng.integers(-8, 8, size=(N, K)).astype(np.int32)
+    wc = oracle.pack(q, 4)
+    ws = np.exp2(rng.uniform(-9, -7, size=N)).astype(np.float32)
+    bias = rng.standard_normal(N).astype(np.float32)
+    x = synth.as_dtype((mean + rng.standard_normal((M, K))).astype(np.float32), xdtype)
+    h = fq.weights_import(to_dev(wc), to_dev(ws), None, to_dev(bias), K, 1, 4)
+    want = oracle.linear_wonly(x, xdtype, wc, ws, bias, 4, "f32")
+    y = fq.linear_w4a16(to_dev(x, xdtype), h, torch.float32)
+    assert_close(to_np(y), want, "f32", f"w4a16 mean {mean} {M}x{N}x{K}")
 
 
 def test_linear_w4a16_exact_on_integer_activations_and_edges():
