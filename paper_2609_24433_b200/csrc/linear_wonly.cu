@@ -475,7 +475,7 @@ bool build_stream_tmap(Weights& W) {
 }
 
 bool gemm_stream_applies(int64_t M, const Weights& W) {
-    // Measured against the tcgen05 kernel over M in {1, 8, 16} x K, N in {4096, 8192, 16384}: ahead (or level) wherever the
+    // Measured against the tcgen05 kernel over M in {1, 8, 16} x K, N in {4096, 8192, 16384}, operands from HBM: ahead wherever the
     // row groups make at most two rounds over the SMs (N <= 64 x SMs: 4096 and 8192 rows) -- every row group ends with a
     // rendezvous and a reduction, which four rounds of short rows (K = 4096, N = 16384: 19 us against 10 us) do not amortise --
     // up to 128 Mi weights for at most 8 tokens and 64 Mi for at most 16 (16 x 16384 x 8192: 23 us against 21 us).
