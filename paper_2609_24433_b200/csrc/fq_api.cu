@@ -398,7 +398,7 @@ fq_status fq_fold_weights_gptq(const void* Wsrc, fq_dtype wt, int64_t N, int64_t
     *out = nullptr;
     fq_status st = check_shape(N, K, hadamard_block, bits);
     if (st != FQ_OK) return st;
-    if (K > 4096) return FQ_ERR_UNSUPPORTED;          // K x K factorisation in shared-nothing column steps
+    if (K > 16384) return FQ_ERR_UNSUPPORTED;         // three K x K binary32 matrices; a row of K floats per CTA in shared memory
     if ((wt != FQ_F32 && wt != FQ_BF16) || (ct != FQ_F32 && ct != FQ_BF16)) return FQ_ERR_INVALID_ARG;
     if (!calib || Mc < 1 || ldc < K || !(damp >= 0.0f)) return FQ_ERR_INVALID_ARG;
     if (N > 0 && (!Wsrc || ldw < K)) return FQ_ERR_INVALID_ARG;

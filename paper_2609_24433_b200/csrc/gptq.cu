@@ -89,10 +89,9 @@ __global__ void damp_kernel(float* __restrict__ H, int K, float damp, uint8_t* _
 // finished entries M[j][k], k > j, into shared memory (all threads load, so the strided reads overlap),
 // then recomputes the diagonal entry from them (one chain of at most K terms) instead of waiting for
 // another CTA to publish it; the off-diagonal chains read the same copy.
-constexpr int kMaxK = 4096;
 __global__ void __launch_bounds__(256)
 rev_chol_col_kernel(const float* __restrict__ H, float* __restrict__ Mt, int K, int j, int* __restrict__ bad) {
-    __shared__ float s_mj[kMaxK];                    // s_mj[k - j - 1] = M[j][k]
+    extern __shared__ float s_mj[];                  // K floats: s_mj[k - j - 1] = M[j][k]
     __shared__ float s_d;
     const int n = K - 1 - j;
     for (int o = threadIdx.x; o < n; o += blockDim.x) s_mj[o] = Mt[(int64_t)(j + 1 + o) * K + j];
@@ -155,9 +154,9 @@ tri_inverse_kernel(const float* __restrict__ Mt, float* __restrict__ U, int K) {
     }
 }
 
-// The sweep is independent per weight row: a CTA keeps kRows rows in shared memory and walks the channels.
-constexpr int kSweepRows = 4;
-template <int BITS>
+// The sweep is independent per weight row: a CTA keeps kSweepRows rows in shared memory (four; two of the longest
+// rows, which would not fit otherwise) and walks the channels.
+template <int BITS, int kSweepRows>
 __global__ void __launch_bounds__(256)
 gptq_sweep_kernel(const float* __restrict__ Wt, int64_t N, int K, const float* __restrict__ U,
                   const uint8_t* __restrict__ dead, const float* __restrict__ w_scale, uint8_t* __restrict__ codes) {
@@ -237,27 +236,38 @@ cudaError_t launch_gptq_factor(const float* z, int64_t Mc, int64_t K, float damp
     damp_kernel<<<1, 256, 0, stream>>>(H, (int)K, damp, dead);
     cudaError_t e = cudaMemsetAsync(Mt, 0, sizeof(float) * (size_t)K * (size_t)K, stream);
     if (e != cudaSuccess) return e;
+    const size_t col_smem = sizeof(float) * (size_t)K;
+    e = ensure_dynamic_smem(reinterpret_cast<const void*>(rev_chol_col_kernel), col_smem);
+    if (e != cudaSuccess) return e;
     for (int j = (int)K - 1; j >= 0; --j)
-        rev_chol_col_kernel<<<(unsigned)(j / 256 + 1), 256, 0, stream>>>(H, Mt, (int)K, j, bad);
+        rev_chol_col_kernel<<<(unsigned)(j / 256 + 1), 256, col_smem, stream>>>(H, Mt, (int)K, j, bad);
     tri_inverse_kernel<<<(unsigned)((K + 127) / 128), 128, 0, stream>>>(Mt, U, (int)K);
     return cudaGetLastError();
 }
 
+namespace {
+template <int BITS, int ROWS>
+cudaError_t launch_sweep_variant(const float* Wt, int64_t N, int64_t K, const float* U, const uint8_t* dead,
+                                 const float* w_scale, uint8_t* codes, cudaStream_t stream) {
+    const size_t smem = sizeof(float) * (size_t)ROWS * (size_t)K;
+    const unsigned grid = (unsigned)((N + ROWS - 1) / ROWS);
+    auto kern = gptq_sweep_kernel<BITS, ROWS>;
+    cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), smem);
+    if (e != cudaSuccess) return e;
+    kern<<<grid, 256, smem, stream>>>(Wt, N, (int)K, U, dead, w_scale, codes);
+    return cudaGetLastError();
+}
+}  // namespace
+
 cudaError_t launch_gptq_sweep(const float* Wt, int64_t N, int64_t K, const float* U, const uint8_t* dead,
                               const float* w_scale, int bits, uint8_t* codes, cudaStream_t stream) {
     if (N == 0) return cudaSuccess;
-    const size_t smem = sizeof(float) * (size_t)kSweepRows * (size_t)K;
-    const unsigned grid = (unsigned)((N + kSweepRows - 1) / kSweepRows);
-    if (bits == 4) {
-        cudaError_t e = cudaFuncSetAttribute(gptq_sweep_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-        gptq_sweep_kernel<4><<<grid, 256, smem, stream>>>(Wt, N, (int)K, U, dead, w_scale, codes);
-    } else {
-        cudaError_t e = cudaFuncSetAttribute(gptq_sweep_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-        gptq_sweep_kernel<8><<<grid, 256, smem, stream>>>(Wt, N, (int)K, U, dead, w_scale, codes);
-    }
-    return cudaGetLastError();
+    // four rows of K floats per CTA up to K = 8192 (128 KB), two beyond (K <= 16384: 128 KB)
+    if (K <= 8192)
+        return bits == 4 ? launch_sweep_variant<4, 4>(Wt, N, K, U, dead, w_scale, codes, stream)
+                         : launch_sweep_variant<8, 4>(Wt, N, K, U, dead, w_scale, codes, stream);
+    return bits == 4 ? launch_sweep_variant<4, 2>(Wt, N, K, U, dead, w_scale, codes, stream)
+                     : launch_sweep_variant<8, 2>(Wt, N, K, U, dead, w_scale, codes, stream);
 }
 
 }  // namespace fq

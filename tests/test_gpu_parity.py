@@ -995,7 +995,7 @@ def test_fold_weights_gptq_backbone_width_sampled_and_errors():
     assert np.array_equal(to_np(hs).view(np.uint32), ws.view(np.uint32))
     assert np.array_equal(to_np(hc), wc)
     with pytest.raises(fq.FqError) as e:
-        fq.fold_weights_gptq(torch.zeros((8, 8192), device="cuda"), None, None, torch.zeros((4, 8192), device="cuda"), 64, 4)
+        fq.fold_weights_gptq(torch.zeros((8, 32768), device="cuda"), None, None, torch.zeros((4, 32768), device="cuda"), 64, 4)
     assert e.value.status == fq.ERR_UNSUPPORTED
     # two channels that always fire together and no damping: the second moment is exactly singular
     twin = 2.0 * np.eye(32, dtype=np.float32)
@@ -1005,6 +1005,34 @@ def test_fold_weights_gptq_backbone_width_sampled_and_errors():
     assert e.value.status == fq.ERR_INVALID_ARG
     with pytest.raises(RuntimeError):
         oracle.gptq_factor(twin, 0.0)
+
+
+def test_fold_weights_gptq_long_rows_by_properties():
+    """K = 8192: beyond what the oracle's cubic factorisation finishes in test time, so properties instead of codes.
+    The handle keeps the round-to-nearest steps; the codes stay in range; and on the calibration tokens the GPTQ
+    codes reconstruct the transformed weights' outputs better than round-to-nearest does -- the objective of Eq. 7,
+    evaluated in binary64 from the oracle's transformed weights and tokens."""
+    rng = np.random.default_rng(21)
+    N, K, Mc, block = 16, 8192, 192, 256
+    W = synth.draw_weights(rng, N, K)
+    calib = _correlated_calib(rng, Mc, K, rank=32)
+    wc_rtn, ws, g, wt = oracle.fold_weights(W, "f32", None, block, 4, return_wt=True)
+    z = (calib * g[None, :]).astype(np.float32)
+    for t in range(Mc):
+        for b0 in range(0, K, block):
+            z[t, b0:b0 + block] = oracle.fwht_block(z[t, b0:b0 + block])
+    h = fq.fold_weights_gptq(to_dev(W), None, None, to_dev(calib), block, 4, 0.01)
+    hc, hs, _, _ = h.export()
+    assert np.array_equal(to_np(hs).view(np.uint32), ws.view(np.uint32))
+    q_gptq = oracle.unpack(to_np(hc), K, 4).astype(np.float64)
+    q_rtn = oracle.unpack(wc_rtn, K, 4).astype(np.float64)
+    assert np.abs(q_gptq).max() <= 7
+    z64 = z.astype(np.float64)
+
+    def objective(q):
+        return np.linalg.norm((wt.astype(np.float64) - ws.astype(np.float64)[:, None] * q) @ z64.T)
+
+    assert objective(q_gptq) < 0.8 * objective(q_rtn), (objective(q_gptq), objective(q_rtn))
 
 
 # ------------------------------------------------- gate product fused into the prologue ----
