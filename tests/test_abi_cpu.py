@@ -114,7 +114,7 @@ def test_argument_checks_of_the_widened_entry_points(lib):
         return lib.fq_fold_weights_gptq(one, 0, i64(8), i64(K), i64(K), null, null, calib, 0, i64(Mc), i64(K), 64, 4,
                                         f32(damp), null, ctypes.byref(out))
 
-    assert gptq(8192, 16, one, 0.01) == fq.ERR_UNSUPPORTED            # K beyond the factorisation's limit
+    assert gptq(32768, 16, one, 0.01) == fq.ERR_UNSUPPORTED           # K beyond the factorisation's limit
     assert gptq(1024, 16, null, 0.01) == fq.ERR_INVALID_ARG           # no calibration tokens
     assert gptq(1024, 0, one, 0.01) == fq.ERR_INVALID_ARG
     assert gptq(1024, 16, one, -1.0) == fq.ERR_INVALID_ARG
