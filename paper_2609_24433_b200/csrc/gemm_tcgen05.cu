@@ -1169,8 +1169,11 @@ struct Plan {
 // Pairs gain nothing for 4-bit weights, which never pass through shared memory unpacked.
 // K split (single CTAs, and CTA pairs on 8-bit weights): problems with fewer tiles than SMs and a long K (every short batch; down_proj
 // at M = 816: 64 tiles of 128 k-blocks) make `split` work units of every tile, each on a slice of K; the
-// slices leave int32 partial sums in scratch and the one that finishes last adds them up (fitted cost per
-// unit: 1500 + 70*bt cycles, plus 8*bt per extra slice).
+// slices leave int32 partial sums in scratch and the one that finishes last adds them up.  Fitted cost per
+// unit: 12500 + 40*bt cycles, plus 1500 per extra slice -- the constant is what a split costs a call on operands
+// from HBM whatever its size (the node that clears the counters ahead of the prologue, two rendezvous, the
+// round trips of the exchange: 16-25 thousand cycles measured at tiles of 16 and 64 tokens split in 2, 4 and 8,
+// where an earlier model of 1500 + 70*bt chose splits that ran 15-45 % slower than the same tile unsplit).
 Plan plan_gemm(int64_t M, int64_t N, int64_t K, int bits, int sms, size_t scratch_avail) {
     const int bt_max = bits == 4 ? 208 : 256;
     const int64_t kb = (K + kBlockK - 1) / kBlockK;
@@ -1202,7 +1205,7 @@ Plan plan_gemm(int64_t M, int64_t N, int64_t K, int bits, int sms, size_t scratc
                 const size_t scratch = sp > 1 ? kCounterBytes + (size_t)units * c * sp * kTileN * b * sizeof(int32_t) : 0;
                 if (scratch > scratch_avail) continue;
                 const int slots = sms / c;
-                const double unit_cost = (double)kb_per * per_kb + 16.0 * b + 1000.0 + (sp > 1 ? 1500.0 + 70.0 * b + 8.0 * b * (sp - 1) : 0.0);
+                const double unit_cost = (double)kb_per * per_kb + 16.0 * b + 1000.0 + (sp > 1 ? 12500.0 + 40.0 * b + 1500.0 * (sp - 1) : 0.0);
                 const double cost = (double)((units * sp + slots - 1) / slots) * unit_cost;
                 if (best.bt == 0 || cost < best_cost * 0.98) {   // ties: the earlier candidate (larger tile, no split)
                     best.bt = b; best.ctas = c; best.split = sp; best.scratch = scratch;

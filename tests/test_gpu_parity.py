@@ -368,7 +368,7 @@ def test_accumulator_extremes_and_one_hot(bits):
     assert np.array_equal(to_np(got), wi.T)
 
 
-@pytest.mark.parametrize("M,N,K,bits", [(16, 256, 8192, 4), (208, 384, 16384, 8), (9, 128, 16384, 4), (64, 256, 8192, 8)])
+@pytest.mark.parametrize("M,N,K,bits", [(100, 256, 16384, 4), (208, 384, 16384, 8), (130, 128, 16384, 4), (64, 256, 16384, 8)])
 def test_k_split_equals_unsplit_and_oracle(M, N, K, bits):
     """Few tiles and a long K: the planner splits K over a CTA cluster when the workspace has room
     for the partial sums.  With a workspace that holds only the activation codes and steps the same
@@ -677,7 +677,7 @@ def test_one_handle_three_streams_three_workspaces():
     """A weight handle is read-only at run time: consumers of one handle on three streams, each with its own
     workspace (K split included), give what the same calls give one after the other."""
     rng = np.random.default_rng(12)
-    M, K, N = 16, 8192, 256                     # few tiles, long K: the planner splits K when scratch is there
+    M, K, N = 100, 16384, 256                   # few tiles, long K: the planner splits K when scratch is there
     W = synth.draw_weights(rng, N, K)
     h = fq.fold_weights(to_dev(W), None, None, 128, 4)
     need = fq.workspace_bytes(M, K, N, 4)
@@ -700,7 +700,8 @@ def test_one_handle_three_streams_three_workspaces():
 
 
 @pytest.mark.parametrize("M,K,N,bits", [(50, 1024, 3072, 4), (50, 4096, 1024, 4), (16, 8192, 8192, 4), (64, 8192, 8192, 4),
-                                        (256, 4096, 4096, 4), (816, 2048, 2560, 4), (64, 8192, 2048, 8), (816, 2048, 2048, 8)])
+                                        (256, 4096, 4096, 4), (816, 2048, 2560, 4), (64, 8192, 2048, 8), (816, 2048, 2048, 8),
+                                        (100, 16384, 256, 4), (64, 16384, 256, 8)])      # the last two split K
 def test_linear_replayed_in_a_cuda_graph_equals_the_eager_call(M, K, N, bits):
     """The benchmark and any latency-minded caller replay the one-call path from CUDA graphs, where the prologue, the
     GEMM (programmatic dependent launch) and the K split's counter memset really overlap and follow each other
