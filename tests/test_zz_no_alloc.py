@@ -60,3 +60,22 @@ def test_static_scratch_rejects_what_does_not_fit_and_bad_arguments():
     assert fq.lib().fq_linear_w4a4_static(null, 0, ctypes.c_int64(4), ctypes.c_int64(K), h4.handle,
                                           ctypes.c_float(1.0), null, 0, ctypes.c_int64(N), null) == fq.ERR_INVALID_ARG
     torch.cuda.synchronize()
+
+
+def test_static_scratch_calls_leave_the_device_memory_as_it_was():
+    """After the start-up call (zero tokens: it loads the module that holds the scratch), calls of the workspace-free
+    entry point take no device memory: the free-memory figure the driver reports is the same before and after."""
+    data = _site(200, 1024, 264, "bf16", 3)
+    x = to_dev(data.x, "bf16")
+    h = fq.fold_weights(to_dev(data.W["p"]), None, to_dev(data.bias["p"]), 128, 4)
+    y = torch.empty((200, 264), dtype=torch.bfloat16, device="cuda")
+    fq.linear_w4a4_static(x[:0], h, 1.0, y=y[:0])          # start-up call
+    fq.linear_w4a4_static(x, h, 1.0, y=y)                  # and one full call, so that every kernel's module is resident
+    torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info()
+    for _ in range(5):
+        fq.linear_w4a4_static(x, h, 1.0, y=y)
+    torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert free_after == free_before
+    assert torch.equal(y, fq.linear_w4a4(x, h, 1.0, torch.bfloat16))
