@@ -372,12 +372,13 @@ weight_stream_kernel(const __grid_constant__ CUtensorMap map_w, const StreamPara
                     const int row = o % kRowsCta, tok = o / kRowsCta;    // consecutive threads: consecutive channels
                     AccT sum = 0;
 #pragma unroll
-                    for (int k = 0; k < kConsumers; ++k) sum += s_part[((size_t)k * kRowsCta + row) * (kTok + 1) + tok];
-                    if (MODE != kModeInt) {
-                        float xs = 0.0f;
-#pragma unroll
-                        for (int k = 0; k < kConsumers; ++k) xs += s_xsum[k * kTok + tok];
-                        sum = (AccT)fmaf(-kCodeOffset, xs, (float)sum);
+                    for (int k = 0; k < kConsumers; ++k) {
+                        const AccT part_k = s_part[((size_t)k * kRowsCta + row) * (kTok + 1) + tok];
+                        // float modes: the offset comes off warp by warp, each warp's sum of activations against its own
+                        // products (the same channels), before the sixteen slices are added: the cancellation then acts
+                        // on a sixteenth of the row at a time
+                        if (MODE != kModeInt) sum += (AccT)fmaf(-kCodeOffset, s_xsum[k * kTok + tok], (float)part_k);
+                        else sum += part_k;
                     }
                     const int64_t j = j0 + row, tt = t0 + tok;
                     if (j < p.N && tt < p.M) {
