@@ -46,6 +46,21 @@ def test_workspace_bytes_is_a_host_computation(lib):
     assert fq.workspace_bytes(64, 1024, 1024, 8) >= 64 * 1024
 
 
+def test_planner_splits_k_only_where_it_measured_faster(lib):
+    """The workspace a shape asks for tells whether the planner would split K (scratch for the partial sums beyond the
+    codes and steps).  On operands from HBM a split costs a call 16-25 thousand cycles, so short batches on square
+    matrices and the backbone's sites run unsplit; a few tiles on a very long K still split.  (Without a device the
+    planner assumes 148 SMs.)"""
+    def base(M, K):
+        return (M * K + 255) // 256 * 256 + (4 * M + 255) // 256 * 256
+
+    for M, K, N, bits in [(64, 4096, 4096, 8), (50, 4096, 1024, 8), (16, 8192, 8192, 8), (50, 4096, 1024, 4),
+                          (816, 16384, 2048, 8), (816, 2048, 32768, 4), (16384, 8192, 8192, 4)]:
+        assert fq.workspace_bytes(M, K, N, bits) == base(M, K), (M, K, N, bits)
+    for M, K, N, bits in [(50, 16384, 1024, 8), (100, 16384, 256, 4), (208, 16384, 384, 8)]:
+        assert fq.workspace_bytes(M, K, N, bits) > base(M, K), (M, K, N, bits)
+
+
 def test_argument_checks_run_before_any_device_work(lib):
     out = ctypes.c_void_p()
     null = ctypes.c_void_p(0)
