@@ -1,8 +1,8 @@
 // Short-batch weight streaming for 4-bit weights: the projection of a handful of tokens is a
 // matrix-vector product bound by the weight bytes, which must cross HBM once.  Two users:
-//   * the W4A4 integer product of Eq. 8 for batches of at most 16 tokens where it measured faster than the
-//     TMA/TMEM pipeline of the big GEMM (see gemm_stream_applies), whose per-k-block hand-overs cannot be fed
-//     at HBM rate by so thin a tile;
+//   * the W4A4 and W8A8 integer products of Eq. 8 for batches of at most 16 tokens where it measured faster than
+//     the TMA/TMEM pipeline of the big GEMM (see gemm_stream_applies), whose per-k-block hand-overs cannot be fed
+//     at HBM rate by so thin a tile (8-bit weights: a line is 128 channels, the bytes enter the MMAs as they are);
 //   * the weight-only projection with floating-point activations (the adaptive layer-normalisation
 //     modulation of the W4A4 engines):  y[t][j] = s^W_j * sum_c qW[j][c] * x[t][c] + b_j.
 // One persistent CTA per SM walks groups of 32 weight rows.  A producer warp streams the packed rows
@@ -40,11 +40,20 @@ namespace {
 constexpr int kConsumers = 16;                  // consumer warps: (row tile, 128-channel slot of a stage)
 constexpr int kThreads = 32 * (kConsumers + 1); // + one producer warp
 constexpr int kRowsCta = 32;                    // two 16-row MMA tiles
-constexpr int kStageCh = 2048;                  // channels per stage
-constexpr int kLines = kStageCh / 256;          // 128-byte lines (256 channels) per row and stage
-constexpr int kStageBytes = kRowsCta * kStageCh / 2;   // one TMA box: 32 rows x 8 lines of 128 bytes (32 KB)
+constexpr int kLines = 8;                       // 128-byte lines per row and stage
+constexpr int kStageBytes = kRowsCta * kLines * 128;   // one TMA box: 32 rows x 8 lines of 128 bytes (32 KB)
 constexpr int kMaxDepth = 6;
-enum : int { kModeInt = 0, kModeBf16 = 1, kModeF32 = 2 };
+// kModeInt: 4-bit weights x int8 activations; kModeBf16 / kModeF32: 4-bit weights x float activations;
+// kModeInt8: 8-bit weights x int8 activations (a line is 128 channels then, a 16-byte unit 16 channels, and the
+// bytes go into the MMAs as they are)
+enum : int { kModeInt = 0, kModeBf16 = 1, kModeF32 = 2, kModeInt8 = 3 };
+template <int MODE>
+struct Geometry {
+    static constexpr bool kIntegers = MODE == kModeInt || MODE == kModeInt8;
+    static constexpr int kLineCh = MODE == kModeInt8 ? 128 : 256;     // channels of a 128-byte line
+    static constexpr int kUnitCh = kLineCh / 8;                       // channels of a 16-byte unit
+    static constexpr int kStageCh = kLines * kLineCh;                 // channels per stage
+};
 
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, uint32_t bar) {
     asm volatile(
@@ -100,6 +109,18 @@ struct XFrag<kModeInt> {
             b[0][4 * h + 0] = raw[h].x; b[0][4 * h + 1] = raw[h].y; b[0][4 * h + 2] = raw[h].z; b[0][4 * h + 3] = raw[h].w;
         }
     }
+};
+// int8 codes in channel order against 8-bit weights: the unit's 16 channels, four per register, as they are
+template <>
+struct XFrag<kModeInt8> {
+    typedef int8_t elem;
+    static constexpr int kTerms = 1;
+    uint4 raw[1];
+    uint32_t b[1][4];
+    __device__ __forceinline__ void fetch(const int8_t* p, bool ok) {
+        raw[0] = ok ? __ldg(reinterpret_cast<const uint4*>(p)) : make_uint4(0u, 0u, 0u, 0u);
+    }
+    __device__ __forceinline__ void permute() { b[0][0] = raw[0].x; b[0][1] = raw[0].y; b[0][2] = raw[0].z; b[0][3] = raw[0].w; }
 };
 // bf16: for word w, b[4w + j] = (channel j, channel j + 4), j = 0..3
 template <>
@@ -179,9 +200,11 @@ __global__ void __launch_bounds__(kThreads, 1)
 weight_stream_kernel(const __grid_constant__ CUtensorMap map_w, const StreamParams p) {
     extern __shared__ uint8_t smem_raw[];
     typedef typename XFrag<MODE>::elem XT;
-    typedef typename std::conditional<MODE == kModeInt, int, float>::type AccT;
+    typedef typename std::conditional<Geometry<MODE>::kIntegers, int, float>::type AccT;
     constexpr int kTerms = XFrag<MODE>::kTerms;
     constexpr int kTok = 8 * GROUPS;
+    constexpr bool kIntegers = Geometry<MODE>::kIntegers;
+    constexpr int kStageCh = Geometry<MODE>::kStageCh, kLineCh = Geometry<MODE>::kLineCh, kUnitCh = Geometry<MODE>::kUnitCh;
     __shared__ uint64_t s_full[kMaxDepth], s_empty[kMaxDepth];
     __shared__ uint64_t s_sync;                       // rendezvous of the consumer warps (bounded, unlike bar.sync)
     __shared__ int s_abort;
@@ -265,7 +288,7 @@ weight_stream_kernel(const __grid_constant__ CUtensorMap map_w, const StreamPara
                         for (int i = 0; i < 4; ++i) acc[r][q][i] = 0;
                 // float modes: sum of the tokens' activations over this warp's channels (see codes_plus136_bf16x2).  It does
                 // not depend on the rows: with one pass per row group the CTA's first row group computes it for all
-                [[maybe_unused]] const bool do_sum = MODE != kModeInt && (passes > 1 || rg == (int)blockIdx.x);
+                [[maybe_unused]] const bool do_sum = !kIntegers && (passes > 1 || rg == (int)blockIdx.x);
                 [[maybe_unused]] float acc_s[GROUPS][4];
 #pragma unroll
                 for (int q = 0; q < GROUPS; ++q)
@@ -274,7 +297,7 @@ weight_stream_kernel(const __grid_constant__ CUtensorMap map_w, const StreamPara
                 XFrag<MODE> xf[GROUPS];
                 // the lane's 32 channels of stage s
                 auto load_x = [&](int s) {
-                    const int c = s * kStageCh + kq * 256 + 32 * (2 * t + h);
+                    const int c = s * kStageCh + kq * kLineCh + kUnitCh * (2 * t + h);
 #pragma unroll
                     for (int q = 0; q < GROUPS; ++q) {
                         const int64_t tok = t0 + 8 * q + g;
@@ -292,7 +315,7 @@ weight_stream_kernel(const __grid_constant__ CUtensorMap map_w, const StreamPara
                     __syncwarp();
                     if (elect_one()) mbar_arrive(smem_u32(&s_empty[slot]));
                     if (++slot == p.depth) { slot = 0; ph ^= 1u; }
-                    const bool exists = s * kStageCh + kq * 256 < p.K;     // (warp-uniform) the line is inside the row
+                    const bool exists = s * kStageCh + kq * kLineCh < p.K;     // (warp-uniform) the line is inside the row
                     // this stage's activations arrived a stage ago: form the fragments, then put the next stage's loads in
                     // flight behind this stage's MMAs (after them for binary32 activations, whose three fragments per token
                     // leave no registers for both)
@@ -306,7 +329,15 @@ weight_stream_kernel(const __grid_constant__ CUtensorMap map_w, const StreamPara
                         for (int r = 0; r < 2; ++r) {
                             const uint32_t w0[4] = {wq[2 * r].x, wq[2 * r].y, wq[2 * r].z, wq[2 * r].w};                   // row 16 r + g
                             const uint32_t w1[4] = {wq[2 * r + 1].x, wq[2 * r + 1].y, wq[2 * r + 1].z, wq[2 * r + 1].w};   // row 16 r + g + 8
-                            if (MODE == kModeInt) {
+                            if constexpr (MODE == kModeInt8) {
+#pragma unroll
+                                for (int w = 0; w < 2; ++w) {      // two MMAs: the unit's bytes 0-7 and 8-15
+                                    const uint32_t a[4] = {w0[2 * w], w1[2 * w], w0[2 * w + 1], w1[2 * w + 1]};
+#pragma unroll
+                                    for (int q = 0; q < GROUPS; ++q)
+                                        mma_s8(reinterpret_cast<int*>(acc[r][q]), a, xc[q].b[0][2 * w], xc[q].b[0][2 * w + 1]);
+                                }
+                            } else if constexpr (MODE == kModeInt) {
 #pragma unroll
                                 for (int w = 0; w < 4; ++w) {
                                     const uint32_t a[4] = {(w0[w] << 4) & 0xF0F0F0F0u, (w1[w] << 4) & 0xF0F0F0F0u,
@@ -331,7 +362,7 @@ weight_stream_kernel(const __grid_constant__ CUtensorMap map_w, const StreamPara
                                     }
                             }
                         }
-                        if (MODE != kModeInt && do_sum) {
+                        if constexpr (!kIntegers) if (do_sum) {
                             const uint32_t ones[4] = {0x3F803F80u, 0x3F803F80u, 0x3F803F80u, 0x3F803F80u};   // bf16 1.0
 #pragma unroll
                             for (int i = 0; i < 8; ++i)
@@ -356,7 +387,7 @@ weight_stream_kernel(const __grid_constant__ CUtensorMap map_w, const StreamPara
                         part[(16 * r + g + 8) * (kTok + 1) + 8 * q + 2 * t] = acc[r][q][2];
                         part[(16 * r + g + 8) * (kTok + 1) + 8 * q + 2 * t + 1] = acc[r][q][3];
                     }
-                if (MODE != kModeInt && do_sum && g == 0) {      // every row of the ones product holds the same sums: row 0
+                if (!kIntegers && do_sum && g == 0) {      // every row of the ones product holds the same sums: row 0
 #pragma unroll
                     for (int q = 0; q < GROUPS; ++q) {
                         s_xsum[warp * kTok + 8 * q + 2 * t] = acc_s[q][0];
@@ -377,16 +408,16 @@ weight_stream_kernel(const __grid_constant__ CUtensorMap map_w, const StreamPara
                         // float modes: the offset comes off warp by warp, each warp's sum of activations against its own
                         // products (the same channels), before the sixteen slices are added: the cancellation then acts
                         // on a sixteenth of the row at a time
-                        if (MODE != kModeInt) sum += (AccT)fmaf(-kCodeOffset, s_xsum[k * kTok + tok], (float)part_k);
+                        if (!kIntegers) sum += (AccT)fmaf(-kCodeOffset, s_xsum[k * kTok + tok], (float)part_k);
                         else sum += part_k;
                     }
                     const int64_t j = j0 + row, tt = t0 + tok;
                     if (j < p.N && tt < p.M) {
-                        if (MODE == kModeInt && p.acc_out != nullptr) {
+                        if (kIntegers && p.acc_out != nullptr) {
                             p.acc_out[tt * p.N + j] = (int)sum >> p.acc_shift;
                         } else {
                             float v;
-                            if (MODE == kModeInt) {
+                            if (kIntegers) {
                                 // (float)sum * 2^-shift is exact: the shift is folded into the channel scale
                                 const float sw = __ldg(p.w_scale + j) * (1.0f / (float)(1 << p.acc_shift));
                                 v = fmaf((float)sum, __ldg(p.a_delta + tt) * sw, __ldg(p.bias + j));
@@ -411,7 +442,7 @@ weight_stream_kernel(const __grid_constant__ CUtensorMap map_w, const StreamPara
 
 template <int MODE, int GROUPS>
 cudaError_t launch_stream(const CUtensorMap& map, StreamParams p, cudaStream_t stream) {
-    typedef typename std::conditional<MODE == kModeInt, int, float>::type AccT;
+    typedef typename std::conditional<Geometry<MODE>::kIntegers, int, float>::type AccT;
     const int sms = device_sm_count();
     const size_t part_bytes = (size_t)kConsumers * kRowsCta * (8 * GROUPS + 1) * sizeof(AccT) + (size_t)kConsumers * 8 * GROUPS * sizeof(float);
     const size_t budget = 227 * 1024 - 1024 /*alignment*/ - 1024 /*static*/ - part_bytes;
@@ -466,10 +497,11 @@ __global__ void linear_wonly4_small_kernel(const XT* __restrict__ x, int64_t M, 
 
 bool build_stream_tmap(Weights& W) {
     W.tmap_stream_valid = false;
-    // rows of whole 128-byte lines only (K a multiple of 256); other widths take the general kernels
-    if (W.bits != 4 || W.N == 0 || W.K % 256 != 0) return true;
-    const uint64_t dims[3] = {128, (uint64_t)W.K / 256, (uint64_t)W.N};
-    const uint64_t strides[2] = {128, (uint64_t)W.K / 2};
+    // rows of whole 128-byte lines only (K a multiple of 256 at 4 bits, of 128 at 8); other widths take the general kernels
+    const int64_t row_bytes = W.bits == 4 ? W.K / 2 : W.K;
+    if (W.N == 0 || W.K % (W.bits == 4 ? 256 : 128) != 0) return true;
+    const uint64_t dims[3] = {128, (uint64_t)row_bytes / 128, (uint64_t)W.N};
+    const uint64_t strides[2] = {128, (uint64_t)row_bytes};
     const uint32_t box[3] = {128, (uint32_t)kLines, (uint32_t)kRowsCta};
     W.tmap_stream_valid = encode_tiled(&W.tmap_stream, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, W.codes, dims, strides, box, true);
     return W.tmap_stream_valid;
@@ -480,7 +512,10 @@ bool gemm_stream_applies(int64_t M, const Weights& W) {
     // row groups make at most two rounds over the SMs (N <= 64 x SMs: 4096 and 8192 rows) -- every row group ends with a
     // rendezvous and a reduction, which four rounds of short rows (K = 4096, N = 16384: 19 us against 10 us) do not amortise --
     // up to 128 Mi weights for at most 8 tokens and 64 Mi for at most 16 (16 x 16384 x 8192: 23 us against 21 us).
-    if (W.bits != 4 || !W.tmap_stream_valid || M < 1 || M > 16) return false;
+    if (!W.tmap_stream_valid || M < 1 || M > 16) return false;
+    // 8-bit weights (twice the bytes per row): ahead where the row groups make ONE round over the SMs, up to 64 Mi
+    // weights (16 tokens, K = 8192, N = 4096: 12.8 us against 17.5 us; K = 4096, N = 8192: 14.0 against 11.5 us)
+    if (W.bits == 8) return W.N <= 32ll * device_sm_count() && W.N * W.K <= (1ll << 26);
     if (W.N > 64ll * device_sm_count()) return false;
     return W.N * W.K <= (M <= 8 ? (1ll << 27) : (1ll << 26));
 }
@@ -491,6 +526,8 @@ cudaError_t launch_gemm_stream(const int8_t* a8, int64_t M, const Weights& W, in
     p.x = a8; p.ldx = W.K; p.M = M; p.N = W.N; p.K = (int)W.K; p.acc_shift = acc_shift;
     p.a_delta = out.a_delta; p.w_scale = W.w_scale; p.bias = W.bias;
     p.y = out.y; p.yt = out.yt; p.ldy = out.ldy; p.acc_out = out.acc;
+    if (W.bits == 8)
+        return M <= 8 ? launch_stream<kModeInt8, 1>(W.tmap_stream, p, stream) : launch_stream<kModeInt8, 2>(W.tmap_stream, p, stream);
     if (M <= 8) return launch_stream<kModeInt, 1>(W.tmap_stream, p, stream);
     return launch_stream<kModeInt, 2>(W.tmap_stream, p, stream);
 }

@@ -612,6 +612,7 @@ SWEEP_SAMPLE = [
     (1, 1024, 32, 4), (1, 4096, 256, 8), (16, 2048, 64, 4), (64, 1024, 128, 8), (256, 4096, 32, 8),
     (256, 2048, 256, 4), (1024, 1024, 64, 4), (1024, 4096, 128, 8), (4096, 2048, 128, 4),
     (8, 8192, 128, 4), (16, 8192, 64, 4),      # the weight-streaming kernel at its largest square (64 Mi weights)
+    (3, 1024, 32, 8), (16, 4096, 64, 8), (9, 2048, 256, 8),   # ... and on 8-bit weights
 ]
 
 
