@@ -466,6 +466,25 @@ def test_random_shapes_against_the_second_witness():
         assert st == fq.OK, (M, N, K, bits, hex(word))
 
 
+@pytest.mark.parametrize("M,N,K", [(1, 72, 1152), (9, 136, 640), (16, 1032, 2176), (5, 8, 128), (16, 4096, 16384)])
+def test_short_batches_on_8bit_weights_take_the_streaming_kernel_bit_exact(M, N, K):
+    """At most 16 tokens on 8-bit weights of at most 32 x SMs rows: rows that end inside a stage (K not a multiple of
+    1024), row groups that end inside the matrix (N not a multiple of 32), one and two token groups, and the longest
+    rows it is given -- integer sums against the oracle, outputs against its epilogue."""
+    rng = np.random.default_rng(M + N + K)
+    a, w = random_codes(rng, M, K, 8), random_codes(rng, N, K, 8)
+    ws = np.exp2(rng.uniform(-10, -6, size=N)).astype(np.float32)
+    bias = rng.standard_normal(N).astype(np.float32)
+    h = fq.weights_import(to_dev(w), to_dev(ws), None, to_dev(bias), K, 32, 8)
+    want = oracle.gemm_i32(a, w, K, 8)
+    assert np.array_equal(to_np(fq.gemm_acc_i32(to_dev(a), h)), want)
+    delta = (rng.random(M) + 0.5).astype(np.float32)
+    y = fq.gemm_w8a8(to_dev(a), to_dev(delta), h, out_dtype=torch.float32)
+    assert_close(to_np(y), oracle.epilogue(want, delta, ws, bias, "f32"), "f32", f"w8 stream {M}x{N}x{K}")
+    st, word = fq.device_status()
+    assert st == fq.OK, hex(word)
+
+
 @pytest.mark.parametrize("M", [1, 16, 64])
 def test_short_batch_on_a_large_matrix(M):
     """Long K loops on many tiles (128 stages of four atoms, or a K split): the regime where a pipeline that
