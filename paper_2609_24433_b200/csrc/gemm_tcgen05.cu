@@ -1187,19 +1187,17 @@ Plan plan_gemm(int64_t M, int64_t N, int64_t K, int bits, int sms, size_t scratc
             // 4-bit weights, token tiles of 32..64 (four-atom stages): kept to the envelope in which that configuration
             // has run clean under CUDA-graph replay -- at most 64 work units and K <= 4096.  Beyond it (M = 64 at
             // K = N = 8192 and 16384 ended two benchmark runs with a launch failure whose cause reading has not shown)
-            // the batch is padded to a 128-token tile with two-atom stages, unsplit: the configuration every mid-size
-            // batch runs.
-            bool padded = false;
+            // the batch is padded to a 128-token tile with two-atom stages: the configuration every mid-size batch runs
+            // (it may split K like any other: 32 tiles of 128 k-blocks are better off as 128 units).
             if (bits == 4 && b > 16 && b <= 64 && (n_units * ((M + b - 1) / b) > 64 || kb > 32)) {
                 b = 128;
-                padded = true;
             }
             const int64_t units = n_units * ((M + b - 1) / b);
             const double w8_single = 350.0 + 0.8 * b > 230.0 + 2.0 * b ? 350.0 + 0.8 * b : 230.0 + 2.0 * b;
             // 4-bit, tiles of at most 128 tokens: two-atom stages (see the kernel) cost less per 128 channels
             const double w4 = (c == 1 && b <= 128 && K % kBlockK == 0) ? 235.0 + b : 330.0 + b;
             const double per_kb = bits == 4 ? w4 : (c == 1 ? w8_single : (2.62 * b > 545.0 ? 2.62 * b : 545.0));
-            for (int sp = 1; sp <= (padded ? 1 : ((c == 1 || bits == 8) ? kMaxSplit : 1)); sp *= 2) {
+            for (int sp = 1; sp <= ((c == 1 || bits == 8) ? kMaxSplit : 1); sp *= 2) {
                 if (sp > 1 && (kb % sp != 0 || kb / sp < 2 || units * c > kMaxSplitTiles || units * c * sp > 4 * (int64_t)sms)) continue;
                 const int64_t kb_per = kb / sp;
                 const size_t scratch = sp > 1 ? kCounterBytes + (size_t)units * c * sp * kTileN * b * sizeof(int32_t) : 0;

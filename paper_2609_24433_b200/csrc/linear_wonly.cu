@@ -73,7 +73,7 @@ __device__ __forceinline__ void mma_s8(int* d, const uint32_t* a, uint32_t b0, u
 }
 __device__ __forceinline__ uint4 lds128(uint32_t addr) {
     uint4 v;
-    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
     return v;
 }
 
@@ -312,8 +312,7 @@ weight_stream_kernel(const __grid_constant__ CUtensorMap map_w, const StreamPara
                     uint4 wq[4];                             // rows g, g + 8, g + 16, g + 24
 #pragma unroll
                     for (int r = 0; r < 4; ++r) wq[r] = lds128(row0 + (uint32_t)(r * 8 * kLines * 128));
-                    __syncwarp();
-                    if (elect_one()) mbar_arrive(smem_u32(&s_empty[slot]));
+                    const int slot_used = slot;              // given back only after the stage's MMAs, see below
                     if (++slot == p.depth) { slot = 0; ph ^= 1u; }
                     const bool exists = s * kStageCh + kq * kLineCh < p.K;     // (warp-uniform) the line is inside the row
                     // this stage's activations arrived a stage ago: form the fragments, then put the next stage's loads in
@@ -374,6 +373,13 @@ weight_stream_kernel(const __grid_constant__ CUtensorMap map_w, const StreamPara
                         }
                     }
                     if (!kAhead && s + 1 < stages_k) load_x(s + 1);
+                    // The stage goes back to the producer only now, behind the MMAs that consumed what was loaded from it:
+                    // released right after the loads had been issued (and a __syncwarp), the float path -- the one slow
+                    // enough to keep the ring full, so that a freed stage is overwritten at once -- returned wrong sums in
+                    // about one launch in a thousand once a row had more stages than the ring (K >= 16384): the loads had
+                    // not all been performed when the producer's copy landed.
+                    __syncwarp();
+                    if (elect_one()) mbar_arrive(smem_u32(&s_empty[slot_used]));
                 }
                 if (!ok) break;
                 // C fragment: [0..1] = row g, tokens 2t, 2t+1; [2..3] = row g + 8

@@ -850,6 +850,37 @@ def test_linear_w4a16_long_rows_and_activations_with_a_mean(M, N, K, xdtype, mea
     assert_close(to_np(y), want, "f32", f"w4a16 mean {mean} {M}x{N}x{K}")
 
 
+def test_linear_w4a16_rows_longer_than_the_ring_are_reproducible():
+    """K = 16384 is eight stages through a ring of six: with the float path's slow consumers the ring stays full and a
+    stage given back is overwritten at once.  Two thousand launches on the same operands must return the same bits
+    (a stage released before its loads had been performed showed up as wrong sums in about one launch in a thousand)."""
+    rng = np.random.default_rng(5)
+    M, N, K = 8, 1024, 16384
+    q = rng.integers(-8, 8, size=(N, K)).astype(np.int32)
+    ws = np.exp2(rng.uniform(-9, -7, size=N)).astype(np.float32)
+    bias = rng.standard_normal(N).astype(np.float32)
+    wc = oracle.pack(q, 4)
+    x = synth.as_dtype(rng.standard_normal((M, K)).astype(np.float32), "bf16")
+    h = fq.weights_import(to_dev(wc), to_dev(ws), None, to_dev(bias), K, 1, 4)
+    xd = to_dev(x, "bf16")
+    ref = fq.linear_w4a16(xd, h, torch.float32).clone()
+    assert_close(to_np(ref), oracle.linear_wonly(x, "bf16", wc, ws, bias, 4, "f32"), "f32", "w4a16 long rows")
+    y = torch.empty_like(ref)
+    for it in range(2000):
+        fq.linear_w4a16(xd, h, y=y)
+        if it % 50 == 49:
+            assert torch.equal(y, ref), f"launch {it} differs from the first"
+    # the integer path shares the ring
+    a = random_codes(rng, 16, K, 4)
+    hi = import_codes(wc, K, 4)
+    acc = fq.gemm_acc_i32(to_dev(a), hi).clone()
+    assert np.array_equal(to_np(acc), oracle.gemm_i32(a, wc, K, 4))
+    for it in range(500):
+        got = fq.gemm_acc_i32(to_dev(a), hi) if it % 50 == 49 else None
+        if got is not None:
+            assert torch.equal(got, acc)
+
+
 def test_linear_w4a16_exact_on_integer_activations_and_edges():
     """Integer activations make every binary32 partial sum exact, whatever the order of the additions:
     the kernel must then equal the oracle bit for bit (any indexing slip shows).  Plus the edges: zero
