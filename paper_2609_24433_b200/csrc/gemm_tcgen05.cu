@@ -140,6 +140,7 @@ struct Params {
     int32_t* partials;   // [tile][slice][bt tokens][128 channels] int32 raw sums of the slices (K split)
     uint32_t* counters;  // [tile] slices finished so far; zeroed by the host before the launch (K split)
     int delta_vec;       // a_delta is 16-byte aligned: the epilogue may read four steps per load
+    uint32_t zero;       // 0, as a run-time value (see the unpack warps' release of a packed stage)
 };
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
@@ -973,10 +974,6 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                         // is the TMEM slot free?  (tested now, needed only after the expansion below)
                         slot_free = m < 0 || mbar_test_wait(smem_u32(&s_empty[es]), eph);
                     }
-                    if (h == ATOMS - 1) {
-                        __syncwarp();
-                        if (elect_one()) mbar_arrive(smem_u32(&s_empty_p[ps]));   // packed stage read: give it back
-                    }
                     uint32_t o[32];                          // 128 codes -> 128 int8 = 32 TMEM columns
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
@@ -988,6 +985,16 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                             o[8 * c + 2 * q + 0] = lo;   // same (even, odd) channel order as the int8 activations
                             o[8 * c + 2 * q + 1] = hi;
                         }
+                    }
+                    if (h == ATOMS - 1) {
+                        // The packed stage goes back to its producer behind the expansion that consumed what was loaded
+                        // from it, and the barrier's address is formed from one expanded word of each load and a run-time
+                        // zero: neither the compiler nor the load/store unit may let the arrival overtake the loads (the
+                        // ring is always full, a freed stage is overwritten at once; the weight-streaming kernel, which
+                        // released its stages right behind the loads, returned wrong sums once in a thousand launches).
+                        const uint32_t dep = (o[0] ^ o[9] ^ o[18] ^ o[27]) & p.zero;
+                        __syncwarp();
+                        if (elect_one()) mbar_arrive(smem_u32(&s_empty_p[ps]) + dep);
                     }
                     if (h == 0) {
                         ok = mbar_wait_all(smem_u32(&s_empty[es]), eph, abort_flag, p.watchdog, kWdUnpackEmpty, slot_free);

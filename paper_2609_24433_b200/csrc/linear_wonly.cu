@@ -190,6 +190,7 @@ struct StreamParams {
     int64_t ldy;
     int32_t* acc_out;         // int8: raw sums instead of y (parity/debug)
     uint32_t* watchdog;
+    uint32_t zero;            // 0, as a run-time value (see the consumers' release of a stage)
 };
 
 enum : uint32_t { kWdStreamFull = 0x400u, kWdStreamEmpty = 0x800u, kWdStreamSync = 0x1000u };
@@ -378,8 +379,12 @@ weight_stream_kernel(const __grid_constant__ CUtensorMap map_w, const StreamPara
                     // enough to keep the ring full, so that a freed stage is overwritten at once -- returned wrong sums in
                     // about one launch in a thousand once a row had more stages than the ring (K >= 16384): the loads had
                     // not all been performed when the producer's copy landed.
+                    // (and its barrier's address is formed from an accumulator and a run-time zero: a true dependence)
+                    uint32_t dep;
+                    if constexpr (kIntegers) dep = (uint32_t)(acc[0][0][0] ^ acc[1][0][0]) & p.zero;
+                    else dep = (__float_as_uint(acc[0][0][0]) ^ __float_as_uint(acc[1][0][0])) & p.zero;
                     __syncwarp();
-                    if (elect_one()) mbar_arrive(smem_u32(&s_empty[slot_used]));
+                    if (elect_one()) mbar_arrive(smem_u32(&s_empty[slot_used]) + dep);
                 }
                 if (!ok) break;
                 // C fragment: [0..1] = row g, tokens 2t, 2t+1; [2..3] = row g + 8
