@@ -485,6 +485,34 @@ def test_short_batches_on_8bit_weights_take_the_streaming_kernel_bit_exact(M, N,
     assert st == fq.OK, hex(word)
 
 
+@pytest.mark.parametrize("M,K,N,bits", [(816, 2048, 4096, 4), (50, 4096, 1024, 4), (256, 4096, 4096, 4), (64, 8192, 2048, 8),
+                                        (16, 16384, 1024, 4), (100, 16384, 256, 4)])
+def test_repeated_launches_return_the_same_bits(M, K, N, bits):
+    """Rings that are full all the time (weights prefetched far ahead) hand their stages over thousands of times per
+    launch: a stage given back an instant too early shows up as a rare wrong output, not as a failure.  Six hundred
+    launches per configuration (one-, two- and four-atom stages, 8-bit operands, the streaming kernel, a K split)
+    must return the bits of the first, which match the dp4a witness."""
+    q = 7 if bits == 4 else 127
+    gen = torch.Generator(device="cuda").manual_seed(M + K + N)
+    wc = torch.randint(-q, q + 1, (N, K), dtype=torch.int8, device="cuda", generator=gen)
+    ac = torch.randint(-q, q + 1, (M, K), dtype=torch.int8, device="cuda", generator=gen)
+    h = fq.weights_import(_pack_dev(wc, bits), torch.rand(N, device="cuda", generator=gen) * 0.01 + 0.001, None,
+                          torch.randn(N, device="cuda", generator=gen), K, 32, bits)
+    a = _pack_dev(ac, bits)
+    d = torch.rand(M, device="cuda", generator=gen) + 0.5
+    ws = torch.empty(fq.workspace_bytes(M, K, N, bits), dtype=torch.uint8, device="cuda")
+    f = fq.gemm_w4a4 if bits == 4 else fq.gemm_w8a8
+    ref = f(a, d, h, torch.float32, workspace=ws).clone()
+    assert torch.allclose(ref, fq.gemm_simt(a, d, h, torch.float32), rtol=1e-5, atol=1e-5)
+    y = torch.empty_like(ref)
+    for it in range(600):
+        f(a, d, h, y=y, workspace=ws)
+        if it % 50 == 49:
+            assert torch.equal(y, ref), f"launch {it} differs from the first"
+    st, word = fq.device_status()
+    assert st == fq.OK, hex(word)
+
+
 @pytest.mark.parametrize("M", [1, 16, 64])
 def test_short_batch_on_a_large_matrix(M):
     """Long K loops on many tiles (128 stages of four atoms, or a K split): the regime where a pipeline that
