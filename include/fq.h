@@ -221,10 +221,9 @@ fq_status fq_linear_w8a8(const void* x, fq_dtype xt, int64_t M, int64_t ldx, con
  * W is any 4-bit handle; its codes multiply x as given, so a handle meant for this call is made with the
  * identity transform (fq_fold_weights with hadamard_block = 1 and smooth = NULL: plain per-output-channel
  * RTN of W), or x must already be in the handle's transformed coordinates.  No quantization of x, no
- * workspace.  x device [M, K] of dtype xt (FQ_F32 or FQ_BF16); binary32 accumulation.  The kernel multiplies
- * (136 + code) * x exactly and takes 136 * sum_c x[t][c] off afterwards (slice by slice of K / 16 channels), so the
- * rounding of its sums grows with |sum_c x[t][c]|: about 2^-24 * 136 * |sum over a slice| per output, negligible
- * for activations centred near zero, within the 1e-3 of the tests up to mean / sigma = 4 over 16384 channels.
+ * workspace.  x device [M, K] of dtype xt (FQ_F32 or FQ_BF16); binary32 accumulation (the products are exact; the
+ * expanded codes carry an offset that a second MMA removes sixteen channels at a time, so the sums' rounding does not
+ * depend on the activations' mean).
  * These projections see
  * one conditioning vector per sample: the kernel streams the weights once per eight tokens and is meant for
  * short batches (any M is accepted).  Errors as for fq_linear_w4a4; FQ_ERR_UNSUPPORTED for 8-bit handles. */

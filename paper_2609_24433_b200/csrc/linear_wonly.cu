@@ -79,13 +79,13 @@ __device__ __forceinline__ uint4 lds128(uint32_t addr) {
 
 // Codes of channels j and j + 4 of a packed word (eight two's-complement nibbles, channel i at bits
 // 4 i) as two bf16, each 136 too large: (n & 15) ^ 8 = n + 8 goes into the mantissa of 128 (0x4300).
-// The exact value 136 + n is what the MMAs multiply; 136 times the sum of the token's activations --
-// accumulated beside the products by MMAs against a matrix of ones -- comes off once per output.  (Taking
-// 136 off every pair with a packed subtract cost a third of the kernel's integer instructions.)
+// The exact value 136 + n is what the product MMA multiplies; a second MMA of the constant -136 against the same
+// activations takes the offset off again at once, sixteen channels at a time, so the accumulator never carries more
+// than one MMA's worth of it.  (Taking 136 off every pair with a packed subtract cost a third of the kernel's
+// integer instructions -- the pipe that bounds it; the tensor pipe has room for twice the MMAs.)
 __device__ __forceinline__ uint32_t codes_plus136_bf16x2(uint32_t w, int j) {
     return ((w >> (4 * j)) & 0x000F000Fu) ^ 0x43084308u;
 }
-constexpr float kCodeOffset = 136.0f;
 
 // The activations of one token at a lane's 32 channels: fetch() issues the loads into raw registers, permute() --
 // called a stage later, when they have long arrived -- forms the B-fragment registers.  (With the byte permutes right
@@ -214,7 +214,6 @@ weight_stream_kernel(const __grid_constant__ CUtensorMap map_w, const StreamPara
     const uint32_t ring = (smem_u32(smem_raw) + 1023u) & ~1023u;
     AccT* s_part = reinterpret_cast<AccT*>(smem_raw + (ring - smem_u32(smem_raw)) + (size_t)p.depth * kStageBytes);
     // s_part[consumer warp][row 0..31][token, padded to kTok + 1]
-    [[maybe_unused]] float* s_xsum = reinterpret_cast<float*>(s_part + (size_t)kConsumers * kRowsCta * (kTok + 1));   // [consumer warp][token]
 
     if (threadIdx.x == 0) {
         s_abort = 0;
@@ -287,14 +286,7 @@ weight_stream_kernel(const __grid_constant__ CUtensorMap map_w, const StreamPara
                     for (int q = 0; q < GROUPS; ++q)
 #pragma unroll
                         for (int i = 0; i < 4; ++i) acc[r][q][i] = 0;
-                // float modes: sum of the tokens' activations over this warp's channels (see codes_plus136_bf16x2).  It does
-                // not depend on the rows: with one pass per row group the CTA's first row group computes it for all
-                [[maybe_unused]] const bool do_sum = !kIntegers && (passes > 1 || rg == (int)blockIdx.x);
-                [[maybe_unused]] float acc_s[GROUPS][4];
-#pragma unroll
-                for (int q = 0; q < GROUPS; ++q)
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) acc_s[q][i] = 0.0f;
+                [[maybe_unused]] const uint32_t minus136[4] = {0xC308C308u, 0xC308C308u, 0xC308C308u, 0xC308C308u};   // bf16 -136
                 XFrag<MODE> xf[GROUPS];
                 // the lane's 32 channels of stage s
                 auto load_x = [&](int s) {
@@ -357,20 +349,14 @@ weight_stream_kernel(const __grid_constant__ CUtensorMap map_w, const StreamPara
                                         for (int q = 0; q < GROUPS; ++q)
 #pragma unroll
                                             for (int tm = 0; tm < kTerms; ++tm)
+                                            {
                                                 mma_bf16(reinterpret_cast<float*>(acc[r][q]), a, xc[q].b[tm][4 * w + 2 * m],
                                                          xc[q].b[tm][4 * w + 2 * m + 1]);
+                                                mma_bf16(reinterpret_cast<float*>(acc[r][q]), minus136, xc[q].b[tm][4 * w + 2 * m],
+                                                         xc[q].b[tm][4 * w + 2 * m + 1]);
+                                            }
                                     }
                             }
-                        }
-                        if constexpr (!kIntegers) if (do_sum) {
-                            const uint32_t ones[4] = {0x3F803F80u, 0x3F803F80u, 0x3F803F80u, 0x3F803F80u};   // bf16 1.0
-#pragma unroll
-                            for (int i = 0; i < 8; ++i)
-#pragma unroll
-                                for (int q = 0; q < GROUPS; ++q)
-#pragma unroll
-                                    for (int tm = 0; tm < kTerms; ++tm)
-                                        mma_bf16(acc_s[q], ones, xc[q].b[tm][2 * i], xc[q].b[tm][2 * i + 1]);
                         }
                     }
                     if (!kAhead && s + 1 < stages_k) load_x(s + 1);
@@ -398,13 +384,6 @@ weight_stream_kernel(const __grid_constant__ CUtensorMap map_w, const StreamPara
                         part[(16 * r + g + 8) * (kTok + 1) + 8 * q + 2 * t] = acc[r][q][2];
                         part[(16 * r + g + 8) * (kTok + 1) + 8 * q + 2 * t + 1] = acc[r][q][3];
                     }
-                if (!kIntegers && do_sum && g == 0) {      // every row of the ones product holds the same sums: row 0
-#pragma unroll
-                    for (int q = 0; q < GROUPS; ++q) {
-                        s_xsum[warp * kTok + 8 * q + 2 * t] = acc_s[q][0];
-                        s_xsum[warp * kTok + 8 * q + 2 * t + 1] = acc_s[q][1];
-                    }
-                }
                 __syncwarp();
                 if (elect_one()) mbar_arrive(smem_u32(&s_sync));
                 ok = mbar_wait_all(smem_u32(&s_sync), sync_ph, abort_flag, p.watchdog, kWdStreamSync);
@@ -414,14 +393,7 @@ weight_stream_kernel(const __grid_constant__ CUtensorMap map_w, const StreamPara
                     const int row = o % kRowsCta, tok = o / kRowsCta;    // consecutive threads: consecutive channels
                     AccT sum = 0;
 #pragma unroll
-                    for (int k = 0; k < kConsumers; ++k) {
-                        const AccT part_k = s_part[((size_t)k * kRowsCta + row) * (kTok + 1) + tok];
-                        // float modes: the offset comes off warp by warp, each warp's sum of activations against its own
-                        // products (the same channels), before the sixteen slices are added: the cancellation then acts
-                        // on a sixteenth of the row at a time
-                        if (!kIntegers) sum += (AccT)fmaf(-kCodeOffset, s_xsum[k * kTok + tok], (float)part_k);
-                        else sum += part_k;
-                    }
+                    for (int k = 0; k < kConsumers; ++k) sum += s_part[((size_t)k * kRowsCta + row) * (kTok + 1) + tok];
                     const int64_t j = j0 + row, tt = t0 + tok;
                     if (j < p.N && tt < p.M) {
                         if (kIntegers && p.acc_out != nullptr) {
@@ -455,7 +427,7 @@ template <int MODE, int GROUPS>
 cudaError_t launch_stream(const CUtensorMap& map, StreamParams p, cudaStream_t stream) {
     typedef typename std::conditional<Geometry<MODE>::kIntegers, int, float>::type AccT;
     const int sms = device_sm_count();
-    const size_t part_bytes = (size_t)kConsumers * kRowsCta * (8 * GROUPS + 1) * sizeof(AccT) + (size_t)kConsumers * 8 * GROUPS * sizeof(float);
+    const size_t part_bytes = (size_t)kConsumers * kRowsCta * (8 * GROUPS + 1) * sizeof(AccT);
     const size_t budget = 227 * 1024 - 1024 /*alignment*/ - 1024 /*static*/ - part_bytes;
     int depth = (int)(budget / kStageBytes);
     if (depth > kMaxDepth) depth = kMaxDepth;

@@ -861,11 +861,13 @@ def test_linear_w4a16_matches_oracle(M, N, K, xdtype, ydtype):
     assert np.linalg.norm(as_f64(to_np(y)) - ref) / np.linalg.norm(ref) < 0.2
 
 
-@pytest.mark.parametrize("M,N,K,xdtype,mean", [(9, 512, 8192, "f32", 4.0), (1, 8192, 8192, "bf16", 0.0), (8, 1024, 16384, "bf16", -2.0)])
+@pytest.mark.parametrize("M,N,K,xdtype,mean", [(9, 512, 8192, "f32", 4.0), (1, 8192, 8192, "bf16", 0.0), (8, 1024, 16384, "bf16", -2.0),
+                                               (3, 264, 16384, "f32", 50.0)])
 def test_linear_w4a16_long_rows_and_activations_with_a_mean(M, N, K, xdtype, mean):
-    """The kernel multiplies the codes 136 too large and takes 136 x (sum of the token's activations) off each output:
-    activations whose sum is far from zero (mean / sigma up to 4, K up to 16384) are where that cancellation costs the
-    most binary32 digits.  Same tolerance as everywhere; also the largest rows the streaming ring sees here."""
+    """The kernel multiplies the codes 136 too large and cancels the offset with a second MMA of -136 against the same
+    activations, sixteen channels at a time: activations whose sum is far from zero (mean / sigma up to 50, K up to
+    16384) must cost it no accuracy (taking 136 x the whole row's sum off at the end left such rows at the edge of
+    the tolerance).  Same tolerance as everywhere; also the largest rows the streaming ring sees here."""
     rng = np.random.default_rng(M + N + K)
     q = rng.integers(-8, 8, size=(N, K)).astype(np.int32)
     wc = oracle.pack(q, 4)
