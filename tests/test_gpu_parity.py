@@ -513,6 +513,47 @@ def test_repeated_launches_return_the_same_bits(M, K, N, bits):
     assert st == fq.OK, hex(word)
 
 
+@pytest.mark.parametrize("M,sites", [
+    (50, [(1024, 3072, 4), (1024, 1024, 4), (1024, 8192, 4), (4096, 1024, 4)]),          # an action-expert layer
+    (100, [(16384, 256, 4), (2048, 2048, 4), (16384, 256, 8), (1024, 1024, 8)]),         # K splits between unsplit calls
+    (16, [(4096, 4096, 4), (4096, 4096, 8), (8192, 1024, 4), (1024, 4096, 8)]),          # the streaming kernel, both widths
+])
+def test_calls_of_a_layer_share_one_workspace_in_a_graph(M, sites):
+    """A model runs its layers' projections one after the other on one stream with ONE workspace.  Each call's prologue
+    overwrites the codes and steps that the call before it may still be reading when it starts early (programmatic
+    dependent launch), and a K split's counters are cleared between unrelated launches: a graph of three such layers,
+    replayed a hundred times, must give what the calls give with workspaces of their own."""
+    gen = torch.Generator(device="cuda").manual_seed(M)
+    hs, xs, ys, need = [], [], [], 0
+    for K, N, bits in sites:
+        W = torch.randn((N, K), device="cuda", generator=gen) * 0.02
+        hs.append(fq.fold_weights(W, None, torch.randn(N, device="cuda", generator=gen), 64, bits))
+        xs.append(torch.randn((M, K), device="cuda", generator=gen).to(torch.bfloat16))
+        ys.append(torch.empty((M, N), dtype=torch.bfloat16, device="cuda"))
+        need = max(need, fq.workspace_bytes(M, K, N, bits))
+    want = [fq.linear(x, h, 1.0, torch.bfloat16) for x, h in zip(xs, hs)]
+    ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+    for x, h, y in zip(xs, hs, ys):
+        fq.linear(x, h, 1.0, y=y, workspace=ws)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        for _ in range(3):
+            for x, h, y in zip(xs, hs, ys):
+                fq.linear(x, h, 1.0, y=y, workspace=ws)
+    for it in range(100):
+        if it % 10 == 0:
+            for y in ys:
+                y.zero_()
+        g.replay()
+        if it % 10 == 9:
+            torch.cuda.synchronize()
+            for a, b in zip(ys, want):
+                assert torch.equal(a, b), f"replay {it}"
+    st, word = fq.device_status()
+    assert st == fq.OK, hex(word)
+
+
 @pytest.mark.parametrize("M", [1, 16, 64])
 def test_short_batch_on_a_large_matrix(M):
     """Long K loops on many tiles (128 stages of four atoms, or a K split): the regime where a pipeline that
